@@ -1,0 +1,420 @@
+"""Pins for the CPU oracle: each check ties it to something other than itself —
+published known-answer vectors, the paper's worked example, brute force on tiny
+graphs, closed forms, whole-graph linear algebra, library routines."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import dense_oracle as O
+from paper_2202_02365_b200 import inputs
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _fields(path):
+    out = {}
+    for line in open(path):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        key, val = line.split(":", 1)
+        out[key.strip()] = val.strip()
+    return out
+
+
+def _ints(s):
+    return [int(x) for x in s.split()]
+
+
+def _csr_from_edges(n, edges):
+    rows = [[] for _ in range(n)]
+    for s, d in edges:
+        rows[d].append(s)
+    off, nb = [0], []
+    for r in rows:
+        nb.extend(sorted(r))
+        off.append(len(nb))
+    return np.array(off), np.array(nb, dtype=np.int64)
+
+
+def _random_graph(n, m, seed):
+    g = inputs.erdos_renyi_graph(n, m, seed)
+    return g.row_offsets.numpy(), g.nbrs.numpy().astype(np.int64)
+
+
+# ---------------------------------------------------------------- Philox
+def test_philox_known_answers():
+    n = 0
+    for line in open(os.path.join(GOLD, "philox4x32_10_kat.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        w = [int(x, 16) for x in line.split()]
+        assert list(O.philox4x32_10(w[0:4], w[4:6])) == w[6:10]
+        n += 1
+    assert n == 3
+
+
+def test_draw_word_keying():
+    # word t of a block is output (t % 4) of counter (node, 0, hop, t // 4)
+    blk = O.philox4x32_10((12345, 0, 2, 1), (0xDEADBEEF, 0x1234))
+    seed = (0x1234 << 32) | 0xDEADBEEF
+    assert [O.draw_word(seed, 12345, 2, 4 + i) for i in range(4)] == list(blk)
+    # every key component matters
+    base = O.draw_word(seed, 12345, 2, 5)
+    assert len({base, O.draw_word(seed + 1, 12345, 2, 5), O.draw_word(seed, 12346, 2, 5),
+                O.draw_word(seed, 12345, 1, 5), O.draw_word(seed, 12345, 2, 6),
+                O.draw_word(seed ^ (1 << 40), 12345, 2, 5)}) == 6
+
+
+def test_to_range_is_floor_of_scaled_word():
+    for w, n in [(0, 7), (0xFFFFFFFF, 7), (0x80000000, 10), (0x12345678, 1000003)]:
+        assert O.to_range(w, n) == int(np.floor(w / 2.0**32 * n))
+        assert 0 <= O.to_range(w, n) < n
+
+
+# ---------------------------------------------------------------- one-hop sample
+def test_small_degree_returns_whole_row():
+    row = [4, 9, 9, 17]
+    for f in (4, 5, 100):
+        assert O.one_hop_sample(row, f, 1, 3, 0) == row
+
+
+def test_large_degree_returns_f_distinct_positions_in_order():
+    row = list(range(100, 160))       # distinct values -> positions are recoverable
+    for f in (1, 2, 7, 31, 33, 59):
+        for node in range(20):
+            s = O.one_hop_sample(row, f, 99, node, 1)
+            assert len(s) == f
+            assert len(set(s)) == f
+            assert s == sorted(s)
+            assert set(s) <= set(row)
+
+
+def test_sample_depends_only_on_its_key():
+    row = list(range(50))
+    a = O.one_hop_sample(row, 5, 7, 11, 0)
+    assert a == O.one_hop_sample(row, 5, 7, 11, 0)
+    others = [O.one_hop_sample(row, 5, 8, 11, 0), O.one_hop_sample(row, 5, 7, 12, 0),
+              O.one_hop_sample(row, 5, 7, 11, 1)]
+    assert any(o != a for o in others)
+
+
+def test_inclusion_is_uniform():
+    # every position is kept with probability f/d, every pair with f(f-1)/(d(d-1))
+    d, f, trials = 12, 4, 6000
+    row = list(range(d))
+    single = np.zeros(d)
+    pair = np.zeros((d, d))
+    for node in range(trials):
+        s = O.one_hop_sample(row, f, 2024, node, 0)
+        for x in s:
+            single[x] += 1
+        for x, y in itertools.combinations(s, 2):
+            pair[x, y] += 1
+    exp = trials * f / d
+    chi2 = ((single - exp) ** 2 / exp).sum()
+    assert chi2 < 35.0                      # 11 dof, p ~ 2e-4
+    exp2 = trials * f * (f - 1) / (d * (d - 1))
+    vals = pair[np.triu_indices(d, 1)]
+    chi2p = ((vals - exp2) ** 2 / exp2).sum()
+    assert chi2p < 120.0                    # 65 dof, p ~ 4e-5
+
+
+def test_all_subsets_reachable_tiny():
+    # d = 5, f = 2: all 10 subsets appear, about equally often
+    seen = {}
+    for node in range(4000):
+        s = tuple(O.one_hop_sample([0, 1, 2, 3, 4], 2, 5, node, 0))
+        seen[s] = seen.get(s, 0) + 1
+    assert len(seen) == 10
+    assert min(seen.values()) > 300 and max(seen.values()) < 500
+
+
+# ---------------------------------------------------------------- Algorithm 1
+def test_worked_example_layout():
+    g = _fields(os.path.join(GOLD, "dense_worked_example.txt"))
+    edges = [tuple(_ints(e)) for e in g["edges"].split(",")]
+    off, nb = _csr_from_edges(5, edges)
+    d = O.sample_dense(O.GraphView(off, nb), _ints(g["targets"]), _ints(g["fanouts"]), seed=0)
+    for key in ("node_ids", "node_id_offsets", "nbrs", "nbr_offsets", "repr_map"):
+        assert d[key] == _ints(g[key]), key
+    u = O.update_dense(d)
+    assert u["node_ids"] == _ints(g["after_layer1_node_ids"])
+    assert u["nbrs"] == _ints(g["after_layer1_nbrs"])
+    assert u["repr_map"] == _ints(g["after_layer1_repr_map"])
+    assert u["nbr_offsets"] == _ints(g["after_layer1_nbr_offsets"])
+    assert u["node_id_offsets"] == _ints(g["after_layer1_node_id_offsets"])
+
+
+def _bfs_levels(off, nb, targets, k, allowed=None):
+    seen = set(targets)
+    levels = [list(targets)]
+    frontier = list(targets)
+    for _ in range(k):
+        nxt = set()
+        for v in frontier:
+            for u in nb[off[v]:off[v + 1]]:
+                u = int(u)
+                if (allowed is None or u in allowed) and u not in seen:
+                    nxt.add(u)
+        seen |= nxt
+        frontier = sorted(nxt)
+        levels.append(frontier)
+    return levels
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_full_fanout_gives_bfs_levels(seed):
+    off, nb = _random_graph(60, 150, seed)
+    maxdeg = int(np.diff(off).max())
+    targets = [5, 17, 3]
+    k = 3
+    d = O.sample_dense(O.GraphView(off, nb), targets, [maxdeg] * k, seed=4)
+    levels = _bfs_levels(off, nb, targets, k)
+    nio = d["node_id_offsets"]
+    for j in range(k + 1):                       # Delta_{k-j} = BFS level j
+        i = k - j
+        assert d["node_ids"][nio[i]:nio[i + 1]] == levels[j]
+    # every sampled node carries its exact neighbourhood
+    sampled = d["node_ids"][nio[1]:]
+    for r, v in enumerate(sampled):
+        got = d["nbrs"][d["nbr_offsets"][r]:d["nbr_offsets"][r + 1]]
+        assert got == [int(u) for u in nb[off[v]:off[v + 1]]]
+
+
+def _memoised_khop(view, targets, fanouts, seed):
+    """Ordinary layer-by-layer k-hop sampling over the *whole* frontier, with a
+    node's one-hop sample remembered from the first hop that needed it."""
+    memo = {}
+    known = list(targets)
+    for hop, f in enumerate(fanouts):
+        for v in list(known):
+            if v not in memo:
+                memo[v] = O.one_hop_sample(view.row(v), f, seed, v, hop)
+        for v in list(known):
+            for u in memo[v]:
+                if u not in known:
+                    known.append(u)
+    return memo, set(known)
+
+
+@pytest.mark.parametrize("seed", [0, 3])
+def test_delta_sampling_equals_memoised_full_frontier_sampling(seed):
+    off, nb = _random_graph(200, 1600, seed)
+    view = O.GraphView(off, nb)
+    targets = [1, 50, 7, 120, 33]
+    fanouts = [4, 3, 2]
+    d = O.sample_dense(view, targets, fanouts, seed=11)
+    memo, known = _memoised_khop(view, targets, fanouts, 11)
+    assert set(d["node_ids"]) == known
+    assert len(d["node_ids"]) == len(known)                      # no duplicates
+    nio = d["node_id_offsets"]
+    sampled = d["node_ids"][nio[1]:]
+    assert set(sampled) == set(memo)                             # sampled exactly once each
+    for r, v in enumerate(sampled):
+        assert d["nbrs"][d["nbr_offsets"][r]:d["nbr_offsets"][r + 1]] == memo[v]
+    # a node's fanout is that of the first hop that needed it
+    k = len(fanouts)
+    for i in range(1, k + 1):
+        f = fanouts[k - i]
+        for r in range(nio[i] - nio[1], nio[i + 1] - nio[1]):
+            v = sampled[r]
+            deg = off[v + 1] - off[v]
+            assert d["nbr_offsets"][r + 1] - d["nbr_offsets"][r] == min(deg, f)
+    # each delta ascending (targets keep caller order)
+    for i in range(k):
+        seg = d["node_ids"][nio[i]:nio[i + 1]]
+        assert seg == sorted(seg)
+    assert d["node_ids"][nio[k]:] == targets
+    # repr_map points at the right rows, and never before the delta it may use
+    for e, r in enumerate(d["repr_map"]):
+        assert d["node_ids"][r] == d["nbrs"][e]
+
+
+def test_neighbours_of_delta_j_live_in_later_rows():
+    # neighbours of Delta_j lie in Delta_{j-1} .. Delta_k, so Algorithm 2's shift
+    # of repr_map never goes negative
+    off, nb = _random_graph(300, 3000, 5)
+    d = O.sample_dense(O.GraphView(off, nb), list(range(0, 40, 2)), [3, 3, 3], seed=1)
+    cur = d
+    for _ in range(2):
+        cur = O.update_dense(cur)
+        assert min(cur["repr_map"]) >= 0
+        for e, r in enumerate(cur["repr_map"]):
+            assert cur["node_ids"][r] == cur["nbrs"][e]
+        assert cur["nbr_offsets"][0] == 0 and cur["node_id_offsets"][0] == 0
+        assert cur["nbr_offsets"][-1] == len(cur["nbrs"])
+        assert cur["node_id_offsets"][-1] == len(cur["node_ids"])
+
+
+def test_input_errors():
+    off, nb = _random_graph(20, 40, 0)
+    v = O.GraphView(off, nb, n_parts=4, resident_parts=[0, 1])
+    with pytest.raises(ValueError):
+        O.sample_dense(v, [1, 1], [2], 0)
+    with pytest.raises(ValueError):
+        O.sample_dense(v, [19], [2], 0)           # partition 3 is not resident
+    with pytest.raises(ValueError):
+        O.sample_dense(v, [20], [2], 0)
+
+
+# ---------------------------------------------------------------- in-buffer filter
+@pytest.mark.parametrize("resident", [[0, 2], [1, 2, 3], [3]])
+def test_buffer_filter_equals_sampling_the_induced_subgraph(resident):
+    n, parts = 120, 4
+    off, nb = _random_graph(n, 1500, 9)
+    size = (n + parts - 1) // parts
+    res = lambda u: (u // size) in resident
+    # induced subgraph built edge by edge
+    edges = [(int(u), v) for v in range(n) for u in nb[off[v]:off[v + 1]] if res(int(u)) and res(v)]
+    off2, nb2 = _csr_from_edges(n, edges)
+    targets = [v for v in range(n) if res(v)][::7]
+    a = O.sample_dense(O.GraphView(off, nb, parts, resident), targets, [3, 2], seed=5)
+    b = O.sample_dense(O.GraphView(off2, nb2), targets, [3, 2], seed=5)
+    assert a == b
+    assert all(res(u) for u in a["node_ids"])
+    # with full fanout: BFS levels of the resident subgraph only
+    maxdeg = int(np.diff(off).max())
+    c = O.sample_dense(O.GraphView(off, nb, parts, resident), targets[:3], [maxdeg] * 2, seed=5)
+    lv = _bfs_levels(off, nb, targets[:3], 2, allowed={u for u in range(n) if res(u)})
+    nio = c["node_id_offsets"]
+    assert c["node_ids"][nio[0]:nio[1]] == lv[2] and c["node_ids"][nio[1]:nio[2]] == lv[1]
+
+
+# ---------------------------------------------------------------- forward
+def test_hand_computed_means():
+    g = _fields(os.path.join(GOLD, "dense_worked_example.txt"))
+    hm = _fields(os.path.join(GOLD, "hand_means.txt"))
+    edges = [tuple(_ints(e)) for e in g["edges"].split(",")]
+    off, nb = _csr_from_edges(5, edges)
+    d = O.sample_dense(O.GraphView(off, nb), _ints(g["targets"]), [10, 10], seed=0)
+    h0 = np.array([float(x) for x in hm["h0"].split()]).reshape(5, 2)
+    layer = (np.eye(2), 2 * np.eye(2), np.array([0.5, -0.5]))
+    outs = O.forward(d, h0, [layer, layer], return_all=True)
+    np.testing.assert_allclose(outs[0].ravel(), [float(x) for x in hm["layer1"].split()], rtol=0, atol=1e-12)
+    np.testing.assert_allclose(outs[1].ravel(), [float(x) for x in hm["layer2"].split()], rtol=0, atol=1e-12)
+
+
+def _whole_graph_sage(off, nb, feats, layers):
+    """GraphSage-mean on every node of the graph with dense adjacency algebra."""
+    n = len(off) - 1
+    a = np.zeros((n, n))
+    for v in range(n):
+        for u in nb[off[v]:off[v + 1]]:
+            a[v, int(u)] += 1.0                   # multi-edges count
+    deg = a.sum(1, keepdims=True)
+    a_mean = np.divide(a, deg, out=np.zeros_like(a), where=deg > 0)
+    h = feats.astype(np.float64)
+    for i, (ws, wn, b) in enumerate(layers):
+        h = h @ ws.astype(np.float64) + (a_mean @ h) @ wn.astype(np.float64) + b.astype(np.float64)
+        if i + 1 < len(layers):
+            h = np.maximum(h, 0)
+    return h
+
+
+@pytest.mark.parametrize("k", [1, 2, 3])
+def test_full_fanout_forward_equals_whole_graph_graphsage(k):
+    off, nb = _random_graph(80, 400, 21)
+    rng = np.random.default_rng(0)
+    feats = rng.standard_normal((80, 6))
+    dims = [6, 5, 4, 3][:k + 1]
+    layers = [(w.numpy(), n_.numpy(), b.numpy()) for w, n_, b in inputs.random_bias_layers(dims, 3)]
+    targets = [9, 2, 40, 77, 31]
+    maxdeg = int(np.diff(off).max())
+    d = O.sample_dense(O.GraphView(off, nb), targets, [maxdeg] * k, seed=0)
+    out = O.forward(d, feats[d["node_ids"]], layers)
+    ref = _whole_graph_sage(off, nb, feats, layers)[targets]
+    np.testing.assert_allclose(out, ref, rtol=1e-12, atol=1e-12)
+
+
+def test_forward_special_cases_and_library_crosscheck():
+    off, nb = _random_graph(150, 1200, 2)
+    d = O.sample_dense(O.GraphView(off, nb), [3, 100, 42, 7], [4, 3], seed=8)
+    rng = np.random.default_rng(1)
+    h0 = rng.standard_normal((len(d["node_ids"]), 5))
+    eye, zero, b0 = np.eye(5), np.zeros((5, 5)), np.zeros(5)
+    n0 = d["node_id_offsets"][1]
+    # W_nbr = 0, W_self = I: layer output is the self rows
+    np.testing.assert_array_equal(O.sage_layer(d, h0, eye, zero, b0, relu=False), h0[n0:])
+    # additive layer of Algorithm 3 = self + count * mean
+    mean_only = O.sage_layer(d, h0, zero, eye, b0, relu=False)
+    cnt = np.diff(d["nbr_offsets"])[:, None]
+    np.testing.assert_allclose(O.additive_layer(d, h0), h0[n0:] + cnt * mean_only, rtol=1e-12, atol=1e-12)
+    # library cross-check: index_select + index_add_ + matmul in fp64
+    layers = [(w.double(), n_.double(), b.double()) for w, n_, b in inputs.random_bias_layers([5, 4], 5)]
+    ws, wn, b = layers[0]
+    ht = torch.from_numpy(h0)
+    rm = torch.tensor(d["repr_map"])
+    seg = torch.repeat_interleave(torch.arange(len(cnt)), torch.from_numpy(cnt.ravel()))
+    agg = torch.zeros((len(cnt), 5), dtype=torch.float64).index_add_(0, seg, ht.index_select(0, rm))
+    agg = agg / torch.clamp(torch.from_numpy(cnt).double(), min=1)
+    ref = torch.relu(ht[n0:] @ ws + agg @ wn + b)
+    got = O.sage_layer(d, h0, ws.numpy(), wn.numpy(), b.numpy(), relu=True)
+    np.testing.assert_allclose(got, ref.numpy(), rtol=1e-12, atol=1e-12)
+
+
+def test_isolated_node_gets_self_term_only():
+    off, nb = _csr_from_edges(3, [(0, 1)])
+    d = O.sample_dense(O.GraphView(off, nb), [2, 1], [2], seed=0)
+    h0 = np.array([[1.0, 1.0], [2.0, 3.0], [5.0, 7.0]])[d["node_ids"]]
+    out = O.forward(d, h0, [(np.eye(2), np.eye(2), np.zeros(2))])
+    np.testing.assert_array_equal(out, [[5.0, 7.0], [3.0, 4.0]])
+
+
+# ---------------------------------------------------------------- link prediction
+def test_negatives_are_resident_and_uniform():
+    off, nb = _random_graph(100, 300, 0)
+    v = O.GraphView(off, nb, n_parts=5, resident_parts=[1, 3])
+    negs = O.lp_negatives(v, n_chunks=4, negs_per_chunk=500, seed=77)
+    flat = [u for row in negs for u in row]
+    assert all(v.is_resident(u) for u in flat)
+    counts = np.bincount(flat, minlength=100)
+    res = np.array([v.is_resident(u) for u in range(100)])
+    assert counts[~res].sum() == 0
+    exp = len(flat) / res.sum()
+    assert ((counts[res] - exp) ** 2 / exp).sum() < 80.0        # 39 dof
+    assert v.resident_nodes() == [v.resident_node_at(i) for i in range(v.n_resident_nodes())]
+    assert negs != O.lp_negatives(v, 4, 500, seed=78)
+
+
+def test_lp_prepare_indices():
+    off, nb = _random_graph(50, 200, 0)
+    v = O.GraphView(off, nb)
+    src, dst = [3, 9, 3, 44], [9, 1, 20, 3]
+    p = O.lp_prepare(v, src, dst, n_chunks=2, negs_per_chunk=3, seed=1)
+    t = p["targets"]
+    assert t == sorted(set(t))
+    assert [t[i] for i in p["src_idx"]] == src and [t[i] for i in p["dst_idx"]] == dst
+    for row_ids, row_idx in zip(p["neg_ids"], p["neg_idx"]):
+        assert [t[i] for i in row_idx] == row_ids
+    assert set(t) == set(src) | set(dst) | {u for r in p["neg_ids"] for u in r}
+
+
+def test_distmult_closed_forms():
+    rng = np.random.default_rng(3)
+    h = rng.standard_normal((30, 8))
+    rel_emb = rng.standard_normal((5, 8))
+    n, chunks, negs = 12, 3, 4
+    prep = {"src_idx": list(rng.integers(0, 30, n)), "dst_idx": list(rng.integers(0, 30, n)),
+            "neg_idx": [list(rng.integers(0, 30, negs)) for _ in range(chunks)]}
+    rel = rng.integers(0, 5, n)
+    pos, nd, ns = O.distmult_scores(h, rel_emb, prep, rel, chunks)
+    s, o = np.array(prep["src_idx"]), np.array(prep["dst_idx"])
+    chunk_of = (np.arange(n) * chunks) // n
+    neg = np.array(prep["neg_idx"])[chunk_of]                      # [n, negs]
+    ht, rt = torch.from_numpy(h), torch.from_numpy(rel_emb)
+    np.testing.assert_allclose(pos, torch.einsum("id,id,id->i", ht[s], rt[rel], ht[o]).numpy(), rtol=1e-12)
+    np.testing.assert_allclose(nd, torch.einsum("id,id,itd->it", ht[s], rt[rel], ht[neg]).numpy(), rtol=1e-12)
+    np.testing.assert_allclose(ns, torch.einsum("itd,id,id->it", ht[neg], rt[rel], ht[o]).numpy(), rtol=1e-12)
+    # relation == 1: a plain dot product / matmul
+    pos1, nd1, _ = O.distmult_scores(h, np.ones((5, 8)), prep, rel, chunks)
+    np.testing.assert_allclose(pos1, (h[s] * h[o]).sum(1), rtol=1e-12)
+    np.testing.assert_allclose(nd1, np.stack([h[neg[i]] @ h[s[i]] for i in range(n)]), rtol=1e-12)
+    # symmetric in source and destination
+    prep2 = dict(prep, src_idx=prep["dst_idx"], dst_idx=prep["src_idx"])
+    pos2, nd2, ns2 = O.distmult_scores(h, rel_emb, prep2, rel, chunks)
+    np.testing.assert_allclose(pos2, pos, rtol=1e-12)
+    np.testing.assert_allclose(nd2, ns, rtol=1e-12)
