@@ -1,0 +1,252 @@
+/*
+ * mgdense — DENSE multi-hop neighbourhood sampling, GraphSage forward over DENSE and
+ * DistMult link scoring on one NVIDIA B200 (sm_100a), behind a plain C ABI.
+ *
+ * The operations are those of MariusGNN (EuroSys '23): Algorithm 1 (multi-hop sampling
+ * into the DENSE arrays), Section 4.1 (oneHopSample / computeNextDelta over the in-memory
+ * subgraph), Section 4.2 (repr_map, layer evaluation, Algorithm 2's update, Algorithm 3's
+ * aggregation) and the partition buffer of Section 3.
+ *
+ * Conventions
+ *  - Every call returns an int32 status: MG_OK (0) or a negative MG_ERR_* code; nothing
+ *    throws, aborts or traps.  mg_last_error(ctx) gives a message owned by the context.
+ *  - "host" / "device" is stated per pointer.  Input arrays are caller-owned and only read
+ *    during the call unless a parameter says the library keeps (borrows) the pointer.
+ *  - Opaque handles are created and destroyed by the library.  A context is bound to one
+ *    device and one stream (the stream handed to mg_create; 0 = the default stream); all
+ *    kernels run on it.  Partition swaps run on a library-owned side stream.
+ *  - Node ids are int32.  CSR row offsets are int32 or int64 on input.
+ *  - A context is not thread-safe; use one per host thread.
+ */
+#ifndef MGDENSE_H
+#define MGDENSE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MG_OK 0
+#define MG_ERR_ARG (-1)         /* null pointer, negative size, k <= 0, fanout <= 0, id out of range */
+#define MG_ERR_STATE (-2)       /* call made before the data it needs was loaded */
+#define MG_ERR_NONRESIDENT (-3) /* a target lies in a partition that is not in the buffer */
+#define MG_ERR_DUPLICATE (-4)   /* a batch lists the same target twice (Algorithm 1 wants unique ids) */
+#define MG_ERR_CAPACITY (-5)    /* a caller-set capacity was exceeded; nothing was written out of bounds */
+#define MG_ERR_OOM (-6)         /* a device or host allocation failed */
+#define MG_ERR_TIMEOUT (-7)     /* a bounded wait on the side stream ran out */
+#define MG_ERR_CUDA (-8)        /* a CUDA runtime call failed; see mg_last_error */
+
+#define MG_DTYPE_F32 0
+#define MG_DTYPE_F16 1
+
+#define MG_BACKING_HBM 0  /* the whole feature table lives in device memory */
+#define MG_BACKING_HOST 1 /* the table stays in (preferably pinned) host memory; only the
+                             buffer's partitions are copied into device slots */
+
+#define MG_GEMM_TF32 0 /* tcgen05 kind::tf32, operands rounded to nearest TF32, fp32 accumulate */
+#define MG_GEMM_FP32 1 /* CUDA-core fp32 FMA; slow, for isolating tensor-core rounding */
+
+#define MG_CORRUPT_DST 1
+#define MG_CORRUPT_SRC 2
+#define MG_CORRUPT_BOTH 3
+
+#define MG_MAX_HOPS 8
+#define MG_MAX_FANOUT 1024
+#define MG_MAX_BATCHES 4096
+#define MG_MAX_PARTS 256
+
+typedef struct mg_ctx mg_ctx;
+typedef struct mg_dense mg_dense;
+typedef struct mg_model mg_model;
+typedef struct mg_lp_batch mg_lp_batch;
+
+/* Capacities of one mg_sample_many call.  A zero field selects the worst-case bound
+ * computed from the targets and fanouts, clamped to the graph's size. */
+typedef struct mg_sample_caps {
+    int64_t max_nodes_total;     /* sum over batches of |node_ids| */
+    int64_t max_entries_total;   /* sum over batches of |nbrs| */
+    int32_t max_nodes_per_batch; /* |node_ids| of one batch; sizes the per-batch id table */
+} mg_sample_caps;
+
+/* One batch's DENSE in the paper's layout (Section 4.1): node_ids = [Delta_0 .. Delta_k],
+ * nbrs = [nbrs(Delta_1) .. nbrs(Delta_k)].  All pointers are DEVICE pointers into a buffer
+ * owned by the mg_dense, valid until the next mg_dense_view / mg_sample* on it or its free.
+ * node_id_offsets has k+2 entries (last = n_nodes); nbr_offsets has n_sampled+1 entries
+ * (last = n_entries) — the terminal entries Algorithm 2 reads on the last layer. */
+typedef struct mg_dense_arrays {
+    int32_t k;
+    int32_t n_nodes;   /* |node_ids| */
+    int32_t n_sampled; /* nodes that carry neighbours = n_nodes - |Delta_0| */
+    int32_t n_entries; /* |nbrs| */
+    const int32_t* node_ids;
+    const int32_t* node_id_offsets;
+    const int32_t* nbrs;
+    const int32_t* nbr_offsets;
+    const int32_t* repr_map;
+} mg_dense_arrays;
+
+/* ---- context ---------------------------------------------------------------------- */
+
+/* Create a context on `device`, issuing work on `stream` (a cudaStream_t; NULL = default
+ * stream).  *out receives the handle. */
+int mg_create(mg_ctx** out, int device, void* stream);
+/* Free everything the context owns (graph copy, buffer slots, workspaces).  Handles made
+ * from it (mg_dense, mg_model, mg_lp_batch) must be freed first. */
+int mg_destroy(mg_ctx* ctx);
+/* Message of the last failed call on this context ("" if none).  Owned by the context. */
+const char* mg_last_error(const mg_ctx* ctx);
+
+/* ---- graph store and partition buffer (Section 3) ------------------------------------- */
+
+/* Load the sampling adjacency as CSR: row v lists the nodes v aggregates from (Figure 1:
+ * the incoming neighbourhood), each row sorted by neighbour id.  row_offsets has
+ * n_nodes+1 entries of int32 (offsets_are_i64 = 0) or int64; nbrs has n_edges int32
+ * entries.  Both pointers are host (ptrs_are_device = 0) or device pointers; the library
+ * copies them.  Resets partitioning to one resident partition.  Errors: MG_ERR_ARG on
+ * null/negative/non-monotone sizes (offsets[0] != 0 or offsets[n] != n_edges), MG_ERR_OOM. */
+int mg_load_graph(mg_ctx* ctx, int64_t n_nodes, int64_t n_edges, const void* row_offsets,
+                  int offsets_are_i64, const int32_t* nbrs, int ptrs_are_device);
+
+/* Split the nodes into n_parts physical partitions of ceil(n_nodes / n_parts) contiguous
+ * ids (the last one short) — the sequential lookup table of Section 3.  All partitions
+ * start non-resident except when n_parts == 1.  Drops any loaded feature table. */
+int mg_set_partitioning(mg_ctx* ctx, int32_t n_parts);
+
+/* Attach the table of base representations (Section 2): n_nodes rows of `dim` values of
+ * `dtype`, row-major.  dim * sizeof(dtype) must be a multiple of 16 bytes.
+ *  - MG_BACKING_HBM: every row is kept in device memory.  A device `table`
+ *    (table_is_device = 1) is BORROWED — it must outlive the context's use of it; a host
+ *    table is copied.  buffer_capacity_parts only bounds how many partitions may be
+ *    resident for sampling.
+ *  - MG_BACKING_HOST: `table` is a host pointer the caller keeps valid (pinned memory makes
+ *    the swaps asynchronous).  The library allocates buffer_capacity_parts + 1 device slots
+ *    of one partition each (the spare slot lets a one-partition swap load while the old
+ *    set is still in use) and copies partitions in as mg_set_resident asks. */
+int mg_load_features(mg_ctx* ctx, const void* table, int table_is_device, int dtype, int32_t dim,
+                     int32_t buffer_capacity_parts, int backing);
+
+/* Ask for the set of resident partitions (the S_i of Section 3).  The difference to the
+ * current set is computed; partitions to be added are copied host->device on the side
+ * stream (MG_BACKING_HOST).  Sampling and forward calls keep using the current set until
+ * mg_commit_resident.  async = 0 commits before returning.  Errors: MG_ERR_ARG (id out of
+ * range, duplicates), MG_ERR_CAPACITY (n > buffer capacity), MG_ERR_STATE. */
+int mg_set_resident(mg_ctx* ctx, const int32_t* part_ids /*host*/, int32_t n, int async);
+
+/* Wait at most timeout_ms for the pending copies (polling, never an unbounded wait), then
+ * switch the slot map to the pending set and rebuild the in-buffer view of the graph: the
+ * rows of resident nodes restricted to resident neighbours (sampling sees only in-memory
+ * nodes and edges, Section 3).  MG_ERR_TIMEOUT leaves the pending set pending. */
+int mg_commit_resident(mg_ctx* ctx, int32_t timeout_ms);
+
+/* ---- DENSE sampling (Algorithm 1) ---------------------------------------------------- */
+
+/* Sample n_batches independent mini-batches in one pass.  Batch b has targets
+ * targets[target_offsets[b] .. target_offsets[b+1]) (unique, resident node ids; caller order
+ * is kept as Delta_k), seed seeds[b].  fanouts[h], h = 0..k-1, is the maximum number of
+ * neighbours for the nodes first reached at hop h (h = 0: the targets) — ordered away from
+ * the targets.  A node with at most f resident neighbours gets all of them; otherwise f
+ * distinct row positions chosen by Floyd's algorithm from Philox4x32-10 words keyed by
+ * (seed, node, hop, slot), kept in row order.  Each new delta is the ascending list of
+ * unique new neighbours not yet in node_ids (computeNextDelta).
+ * `targets` is a host pointer, or a device pointer if targets_on_device; target_offsets,
+ * fanouts and seeds are host pointers.  *out: NULL to allocate a new mg_dense, or an
+ * existing one (of this context) to reuse its buffers.
+ * The call is synchronous: on return the sample is complete and its status checked.
+ * Errors: MG_ERR_ARG, MG_ERR_STATE, MG_ERR_NONRESIDENT, MG_ERR_DUPLICATE, MG_ERR_CAPACITY,
+ * MG_ERR_OOM. */
+int mg_sample_many(mg_ctx* ctx, const int32_t* targets, int targets_on_device,
+                   const int64_t* target_offsets, int32_t n_batches, const int32_t* fanouts,
+                   int32_t k, const uint64_t* seeds, const mg_sample_caps* caps /*nullable*/,
+                   mg_dense** out);
+
+/* One batch: mg_sample_many with n_batches = 1. */
+int mg_sample(mg_ctx* ctx, const int32_t* targets, int targets_on_device, int32_t n_targets,
+              const int32_t* fanouts, int32_t k, uint64_t seed, const mg_sample_caps* caps,
+              mg_dense** out);
+
+/* Sizes of a sample: nodes_per_hop is a HOST array of n_batches * (k+1) entries,
+ * [b * (k+1) + h] = |Delta_{k-h}| of batch b; entries_per_hop a HOST array of n_batches * k,
+ * [b * k + h] = neighbours sampled for hop h's nodes.  Either may be NULL. */
+int mg_dense_counts(const mg_dense* d, int32_t* n_batches, int32_t* k, int64_t* nodes_per_hop,
+                    int64_t* entries_per_hop);
+
+/* Materialise batch `batch` in the paper's array layout (Section 4.1 plus repr_map,
+ * Section 4.2) into a device buffer owned by `d`. */
+int mg_dense_view(mg_ctx* ctx, mg_dense* d, int32_t batch, mg_dense_arrays* out);
+
+int mg_dense_free(mg_dense* d);
+
+/* ---- GraphSage forward over DENSE (Section 4.2, Algorithms 2 and 3) -------------------- */
+
+/* k layers of widths dims[0] -> dims[1] -> ... -> dims[k]; w_self[l], w_nbr[l] are HOST
+ * row-major [dims[l], dims[l+1]] fp32, bias[l] HOST [dims[l+1]] (copied).  Layer l+1
+ * computes act(self . w_self + mean(sampled neighbours) . w_nbr + bias) with ReLU on all
+ * but the last layer.  dims must be multiples of 4. */
+int mg_model_create(mg_ctx* ctx, int32_t k, const int32_t* dims, const float* const* w_self,
+                    const float* const* w_nbr, const float* const* bias, int gemm_precision,
+                    mg_model** out);
+int mg_model_free(mg_model* m);
+
+/* Forward pass for every batch of `d`.  H^0 is read straight from the feature buffer (rows
+ * of d's node ids through the partition->slot map); layer l aggregates over the part of
+ * DENSE Algorithm 2 would leave after l-1 updates.  `out` receives H^k: one row of dims[k]
+ * fp32 per target, batches concatenated, caller's target order; a device pointer, or a host
+ * pointer if out_on_device = 0.  Errors: MG_ERR_STATE (no features / sample and model
+ * depths differ / feature dim != dims[0]), MG_ERR_OOM. */
+int mg_forward(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out, int out_on_device);
+
+/* H^0 of one batch: base representations of its node_ids, rows in the order of
+ * mg_dense_view's node_ids, widened to fp32.  out_dev: DEVICE [n_nodes, feature dim]. */
+int mg_gather_h0(mg_ctx* ctx, mg_dense* d, int32_t batch, float* out_dev);
+
+/* After mg_forward: H^layer (1..k) of one batch, rows in the order of the paper's node_ids
+ * from node_id_offsets[layer] on.  out_dev: DEVICE [rows, dims[layer]]. */
+int mg_layer_output(mg_ctx* ctx, const mg_model* m, mg_dense* d, int32_t layer, int32_t batch,
+                    float* out_dev);
+
+/* ---- link prediction: shared negatives, target union, DistMult ------------------------ */
+
+/* Prepare a batch of n_edges training edges (HOST int32 src / rel / dst; dst aggregates
+ * from src).  Edge i belongs to chunk floor(i * n_chunks / n_edges); chunk c shares
+ * negs_per_chunk negatives, negative t being the resident node number
+ * mulhi(Philox4x32-10(counter = (c, t, 0xFFFFFFFF, 0), key = seed).word0, #resident nodes)
+ * counted in ascending partition order.  The targets of the batch are the ascending unique
+ * union of all sources, destinations and negatives.  Errors as mg_sample_many. */
+int mg_lp_prepare(mg_ctx* ctx, const int32_t* src, const int32_t* rel, const int32_t* dst,
+                  int64_t n_edges, int32_t n_chunks, int32_t negs_per_chunk, uint64_t seed,
+                  mg_lp_batch** out);
+/* DEVICE pointers owned by the batch: the target ids (ascending), and for each edge /
+ * negative its row in the target list.  Any out pointer may be NULL. */
+int mg_lp_view(const mg_lp_batch* lp, int32_t* n_targets, const int32_t** targets,
+               const int32_t** src_idx, const int32_t** dst_idx, const int32_t** neg_ids,
+               const int32_t** neg_idx);
+int mg_lp_free(mg_lp_batch* lp);
+
+/* DistMult: pos[i] = sum_d h[s_i,d] rel_emb[r_i,d] h[o_i,d]; neg_dst[i,t] the same with the
+ * destination replaced by negative t of edge i's chunk, neg_src[i,t] with the source
+ * replaced.  h_dev: DEVICE [n_targets, dim] (mg_forward's output for the batch's targets);
+ * rel_emb_dev: DEVICE [n_relations, dim]; outputs DEVICE: pos [n_edges],
+ * neg_* [n_edges, negs_per_chunk] (only the sides `corrupt` names are written).  The kernels are
+ * queued on the context's stream; the call does not wait for them. */
+int mg_distmult_score(mg_ctx* ctx, const mg_lp_batch* lp, const float* h_dev, int32_t dim,
+                      const float* rel_emb_dev, int32_t n_relations, int corrupt, float* pos_out,
+                      float* neg_dst_out, float* neg_src_out);
+
+/* ---- instrumentation ------------------------------------------------------------------ */
+
+/* Number of kernels this context has launched since creation. */
+int64_t mg_kernel_launches(const mg_ctx* ctx);
+
+/* Per-phase device timing.  While enabled, every group of kernels the library issues is
+ * bracketed by CUDA events on the context's stream.  mg_profile_read synchronises the stream
+ * and returns, for each phase, its name (static string), the summed milliseconds and the
+ * number of kernel launches since the last reset; arrays must hold 32 entries. */
+int mg_profile(mg_ctx* ctx, int enable);
+int mg_profile_read(mg_ctx* ctx, int32_t* n_phases, const char** names, double* ms, int64_t* launches,
+                    int reset);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MGDENSE_H */

@@ -1,0 +1,345 @@
+"""Thin ctypes binding over libmgdense.so: argument marshalling only.
+
+Every step of the path (sampling, relabelling, aggregation, GEMMs, scoring) runs in the
+library's CUDA kernels; torch is used here for device memory and streams.  There is no
+CPU fallback: a missing library or a failing call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import numpy as np
+import torch
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libmgdense.so")
+
+MG_OK = 0
+ERR_NAMES = {-1: "MG_ERR_ARG", -2: "MG_ERR_STATE", -3: "MG_ERR_NONRESIDENT", -4: "MG_ERR_DUPLICATE",
+             -5: "MG_ERR_CAPACITY", -6: "MG_ERR_OOM", -7: "MG_ERR_TIMEOUT", -8: "MG_ERR_CUDA"}
+DTYPE_F32, DTYPE_F16 = 0, 1
+BACKING_HBM, BACKING_HOST = 0, 1
+GEMM_TF32, GEMM_FP32 = 0, 1
+CORRUPT_DST, CORRUPT_SRC, CORRUPT_BOTH = 1, 2, 3
+
+# every symbol include/mgdense.h declares
+EXPORTS = [
+    "mg_create", "mg_destroy", "mg_last_error", "mg_load_graph", "mg_set_partitioning",
+    "mg_load_features", "mg_set_resident", "mg_commit_resident", "mg_sample_many", "mg_sample",
+    "mg_dense_counts", "mg_dense_view", "mg_dense_free", "mg_model_create", "mg_model_free",
+    "mg_forward", "mg_gather_h0", "mg_layer_output", "mg_lp_prepare", "mg_lp_view", "mg_lp_free",
+    "mg_distmult_score", "mg_kernel_launches", "mg_profile", "mg_profile_read",
+]
+
+
+class MgError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"{ERR_NAMES.get(code, code)}: {msg}")
+        self.code = code
+
+
+class SampleCaps(C.Structure):
+    _fields_ = [("max_nodes_total", C.c_int64), ("max_entries_total", C.c_int64),
+                ("max_nodes_per_batch", C.c_int32)]
+
+
+class DenseArrays(C.Structure):
+    _fields_ = [("k", C.c_int32), ("n_nodes", C.c_int32), ("n_sampled", C.c_int32), ("n_entries", C.c_int32),
+                ("node_ids", C.c_void_p), ("node_id_offsets", C.c_void_p), ("nbrs", C.c_void_p),
+                ("nbr_offsets", C.c_void_p), ("repr_map", C.c_void_p)]
+
+
+_lib = None
+
+
+def load_library(path: str = LIB_PATH) -> C.CDLL:
+    """dlopen the library (works without a GPU; calls then fail with MG_ERR_CUDA)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(path):
+            raise RuntimeError(f"{path} is missing: run `python -m paper_2202_02365_b200.build` "
+                               "(there is no fallback implementation)")
+        _lib = C.CDLL(path)
+        _lib.mg_last_error.restype = C.c_char_p
+        _lib.mg_kernel_launches.restype = C.c_int64
+    return _lib
+
+
+def _ptr(t: torch.Tensor | None):
+    return C.c_void_p(t.data_ptr()) if t is not None else C.c_void_p(0)
+
+
+def _host(x, dtype) -> torch.Tensor:
+    t = torch.as_tensor(x, dtype=dtype)
+    return t.cpu().contiguous()
+
+
+class _DeviceInts:
+    """A library-owned device buffer of n int32 values, exposed through the CUDA array interface."""
+
+    def __init__(self, ptr: int, n: int):
+        self.__cuda_array_interface__ = {"shape": (n,), "typestr": "<i4", "data": (int(ptr), True), "version": 2}
+
+
+def _from_dev(ptr, n: int, device) -> torch.Tensor:
+    """Copy n int32 values out of a library-owned device buffer into a torch tensor."""
+    if n == 0 or not ptr:
+        return torch.empty(0, dtype=torch.int32, device=device)
+    return torch.as_tensor(_DeviceInts(ptr, n), device=device).clone()
+
+
+@dataclass
+class DenseView:
+    """One batch's DENSE in the paper's layout (device int32 tensors)."""
+    node_ids: torch.Tensor
+    node_id_offsets: torch.Tensor
+    nbrs: torch.Tensor
+    nbr_offsets: torch.Tensor
+    repr_map: torch.Tensor
+
+
+class Dense:
+    def __init__(self, ctx: "Context"):
+        self.ctx = ctx
+        self.handle = C.c_void_p(0)
+
+    def counts(self):
+        lib = self.ctx.lib
+        nb, k = C.c_int32(0), C.c_int32(0)
+        self.ctx._check(lib.mg_dense_counts(self.handle, C.byref(nb), C.byref(k), None, None))
+        nodes = torch.zeros((nb.value, k.value + 1), dtype=torch.int64)
+        ents = torch.zeros((nb.value, k.value), dtype=torch.int64)
+        self.ctx._check(lib.mg_dense_counts(self.handle, None, None, _ptr(nodes), _ptr(ents)))
+        return nodes, ents
+
+    def view(self, batch: int = 0) -> DenseView:
+        arr = DenseArrays()
+        self.ctx._check(self.ctx.lib.mg_dense_view(self.ctx.handle, self.handle, C.c_int32(batch), C.byref(arr)))
+        dev = self.ctx.device
+        return DenseView(
+            _from_dev(arr.node_ids, arr.n_nodes, dev), _from_dev(arr.node_id_offsets, arr.k + 2, dev),
+            _from_dev(arr.nbrs, arr.n_entries, dev), _from_dev(arr.nbr_offsets, arr.n_sampled + 1, dev),
+            _from_dev(arr.repr_map, arr.n_entries, dev))
+
+    def free(self):
+        if self.handle:
+            self.ctx.lib.mg_dense_free(self.handle)
+            self.handle = C.c_void_p(0)
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+class Model:
+    def __init__(self, ctx: "Context", layers, precision: int = GEMM_TF32):
+        self.ctx = ctx
+        self.handle = C.c_void_p(0)
+        k = len(layers)
+        self.dims = [int(layers[0][0].shape[0])] + [int(l[0].shape[1]) for l in layers]
+        keep = []
+        arrs = []
+        for idx in range(3):
+            ptrs = (C.c_void_p * k)()
+            for i, l in enumerate(layers):
+                t = _host(l[idx], torch.float32)
+                keep.append(t)
+                ptrs[i] = t.data_ptr()
+            arrs.append(ptrs)
+        dims = (C.c_int32 * (k + 1))(*self.dims)
+        ctx._check(ctx.lib.mg_model_create(ctx.handle, C.c_int32(k), dims, arrs[0], arrs[1], arrs[2],
+                                           C.c_int(precision), C.byref(self.handle)))
+
+    def free(self):
+        if self.handle:
+            self.ctx.lib.mg_model_free(self.handle)
+            self.handle = C.c_void_p(0)
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+class LpBatch:
+    def __init__(self, ctx: "Context"):
+        self.ctx = ctx
+        self.handle = C.c_void_p(0)
+        self.n_edges = 0
+        self.negs = 0
+
+    def view(self):
+        n = C.c_int32(0)
+        p = [C.c_void_p(0) for _ in range(5)]
+        self.ctx._check(self.ctx.lib.mg_lp_view(self.handle, C.byref(n), *[C.byref(x) for x in p]))
+        dev = self.ctx.device
+        nt = n.value
+        return {
+            "targets": _from_dev(p[0].value, nt, dev), "src_idx": _from_dev(p[1].value, self.n_edges, dev),
+            "dst_idx": _from_dev(p[2].value, self.n_edges, dev),
+            "neg_ids": _from_dev(p[3].value, self.n_chunks * self.negs, dev).view(self.n_chunks, self.negs),
+            "neg_idx": _from_dev(p[4].value, self.n_chunks * self.negs, dev).view(self.n_chunks, self.negs),
+        }
+
+    def free(self):
+        if self.handle:
+            self.ctx.lib.mg_lp_free(self.handle)
+            self.handle = C.c_void_p(0)
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+class Context:
+    """One device, one stream.  Mirrors the C calls one to one."""
+
+    def __init__(self, device: int = 0, stream: torch.cuda.Stream | None = None):
+        self.lib = load_library()
+        if not torch.cuda.is_available():
+            raise RuntimeError("mgdense needs a CUDA device; there is no CPU path")
+        self.device = torch.device("cuda", device)
+        self.stream = stream
+        self.handle = C.c_void_p(0)
+        sptr = C.c_void_p(stream.cuda_stream if stream is not None else 0)
+        rc = self.lib.mg_create(C.byref(self.handle), C.c_int(device), sptr)
+        if rc != MG_OK:
+            raise MgError(rc, "mg_create failed")
+        self._keep = {}
+
+    # -- plumbing
+    def _check(self, rc: int):
+        if rc != MG_OK:
+            msg = self.lib.mg_last_error(self.handle)
+            raise MgError(rc, msg.decode() if msg else "")
+
+    def close(self):
+        if self.handle:
+            self.lib.mg_destroy(self.handle)
+            self.handle = C.c_void_p(0)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def kernel_launches(self) -> int:
+        return int(self.lib.mg_kernel_launches(self.handle))
+
+    def profile(self, on: bool):
+        self._check(self.lib.mg_profile(self.handle, C.c_int(1 if on else 0)))
+
+    def profile_read(self, reset: bool = True):
+        n = C.c_int32(0)
+        names = (C.c_char_p * 32)()
+        ms = (C.c_double * 32)()
+        launches = (C.c_int64 * 32)()
+        self._check(self.lib.mg_profile_read(self.handle, C.byref(n), names, ms, launches, C.c_int(1 if reset else 0)))
+        return {names[i].decode(): {"ms": ms[i], "launches": launches[i]} for i in range(n.value)}
+
+    # -- graph store and buffer
+    def load_graph(self, row_offsets: torch.Tensor, nbrs: torch.Tensor):
+        assert row_offsets.dtype in (torch.int32, torch.int64) and nbrs.dtype == torch.int32
+        assert row_offsets.is_cuda == nbrs.is_cuda
+        row_offsets, nbrs = row_offsets.contiguous(), nbrs.contiguous()
+        n_nodes, n_edges = row_offsets.numel() - 1, nbrs.numel()
+        self._check(self.lib.mg_load_graph(self.handle, C.c_int64(n_nodes), C.c_int64(n_edges), _ptr(row_offsets),
+                                           C.c_int(row_offsets.dtype == torch.int64), _ptr(nbrs),
+                                           C.c_int(row_offsets.is_cuda)))
+        self.n_nodes = n_nodes
+
+    def set_partitioning(self, n_parts: int):
+        self._check(self.lib.mg_set_partitioning(self.handle, C.c_int32(n_parts)))
+
+    def load_features(self, table: torch.Tensor, capacity_parts: int = 1, backing: int = BACKING_HBM):
+        assert table.dim() == 2 and table.is_contiguous()
+        dt = {torch.float32: DTYPE_F32, torch.float16: DTYPE_F16}[table.dtype]
+        self._keep["features"] = table          # device tables are borrowed, host tables stay the backing store
+        self._check(self.lib.mg_load_features(self.handle, _ptr(table), C.c_int(table.is_cuda), C.c_int(dt),
+                                              C.c_int32(table.shape[1]), C.c_int32(capacity_parts), C.c_int(backing)))
+
+    def set_resident(self, parts, async_: bool = False):
+        p = _host(list(parts), torch.int32)
+        self._check(self.lib.mg_set_resident(self.handle, _ptr(p), C.c_int32(p.numel()), C.c_int(1 if async_ else 0)))
+
+    def commit_resident(self, timeout_ms: int = 60000):
+        self._check(self.lib.mg_commit_resident(self.handle, C.c_int32(timeout_ms)))
+
+    # -- sampling
+    def sample_many(self, targets: torch.Tensor, target_offsets, fanouts, seeds, caps=None, out: Dense | None = None) -> Dense:
+        assert targets.dtype == torch.int32
+        targets = targets.contiguous()
+        offs = _host(target_offsets, torch.int64)
+        fo = _host(list(fanouts), torch.int32)
+        sd = np.ascontiguousarray(np.array([int(s) & 0xFFFFFFFFFFFFFFFF for s in seeds], dtype=np.uint64))
+        d = out if out is not None else Dense(self)
+        cp = None
+        if caps is not None:
+            cp = SampleCaps(int(caps.get("max_nodes_total", 0)), int(caps.get("max_entries_total", 0)),
+                            int(caps.get("max_nodes_per_batch", 0)))
+        self._check(self.lib.mg_sample_many(self.handle, _ptr(targets), C.c_int(targets.is_cuda), _ptr(offs),
+                                            C.c_int32(offs.numel() - 1), _ptr(fo), C.c_int32(fo.numel()), C.c_void_p(sd.ctypes.data),
+                                            C.byref(cp) if cp is not None else None, C.byref(d.handle)))
+        return d
+
+    def sample(self, targets: torch.Tensor, fanouts, seed: int, caps=None, out: Dense | None = None) -> Dense:
+        assert targets.dtype == torch.int32
+        targets = targets.contiguous()
+        fo = _host(list(fanouts), torch.int32)
+        d = out if out is not None else Dense(self)
+        cp = None
+        if caps is not None:
+            cp = SampleCaps(int(caps.get("max_nodes_total", 0)), int(caps.get("max_entries_total", 0)),
+                            int(caps.get("max_nodes_per_batch", 0)))
+        self._check(self.lib.mg_sample(self.handle, _ptr(targets), C.c_int(targets.is_cuda), C.c_int32(targets.numel()),
+                                       _ptr(fo), C.c_int32(fo.numel()), C.c_uint64(int(seed) & 0xFFFFFFFFFFFFFFFF),
+                                       C.byref(cp) if cp is not None else None, C.byref(d.handle)))
+        return d
+
+    # -- forward
+    def model(self, layers, precision: int = GEMM_TF32) -> Model:
+        return Model(self, layers, precision)
+
+    def forward(self, model: Model, dense: Dense, out: torch.Tensor) -> torch.Tensor:
+        assert out.dtype == torch.float32 and out.is_contiguous()
+        self._check(self.lib.mg_forward(self.handle, model.handle, dense.handle, _ptr(out), C.c_int(out.is_cuda)))
+        return out
+
+    def gather_h0(self, dense: Dense, batch: int, n_nodes: int, dim: int) -> torch.Tensor:
+        out = torch.empty((n_nodes, dim), dtype=torch.float32, device=self.device)
+        self._check(self.lib.mg_gather_h0(self.handle, dense.handle, C.c_int32(batch), _ptr(out)))
+        return out
+
+    def layer_output(self, model: Model, dense: Dense, layer: int, batch: int, n_rows: int) -> torch.Tensor:
+        out = torch.empty((n_rows, model.dims[layer]), dtype=torch.float32, device=self.device)
+        self._check(self.lib.mg_layer_output(self.handle, model.handle, dense.handle, C.c_int32(layer),
+                                             C.c_int32(batch), _ptr(out)))
+        return out
+
+    # -- link prediction
+    def lp_prepare(self, src, rel, dst, n_chunks: int, negs_per_chunk: int, seed: int) -> LpBatch:
+        s, r, d = _host(src, torch.int32), _host(rel, torch.int32), _host(dst, torch.int32)
+        lp = LpBatch(self)
+        lp.n_edges, lp.negs, lp.n_chunks = s.numel(), negs_per_chunk, n_chunks
+        self._check(self.lib.mg_lp_prepare(self.handle, _ptr(s), _ptr(r), _ptr(d), C.c_int64(s.numel()),
+                                           C.c_int32(n_chunks), C.c_int32(negs_per_chunk),
+                                           C.c_uint64(int(seed) & 0xFFFFFFFFFFFFFFFF), C.byref(lp.handle)))
+        return lp
+
+    def distmult_score(self, lp: LpBatch, h: torch.Tensor, rel_emb: torch.Tensor, corrupt: int = CORRUPT_BOTH):
+        assert h.is_cuda and rel_emb.is_cuda and h.dtype == torch.float32 and rel_emb.dtype == torch.float32
+        h, rel_emb = h.contiguous(), rel_emb.contiguous()
+        pos = torch.empty(lp.n_edges, dtype=torch.float32, device=self.device)
+        nd = torch.empty((lp.n_edges, lp.negs), dtype=torch.float32, device=self.device) if corrupt & CORRUPT_DST else None
+        ns = torch.empty((lp.n_edges, lp.negs), dtype=torch.float32, device=self.device) if corrupt & CORRUPT_SRC else None
+        self._check(self.lib.mg_distmult_score(self.handle, lp.handle, _ptr(h), C.c_int32(h.shape[1]), _ptr(rel_emb),
+                                               C.c_int32(rel_emb.shape[0]), C.c_int(corrupt), _ptr(pos), _ptr(nd), _ptr(ns)))
+        return pos, nd, ns

@@ -1,0 +1,589 @@
+// Context, graph store and partition buffer (Section 3): CSR in device memory, the resident
+// set with its partition -> slot map, host-backed feature slots filled on a side stream, and
+// the in-buffer view of the graph that sampling reads.
+
+#include <stdarg.h>
+
+#include <algorithm>
+#include <chrono>
+#include <thread>
+
+#include "mg_device.cuh"
+#include "mg_internal.cuh"
+
+static const char* kPhaseNames[PH_COUNT] = {
+    "sample_init", "sample_count", "sample_scan", "sample_pick", "sample_sort", "sample_place",
+    "sample_relabel", "sample_final", "aggregate_l1", "aggregate_rest", "gemm", "distmult", "other"};
+
+int mg_fail(mg_ctx* ctx, int code, const char* fmt, ...) {
+    if (ctx) {
+        char buf[512];
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(buf, sizeof(buf), fmt, ap);
+        va_end(ap);
+        ctx->err = buf;
+    }
+    return code;
+}
+
+int mg_cuda_fail(mg_ctx* ctx, cudaError_t e, const char* what) {
+    cudaGetLastError();
+    const int code = (e == cudaErrorMemoryAllocation) ? MG_ERR_OOM : MG_ERR_CUDA;
+    return mg_fail(ctx, code, "%s: %s", what, cudaGetErrorString(e));
+}
+
+void mg_prof_begin(mg_ctx* ctx, int phase) {
+    if (!ctx->prof_on) return;
+    cudaEvent_t a, b;
+    cudaEventCreate(&a);
+    cudaEventCreate(&b);
+    cudaEventRecord(a, ctx->stream);
+    ctx->prof_pending.push_back({phase, {a, b}});
+}
+
+void mg_prof_end(mg_ctx* ctx, int phase, int n_launches) {
+    if (!ctx->prof_on) return;
+    for (size_t i = ctx->prof_pending.size(); i-- > 0;) {
+        if (ctx->prof_pending[i].first == phase) {
+            cudaEventRecord(ctx->prof_pending[i].second.second, ctx->stream);
+            break;
+        }
+    }
+    ctx->prof[phase].launches += n_launches;
+}
+
+namespace {
+
+constexpr int kThreads = 256;
+
+__global__ void k_widen_offsets(const int32_t* in, int64_t* out, int64_t n) {
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        out[i] = in[i];
+}
+
+// checks that offsets are non-decreasing and neighbour ids are in range; flags[0] |= 1 / 2
+__global__ void k_check_graph(const int64_t* off, int64_t n_nodes, const int32_t* nbrs, int64_t n_edges, uint32_t* flags) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int64_t tid = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    for (int64_t i = tid; i < n_nodes; i += stride)
+        if (off[i + 1] < off[i]) atomicOr(flags, 1u);
+    for (int64_t e = tid; e < n_edges; e += stride)
+        if (nbrs[e] < 0 || (int64_t)nbrs[e] >= n_nodes) atomicOr(flags, 2u);
+}
+
+// ---- in-buffer view: rows of resident nodes restricted to resident neighbours -------------
+constexpr int kRowLanes = 8;
+
+__global__ void __launch_bounds__(kThreads)
+k_view_count(const int64_t* __restrict__ off, const int32_t* __restrict__ nbrs, int64_t n_nodes, uint32_t part_size,
+             const int32_t* __restrict__ slot_of_part, int32_t* cnt) {
+    const int gl = threadIdx.x % kRowLanes;
+    const int64_t groups = (int64_t)gridDim.x * (kThreads / kRowLanes);
+    const int64_t n_round = (n_nodes + groups - 1) / groups * groups;  // whole warps stay in the loop together
+    for (int64_t v = blockIdx.x * (int64_t)(kThreads / kRowLanes) + threadIdx.x / kRowLanes; v < n_round; v += groups) {
+        int32_t c = 0;
+        if (v < n_nodes && slot_of_part[(uint32_t)v / part_size] >= 0) {
+            const int64_t lo = off[v], hi = off[v + 1];
+            for (int64_t e = lo + gl; e < hi; e += kRowLanes)
+                c += slot_of_part[(uint32_t)nbrs[e] / part_size] >= 0 ? 1 : 0;
+        }
+#pragma unroll
+        for (int o = kRowLanes / 2; o > 0; o >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
+        if (gl == 0 && v < n_nodes) cnt[v] = c;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_view_fill(const int64_t* __restrict__ off, const int32_t* __restrict__ nbrs, int64_t n_nodes, uint32_t part_size,
+            const int32_t* __restrict__ slot_of_part, const int64_t* __restrict__ view_off, int32_t* view_nbrs) {
+    const int lane = threadIdx.x & 31;
+    const int gl = threadIdx.x % kRowLanes;
+    const int gshift = lane - gl;
+    const int64_t groups = (int64_t)gridDim.x * (kThreads / kRowLanes);
+    const int64_t n_round = (n_nodes + groups - 1) / groups * groups;  // whole warps stay in the loop together
+    for (int64_t v = blockIdx.x * (int64_t)(kThreads / kRowLanes) + threadIdx.x / kRowLanes; v < n_round; v += groups) {
+        int64_t lo = 0, hi = 0, out = 0;
+        if (v < n_nodes && slot_of_part[(uint32_t)v / part_size] >= 0) {
+            lo = off[v]; hi = off[v + 1]; out = view_off[v];
+        }
+        // the longest row of the warp's four groups sets the trip count, so ballots stay converged
+        int64_t len = hi - lo;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) len = max(len, __shfl_xor_sync(0xFFFFFFFFu, len, o));
+        for (int64_t base = 0; base < len; base += kRowLanes) {
+            const int64_t e = lo + base + gl;
+            int32_t u = 0;
+            bool keep = false;
+            if (e < hi) { u = nbrs[e]; keep = slot_of_part[(uint32_t)u / part_size] >= 0; }
+            const uint32_t bal = (__ballot_sync(0xFFFFFFFFu, keep) >> gshift) & ((1u << kRowLanes) - 1u);
+            if (keep) view_nbrs[out + __popc(bal & ((1u << gl) - 1u))] = u;
+            out += __popc(bal);
+        }
+    }
+}
+
+// ---- 64-bit exclusive scan of int32 counts: out[i] = sum_{j<i} in[j], i in [0, n] ----------
+constexpr int kTile = 2048;
+
+__device__ __forceinline__ uint64_t block_scan64(uint64_t v, uint64_t* sm /*9*/, uint64_t* total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint64_t inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint64_t t = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+        if (lane >= o) inc += t;
+    }
+    if (lane == 31) sm[warp] = inc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint64_t run = 0;
+        for (int w = 0; w < 8; ++w) { const uint64_t t = sm[w]; sm[w] = run; run += t; }
+        sm[8] = run;
+    }
+    __syncthreads();
+    const uint64_t res = inc - v + sm[warp];
+    *total = sm[8];
+    __syncthreads();
+    return res;
+}
+
+__global__ void __launch_bounds__(kThreads) k_scan64_reduce(const int32_t* in, int64_t n, uint64_t* tile_sums) {
+    __shared__ uint64_t sm[9];
+    const int64_t ntiles = (n + kTile - 1) / kTile;
+    for (int64_t t = blockIdx.x; t < ntiles; t += gridDim.x) {
+        uint64_t s = 0;
+        const int64_t start = t * kTile + threadIdx.x * 8;
+        for (int j = 0; j < 8; ++j)
+            if (start + j < n) s += (uint64_t)in[start + j];
+        uint64_t total;
+        block_scan64(s, sm, &total);
+        if (threadIdx.x == 0) tile_sums[t] = total;
+    }
+}
+
+__global__ void k_scan64_tiles(uint64_t* tile_sums, int64_t ntiles, int64_t* total_out) {
+    // one thread block, sequential over chunks; ntiles is at most a few 10^4
+    __shared__ uint64_t sm[9];
+    __shared__ uint64_t carry_s;
+    if (threadIdx.x == 0) carry_s = 0;
+    __syncthreads();
+    for (int64_t start = 0; start < ntiles; start += kThreads) {
+        const int64_t i = start + threadIdx.x;
+        const uint64_t v = i < ntiles ? tile_sums[i] : 0ull;
+        uint64_t total;
+        const uint64_t ex = block_scan64(v, sm, &total);
+        if (i < ntiles) tile_sums[i] = carry_s + ex;
+        __syncthreads();
+        if (threadIdx.x == 0) carry_s += total;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *total_out = (int64_t)carry_s;
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_scan64_down(const int32_t* in, int64_t n, const uint64_t* tile_sums, int64_t* out) {
+    __shared__ uint64_t sm[9];
+    const int64_t ntiles = (n + kTile - 1) / kTile;
+    for (int64_t t = blockIdx.x; t < ntiles; t += gridDim.x) {
+        uint32_t v[8];
+        uint64_t s = 0;
+        const int64_t start = t * kTile + threadIdx.x * 8;
+        for (int j = 0; j < 8; ++j) { v[j] = (start + j < n) ? (uint32_t)in[start + j] : 0u; s += v[j]; }
+        uint64_t total;
+        uint64_t run = block_scan64(s, sm, &total) + tile_sums[t];
+        for (int j = 0; j < 8; ++j) {
+            if (start + j < n) out[start + j] = (int64_t)run;
+            run += v[j];
+        }
+        if (t == ntiles - 1 && threadIdx.x == kThreads - 1) out[n] = (int64_t)(tile_sums[t] + total);
+    }
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------
+extern "C" int mg_create(mg_ctx** out, int device, void* stream) {
+    if (!out) return MG_ERR_ARG;
+    *out = nullptr;
+    int n_dev = 0;
+    cudaError_t e = cudaGetDeviceCount(&n_dev);
+    if (e != cudaSuccess || device < 0 || device >= n_dev) { cudaGetLastError(); return MG_ERR_CUDA; }
+    if (cudaSetDevice(device) != cudaSuccess) { cudaGetLastError(); return MG_ERR_CUDA; }
+    mg_ctx* c = new mg_ctx();
+    c->device = device;
+    c->stream = (cudaStream_t)stream;
+    cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, device);
+    if (c->n_sms <= 0) c->n_sms = 148;
+    for (int i = 0; i < PH_COUNT; ++i) c->prof[i] = ProfPhase{kPhaseNames[i], 0.0, 0};
+    if (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaMalloc((void**)&c->d_slot_of_part, sizeof(int32_t) * MG_MAX_PARTS) != cudaSuccess ||
+        cudaMalloc((void**)&c->d_res_prefix, sizeof(int64_t) * (MG_MAX_PARTS + 1)) != cudaSuccess) {
+        cudaGetLastError();
+        delete c;
+        return MG_ERR_CUDA;
+    }
+    *out = c;
+    return MG_OK;
+}
+
+static void free_view(mg_ctx* c) {
+    if (c->view_owned) { cudaFree(c->view_off); cudaFree(c->view_nbrs); }
+    c->view_off = nullptr; c->view_nbrs = nullptr; c->view_owned = false; c->view_edges = 0;
+}
+
+static void free_features(mg_ctx* c) {
+    if (c->slots_owned) cudaFree(c->slots);
+    c->slots = nullptr; c->slots_owned = false; c->host_table = nullptr; c->feat_dim = 0; c->n_slots = 0;
+}
+
+extern "C" int mg_destroy(mg_ctx* c) {
+    if (!c) return MG_OK;
+    cudaSetDevice(c->device);
+    cudaStreamSynchronize(c->stream);
+    cudaStreamSynchronize(c->side);
+    for (auto ev : c->pending_events) cudaEventDestroy(ev);
+    for (auto& p : c->prof_pending) { cudaEventDestroy(p.second.first); cudaEventDestroy(p.second.second); }
+    free_view(c);
+    free_features(c);
+    cudaFree(c->row_off); cudaFree(c->nbrs); cudaFree(c->d_slot_of_part); cudaFree(c->d_res_prefix);
+    cudaFree(c->ws_x); cudaFree(c->ws_h[0]); cudaFree(c->ws_h[1]);
+    cudaStreamDestroy(c->side);
+    delete c;
+    return MG_OK;
+}
+
+extern "C" const char* mg_last_error(const mg_ctx* c) { return c ? c->err.c_str() : "null context"; }
+extern "C" int64_t mg_kernel_launches(const mg_ctx* c) { return c ? c->launches : 0; }
+
+extern "C" int mg_profile(mg_ctx* c, int enable) {
+    if (!c) return MG_ERR_ARG;
+    c->prof_on = enable != 0;
+    return MG_OK;
+}
+
+extern "C" int mg_profile_read(mg_ctx* c, int32_t* n_phases, const char** names, double* ms, int64_t* launches, int reset) {
+    if (!c) return MG_ERR_ARG;
+    cudaSetDevice(c->device);
+    cudaStreamSynchronize(c->stream);
+    for (auto& p : c->prof_pending) {
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, p.second.first, p.second.second) == cudaSuccess) c->prof[p.first].ms += t;
+        else cudaGetLastError();
+        cudaEventDestroy(p.second.first);
+        cudaEventDestroy(p.second.second);
+    }
+    c->prof_pending.clear();
+    if (n_phases) *n_phases = PH_COUNT;
+    for (int i = 0; i < PH_COUNT; ++i) {
+        if (names) names[i] = c->prof[i].name;
+        if (ms) ms[i] = c->prof[i].ms;
+        if (launches) launches[i] = c->prof[i].launches;
+        if (reset) { c->prof[i].ms = 0; c->prof[i].launches = 0; }
+    }
+    return MG_OK;
+}
+
+// upload the committed slot map and the resident-node prefix counts
+static int upload_slot_map(mg_ctx* c) {
+    int32_t slots[MG_MAX_PARTS];
+    int64_t prefix[MG_MAX_PARTS + 1];
+    prefix[0] = 0;
+    for (int p = 0; p < MG_MAX_PARTS; ++p) {
+        slots[p] = p < c->n_parts ? c->slot_of_part[p] : -1;
+        int64_t sz = 0;
+        if (p < c->n_parts && slots[p] >= 0) sz = std::min<int64_t>(c->part_size, c->n_nodes - (int64_t)p * c->part_size);
+        prefix[p + 1] = prefix[p] + std::max<int64_t>(sz, 0);
+    }
+    c->n_resident_nodes = prefix[MG_MAX_PARTS];
+    MG_CUDA(c, cudaMemcpyAsync(c->d_slot_of_part, slots, sizeof(slots), cudaMemcpyHostToDevice, c->stream));
+    MG_CUDA(c, cudaMemcpyAsync(c->d_res_prefix, prefix, sizeof(prefix), cudaMemcpyHostToDevice, c->stream));
+    MG_CUDA(c, cudaStreamSynchronize(c->stream));
+    return MG_OK;
+}
+
+static int rebuild_view(mg_ctx* c) {
+    bool all = true;
+    for (int p = 0; p < c->n_parts; ++p) all = all && c->slot_of_part[p] >= 0;
+    if (all) {
+        free_view(c);
+        c->view_off = c->row_off; c->view_nbrs = c->nbrs; c->view_edges = c->n_edges; c->view_owned = false;
+        return MG_OK;
+    }
+    if (!c->view_owned) {
+        c->view_off = nullptr; c->view_nbrs = nullptr;
+        if (cudaMalloc((void**)&c->view_off, sizeof(int64_t) * (c->n_nodes + 1)) != cudaSuccess ||
+            cudaMalloc((void**)&c->view_nbrs, sizeof(int32_t) * std::max<int64_t>(c->n_edges, 1)) != cudaSuccess) {
+            cudaGetLastError();
+            cudaFree(c->view_off);
+            c->view_off = nullptr; c->view_nbrs = nullptr;
+            return mg_fail(c, MG_ERR_OOM, "allocation of the in-buffer graph view failed");
+        }
+        c->view_owned = true;
+    }
+    const int64_t n = c->n_nodes;
+    const int64_t ntiles = (n + kTile - 1) / kTile;
+    int32_t* cnt = nullptr;
+    uint64_t* tiles = nullptr;
+    int64_t* d_total = nullptr;
+    if (cudaMalloc((void**)&cnt, sizeof(int32_t) * std::max<int64_t>(n, 1)) != cudaSuccess ||
+        cudaMalloc((void**)&tiles, sizeof(uint64_t) * (ntiles + 1)) != cudaSuccess ||
+        cudaMalloc((void**)&d_total, sizeof(int64_t)) != cudaSuccess) {
+        cudaGetLastError();
+        cudaFree(cnt); cudaFree(tiles); cudaFree(d_total);
+        return mg_fail(c, MG_ERR_OOM, "scratch allocation for the in-buffer graph view failed");
+    }
+    const int grid = mg_grid(c, 8);
+    cudaStream_t st = c->stream;
+    k_view_count<<<grid, kThreads, 0, st>>>(c->row_off, c->nbrs, n, (uint32_t)c->part_size, c->d_slot_of_part, cnt);
+    k_scan64_reduce<<<grid, kThreads, 0, st>>>(cnt, n, tiles);
+    k_scan64_tiles<<<1, kThreads, 0, st>>>(tiles, ntiles, d_total);
+    k_scan64_down<<<grid, kThreads, 0, st>>>(cnt, n, tiles, c->view_off);
+    k_view_fill<<<grid, kThreads, 0, st>>>(c->row_off, c->nbrs, n, (uint32_t)c->part_size, c->d_slot_of_part, c->view_off, c->view_nbrs);
+    c->launches += 5;
+    int64_t total = 0;
+    cudaError_t e = cudaMemcpyAsync(&total, d_total, sizeof(int64_t), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    cudaFree(cnt); cudaFree(tiles); cudaFree(d_total);
+    if (e != cudaSuccess) return mg_cuda_fail(c, e, "rebuild of the in-buffer graph view");
+    c->view_edges = total;
+    return MG_OK;
+}
+
+extern "C" int mg_load_graph(mg_ctx* c, int64_t n_nodes, int64_t n_edges, const void* row_offsets, int offsets_are_i64,
+                             const int32_t* nbrs, int ptrs_are_device) {
+    if (!c) return MG_ERR_ARG;
+    if (!row_offsets || (n_edges > 0 && !nbrs)) return mg_fail(c, MG_ERR_ARG, "null argument");
+    if (n_nodes <= 0 || n_nodes >= (1ll << 31) - 1 || n_edges < 0) return mg_fail(c, MG_ERR_ARG, "n_nodes must be in [1, 2^31 - 2], n_edges >= 0");
+    MG_CUDA(c, cudaSetDevice(c->device));
+    MG_CUDA(c, cudaStreamSynchronize(c->stream));
+    free_view(c);
+    free_features(c);
+    cudaFree(c->row_off); cudaFree(c->nbrs);
+    c->row_off = nullptr; c->nbrs = nullptr; c->n_nodes = 0; c->n_edges = 0;
+    const cudaMemcpyKind kind = ptrs_are_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+    if (cudaMalloc((void**)&c->row_off, sizeof(int64_t) * (n_nodes + 1)) != cudaSuccess ||
+        cudaMalloc((void**)&c->nbrs, sizeof(int32_t) * std::max<int64_t>(n_edges, 1)) != cudaSuccess) {
+        cudaGetLastError();
+        cudaFree(c->row_off); c->row_off = nullptr;
+        return mg_fail(c, MG_ERR_OOM, "allocation of the graph store failed");
+    }
+    cudaStream_t st = c->stream;
+    if (offsets_are_i64) {
+        MG_CUDA(c, cudaMemcpyAsync(c->row_off, row_offsets, sizeof(int64_t) * (n_nodes + 1), kind, st));
+    } else {
+        int32_t* tmp = nullptr;
+        MG_CUDA(c, cudaMalloc((void**)&tmp, sizeof(int32_t) * (n_nodes + 1)));
+        cudaError_t e = cudaMemcpyAsync(tmp, row_offsets, sizeof(int32_t) * (n_nodes + 1), kind, st);
+        if (e == cudaSuccess) {
+            k_widen_offsets<<<mg_grid(c, 4), kThreads, 0, st>>>(tmp, c->row_off, n_nodes + 1);
+            c->launches++;
+            e = cudaStreamSynchronize(st);
+        }
+        cudaFree(tmp);
+        if (e != cudaSuccess) return mg_cuda_fail(c, e, "offset upload");
+    }
+    if (n_edges > 0) MG_CUDA(c, cudaMemcpyAsync(c->nbrs, nbrs, sizeof(int32_t) * n_edges, kind, st));
+    // validate on the device; only the two end offsets come back
+    uint32_t* flags = nullptr;
+    MG_CUDA(c, cudaMalloc((void**)&flags, sizeof(uint32_t)));
+    cudaMemsetAsync(flags, 0, sizeof(uint32_t), st);
+    k_check_graph<<<mg_grid(c, 8), kThreads, 0, st>>>(c->row_off, n_nodes, c->nbrs, n_edges, flags);
+    c->launches++;
+    uint32_t h_flags = 0;
+    int64_t ends[2] = {0, 0};
+    cudaMemcpyAsync(&h_flags, flags, sizeof(uint32_t), cudaMemcpyDeviceToHost, st);
+    cudaMemcpyAsync(&ends[0], c->row_off, sizeof(int64_t), cudaMemcpyDeviceToHost, st);
+    cudaMemcpyAsync(&ends[1], c->row_off + n_nodes, sizeof(int64_t), cudaMemcpyDeviceToHost, st);
+    cudaError_t e = cudaStreamSynchronize(st);
+    cudaFree(flags);
+    if (e != cudaSuccess) return mg_cuda_fail(c, e, "graph upload");
+    if (h_flags || ends[0] != 0 || ends[1] != n_edges) {
+        cudaFree(c->row_off); cudaFree(c->nbrs);
+        c->row_off = nullptr; c->nbrs = nullptr;
+        return mg_fail(c, MG_ERR_ARG, "malformed CSR: %s", (h_flags & 2) ? "neighbour id out of range"
+                                                            : (h_flags & 1) ? "row offsets decrease"
+                                                                            : "row_offsets[0] != 0 or row_offsets[n_nodes] != n_edges");
+    }
+    c->n_nodes = n_nodes;
+    c->n_edges = n_edges;
+    return mg_set_partitioning(c, 1);
+}
+
+extern "C" int mg_set_partitioning(mg_ctx* c, int32_t n_parts) {
+    if (!c) return MG_ERR_ARG;
+    if (!c->row_off) return mg_fail(c, MG_ERR_STATE, "no graph loaded");
+    if (n_parts <= 0 || n_parts > MG_MAX_PARTS) return mg_fail(c, MG_ERR_ARG, "n_parts must be in [1, %d]", MG_MAX_PARTS);
+    MG_CUDA(c, cudaSetDevice(c->device));
+    MG_CUDA(c, cudaStreamSynchronize(c->stream));
+    free_features(c);
+    c->n_parts = n_parts;
+    c->part_size = (c->n_nodes + n_parts - 1) / n_parts;
+    c->capacity = n_parts;
+    c->slot_of_part.assign(n_parts, n_parts == 1 ? 0 : -1);
+    c->pending_slot.clear();
+    c->has_pending = false;
+    int rc = upload_slot_map(c);
+    if (rc) return rc;
+    return rebuild_view(c);
+}
+
+extern "C" int mg_load_features(mg_ctx* c, const void* table, int table_is_device, int dtype, int32_t dim,
+                                int32_t buffer_capacity_parts, int backing) {
+    if (!c) return MG_ERR_ARG;
+    if (!c->row_off) return mg_fail(c, MG_ERR_STATE, "no graph loaded");
+    if (!table) return mg_fail(c, MG_ERR_ARG, "null table");
+    if (dtype != MG_DTYPE_F32 && dtype != MG_DTYPE_F16) return mg_fail(c, MG_ERR_ARG, "unknown dtype");
+    const int64_t esz = dtype == MG_DTYPE_F32 ? 4 : 2;
+    if (dim <= 0 || (dim * esz) % 16 != 0) return mg_fail(c, MG_ERR_ARG, "dim * sizeof(dtype) must be a positive multiple of 16 bytes");
+    if (buffer_capacity_parts <= 0 || buffer_capacity_parts > c->n_parts) return mg_fail(c, MG_ERR_ARG, "buffer capacity must be in [1, n_parts]");
+    if (backing != MG_BACKING_HBM && backing != MG_BACKING_HOST) return mg_fail(c, MG_ERR_ARG, "unknown backing");
+    if (backing == MG_BACKING_HOST && table_is_device) return mg_fail(c, MG_ERR_ARG, "host backing needs a host table");
+    MG_CUDA(c, cudaSetDevice(c->device));
+    MG_CUDA(c, cudaStreamSynchronize(c->stream));
+    free_features(c);
+    c->feat_dtype = dtype;
+    c->row_bytes = dim * esz;
+    c->slot_bytes = c->part_size * c->row_bytes;
+    c->capacity = buffer_capacity_parts;
+    c->backing = backing;
+    int n_res = 0;
+    for (int p = 0; p < c->n_parts; ++p) n_res += c->slot_of_part[p] >= 0;
+    if (backing == MG_BACKING_HBM) {
+        if (table_is_device) {
+            c->slots = (char*)const_cast<void*>(table);
+            c->slots_owned = false;
+        } else {
+            const size_t bytes = (size_t)c->n_nodes * c->row_bytes;
+            if (cudaMalloc((void**)&c->slots, bytes) != cudaSuccess) { cudaGetLastError(); c->slots = nullptr; return mg_fail(c, MG_ERR_OOM, "feature table allocation failed"); }
+            c->slots_owned = true;
+            MG_CUDA(c, cudaMemcpyAsync(c->slots, table, bytes, cudaMemcpyHostToDevice, c->stream));
+            MG_CUDA(c, cudaStreamSynchronize(c->stream));
+        }
+        c->n_slots = c->n_parts;
+        // resident partitions keep slot == partition id
+        for (int p = 0; p < c->n_parts; ++p)
+            if (c->slot_of_part[p] >= 0) c->slot_of_part[p] = p;
+    } else {
+        c->n_slots = buffer_capacity_parts + 1;
+        const size_t bytes = (size_t)c->n_slots * c->slot_bytes;
+        if (cudaMalloc((void**)&c->slots, bytes) != cudaSuccess) { cudaGetLastError(); c->slots = nullptr; return mg_fail(c, MG_ERR_OOM, "buffer slot allocation failed"); }
+        c->slots_owned = true;
+        c->host_table = (const char*)table;
+        // whatever was resident for sampling only is reloaded into slots
+        std::vector<int32_t> keep;
+        for (int p = 0; p < c->n_parts; ++p)
+            if (c->slot_of_part[p] >= 0) keep.push_back(p);
+        c->slot_of_part.assign(c->n_parts, -1);
+        c->feat_dim = dim;
+        if ((int)keep.size() > c->capacity) keep.resize(c->capacity);
+        if (!keep.empty()) {
+            int rc = mg_set_resident(c, keep.data(), (int32_t)keep.size(), 0);
+            if (rc) return rc;
+        } else {
+            int rc = upload_slot_map(c);
+            if (rc) return rc;
+            rc = rebuild_view(c);
+            if (rc) return rc;
+        }
+    }
+    if (n_res > c->capacity && backing == MG_BACKING_HBM) {
+        // more partitions resident than the new capacity allows: keep the lowest ids
+        int kept = 0;
+        for (int p = 0; p < c->n_parts; ++p)
+            if (c->slot_of_part[p] >= 0 && ++kept > c->capacity) c->slot_of_part[p] = -1;
+    }
+    c->feat_dim = dim;
+    int rc = upload_slot_map(c);
+    if (rc) return rc;
+    return rebuild_view(c);
+}
+
+extern "C" int mg_set_resident(mg_ctx* c, const int32_t* part_ids, int32_t n, int async) {
+    if (!c) return MG_ERR_ARG;
+    if (!c->row_off) return mg_fail(c, MG_ERR_STATE, "no graph loaded");
+    if (n < 0 || (n > 0 && !part_ids)) return mg_fail(c, MG_ERR_ARG, "bad partition list");
+    if (n > c->capacity) return mg_fail(c, MG_ERR_CAPACITY, "%d partitions asked, buffer holds %d", n, c->capacity);
+    if (c->has_pending) return mg_fail(c, MG_ERR_STATE, "a resident set is already pending; commit it first");
+    std::vector<char> want(c->n_parts, 0);
+    for (int i = 0; i < n; ++i) {
+        if (part_ids[i] < 0 || part_ids[i] >= c->n_parts) return mg_fail(c, MG_ERR_ARG, "partition id out of range");
+        if (want[part_ids[i]]) return mg_fail(c, MG_ERR_ARG, "partition listed twice");
+        want[part_ids[i]] = 1;
+    }
+    MG_CUDA(c, cudaSetDevice(c->device));
+    std::vector<int32_t> next(c->n_parts, -1);
+    const bool host_backed = c->slots && c->backing == MG_BACKING_HOST;
+    if (!host_backed) {
+        for (int p = 0; p < c->n_parts; ++p) next[p] = want[p] ? p : -1;
+    } else {
+        // slots free right now can be filled at once; slots of evicted partitions only after the
+        // work already queued on the main stream has finished with them
+        std::vector<char> used(c->n_slots, 0), evicted_slot(c->n_slots, 0);
+        for (int p = 0; p < c->n_parts; ++p) {
+            const int s = c->slot_of_part[p];
+            if (s < 0) continue;
+            if (want[p]) { next[p] = s; used[s] = 1; }
+            else evicted_slot[s] = 1;
+        }
+        std::vector<int> free_now, free_later;
+        for (int s = 0; s < c->n_slots; ++s) {
+            if (used[s]) continue;
+            (evicted_slot[s] ? free_later : free_now).push_back(s);
+        }
+        cudaEvent_t main_done = nullptr;
+        for (int p = 0; p < c->n_parts; ++p) {
+            if (!want[p] || next[p] >= 0) continue;
+            int s;
+            if (!free_now.empty()) { s = free_now.back(); free_now.pop_back(); }
+            else if (!free_later.empty()) {
+                s = free_later.back(); free_later.pop_back();
+                if (!main_done) {
+                    MG_CUDA(c, cudaEventCreateWithFlags(&main_done, cudaEventDisableTiming));
+                    MG_CUDA(c, cudaEventRecord(main_done, c->stream));
+                    MG_CUDA(c, cudaStreamWaitEvent(c->side, main_done, 0));
+                }
+            } else return mg_fail(c, MG_ERR_CAPACITY, "no free buffer slot");
+            next[p] = s;
+            const int64_t first = (int64_t)p * c->part_size;
+            const int64_t rows = std::min<int64_t>(c->part_size, c->n_nodes - first);
+            if (rows > 0)
+                MG_CUDA(c, cudaMemcpyAsync(c->slots + (size_t)s * c->slot_bytes, c->host_table + (size_t)first * c->row_bytes,
+                                           (size_t)rows * c->row_bytes, cudaMemcpyHostToDevice, c->side));
+        }
+        if (main_done) cudaEventDestroy(main_done);
+        cudaEvent_t done;
+        MG_CUDA(c, cudaEventCreateWithFlags(&done, cudaEventDisableTiming));
+        MG_CUDA(c, cudaEventRecord(done, c->side));
+        c->pending_events.push_back(done);
+    }
+    c->pending_slot = next;
+    c->has_pending = true;
+    if (!async) return mg_commit_resident(c, 600000);
+    return MG_OK;
+}
+
+extern "C" int mg_commit_resident(mg_ctx* c, int32_t timeout_ms) {
+    if (!c) return MG_ERR_ARG;
+    if (!c->has_pending) return mg_fail(c, MG_ERR_STATE, "no pending resident set");
+    MG_CUDA(c, cudaSetDevice(c->device));
+    const auto t0 = std::chrono::steady_clock::now();
+    for (auto ev : c->pending_events) {
+        for (;;) {
+            const cudaError_t q = cudaEventQuery(ev);
+            if (q == cudaSuccess) break;
+            if (q != cudaErrorNotReady) return mg_cuda_fail(c, q, "waiting for a partition copy");
+            const auto ms = std::chrono::duration_cast<std::chrono::milliseconds>(std::chrono::steady_clock::now() - t0).count();
+            if (ms > timeout_ms) return mg_fail(c, MG_ERR_TIMEOUT, "partition copies still running after %d ms", timeout_ms);
+            std::this_thread::sleep_for(std::chrono::microseconds(200));
+        }
+    }
+    for (auto ev : c->pending_events) cudaEventDestroy(ev);
+    c->pending_events.clear();
+    c->slot_of_part = c->pending_slot;
+    c->has_pending = false;
+    int rc = upload_slot_map(c);
+    if (rc) return rc;
+    return rebuild_view(c);
+}

@@ -1,0 +1,502 @@
+// GraphSage forward over DENSE (Section 4.2): per layer a segment-mean over the sampled
+// neighbours (Algorithm 3 with mean instead of sum) and the self / neighbour linear maps.
+//
+// Rows are kept in sampling order (targets first), so layer l's output rows of a batch are the
+// prefix [0, N_l) of its local rows and the "update" of Algorithm 2 is only a smaller row count.
+// All batches are packed: H^l holds rowbase[l][b] .. rowbase[l][b+1] for batch b.
+// Layer 1 reads base representations straight from the partition buffer (H^0 is never stored).
+
+#include <cuda_fp16.h>
+
+#include <algorithm>
+
+#include "mg_device.cuh"
+#include "mg_internal.cuh"
+
+int mg_gemm_tf32(mg_ctx* ctx, const float* x, const float* w_t, const float* bias, float* out, int64_t M, int N, int K,
+                 bool relu);  // mg_gemm_tcgen05.cu
+
+namespace {
+
+constexpr int kThreads = 256;
+
+struct AggArgs {
+    int32_t B, k, layer;     // layer l = 1..k
+    int32_t d_in;
+    int32_t row_lo, row_hi;  // packed output rows handled by this launch
+    const int32_t* rowbase_out;  // [B+1] of layer l
+    const int32_t* rowbase_in;   // [B+1] of layer l-1
+    const int32_t* cum;          // [B][k+2]
+    const int32_t* node_off;     // [k+1][B+1]
+    const int32_t* nodes;
+    const int32_t* ent_off;
+    const int32_t* ent_nbrs;
+    const int32_t* ent_repr;
+    const float* h_prev;         // layers >= 2
+    // layer 1: the partition buffer
+    const char* slots;
+    const int32_t* slot_of_part;
+    int64_t slot_bytes, row_bytes;
+    uint32_t part_size;
+    float* x;                    // [rows, 2 * d_in], row r of this launch at x + (r - row_lo) * 2 * d_in
+    int round_tf32;
+};
+
+__device__ __forceinline__ float to_tf32(float v) {
+    uint32_t u;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(v));
+    return __uint_as_float(u);
+}
+
+__device__ __forceinline__ const char* feature_row(const AggArgs& a, int32_t node) {
+    const uint32_t p = (uint32_t)node / a.part_size;
+    return a.slots + (int64_t)a.slot_of_part[p] * a.slot_bytes + (int64_t)((uint32_t)node - p * a.part_size) * a.row_bytes;
+}
+
+// one 16-byte chunk -> 4 (fp32) or 8 (fp16) floats
+template <bool HALF>
+struct Chunk {
+    static constexpr int kVals = HALF ? 8 : 4;
+    float v[kVals];
+    __device__ __forceinline__ void zero() {
+#pragma unroll
+        for (int i = 0; i < kVals; ++i) v[i] = 0.f;
+    }
+    __device__ __forceinline__ void load(const char* row, int chunk) {
+        const uint4 raw = __ldg(reinterpret_cast<const uint4*>(row) + chunk);
+        if (HALF) {
+            const __half2* h = reinterpret_cast<const __half2*>(&raw);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 f = __half22float2(h[i]);
+                v[2 * i] = f.x;
+                v[2 * i + 1] = f.y;
+            }
+        } else {
+            v[0] = __uint_as_float(raw.x); v[1] = __uint_as_float(raw.y);
+            v[2] = __uint_as_float(raw.z); v[3] = __uint_as_float(raw.w);
+        }
+    }
+    __device__ __forceinline__ void add(const Chunk& o) {
+#pragma unroll
+        for (int i = 0; i < kVals; ++i) v[i] += o.v[i];
+    }
+    __device__ __forceinline__ void store(float* dst, float scale, bool round) const {
+#pragma unroll
+        for (int i = 0; i < kVals; i += 4) {
+            float4 o = make_float4(v[i] * scale, v[i + 1] * scale, v[i + 2] * scale, v[i + 3] * scale);
+            if (round) { o.x = to_tf32(o.x); o.y = to_tf32(o.y); o.z = to_tf32(o.z); o.w = to_tf32(o.w); }
+            *reinterpret_cast<float4*>(dst + i) = o;
+        }
+    }
+};
+
+// G lanes per output row; each lane owns NCH 16-byte chunks of the row (chunk = gl + j * G).
+template <int G, int NCH, bool FIRST, bool HALF>
+__global__ void __launch_bounds__(kThreads) k_aggregate(AggArgs a) {
+    using C = Chunk<HALF>;
+    constexpr int kRowsPerBlock = kThreads / G;
+    const int gl = threadIdx.x % G;
+    const int n_chunks = a.d_in / C::kVals;
+    const int kk = a.k;
+    for (int32_t r = a.row_lo + blockIdx.x * kRowsPerBlock + threadIdx.x / G; r < a.row_hi; r += gridDim.x * kRowsPerBlock) {
+        const int b = upper_segment(a.rowbase_out, a.B + 1, r);
+        const int32_t l = r - a.rowbase_out[b];
+        const int32_t* cum = a.cum + b * (kk + 2);
+        int h = 0;
+        while (h < kk - a.layer && l >= cum[h + 1]) ++h;
+        const int32_t idx = a.node_off[h * (a.B + 1) + b] + (l - cum[h]);
+        const int32_t e0 = a.ent_off[idx], e1 = a.ent_off[idx + 1];
+        const int64_t in_base = FIRST ? 0 : (int64_t)a.rowbase_in[b];
+        float* xrow = a.x + (int64_t)(r - a.row_lo) * 2 * a.d_in;
+
+        // self row
+        const char* self_row = FIRST ? feature_row(a, a.nodes[idx])
+                                     : reinterpret_cast<const char*>(a.h_prev + (in_base + l) * a.d_in);
+        C acc[NCH];
+#pragma unroll
+        for (int j = 0; j < NCH; ++j) {
+            const int c = gl + j * G;
+            if (c < n_chunks) {
+                C s;
+                s.load(self_row, c);
+                s.store(xrow + c * C::kVals, 1.f, a.round_tf32);
+            }
+            acc[j].zero();
+        }
+        // neighbours, in entry order, two rows in flight
+        int32_t e = e0;
+        for (; e + 1 < e1; e += 2) {
+            const char* r0 = FIRST ? feature_row(a, a.ent_nbrs[e])
+                                   : reinterpret_cast<const char*>(a.h_prev + (in_base + a.ent_repr[e]) * a.d_in);
+            const char* r1 = FIRST ? feature_row(a, a.ent_nbrs[e + 1])
+                                   : reinterpret_cast<const char*>(a.h_prev + (in_base + a.ent_repr[e + 1]) * a.d_in);
+            C t0[NCH], t1[NCH];
+#pragma unroll
+            for (int j = 0; j < NCH; ++j) {
+                const int c = gl + j * G;
+                if (c < n_chunks) { t0[j].load(r0, c); t1[j].load(r1, c); }
+            }
+#pragma unroll
+            for (int j = 0; j < NCH; ++j) {
+                const int c = gl + j * G;
+                if (c < n_chunks) { acc[j].add(t0[j]); acc[j].add(t1[j]); }
+            }
+        }
+        if (e < e1) {
+            const char* r0 = FIRST ? feature_row(a, a.ent_nbrs[e])
+                                   : reinterpret_cast<const char*>(a.h_prev + (in_base + a.ent_repr[e]) * a.d_in);
+#pragma unroll
+            for (int j = 0; j < NCH; ++j) {
+                const int c = gl + j * G;
+                if (c < n_chunks) { C t; t.load(r0, c); acc[j].add(t); }
+            }
+        }
+        const float inv = e1 > e0 ? 1.f / (float)(e1 - e0) : 0.f;
+#pragma unroll
+        for (int j = 0; j < NCH; ++j) {
+            const int c = gl + j * G;
+            if (c < n_chunks) acc[j].store(xrow + a.d_in + c * C::kVals, inv, a.round_tf32);
+        }
+    }
+}
+
+// ---- CUDA-core fp32 GEMM with bias / ReLU epilogue (MG_GEMM_FP32) ---------------------------
+// out[M, N] = act(x[M, K] . w[K, N] + bias)
+template <bool RELU>
+__global__ void __launch_bounds__(256) k_gemm_fp32(const float* __restrict__ x, const float* __restrict__ w,
+                                                   const float* __restrict__ bias, float* __restrict__ out, int64_t M,
+                                                   int N, int K) {
+    constexpr int BM = 64, BN = 64, BK = 16;
+    __shared__ float As[BK][BM + 4];
+    __shared__ float Bs[BK][BN + 4];
+    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
+    const int64_t m0 = (int64_t)blockIdx.x * BM;
+    const int n0 = blockIdx.y * BN;
+    float acc[4][4] = {};
+    for (int k0 = 0; k0 < K; k0 += BK) {
+        for (int i = threadIdx.x; i < BM * BK; i += 256) {
+            const int mm = i / BK, kk = i % BK;
+            As[kk][mm] = (m0 + mm < M && k0 + kk < K) ? x[(m0 + mm) * K + k0 + kk] : 0.f;
+        }
+        for (int i = threadIdx.x; i < BK * BN; i += 256) {
+            const int kk = i / BN, nn = i % BN;
+            Bs[kk][nn] = (k0 + kk < K && n0 + nn < N) ? w[(int64_t)(k0 + kk) * N + n0 + nn] : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < BK; ++kk) {
+            float av[4], bv[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { av[i] = As[kk][ty * 4 + i]; bv[i] = Bs[kk][tx * 4 + i]; }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+    for (int i = 0; i < 4; ++i) {
+        const int64_t m = m0 + ty * 4 + i;
+        if (m >= M) continue;
+        for (int j = 0; j < 4; ++j) {
+            const int n = n0 + tx * 4 + j;
+            if (n >= N) continue;
+            float v = acc[i][j] + bias[n];
+            if (RELU) v = fmaxf(v, 0.f);
+            out[m * N + n] = v;
+        }
+    }
+}
+
+// ---- canonical-order exports ---------------------------------------------------------------
+struct RowExportArgs {
+    int32_t k, n_rows, first_delta;  // rows of Delta_{first_delta} .. Delta_k in the paper's order
+    int32_t nio[MG_MAX_HOPS + 2];    // canonical offsets of the deltas of this batch
+    int32_t cum[MG_MAX_HOPS + 2];
+    int32_t dim;
+};
+
+// out[c, :] = src[local(c), :] where c runs over the paper's row order
+__global__ void __launch_bounds__(kThreads) k_export_rows(RowExportArgs a, const float* __restrict__ src, float* __restrict__ out) {
+    const int vec = a.dim / 4;
+    const int64_t total = (int64_t)a.n_rows * vec;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int32_t c = (int32_t)(i / vec) + a.nio[a.first_delta];
+        const int q = (int)(i % vec);
+        int j = a.first_delta;
+        while (j < a.k && c >= a.nio[j + 1]) ++j;
+        const int32_t l = a.cum[a.k - j] + (c - a.nio[j]);
+        reinterpret_cast<float4*>(out)[i] = reinterpret_cast<const float4*>(src + (int64_t)l * a.dim)[q];
+    }
+}
+
+struct H0Args {
+    RowExportArgs r;
+    int32_t node_off[MG_MAX_HOPS + 1];
+    const int32_t* nodes;
+    const char* slots;
+    const int32_t* slot_of_part;
+    int64_t slot_bytes, row_bytes;
+    uint32_t part_size;
+};
+
+template <bool HALF>
+__global__ void __launch_bounds__(kThreads) k_gather_h0(H0Args a, float* __restrict__ out) {
+    using C = Chunk<HALF>;
+    const int n_chunks = a.r.dim / C::kVals;
+    const int64_t total = (int64_t)a.r.n_rows * n_chunks;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int32_t c = (int32_t)(i / n_chunks);
+        const int q = (int)(i % n_chunks);
+        int j = 0;
+        while (j < a.r.k && c >= a.r.nio[j + 1]) ++j;
+        const int h = a.r.k - j;
+        const int32_t node = a.nodes[a.node_off[h] + (c - a.r.nio[j])];
+        const uint32_t p = (uint32_t)node / a.part_size;
+        const char* row = a.slots + (int64_t)a.slot_of_part[p] * a.slot_bytes + (int64_t)((uint32_t)node - p * a.part_size) * a.row_bytes;
+        C v;
+        v.load(row, q);
+        v.store(out + (int64_t)c * a.r.dim + q * C::kVals, 1.f, false);
+    }
+}
+
+__global__ void k_transpose(const float* __restrict__ in, float* __restrict__ out, int rows, int cols, int round_tf32) {
+    const int64_t n = (int64_t)rows * cols;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const int r = (int)(i / cols), c = (int)(i % cols);
+        const float v = in[i];
+        out[(int64_t)c * rows + r] = round_tf32 ? to_tf32(v) : v;
+    }
+}
+
+template <bool FIRST, bool HALF>
+void launch_aggregate(const AggArgs& a, int grid, cudaStream_t st) {
+    const int vals = HALF ? 8 : 4;
+    const int n_chunks = a.d_in / vals;
+    int G = 4;
+    while (G < 32 && G < n_chunks) G <<= 1;
+    const int nch = (n_chunks + G - 1) / G;
+#define MG_AGG(GG, NN) k_aggregate<GG, NN, FIRST, HALF><<<grid, kThreads, 0, st>>>(a)
+    if (G == 4) MG_AGG(4, 1);
+    else if (G == 8) MG_AGG(8, 1);
+    else if (G == 16) MG_AGG(16, 1);
+    else if (nch == 1) MG_AGG(32, 1);
+    else if (nch == 2) MG_AGG(32, 2);
+    else if (nch == 3) MG_AGG(32, 3);
+    else if (nch == 4) MG_AGG(32, 4);
+    else if (nch <= 6) MG_AGG(32, 6);
+    else MG_AGG(32, 8);
+#undef MG_AGG
+}
+
+void fill_row_export(const mg_dense* d, int batch, int first_delta, int dim, RowExportArgs* r) {
+    const int k = d->k;
+    memset(r, 0, sizeof(*r));
+    r->k = k;
+    r->dim = dim;
+    r->first_delta = first_delta;
+    for (int h = 0; h <= k + 1; ++h) r->cum[h] = d->h_cum[(size_t)batch * (k + 2) + h];
+    r->nio[0] = 0;
+    for (int j = 0; j <= k; ++j) r->nio[j + 1] = r->nio[j] + (r->cum[k - j + 1] - r->cum[k - j]);
+    r->n_rows = r->nio[k + 1] - r->nio[first_delta];
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------
+extern "C" int mg_model_create(mg_ctx* ctx, int32_t k, const int32_t* dims, const float* const* w_self,
+                               const float* const* w_nbr, const float* const* bias, int gemm_precision, mg_model** out) {
+    if (!ctx) return MG_ERR_ARG;
+    if (!out || !dims || !w_self || !w_nbr || !bias) return mg_fail(ctx, MG_ERR_ARG, "null argument");
+    if (k <= 0 || k > MG_MAX_HOPS) return mg_fail(ctx, MG_ERR_ARG, "k must be in [1, %d]", MG_MAX_HOPS);
+    if (gemm_precision != MG_GEMM_TF32 && gemm_precision != MG_GEMM_FP32) return mg_fail(ctx, MG_ERR_ARG, "unknown gemm precision");
+    for (int l = 0; l <= k; ++l)
+        if (dims[l] <= 0 || dims[l] % 4 != 0 || dims[l] > 1024) return mg_fail(ctx, MG_ERR_ARG, "layer widths must be multiples of 4 in [4, 1024]");
+    for (int l = 0; l < k; ++l)
+        if (!w_self[l] || !w_nbr[l] || !bias[l]) return mg_fail(ctx, MG_ERR_ARG, "null weight pointer");
+    MG_CUDA(ctx, cudaSetDevice(ctx->device));
+    mg_model* m = new mg_model();
+    m->ctx = ctx;
+    m->k = k;
+    m->precision = gemm_precision;
+    for (int l = 0; l <= k; ++l) m->dims[l] = dims[l];
+    for (int l = 0; l < k; ++l) {
+        const size_t di = dims[l], dn = dims[l + 1];
+        if (cudaMalloc((void**)&m->w_cat[l], sizeof(float) * 2 * di * dn) != cudaSuccess ||
+            cudaMalloc((void**)&m->w_cat_t[l], sizeof(float) * 2 * di * dn) != cudaSuccess ||
+            cudaMalloc((void**)&m->bias[l], sizeof(float) * dn) != cudaSuccess) {
+            cudaGetLastError();
+            mg_model_free(m);
+            return mg_fail(ctx, MG_ERR_OOM, "weight allocation failed");
+        }
+        cudaMemcpyAsync(m->w_cat[l], w_self[l], sizeof(float) * di * dn, cudaMemcpyHostToDevice, ctx->stream);
+        cudaMemcpyAsync(m->w_cat[l] + di * dn, w_nbr[l], sizeof(float) * di * dn, cudaMemcpyHostToDevice, ctx->stream);
+        cudaMemcpyAsync(m->bias[l], bias[l], sizeof(float) * dn, cudaMemcpyHostToDevice, ctx->stream);
+        // K-major copy [d_out, 2 d_in], rounded to nearest TF32 once, for the tensor-core path
+        k_transpose<<<mg_grid(ctx, 2), kThreads, 0, ctx->stream>>>(m->w_cat[l], m->w_cat_t[l], (int)(2 * di), (int)dn,
+                                                                  gemm_precision == MG_GEMM_TF32);
+        ctx->launches++;
+    }
+    cudaError_t e = cudaStreamSynchronize(ctx->stream);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    if (e != cudaSuccess) { mg_model_free(m); return mg_cuda_fail(ctx, e, "weight upload"); }
+    *out = m;
+    return MG_OK;
+}
+
+extern "C" int mg_model_free(mg_model* m) {
+    if (!m) return MG_OK;
+    if (m->ctx) cudaSetDevice(m->ctx->device);
+    for (int l = 0; l < MG_MAX_HOPS; ++l) { cudaFree(m->w_cat[l]); cudaFree(m->w_cat_t[l]); cudaFree(m->bias[l]); }
+    delete m;
+    return MG_OK;
+}
+
+static int forward_checks(mg_ctx* ctx, const mg_model* m, const mg_dense* d) {
+    if (!m || !d) return mg_fail(ctx, MG_ERR_ARG, "null argument");
+    if (!d->valid) return mg_fail(ctx, MG_ERR_STATE, "mg_dense holds no completed sample");
+    if (d->ctx != ctx || m->ctx != ctx) return mg_fail(ctx, MG_ERR_ARG, "handle belongs to another context");
+    if (!ctx->slots || ctx->feat_dim <= 0) return mg_fail(ctx, MG_ERR_STATE, "no feature table loaded");
+    if (m->k != d->k) return mg_fail(ctx, MG_ERR_STATE, "model has %d layers, sample has %d hops", m->k, d->k);
+    if (m->dims[0] != ctx->feat_dim) return mg_fail(ctx, MG_ERR_STATE, "model input width %d != feature dim %d", m->dims[0], ctx->feat_dim);
+    return MG_OK;
+}
+
+// rows of a layer are processed in chunks small enough for the [self | mean] staging matrix to
+// stay in L2 between the aggregation kernel that writes it and the GEMM that reads it
+static int64_t chunk_rows_for(int d_in) {
+    const int64_t bytes_per_row = (int64_t)2 * d_in * 4;
+    int64_t rows = (48ll << 20) / bytes_per_row;
+    rows = std::max<int64_t>(rows / 128 * 128, 128);
+    return rows;
+}
+
+extern "C" int mg_forward(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out, int out_on_device) {
+    if (!ctx) return MG_ERR_ARG;
+    int rc = forward_checks(ctx, m, d);
+    if (rc) return rc;
+    if (!out) return mg_fail(ctx, MG_ERR_ARG, "null output");
+    MG_CUDA(ctx, cudaSetDevice(ctx->device));
+    const int k = d->k, B = d->n_batches;
+    cudaStream_t st = ctx->stream;
+
+    // per-layer outputs H^1..H^k live in one workspace (kept for mg_layer_output)
+    size_t total = 0;
+    size_t off[MG_MAX_HOPS + 1];
+    for (int l = 1; l <= k; ++l) {
+        off[l] = total;
+        total += (size_t)d->h_hdr.rows_total[l] * m->dims[l];
+    }
+    {
+        size_t have = ctx->ws_h_bytes[0] / sizeof(float);
+        if ((rc = mg_ensure(ctx, &ctx->ws_h[0], &have, total))) return rc;
+        ctx->ws_h_bytes[0] = have * sizeof(float);
+    }
+    int64_t max_x = 0;
+    for (int l = 1; l <= k; ++l) {
+        const int64_t rows = std::min<int64_t>(chunk_rows_for(m->dims[l - 1]), d->h_hdr.rows_total[l]);
+        max_x = std::max<int64_t>(max_x, rows * 2 * m->dims[l - 1]);
+    }
+    {
+        size_t have = ctx->ws_x_bytes / sizeof(float);
+        if ((rc = mg_ensure(ctx, &ctx->ws_x, &have, (size_t)max_x))) return rc;
+        ctx->ws_x_bytes = have * sizeof(float);
+    }
+
+    const bool half = ctx->feat_dtype == MG_DTYPE_F16;
+    for (int l = 1; l <= k; ++l) {
+        const int d_in = m->dims[l - 1], d_out = m->dims[l];
+        const int64_t M = d->h_hdr.rows_total[l];
+        float* h_out = ctx->ws_h[0] + off[l];
+        const float* h_prev = l > 1 ? ctx->ws_h[0] + off[l - 1] : nullptr;
+        const int64_t chunk = chunk_rows_for(d_in);
+        for (int64_t r0 = 0; r0 < M; r0 += chunk) {
+            const int64_t r1 = std::min(M, r0 + chunk);
+            AggArgs a;
+            a.B = B; a.k = k; a.layer = l; a.d_in = d_in;
+            a.row_lo = (int32_t)r0; a.row_hi = (int32_t)r1;
+            a.rowbase_out = d->rowbase + (size_t)l * (B + 1);
+            a.rowbase_in = d->rowbase + (size_t)(l - 1) * (B + 1);
+            a.cum = d->cum; a.node_off = d->node_off; a.nodes = d->nodes;
+            a.ent_off = d->ent_off; a.ent_nbrs = d->ent_nbrs; a.ent_repr = d->ent_repr;
+            a.h_prev = h_prev;
+            a.slots = ctx->slots; a.slot_of_part = ctx->d_slot_of_part;
+            a.slot_bytes = ctx->slot_bytes; a.row_bytes = ctx->row_bytes; a.part_size = (uint32_t)ctx->part_size;
+            a.x = ctx->ws_x;
+            a.round_tf32 = m->precision == MG_GEMM_TF32;
+            {
+                ProfScope ps(ctx, l == 1 ? PH_AGG_L1 : PH_AGG_REST, 1);
+                const int grid = mg_grid(ctx, 8);
+                if (l == 1) { if (half) launch_aggregate<true, true>(a, grid, st); else launch_aggregate<true, false>(a, grid, st); }
+                else launch_aggregate<false, false>(a, grid, st);
+                ctx->launches++;
+            }
+            {
+                ProfScope ps(ctx, PH_GEMM, 1);
+                const int64_t rows = r1 - r0;
+                const bool relu = l < k;
+                if (m->precision == MG_GEMM_FP32) {
+                    dim3 grid((unsigned)((rows + 63) / 64), (unsigned)((d_out + 63) / 64));
+                    if (relu) k_gemm_fp32<true><<<grid, 256, 0, st>>>(ctx->ws_x, m->w_cat[l - 1], m->bias[l - 1], h_out + r0 * d_out, rows, d_out, 2 * d_in);
+                    else k_gemm_fp32<false><<<grid, 256, 0, st>>>(ctx->ws_x, m->w_cat[l - 1], m->bias[l - 1], h_out + r0 * d_out, rows, d_out, 2 * d_in);
+                    ctx->launches++;
+                } else {
+                    rc = mg_gemm_tf32(ctx, ctx->ws_x, m->w_cat_t[l - 1], m->bias[l - 1], h_out + r0 * d_out, rows, d_out, 2 * d_in, relu);
+                    if (rc) return rc;
+                }
+            }
+        }
+    }
+    MG_CUDA(ctx, cudaGetLastError());
+    const size_t out_bytes = (size_t)d->h_hdr.rows_total[k] * m->dims[k] * sizeof(float);
+    MG_CUDA(ctx, cudaMemcpyAsync(out, ctx->ws_h[0] + off[k], out_bytes, out_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, st));
+    MG_CUDA(ctx, cudaStreamSynchronize(st));
+    return MG_OK;
+}
+
+extern "C" int mg_gather_h0(mg_ctx* ctx, mg_dense* d, int32_t batch, float* out_dev) {
+    if (!ctx) return MG_ERR_ARG;
+    if (!d || !out_dev) return mg_fail(ctx, MG_ERR_ARG, "null argument");
+    if (!d->valid) return mg_fail(ctx, MG_ERR_STATE, "mg_dense holds no completed sample");
+    if (!ctx->slots || ctx->feat_dim <= 0) return mg_fail(ctx, MG_ERR_STATE, "no feature table loaded");
+    if (batch < 0 || batch >= d->n_batches) return mg_fail(ctx, MG_ERR_ARG, "batch out of range");
+    MG_CUDA(ctx, cudaSetDevice(ctx->device));
+    H0Args a;
+    fill_row_export(d, batch, 0, ctx->feat_dim, &a.r);
+    for (int h = 0; h <= d->k; ++h) a.node_off[h] = d->h_node_off[(size_t)h * (d->n_batches + 1) + batch];
+    a.nodes = d->nodes; a.slots = ctx->slots; a.slot_of_part = ctx->d_slot_of_part;
+    a.slot_bytes = ctx->slot_bytes; a.row_bytes = ctx->row_bytes; a.part_size = (uint32_t)ctx->part_size;
+    if (a.r.n_rows > 0) {
+        if (ctx->feat_dtype == MG_DTYPE_F16) k_gather_h0<true><<<mg_grid(ctx, 4), kThreads, 0, ctx->stream>>>(a, out_dev);
+        else k_gather_h0<false><<<mg_grid(ctx, 4), kThreads, 0, ctx->stream>>>(a, out_dev);
+        ctx->launches++;
+    }
+    MG_CUDA(ctx, cudaGetLastError());
+    MG_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return MG_OK;
+}
+
+extern "C" int mg_layer_output(mg_ctx* ctx, const mg_model* m, mg_dense* d, int32_t layer, int32_t batch, float* out_dev) {
+    if (!ctx) return MG_ERR_ARG;
+    int rc = forward_checks(ctx, m, d);
+    if (rc) return rc;
+    if (!out_dev) return mg_fail(ctx, MG_ERR_ARG, "null output");
+    if (layer < 1 || layer > d->k) return mg_fail(ctx, MG_ERR_ARG, "layer must be in [1, k]");
+    if (batch < 0 || batch >= d->n_batches) return mg_fail(ctx, MG_ERR_ARG, "batch out of range");
+    if (!ctx->ws_h[0]) return mg_fail(ctx, MG_ERR_STATE, "mg_forward has not run");
+    MG_CUDA(ctx, cudaSetDevice(ctx->device));
+    size_t off = 0;
+    for (int l = 1; l < layer; ++l) off += (size_t)d->h_hdr.rows_total[l] * m->dims[l];
+    const int B = d->n_batches;
+    const float* src = ctx->ws_h[0] + off + (size_t)d->h_rowbase[(size_t)layer * (B + 1) + batch] * m->dims[layer];
+    RowExportArgs r;
+    fill_row_export(d, batch, layer, m->dims[layer], &r);
+    if (r.n_rows > 0) {
+        k_export_rows<<<mg_grid(ctx, 4), kThreads, 0, ctx->stream>>>(r, src, out_dev);
+        ctx->launches++;
+    }
+    MG_CUDA(ctx, cudaGetLastError());
+    MG_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return MG_OK;
+}

@@ -1,0 +1,226 @@
+// Internal declarations shared by the translation units of libmgdense.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <string>
+#include <vector>
+
+#include "mgdense.h"
+
+// ---------------------------------------------------------------------------------------
+// status word written by kernels (never a trap): bit flags, read by the host after a call
+// ---------------------------------------------------------------------------------------
+enum : uint32_t {
+    ST_RANGE = 1u,         // target id outside [0, n_nodes)
+    ST_NONRESIDENT = 2u,   // target in a non-resident partition
+    ST_DUPLICATE = 4u,     // same target twice in a batch
+    ST_CAP_ENTRIES = 8u,   // neighbour arena too small
+    ST_CAP_NODES = 16u,    // node arena too small
+    ST_CAP_TABLE = 32u,    // per-batch id table full (max_nodes_per_batch too small)
+    ST_INTERNAL = 64u,     // an invariant did not hold (bug guard; access skipped)
+};
+
+// Device-side header of a sample: counters every kernel sizes itself from.
+struct DenseHeader {
+    uint32_t status;
+    uint32_t n_new;                       // length of the new-node list of the current hop
+    int32_t hop_base[MG_MAX_HOPS + 2];    // node arena: hop h occupies [hop_base[h], hop_base[h+1])
+    int32_t ent_base[MG_MAX_HOPS + 1];    // entry arena: hop h occupies [ent_base[h], ent_base[h+1])
+    int32_t rows_total[MG_MAX_HOPS + 1];  // rows of H^l summed over batches, l = 0..k
+};
+
+struct ProfPhase {
+    const char* name;
+    double ms;
+    int64_t launches;
+};
+
+enum {
+    PH_SAMPLE_INIT = 0,
+    PH_SAMPLE_COUNT,
+    PH_SAMPLE_SCAN,
+    PH_SAMPLE_PICK,
+    PH_SAMPLE_SORT,
+    PH_SAMPLE_PLACE,
+    PH_SAMPLE_RELABEL,
+    PH_SAMPLE_FINAL,
+    PH_AGG_L1,
+    PH_AGG_REST,
+    PH_GEMM,
+    PH_DISTMULT,
+    PH_OTHER,
+    PH_COUNT
+};
+
+struct mg_ctx {
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    cudaStream_t side = nullptr;  // partition swaps
+    std::string err;
+    int64_t launches = 0;
+    int n_sms = 148;
+
+    // graph store (device)
+    int64_t n_nodes = 0, n_edges = 0;
+    int64_t* row_off = nullptr;  // [n_nodes + 1]
+    int32_t* nbrs = nullptr;     // [n_edges]
+    // in-buffer view (device); equal to the store when everything is resident
+    int64_t* view_off = nullptr;
+    int32_t* view_nbrs = nullptr;
+    int64_t view_edges = 0;
+    bool view_owned = false;
+
+    // partitioning and buffer
+    int32_t n_parts = 1;
+    int64_t part_size = 0;
+    int32_t capacity = 1;
+    std::vector<int32_t> slot_of_part;  // committed; -1 = not resident
+    std::vector<int32_t> pending_slot;  // after set_resident, before commit
+    bool has_pending = false;
+    std::vector<cudaEvent_t> pending_events;
+    int32_t* d_slot_of_part = nullptr;   // [MG_MAX_PARTS]
+    int64_t* d_res_prefix = nullptr;     // [MG_MAX_PARTS + 1] resident-node prefix counts
+    int64_t n_resident_nodes = 0;
+
+    // features
+    int feat_dtype = MG_DTYPE_F32;
+    int32_t feat_dim = 0;
+    int backing = MG_BACKING_HBM;
+    const char* host_table = nullptr;  // MG_BACKING_HOST
+    char* slots = nullptr;             // device: slot s at slots + s * slot_bytes
+    bool slots_owned = false;
+    int32_t n_slots = 0;
+    int64_t slot_bytes = 0;
+    int64_t row_bytes = 0;
+
+    // forward workspaces (grown on demand)
+    float* ws_x = nullptr; size_t ws_x_bytes = 0;
+    float* ws_h[2] = {nullptr, nullptr}; size_t ws_h_bytes[2] = {0, 0};
+    float** ws_layer = nullptr;
+
+    // profiling
+    bool prof_on = false;
+    ProfPhase prof[PH_COUNT];
+    std::vector<std::pair<int, std::pair<cudaEvent_t, cudaEvent_t>>> prof_pending;
+};
+
+struct mg_dense {
+    mg_ctx* ctx = nullptr;
+    int32_t k = 0, n_batches = 0;
+    int32_t fanouts[MG_MAX_HOPS] = {0};
+    int64_t cap_nodes = 0, cap_entries = 0;
+    int32_t table_size = 0;  // slots per batch, power of two
+    int32_t table_shift = 0; // 32 - log2(table_size)
+    int64_t n_targets_total = 0;
+
+    // device arrays
+    DenseHeader* hdr = nullptr;
+    int32_t* nodes = nullptr;       // [cap_nodes] hop-major, batch-major inside a hop
+    int32_t* node_batch = nullptr;  // [cap_nodes]
+    int32_t* ent_off = nullptr;     // [cap_nodes + 1] start of each sampled node's entries
+    int32_t* ent_nbrs = nullptr;    // [cap_entries] neighbour ids
+    int32_t* ent_repr = nullptr;    // [cap_entries] neighbour's local row in its batch
+    int32_t* node_off = nullptr;    // [(k+1) * (B+1)] arena index where batch b's hop-h nodes start
+    int32_t* cum = nullptr;         // [B * (k+2)] local row of the first node of hop h; [k+1] = V
+    int32_t* rowbase = nullptr;     // [(k+1) * (B+1)] first packed row of batch b in H^l
+    int32_t* hkeys = nullptr;       // [B * table_size]
+    int32_t* hvals = nullptr;       // [B * table_size]
+    uint64_t* newlist[2] = {nullptr, nullptr};  // [cap_nodes] composite keys
+    uint64_t* d_seeds = nullptr;    // [B]
+    int32_t* scan_tmp = nullptr;    // block sums
+    uint32_t* sort_hist = nullptr;  // radix histograms
+    size_t scan_tmp_elems = 0, sort_hist_elems = 0;
+    int64_t alloc_batches = 0, alloc_table = 0;
+
+    // export buffer for mg_dense_view
+    int32_t* exp_buf = nullptr; size_t exp_elems = 0;
+
+    // host mirror
+    DenseHeader h_hdr;
+    std::vector<int32_t> h_cum;      // [B * (k+2)]
+    std::vector<int32_t> h_node_off; // [(k+1) * (B+1)]
+    std::vector<int32_t> h_rowbase;  // [(k+1) * (B+1)]
+    std::vector<int32_t> h_ent_hop;  // [k * (B+1)] arena entry index where batch b's hop-h entries start
+    int32_t* d_ent_hop = nullptr;    // device copy of the same
+    bool valid = false;
+};
+
+struct mg_model {
+    mg_ctx* ctx = nullptr;
+    int32_t k = 0;
+    int32_t dims[MG_MAX_HOPS + 1] = {0};
+    int precision = MG_GEMM_TF32;
+    float* w_cat[MG_MAX_HOPS] = {nullptr};  // device [2*d_in, d_out]: rows 0..d_in-1 self, then neighbour
+    float* w_cat_t[MG_MAX_HOPS] = {nullptr}; // device [d_out, 2*d_in] (K-major copy for the tensor-core path)
+    float* bias[MG_MAX_HOPS] = {nullptr};
+};
+
+struct mg_lp_batch {
+    mg_ctx* ctx = nullptr;
+    int64_t n_edges = 0;
+    int32_t n_chunks = 0, negs = 0, n_targets = 0;
+    int32_t* targets = nullptr;  // device
+    int32_t* src_idx = nullptr;
+    int32_t* dst_idx = nullptr;
+    int32_t* rel = nullptr;
+    int32_t* neg_ids = nullptr;
+    int32_t* neg_idx = nullptr;
+};
+
+// ---------------------------------------------------------------------------------------
+// host helpers
+// ---------------------------------------------------------------------------------------
+int mg_fail(mg_ctx* ctx, int code, const char* fmt, ...);
+int mg_cuda_fail(mg_ctx* ctx, cudaError_t e, const char* what);
+
+#define MG_CUDA(ctx, call)                                      \
+    do {                                                        \
+        cudaError_t e__ = (call);                               \
+        if (e__ != cudaSuccess) return mg_cuda_fail(ctx, e__, #call); \
+    } while (0)
+
+// grow-only device buffer
+template <typename T>
+static inline int mg_ensure(mg_ctx* ctx, T** ptr, size_t* have_elems, size_t need_elems) {
+    if (*ptr && *have_elems >= need_elems) return MG_OK;
+    if (*ptr) cudaFree(*ptr);
+    *ptr = nullptr;
+    *have_elems = 0;
+    if (need_elems == 0) need_elems = 1;
+    cudaError_t e = cudaMalloc((void**)ptr, need_elems * sizeof(T));
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return mg_fail(ctx, MG_ERR_OOM, "device allocation of %zu bytes failed", need_elems * sizeof(T));
+    }
+    *have_elems = need_elems;
+    return MG_OK;
+}
+
+void mg_prof_begin(mg_ctx* ctx, int phase);
+void mg_prof_end(mg_ctx* ctx, int phase, int n_launches);
+
+struct ProfScope {
+    mg_ctx* c; int ph; int n;
+    ProfScope(mg_ctx* ctx, int phase, int launches) : c(ctx), ph(phase), n(launches) { mg_prof_begin(c, ph); }
+    ~ProfScope() { mg_prof_end(c, ph, n); }
+};
+
+static inline int mg_grid(const mg_ctx* ctx, int ctas_per_sm) { return ctx->n_sms * ctas_per_sm; }
+
+// ---- generic device-sized scan and sort (mg_sample.cu) -------------------------------------
+struct SortParams {   // device-resident
+    int32_t zero;
+    int32_t n;        // keys
+    int32_t ntiles;   // ceil(n / 4096)
+    int32_t hist_len; // 256 * ntiles
+};
+size_t mg_sort_hist_elems(int64_t max_keys);
+size_t mg_scan_tmp_elems(int64_t max_elems);
+void mg_sort_u64(mg_ctx* ctx, uint64_t* const buf[2], const SortParams* sp, int lo_bit, int bits, uint32_t* hist,
+                 uint32_t* scan_tmp, int* res_buf);
+void mg_scan_u32(mg_ctx* ctx, uint32_t* data, const int32_t* lo, const int32_t* hi, const int32_t* base,
+                 uint32_t* scan_tmp, uint32_t* total_out);

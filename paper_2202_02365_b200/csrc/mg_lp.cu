@@ -1,0 +1,279 @@
+// Link prediction: shared uniform negatives per chunk, the batch's target union, and DistMult
+// scoring (the decoder of the paper's link-prediction configuration, Section 7.1).
+
+#include <algorithm>
+
+#include "mg_device.cuh"
+#include "mg_internal.cuh"
+
+namespace {
+
+constexpr int kThreads = 256;
+
+// Builds the sort keys (id << 32 | origin) for sources, destinations and negatives.
+// origin: [0, E) sources, [E, 2E) destinations, [2E, 2E + C * negs) negatives.
+__global__ void __launch_bounds__(kThreads)
+k_lp_keys(const int32_t* __restrict__ src, const int32_t* __restrict__ dst, int64_t E, int32_t n_chunks, int32_t negs,
+          uint64_t seed, const int64_t* __restrict__ res_prefix, int32_t n_parts, int64_t part_size, int64_t n_resident,
+          int64_t n_nodes, const int32_t* __restrict__ slot_of_part, int32_t* neg_ids, uint64_t* keys, uint32_t* status) {
+    const int64_t total = 2 * E + (int64_t)n_chunks * negs;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        int32_t id;
+        if (i < 2 * E) {
+            id = i < E ? src[i] : dst[i - E];
+            if (id < 0 || (int64_t)id >= n_nodes) { atomicOr(status, ST_RANGE); id = 0; }
+            else if (slot_of_part[(int64_t)id / part_size] < 0) atomicOr(status, ST_NONRESIDENT);
+        } else {
+            const int64_t j = i - 2 * E;
+            const uint32_t c = (uint32_t)(j / negs), t = (uint32_t)(j % negs);
+            uint32_t o[4];
+            philox4x32_10(c, t, 0xFFFFFFFFu, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), o);
+            // index among the resident nodes, counted in ascending partition order
+            const int64_t r = (int64_t)(((unsigned __int128)o[0] * (unsigned __int128)(uint64_t)n_resident) >> 32);
+            int p = 0;
+            while (p + 1 < n_parts && res_prefix[p + 1] <= r) ++p;
+            id = (int32_t)((int64_t)p * part_size + (r - res_prefix[p]));
+            neg_ids[j] = id;
+        }
+        keys[i] = ((uint64_t)(uint32_t)id << 32) | (uint64_t)(uint32_t)i;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads) k_lp_heads(const uint64_t* __restrict__ sorted, int32_t n, uint32_t* heads) {
+    for (int32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
+        heads[i] = (i > 0 && (sorted[i] >> 32) != (sorted[i - 1] >> 32)) ? 1u : 0u;
+}
+
+// after an exclusive scan of heads: rank[i] = scanned[i] + heads[i] is the target row of key i.
+// An exclusive scan of h gives rank[i] - h[i]; recompute h from the keys.
+__global__ void __launch_bounds__(kThreads)
+k_lp_scatter(const uint64_t* __restrict__ sorted, const uint32_t* __restrict__ scanned, int32_t n, int64_t E,
+             int32_t* targets, int32_t* src_idx, int32_t* dst_idx, int32_t* neg_idx, int32_t* n_targets) {
+    for (int32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        const uint64_t key = sorted[i];
+        const bool head = i > 0 && (key >> 32) != (sorted[i - 1] >> 32);
+        const int32_t rank = (int32_t)scanned[i] + (head ? 1 : 0);
+        const uint32_t origin = (uint32_t)key;
+        if (i == 0 || head) targets[rank] = (int32_t)(key >> 32);
+        if ((int64_t)origin < E) src_idx[origin] = rank;
+        else if ((int64_t)origin < 2 * E) dst_idx[origin - E] = rank;
+        else neg_idx[origin - 2 * E] = rank;
+        if (i == n - 1) *n_targets = rank + 1;
+    }
+}
+
+// pos[i] = sum_d h[s_i, d] * rel[r_i, d] * h[o_i, d]; one warp per edge, fixed summation order
+__global__ void __launch_bounds__(kThreads)
+k_distmult_pos(const float* __restrict__ h, const float* __restrict__ rel_emb, const int32_t* __restrict__ src_idx,
+               const int32_t* __restrict__ dst_idx, const int32_t* __restrict__ rel, int64_t E, int dim, float* pos) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warps = (int64_t)gridDim.x * (kThreads / 32);
+    for (int64_t i = blockIdx.x * (int64_t)(kThreads / 32) + (threadIdx.x >> 5); i < E; i += warps) {
+        const float* hs = h + (int64_t)src_idx[i] * dim;
+        const float* ho = h + (int64_t)dst_idx[i] * dim;
+        const float* r = rel_emb + (int64_t)rel[i] * dim;
+        float s = 0.f;
+        for (int d = lane; d < dim; d += 32) s = fmaf(hs[d] * r[d], ho[d], s);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+        if (lane == 0) pos[i] = s;
+    }
+}
+
+// neg[i, t] = sum_d (h[a_i, d] * rel[r_i, d]) * h[neg_{c(i), t}, d], a = source (destination side
+// corrupted) or destination (source side corrupted).  Tiles of 64 edges x 64 negatives inside one
+// chunk; both operands are gathered into shared memory.
+struct NegArgs {
+    const float* h;
+    const float* rel_emb;
+    const int32_t* keep_idx;  // src_idx when the destination is corrupted, dst_idx otherwise
+    const int32_t* rel;
+    const int32_t* neg_idx;   // [n_chunks, negs]
+    int64_t E;
+    int32_t n_chunks, negs, dim, tiles_per_chunk;
+    float* out;               // [E, negs]
+};
+
+__global__ void __launch_bounds__(256) k_distmult_neg(NegArgs a) {
+    constexpr int BM = 64, BN = 64, BK = 16;
+    __shared__ float As[BK][BM + 4];
+    __shared__ float Bs[BK][BN + 4];
+    __shared__ int32_t a_row[BM], a_rel[BM], b_row[BN];
+    const int c = blockIdx.x / a.tiles_per_chunk;
+    const int tile = blockIdx.x % a.tiles_per_chunk;
+    // chunk c holds the edges i with floor(i * n_chunks / E) == c
+    const int64_t lo = ((int64_t)c * a.E + a.n_chunks - 1) / a.n_chunks;
+    const int64_t hi = ((int64_t)(c + 1) * a.E + a.n_chunks - 1) / a.n_chunks;
+    const int64_t m0 = lo + (int64_t)tile * BM;
+    if (m0 >= hi) return;
+    const int n0 = blockIdx.y * BN;
+    if (threadIdx.x < BM) {
+        const int64_t i = m0 + threadIdx.x;
+        a_row[threadIdx.x] = i < hi ? a.keep_idx[i] : -1;
+        a_rel[threadIdx.x] = i < hi ? a.rel[i] : 0;
+    } else if (threadIdx.x < BM + BN) {
+        const int t = n0 + (threadIdx.x - BM);
+        b_row[threadIdx.x - BM] = t < a.negs ? a.neg_idx[(int64_t)c * a.negs + t] : -1;
+    }
+    __syncthreads();
+    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
+    float acc[4][4] = {};
+    for (int k0 = 0; k0 < a.dim; k0 += BK) {
+        for (int i = threadIdx.x; i < BM * BK; i += 256) {
+            const int mm = i / BK, kk = i % BK;
+            float v = 0.f;
+            if (a_row[mm] >= 0 && k0 + kk < a.dim)
+                v = a.h[(int64_t)a_row[mm] * a.dim + k0 + kk] * a.rel_emb[(int64_t)a_rel[mm] * a.dim + k0 + kk];
+            As[kk][mm] = v;
+        }
+        for (int i = threadIdx.x; i < BN * BK; i += 256) {
+            const int nn = i / BK, kk = i % BK;
+            Bs[kk][nn] = (b_row[nn] >= 0 && k0 + kk < a.dim) ? a.h[(int64_t)b_row[nn] * a.dim + k0 + kk] : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < BK; ++kk) {
+            float av[4], bv[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { av[i] = As[kk][ty * 4 + i]; bv[i] = Bs[kk][tx * 4 + i]; }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+    for (int i = 0; i < 4; ++i) {
+        const int64_t m = m0 + ty * 4 + i;
+        if (m >= hi) continue;
+        for (int j = 0; j < 4; ++j) {
+            const int n = n0 + tx * 4 + j;
+            if (n < a.negs) a.out[m * a.negs + n] = acc[i][j];
+        }
+    }
+}
+
+}  // namespace
+
+extern "C" int mg_lp_free(mg_lp_batch* lp) {
+    if (!lp) return MG_OK;
+    if (lp->ctx) cudaSetDevice(lp->ctx->device);
+    cudaFree(lp->targets); cudaFree(lp->src_idx); cudaFree(lp->dst_idx); cudaFree(lp->rel);
+    cudaFree(lp->neg_ids); cudaFree(lp->neg_idx);
+    delete lp;
+    return MG_OK;
+}
+
+extern "C" int mg_lp_prepare(mg_ctx* ctx, const int32_t* src, const int32_t* rel, const int32_t* dst, int64_t n_edges,
+                             int32_t n_chunks, int32_t negs, uint64_t seed, mg_lp_batch** out) {
+    if (!ctx) return MG_ERR_ARG;
+    if (!out || !src || !rel || !dst) return mg_fail(ctx, MG_ERR_ARG, "null argument");
+    if (n_edges <= 0 || n_chunks <= 0 || negs < 0 || n_chunks > n_edges) return mg_fail(ctx, MG_ERR_ARG, "need n_edges >= n_chunks >= 1 and negs >= 0");
+    if (!ctx->row_off) return mg_fail(ctx, MG_ERR_STATE, "no graph loaded");
+    if (ctx->n_resident_nodes <= 0) return mg_fail(ctx, MG_ERR_STATE, "no resident partition");
+    const int64_t total = 2 * n_edges + (int64_t)n_chunks * negs;
+    if (total >= (1ll << 31)) return mg_fail(ctx, MG_ERR_ARG, "batch too large");
+    MG_CUDA(ctx, cudaSetDevice(ctx->device));
+    cudaStream_t st = ctx->stream;
+    mg_lp_batch* lp = new mg_lp_batch();
+    lp->ctx = ctx; lp->n_edges = n_edges; lp->n_chunks = n_chunks; lp->negs = negs;
+
+    int32_t *d_src = nullptr, *d_dst = nullptr, *d_nt = nullptr;
+    uint64_t* keys[2] = {nullptr, nullptr};
+    uint32_t *heads = nullptr, *hist = nullptr, *scan_tmp = nullptr, *d_status = nullptr;
+    SortParams* sp = nullptr;
+    const size_t n_neg = (size_t)std::max<int64_t>((int64_t)n_chunks * negs, 1);
+    auto cleanup = [&]() {
+        cudaFree(d_src); cudaFree(d_dst); cudaFree(d_nt); cudaFree(keys[0]); cudaFree(keys[1]);
+        cudaFree(heads); cudaFree(hist); cudaFree(scan_tmp); cudaFree(d_status); cudaFree(sp);
+    };
+    const size_t hist_elems = mg_sort_hist_elems(total);
+    const size_t scan_elems = std::max(mg_scan_tmp_elems(total), mg_scan_tmp_elems((int64_t)hist_elems));
+    bool ok = cudaMalloc((void**)&d_src, 4 * n_edges) == cudaSuccess && cudaMalloc((void**)&d_dst, 4 * n_edges) == cudaSuccess &&
+              cudaMalloc((void**)&d_nt, 4) == cudaSuccess && cudaMalloc((void**)&keys[0], 8 * total) == cudaSuccess &&
+              cudaMalloc((void**)&keys[1], 8 * total) == cudaSuccess && cudaMalloc((void**)&heads, 4 * total) == cudaSuccess &&
+              cudaMalloc((void**)&hist, 4 * hist_elems) == cudaSuccess && cudaMalloc((void**)&scan_tmp, 4 * scan_elems) == cudaSuccess &&
+              cudaMalloc((void**)&d_status, 4) == cudaSuccess && cudaMalloc((void**)&sp, sizeof(SortParams)) == cudaSuccess &&
+              cudaMalloc((void**)&lp->targets, 4 * total) == cudaSuccess && cudaMalloc((void**)&lp->src_idx, 4 * n_edges) == cudaSuccess &&
+              cudaMalloc((void**)&lp->dst_idx, 4 * n_edges) == cudaSuccess && cudaMalloc((void**)&lp->rel, 4 * n_edges) == cudaSuccess &&
+              cudaMalloc((void**)&lp->neg_ids, 4 * n_neg) == cudaSuccess && cudaMalloc((void**)&lp->neg_idx, 4 * n_neg) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); cleanup(); mg_lp_free(lp); return mg_fail(ctx, MG_ERR_OOM, "allocation of the link-prediction batch failed"); }
+
+    SortParams h_sp;
+    h_sp.zero = 0; h_sp.n = (int32_t)total; h_sp.ntiles = (int32_t)((total + 4095) / 4096); h_sp.hist_len = 256 * h_sp.ntiles;
+    cudaMemcpyAsync(sp, &h_sp, sizeof(h_sp), cudaMemcpyHostToDevice, st);
+    cudaMemcpyAsync(d_src, src, 4 * n_edges, cudaMemcpyHostToDevice, st);
+    cudaMemcpyAsync(d_dst, dst, 4 * n_edges, cudaMemcpyHostToDevice, st);
+    cudaMemcpyAsync(lp->rel, rel, 4 * n_edges, cudaMemcpyHostToDevice, st);
+    cudaMemsetAsync(d_status, 0, 4, st);
+    const int grid = mg_grid(ctx, 4);
+    k_lp_keys<<<grid, kThreads, 0, st>>>(d_src, d_dst, n_edges, n_chunks, negs, seed, ctx->d_res_prefix, ctx->n_parts,
+                                         ctx->part_size, ctx->n_resident_nodes, ctx->n_nodes, ctx->d_slot_of_part,
+                                         lp->neg_ids, keys[0], d_status);
+    int id_bits = 1;
+    while ((1ll << id_bits) < ctx->n_nodes) ++id_bits;
+    int res = 0;
+    mg_sort_u64(ctx, keys, sp, 32, id_bits, hist, scan_tmp, &res);
+    k_lp_heads<<<grid, kThreads, 0, st>>>(keys[res], (int32_t)total, heads);
+    mg_scan_u32(ctx, heads, &sp->zero, &sp->n, nullptr, scan_tmp, nullptr);
+    k_lp_scatter<<<grid, kThreads, 0, st>>>(keys[res], heads, (int32_t)total, n_edges, lp->targets, lp->src_idx, lp->dst_idx,
+                                            lp->neg_idx, d_nt);
+    ctx->launches += 3;
+    uint32_t h_status = 0;
+    cudaMemcpyAsync(&h_status, d_status, 4, cudaMemcpyDeviceToHost, st);
+    cudaMemcpyAsync(&lp->n_targets, d_nt, 4, cudaMemcpyDeviceToHost, st);
+    cudaError_t e = cudaStreamSynchronize(st);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    cleanup();
+    if (e != cudaSuccess) { mg_lp_free(lp); return mg_cuda_fail(ctx, e, "mg_lp_prepare"); }
+    if (h_status & ST_RANGE) { mg_lp_free(lp); return mg_fail(ctx, MG_ERR_ARG, "an edge endpoint is outside [0, n_nodes)"); }
+    if (h_status & ST_NONRESIDENT) { mg_lp_free(lp); return mg_fail(ctx, MG_ERR_NONRESIDENT, "an edge endpoint lies in a partition that is not resident"); }
+    *out = lp;
+    return MG_OK;
+}
+
+extern "C" int mg_lp_view(const mg_lp_batch* lp, int32_t* n_targets, const int32_t** targets, const int32_t** src_idx,
+                          const int32_t** dst_idx, const int32_t** neg_ids, const int32_t** neg_idx) {
+    if (!lp) return MG_ERR_ARG;
+    if (n_targets) *n_targets = lp->n_targets;
+    if (targets) *targets = lp->targets;
+    if (src_idx) *src_idx = lp->src_idx;
+    if (dst_idx) *dst_idx = lp->dst_idx;
+    if (neg_ids) *neg_ids = lp->neg_ids;
+    if (neg_idx) *neg_idx = lp->neg_idx;
+    return MG_OK;
+}
+
+extern "C" int mg_distmult_score(mg_ctx* ctx, const mg_lp_batch* lp, const float* h_dev, int32_t dim, const float* rel_emb_dev,
+                                 int32_t n_relations, int corrupt, float* pos_out, float* neg_dst_out, float* neg_src_out) {
+    if (!ctx) return MG_ERR_ARG;
+    if (!lp || !h_dev || !rel_emb_dev || !pos_out) return mg_fail(ctx, MG_ERR_ARG, "null argument");
+    if (dim <= 0 || n_relations <= 0) return mg_fail(ctx, MG_ERR_ARG, "dim and n_relations must be positive");
+    if ((corrupt & MG_CORRUPT_DST) && lp->negs > 0 && !neg_dst_out) return mg_fail(ctx, MG_ERR_ARG, "null neg_dst_out");
+    if ((corrupt & MG_CORRUPT_SRC) && lp->negs > 0 && !neg_src_out) return mg_fail(ctx, MG_ERR_ARG, "null neg_src_out");
+    MG_CUDA(ctx, cudaSetDevice(ctx->device));
+    cudaStream_t st = ctx->stream;
+    ProfScope ps(ctx, PH_DISTMULT, 3);
+    k_distmult_pos<<<mg_grid(ctx, 8), kThreads, 0, st>>>(h_dev, rel_emb_dev, lp->src_idx, lp->dst_idx, lp->rel, lp->n_edges, dim, pos_out);
+    ctx->launches++;
+    if (lp->negs > 0) {
+        const int64_t max_chunk = (lp->n_edges + lp->n_chunks - 1) / lp->n_chunks;
+        NegArgs a;
+        a.h = h_dev; a.rel_emb = rel_emb_dev; a.rel = lp->rel; a.neg_idx = lp->neg_idx; a.E = lp->n_edges;
+        a.n_chunks = lp->n_chunks; a.negs = lp->negs; a.dim = dim;
+        a.tiles_per_chunk = (int32_t)((max_chunk + 63) / 64);
+        dim3 grid((unsigned)(a.tiles_per_chunk * lp->n_chunks), (unsigned)((lp->negs + 63) / 64));
+        if (corrupt & MG_CORRUPT_DST) {
+            a.keep_idx = lp->src_idx; a.out = neg_dst_out;
+            k_distmult_neg<<<grid, 256, 0, st>>>(a);
+            ctx->launches++;
+        }
+        if (corrupt & MG_CORRUPT_SRC) {
+            a.keep_idx = lp->dst_idx; a.out = neg_src_out;
+            k_distmult_neg<<<grid, 256, 0, st>>>(a);
+            ctx->launches++;
+        }
+    }
+    MG_CUDA(ctx, cudaGetLastError());
+    return MG_OK;
+}

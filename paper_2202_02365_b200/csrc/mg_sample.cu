@@ -1,0 +1,964 @@
+// DENSE multi-hop sampling (Algorithm 1) for many independent mini-batches per pass.
+//
+// Layout kept on the device (hop-major, sampling order):
+//   nodes[]     hop 0 = the targets of all batches, hop h+1 = the deltas found from hop h,
+//               inside a hop batch after batch, inside a batch ascending id (targets: caller order)
+//   ent_off[]   for each sampled node its first entry in ent_nbrs / ent_repr (same order as nodes)
+//   ent_repr[]  the neighbour's LOCAL row: its position in the batch's node list taken in
+//               sampling order (targets first).  In that order the rows layer l needs are the
+//               prefix [0, N_l) of the batch, which is what Algorithm 2 achieves by cutting the
+//               front of node_ids in the paper's (reversed) order.
+// The paper's arrays are produced from this by mg_dense_view.
+//
+// Every kernel sizes itself from counters in device memory (DenseHeader), so a k-hop sample is
+// issued without a host round trip per hop; the host reads the header once at the end.
+
+#include <stdarg.h>
+
+#include <algorithm>
+
+#include "mg_device.cuh"
+#include "mg_internal.cuh"
+
+namespace {
+
+constexpr int kThreads = 256;
+
+// -------------------------------------------------------------------------------------
+// generic exclusive scan over a device-sized range (three kernels, no inter-block waits)
+// -------------------------------------------------------------------------------------
+constexpr int kScanTile = 2048;  // 256 threads x 8
+
+struct ScanRange {       // all device pointers
+    const int32_t* lo;   // range is data[*lo .. *hi)
+    const int32_t* hi;
+    const int32_t* base; // value added to every output (nullable)
+};
+
+__device__ __forceinline__ uint32_t block_excl_scan_256(uint32_t v, uint32_t* smem /*>= 9*/, uint32_t* total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t inc = warp_incl_scan(v);
+    if (lane == 31) smem[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t w = lane < 8 ? smem[lane] : 0u;
+        const uint32_t wi = warp_incl_scan(w);
+        if (lane < 8) smem[lane] = wi - w;
+        if (lane == 7) smem[8] = wi;
+    }
+    __syncthreads();
+    const uint32_t res = inc - v + smem[warp];
+    *total = smem[8];
+    __syncthreads();
+    return res;
+}
+
+__global__ void __launch_bounds__(kThreads) k_scan_reduce(const uint32_t* data, ScanRange r, uint32_t* tile_sums) {
+    __shared__ uint32_t sm[9];
+    const int32_t lo = *r.lo, n = *r.hi - lo;
+    const int ntiles = (n + kScanTile - 1) / kScanTile;
+    for (int t = blockIdx.x; t < ntiles; t += gridDim.x) {
+        uint32_t s = 0;
+        const int start = t * kScanTile + threadIdx.x * 8;
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            if (start + j < n) s += data[lo + start + j];
+        uint32_t total;
+        block_excl_scan_256(s, sm, &total);
+        if (threadIdx.x == 0) tile_sums[t] = total;
+    }
+}
+
+// single block: exclusive scan of the tile sums in place; total (plus base) to *total_out
+__global__ void __launch_bounds__(1024) k_scan_tiles(uint32_t* tile_sums, ScanRange r, uint32_t* total_out) {
+    __shared__ uint32_t warp_tot[33];
+    const int n = *r.hi - *r.lo;
+    const int ntiles = (n + kScanTile - 1) / kScanTile;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t carry = 0;
+    for (int start = 0; start < ntiles; start += 1024) {
+        const int i = start + threadIdx.x;
+        const uint32_t v = i < ntiles ? tile_sums[i] : 0u;
+        const uint32_t inc = warp_incl_scan(v);
+        if (lane == 31) warp_tot[warp] = inc;
+        __syncthreads();
+        if (warp == 0) {
+            const uint32_t w = warp_tot[lane];
+            const uint32_t wi = warp_incl_scan(w);
+            warp_tot[lane] = wi - w;
+            if (lane == 31) warp_tot[32] = wi;
+        }
+        __syncthreads();
+        if (i < ntiles) tile_sums[i] = carry + warp_tot[warp] + inc - v;
+        carry += warp_tot[32];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0 && total_out) *total_out = carry + (r.base ? (uint32_t)*r.base : 0u);
+}
+
+__global__ void __launch_bounds__(kThreads) k_scan_down(uint32_t* data, ScanRange r, const uint32_t* tile_sums) {
+    __shared__ uint32_t sm[9];
+    const int32_t lo = *r.lo, n = *r.hi - lo;
+    const uint32_t base = r.base ? (uint32_t)*r.base : 0u;
+    const int ntiles = (n + kScanTile - 1) / kScanTile;
+    for (int t = blockIdx.x; t < ntiles; t += gridDim.x) {
+        uint32_t v[8], s = 0;
+        const int start = t * kScanTile + threadIdx.x * 8;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            v[j] = (start + j < n) ? data[lo + start + j] : 0u;
+            s += v[j];
+        }
+        uint32_t total;
+        uint32_t run = block_excl_scan_256(s, sm, &total) + tile_sums[t] + base;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (start + j < n) data[lo + start + j] = run;
+            run += v[j];
+        }
+    }
+}
+
+// -------------------------------------------------------------------------------------
+// hop 0: targets
+// -------------------------------------------------------------------------------------
+struct TableGeom {
+    int32_t size;   // slots per batch
+    int32_t shift;  // 32 - log2(size)
+};
+
+__global__ void __launch_bounds__(kThreads)
+k_init_targets(DenseHeader* hdr, const int32_t* __restrict__ targets, int32_t n_total,
+               const int32_t* __restrict__ tgt_off, int32_t B, int32_t* nodes, int32_t* node_batch,
+               int32_t* hkeys, int32_t* hvals, TableGeom tg, int64_t n_nodes, int64_t part_size,
+               const int32_t* __restrict__ slot_of_part) {
+    for (int32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n_total; i += gridDim.x * blockDim.x) {
+        const int b = upper_segment(tgt_off, B + 1, i);
+        const int32_t v = targets[i];
+        nodes[i] = v;
+        node_batch[i] = b;
+        if (v < 0 || (int64_t)v >= n_nodes) { atomicOr(&hdr->status, ST_RANGE); continue; }
+        if (slot_of_part[(int64_t)v / part_size] < 0) { atomicOr(&hdr->status, ST_NONRESIDENT); continue; }
+        bool is_new;
+        const int32_t slot = table_insert(hkeys + (int64_t)b * tg.size, tg.size, tg.shift, v, &is_new);
+        if (slot < 0) { atomicOr(&hdr->status, ST_CAP_TABLE); continue; }
+        if (!is_new) { atomicOr(&hdr->status, ST_DUPLICATE); continue; }
+        hvals[(int64_t)b * tg.size + slot] = i - tgt_off[b];
+    }
+}
+
+// -------------------------------------------------------------------------------------
+// per hop: degree -> count, (scan), pick + id-table insert, (sort), place, relabel
+// -------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+k_count(const DenseHeader* hdr, int hop, int32_t fanout, const int32_t* __restrict__ nodes,
+        const int64_t* __restrict__ row_off, int32_t* ent_off) {
+    if (hdr->status) return;
+    const int32_t lo = hdr->hop_base[hop], hi = hdr->hop_base[hop + 1];
+    for (int32_t i = lo + blockIdx.x * blockDim.x + threadIdx.x; i < hi; i += gridDim.x * blockDim.x) {
+        const int32_t v = nodes[i];
+        const int64_t d = row_off[v + 1] - row_off[v];
+        ent_off[i] = (int32_t)(d < (int64_t)fanout ? d : (int64_t)fanout);
+    }
+}
+
+// after the scan: close the hop's entry range and check the arena
+__global__ void k_entries_done(DenseHeader* hdr, int hop, const uint32_t* total, int32_t* ent_off, int64_t cap_entries) {
+    if (hdr->status) return;
+    const uint32_t end = *total;  // already includes ent_base[hop]
+    if ((int64_t)end > cap_entries) { atomicOr(&hdr->status, ST_CAP_ENTRIES); return; }
+    hdr->ent_base[hop + 1] = (int32_t)end;
+    ent_off[hdr->hop_base[hop + 1]] = (int32_t)end;
+    hdr->n_new = 0;
+}
+
+struct PickArgs {
+    DenseHeader* hdr;
+    int hop;
+    int32_t fanout;
+    const int32_t* nodes;
+    const int32_t* node_batch;
+    const int64_t* row_off;
+    const int32_t* row_nbrs;
+    const int32_t* ent_off;
+    int32_t* ent_nbrs;
+    int32_t* ent_repr;  // receives batch * table_size + slot until k_relabel
+    int32_t* hkeys;
+    TableGeom tg;
+    const uint64_t* seeds;
+    uint64_t* newlist;
+    int64_t cap_new;
+    int id_bits;
+};
+
+// Appends this block's new composite keys to the list: one global atomic per block call.
+__device__ __forceinline__ void block_append(const PickArgs& a, bool is_new, uint64_t key, uint32_t* sm_cnt /*[2]*/) {
+    const int lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) sm_cnt[0] = 0;
+    __syncthreads();
+    const uint32_t bal = __ballot_sync(0xFFFFFFFFu, is_new);
+    uint32_t warp_off = 0;
+    if (lane == 0 && bal) warp_off = atomicAdd(&sm_cnt[0], __popc(bal));
+    warp_off = __shfl_sync(0xFFFFFFFFu, warp_off, 0);
+    __syncthreads();
+    if (threadIdx.x == 0) sm_cnt[1] = sm_cnt[0] ? atomicAdd(&a.hdr->n_new, sm_cnt[0]) : 0u;
+    __syncthreads();
+    if (is_new) {
+        const int64_t pos = (int64_t)sm_cnt[1] + warp_off + __popc(bal & ((1u << lane) - 1u));
+        if (pos < a.cap_new) a.newlist[pos] = key;
+        else atomicOr(&a.hdr->status, ST_CAP_NODES);
+    }
+    __syncthreads();
+}
+
+__device__ __forceinline__ void insert_pick(const PickArgs& a, bool valid, int32_t b, int32_t u, int32_t out_pos,
+                                            bool* is_new, uint64_t* key) {
+    *is_new = false;
+    *key = 0;
+    if (!valid) return;
+    a.ent_nbrs[out_pos] = u;
+    bool fresh;
+    const int32_t slot = table_insert(a.hkeys + (int64_t)b * a.tg.size, a.tg.size, a.tg.shift, u, &fresh);
+    if (slot < 0) { atomicOr(&a.hdr->status, ST_CAP_TABLE); a.ent_repr[out_pos] = 0; return; }
+    a.ent_repr[out_pos] = b * a.tg.size + slot;
+    if (fresh) {
+        *is_new = true;
+        *key = (uint64_t)(uint32_t)slot | ((uint64_t)(uint32_t)u << MG_SLOT_BITS) |
+               ((uint64_t)(uint32_t)b << (MG_SLOT_BITS + a.id_bits));
+    }
+}
+
+// G lanes per node, fanout <= G <= 32.
+template <int G>
+__global__ void __launch_bounds__(kThreads) k_pick(PickArgs a) {
+    __shared__ uint32_t sm_cnt[2];
+    if (a.hdr->status) return;
+    constexpr int kGroups = kThreads / G;
+    const int32_t lo = a.hdr->hop_base[a.hop], hi = a.hdr->hop_base[a.hop + 1];
+    const int lane = threadIdx.x & 31;
+    const int gl = threadIdx.x % G;               // lane inside the group
+    const int gshift = lane - gl;                 // first warp lane of the group
+    const uint32_t gmask = (G == 32) ? 0xFFFFFFFFu : (((1u << G) - 1u) << gshift);
+    const int32_t f = a.fanout;
+    for (int32_t base = lo + blockIdx.x * kGroups; base < hi; base += gridDim.x * kGroups) {
+        const int32_t i = base + threadIdx.x / G;
+        const bool node_ok = i < hi;
+        int32_t v = 0, b = 0, out0 = 0;
+        int64_t r0 = 0, d = 0;
+        if (node_ok) {
+            v = a.nodes[i];
+            b = a.node_batch[i];
+            out0 = a.ent_off[i];
+            r0 = a.row_off[v];
+            d = a.row_off[v + 1] - r0;
+        }
+        bool valid = false;
+        int32_t u = 0, pos = 0;
+        const bool floyd = node_ok && d > (int64_t)f;
+        // Floyd's subset algorithm: slot t draws x in [0, d-f+t]; it keeps x unless an earlier slot
+        // already holds x, in which case it keeps d-f+t.  Draws are independent of each other, so
+        // all lanes draw at once and only the "already held" test runs slot by slot.
+        uint32_t x = 0xFFFFFFFFu, jt = 0, pick = 0xFFFFFFFFu;
+        if (floyd && gl < f) {
+            jt = (uint32_t)(d - f) + (uint32_t)gl;
+            x = __umulhi(draw_word(a.seeds[b], (uint32_t)v, (uint32_t)a.hop, (uint32_t)gl), jt + 1u);
+        }
+        for (int t = 0; t < f; ++t) {
+            const uint32_t xt = __shfl_sync(0xFFFFFFFFu, x, gshift + t);
+            const uint32_t hit = __ballot_sync(0xFFFFFFFFu, gl < t && pick == xt) & gmask;
+            if (gl == t) pick = hit ? jt : xt;
+        }
+        // rank of this lane's position among the f picks (they are distinct); every lane of the warp
+        // takes part in the shuffles, whatever its node needs
+        int rank = 0;
+        for (int t = 0; t < f; ++t) {
+            const uint32_t pt = __shfl_sync(0xFFFFFFFFu, pick, gshift + t);
+            rank += (pt < pick) ? 1 : 0;
+        }
+        if (floyd) {
+            if (gl < f) {
+                valid = true;
+                u = a.row_nbrs[r0 + (int64_t)pick];
+                pos = out0 + rank;
+            }
+        } else if (node_ok && (int64_t)gl < d) {
+            valid = true;
+            u = a.row_nbrs[r0 + gl];
+            pos = out0 + gl;
+        }
+        bool is_new;
+        uint64_t key;
+        insert_pick(a, valid, b, u, pos, &is_new, &key);
+        block_append(a, is_new, key, sm_cnt);
+    }
+}
+
+// Any fanout up to MG_MAX_FANOUT: one warp per node, picks staged in shared memory.
+__global__ void __launch_bounds__(kThreads) k_pick_wide(PickArgs a) {
+    __shared__ uint32_t sm_cnt[2];
+    extern __shared__ uint32_t sm_dyn[];  // per warp: x[f], pick[f]
+    if (a.hdr->status) return;
+    constexpr int kWarps = kThreads / 32;
+    const int32_t lo = a.hdr->hop_base[a.hop], hi = a.hdr->hop_base[a.hop + 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int32_t f = a.fanout;
+    uint32_t* xs = sm_dyn + (size_t)warp * 2 * f;
+    uint32_t* picks = xs + f;
+    const int rounds = (f + 31) / 32;
+    for (int32_t base = lo + blockIdx.x * kWarps; base < hi; base += gridDim.x * kWarps) {
+        const int32_t i = base + warp;
+        const bool node_ok = i < hi;
+        int32_t v = 0, b = 0, out0 = 0;
+        int64_t r0 = 0, d = 0;
+        if (node_ok) {
+            v = a.nodes[i];
+            b = a.node_batch[i];
+            out0 = a.ent_off[i];
+            r0 = a.row_off[v];
+            d = a.row_off[v + 1] - r0;
+        }
+        const bool floyd = node_ok && d > (int64_t)f;
+        if (floyd) {
+            for (int t = lane; t < f; t += 32) {
+                const uint32_t jt = (uint32_t)(d - f) + (uint32_t)t;
+                xs[t] = __umulhi(draw_word(a.seeds[b], (uint32_t)v, (uint32_t)a.hop, (uint32_t)t), jt + 1u);
+            }
+            __syncwarp();
+            for (int t = 0; t < f; ++t) {
+                const uint32_t xt = xs[t];
+                bool hit = false;
+                for (int s = lane; s < t; s += 32) hit |= (picks[s] == xt);
+                const bool any = __any_sync(0xFFFFFFFFu, hit);
+                if (lane == 0) picks[t] = any ? ((uint32_t)(d - f) + (uint32_t)t) : xt;
+                __syncwarp();
+            }
+        }
+        // every warp of the block runs the same number of append rounds
+        for (int rd = 0; rd < rounds; ++rd) {
+            const int t = rd * 32 + lane;
+            bool valid = false;
+            int32_t u = 0, pos = 0;
+            if (floyd && t < f) {
+                const uint32_t p = picks[t];
+                int rank = 0;
+                for (int s = 0; s < f; ++s) rank += (picks[s] < p) ? 1 : 0;
+                valid = true;
+                u = a.row_nbrs[r0 + (int64_t)p];
+                pos = out0 + rank;
+            } else if (node_ok && !floyd && (int64_t)t < d) {
+                valid = true;
+                u = a.row_nbrs[r0 + t];
+                pos = out0 + t;
+            }
+            bool is_new;
+            uint64_t key;
+            insert_pick(a, valid, b, u, pos, &is_new, &key);
+            block_append(a, is_new, key, sm_cnt);
+        }
+        __syncwarp();
+    }
+}
+
+// -------------------------------------------------------------------------------------
+// radix sort of the new-node list on bits [lo_bit, lo_bit + bits) of the composite key
+// -------------------------------------------------------------------------------------
+constexpr int kSortKeysPerThread = 16;
+constexpr int kSortTile = kThreads * kSortKeysPerThread;  // 4096
+
+__global__ void k_sort_setup(const DenseHeader* hdr, SortParams* sp) {
+    const int32_t n = hdr->status ? 0 : (int32_t)hdr->n_new;
+    sp->zero = 0;
+    sp->n = n;
+    sp->ntiles = (n + kSortTile - 1) / kSortTile;
+    sp->hist_len = 256 * sp->ntiles;
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_radix_hist(const uint64_t* __restrict__ keys, const SortParams* sp, int shift, uint32_t* hist) {
+    __shared__ uint32_t sh[256];
+    const int32_t n = sp->n, ntiles = sp->ntiles;
+    for (int t = blockIdx.x; t < ntiles; t += gridDim.x) {
+        sh[threadIdx.x] = 0;
+        __syncthreads();
+        const int32_t tb = t * kSortTile;
+#pragma unroll 4
+        for (int j = 0; j < kSortKeysPerThread; ++j) {
+            const int32_t i = tb + j * kThreads + threadIdx.x;
+            if (i < n) atomicAdd(&sh[(uint32_t)(keys[i] >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        hist[(size_t)threadIdx.x * ntiles + t] = sh[threadIdx.x];
+        __syncthreads();
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_radix_scatter(const uint64_t* __restrict__ keys, uint64_t* __restrict__ out, const SortParams* sp, int shift,
+                const uint32_t* __restrict__ hist_scanned) {
+    __shared__ uint32_t cnt[kThreads / 32][256];
+    const int32_t n = sp->n, ntiles = sp->ntiles;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr int kPerWarp = kSortTile / (kThreads / 32);  // 512 consecutive keys per warp
+    for (int t = blockIdx.x; t < ntiles; t += gridDim.x) {
+        for (int w = 0; w < kThreads / 32; ++w) cnt[w][threadIdx.x] = 0;
+        __syncthreads();
+        uint64_t key[kSortKeysPerThread];
+        uint32_t rank[kSortKeysPerThread];
+        const int32_t wb = t * kSortTile + warp * kPerWarp;
+#pragma unroll
+        for (int r = 0; r < kSortKeysPerThread; ++r) {
+            const int32_t i = wb + r * 32 + lane;
+            const bool ok = i < n;
+            key[r] = ok ? keys[i] : 0ull;
+            const uint32_t dg = ok ? ((uint32_t)(key[r] >> shift) & 255u) : 0xFFFFFFFFu;
+            const uint32_t peers = __match_any_sync(0xFFFFFFFFu, dg);
+            const int leader = __ffs(peers) - 1;
+            uint32_t old = 0;
+            if (ok && lane == leader) {
+                old = cnt[warp][dg];
+                cnt[warp][dg] = old + __popc(peers);
+            }
+            old = __shfl_sync(0xFFFFFFFFu, old, leader);
+            rank[r] = old + __popc(peers & ((1u << lane) - 1u));
+            __syncwarp();
+        }
+        __syncthreads();
+        {   // turn per-warp counts of digit `threadIdx.x` into global start positions
+            uint32_t run = hist_scanned[(size_t)threadIdx.x * ntiles + t];
+            for (int w = 0; w < kThreads / 32; ++w) {
+                const uint32_t c = cnt[w][threadIdx.x];
+                cnt[w][threadIdx.x] = run;
+                run += c;
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int r = 0; r < kSortKeysPerThread; ++r) {
+            const int32_t i = wb + r * 32 + lane;
+            if (i < n) out[cnt[warp][(uint32_t)(key[r] >> shift) & 255u] + rank[r]] = key[r];
+        }
+        __syncthreads();
+    }
+}
+
+// -------------------------------------------------------------------------------------
+// place the sorted new nodes as the next hop
+// -------------------------------------------------------------------------------------
+__global__ void k_hop_advance(DenseHeader* hdr, int hop, int32_t B, int32_t* node_off_next, int64_t cap_nodes) {
+    if (hdr->status) return;
+    const int32_t start = hdr->hop_base[hop + 1];
+    const int64_t end = (int64_t)start + hdr->n_new;
+    if (end > cap_nodes) { if (threadIdx.x == 0) atomicOr(&hdr->status, ST_CAP_NODES); return; }
+    if (threadIdx.x == 0) hdr->hop_base[hop + 2] = (int32_t)end;
+    if (hdr->n_new == 0)
+        for (int b = threadIdx.x; b <= B; b += blockDim.x) node_off_next[b] = start;
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_place_nodes(const DenseHeader* hdr, int hop, int32_t B, const uint64_t* __restrict__ sorted, int id_bits,
+              int32_t* nodes, int32_t* node_batch, int32_t* node_off_next) {
+    if (hdr->status) return;
+    const int32_t n = (int32_t)hdr->n_new, start = hdr->hop_base[hop + 1];
+    const uint64_t id_mask = (1ull << id_bits) - 1ull;
+    for (int32_t j = blockIdx.x * blockDim.x + threadIdx.x; j < n; j += gridDim.x * blockDim.x) {
+        const uint64_t key = sorted[j];
+        const int32_t b = (int32_t)(key >> (MG_SLOT_BITS + id_bits));
+        nodes[start + j] = (int32_t)((key >> MG_SLOT_BITS) & id_mask);
+        node_batch[start + j] = b;
+        const int32_t prev_b = j == 0 ? -1 : (int32_t)(sorted[j - 1] >> (MG_SLOT_BITS + id_bits));
+        for (int bb = prev_b + 1; bb <= b; ++bb) node_off_next[bb] = start + j;
+        if (j == n - 1)
+            for (int bb = b + 1; bb <= B; ++bb) node_off_next[bb] = start + n;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_place_rows(DenseHeader* hdr, int hop, int32_t B, int32_t k, const uint64_t* __restrict__ sorted, int id_bits,
+             const int32_t* __restrict__ node_off_next, int32_t* cum, int32_t* hvals, TableGeom tg,
+             int32_t max_nodes_per_batch) {
+    if (hdr->status) return;
+    const int32_t n = (int32_t)hdr->n_new, start = hdr->hop_base[hop + 1];
+    const int32_t tid = blockIdx.x * blockDim.x + threadIdx.x;
+    for (int32_t j = tid; j < n; j += gridDim.x * blockDim.x) {
+        const uint64_t key = sorted[j];
+        const int32_t b = (int32_t)(key >> (MG_SLOT_BITS + id_bits));
+        const int32_t slot = (int32_t)(key & ((1u << MG_SLOT_BITS) - 1u));
+        hvals[(int64_t)b * tg.size + slot] = cum[b * (k + 2) + hop + 1] + (start + j - node_off_next[b]);
+    }
+    for (int32_t b = tid; b < B; b += gridDim.x * blockDim.x) {
+        const int32_t v = cum[b * (k + 2) + hop + 1] + (node_off_next[b + 1] - node_off_next[b]);
+        cum[b * (k + 2) + hop + 2] = v;
+        if (v > max_nodes_per_batch) atomicOr(&hdr->status, ST_CAP_TABLE);
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_relabel(const DenseHeader* hdr, int hop, const int32_t* __restrict__ hvals, int32_t* ent_repr) {
+    if (hdr->status) return;
+    const int32_t lo = hdr->ent_base[hop], hi = hdr->ent_base[hop + 1];
+    for (int32_t e = lo + blockIdx.x * blockDim.x + threadIdx.x; e < hi; e += gridDim.x * blockDim.x)
+        ent_repr[e] = hvals[ent_repr[e]];
+}
+
+// one block: packed row bases of every layer and the per-batch entry bounds of every hop
+__global__ void __launch_bounds__(1024)
+k_finalize(DenseHeader* hdr, int32_t B, int32_t k, const int32_t* __restrict__ cum, const int32_t* __restrict__ node_off,
+           const int32_t* __restrict__ ent_off, int32_t* rowbase, int32_t* ent_hop) {
+    __shared__ uint32_t warp_tot[33];
+    if (hdr->status) return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int l = 0; l <= k; ++l) {
+        uint32_t carry = 0;
+        for (int start = 0; start < B; start += 1024) {
+            const int b = start + threadIdx.x;
+            const uint32_t v = b < B ? (uint32_t)cum[b * (k + 2) + (k - l + 1)] : 0u;
+            const uint32_t inc = warp_incl_scan(v);
+            if (lane == 31) warp_tot[warp] = inc;
+            __syncthreads();
+            if (warp == 0) {
+                const uint32_t w = warp_tot[lane];
+                const uint32_t wi = warp_incl_scan(w);
+                warp_tot[lane] = wi - w;
+                if (lane == 31) warp_tot[32] = wi;
+            }
+            __syncthreads();
+            if (b < B) rowbase[l * (B + 1) + b] = (int32_t)(carry + warp_tot[warp] + inc - v);
+            carry += warp_tot[32];
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) {
+            rowbase[l * (B + 1) + B] = (int32_t)carry;
+            hdr->rows_total[l] = (int32_t)carry;
+        }
+    }
+    for (int h = 0; h < k; ++h)
+        for (int b = threadIdx.x; b <= B; b += blockDim.x)
+            ent_hop[h * (B + 1) + b] = ent_off[node_off[h * (B + 1) + b]];
+}
+
+// -------------------------------------------------------------------------------------
+// export to the paper's layout (mg_dense_view)
+// -------------------------------------------------------------------------------------
+struct ExportArgs {
+    int32_t k, b, B;
+    int32_t V, n0, E;
+    int32_t nio[MG_MAX_HOPS + 2];     // canonical node_id_offsets
+    int32_t ebase[MG_MAX_HOPS + 1];   // canonical first entry of Delta_j's neighbours, j = 1..k
+    int32_t cum[MG_MAX_HOPS + 2];     // local row base per hop
+    int32_t node_off[MG_MAX_HOPS + 1];
+    int32_t ent_hop[MG_MAX_HOPS + 1];
+    const int32_t *nodes, *ent_off, *ent_nbrs, *ent_repr;
+    int32_t *o_node_ids, *o_nio, *o_nbrs, *o_nbr_off, *o_repr;
+};
+
+__global__ void __launch_bounds__(kThreads) k_export(ExportArgs a) {
+    const int32_t tid = blockIdx.x * blockDim.x + threadIdx.x;
+    if (tid <= a.k + 1) a.o_nio[tid] = a.nio[tid];
+    if (tid == 0) a.o_nbr_off[a.V - a.n0] = a.E;
+    for (int32_t c = tid; c < a.V; c += gridDim.x * blockDim.x) {
+        int j = 0;
+        while (j < a.k && c >= a.nio[j + 1]) ++j;
+        const int h = a.k - j;
+        const int32_t idx = a.node_off[h] + (c - a.nio[j]);
+        a.o_node_ids[c] = a.nodes[idx];
+        if (j == 0) continue;
+        const int32_t e0 = a.ent_off[idx], e1 = a.ent_off[idx + 1];
+        const int32_t o0 = a.ebase[j] + (e0 - a.ent_hop[h]);
+        a.o_nbr_off[c - a.n0] = o0;
+        for (int32_t e = e0; e < e1; ++e) {
+            a.o_nbrs[o0 + (e - e0)] = a.ent_nbrs[e];
+            const int32_t l = a.ent_repr[e];
+            int hh = 0;
+            while (hh < a.k && l >= a.cum[hh + 1]) ++hh;
+            a.o_repr[o0 + (e - e0)] = a.nio[a.k - hh] + (l - a.cum[hh]);
+        }
+    }
+}
+
+int ilog2_ceil(int64_t x) {
+    int b = 0;
+    while (((int64_t)1 << b) < x) ++b;
+    return b;
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------
+// generic pieces other translation units use
+// ---------------------------------------------------------------------------------------
+size_t mg_sort_hist_elems(int64_t max_keys) { return (size_t)256 * ((max_keys + kSortTile - 1) / kSortTile) + 256; }
+size_t mg_scan_tmp_elems(int64_t max_elems) { return (size_t)((max_elems + kScanTile - 1) / kScanTile) + 16; }
+
+// LSD radix sort of 64-bit keys on bits [lo_bit, lo_bit + bits); sp (device) holds the key count.
+// Keys start in buf[0]; *res_buf tells which buffer holds the result.
+void mg_sort_u64(mg_ctx* ctx, uint64_t* const buf[2], const SortParams* sp, int lo_bit, int bits, uint32_t* hist,
+                 uint32_t* scan_tmp, int* res_buf) {
+    cudaStream_t st = ctx->stream;
+    const int grid = mg_grid(ctx, 8);
+    const int passes = (bits + 7) / 8;
+    ScanRange r{&sp->zero, &sp->hist_len, nullptr};
+    int cur = 0;
+    for (int p = 0; p < passes; ++p) {
+        const int shift = lo_bit + 8 * p;
+        k_radix_hist<<<grid, kThreads, 0, st>>>(buf[cur], sp, shift, hist);
+        k_scan_reduce<<<grid, kThreads, 0, st>>>(hist, r, scan_tmp);
+        k_scan_tiles<<<1, 1024, 0, st>>>(scan_tmp, r, nullptr);
+        k_scan_down<<<grid, kThreads, 0, st>>>(hist, r, scan_tmp);
+        k_radix_scatter<<<grid, kThreads, 0, st>>>(buf[cur], buf[cur ^ 1], sp, shift, hist);
+        cur ^= 1;
+    }
+    ctx->launches += 5 * passes;
+    *res_buf = cur;
+}
+
+// in-place exclusive scan of data[*lo .. *hi) (+ *base); total (+ *base) to *total_out (nullable)
+void mg_scan_u32(mg_ctx* ctx, uint32_t* data, const int32_t* lo, const int32_t* hi, const int32_t* base,
+                 uint32_t* scan_tmp, uint32_t* total_out) {
+    cudaStream_t st = ctx->stream;
+    const int grid = mg_grid(ctx, 8);
+    ScanRange r{lo, hi, base};
+    k_scan_reduce<<<grid, kThreads, 0, st>>>(data, r, scan_tmp);
+    k_scan_tiles<<<1, 1024, 0, st>>>(scan_tmp, r, total_out);
+    k_scan_down<<<grid, kThreads, 0, st>>>(data, r, scan_tmp);
+    ctx->launches += 3;
+}
+
+// ---------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------
+template <typename T>
+static int dev_realloc(mg_ctx* ctx, T** p, size_t elems) {
+    if (*p) cudaFree(*p);
+    *p = nullptr;
+    if (cudaMalloc((void**)p, std::max<size_t>(elems, 1) * sizeof(T)) != cudaSuccess) {
+        cudaGetLastError();
+        *p = nullptr;
+        return mg_fail(ctx, MG_ERR_OOM, "device allocation of %zu bytes failed", elems * sizeof(T));
+    }
+    return MG_OK;
+}
+
+static int dense_alloc(mg_ctx* ctx, mg_dense* d, int32_t B, int32_t k, int64_t cap_nodes, int64_t cap_entries,
+                       int32_t table_size) {
+    int rc;
+    if (!d->hdr && (rc = dev_realloc(ctx, &d->hdr, 1))) return rc;
+    if (d->cap_nodes < cap_nodes) {
+        d->cap_nodes = 0;
+        if ((rc = dev_realloc(ctx, &d->nodes, (size_t)cap_nodes))) return rc;
+        if ((rc = dev_realloc(ctx, &d->node_batch, (size_t)cap_nodes))) return rc;
+        if ((rc = dev_realloc(ctx, &d->ent_off, (size_t)cap_nodes + 1))) return rc;
+        if ((rc = dev_realloc(ctx, &d->newlist[0], (size_t)cap_nodes))) return rc;
+        if ((rc = dev_realloc(ctx, &d->newlist[1], (size_t)cap_nodes))) return rc;
+        const int64_t sort_tiles = (cap_nodes + kSortTile - 1) / kSortTile;
+        const int64_t scan_tiles = std::max<int64_t>((cap_nodes + kScanTile - 1) / kScanTile,
+                                                     (256 * sort_tiles + kScanTile - 1) / kScanTile);
+        d->scan_tmp_elems = (size_t)scan_tiles + 16;
+        (void)scan_tiles;
+        if ((rc = dev_realloc(ctx, &d->scan_tmp, d->scan_tmp_elems))) return rc;
+        d->sort_hist_elems = (size_t)256 * sort_tiles + 256;
+        if ((rc = dev_realloc(ctx, &d->sort_hist, d->sort_hist_elems))) return rc;
+        d->cap_nodes = cap_nodes;
+    }
+    if (d->cap_entries < cap_entries) {
+        d->cap_entries = 0;
+        if ((rc = dev_realloc(ctx, &d->ent_nbrs, (size_t)cap_entries))) return rc;
+        if ((rc = dev_realloc(ctx, &d->ent_repr, (size_t)cap_entries))) return rc;
+        d->cap_entries = cap_entries;
+    }
+    const int64_t need_table = (int64_t)B * table_size;
+    if (d->alloc_table < need_table) {
+        d->alloc_table = 0;
+        if ((rc = dev_realloc(ctx, &d->hkeys, (size_t)need_table))) return rc;
+        if ((rc = dev_realloc(ctx, &d->hvals, (size_t)need_table))) return rc;
+        d->alloc_table = need_table;
+    }
+    const int64_t need_b = (int64_t)(MG_MAX_HOPS + 2) * (B + 1);
+    if (d->alloc_batches < need_b) {
+        d->alloc_batches = 0;
+        if ((rc = dev_realloc(ctx, &d->node_off, (size_t)need_b))) return rc;
+        if ((rc = dev_realloc(ctx, &d->cum, (size_t)need_b))) return rc;
+        if ((rc = dev_realloc(ctx, &d->rowbase, (size_t)need_b))) return rc;
+        if ((rc = dev_realloc(ctx, &d->d_ent_hop, (size_t)need_b))) return rc;
+        if ((rc = dev_realloc(ctx, &d->d_seeds, (size_t)need_b))) return rc;
+        d->alloc_batches = need_b;
+    }
+    d->k = k;
+    d->n_batches = B;
+    d->table_size = table_size;
+    d->table_shift = 32 - ilog2_ceil(table_size);
+    return MG_OK;
+}
+
+static const char* status_text(uint32_t st) {
+    if (st & ST_RANGE) return "a target id is outside [0, n_nodes)";
+    if (st & ST_NONRESIDENT) return "a target lies in a partition that is not resident";
+    if (st & ST_DUPLICATE) return "a batch lists a target twice";
+    if (st & ST_CAP_ENTRIES) return "neighbour capacity (max_entries_total) exceeded";
+    if (st & ST_CAP_NODES) return "node capacity (max_nodes_total) exceeded";
+    if (st & ST_CAP_TABLE) return "per-batch node capacity (max_nodes_per_batch) exceeded";
+    return "internal invariant violated";
+}
+
+static int status_code(uint32_t st) {
+    if (st & ST_RANGE) return MG_ERR_ARG;
+    if (st & ST_NONRESIDENT) return MG_ERR_NONRESIDENT;
+    if (st & ST_DUPLICATE) return MG_ERR_DUPLICATE;
+    if (st & (ST_CAP_ENTRIES | ST_CAP_NODES | ST_CAP_TABLE)) return MG_ERR_CAPACITY;
+    return MG_ERR_CUDA;
+}
+
+extern "C" int mg_sample_many(mg_ctx* ctx, const int32_t* targets, int targets_on_device,
+                              const int64_t* target_offsets, int32_t n_batches, const int32_t* fanouts,
+                              int32_t k, const uint64_t* seeds, const mg_sample_caps* caps, mg_dense** out) {
+    if (!ctx) return MG_ERR_ARG;
+    if (!out || !target_offsets || !fanouts || !seeds) return mg_fail(ctx, MG_ERR_ARG, "null argument");
+    if (n_batches <= 0 || n_batches > MG_MAX_BATCHES) return mg_fail(ctx, MG_ERR_ARG, "n_batches must be in [1, %d]", MG_MAX_BATCHES);
+    if (k <= 0 || k > MG_MAX_HOPS) return mg_fail(ctx, MG_ERR_ARG, "k must be in [1, %d]", MG_MAX_HOPS);
+    for (int h = 0; h < k; ++h)
+        if (fanouts[h] <= 0 || fanouts[h] > MG_MAX_FANOUT) return mg_fail(ctx, MG_ERR_ARG, "fanouts must be in [1, %d]", MG_MAX_FANOUT);
+    if (!ctx->row_off) return mg_fail(ctx, MG_ERR_STATE, "no graph loaded");
+    if (target_offsets[0] != 0) return mg_fail(ctx, MG_ERR_ARG, "target_offsets[0] must be 0");
+    for (int b = 0; b < n_batches; ++b)
+        if (target_offsets[b + 1] < target_offsets[b]) return mg_fail(ctx, MG_ERR_ARG, "target_offsets must be non-decreasing");
+    const int64_t T = target_offsets[n_batches];
+    if (T > 0 && !targets) return mg_fail(ctx, MG_ERR_ARG, "null targets");
+    if (T >= (1ll << 31)) return mg_fail(ctx, MG_ERR_ARG, "too many targets");
+    MG_CUDA(ctx, cudaSetDevice(ctx->device));
+
+    // capacities: worst case unless the caller bounds them
+    const int64_t N = ctx->n_nodes;
+    int64_t worst_nodes_total = 0, worst_entries_total = 0, worst_nodes_batch = 0;
+    for (int b = 0; b < n_batches; ++b) {
+        double level = (double)(target_offsets[b + 1] - target_offsets[b]);  // nodes that can be new at this hop
+        double nodes = level, entries = 0;
+        for (int h = 0; h < k; ++h) {
+            level = std::min(level, (double)N) * fanouts[h];
+            entries += level;
+            nodes += level;
+        }
+        const int64_t nb = (int64_t)std::min(nodes, (double)N);
+        worst_nodes_total += nb;
+        worst_entries_total += (int64_t)std::min(entries, 4.0e18);
+        worst_nodes_batch = std::max(worst_nodes_batch, nb);
+    }
+    int64_t cap_nodes = (caps && caps->max_nodes_total > 0) ? caps->max_nodes_total : worst_nodes_total;
+    int64_t cap_entries = (caps && caps->max_entries_total > 0) ? caps->max_entries_total : worst_entries_total;
+    int64_t cap_batch = (caps && caps->max_nodes_per_batch > 0) ? caps->max_nodes_per_batch : worst_nodes_batch;
+    cap_nodes = std::max<int64_t>(cap_nodes, T);
+    cap_batch = std::max<int64_t>(cap_batch, 1);
+    for (int b = 0; b < n_batches; ++b) cap_batch = std::max<int64_t>(cap_batch, target_offsets[b + 1] - target_offsets[b]);
+    if (cap_nodes >= (1ll << 31) - 1 || cap_entries >= (1ll << 31) - 1)
+        return mg_fail(ctx, MG_ERR_CAPACITY, "capacities must stay below 2^31 (nodes %lld, entries %lld): pass tighter mg_sample_caps or fewer batches",
+                       (long long)cap_nodes, (long long)cap_entries);
+    const int tbits = std::max(4, ilog2_ceil(cap_batch * 2));
+    if (tbits > MG_SLOT_BITS) return mg_fail(ctx, MG_ERR_CAPACITY, "max_nodes_per_batch above %d", 1 << (MG_SLOT_BITS - 1));
+    const int32_t table_size = 1 << tbits;
+    if ((int64_t)table_size * n_batches >= (1ll << 31))
+        return mg_fail(ctx, MG_ERR_CAPACITY, "n_batches x id-table size must stay below 2^31: pass a smaller max_nodes_per_batch or fewer batches");
+    const int id_bits = std::max(1, ilog2_ceil(N));
+    const int b_bits = std::max(1, ilog2_ceil(n_batches));
+    if (MG_SLOT_BITS + id_bits + b_bits > 64) return mg_fail(ctx, MG_ERR_ARG, "id and batch bits do not fit the sort key");
+
+    mg_dense* d = *out;
+    const bool created = (d == nullptr);
+    if (created) { d = new mg_dense(); d->ctx = ctx; }
+    else if (d->ctx != ctx) return mg_fail(ctx, MG_ERR_ARG, "mg_dense belongs to another context");
+    d->valid = false;
+    int rc = dense_alloc(ctx, d, n_batches, k, cap_nodes, std::max<int64_t>(cap_entries, 1), table_size);
+    if (rc) { if (created) mg_dense_free(d); return rc; }
+    *out = d;
+    for (int h = 0; h < k; ++h) d->fanouts[h] = fanouts[h];
+    d->n_targets_total = T;
+
+    cudaStream_t st = ctx->stream;
+    const int B = n_batches;
+    const TableGeom tg{table_size, d->table_shift};
+
+    // host-known part of the header and per-batch tables
+    DenseHeader hh;
+    memset(&hh, 0, sizeof(hh));
+    hh.hop_base[0] = 0;
+    hh.hop_base[1] = (int32_t)T;
+    std::vector<int32_t> off32(B + 1), cum0((size_t)B * (k + 2), 0);
+    for (int b = 0; b <= B; ++b) off32[b] = (int32_t)target_offsets[b];
+    for (int b = 0; b < B; ++b) cum0[(size_t)b * (k + 2) + 1] = off32[b + 1] - off32[b];
+    {
+        ProfScope ps(ctx, PH_SAMPLE_INIT, 1);
+        MG_CUDA(ctx, cudaMemcpyAsync(d->hdr, &hh, sizeof(hh), cudaMemcpyHostToDevice, st));
+        MG_CUDA(ctx, cudaMemcpyAsync(d->node_off, off32.data(), sizeof(int32_t) * (B + 1), cudaMemcpyHostToDevice, st));
+        MG_CUDA(ctx, cudaMemcpyAsync(d->cum, cum0.data(), sizeof(int32_t) * cum0.size(), cudaMemcpyHostToDevice, st));
+        MG_CUDA(ctx, cudaMemcpyAsync(d->d_seeds, seeds, sizeof(uint64_t) * B, cudaMemcpyHostToDevice, st));
+        MG_CUDA(ctx, cudaMemsetAsync(d->hkeys, 0xFF, sizeof(int32_t) * (size_t)B * table_size, st));
+        // the targets are staged in newlist[1] when they come from the host
+        const int32_t* tgt_dev = targets;
+        if (!targets_on_device && T > 0) {
+            MG_CUDA(ctx, cudaMemcpyAsync(d->newlist[1], targets, sizeof(int32_t) * T, cudaMemcpyHostToDevice, st));
+            tgt_dev = (const int32_t*)d->newlist[1];
+        }
+        if (T > 0) {
+            k_init_targets<<<mg_grid(ctx, 4), kThreads, 0, st>>>(d->hdr, tgt_dev, (int32_t)T, d->node_off, B, d->nodes,
+                                                               d->node_batch, d->hkeys, d->hvals, tg, ctx->n_nodes,
+                                                               ctx->part_size, ctx->d_slot_of_part);
+            ctx->launches++;
+        }
+    }
+
+    SortParams* sp = (SortParams*)(d->scan_tmp + d->scan_tmp_elems - 8);  // tail of the scratch block
+    uint32_t* scan_total = (uint32_t*)(d->scan_tmp + d->scan_tmp_elems - 4);
+    const int grid = mg_grid(ctx, 8);
+    for (int h = 0; h < k; ++h) {
+        const int32_t f = fanouts[h];
+        {
+            ProfScope ps(ctx, PH_SAMPLE_COUNT, 1);
+            k_count<<<grid, kThreads, 0, st>>>(d->hdr, h, f, d->nodes, ctx->view_off, d->ent_off);
+        }
+        {
+            ProfScope ps(ctx, PH_SAMPLE_SCAN, 4);
+            mg_scan_u32(ctx, (uint32_t*)d->ent_off, &d->hdr->hop_base[h], &d->hdr->hop_base[h + 1], &d->hdr->ent_base[h],
+                        (uint32_t*)d->scan_tmp, scan_total);
+            k_entries_done<<<1, 1, 0, st>>>(d->hdr, h, scan_total, d->ent_off, d->cap_entries);
+        }
+        {
+            ProfScope ps(ctx, PH_SAMPLE_PICK, 1);
+            PickArgs a{d->hdr, h, f, d->nodes, d->node_batch, ctx->view_off, ctx->view_nbrs, d->ent_off, d->ent_nbrs,
+                       d->ent_repr, d->hkeys, tg, d->d_seeds, d->newlist[0], d->cap_nodes, id_bits};
+            if (f <= 4) k_pick<4><<<grid, kThreads, 0, st>>>(a);
+            else if (f <= 8) k_pick<8><<<grid, kThreads, 0, st>>>(a);
+            else if (f <= 16) k_pick<16><<<grid, kThreads, 0, st>>>(a);
+            else if (f <= 32) k_pick<32><<<grid, kThreads, 0, st>>>(a);
+            else k_pick_wide<<<grid, kThreads, (size_t)(kThreads / 32) * 2 * f * sizeof(uint32_t), st>>>(a);
+        }
+        int res_buf = 0;
+        {
+            const int key_bits = id_bits + b_bits;
+            const int passes = (key_bits + 7) / 8;
+            ProfScope ps(ctx, PH_SAMPLE_SORT, 1 + passes * 5);
+            k_sort_setup<<<1, 1, 0, st>>>(d->hdr, sp);
+            mg_sort_u64(ctx, d->newlist, sp, MG_SLOT_BITS, key_bits, d->sort_hist, (uint32_t*)d->scan_tmp, &res_buf);
+        }
+        {
+            ProfScope ps(ctx, PH_SAMPLE_PLACE, 3);
+            int32_t* off_next = d->node_off + (size_t)(h + 1) * (B + 1);
+            k_hop_advance<<<1, 256, 0, st>>>(d->hdr, h, B, off_next, d->cap_nodes);
+            k_place_nodes<<<grid, kThreads, 0, st>>>(d->hdr, h, B, d->newlist[res_buf], id_bits, d->nodes, d->node_batch, off_next);
+            k_place_rows<<<grid, kThreads, 0, st>>>(d->hdr, h, B, k, d->newlist[res_buf], id_bits, off_next, d->cum, d->hvals, tg,
+                                                    (int32_t)cap_batch);
+        }
+        {
+            ProfScope ps(ctx, PH_SAMPLE_RELABEL, 1);
+            k_relabel<<<grid, kThreads, 0, st>>>(d->hdr, h, d->hvals, d->ent_repr);
+        }
+        ctx->launches += 1 + 1 + 1 + 1 + 3 + 1;  // count, entries_done, pick, sort_setup, place x3, relabel
+    }
+    {
+        ProfScope ps(ctx, PH_SAMPLE_FINAL, 1);
+        k_finalize<<<1, 1024, 0, st>>>(d->hdr, B, k, d->cum, d->node_off, d->ent_off, d->rowbase, d->d_ent_hop);
+        ctx->launches++;
+    }
+    MG_CUDA(ctx, cudaGetLastError());
+
+    // read the summary back (the one host sync of a sample)
+    d->h_cum.resize((size_t)B * (k + 2));
+    d->h_node_off.resize((size_t)(k + 1) * (B + 1));
+    d->h_rowbase.resize((size_t)(k + 1) * (B + 1));
+    d->h_ent_hop.resize((size_t)k * (B + 1));
+    MG_CUDA(ctx, cudaMemcpyAsync(&d->h_hdr, d->hdr, sizeof(DenseHeader), cudaMemcpyDeviceToHost, st));
+    MG_CUDA(ctx, cudaMemcpyAsync(d->h_cum.data(), d->cum, sizeof(int32_t) * d->h_cum.size(), cudaMemcpyDeviceToHost, st));
+    MG_CUDA(ctx, cudaMemcpyAsync(d->h_node_off.data(), d->node_off, sizeof(int32_t) * d->h_node_off.size(), cudaMemcpyDeviceToHost, st));
+    MG_CUDA(ctx, cudaMemcpyAsync(d->h_rowbase.data(), d->rowbase, sizeof(int32_t) * d->h_rowbase.size(), cudaMemcpyDeviceToHost, st));
+    MG_CUDA(ctx, cudaMemcpyAsync(d->h_ent_hop.data(), d->d_ent_hop, sizeof(int32_t) * d->h_ent_hop.size(), cudaMemcpyDeviceToHost, st));
+    MG_CUDA(ctx, cudaStreamSynchronize(st));
+    if (d->h_hdr.status) return mg_fail(ctx, status_code(d->h_hdr.status), "%s", status_text(d->h_hdr.status));
+    d->valid = true;
+    return MG_OK;
+}
+
+extern "C" int mg_sample(mg_ctx* ctx, const int32_t* targets, int targets_on_device, int32_t n_targets,
+                         const int32_t* fanouts, int32_t k, uint64_t seed, const mg_sample_caps* caps, mg_dense** out) {
+    if (!ctx) return MG_ERR_ARG;
+    if (n_targets < 0) return mg_fail(ctx, MG_ERR_ARG, "negative n_targets");
+    const int64_t off[2] = {0, n_targets};
+    return mg_sample_many(ctx, targets, targets_on_device, off, 1, fanouts, k, &seed, caps, out);
+}
+
+extern "C" int mg_dense_counts(const mg_dense* d, int32_t* n_batches, int32_t* k, int64_t* nodes_per_hop,
+                               int64_t* entries_per_hop) {
+    if (!d) return MG_ERR_ARG;
+    if (!d->valid) return MG_ERR_STATE;
+    const int B = d->n_batches, K = d->k;
+    if (n_batches) *n_batches = B;
+    if (k) *k = K;
+    if (nodes_per_hop)
+        for (int b = 0; b < B; ++b)
+            for (int h = 0; h <= K; ++h)
+                nodes_per_hop[(size_t)b * (K + 1) + h] = d->h_cum[(size_t)b * (K + 2) + h + 1] - d->h_cum[(size_t)b * (K + 2) + h];
+    if (entries_per_hop)
+        for (int b = 0; b < B; ++b)
+            for (int h = 0; h < K; ++h)
+                entries_per_hop[(size_t)b * K + h] = d->h_ent_hop[(size_t)h * (B + 1) + b + 1] - d->h_ent_hop[(size_t)h * (B + 1) + b];
+    return MG_OK;
+}
+
+extern "C" int mg_dense_view(mg_ctx* ctx, mg_dense* d, int32_t batch, mg_dense_arrays* out) {
+    if (!ctx) return MG_ERR_ARG;
+    if (!d || !out) return mg_fail(ctx, MG_ERR_ARG, "null argument");
+    if (!d->valid) return mg_fail(ctx, MG_ERR_STATE, "mg_dense holds no completed sample");
+    if (batch < 0 || batch >= d->n_batches) return mg_fail(ctx, MG_ERR_ARG, "batch out of range");
+    MG_CUDA(ctx, cudaSetDevice(ctx->device));
+    const int k = d->k, B = d->n_batches, b = batch;
+    ExportArgs a;
+    memset(&a, 0, sizeof(a));
+    a.k = k; a.b = b; a.B = B;
+    for (int h = 0; h <= k + 1; ++h) a.cum[h] = d->h_cum[(size_t)b * (k + 2) + h];
+    a.V = a.cum[k + 1];
+    // canonical Delta_j = hop k - j
+    a.nio[0] = 0;
+    for (int j = 0; j <= k; ++j) a.nio[j + 1] = a.nio[j] + (a.cum[k - j + 1] - a.cum[k - j]);
+    a.n0 = a.nio[1];
+    for (int h = 0; h <= k; ++h) a.node_off[h] = d->h_node_off[(size_t)h * (B + 1) + b];
+    int32_t e_run = 0;
+    for (int j = 1; j <= k; ++j) {
+        const int h = k - j;
+        a.ebase[j] = e_run;
+        a.ent_hop[h] = d->h_ent_hop[(size_t)h * (B + 1) + b];
+        e_run += d->h_ent_hop[(size_t)h * (B + 1) + b + 1] - a.ent_hop[h];
+    }
+    a.E = e_run;
+    const int32_t n_s = a.V - a.n0;
+    const size_t need = (size_t)a.V + (k + 2) + 2 * (size_t)a.E + (size_t)n_s + 1 + 16;
+    int rc = mg_ensure(ctx, &d->exp_buf, &d->exp_elems, need);
+    if (rc) return rc;
+    a.nodes = d->nodes; a.ent_off = d->ent_off; a.ent_nbrs = d->ent_nbrs; a.ent_repr = d->ent_repr;
+    a.o_node_ids = d->exp_buf;
+    a.o_nio = a.o_node_ids + a.V;
+    a.o_nbrs = a.o_nio + (k + 2);
+    a.o_nbr_off = a.o_nbrs + a.E;
+    a.o_repr = a.o_nbr_off + n_s + 1;
+    const int grid = std::max(1, std::min(mg_grid(ctx, 4), (a.V + kThreads - 1) / kThreads));
+    k_export<<<grid, kThreads, 0, ctx->stream>>>(a);
+    ctx->launches++;
+    MG_CUDA(ctx, cudaGetLastError());
+    MG_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    out->k = k;
+    out->n_nodes = a.V;
+    out->n_sampled = n_s;
+    out->n_entries = a.E;
+    out->node_ids = a.o_node_ids;
+    out->node_id_offsets = a.o_nio;
+    out->nbrs = a.o_nbrs;
+    out->nbr_offsets = a.o_nbr_off;
+    out->repr_map = a.o_repr;
+    return MG_OK;
+}
+
+extern "C" int mg_dense_free(mg_dense* d) {
+    if (!d) return MG_OK;
+    if (d->ctx) cudaSetDevice(d->ctx->device);
+    cudaFree(d->hdr); cudaFree(d->nodes); cudaFree(d->node_batch); cudaFree(d->ent_off);
+    cudaFree(d->ent_nbrs); cudaFree(d->ent_repr); cudaFree(d->node_off); cudaFree(d->cum);
+    cudaFree(d->rowbase); cudaFree(d->hkeys); cudaFree(d->hvals); cudaFree(d->newlist[0]);
+    cudaFree(d->newlist[1]); cudaFree(d->d_seeds); cudaFree(d->scan_tmp); cudaFree(d->sort_hist);
+    cudaFree(d->exp_buf); cudaFree(d->d_ent_hop);
+    delete d;
+    return MG_OK;
+}

@@ -1,0 +1,257 @@
+"""GPU parity: the CUDA path through the C ABI against the CPU oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2202_02365_b200 as mg
+from oracle import dense_oracle as O
+from paper_2202_02365_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+RTOL_AGG = 1e-5     # fp32 aggregation / fp32 GEMM outputs
+RTOL_TC = 5e-3      # TF32 tensor-core GEMM outputs
+
+
+def close(got, ref, rtol):
+    """|got - ref| <= rtol * max(|ref|, rms(ref)) element-wise."""
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    assert got.shape == ref.shape
+    if ref.size == 0:
+        return
+    rms = np.sqrt(np.mean(ref ** 2))
+    bound = rtol * np.maximum(np.abs(ref), rms)
+    err = np.abs(got - ref)
+    worst = np.max(err / np.maximum(bound, 1e-300))
+    assert worst <= 1.0, f"worst error {worst:.3f} x the bound (rtol {rtol})"
+
+
+def oracle_view(graph, n_parts=1, resident=None):
+    return O.GraphView(graph.row_offsets.cpu().numpy(), graph.nbrs.cpu().numpy(), n_parts, resident)
+
+
+def assert_dense_equal(view, ref):
+    for key in ("node_ids", "node_id_offsets", "nbrs", "nbr_offsets", "repr_map"):
+        got = getattr(view, key).cpu().numpy().tolist()
+        assert got == ref[key], f"{key} differs"
+
+
+def make_ctx(graph, feats=None, offsets_dtype=torch.int64):
+    ctx = mg.Context(0)
+    ctx.load_graph(graph.row_offsets.to(offsets_dtype).cuda(), graph.nbrs.cuda())
+    if feats is not None:
+        ctx.load_features(feats.cuda())
+    return ctx
+
+
+@pytest.fixture(scope="module")
+def tiny():
+    g = inputs.erdos_renyi_graph(10_000, 200_000, seed=0)
+    feats = inputs.normal_features(10_000, 16, seed=1)
+    return g, feats
+
+
+def test_config1_sample_bit_exact(tiny):
+    g, feats = tiny
+    ctx = make_ctx(g, feats, torch.int32)
+    targets = inputs.distinct_targets(10_000, 512, seed=2)
+    d = ctx.sample(targets, [10, 5], seed=123)
+    ref = O.sample_dense(oracle_view(g), targets.tolist(), [10, 5], 123)
+    assert_dense_equal(d.view(0), ref)
+    nodes, ents = d.counts()
+    nio = ref["node_id_offsets"]
+    assert nodes[0].tolist() == [nio[3] - nio[2], nio[2] - nio[1], nio[1] - nio[0]]
+    assert int(ents.sum()) == len(ref["nbrs"])
+
+
+def test_config1_forward(tiny):
+    g, feats = tiny
+    ctx = make_ctx(g, feats)
+    targets = inputs.distinct_targets(10_000, 512, seed=3)
+    layers = inputs.random_bias_layers([16, 16, 16], seed=4)
+    d = ctx.sample(targets, [10, 5], seed=7)
+    ref = O.sample_dense(oracle_view(g), targets.tolist(), [10, 5], 7)
+    h0 = feats.numpy()[ref["node_ids"]]
+    got_h0 = ctx.gather_h0(d, 0, len(ref["node_ids"]), 16).cpu().numpy()
+    np.testing.assert_array_equal(got_h0, h0)
+    ref_outs = O.forward(ref, h0, [(w.numpy(), n.numpy(), b.numpy()) for w, n, b in layers], return_all=True)
+    for prec, rtol in ((mg.GEMM_FP32, RTOL_AGG), (mg.GEMM_TF32, RTOL_TC)):
+        model = ctx.model(layers, prec)
+        out = torch.empty((512, 16), dtype=torch.float32, device="cuda")
+        ctx.forward(model, d, out)
+        close(out.cpu().numpy(), ref_outs[-1], rtol)
+        l1 = ctx.layer_output(model, d, 1, 0, ref_outs[0].shape[0]).cpu().numpy()
+        close(l1, ref_outs[0], rtol)
+        host_out = torch.empty((512, 16), dtype=torch.float32)
+        ctx.forward(model, d, host_out)
+        np.testing.assert_array_equal(host_out.numpy(), out.cpu().numpy())
+
+
+def test_many_batches_match_single_and_oracle(tiny):
+    g, feats = tiny
+    ctx = make_ctx(g, feats)
+    B, T = 7, 200
+    sizes = [T, 0, 13, T, 1, 300, 64]
+    tg = [inputs.distinct_targets(10_000, s, seed=10 + i) for i, s in enumerate(sizes)]
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    seeds = [1000 + 17 * i for i in range(B)]
+    d = ctx.sample_many(torch.cat(tg), offs, [4, 3, 2], seeds)
+    view = oracle_view(g)
+    layers = inputs.random_bias_layers([16, 8, 8, 4], seed=5)
+    model = ctx.model(layers, mg.GEMM_FP32)
+    out = torch.empty((int(offs[-1]), 4), dtype=torch.float32, device="cuda")
+    ctx.forward(model, d, out)
+    for b in range(B):
+        ref = O.sample_dense(view, tg[b].tolist(), [4, 3, 2], seeds[b])
+        assert_dense_equal(d.view(b), ref)
+        if sizes[b]:
+            ref_out = O.forward(ref, feats.numpy()[ref["node_ids"]], [(w.numpy(), n.numpy(), bb.numpy()) for w, n, bb in layers])
+            close(out[offs[b]:offs[b + 1]].cpu().numpy(), ref_out, RTOL_AGG)
+    # device-resident targets give the same sample; so does reusing the handle
+    d2 = ctx.sample_many(torch.cat(tg).cuda(), offs, [4, 3, 2], seeds, out=d)
+    assert d2 is d
+    assert_dense_equal(d.view(3), O.sample_dense(view, tg[3].tolist(), [4, 3, 2], seeds[3]))
+
+
+@pytest.mark.parametrize("fanouts", [[1], [3, 1], [33, 2], [40, 70]])
+def test_odd_fanouts(fanouts):
+    g = inputs.rmat_graph(3000, 60_000, seed=3)
+    ctx = make_ctx(g)
+    targets = inputs.distinct_targets(3000, 50, seed=1)
+    d = ctx.sample(targets, fanouts, seed=99)
+    assert_dense_equal(d.view(0), O.sample_dense(oracle_view(g), targets.tolist(), fanouts, 99))
+
+
+def test_full_fanout_is_exact_neighbourhood():
+    g = inputs.erdos_renyi_graph(500, 3000, seed=8)
+    ctx = make_ctx(g)
+    maxdeg = int((g.row_offsets[1:] - g.row_offsets[:-1]).max())
+    targets = torch.tensor([4, 99, 250], dtype=torch.int32)
+    d = ctx.sample(targets, [maxdeg, maxdeg], seed=0)
+    assert_dense_equal(d.view(0), O.sample_dense(oracle_view(g), targets.tolist(), [maxdeg, maxdeg], 0))
+
+
+def test_run_to_run_determinism(tiny):
+    g, _ = tiny
+    ctx = make_ctx(g)
+    targets = inputs.distinct_targets(10_000, 512, seed=5)
+    a = ctx.sample(targets, [10, 5], seed=1).view(0)
+    b = ctx.sample(targets, [10, 5], seed=1).view(0)
+    for key in ("node_ids", "nbrs", "nbr_offsets", "repr_map"):
+        assert torch.equal(getattr(a, key), getattr(b, key))
+    c = ctx.sample(targets, [10, 5], seed=2).view(0)
+    assert not torch.equal(a.nbrs, c.nbrs) or a.nbrs.numel() != c.nbrs.numel()
+
+
+def test_errors(tiny):
+    g, feats = tiny
+    ctx = make_ctx(g, feats)
+    t = torch.tensor([1, 2, 3], dtype=torch.int32)
+    with pytest.raises(mg.MgError) as e:
+        ctx.sample(torch.tensor([1, 2, 1], dtype=torch.int32), [2], 0)
+    assert e.value.code == -4
+    with pytest.raises(mg.MgError) as e:
+        ctx.sample(torch.tensor([1, 10_000], dtype=torch.int32), [2], 0)
+    assert e.value.code == -1
+    with pytest.raises(mg.MgError) as e:
+        ctx.sample(t, [0], 0)
+    assert e.value.code == -1
+    with pytest.raises(mg.MgError) as e:
+        ctx.sample(t, [5, 5], 0, caps={"max_entries_total": 4})
+    assert e.value.code == -5
+    with pytest.raises(mg.MgError) as e:
+        ctx.sample(inputs.distinct_targets(10_000, 100, 0), [10, 10], 0, caps={"max_nodes_total": 150})
+    assert e.value.code == -5
+    # the context stays usable after every failure
+    d = ctx.sample(t, [2], 0)
+    assert d.view(0).node_ids.numel() >= 3
+    empty = mg.Context(0)
+    with pytest.raises(mg.MgError) as e:
+        empty.sample(t, [2], 0)
+    assert e.value.code == -2
+    # a model whose depth differs from the sample
+    model = ctx.model(inputs.glorot_layers([16, 16, 16], 0), mg.GEMM_FP32)
+    with pytest.raises(mg.MgError) as e:
+        ctx.forward(model, d, torch.empty((3, 16), device="cuda"))
+    assert e.value.code == -2
+
+
+def test_partition_buffer_filter_and_host_backing():
+    n, parts, cap = 6000, 6, 3
+    g = inputs.rmat_graph(n, 90_000, seed=4)
+    feats16 = inputs.normal_features(n, 24, seed=2, dtype=torch.float16, pin=False).pin_memory()
+    ctx = mg.Context(0)
+    ctx.load_graph(g.row_offsets.cuda(), g.nbrs.cuda())
+    ctx.set_partitioning(parts)
+    ctx.load_features(feats16, capacity_parts=cap, backing=mg.BACKING_HOST)
+    layers = inputs.random_bias_layers([24, 8, 8], seed=6)
+    model = ctx.model(layers, mg.GEMM_FP32)
+    states = inputs.swap_order(parts, cap, seed=1)
+    assert len(states) == parts - cap + 1
+    for step, resident in enumerate(states):
+        ctx.set_resident(resident, async_=True)
+        ctx.commit_resident(10_000)
+        mask = inputs.resident_node_mask(n, parts, resident)
+        pool = torch.nonzero(mask).flatten()
+        targets = inputs.distinct_targets(pool, 64, seed=step)
+        d = ctx.sample(targets, [5, 3], seed=50 + step)
+        view = oracle_view(g, parts, resident)
+        ref = O.sample_dense(view, targets.tolist(), [5, 3], 50 + step)
+        assert_dense_equal(d.view(0), ref)
+        assert all(view.is_resident(u) for u in ref["node_ids"])
+        out = torch.empty((64, 8), dtype=torch.float32, device="cuda")
+        ctx.forward(model, d, out)
+        h0 = feats16.float().numpy()[ref["node_ids"]]
+        np.testing.assert_array_equal(ctx.gather_h0(d, 0, len(ref["node_ids"]), 24).cpu().numpy(), h0)
+        ref_out = O.forward(ref, h0, [(w.numpy(), nn.numpy(), b.numpy()) for w, nn, b in layers])
+        close(out.cpu().numpy(), ref_out, RTOL_AGG)
+    # a target outside the buffer is refused
+    outside = int(torch.nonzero(~inputs.resident_node_mask(n, parts, states[-1])).flatten()[0])
+    with pytest.raises(mg.MgError) as e:
+        ctx.sample(torch.tensor([outside], dtype=torch.int32), [2], 0)
+    assert e.value.code == -3
+    with pytest.raises(mg.MgError) as e:
+        ctx.set_resident([0, 1, 2, 3])
+    assert e.value.code == -5
+
+
+def test_link_prediction_distmult():
+    n, parts, cap = 8000, 4, 2
+    g = inputs.rmat_graph(n, 100_000, seed=5, n_relations=37)
+    emb = inputs.normal_features(n, 20, seed=3, std=0.001)
+    rel_emb = inputs.normal_features(37, 12, seed=9)
+    ctx = mg.Context(0)
+    ctx.load_graph(g.row_offsets.cuda(), g.nbrs.cuda())
+    ctx.set_partitioning(parts)
+    ctx.load_features(emb.cuda(), capacity_parts=cap)
+    resident = [1, 3]
+    ctx.set_resident(resident)
+    mask = inputs.resident_node_mask(n, parts, resident)
+    src, rel, dst = inputs.lp_edges(g, mask, 500, seed=1)
+    n_chunks, negs = 3, 70
+    lp = ctx.lp_prepare(src, rel, dst, n_chunks, negs, seed=2024)
+    view = oracle_view(g, parts, resident)
+    prep = O.lp_prepare(view, src.tolist(), dst.tolist(), n_chunks, negs, 2024)
+    got = lp.view()
+    assert got["targets"].cpu().tolist() == prep["targets"]
+    assert got["src_idx"].cpu().tolist() == prep["src_idx"]
+    assert got["dst_idx"].cpu().tolist() == prep["dst_idx"]
+    assert got["neg_ids"].cpu().tolist() == prep["neg_ids"]
+    assert got["neg_idx"].cpu().tolist() == prep["neg_idx"]
+    # one GraphSage layer over the targets, then DistMult
+    layers = inputs.random_bias_layers([20, 12], seed=8)
+    model = ctx.model(layers, mg.GEMM_FP32)
+    d = ctx.sample(got["targets"], [20], seed=5)
+    ref = O.sample_dense(view, prep["targets"], [20], 5)
+    assert_dense_equal(d.view(0), ref)
+    h = torch.empty((len(prep["targets"]), 12), dtype=torch.float32, device="cuda")
+    ctx.forward(model, d, h)
+    ref_h = O.forward(ref, emb.numpy()[ref["node_ids"]], [(w.numpy(), nn.numpy(), b.numpy()) for w, nn, b in layers])
+    close(h.cpu().numpy(), ref_h, RTOL_AGG)
+    pos, nd, ns = ctx.distmult_score(lp, h, rel_emb.cuda())
+    torch.cuda.synchronize()
+    rpos, rnd, rns = O.distmult_scores(ref_h, rel_emb.numpy(), prep, rel.tolist(), n_chunks)
+    close(pos.cpu().numpy(), rpos, RTOL_AGG)
+    close(nd.cpu().numpy(), rnd, RTOL_AGG)
+    close(ns.cpu().numpy(), rns, RTOL_AGG)
