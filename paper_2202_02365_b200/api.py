@@ -8,6 +8,7 @@ from __future__ import annotations
 
 import ctypes as C
 import os
+import weakref
 from dataclasses import dataclass
 
 import numpy as np
@@ -80,7 +81,7 @@ class _DeviceInts:
     """A library-owned device buffer of n int32 values, exposed through the CUDA array interface."""
 
     def __init__(self, ptr: int, n: int):
-        self.__cuda_array_interface__ = {"shape": (n,), "typestr": "<i4", "data": (int(ptr), True), "version": 2}
+        self.__cuda_array_interface__ = {"shape": (n,), "typestr": "<i4", "data": (int(ptr), False), "version": 2}
 
 
 def _from_dev(ptr, n: int, device) -> torch.Tensor:
@@ -104,6 +105,7 @@ class Dense:
     def __init__(self, ctx: "Context"):
         self.ctx = ctx
         self.handle = C.c_void_p(0)
+        ctx._children.add(self)
 
     def counts(self):
         lib = self.ctx.lib
@@ -139,6 +141,7 @@ class Model:
     def __init__(self, ctx: "Context", layers, precision: int = GEMM_TF32):
         self.ctx = ctx
         self.handle = C.c_void_p(0)
+        ctx._children.add(self)
         k = len(layers)
         self.dims = [int(layers[0][0].shape[0])] + [int(l[0].shape[1]) for l in layers]
         keep = []
@@ -170,6 +173,7 @@ class LpBatch:
     def __init__(self, ctx: "Context"):
         self.ctx = ctx
         self.handle = C.c_void_p(0)
+        ctx._children.add(self)
         self.n_edges = 0
         self.negs = 0
 
@@ -208,6 +212,7 @@ class Context:
         self.device = torch.device("cuda", device)
         self.stream = stream
         self.handle = C.c_void_p(0)
+        self._children = weakref.WeakSet()
         sptr = C.c_void_p(stream.cuda_stream if stream is not None else 0)
         rc = self.lib.mg_create(C.byref(self.handle), C.c_int(device), sptr)
         if rc != MG_OK:
@@ -222,6 +227,8 @@ class Context:
 
     def close(self):
         if self.handle:
+            for child in list(self._children):
+                child.free()
             self.lib.mg_destroy(self.handle)
             self.handle = C.c_void_p(0)
 

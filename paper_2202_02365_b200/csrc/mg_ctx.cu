@@ -218,7 +218,9 @@ extern "C" int mg_create(mg_ctx** out, int device, void* stream) {
     for (int i = 0; i < PH_COUNT; ++i) c->prof[i] = ProfPhase{kPhaseNames[i], 0.0, 0};
     if (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
         cudaMalloc((void**)&c->d_slot_of_part, sizeof(int32_t) * MG_MAX_PARTS) != cudaSuccess ||
-        cudaMalloc((void**)&c->d_res_prefix, sizeof(int64_t) * (MG_MAX_PARTS + 1)) != cudaSuccess) {
+        cudaMalloc((void**)&c->d_res_prefix, sizeof(int64_t) * (MG_MAX_PARTS + 1)) != cudaSuccess ||
+        cudaMalloc((void**)&c->d_flags, sizeof(uint32_t)) != cudaSuccess ||
+        cudaMemset(c->d_flags, 0, sizeof(uint32_t)) != cudaSuccess) {
         cudaGetLastError();
         delete c;
         return MG_ERR_CUDA;
@@ -246,7 +248,7 @@ extern "C" int mg_destroy(mg_ctx* c) {
     for (auto& p : c->prof_pending) { cudaEventDestroy(p.second.first); cudaEventDestroy(p.second.second); }
     free_view(c);
     free_features(c);
-    cudaFree(c->row_off); cudaFree(c->nbrs); cudaFree(c->d_slot_of_part); cudaFree(c->d_res_prefix);
+    cudaFree(c->row_off); cudaFree(c->nbrs); cudaFree(c->d_slot_of_part); cudaFree(c->d_res_prefix); cudaFree(c->d_flags);
     cudaFree(c->ws_x); cudaFree(c->ws_h[0]); cudaFree(c->ws_h[1]);
     cudaStreamDestroy(c->side);
     delete c;

@@ -15,6 +15,7 @@
 
 int mg_gemm_tf32(mg_ctx* ctx, const float* x, const float* w_t, const float* bias, float* out, int64_t M, int N, int K,
                  bool relu);  // mg_gemm_tcgen05.cu
+int mg_gemm_tf32_status(mg_ctx* ctx);
 
 namespace {
 
@@ -318,6 +319,7 @@ extern "C" int mg_model_create(mg_ctx* ctx, int32_t k, const int32_t* dims, cons
     MG_CUDA(ctx, cudaSetDevice(ctx->device));
     mg_model* m = new mg_model();
     m->ctx = ctx;
+    m->device = ctx->device;
     m->k = k;
     m->precision = gemm_precision;
     for (int l = 0; l <= k; ++l) m->dims[l] = dims[l];
@@ -347,7 +349,7 @@ extern "C" int mg_model_create(mg_ctx* ctx, int32_t k, const int32_t* dims, cons
 
 extern "C" int mg_model_free(mg_model* m) {
     if (!m) return MG_OK;
-    if (m->ctx) cudaSetDevice(m->ctx->device);
+    cudaSetDevice(m->device);
     for (int l = 0; l < MG_MAX_HOPS; ++l) { cudaFree(m->w_cat[l]); cudaFree(m->w_cat_t[l]); cudaFree(m->bias[l]); }
     delete m;
     return MG_OK;
@@ -452,6 +454,7 @@ extern "C" int mg_forward(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* ou
     const size_t out_bytes = (size_t)d->h_hdr.rows_total[k] * m->dims[k] * sizeof(float);
     MG_CUDA(ctx, cudaMemcpyAsync(out, ctx->ws_h[0] + off[k], out_bytes, out_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, st));
     MG_CUDA(ctx, cudaStreamSynchronize(st));
+    if (m->precision == MG_GEMM_TF32) return mg_gemm_tf32_status(ctx);
     return MG_OK;
 }
 

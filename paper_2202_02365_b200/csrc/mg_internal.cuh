@@ -63,6 +63,7 @@ struct mg_ctx {
     std::string err;
     int64_t launches = 0;
     int n_sms = 148;
+    uint32_t* d_flags = nullptr;  // device word the tensor-core GEMM reports a barrier time-out in
 
     // graph store (device)
     int64_t n_nodes = 0, n_edges = 0;
@@ -110,6 +111,7 @@ struct mg_ctx {
 
 struct mg_dense {
     mg_ctx* ctx = nullptr;
+    int device = 0;
     int32_t k = 0, n_batches = 0;
     int32_t fanouts[MG_MAX_HOPS] = {0};
     int64_t cap_nodes = 0, cap_entries = 0;
@@ -151,6 +153,7 @@ struct mg_dense {
 
 struct mg_model {
     mg_ctx* ctx = nullptr;
+    int device = 0;
     int32_t k = 0;
     int32_t dims[MG_MAX_HOPS + 1] = {0};
     int precision = MG_GEMM_TF32;
@@ -161,6 +164,7 @@ struct mg_model {
 
 struct mg_lp_batch {
     mg_ctx* ctx = nullptr;
+    int device = 0;
     int64_t n_edges = 0;
     int32_t n_chunks = 0, negs = 0, n_targets = 0;
     int32_t* targets = nullptr;  // device

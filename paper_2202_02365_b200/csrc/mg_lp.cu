@@ -157,7 +157,7 @@ __global__ void __launch_bounds__(256) k_distmult_neg(NegArgs a) {
 
 extern "C" int mg_lp_free(mg_lp_batch* lp) {
     if (!lp) return MG_OK;
-    if (lp->ctx) cudaSetDevice(lp->ctx->device);
+    cudaSetDevice(lp->device);
     cudaFree(lp->targets); cudaFree(lp->src_idx); cudaFree(lp->dst_idx); cudaFree(lp->rel);
     cudaFree(lp->neg_ids); cudaFree(lp->neg_idx);
     delete lp;
@@ -176,7 +176,7 @@ extern "C" int mg_lp_prepare(mg_ctx* ctx, const int32_t* src, const int32_t* rel
     MG_CUDA(ctx, cudaSetDevice(ctx->device));
     cudaStream_t st = ctx->stream;
     mg_lp_batch* lp = new mg_lp_batch();
-    lp->ctx = ctx; lp->n_edges = n_edges; lp->n_chunks = n_chunks; lp->negs = negs;
+    lp->ctx = ctx; lp->device = ctx->device; lp->n_edges = n_edges; lp->n_chunks = n_chunks; lp->negs = negs;
 
     int32_t *d_src = nullptr, *d_dst = nullptr, *d_nt = nullptr;
     uint64_t* keys[2] = {nullptr, nullptr};

@@ -761,7 +761,7 @@ extern "C" int mg_sample_many(mg_ctx* ctx, const int32_t* targets, int targets_o
 
     mg_dense* d = *out;
     const bool created = (d == nullptr);
-    if (created) { d = new mg_dense(); d->ctx = ctx; }
+    if (created) { d = new mg_dense(); d->ctx = ctx; d->device = ctx->device; }
     else if (d->ctx != ctx) return mg_fail(ctx, MG_ERR_ARG, "mg_dense belongs to another context");
     d->valid = false;
     int rc = dense_alloc(ctx, d, n_batches, k, cap_nodes, std::max<int64_t>(cap_entries, 1), table_size);
@@ -953,7 +953,7 @@ extern "C" int mg_dense_view(mg_ctx* ctx, mg_dense* d, int32_t batch, mg_dense_a
 
 extern "C" int mg_dense_free(mg_dense* d) {
     if (!d) return MG_OK;
-    if (d->ctx) cudaSetDevice(d->ctx->device);
+    cudaSetDevice(d->device);
     cudaFree(d->hdr); cudaFree(d->nodes); cudaFree(d->node_batch); cudaFree(d->ent_off);
     cudaFree(d->ent_nbrs); cudaFree(d->ent_repr); cudaFree(d->node_off); cudaFree(d->cum);
     cudaFree(d->rowbase); cudaFree(d->hkeys); cudaFree(d->hvals); cudaFree(d->newlist[0]);

@@ -255,3 +255,51 @@ def test_link_prediction_distmult():
     close(pos.cpu().numpy(), rpos, RTOL_AGG)
     close(nd.cpu().numpy(), rnd, RTOL_AGG)
     close(ns.cpu().numpy(), rns, RTOL_AGG)
+
+
+@pytest.mark.parametrize("d_in,d_out", [(100, 100), (256, 256), (128, 256), (768, 256), (16, 520), (36, 4)])
+def test_tensor_core_linear_layer_shapes(d_in, d_out):
+    """One GraphSage layer at the widths of the five configurations (and ragged ones): several
+    K slices, ring wrap-around, padded N tiles, more than one N tile, a ragged last row tile."""
+    n = 5000
+    g = inputs.rmat_graph(n, 60_000, seed=11)
+    feats = inputs.normal_features(n, d_in, seed=12)
+    ctx = make_ctx(g, feats)
+    targets = inputs.distinct_targets(n, 777, seed=13)
+    d = ctx.sample(targets, [6], seed=3)
+    ref = O.sample_dense(oracle_view(g), targets.tolist(), [6], 3)
+    assert_dense_equal(d.view(0), ref)
+    layers = inputs.random_bias_layers([d_in, d_out], seed=14)
+    want = O.forward(ref, feats.numpy()[ref["node_ids"]], [(w.numpy(), nn.numpy(), b.numpy()) for w, nn, b in layers])
+    for prec, rtol in ((mg.GEMM_TF32, RTOL_TC), (mg.GEMM_FP32, RTOL_AGG)):
+        out = torch.empty((777, d_out), dtype=torch.float32, device="cuda")
+        ctx.forward(ctx.model(layers, prec), d, out)
+        close(out.cpu().numpy(), want, rtol)
+
+
+def test_config2_shaped_power_law_three_layers():
+    """R-MAT, dim 128, hidden 256, fanouts [15, 10, 5], batches of 1000 (config 2 at 1/5 scale so
+    the oracle finishes in seconds); hub rows, zero-degree nodes, several batches per pass."""
+    n = 200_000
+    g = inputs.rmat_graph(n, 4_000_000, seed=21)
+    feats = inputs.normal_features(n, 128, seed=22)
+    ctx = make_ctx(g, feats)
+    B = 4
+    tg = inputs.train_set_batches(n, 20_000, 1000, B, seed=23)
+    offs = [1000 * i for i in range(B + 1)]
+    seeds = [7 + i for i in range(B)]
+    d = ctx.sample_many(tg.flatten(), offs, [15, 10, 5], seeds)
+    layers = inputs.glorot_layers([128, 256, 256, 256], seed=24)
+    model = ctx.model(layers, mg.GEMM_TF32)
+    out = torch.empty((B * 1000, 256), dtype=torch.float32, device="cuda")
+    ctx.forward(model, d, out)
+    view = oracle_view(g)
+    for b in (0, B - 1):
+        ref = O.sample_dense(view, tg[b].tolist(), [15, 10, 5], seeds[b])
+        assert_dense_equal(d.view(b), ref)
+        outs = O.forward(ref, feats.numpy()[ref["node_ids"]], [(w.numpy(), nn.numpy(), bb.numpy()) for w, nn, bb in layers],
+                         return_all=True)
+        close(out[b * 1000:(b + 1) * 1000].cpu().numpy(), outs[-1], RTOL_TC)
+        for layer in (1, 2):
+            got = ctx.layer_output(model, d, layer, b, outs[layer - 1].shape[0]).cpu().numpy()
+            close(got, outs[layer - 1], RTOL_TC)
