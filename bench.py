@@ -1,0 +1,378 @@
+#!/usr/bin/env python
+"""Benchmark of the DENSE sample + GraphSage forward hot path on synthetic paper-shaped graphs.
+
+One step = one pass of the whole path (k-hop DENSE sampling, relabelling, feature gather +
+segment-mean, linear layers) over one group of independent mini-batches through the C ABI.
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2202_02365_b200 import inputs  # noqa: E402
+
+CONFIGS = {
+    # name: nodes, edges, graph kind, feature dim, hidden, fanouts, targets per mini-batch, partitions
+    "config1_er_10k": dict(n=10_000, m=200_000, kind="er", dim=16, hidden=16, fanouts=[10, 5], batch=512, parts=1,
+                           train=10_000),
+    "config2_rmat_1m": dict(n=1_000_000, m=20_000_000, kind="rmat", dim=128, hidden=256, fanouts=[15, 10, 5],
+                            batch=1000, parts=1, train=1_000_000),
+    "config3_papers100m_shaped": dict(n=111_000_000, m=1_620_000_000, kind="rmat", dim=128, hidden=256,
+                                      fanouts=[15, 10, 5], batch=1000, parts=16, train=1_100_000),
+}
+DEFAULT_WORKLOAD = "config3_papers100m_shaped"
+HBM_NOMINAL_GBS = 8000.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def build_workload(cfg, device, seed=0):
+    t0 = time.time()
+    if cfg["kind"] == "er":
+        g = inputs.erdos_renyi_graph(cfg["n"], cfg["m"], seed, device)
+    else:
+        g = inputs.rmat_graph(cfg["n"], cfg["m"], seed, device)
+    torch.cuda.synchronize()
+    t1 = time.time()
+    feats = inputs.normal_features(cfg["n"], cfg["dim"], seed + 1, device)
+    torch.cuda.synchronize()
+    dims = [cfg["dim"]] + [cfg["hidden"]] * len(cfg["fanouts"])
+    layers = inputs.glorot_layers(dims, seed + 2)
+    return g, feats, layers, {"graph_s": round(t1 - t0, 1), "features_s": round(time.time() - t1, 1)}
+
+
+def algorithmic_bytes(nodes, ents, cfg, feat_bytes=4):
+    """Bytes the method must move for the sampled batches (per-unit figures of the scope table):
+    sampling 12 E_s + 20 n_s + 4 V, features V d0 s, aggregation indices sum_l 4 (E_l + N_l),
+    output n_k d_k 4.  nodes: [B, k+1] (hop 0 = targets), ents: [B, k]."""
+    k = ents.shape[1]
+    V = nodes.sum()
+    n_s = nodes[:, :k].sum()
+    E_s = ents.sum()
+    a_s = 12 * E_s + 20 * n_s + 4 * V
+    a_f = V * cfg["dim"] * feat_bytes
+    a_i = 0
+    for l in range(1, k + 1):                       # layer l aggregates hops 0 .. k-l
+        a_i += 4 * (ents[:, :k - l + 1].sum() + nodes[:, :k - l + 1].sum())
+    a_o = nodes[:, 0].sum() * cfg["hidden"] * 4
+    flops = 0
+    dims = [cfg["dim"]] + [cfg["hidden"]] * k
+    for l in range(1, k + 1):
+        flops += 2 * nodes[:, :k - l + 1].sum() * 2 * dims[l - 1] * dims[l]
+    agg_l1 = a_f + 4 * (ents.sum() + nodes[:, :k].sum())
+    return {"sampling": int(a_s), "features": int(a_f), "agg_index": int(a_i), "output": int(a_o),
+            "a_min": int(a_s + a_f + a_i + a_o), "flops": int(flops), "agg_l1": int(agg_l1)}
+
+
+def oracle_time(g_host, feats, layers, cfg, target_rows, seeds, budget_s=20.0):
+    """The CPU oracle as it stands on a bounded sample of the same mini-batches."""
+    from oracle import dense_oracle as O
+    view = O.GraphView(g_host[0], g_host[1])
+    np_layers = [(w.numpy(), n.numpy(), b.numpy()) for w, n, b in layers]
+    done, edges, t0 = 0, 0, time.time()
+    for tg, seed in zip(target_rows, seeds):
+        ref = O.sample_dense(view, tg.tolist(), cfg["fanouts"], int(seed))
+        ids = torch.as_tensor(ref["node_ids"], dtype=torch.int64)
+        h0 = feats[ids.to(feats.device)].float().cpu().numpy()
+        O.forward(ref, h0, np_layers)
+        done += 1
+        edges += len(ref["nbrs"])
+        if time.time() - t0 > budget_s:
+            break
+    dt = time.time() - t0
+    return {"batches": done, "seconds": dt, "batches_per_s": done / dt, "edges_per_s": edges / dt}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=8)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="mgdense", choices=["mgdense", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(CONFIGS))
+    ap.add_argument("--group", type=int, default=128, help="mini-batches per step")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-budget", type=float, default=20.0)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "mgdense" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    cfg = CONFIGS[args.workload]
+    peaks = measured_peaks()
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        run_reference(args, cfg)
+        return
+
+    import paper_2202_02365_b200 as mg
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    g, feats, layers, setup = build_workload(cfg, device, seed=0)
+    ctx = mg.Context(local_rank)
+    ctx.load_graph(g.row_offsets, g.nbrs)
+    g_host = None
+    if rank == 0 and not args.no_cpu_baseline:
+        g_host = (g.row_offsets.cpu().numpy(), g.nbrs.cpu().numpy())
+    n_edges = g.n_edges
+    del g
+    torch.cuda.empty_cache()
+    if cfg["parts"] > 1:
+        ctx.set_partitioning(cfg["parts"])
+        ctx.load_features(feats, capacity_parts=cfg["parts"])
+        ctx.set_resident(list(range(cfg["parts"])))
+    else:
+        ctx.load_features(feats)
+    model = ctx.model(layers, mg.GEMM_TF32)
+
+    G, T, k = args.group, cfg["batch"], len(cfg["fanouts"])
+    n_steps_total = args.warmup + 2 * args.steps + 1
+    # every rank draws its own mini-batches from the shuffled train set
+    all_targets = inputs.train_set_batches(cfg["n"], cfg["train"], T, G * n_steps_total, seed=100 + rank)
+    offs = torch.arange(0, G + 1, dtype=torch.int64) * T
+
+    def step_targets(i):
+        return all_targets[i * G:(i + 1) * G].reshape(-1)
+
+    def step_seeds(i):
+        return [(rank << 40) + i * G + b for b in range(G)]
+
+    # capacities from a probe group (worst-case bounds would waste memory by ~10x)
+    probe = ctx.sample_many(step_targets(0).to(device), offs, cfg["fanouts"], step_seeds(0),
+                            caps=None if cfg["n"] < 2_000_000 else {"max_nodes_per_batch": 1 << 19})
+    nodes, ents = probe.counts()
+    caps = {"max_nodes_total": int(nodes.sum() * 1.3) + 1024, "max_entries_total": int(ents.sum() * 1.3) + 1024,
+            "max_nodes_per_batch": int(nodes.sum(1).max() * 1.5) + 64}
+    probe.free()
+    dense = ctx.sample_many(step_targets(0).to(device), offs, cfg["fanouts"], step_seeds(0), caps=caps)
+
+    out_dev = torch.empty((G * T, cfg["hidden"]), dtype=torch.float32, device=device)
+    out_host = torch.empty((G * T, cfg["hidden"]), dtype=torch.float32).pin_memory()
+    dev_targets = [step_targets(i).to(device) for i in range(n_steps_total)]
+    host_targets = [step_targets(i).pin_memory() for i in range(n_steps_total)]
+
+    def run_step(i, e2e):
+        tg = host_targets[i] if e2e else dev_targets[i]
+        ctx.sample_many(tg, offs, cfg["fanouts"], step_seeds(i), caps=caps, out=dense)
+        ctx.forward(model, dense, out_host if e2e else out_dev)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+
+    for i in range(args.warmup):
+        run_step(i, False)
+
+    # ---- device-resident timing -------------------------------------------------------
+    stats = {"nodes": [], "ents": []}
+    ctx.profile(True)
+    ctx.profile_read(reset=True)
+    launches0 = ctx.kernel_launches()
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for s in range(args.steps):
+        run_step(args.warmup + s, False)
+        n_, e_ = dense.counts()
+        stats["nodes"].append(n_); stats["ents"].append(e_)
+    ev1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms_dev = ev0.elapsed_time(ev1)
+    launches = ctx.kernel_launches() - launches0
+    phases = ctx.profile_read(reset=True)
+    ctx.profile(False)
+
+    # ---- end to end: host targets in, host H^k out --------------------------------------
+    barrier()
+    ev2, ev3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev2.record()
+    for s in range(args.steps):
+        run_step(args.warmup + args.steps + s, True)
+    ev3.record()
+    barrier()
+    ms_e2e = ev2.elapsed_time(ev3)
+
+    if world > 1:
+        t = torch.tensor([ms_dev, ms_e2e], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_dev, ms_e2e = float(t[0]), float(t[1])
+
+    nodes = torch.cat(stats["nodes"]).numpy()
+    ents = torch.cat(stats["ents"]).numpy()
+    alg = algorithmic_bytes(nodes, ents, cfg)
+    n_batches = args.steps * G * world
+    value = n_batches / (ms_dev / 1e3)
+    e2e_value = n_batches / (ms_e2e / 1e3)
+    sampled_edges = float(ents.sum()) * world
+
+    # ---- rooflines per phase (CUDA-event times of the library's own kernels) --------------
+    sample_ms = sum(v["ms"] for name, v in phases.items() if name.startswith("sample_"))
+    agg1 = phases["aggregate_l1"]
+    gemm = phases["gemm"]
+    tf32_peak = peaks["bf16_tflops_sustained"] * 0.5     # nominal TF32 : bf16 dense ratio is 1 : 2
+    rl_agg = {"kernel": "k_aggregate (layer 1: feature gather + segment mean)", "bound": "hbm",
+              "achieved": alg["agg_l1"] / (agg1["ms"] / 1e3) / 1e9 if agg1["ms"] else None,
+              "peak": peaks["hbm_gbs"], "unit": "GB/s",
+              "bytes_per_launch": alg["agg_l1"] / max(1, agg1["launches"]),
+              "ms_per_launch": agg1["ms"] / max(1, agg1["launches"]), "launches": agg1["launches"]}
+    rl_agg["frac"] = rl_agg["achieved"] / rl_agg["peak"] if rl_agg["achieved"] else None
+    rl_gemm = {"kernel": "k_gemm_tf32 (tcgen05)", "bound": "tensor",
+               "achieved": alg["flops"] / (gemm["ms"] / 1e3) / 1e12 if gemm["ms"] else None,
+               "peak": tf32_peak, "unit": "TFLOP/s", "launches": gemm["launches"],
+               "ms_per_launch": gemm["ms"] / max(1, gemm["launches"])}
+    rl_gemm["frac"] = rl_gemm["achieved"] / rl_gemm["peak"] if rl_gemm["achieved"] else None
+    mem_ms = sample_ms + agg1["ms"] + phases["aggregate_rest"]["ms"]
+    path_gbs = alg["a_min"] / (mem_ms / 1e3) / 1e9 if mem_ms else None
+    dominant = rl_agg if agg1["ms"] >= gemm["ms"] else rl_gemm
+    roofline = dict(dominant)
+    roofline["traffic"] = None
+    roofline["peak_source"] = peaks["source"]
+
+    line = {
+        "metric": "DENSE sample+aggregate mini-batches/s", "value": value, "unit": "mini-batches/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_dev / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32 (TF32 tensor-core GEMM)",
+        "data": "synthetic",
+        "config": {"workload": args.workload, "nodes": cfg["n"], "edges": n_edges, "feature_dim": cfg["dim"],
+                   "hidden": cfg["hidden"], "fanouts": cfg["fanouts"], "targets_per_batch": T,
+                   "mini_batches_per_step": G, "partitions": cfg["parts"], "resident": cfg["parts"],
+                   "l2": "inputs larger than L2 (feature table and CSR far exceed 126 MB; no flush)",
+                   "setup_s": setup},
+        "sampled_edges_per_s": sampled_edges / (ms_dev / 1e3),
+        "per_batch": {"nodes": float(nodes.sum(1).mean()), "sampled_edges": float(ents.sum(1).mean()),
+                      "algorithmic_bytes": alg["a_min"] / (args.steps * G),
+                      "gemm_flops": alg["flops"] / (args.steps * G)},
+        "e2e": {"value": e2e_value, "unit": "mini-batches/s", "h2d_bytes_per_step": int(G * T * 4),
+                "d2h_bytes_per_step": int(G * T * cfg["hidden"] * 4), "ms_per_step": ms_e2e / args.steps},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": roofline,
+        "roofline_gemm": rl_gemm,
+        "roofline_aggregate_l1": rl_agg,
+        "path_hbm": {"what": "A_min over the sampling + aggregation kernel time (GEMMs excluded)",
+                     "achieved_gbs": path_gbs, "frac_of_measured": path_gbs / peaks["hbm_gbs"] if path_gbs else None,
+                     "frac_of_8tbs": path_gbs / HBM_NOMINAL_GBS if path_gbs else None, "kernel_ms": mem_ms},
+        "phases_ms_per_step": {name: round(v["ms"] / args.steps, 4) for name, v in phases.items() if v["launches"]},
+    }
+    if rank == 0:
+        if g_host is not None:
+            r = oracle_time(g_host, feats, layers, cfg, all_targets[args.warmup * G:], step_seeds(args.warmup),
+                            budget_s=args.cpu_budget)
+            line["cpu_baseline"] = {"value": r["batches_per_s"], "unit": "mini-batches/s", "cores": 1, "kind": "oracle",
+                                    "sample": f"{r['batches']} mini-batches of the timed workload in {r['seconds']:.1f} s",
+                                    "sampled_edges_per_s": r["edges_per_s"]}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_reference(args, cfg):
+    """The CPU oracle on the host cores: a bounded sample of the same workload per step."""
+    from oracle import dense_oracle as O  # noqa: F401
+    device = torch.device("cuda", 0) if torch.cuda.is_available() else torch.device("cpu")
+    g, feats, layers, _ = build_workload(cfg, device, seed=0)
+    g_host = (g.row_offsets.cpu().numpy(), g.nbrs.cpu().numpy())
+    n_edges = g.n_edges
+    del g
+    per_step = 1
+    total = (args.warmup + args.steps) * per_step
+    targets = inputs.train_set_batches(cfg["n"], cfg["train"], cfg["batch"], max(total, 1), seed=100)
+    seeds = list(range(total))
+    if args.warmup:
+        oracle_time(g_host, feats, layers, cfg, targets[:args.warmup], seeds[:args.warmup], budget_s=1e9)
+    r = oracle_time(g_host, feats, layers, cfg, targets[args.warmup:], seeds[args.warmup:], budget_s=1e9)
+    line = {
+        "impl": "reference", "metric": "DENSE sample+aggregate mini-batches/s", "value": r["batches_per_s"],
+        "unit": "mini-batches/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": r["seconds"] / max(1, r["batches"]) * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "nodes": cfg["n"], "edges": n_edges, "feature_dim": cfg["dim"],
+                   "hidden": cfg["hidden"], "fanouts": cfg["fanouts"], "targets_per_batch": cfg["batch"],
+                   "mini_batches_per_step": per_step},
+        "cpu_baseline": {"value": r["batches_per_s"], "unit": "mini-batches/s", "cores": 1, "kind": "oracle",
+                         "sample": f"{per_step} mini-batch per step, {r['batches']} steps"},
+        "e2e": {"value": r["batches_per_s"], "unit": "mini-batches/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "sampled_edges_per_s": r["edges_per_s"],
+    }
+    print(json.dumps(line))
+
+
+if __name__ == "__main__":
+    main()

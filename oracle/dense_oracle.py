@@ -91,7 +91,7 @@ class GraphView:
 
     def __init__(self, row_offsets, nbrs, n_parts: int = 1, resident_parts=None):
         self.row_offsets = np.asarray(row_offsets, dtype=np.int64)
-        self.nbrs = np.asarray(nbrs, dtype=np.int64)
+        self.nbrs = np.asarray(nbrs)
         self.n_nodes = len(self.row_offsets) - 1
         self.n_parts = int(n_parts)
         self.part_size = (self.n_nodes + self.n_parts - 1) // self.n_parts
