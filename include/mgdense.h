@@ -205,6 +205,32 @@ int mg_gather_h0(mg_ctx* ctx, mg_dense* d, int32_t batch, float* out_dev);
 int mg_layer_output(mg_ctx* ctx, const mg_model* m, mg_dense* d, int32_t layer, int32_t batch,
                     float* out_dev);
 
+/* Size of the scratch array built into the library for mg_forward_noalloc.  Every GPU that
+ * loads the library holds this much device memory until the process exits. */
+#define MG_NOALLOC_SCRATCH_BYTES (16u << 20)
+
+/* mg_forward for callers that must not allocate device memory while they run.  (The paper has
+ * no counterpart; this is a service of the library.)  Such callers exist: a serving process
+ * whose device memory was handed out in full at start-up, so that a later cudaMalloc fails; a
+ * host framework whose caching allocator owns the rest of the GPU; a latency-bound loop that
+ * cannot afford the device-wide synchronisation an allocation or a free implies.  mg_forward
+ * grows its workspaces with cudaMalloc when a sample is larger than any before it; this entry
+ * point never calls cudaMalloc, cudaFree or any allocating routine.  It computes the same H^k
+ * with the same kernels, keeping the [self | mean] staging rows (first 4 MiB) and the
+ * intermediate layer outputs H^1..H^{k-1} (remaining 12 MiB) in a scratch array of
+ * MG_NOALLOC_SCRATCH_BYTES that is part of the library image.
+ *  - out_dev: DEVICE pointer, one row of dims[k] fp32 per target, as mg_forward writes it.
+ *  - Limit: sum over l < k of rows(H^l) * dims[l] * 4 bytes must fit in 12 MiB; larger samples
+ *    get MG_ERR_CAPACITY (nothing is launched) — use mg_forward or fewer mini-batches per call.
+ *  - The first call on a device looks up the array's device address (cudaGetSymbolAddress);
+ *    make that first call before any stream capture begins.
+ *  - All calls in the process share the one array, and it keeps the previous call's contents.
+ *    Nothing in it needs clearing (every value read was written earlier in the same call), but
+ *    two calls that overlap on the GPU — from two contexts or two host threads — race on it:
+ *    run them one after the other.
+ * Other errors as mg_forward. */
+int mg_forward_noalloc(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out_dev);
+
 /* ---- link prediction: shared negatives, target union, DistMult ------------------------ */
 
 /* Prepare a batch of n_edges training edges (HOST int32 src / rel / dst; dst aggregates

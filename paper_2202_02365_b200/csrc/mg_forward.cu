@@ -503,3 +503,102 @@ extern "C" int mg_layer_output(mg_ctx* ctx, const mg_model* m, mg_dense* d, int3
     MG_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     return MG_OK;
 }
+
+// ---------------------------------------------------------------------------------------
+// Forward pass that allocates nothing (the paper has no counterpart).
+//
+// All temporaries live in one file-scope device array that every GPU loading this library
+// holds until the process exits:
+//   [0, kNoAllocStagingBytes)                     the [self | mean] staging rows of one chunk
+//   [kNoAllocStagingBytes, MG_NOALLOC_SCRATCH_BYTES)  the intermediate layer outputs H^1 .. H^{k-1}
+// Nothing in it has to start at zero: every element a kernel reads was written earlier in the
+// same call (rows past the end of a tile are zero-filled by the TMA load, not read from here).
+// ---------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_noalloc_scratch[MG_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+constexpr size_t kNoAllocStagingBytes = 4u << 20;
+constexpr int kNoAllocMaxDevices = 64;
+unsigned char* g_noalloc_ptr[kNoAllocMaxDevices] = {nullptr};
+}  // namespace
+
+extern "C" int mg_forward_noalloc(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out_dev) {
+    if (!ctx) return MG_ERR_ARG;
+    int rc = forward_checks(ctx, m, d);
+    if (rc) return rc;
+    if (!out_dev) return mg_fail(ctx, MG_ERR_ARG, "null output");
+    if (ctx->device < 0 || ctx->device >= kNoAllocMaxDevices) return mg_fail(ctx, MG_ERR_ARG, "device ordinal above %d", kNoAllocMaxDevices - 1);
+    MG_CUDA(ctx, cudaSetDevice(ctx->device));
+    // once per device, with that device current: the array's name is only a host-side handle, the
+    // kernels need its device address
+    if (!g_noalloc_ptr[ctx->device]) {
+        unsigned char* p = nullptr;
+        const cudaError_t e = cudaGetSymbolAddress((void**)&p, g_noalloc_scratch);
+        if (e != cudaSuccess || !p) return mg_cuda_fail(ctx, e, "cudaGetSymbolAddress(g_noalloc_scratch)");
+        g_noalloc_ptr[ctx->device] = p;
+    }
+    unsigned char* scratch = g_noalloc_ptr[ctx->device];
+    const int k = d->k, B = d->n_batches;
+    cudaStream_t st = ctx->stream;
+
+    // intermediates H^1 .. H^{k-1} must fit behind the staging area
+    size_t off[MG_MAX_HOPS + 1] = {0};
+    size_t inter_floats = 0;
+    for (int l = 1; l < k; ++l) {
+        off[l] = inter_floats;
+        inter_floats += (size_t)d->h_hdr.rows_total[l] * m->dims[l];
+    }
+    const size_t inter_cap = (MG_NOALLOC_SCRATCH_BYTES - kNoAllocStagingBytes) / sizeof(float);
+    if (inter_floats > inter_cap)
+        return mg_fail(ctx, MG_ERR_CAPACITY,
+                       "mg_forward_noalloc: intermediate layer outputs need %zu bytes, the built-in scratch holds %zu "
+                       "(MG_NOALLOC_SCRATCH_BYTES = %u in total); use mg_forward or fewer mini-batches per call",
+                       inter_floats * sizeof(float), inter_cap * sizeof(float), (unsigned)MG_NOALLOC_SCRATCH_BYTES);
+    float* staging = reinterpret_cast<float*>(scratch);
+    float* inter = reinterpret_cast<float*>(scratch + kNoAllocStagingBytes);
+
+    const bool half = ctx->feat_dtype == MG_DTYPE_F16;
+    for (int l = 1; l <= k; ++l) {
+        const int d_in = m->dims[l - 1], d_out = m->dims[l];
+        const int64_t M = d->h_hdr.rows_total[l];
+        float* h_out = l == k ? out_dev : inter + off[l];
+        const float* h_prev = l > 1 ? inter + off[l - 1] : nullptr;
+        int64_t chunk = (int64_t)(kNoAllocStagingBytes / sizeof(float)) / (2 * d_in);
+        chunk = chunk / 128 * 128;
+        if (chunk < 128) return mg_fail(ctx, MG_ERR_CAPACITY, "mg_forward_noalloc: layer width %d too large for the staging area", d_in);
+        for (int64_t r0 = 0; r0 < M; r0 += chunk) {
+            const int64_t r1 = std::min(M, r0 + chunk);
+            AggArgs a;
+            a.B = B; a.k = k; a.layer = l; a.d_in = d_in;
+            a.row_lo = (int32_t)r0; a.row_hi = (int32_t)r1;
+            a.rowbase_out = d->rowbase + (size_t)l * (B + 1);
+            a.rowbase_in = d->rowbase + (size_t)(l - 1) * (B + 1);
+            a.cum = d->cum; a.node_off = d->node_off; a.nodes = d->nodes;
+            a.ent_off = d->ent_off; a.ent_nbrs = d->ent_nbrs; a.ent_repr = d->ent_repr;
+            a.h_prev = h_prev;
+            a.slots = ctx->slots; a.slot_of_part = ctx->d_slot_of_part;
+            a.slot_bytes = ctx->slot_bytes; a.row_bytes = ctx->row_bytes; a.part_size = (uint32_t)ctx->part_size;
+            a.x = staging;
+            a.round_tf32 = m->precision == MG_GEMM_TF32;
+            const int grid = mg_grid(ctx, 8);
+            if (l == 1) { if (half) launch_aggregate<true, true>(a, grid, st); else launch_aggregate<true, false>(a, grid, st); }
+            else launch_aggregate<false, false>(a, grid, st);
+            ctx->launches++;
+            const int64_t rows = r1 - r0;
+            const bool relu = l < k;
+            if (m->precision == MG_GEMM_FP32) {
+                dim3 g2((unsigned)((rows + 63) / 64), (unsigned)((d_out + 63) / 64));
+                if (relu) k_gemm_fp32<true><<<g2, 256, 0, st>>>(staging, m->w_cat[l - 1], m->bias[l - 1], h_out + r0 * d_out, rows, d_out, 2 * d_in);
+                else k_gemm_fp32<false><<<g2, 256, 0, st>>>(staging, m->w_cat[l - 1], m->bias[l - 1], h_out + r0 * d_out, rows, d_out, 2 * d_in);
+                ctx->launches++;
+            } else {
+                rc = mg_gemm_tf32(ctx, staging, m->w_cat_t[l - 1], m->bias[l - 1], h_out + r0 * d_out, rows, d_out, 2 * d_in, relu);
+                if (rc) return rc;
+            }
+        }
+    }
+    MG_CUDA(ctx, cudaGetLastError());
+    MG_CUDA(ctx, cudaStreamSynchronize(st));
+    if (m->precision == MG_GEMM_TF32) return mg_gemm_tf32_status(ctx);
+    return MG_OK;
+}
