@@ -16,6 +16,11 @@
 int mg_gemm_tf32(mg_ctx* ctx, const float* x, const float* w_t, const float* bias, float* out, int64_t M, int N, int K,
                  bool relu);  // mg_gemm_tcgen05.cu
 int mg_gemm_tf32_status(mg_ctx* ctx);
+// mg_layer_fused.cu
+int mg_pack_layer_weights(mg_ctx* ctx, const float* w_cat_dev, float* w_pad_t_dev, int d_in, int N);
+bool mg_layer_fused_supported(int d_in, int d_out);
+int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_out, const float* w_pad_t, const float* bias,
+                   const float* h_prev, float* h_out, bool relu);
 
 namespace {
 
@@ -327,6 +332,7 @@ extern "C" int mg_model_create(mg_ctx* ctx, int32_t k, const int32_t* dims, cons
         const size_t di = dims[l], dn = dims[l + 1];
         if (cudaMalloc((void**)&m->w_cat[l], sizeof(float) * 2 * di * dn) != cudaSuccess ||
             cudaMalloc((void**)&m->w_cat_t[l], sizeof(float) * 2 * di * dn) != cudaSuccess ||
+            cudaMalloc((void**)&m->w_pad_t[l], sizeof(float) * 2 * ((di + 31) / 32 * 32) * dn) != cudaSuccess ||
             cudaMalloc((void**)&m->bias[l], sizeof(float) * dn) != cudaSuccess) {
             cudaGetLastError();
             mg_model_free(m);
@@ -339,6 +345,7 @@ extern "C" int mg_model_create(mg_ctx* ctx, int32_t k, const int32_t* dims, cons
         k_transpose<<<mg_grid(ctx, 2), kThreads, 0, ctx->stream>>>(m->w_cat[l], m->w_cat_t[l], (int)(2 * di), (int)dn,
                                                                   gemm_precision == MG_GEMM_TF32);
         ctx->launches++;
+        mg_pack_layer_weights(ctx, m->w_cat[l], m->w_pad_t[l], (int)di, (int)dn);
     }
     cudaError_t e = cudaStreamSynchronize(ctx->stream);
     if (e == cudaSuccess) e = cudaGetLastError();
@@ -350,7 +357,7 @@ extern "C" int mg_model_create(mg_ctx* ctx, int32_t k, const int32_t* dims, cons
 extern "C" int mg_model_free(mg_model* m) {
     if (!m) return MG_OK;
     cudaSetDevice(m->device);
-    for (int l = 0; l < MG_MAX_HOPS; ++l) { cudaFree(m->w_cat[l]); cudaFree(m->w_cat_t[l]); cudaFree(m->bias[l]); }
+    for (int l = 0; l < MG_MAX_HOPS; ++l) { cudaFree(m->w_cat[l]); cudaFree(m->w_cat_t[l]); cudaFree(m->w_pad_t[l]); cudaFree(m->bias[l]); }
     delete m;
     return MG_OK;
 }
@@ -412,6 +419,13 @@ extern "C" int mg_forward(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* ou
         const int64_t M = d->h_hdr.rows_total[l];
         float* h_out = ctx->ws_h[0] + off[l];
         const float* h_prev = l > 1 ? ctx->ws_h[0] + off[l - 1] : nullptr;
+        if (m->precision == MG_GEMM_TF32 && mg_layer_fused_supported(d_in, d_out)) {
+            // gather + segment mean + both linear maps in one persistent tensor-core kernel
+            ProfScope ps(ctx, l == 1 ? PH_AGG_L1 : PH_AGG_REST, 1);
+            rc = mg_layer_fused(ctx, d, l, d_in, d_out, m->w_pad_t[l - 1], m->bias[l - 1], h_prev, h_out, l < k);
+            if (rc) return rc;
+            continue;
+        }
         const int64_t chunk = chunk_rows_for(d_in);
         for (int64_t r0 = 0; r0 < M; r0 += chunk) {
             const int64_t r1 = std::min(M, r0 + chunk);

@@ -159,6 +159,7 @@ struct mg_model {
     int precision = MG_GEMM_TF32;
     float* w_cat[MG_MAX_HOPS] = {nullptr};  // device [2*d_in, d_out]: rows 0..d_in-1 self, then neighbour
     float* w_cat_t[MG_MAX_HOPS] = {nullptr}; // device [d_out, 2*d_in] (K-major copy for the tensor-core path)
+    float* w_pad_t[MG_MAX_HOPS] = {nullptr}; // device [d_out, 2*roundup32(d_in)], zero padded, for the fused layer kernel
     float* bias[MG_MAX_HOPS] = {nullptr};
 };
 
