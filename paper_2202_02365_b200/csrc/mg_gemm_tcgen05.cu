@@ -100,28 +100,16 @@ k_gemm_tf32(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         if (!ok && lane == 0) atomicExch(p.error, 3u);
         tc_fence_after();
         const int lane_group = warp & 3;                 // tensor-memory lanes this warp may read
-        const int64_t row = m0 + lane_group * 32 + lane;
+        const int64_t row0 = m0 + lane_group * 32;
+        // the operand ring is idle once the accumulator is complete: its first 17 KiB serve as the four
+        // warps' transpose buffers for coalesced stores
+        float* out_stage = reinterpret_cast<float*>(stage_base);
         if (ok) {
             for (int c0 = 0; c0 < p.BN; c0 += 32) {
                 uint32_t v[32];
                 tmem_ld_32(tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)c0, v);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (row < p.M) {
-                    float* orow = p.out + row * p.N + n0 + c0;
-#pragma unroll
-                    for (int j = 0; j < 32; j += 4) {
-                        const int n = n0 + c0 + j;
-                        if (c0 + j < p.BN && n < p.N) {
-                            float4 o;
-                            o.x = __uint_as_float(v[j]) + p.bias[n];
-                            o.y = __uint_as_float(v[j + 1]) + p.bias[n + 1];
-                            o.z = __uint_as_float(v[j + 2]) + p.bias[n + 2];
-                            o.w = __uint_as_float(v[j + 3]) + p.bias[n + 3];
-                            if (p.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f); }
-                            *reinterpret_cast<float4*>(orow + j) = o;
-                        }
-                    }
-                }
+                if (row0 < p.M) store_slice_coalesced(v, out_stage + lane_group * (32 * 33), p.bias, p.out, row0, p.M, p.N, n0 + c0, p.relu != 0);
             }
         }
     }

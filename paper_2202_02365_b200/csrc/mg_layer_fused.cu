@@ -16,6 +16,7 @@
 #include <cuda_fp16.h>
 
 #include <algorithm>
+#include <cstdlib>
 
 #include "mg_device.cuh"
 #include "mg_internal.cuh"
@@ -31,6 +32,9 @@ constexpr int kProducerWarps = 16;
 constexpr int kFirstProducerWarp = 6; // warp 0 TMA, warp 1 MMA + tensor memory, warps 2..5 epilogue
 constexpr int kFusedThreads = (kFirstProducerWarp + kProducerWarps) * 32;  // 704
 constexpr int kMaxStages = 8;
+constexpr int kGroupCols = 128;                  // input columns whose (self, mean) slices the producers fill together
+constexpr int kRowsInFlight = 2;                 // rows a producer warp builds at the same time
+constexpr int kUnroll = 5;                       // neighbour rows per output row fetched before the first add
 constexpr uint32_t kABytes = BM * KC * 4;  // 16 KiB per A stage
 
 struct FusedArgs {
@@ -44,12 +48,16 @@ struct FusedArgs {
     const int32_t* ent_off;
     const int32_t* ent_nbrs;
     const int32_t* ent_repr;
+    const int4* row_meta;        // [M] (self source row, first entry, entry count, first H^{l-1} row of the batch)
     // input rows
     const float* h_prev;         // layers >= 2: [rows of layer l-1, d_in]
+    const char* src_base;        // layer 1: the feature buffer; later layers: h_prev
+    int64_t src_row_bytes;
     const char* slots;           // layer 1: partition buffer
     const int32_t* slot_of_part;
     int64_t slot_bytes, row_bytes;
     uint32_t part_size;
+    int32_t identity_rows;       // layer 1: slot == partition for every resident partition (whole table in HBM)
     // shapes
     int32_t d_in, d_in_pad;      // d_in_pad = d_in rounded up to 32; K = 2 * d_in_pad
     int32_t N, BN;               // output width and its MMA tile width (multiple of 16, <= 256)
@@ -60,33 +68,40 @@ struct FusedArgs {
     const float* bias;
     float* out;                  // [M, N]
     uint32_t* error;
+    int32_t dbg;
 };
+
+constexpr int kKeyCap = 2048;   // source-row indices of a tile's entries cached in shared memory
 
 struct RowMeta {      // what a producer needs to build one output row
-    int64_t self_off; // layer 1: node id of the row; later layers: row index into h_prev
-    int64_t in_base;  // later layers: first h_prev row of the row's mini-batch
-    int32_t e0, cnt;  // entries of the row
+    int32_t self_src; // source row of the row's own representation
+    int32_t e0, cnt;  // its entries in the sample's entry arrays; cnt < 0: row past the end
+    int32_t koff;     // first cached source-row index of the row, or -1 when the tile's entries do not fit
+    int32_t in_base;  // layers >= 2: first row of the mini-batch in H^{l-1}
 };
 
+// Source row of an entry.  Layer 1: the feature-buffer row of node `key` (its partition's slot);
+// later layers: row of H^{l-1}.  The address is src_base + row * src_row_bytes.
 template <bool FIRST>
-__device__ __forceinline__ const char* input_row(const FusedArgs& a, int64_t in_base, int32_t key) {
+__device__ __forceinline__ int32_t source_row(const FusedArgs& a, int32_t in_base, int32_t key) {
     if (FIRST) {
+        if (a.identity_rows) return key;
         const uint32_t p = (uint32_t)key / a.part_size;
-        return a.slots + (int64_t)a.slot_of_part[p] * a.slot_bytes + (int64_t)((uint32_t)key - p * a.part_size) * a.row_bytes;
+        return (int32_t)((uint32_t)a.slot_of_part[p] * a.part_size + ((uint32_t)key - p * a.part_size));
     }
-    return reinterpret_cast<const char*>(a.h_prev + (in_base + key) * a.d_in);
+    return in_base + key;
 }
 
-// 4 consecutive values of a row starting at column col (a multiple of 4)
+// 4 consecutive values at p (fp16 values are widened exactly)
 template <bool HALF>
-__device__ __forceinline__ float4 load4(const char* row, int col) {
+__device__ __forceinline__ float4 load4(const char* p) {
     if (HALF) {
-        const uint2 raw = __ldg(reinterpret_cast<const uint2*>(row + (size_t)col * 2));
+        const uint2 raw = __ldg(reinterpret_cast<const uint2*>(p));
         const float2 lo = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
         const float2 hi = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
         return make_float4(lo.x, lo.y, hi.x, hi.y);
     }
-    return __ldg(reinterpret_cast<const float4*>(row + (size_t)col * 4));
+    return __ldg(reinterpret_cast<const float4*>(p));
 }
 
 template <bool FIRST, bool HALF>
@@ -97,13 +112,16 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, FusedArgs a) {
     __shared__ uint64_t acc_full[2], acc_empty[2];
     __shared__ uint32_t tmem_slot;
     __shared__ RowMeta meta[BM];
+    __shared__ int32_t src_rows[kKeyCap];
+    __shared__ uint32_t key_warp_sum[BM / 32];
+    __shared__ int32_t key_end[BM];
+    __shared__ float out_stage[4][32 * 33];   // per epilogue warp: transpose buffer for coalesced stores
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t b_bytes = (uint32_t)a.BN * KC * 4;
     uint8_t* a_base = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* b_base = a_base + (size_t)a.sa * kABytes;
     const int n_chunks = 2 * a.d_in_pad / KC;
-    const int self_chunks = a.d_in_pad / KC;
     const int64_t n_tiles = (a.M + BM - 1) / BM;
 
     if (threadIdx.x == 0) {
@@ -159,7 +177,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, FusedArgs a) {
                     const uint64_t db = smem_desc_sw128(smem_u32(b_base + (size_t)sb * b_bytes));
 #pragma unroll
                     for (int kk = 0; kk < KC / 8; ++kk)
-                        mma_tf32(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (c | kk) ? 1u : 0u);
+                        if (!(a.dbg & 4)) mma_tf32(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (c | kk) ? 1u : 0u);
                     mma_commit(&a_empty[sa]);
                     mma_commit(&b_empty[sb]);
                 }
@@ -176,25 +194,12 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, FusedArgs a) {
             const uint32_t buf = it & 1;
             if (!mbar_wait(&acc_full[buf], (it >> 1) & 1)) { if (lane == 0) atomicExch(a.error, 14u); ok = false; break; }
             tc_fence_after();
-            const int64_t row = t * BM + lane_group * 32 + lane;
+            const int64_t row0 = t * BM + lane_group * 32;
             for (int c0 = 0; c0 < a.BN; c0 += 32) {
                 uint32_t v[32];
                 tmem_ld_32(tmem_base + buf * acc_stride + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)c0, v);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (row < a.M) {
-                    float* orow = a.out + row * a.N + c0;
-#pragma unroll
-                    for (int j = 0; j < 32; j += 4) {
-                        const int n = c0 + j;
-                        if (n < a.N) {
-                            const float4 bb = __ldg(reinterpret_cast<const float4*>(a.bias + n));
-                            float4 o = make_float4(__uint_as_float(v[j]) + bb.x, __uint_as_float(v[j + 1]) + bb.y,
-                                                   __uint_as_float(v[j + 2]) + bb.z, __uint_as_float(v[j + 3]) + bb.w);
-                            if (a.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f); }
-                            *reinterpret_cast<float4*>(orow + j) = o;
-                        }
-                    }
-                }
+                if (row0 < a.M && !(a.dbg & 2)) store_slice_coalesced(v, out_stage[lane_group], a.bias, a.out, row0, a.M, a.N, c0, a.relu != 0);
             }
             tc_fence_before();
             __syncwarp();
@@ -204,81 +209,159 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, FusedArgs a) {
         // ---------------- producers: gather + segment mean -> swizzled A slices ----------------
         const int pw = warp - kFirstProducerWarp;     // 0 .. kProducerWarps-1
         const int ptid = threadIdx.x - kFirstProducerWarp * 32;
-        const int g = lane >> 3, gl = lane & 7;       // 4 rows per warp at a time, 8 lanes x float4 per row slice
+        const int gl = lane & 7;                      // 16-byte slot inside a 128-byte slice row
         constexpr int kRowsPerWarp = BM / kProducerWarps;  // 8
         uint32_t cnt = 0;
         bool ok = true;
         for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
-            // row metadata of the tile, once
+            // row metadata of the tile and the source rows of all its entries, once per tile
             asm volatile("bar.sync 1, %0;" ::"r"(kProducerWarps * 32) : "memory");   // previous tile's readers are done
+            RowMeta mm;
+            mm.self_src = 0; mm.e0 = 0; mm.cnt = -1; mm.koff = -1; mm.in_base = 0;
+            uint32_t incl = 0;
             if (ptid < BM) {
                 const int64_t r = t * BM + ptid;
-                RowMeta mm;
-                mm.self_off = 0; mm.in_base = 0; mm.e0 = 0; mm.cnt = -1;   // cnt < 0: row past the end
                 if (r < a.M) {
-                    const int b = upper_segment(a.rowbase_out, a.B + 1, (int32_t)r);
-                    const int32_t l = (int32_t)r - a.rowbase_out[b];
-                    const int32_t* cum = a.cum + b * (a.k + 2);
-                    int h = 0;
-                    while (h < a.k - a.layer && l >= cum[h + 1]) ++h;
-                    const int32_t idx = a.node_off[h * (a.B + 1) + b] + (l - cum[h]);
-                    mm.e0 = a.ent_off[idx];
-                    mm.cnt = a.ent_off[idx + 1] - mm.e0;
-                    mm.in_base = FIRST ? 0 : (int64_t)a.rowbase_in[b];
-                    mm.self_off = FIRST ? (int64_t)a.nodes[idx] : (int64_t)l;
+                    const int4 rm = __ldg(a.row_meta + r);   // (self_src, e0, cnt, in_base) from the pre-pass
+                    mm.self_src = rm.x; mm.e0 = rm.y; mm.cnt = rm.z; mm.in_base = rm.w;
                 }
-                meta[ptid] = mm;
+                incl = warp_incl_scan((uint32_t)max(mm.cnt, 0));
+                if (lane == 31) key_warp_sum[pw] = incl;
             }
             asm volatile("bar.sync 1, %0;" ::"r"(kProducerWarps * 32) : "memory");
-            for (int c = 0; c < n_chunks; ++c, ++cnt) {
-                const int s = cnt % a.sa;
-                if (ok && cnt >= (uint32_t)a.sa && !mbar_wait(&a_empty[s], ((cnt / a.sa) - 1) & 1)) {
-                    if (lane == 0) atomicExch(a.error, 15u);
-                    ok = false;
-                }
-                ok = __all_sync(0xFFFFFFFFu, ok);
-                if (!ok) continue;   // keep the named barriers balanced, do no more work
-                uint8_t* stage = a_base + (size_t)s * kABytes;
-                const bool is_self = c < self_chunks;
-                const int col = (is_self ? c : c - self_chunks) * KC + gl * 4;
-                const bool col_ok = col < a.d_in;
+            uint32_t total = 0;
 #pragma unroll
-                for (int rr = 0; rr < kRowsPerWarp; rr += 4) {
-                    const int row = pw * kRowsPerWarp + rr + g;
-                    const RowMeta mm = meta[row];
-                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (mm.cnt >= 0 && col_ok) {
-                        if (is_self) {
-                            acc = load4<HALF>(input_row<FIRST>(a, mm.in_base, (int32_t)mm.self_off), col);
-                        } else if (mm.cnt > 0) {
-                            const int32_t* keys = (FIRST ? a.ent_nbrs : a.ent_repr) + mm.e0;
-                            int e = 0;
-                            for (; e + 4 <= mm.cnt; e += 4) {   // four rows in flight, summed in entry order
-                                const float4 v0 = load4<HALF>(input_row<FIRST>(a, mm.in_base, __ldg(keys + e)), col);
-                                const float4 v1 = load4<HALF>(input_row<FIRST>(a, mm.in_base, __ldg(keys + e + 1)), col);
-                                const float4 v2 = load4<HALF>(input_row<FIRST>(a, mm.in_base, __ldg(keys + e + 2)), col);
-                                const float4 v3 = load4<HALF>(input_row<FIRST>(a, mm.in_base, __ldg(keys + e + 3)), col);
-                                acc.x += v0.x; acc.y += v0.y; acc.z += v0.z; acc.w += v0.w;
-                                acc.x += v1.x; acc.y += v1.y; acc.z += v1.z; acc.w += v1.w;
-                                acc.x += v2.x; acc.y += v2.y; acc.z += v2.z; acc.w += v2.w;
-                                acc.x += v3.x; acc.y += v3.y; acc.z += v3.z; acc.w += v3.w;
-                            }
-                            for (; e < mm.cnt; ++e) {
-                                const float4 v0 = load4<HALF>(input_row<FIRST>(a, mm.in_base, __ldg(keys + e)), col);
-                                acc.x += v0.x; acc.y += v0.y; acc.z += v0.z; acc.w += v0.w;
-                            }
-                            const float inv = 1.f / (float)mm.cnt;
-                            acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
-                        }
-                        acc.x = to_tf32(acc.x); acc.y = to_tf32(acc.y); acc.z = to_tf32(acc.z); acc.w = to_tf32(acc.w);
+            for (int w = 0; w < BM / 32; ++w) total += key_warp_sum[w];
+            const bool cached = total <= (uint32_t)kKeyCap;
+            if (ptid < BM) {
+                uint32_t before = 0;
+#pragma unroll
+                for (int w = 0; w < BM / 32; ++w)
+                    if (w < pw) before += key_warp_sum[w];
+                if (cached && mm.cnt >= 0) mm.koff = (int32_t)(before + incl) - mm.cnt;
+                meta[ptid] = mm;
+                key_end[ptid] = (int32_t)(before + incl);   // end of row ptid's cached entries
+            }
+            asm volatile("bar.sync 1, %0;" ::"r"(kProducerWarps * 32) : "memory");
+            if (cached) {
+                // all producer threads copy the tile's entries: entry j belongs to the first row whose end exceeds j
+                const int32_t* keys = FIRST ? a.ent_nbrs : a.ent_repr;
+                for (uint32_t j = ptid; j < total; j += kProducerWarps * 32) {
+                    int lo = 0, hi = BM - 1;
+                    while (lo < hi) {
+                        const int mid = (lo + hi) >> 1;
+                        if (key_end[mid] > (int32_t)j) hi = mid; else lo = mid + 1;
                     }
-                    // K-major, 128-byte swizzle: 16-byte slot gl of row `row` lands in slot gl ^ (row % 8)
-                    uint8_t* dst = stage + (size_t)(row >> 3) * 1024 + (size_t)(row & 7) * 128 + (size_t)((gl ^ (row & 7)) << 4);
-                    *reinterpret_cast<float4*>(dst) = acc;
+                    const RowMeta rm = meta[lo];
+                    src_rows[j] = source_row<FIRST>(a, rm.in_base, __ldg(keys + rm.e0 + ((int32_t)j - rm.koff)));
+                }
+            }
+            asm volatile("bar.sync 1, %0;" ::"r"(kProducerWarps * 32) : "memory");
+            // K slices come in groups of eight: (self, mean) pairs for four consecutive 32-column blocks, i.e.
+            // 128 columns of the input rows.  A warp builds output rows from whole 512-byte row segments (lane
+            // L owns columns 4L..4L+3 of the group) and keeps kRowsInFlight rows x (1 + kUnroll) loads in
+            // flight per lane -- the producers are few and fat on purpose: memory-level parallelism comes from
+            // registers, not from warps.  Each lane scatters its 16-byte pieces into the group's stages: slice
+            // pair L / 8, slot L % 8.
+            const int n_groups = (a.d_in_pad + kGroupCols - 1) / kGroupCols;
+            for (int grp = 0; grp < n_groups; ++grp) {
+                const int pairs = min(kGroupCols / KC, (a.d_in_pad - grp * kGroupCols) / KC);   // slice pairs in this group
+                const int col = grp * kGroupCols + lane * 4;
+                const bool lane_on = (lane >> 3) < pairs;
+                const bool col_ok = lane_on && col < a.d_in;
+                const char* src = a.src_base + (size_t)col * (HALF ? 2 : 4);
+                bool waited = false;
+                for (int rr = 0; rr < kRowsPerWarp; rr += kRowsInFlight) {
+                    const int row0 = pw * kRowsPerWarp + rr;
+                    RowMeta mq[kRowsInFlight];
+                    float4 selfv[kRowsInFlight], acc[kRowsInFlight];
+                    int top = 0;
+#pragma unroll
+                    for (int q = 0; q < kRowsInFlight; ++q) {
+                        mq[q] = meta[row0 + q];
+                        selfv[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        acc[q] = selfv[q];
+                        top = max(top, mq[q].cnt);
+                    }
+                    if (col_ok && !(a.dbg & 1)) {
+#pragma unroll
+                        for (int q = 0; q < kRowsInFlight; ++q)
+                            selfv[q] = load4<HALF>(src + (size_t)(uint32_t)mq[q].self_src * a.src_row_bytes);
+                        if (cached) {
+                            // Every load is issued unconditionally: a slot past the end of a row's entries re-reads
+                            // the row's own representation (a cache hit) and is added as an exact zero.  Branch-free
+                            // code is what lets all loads of a round be in flight together.
+                            for (int e = 0; e < top; e += kUnroll) {
+                                float4 v[kRowsInFlight][kUnroll];
+#pragma unroll
+                                for (int j = 0; j < kUnroll; ++j)
+#pragma unroll
+                                    for (int q = 0; q < kRowsInFlight; ++q) {
+                                        const bool live = e + j < mq[q].cnt;
+                                        const int32_t sr = src_rows[live ? mq[q].koff + e + j : 0];
+                                        v[q][j] = load4<HALF>(src + (size_t)(uint32_t)(live ? sr : mq[q].self_src) * a.src_row_bytes);
+                                    }
+#pragma unroll
+                                for (int j = 0; j < kUnroll; ++j)   // entry order
+#pragma unroll
+                                    for (int q = 0; q < kRowsInFlight; ++q) {
+                                        const bool live = e + j < mq[q].cnt;   // selects, not branches
+                                        acc[q].x += live ? v[q][j].x : 0.f; acc[q].y += live ? v[q][j].y : 0.f;
+                                        acc[q].z += live ? v[q][j].z : 0.f; acc[q].w += live ? v[q][j].w : 0.f;
+                                    }
+                            }
+                        } else {
+                            // a tile with more entries than the shared-memory cache holds: plain per-entry loop
+                            const int32_t* keys = FIRST ? a.ent_nbrs : a.ent_repr;
+#pragma unroll
+                            for (int q = 0; q < kRowsInFlight; ++q)
+                                for (int e = 0; e < mq[q].cnt; ++e) {
+                                    const int32_t sr = source_row<FIRST>(a, mq[q].in_base, __ldg(keys + mq[q].e0 + e));
+                                    const float4 v = load4<HALF>(src + (size_t)(uint32_t)sr * a.src_row_bytes);
+                                    acc[q].x += v.x; acc[q].y += v.y; acc[q].z += v.z; acc[q].w += v.w;
+                                }
+                        }
+#pragma unroll
+                        for (int q = 0; q < kRowsInFlight; ++q) {
+                            const float inv = mq[q].cnt > 0 ? 1.f / (float)mq[q].cnt : 0.f;
+                            acc[q].x = to_tf32(acc[q].x * inv); acc[q].y = to_tf32(acc[q].y * inv);
+                            acc[q].z = to_tf32(acc[q].z * inv); acc[q].w = to_tf32(acc[q].w * inv);
+                            selfv[q].x = to_tf32(selfv[q].x); selfv[q].y = to_tf32(selfv[q].y);
+                            selfv[q].z = to_tf32(selfv[q].z); selfv[q].w = to_tf32(selfv[q].w);
+                        }
+                    }
+                    if (!waited) {
+                        // the group's stages must have been read by the MMAs of their previous use; the loads
+                        // above are already in flight while this waits
+                        for (int j = 0; j < 2 * pairs; ++j) {
+                            const uint32_t cj = cnt + j;
+                            if (ok && cj >= (uint32_t)a.sa && !mbar_wait(&a_empty[cj % a.sa], ((cj / a.sa) - 1) & 1)) {
+                                if (lane == 0) atomicExch(a.error, 15u);
+                                ok = false;
+                            }
+                        }
+                        ok = __all_sync(0xFFFFFFFFu, ok);
+                        waited = true;
+                    }
+                    if (ok && lane_on) {
+                        // K-major, 128-byte swizzle: 16-byte slot gl of row r lands in slot gl ^ (r % 8)
+                        const uint32_t s_self = (cnt + 2 * (lane >> 3)) % a.sa, s_mean = (cnt + 2 * (lane >> 3) + 1) % a.sa;
+                        uint8_t* stage_self = a_base + (size_t)s_self * kABytes;
+                        uint8_t* stage_mean = a_base + (size_t)s_mean * kABytes;
+#pragma unroll
+                        for (int q = 0; q < kRowsInFlight; ++q) {
+                            const int row = row0 + q;
+                            const size_t off = (size_t)(row >> 3) * 1024 + (size_t)(row & 7) * 128 + (size_t)((gl ^ (row & 7)) << 4);
+                            *reinterpret_cast<float4*>(stage_self + off) = selfv[q];
+                            *reinterpret_cast<float4*>(stage_mean + off) = acc[q];
+                        }
+                    }
                 }
                 fence_async_smem();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&a_full[s]);
+                if (ok && lane == 0)
+                    for (int j = 0; j < 2 * pairs; ++j) mbar_arrive(&a_full[(cnt + j) % a.sa]);
+                cnt += 2 * pairs;
             }
         }
     }
@@ -290,13 +373,37 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, FusedArgs a) {
     }
 }
 
+// Pre-pass: for every output row of the layer, where its own representation lives and which
+// entries it aggregates.  One thread per row, full occupancy; the fused kernel then needs a single
+// coalesced load per row instead of a chain of dependent look-ups.
+template <bool FIRST>
+__global__ void __launch_bounds__(256) k_layer_rows(FusedArgs a, int4* __restrict__ row_meta) {
+    for (int64_t r = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; r < a.M; r += (int64_t)gridDim.x * blockDim.x) {
+        const int b = upper_segment(a.rowbase_out, a.B + 1, (int32_t)r);
+        const int32_t l = (int32_t)r - a.rowbase_out[b];
+        const int32_t* cum = a.cum + b * (a.k + 2);
+        int h = 0;
+        while (h < a.k - a.layer && l >= cum[h + 1]) ++h;
+        const int32_t idx = a.node_off[h * (a.B + 1) + b] + (l - cum[h]);
+        const int32_t e0 = a.ent_off[idx];
+        const int32_t in_base = FIRST ? 0 : a.rowbase_in[b];
+        row_meta[r] = make_int4(source_row<FIRST>(a, in_base, FIRST ? a.nodes[idx] : l), e0, a.ent_off[idx + 1] - e0, in_base);
+    }
+}
+
 __global__ void k_pack_weights(const float* __restrict__ w_cat /*[2 d_in, N]*/, float* __restrict__ w_pad_t /*[N, 2 d_in_pad]*/,
                                int d_in, int d_in_pad, int N) {
     const int K = 2 * d_in_pad;
     const int64_t total = (int64_t)N * K;
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
         const int n = (int)(i / K), kx = (int)(i % K);
-        const int part = kx / d_in_pad, col = kx % d_in_pad;
+        // slice order of the fused kernel: groups of 64 input columns; inside a group (self, mean) pairs of
+        // 32-column blocks
+        const int slice = kx / 32;
+        int grp = 0, rem = slice, pairs = min(kGroupCols / 32, d_in_pad / 32);
+        while (rem >= 2 * pairs) { rem -= 2 * pairs; ++grp; pairs = min(kGroupCols / 32, (d_in_pad - grp * kGroupCols) / 32); }
+        const int part = rem & 1;
+        const int col = grp * kGroupCols + (rem >> 1) * 32 + (kx & 31);
         w_pad_t[i] = col < d_in ? to_tf32(w_cat[(int64_t)(part * d_in + col) * N + n]) : 0.f;
     }
 }
@@ -326,6 +433,11 @@ int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_ou
     a.cum = d->cum; a.node_off = d->node_off; a.nodes = d->nodes;
     a.ent_off = d->ent_off; a.ent_nbrs = d->ent_nbrs; a.ent_repr = d->ent_repr;
     a.h_prev = h_prev;
+    a.src_base = layer == 1 ? ctx->slots : reinterpret_cast<const char*>(h_prev);
+    a.src_row_bytes = layer == 1 ? ctx->row_bytes : (int64_t)d_in * 4;
+    a.identity_rows = 1;
+    for (int p = 0; p < ctx->n_parts; ++p)
+        if (ctx->slot_of_part[p] >= 0 && ctx->slot_of_part[p] != p) a.identity_rows = 0;
     a.slots = ctx->slots; a.slot_of_part = ctx->d_slot_of_part;
     a.slot_bytes = ctx->slot_bytes; a.row_bytes = ctx->row_bytes; a.part_size = (uint32_t)ctx->part_size;
     a.d_in = d_in;
@@ -335,20 +447,33 @@ int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_ou
     a.M = M;
     a.relu = relu ? 1 : 0;
     a.bias = bias; a.out = h_out; a.error = ctx->d_flags;
+    a.dbg = getenv("MG_FUSED_DEBUG") ? atoi(getenv("MG_FUSED_DEBUG")) : 0;
     int stride = 32;
     while (stride < a.BN) stride <<= 1;
     a.tmem_cols = 2 * stride;   // two accumulator buffers, each a power of two >= 32 columns
     const int b_bytes = a.BN * KC * 4;
     const int n_chunks = 2 * a.d_in_pad / KC;
-    a.sa = std::min(kMaxStages, std::max(2, std::min(n_chunks, 5)));
-    a.sb = std::max(2, std::min({kMaxStages, n_chunks, (int)((212 * 1024 - a.sa * (int)kABytes) / b_bytes)}));
+    a.sa = std::min(8, n_chunks);   // two groups of (self, mean) slice pairs, 64 input columns each
+    a.sb = std::max(2, std::min({kMaxStages, n_chunks, (int)((194 * 1024 - a.sa * (int)kABytes) / b_bytes)}));
     const size_t smem = (size_t)a.sa * kABytes + (size_t)a.sb * b_bytes + 1024;
     CUtensorMap mw;
     if (!make_map_f32(&mw, w_pad_t, d_out, 2 * a.d_in_pad, a.BN))
         return mg_fail(ctx, MG_ERR_CUDA, "cuTensorMapEncodeTiled failed for the layer weights");
     const bool first = layer == 1, half = first && ctx->feat_dtype == MG_DTYPE_F16;
     auto kern = first ? (half ? k_sage_layer_fused<true, true> : k_sage_layer_fused<true, false>) : k_sage_layer_fused<false, false>;
-    MG_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 216 * 1024));
+    MG_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    {
+        size_t have = ctx->ws_x_bytes / sizeof(int4);
+        int4* buf = reinterpret_cast<int4*>(ctx->ws_x);
+        int rc = mg_ensure(ctx, &buf, &have, (size_t)M);
+        ctx->ws_x = reinterpret_cast<float*>(buf);
+        ctx->ws_x_bytes = have * sizeof(int4);
+        if (rc) return rc;
+        a.row_meta = buf;
+        if (first) k_layer_rows<true><<<mg_grid(ctx, 8), 256, 0, ctx->stream>>>(a, buf);
+        else k_layer_rows<false><<<mg_grid(ctx, 8), 256, 0, ctx->stream>>>(a, buf);
+        ctx->launches++;
+    }
     const int64_t n_tiles = (M + BM - 1) / BM;
     const int grid = (int)std::min<int64_t>(n_tiles, ctx->n_sms);
     kern<<<grid, kFusedThreads, smem, ctx->stream>>>(mw, a);

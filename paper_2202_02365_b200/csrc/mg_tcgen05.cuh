@@ -101,6 +101,30 @@ __device__ __forceinline__ float to_tf32(float v) {
     return __uint_as_float(u);
 }
 
+// Epilogue of one 32-column slice of an accumulator tile.  After tcgen05.ld every lane holds 32
+// consecutive columns of ITS row; storing that directly would touch 32 different rows per
+// instruction.  The slice is transposed through a warp-private padded shared-memory tile so that
+// each store instruction writes one 128-byte row segment.  stage: 32 x 33 floats per warp.
+__device__ __forceinline__ void store_slice_coalesced(const uint32_t* v, float* stage, const float* __restrict__ bias,
+                                                      float* __restrict__ out, int64_t row0, int64_t M, int N, int c0,
+                                                      bool relu) {
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) stage[lane * 33 + j] = __uint_as_float(v[j]);
+    __syncwarp();
+    const int n = c0 + lane;
+    if (n < N) {
+        const float b = __ldg(bias + n);
+        const int rows = (int)min((int64_t)32, M - row0);
+        for (int rr = 0; rr < rows; ++rr) {
+            float o = stage[rr * 33 + lane] + b;
+            if (relu) o = fmaxf(o, 0.f);
+            out[(row0 + rr) * N + n] = o;
+        }
+    }
+    __syncwarp();
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
