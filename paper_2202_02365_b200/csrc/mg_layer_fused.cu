@@ -16,7 +16,6 @@
 #include <cuda_fp16.h>
 
 #include <algorithm>
-#include <cstdlib>
 
 #include "mg_device.cuh"
 #include "mg_internal.cuh"
@@ -33,6 +32,8 @@ constexpr int kFirstProducerWarp = 6; // warp 0 TMA, warp 1 MMA + tensor memory,
 constexpr int kFusedThreads = (kFirstProducerWarp + kProducerWarps) * 32;  // 704
 constexpr int kMaxStages = 8;
 constexpr int kGroupCols = 128;                  // input columns whose (self, mean) slices the producers fill together
+constexpr int kLanesPerRow = kGroupCols / 4;     // lanes covering one row segment with 16-byte loads
+constexpr int kRowsPerInstr = 32 / kLanesPerRow; // rows one warp-wide load instruction covers
 constexpr int kRowsInFlight = 2;                 // rows a producer warp builds at the same time
 constexpr int kUnroll = 5;                       // neighbour rows per output row fetched before the first add
 constexpr uint32_t kABytes = BM * KC * 4;  // 16 KiB per A stage
@@ -68,7 +69,6 @@ struct FusedArgs {
     const float* bias;
     float* out;                  // [M, N]
     uint32_t* error;
-    int32_t dbg;
 };
 
 constexpr int kKeyCap = 2048;   // source-row indices of a tile's entries cached in shared memory
@@ -177,7 +177,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, FusedArgs a) {
                     const uint64_t db = smem_desc_sw128(smem_u32(b_base + (size_t)sb * b_bytes));
 #pragma unroll
                     for (int kk = 0; kk < KC / 8; ++kk)
-                        if (!(a.dbg & 4)) mma_tf32(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (c | kk) ? 1u : 0u);
+                        mma_tf32(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (c | kk) ? 1u : 0u);
                     mma_commit(&a_empty[sa]);
                     mma_commit(&b_empty[sb]);
                 }
@@ -199,7 +199,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, FusedArgs a) {
                 uint32_t v[32];
                 tmem_ld_32(tmem_base + buf * acc_stride + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)c0, v);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (row0 < a.M && !(a.dbg & 2)) store_slice_coalesced(v, out_stage[lane_group], a.bias, a.out, row0, a.M, a.N, c0, a.relu != 0);
+                if (row0 < a.M) store_slice_coalesced(v, out_stage[lane_group], a.bias, a.out, row0, a.M, a.N, c0, a.relu != 0);
             }
             tc_fence_before();
             __syncwarp();
@@ -266,24 +266,25 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, FusedArgs a) {
             const int n_groups = (a.d_in_pad + kGroupCols - 1) / kGroupCols;
             for (int grp = 0; grp < n_groups; ++grp) {
                 const int pairs = min(kGroupCols / KC, (a.d_in_pad - grp * kGroupCols) / KC);   // slice pairs in this group
-                const int col = grp * kGroupCols + lane * 4;
-                const bool lane_on = (lane >> 3) < pairs;
+                const int sub = lane / kLanesPerRow, ll = lane % kLanesPerRow;
+                const int col = grp * kGroupCols + ll * 4;
+                const bool lane_on = (ll >> 3) < pairs;
                 const bool col_ok = lane_on && col < a.d_in;
                 const char* src = a.src_base + (size_t)col * (HALF ? 2 : 4);
                 bool waited = false;
-                for (int rr = 0; rr < kRowsPerWarp; rr += kRowsInFlight) {
-                    const int row0 = pw * kRowsPerWarp + rr;
+                for (int rr = 0; rr < kRowsPerWarp; rr += kRowsInFlight * kRowsPerInstr) {
+                    const int row0 = pw * kRowsPerWarp + rr + sub;   // this lane's rows: row0 + q * kRowsPerInstr
                     RowMeta mq[kRowsInFlight];
                     float4 selfv[kRowsInFlight], acc[kRowsInFlight];
                     int top = 0;
 #pragma unroll
                     for (int q = 0; q < kRowsInFlight; ++q) {
-                        mq[q] = meta[row0 + q];
+                        mq[q] = meta[row0 + q * kRowsPerInstr];
                         selfv[q] = make_float4(0.f, 0.f, 0.f, 0.f);
                         acc[q] = selfv[q];
                         top = max(top, mq[q].cnt);
                     }
-                    if (col_ok && !(a.dbg & 1)) {
+                    if (col_ok) {
 #pragma unroll
                         for (int q = 0; q < kRowsInFlight; ++q)
                             selfv[q] = load4<HALF>(src + (size_t)(uint32_t)mq[q].self_src * a.src_row_bytes);
@@ -345,12 +346,12 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, FusedArgs a) {
                     }
                     if (ok && lane_on) {
                         // K-major, 128-byte swizzle: 16-byte slot gl of row r lands in slot gl ^ (r % 8)
-                        const uint32_t s_self = (cnt + 2 * (lane >> 3)) % a.sa, s_mean = (cnt + 2 * (lane >> 3) + 1) % a.sa;
+                        const uint32_t s_self = (cnt + 2 * (ll >> 3)) % a.sa, s_mean = (cnt + 2 * (ll >> 3) + 1) % a.sa;
                         uint8_t* stage_self = a_base + (size_t)s_self * kABytes;
                         uint8_t* stage_mean = a_base + (size_t)s_mean * kABytes;
 #pragma unroll
                         for (int q = 0; q < kRowsInFlight; ++q) {
-                            const int row = row0 + q;
+                            const int row = row0 + q * kRowsPerInstr;
                             const size_t off = (size_t)(row >> 3) * 1024 + (size_t)(row & 7) * 128 + (size_t)((gl ^ (row & 7)) << 4);
                             *reinterpret_cast<float4*>(stage_self + off) = selfv[q];
                             *reinterpret_cast<float4*>(stage_mean + off) = acc[q];
@@ -447,7 +448,6 @@ int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_ou
     a.M = M;
     a.relu = relu ? 1 : 0;
     a.bias = bias; a.out = h_out; a.error = ctx->d_flags;
-    a.dbg = getenv("MG_FUSED_DEBUG") ? atoi(getenv("MG_FUSED_DEBUG")) : 0;
     int stride = 32;
     while (stride < a.BN) stride <<= 1;
     a.tmem_cols = 2 * stride;   // two accumulator buffers, each a power of two >= 32 columns
