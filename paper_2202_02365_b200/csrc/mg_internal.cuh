@@ -124,6 +124,8 @@ struct mg_dense {
     int32_t* nodes = nullptr;       // [cap_nodes] hop-major, batch-major inside a hop
     int32_t* node_batch = nullptr;  // [cap_nodes]
     int32_t* ent_off = nullptr;     // [cap_nodes + 1] start of each sampled node's entries
+    int64_t* node_r0 = nullptr;     // [cap_nodes] start of the node's row in the in-buffer view
+    uint32_t* node_deg = nullptr;   // [cap_nodes] its (resident) degree
     int32_t* ent_nbrs = nullptr;    // [cap_entries] neighbour ids
     int32_t* ent_repr = nullptr;    // [cap_entries] neighbour's local row in its batch
     int32_t* node_off = nullptr;    // [(k+1) * (B+1)] arena index where batch b's hop-h nodes start

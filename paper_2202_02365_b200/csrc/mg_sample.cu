@@ -152,13 +152,16 @@ k_init_targets(DenseHeader* hdr, const int32_t* __restrict__ targets, int32_t n_
 // -------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads)
 k_count(const DenseHeader* hdr, int hop, int32_t fanout, const int32_t* __restrict__ nodes,
-        const int64_t* __restrict__ row_off, int32_t* ent_off) {
+        const int64_t* __restrict__ row_off, int32_t* ent_off, int64_t* node_r0, uint32_t* node_deg) {
     if (hdr->status) return;
     const int32_t lo = hdr->hop_base[hop], hi = hdr->hop_base[hop + 1];
     for (int32_t i = lo + blockIdx.x * blockDim.x + threadIdx.x; i < hi; i += gridDim.x * blockDim.x) {
         const int32_t v = nodes[i];
-        const int64_t d = row_off[v + 1] - row_off[v];
+        const int64_t r0 = row_off[v];
+        const int64_t d = row_off[v + 1] - r0;
         ent_off[i] = (int32_t)(d < (int64_t)fanout ? d : (int64_t)fanout);
+        node_r0[i] = r0;        // the one random look-up of the row bounds; k_pick reads these coalesced
+        node_deg[i] = (uint32_t)d;
     }
 }
 
@@ -178,60 +181,25 @@ struct PickArgs {
     int32_t fanout;
     const int32_t* nodes;
     const int32_t* node_batch;
-    const int64_t* row_off;
+    const int64_t* node_r0;
+    const uint32_t* node_deg;
     const int32_t* row_nbrs;
     const int32_t* ent_off;
     int32_t* ent_nbrs;
-    int32_t* ent_repr;  // receives batch * table_size + slot until k_relabel
-    int32_t* hkeys;
-    TableGeom tg;
+    int32_t* ent_repr;  // receives the batch id of the entry (k_insert turns it into the id-table slot)
     const uint64_t* seeds;
-    uint64_t* newlist;
-    int64_t cap_new;
-    int id_bits;
 };
 
-// Appends this block's new composite keys to the list: one global atomic per block call.
-__device__ __forceinline__ void block_append(const PickArgs& a, bool is_new, uint64_t key, uint32_t* sm_cnt /*[2]*/) {
-    const int lane = threadIdx.x & 31;
-    if (threadIdx.x == 0) sm_cnt[0] = 0;
-    __syncthreads();
-    const uint32_t bal = __ballot_sync(0xFFFFFFFFu, is_new);
-    uint32_t warp_off = 0;
-    if (lane == 0 && bal) warp_off = atomicAdd(&sm_cnt[0], __popc(bal));
-    warp_off = __shfl_sync(0xFFFFFFFFu, warp_off, 0);
-    __syncthreads();
-    if (threadIdx.x == 0) sm_cnt[1] = sm_cnt[0] ? atomicAdd(&a.hdr->n_new, sm_cnt[0]) : 0u;
-    __syncthreads();
-    if (is_new) {
-        const int64_t pos = (int64_t)sm_cnt[1] + warp_off + __popc(bal & ((1u << lane) - 1u));
-        if (pos < a.cap_new) a.newlist[pos] = key;
-        else atomicOr(&a.hdr->status, ST_CAP_NODES);
-    }
-    __syncthreads();
-}
-
-__device__ __forceinline__ void insert_pick(const PickArgs& a, bool valid, int32_t b, int32_t u, int32_t out_pos,
-                                            bool* is_new, uint64_t* key) {
-    *is_new = false;
-    *key = 0;
+// A pick goes to its place in the entry arena; ent_repr carries the batch id until k_insert replaces it.
+__device__ __forceinline__ void store_pick(const PickArgs& a, bool valid, int32_t b, int32_t u, int32_t out_pos) {
     if (!valid) return;
     a.ent_nbrs[out_pos] = u;
-    bool fresh;
-    const int32_t slot = table_insert(a.hkeys + (int64_t)b * a.tg.size, a.tg.size, a.tg.shift, u, &fresh);
-    if (slot < 0) { atomicOr(&a.hdr->status, ST_CAP_TABLE); a.ent_repr[out_pos] = 0; return; }
-    a.ent_repr[out_pos] = b * a.tg.size + slot;
-    if (fresh) {
-        *is_new = true;
-        *key = (uint64_t)(uint32_t)slot | ((uint64_t)(uint32_t)u << MG_SLOT_BITS) |
-               ((uint64_t)(uint32_t)b << (MG_SLOT_BITS + a.id_bits));
-    }
+    a.ent_repr[out_pos] = b;
 }
 
 // G lanes per node, fanout <= G <= 32.
 template <int G>
 __global__ void __launch_bounds__(kThreads) k_pick(PickArgs a) {
-    __shared__ uint32_t sm_cnt[2];
     if (a.hdr->status) return;
     constexpr int kGroups = kThreads / G;
     const int32_t lo = a.hdr->hop_base[a.hop], hi = a.hdr->hop_base[a.hop + 1];
@@ -249,8 +217,8 @@ __global__ void __launch_bounds__(kThreads) k_pick(PickArgs a) {
             v = a.nodes[i];
             b = a.node_batch[i];
             out0 = a.ent_off[i];
-            r0 = a.row_off[v];
-            d = a.row_off[v + 1] - r0;
+            r0 = a.node_r0[i];
+            d = (int64_t)a.node_deg[i];
         }
         bool valid = false;
         int32_t u = 0, pos = 0;
@@ -286,16 +254,12 @@ __global__ void __launch_bounds__(kThreads) k_pick(PickArgs a) {
             u = a.row_nbrs[r0 + gl];
             pos = out0 + gl;
         }
-        bool is_new;
-        uint64_t key;
-        insert_pick(a, valid, b, u, pos, &is_new, &key);
-        block_append(a, is_new, key, sm_cnt);
+        store_pick(a, valid, b, u, pos);
     }
 }
 
 // Any fanout up to MG_MAX_FANOUT: one warp per node, picks staged in shared memory.
 __global__ void __launch_bounds__(kThreads) k_pick_wide(PickArgs a) {
-    __shared__ uint32_t sm_cnt[2];
     extern __shared__ uint32_t sm_dyn[];  // per warp: x[f], pick[f]
     if (a.hdr->status) return;
     constexpr int kWarps = kThreads / 32;
@@ -314,8 +278,8 @@ __global__ void __launch_bounds__(kThreads) k_pick_wide(PickArgs a) {
             v = a.nodes[i];
             b = a.node_batch[i];
             out0 = a.ent_off[i];
-            r0 = a.row_off[v];
-            d = a.row_off[v + 1] - r0;
+            r0 = a.node_r0[i];
+            d = (int64_t)a.node_deg[i];
         }
         const bool floyd = node_ok && d > (int64_t)f;
         if (floyd) {
@@ -333,7 +297,6 @@ __global__ void __launch_bounds__(kThreads) k_pick_wide(PickArgs a) {
                 __syncwarp();
             }
         }
-        // every warp of the block runs the same number of append rounds
         for (int rd = 0; rd < rounds; ++rd) {
             const int t = rd * 32 + lane;
             bool valid = false;
@@ -350,12 +313,93 @@ __global__ void __launch_bounds__(kThreads) k_pick_wide(PickArgs a) {
                 u = a.row_nbrs[r0 + t];
                 pos = out0 + t;
             }
-            bool is_new;
-            uint64_t key;
-            insert_pick(a, valid, b, u, pos, &is_new, &key);
-            block_append(a, is_new, key, sm_cnt);
+            store_pick(a, valid, b, u, pos);
         }
         __syncwarp();
+    }
+}
+
+// Deduplication: every entry's neighbour id goes into its batch's id table.  One thread owns eight
+// entries; their first-probe compare-and-swaps are issued back to back (eight atomics in flight per
+// thread), collisions are resolved afterwards.  The keys of the ids that were new are appended to the
+// list with one global atomic per 2048 entries.
+struct InsertArgs {
+    DenseHeader* hdr;
+    int hop;
+    const int32_t* ent_nbrs;
+    int32_t* ent_repr;   // in: batch id; out: batch * table_size + slot
+    int32_t* hkeys;
+    TableGeom tg;
+    uint64_t* newlist;
+    int64_t cap_new;
+    int id_bits;
+};
+
+constexpr int kInsertPerThread = 8;
+
+__global__ void __launch_bounds__(kThreads) k_insert(InsertArgs a) {
+    __shared__ uint32_t warp_tot[kThreads / 32 + 1];
+    __shared__ uint32_t block_base;
+    if (a.hdr->status) return;
+    const int32_t lo = a.hdr->ent_base[a.hop], hi = a.hdr->ent_base[a.hop + 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr int kChunk = kThreads * kInsertPerThread;
+    const uint32_t mask = (uint32_t)a.tg.size - 1u;
+    for (int32_t base = lo + blockIdx.x * kChunk; base < hi; base += gridDim.x * kChunk) {
+        int32_t u[kInsertPerThread], b[kInsertPerThread], old[kInsertPerThread];
+        uint32_t slot[kInsertPerThread];
+#pragma unroll
+        for (int j = 0; j < kInsertPerThread; ++j) {
+            const int32_t e = base + j * kThreads + threadIdx.x;
+            u[j] = -1; b[j] = 0; old[j] = 0; slot[j] = 0;
+            if (e < hi) { u[j] = a.ent_nbrs[e]; b[j] = a.ent_repr[e]; }
+        }
+#pragma unroll
+        for (int j = 0; j < kInsertPerThread; ++j)
+            if (u[j] >= 0) {
+                slot[j] = table_hash(u[j], a.tg.shift);
+                old[j] = atomicCAS(&a.hkeys[(int64_t)b[j] * a.tg.size + slot[j]], -1, u[j]);
+            }
+        uint32_t n_mine = 0, new_bits = 0;
+#pragma unroll
+        for (int j = 0; j < kInsertPerThread; ++j) {
+            if (u[j] < 0) continue;
+            bool fresh = old[j] == -1;
+            if (!fresh && old[j] != u[j]) {   // first slot taken by another id: linear probing
+                int32_t* keys = a.hkeys + (int64_t)b[j] * a.tg.size;
+                int32_t probe = 1;
+                for (; probe < a.tg.size; ++probe) {
+                    slot[j] = (slot[j] + 1u) & mask;
+                    const int32_t o = atomicCAS(&keys[slot[j]], -1, u[j]);
+                    if (o == -1) { fresh = true; break; }
+                    if (o == u[j]) break;
+                }
+                if (probe >= a.tg.size) { atomicOr(&a.hdr->status, ST_CAP_TABLE); slot[j] = 0; }
+            }
+            a.ent_repr[base + j * kThreads + threadIdx.x] = b[j] * a.tg.size + (int32_t)slot[j];
+            if (fresh) { new_bits |= 1u << j; ++n_mine; }
+        }
+        // block-wide exclusive scan of the per-thread counts, one global atomic for the block
+        const uint32_t inc = warp_incl_scan(n_mine);
+        if (lane == 31) warp_tot[warp] = inc;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint32_t run = 0;
+            for (int w = 0; w < kThreads / 32; ++w) { const uint32_t t = warp_tot[w]; warp_tot[w] = run; run += t; }
+            block_base = run ? atomicAdd(&a.hdr->n_new, run) : 0u;
+        }
+        __syncthreads();
+        int64_t pos = (int64_t)block_base + warp_tot[warp] + inc - n_mine;
+#pragma unroll
+        for (int j = 0; j < kInsertPerThread; ++j)
+            if (new_bits & (1u << j)) {
+                const uint64_t key = (uint64_t)slot[j] | ((uint64_t)(uint32_t)u[j] << MG_SLOT_BITS) |
+                                     ((uint64_t)(uint32_t)b[j] << (MG_SLOT_BITS + a.id_bits));
+                if (pos < a.cap_new) a.newlist[pos] = key;
+                else atomicOr(&a.hdr->status, ST_CAP_NODES);
+                ++pos;
+            }
+        __syncthreads();
     }
 }
 
@@ -647,6 +691,8 @@ static int dense_alloc(mg_ctx* ctx, mg_dense* d, int32_t B, int32_t k, int64_t c
         if ((rc = dev_realloc(ctx, &d->nodes, (size_t)cap_nodes))) return rc;
         if ((rc = dev_realloc(ctx, &d->node_batch, (size_t)cap_nodes))) return rc;
         if ((rc = dev_realloc(ctx, &d->ent_off, (size_t)cap_nodes + 1))) return rc;
+        if ((rc = dev_realloc(ctx, &d->node_r0, (size_t)cap_nodes))) return rc;
+        if ((rc = dev_realloc(ctx, &d->node_deg, (size_t)cap_nodes))) return rc;
         if ((rc = dev_realloc(ctx, &d->newlist[0], (size_t)cap_nodes))) return rc;
         if ((rc = dev_realloc(ctx, &d->newlist[1], (size_t)cap_nodes))) return rc;
         const int64_t sort_tiles = (cap_nodes + kSortTile - 1) / kSortTile;
@@ -810,7 +856,7 @@ extern "C" int mg_sample_many(mg_ctx* ctx, const int32_t* targets, int targets_o
         const int32_t f = fanouts[h];
         {
             ProfScope ps(ctx, PH_SAMPLE_COUNT, 1);
-            k_count<<<grid, kThreads, 0, st>>>(d->hdr, h, f, d->nodes, ctx->view_off, d->ent_off);
+            k_count<<<grid, kThreads, 0, st>>>(d->hdr, h, f, d->nodes, ctx->view_off, d->ent_off, d->node_r0, d->node_deg);
         }
         {
             ProfScope ps(ctx, PH_SAMPLE_SCAN, 4);
@@ -820,13 +866,16 @@ extern "C" int mg_sample_many(mg_ctx* ctx, const int32_t* targets, int targets_o
         }
         {
             ProfScope ps(ctx, PH_SAMPLE_PICK, 1);
-            PickArgs a{d->hdr, h, f, d->nodes, d->node_batch, ctx->view_off, ctx->view_nbrs, d->ent_off, d->ent_nbrs,
-                       d->ent_repr, d->hkeys, tg, d->d_seeds, d->newlist[0], d->cap_nodes, id_bits};
+            PickArgs a{d->hdr, h, f, d->nodes, d->node_batch, d->node_r0, d->node_deg, ctx->view_nbrs, d->ent_off, d->ent_nbrs,
+                       d->ent_repr, d->d_seeds};
             if (f <= 4) k_pick<4><<<grid, kThreads, 0, st>>>(a);
             else if (f <= 8) k_pick<8><<<grid, kThreads, 0, st>>>(a);
             else if (f <= 16) k_pick<16><<<grid, kThreads, 0, st>>>(a);
             else if (f <= 32) k_pick<32><<<grid, kThreads, 0, st>>>(a);
             else k_pick_wide<<<grid, kThreads, (size_t)(kThreads / 32) * 2 * f * sizeof(uint32_t), st>>>(a);
+            InsertArgs ia{d->hdr, h, d->ent_nbrs, d->ent_repr, d->hkeys, tg, d->newlist[0], d->cap_nodes, id_bits};
+            k_insert<<<grid, kThreads, 0, st>>>(ia);
+            ctx->launches++;
         }
         int res_buf = 0;
         {
@@ -954,7 +1003,7 @@ extern "C" int mg_dense_view(mg_ctx* ctx, mg_dense* d, int32_t batch, mg_dense_a
 extern "C" int mg_dense_free(mg_dense* d) {
     if (!d) return MG_OK;
     cudaSetDevice(d->device);
-    cudaFree(d->hdr); cudaFree(d->nodes); cudaFree(d->node_batch); cudaFree(d->ent_off);
+    cudaFree(d->hdr); cudaFree(d->nodes); cudaFree(d->node_batch); cudaFree(d->ent_off); cudaFree(d->node_r0); cudaFree(d->node_deg);
     cudaFree(d->ent_nbrs); cudaFree(d->ent_repr); cudaFree(d->node_off); cudaFree(d->cum);
     cudaFree(d->rowbase); cudaFree(d->hkeys); cudaFree(d->hvals); cudaFree(d->newlist[0]);
     cudaFree(d->newlist[1]); cudaFree(d->d_seeds); cudaFree(d->scan_tmp); cudaFree(d->sort_hist);
