@@ -223,9 +223,10 @@ struct SortParams {   // device-resident
     int32_t zero;
     int32_t n;        // keys
     int32_t ntiles;   // ceil(n / 4096)
-    int32_t hist_len; // 256 * ntiles
+    int32_t hist_len; // bins * ntiles
 };
 size_t mg_sort_hist_elems(int64_t max_keys);
+void mg_sort_params_host(SortParams* sp, int64_t n);
 size_t mg_scan_tmp_elems(int64_t max_elems);
 void mg_sort_u64(mg_ctx* ctx, uint64_t* const buf[2], const SortParams* sp, int lo_bit, int bits, uint32_t* hist,
                  uint32_t* scan_tmp, int* res_buf);

@@ -200,7 +200,7 @@ extern "C" int mg_lp_prepare(mg_ctx* ctx, const int32_t* src, const int32_t* rel
     if (!ok) { cudaGetLastError(); cleanup(); mg_lp_free(lp); return mg_fail(ctx, MG_ERR_OOM, "allocation of the link-prediction batch failed"); }
 
     SortParams h_sp;
-    h_sp.zero = 0; h_sp.n = (int32_t)total; h_sp.ntiles = (int32_t)((total + 4095) / 4096); h_sp.hist_len = 256 * h_sp.ntiles;
+    mg_sort_params_host(&h_sp, total);
     cudaMemcpyAsync(sp, &h_sp, sizeof(h_sp), cudaMemcpyHostToDevice, st);
     cudaMemcpyAsync(d_src, src, 4 * n_edges, cudaMemcpyHostToDevice, st);
     cudaMemcpyAsync(d_dst, dst, 4 * n_edges, cudaMemcpyHostToDevice, st);

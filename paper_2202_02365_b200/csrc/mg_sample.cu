@@ -408,43 +408,62 @@ __global__ void __launch_bounds__(kThreads) k_insert(InsertArgs a) {
 // -------------------------------------------------------------------------------------
 constexpr int kSortKeysPerThread = 16;
 constexpr int kSortTile = kThreads * kSortKeysPerThread;  // 4096
+constexpr int kRadixBits = 9;                              // 34 key bits (27 id + 7 batch) take four passes
+constexpr int kBins = 1 << kRadixBits;
+constexpr int kBinsPerThread = kBins / kThreads;
 
 __global__ void k_sort_setup(const DenseHeader* hdr, SortParams* sp) {
     const int32_t n = hdr->status ? 0 : (int32_t)hdr->n_new;
     sp->zero = 0;
     sp->n = n;
     sp->ntiles = (n + kSortTile - 1) / kSortTile;
-    sp->hist_len = 256 * sp->ntiles;
+    sp->hist_len = kBins * sp->ntiles;
 }
 
 __global__ void __launch_bounds__(kThreads)
 k_radix_hist(const uint64_t* __restrict__ keys, const SortParams* sp, int shift, uint32_t* hist) {
-    __shared__ uint32_t sh[256];
+    __shared__ uint32_t sh[kBins];
     const int32_t n = sp->n, ntiles = sp->ntiles;
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x) {
-        sh[threadIdx.x] = 0;
+#pragma unroll
+        for (int q = 0; q < kBinsPerThread; ++q) sh[threadIdx.x + q * kThreads] = 0;
         __syncthreads();
         const int32_t tb = t * kSortTile;
 #pragma unroll 4
         for (int j = 0; j < kSortKeysPerThread; ++j) {
             const int32_t i = tb + j * kThreads + threadIdx.x;
-            if (i < n) atomicAdd(&sh[(uint32_t)(keys[i] >> shift) & 255u], 1u);
+            if (i < n) atomicAdd(&sh[(uint32_t)(keys[i] >> shift) & (kBins - 1)], 1u);
         }
         __syncthreads();
-        hist[(size_t)threadIdx.x * ntiles + t] = sh[threadIdx.x];
+#pragma unroll
+        for (int q = 0; q < kBinsPerThread; ++q) {
+            const int bin = threadIdx.x + q * kThreads;
+            hist[(size_t)bin * ntiles + t] = sh[bin];
+        }
         __syncthreads();
     }
 }
 
+// One stable counting pass.  A tile's keys are ranked per digit (warp by warp, 32 keys at a time with
+// match_any), laid out digit by digit in shared memory, and written from there, so that every run of
+// equal digits leaves the SM as consecutive addresses.
 __global__ void __launch_bounds__(kThreads)
 k_radix_scatter(const uint64_t* __restrict__ keys, uint64_t* __restrict__ out, const SortParams* sp, int shift,
                 const uint32_t* __restrict__ hist_scanned) {
-    __shared__ uint32_t cnt[kThreads / 32][256];
+    extern __shared__ __align__(16) uint8_t sort_smem[];
+    uint64_t* stage = reinterpret_cast<uint64_t*>(sort_smem);                          // [kSortTile]
+    uint32_t (*cnt)[kBins] = reinterpret_cast<uint32_t (*)[kBins]>(stage + kSortTile);   // [warps][kBins]
+    uint32_t* tile_base = reinterpret_cast<uint32_t*>(cnt + kThreads / 32);             // [kBins] first slot of a digit in the tile
+    uint32_t* glob_base = tile_base + kBins;                                            // [kBins] first output position
+    __shared__ uint32_t warp_tot[kThreads / 32];
     const int32_t n = sp->n, ntiles = sp->ntiles;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    constexpr int kPerWarp = kSortTile / (kThreads / 32);  // 512 consecutive keys per warp
+    constexpr int kWarps = kThreads / 32;
+    constexpr int kPerWarp = kSortTile / kWarps;  // 512 consecutive keys per warp
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x) {
-        for (int w = 0; w < kThreads / 32; ++w) cnt[w][threadIdx.x] = 0;
+        for (int w = 0; w < kWarps; ++w)
+#pragma unroll
+            for (int q = 0; q < kBinsPerThread; ++q) cnt[w][threadIdx.x + q * kThreads] = 0;
         __syncthreads();
         uint64_t key[kSortKeysPerThread];
         uint32_t rank[kSortKeysPerThread];
@@ -454,7 +473,7 @@ k_radix_scatter(const uint64_t* __restrict__ keys, uint64_t* __restrict__ out, c
             const int32_t i = wb + r * 32 + lane;
             const bool ok = i < n;
             key[r] = ok ? keys[i] : 0ull;
-            const uint32_t dg = ok ? ((uint32_t)(key[r] >> shift) & 255u) : 0xFFFFFFFFu;
+            const uint32_t dg = ok ? ((uint32_t)(key[r] >> shift) & (kBins - 1)) : 0xFFFFFFFFu;
             const uint32_t peers = __match_any_sync(0xFFFFFFFFu, dg);
             const int leader = __ffs(peers) - 1;
             uint32_t old = 0;
@@ -467,23 +486,49 @@ k_radix_scatter(const uint64_t* __restrict__ keys, uint64_t* __restrict__ out, c
             __syncwarp();
         }
         __syncthreads();
-        {   // turn per-warp counts of digit `threadIdx.x` into global start positions
-            uint32_t run = hist_scanned[(size_t)threadIdx.x * ntiles + t];
-            for (int w = 0; w < kThreads / 32; ++w) {
-                const uint32_t c = cnt[w][threadIdx.x];
-                cnt[w][threadIdx.x] = run;
-                run += c;
-            }
+        // per digit: prefix over the warps, total in the tile; then an exclusive scan over the digits
+        uint32_t mine[kBinsPerThread], sum = 0;
+#pragma unroll
+        for (int q = 0; q < kBinsPerThread; ++q) {
+            const int bin = threadIdx.x * kBinsPerThread + q;   // consecutive bins per thread: scan order = bin order
+            uint32_t run = 0;
+            for (int w = 0; w < kWarps; ++w) { const uint32_t c = cnt[w][bin]; cnt[w][bin] = run; run += c; }
+            mine[q] = run;
+            sum += run;
+        }
+        const uint32_t inc = warp_incl_scan(sum);
+        if (lane == 31) warp_tot[warp] = inc;
+        __syncthreads();
+        uint32_t before = inc - sum;
+        for (int w = 0; w < warp; ++w) before += warp_tot[w];
+#pragma unroll
+        for (int q = 0; q < kBinsPerThread; ++q) {
+            const int bin = threadIdx.x * kBinsPerThread + q;
+            tile_base[bin] = before;
+            glob_base[bin] = hist_scanned[(size_t)bin * ntiles + t];
+            before += mine[q];
         }
         __syncthreads();
 #pragma unroll
         for (int r = 0; r < kSortKeysPerThread; ++r) {
             const int32_t i = wb + r * 32 + lane;
-            if (i < n) out[cnt[warp][(uint32_t)(key[r] >> shift) & 255u] + rank[r]] = key[r];
+            if (i < n) {
+                const uint32_t dg = (uint32_t)(key[r] >> shift) & (kBins - 1);
+                stage[tile_base[dg] + cnt[warp][dg] + rank[r]] = key[r];
+            }
+        }
+        __syncthreads();
+        const int32_t tile_n = min(kSortTile, n - t * kSortTile);
+        for (int32_t i = threadIdx.x; i < tile_n; i += kThreads) {
+            const uint64_t kx = stage[i];
+            const uint32_t dg = (uint32_t)(kx >> shift) & (kBins - 1);
+            out[glob_base[dg] + ((uint32_t)i - tile_base[dg])] = kx;
         }
         __syncthreads();
     }
 }
+
+constexpr size_t kScatterSmem = (size_t)kSortTile * 8 + (size_t)(kThreads / 32) * kBins * 4 + 2 * (size_t)kBins * 4;
 
 // -------------------------------------------------------------------------------------
 // place the sorted new nodes as the next hop
@@ -630,7 +675,10 @@ int ilog2_ceil(int64_t x) {
 // ---------------------------------------------------------------------------------------
 // generic pieces other translation units use
 // ---------------------------------------------------------------------------------------
-size_t mg_sort_hist_elems(int64_t max_keys) { return (size_t)256 * ((max_keys + kSortTile - 1) / kSortTile) + 256; }
+size_t mg_sort_hist_elems(int64_t max_keys) { return (size_t)kBins * ((max_keys + kSortTile - 1) / kSortTile) + kBins; }
+void mg_sort_params_host(SortParams* sp, int64_t n) {
+    sp->zero = 0; sp->n = (int32_t)n; sp->ntiles = (int32_t)((n + kSortTile - 1) / kSortTile); sp->hist_len = kBins * sp->ntiles;
+}
 size_t mg_scan_tmp_elems(int64_t max_elems) { return (size_t)((max_elems + kScanTile - 1) / kScanTile) + 16; }
 
 // LSD radix sort of 64-bit keys on bits [lo_bit, lo_bit + bits); sp (device) holds the key count.
@@ -639,16 +687,21 @@ void mg_sort_u64(mg_ctx* ctx, uint64_t* const buf[2], const SortParams* sp, int 
                  uint32_t* scan_tmp, int* res_buf) {
     cudaStream_t st = ctx->stream;
     const int grid = mg_grid(ctx, 8);
-    const int passes = (bits + 7) / 8;
+    const int passes = (bits + kRadixBits - 1) / kRadixBits;
     ScanRange r{&sp->zero, &sp->hist_len, nullptr};
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(k_radix_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScatterSmem);
+        attr_set = true;
+    }
     int cur = 0;
     for (int p = 0; p < passes; ++p) {
-        const int shift = lo_bit + 8 * p;
+        const int shift = lo_bit + kRadixBits * p;
         k_radix_hist<<<grid, kThreads, 0, st>>>(buf[cur], sp, shift, hist);
         k_scan_reduce<<<grid, kThreads, 0, st>>>(hist, r, scan_tmp);
         k_scan_tiles<<<1, 1024, 0, st>>>(scan_tmp, r, nullptr);
         k_scan_down<<<grid, kThreads, 0, st>>>(hist, r, scan_tmp);
-        k_radix_scatter<<<grid, kThreads, 0, st>>>(buf[cur], buf[cur ^ 1], sp, shift, hist);
+        k_radix_scatter<<<grid, kThreads, kScatterSmem, st>>>(buf[cur], buf[cur ^ 1], sp, shift, hist);
         cur ^= 1;
     }
     ctx->launches += 5 * passes;
@@ -697,11 +750,11 @@ static int dense_alloc(mg_ctx* ctx, mg_dense* d, int32_t B, int32_t k, int64_t c
         if ((rc = dev_realloc(ctx, &d->newlist[1], (size_t)cap_nodes))) return rc;
         const int64_t sort_tiles = (cap_nodes + kSortTile - 1) / kSortTile;
         const int64_t scan_tiles = std::max<int64_t>((cap_nodes + kScanTile - 1) / kScanTile,
-                                                     (256 * sort_tiles + kScanTile - 1) / kScanTile);
+                                                     (kBins * sort_tiles + kScanTile - 1) / kScanTile);
         d->scan_tmp_elems = (size_t)scan_tiles + 16;
         (void)scan_tiles;
         if ((rc = dev_realloc(ctx, &d->scan_tmp, d->scan_tmp_elems))) return rc;
-        d->sort_hist_elems = (size_t)256 * sort_tiles + 256;
+        d->sort_hist_elems = (size_t)kBins * sort_tiles + kBins;
         if ((rc = dev_realloc(ctx, &d->sort_hist, d->sort_hist_elems))) return rc;
         d->cap_nodes = cap_nodes;
     }
@@ -880,7 +933,7 @@ extern "C" int mg_sample_many(mg_ctx* ctx, const int32_t* targets, int targets_o
         int res_buf = 0;
         {
             const int key_bits = id_bits + b_bits;
-            const int passes = (key_bits + 7) / 8;
+            const int passes = (key_bits + kRadixBits - 1) / kRadixBits;
             ProfScope ps(ctx, PH_SAMPLE_SORT, 1 + passes * 5);
             k_sort_setup<<<1, 1, 0, st>>>(d->hdr, sp);
             mg_sort_u64(ctx, d->newlist, sp, MG_SLOT_BITS, key_bits, d->sort_hist, (uint32_t*)d->scan_tmp, &res_buf);
