@@ -303,3 +303,81 @@ def test_config2_shaped_power_law_three_layers():
         for layer in (1, 2):
             got = ctx.layer_output(model, d, layer, b, outs[layer - 1].shape[0]).cpu().numpy()
             close(got, outs[layer - 1], RTOL_TC)
+
+
+def _check_batches_against_oracle(g_host, feats, layers, fanouts, targets_by_batch, seeds, dense, out, offs, batches, rtol):
+    view = O.GraphView(g_host[0], g_host[1])
+    np_layers = [(w.numpy(), nn.numpy(), b.numpy()) for w, nn, b in layers]
+    for b in batches:
+        ref = O.sample_dense(view, targets_by_batch[b].tolist(), fanouts, seeds[b])
+        assert_dense_equal(dense.view(b), ref)
+        ids = torch.as_tensor(ref["node_ids"], dtype=torch.int64, device=feats.device)
+        want = O.forward(ref, feats[ids].float().cpu().numpy(), np_layers)
+        close(out[offs[b]:offs[b + 1]].cpu().numpy(), want, rtol)
+
+
+def test_full_size_config2_in_bench_launch_configuration():
+    """Config 2 at full size (R-MAT 1M nodes / 20M edges, dim 128, hidden 256, [15, 10, 5], 1000 targets),
+    128 mini-batches per pass as bench.py runs it; three of the batches checked against the oracle."""
+    import bench
+    cfg = bench.CONFIGS["config2_rmat_1m"]
+    g, feats, layers, _ = bench.build_workload(cfg, torch.device("cuda"), seed=0)
+    ctx = mg.Context(0)
+    ctx.load_graph(g.row_offsets, g.nbrs)
+    ctx.load_features(feats)
+    G, T = 128, cfg["batch"]
+    tg = inputs.train_set_batches(cfg["n"], cfg["train"], T, G, seed=100)
+    offs = [T * i for i in range(G + 1)]
+    seeds = list(range(G))
+    d = ctx.sample_many(tg.reshape(-1).cuda(), offs, cfg["fanouts"], seeds)
+    model = ctx.model(layers, mg.GEMM_TF32)
+    out = torch.empty((G * T, cfg["hidden"]), dtype=torch.float32, device="cuda")
+    ctx.forward(model, d, out)
+    g_host = (g.row_offsets.cpu().numpy(), g.nbrs.cpu().numpy())
+    _check_batches_against_oracle(g_host, feats, layers, cfg["fanouts"], tg, seeds, d, out, offs, [0, 77, G - 1], RTOL_TC)
+
+
+def test_full_size_config3_in_bench_launch_configuration():
+    """Config 3 at full size (R-MAT 111M nodes / 1.62B edges, 16 partitions all resident, int64 offsets),
+    128 mini-batches per pass with the capacities bench.py derives; two batches checked against the oracle."""
+    import bench
+    cfg = bench.CONFIGS["config3_papers100m_shaped"]
+    free, _ = torch.cuda.mem_get_info()
+    if free < 150 * (1 << 30):
+        pytest.skip("needs a GPU with 150 GB free")
+    g, feats, layers, _ = bench.build_workload(cfg, torch.device("cuda"), seed=0)
+    ctx = mg.Context(0)
+    ctx.load_graph(g.row_offsets, g.nbrs)
+    g_host = (g.row_offsets.cpu().numpy(), g.nbrs.cpu().numpy())
+    del g
+    torch.cuda.empty_cache()
+    ctx.set_partitioning(cfg["parts"])
+    ctx.load_features(feats, capacity_parts=cfg["parts"])
+    ctx.set_resident(list(range(cfg["parts"])))
+    G, T = 128, cfg["batch"]
+    tg = inputs.train_set_batches(cfg["n"], cfg["train"], T, G, seed=100)
+    offs = [T * i for i in range(G + 1)]
+    seeds = [(1 << 40) + i for i in range(G)]
+    probe = ctx.sample_many(tg.reshape(-1).cuda(), offs, cfg["fanouts"], seeds, caps={"max_nodes_per_batch": 1 << 19})
+    nodes, ents = probe.counts()
+    caps = {"max_nodes_total": int(nodes.sum() * 1.3) + 1024, "max_entries_total": int(ents.sum() * 1.3) + 1024,
+            "max_nodes_per_batch": int(nodes.sum(1).max() * 1.5) + 64}
+    probe.free()
+    d = ctx.sample_many(tg.reshape(-1).cuda(), offs, cfg["fanouts"], seeds, caps=caps)
+    model = ctx.model(layers, mg.GEMM_TF32)
+    out = torch.empty((G * T, cfg["hidden"]), dtype=torch.float32, device="cuda")
+    ctx.forward(model, d, out)
+    _check_batches_against_oracle(g_host, feats, layers, cfg["fanouts"], tg, seeds, d, out, offs, [0, G - 1], RTOL_TC)
+    # properties that hold at any size, on every batch: no duplicate node, every neighbour has a row
+    n2, e2 = d.counts()
+    assert torch.equal(n2, nodes) and torch.equal(e2, ents)          # same seeds, same sample
+    for b in (1, 64):
+        v = d.view(b)
+        ids = v.node_ids.long()
+        assert torch.unique(ids).numel() == ids.numel()
+        assert torch.equal(ids[v.repr_map.long()], v.nbrs.long())
+        nio = v.node_id_offsets.cpu().tolist()
+        for j in range(len(nio) - 2):                                # deltas ascending (targets keep caller order)
+            seg = ids[nio[j]:nio[j + 1]]
+            assert bool((seg[1:] > seg[:-1]).all())
+        assert ids[nio[-2]:].cpu().tolist() == tg[b].tolist()
