@@ -253,11 +253,14 @@ int mg_lp_free(mg_lp_batch* lp);
  * destination replaced by negative t of edge i's chunk, neg_src[i,t] with the source
  * replaced.  h_dev: DEVICE [n_targets, dim] (mg_forward's output for the batch's targets);
  * rel_emb_dev: DEVICE [n_relations, dim]; outputs DEVICE: pos [n_edges],
- * neg_* [n_edges, negs_per_chunk] (only the sides `corrupt` names are written).  The kernels are
- * queued on the context's stream; the call does not wait for them. */
+ * neg_* [n_edges, negs_per_chunk] (only the sides `corrupt` names are written).  pos is always
+ * computed in fp32; the negative scores are a contraction and run on the tensor cores
+ * (MG_GEMM_TF32: operands rounded to nearest TF32, fp32 accumulate; needs dim % 4 == 0 and
+ * dim <= 128) or on CUDA cores in fp32 (MG_GEMM_FP32, any dim).  The kernels are queued on the
+ * context's stream; the call does not wait for them. */
 int mg_distmult_score(mg_ctx* ctx, const mg_lp_batch* lp, const float* h_dev, int32_t dim,
-                      const float* rel_emb_dev, int32_t n_relations, int corrupt, float* pos_out,
-                      float* neg_dst_out, float* neg_src_out);
+                      const float* rel_emb_dev, int32_t n_relations, int corrupt, int gemm_precision,
+                      float* pos_out, float* neg_dst_out, float* neg_src_out);
 
 /* ---- instrumentation ------------------------------------------------------------------ */
 

@@ -348,12 +348,13 @@ class Context:
                                            C.c_uint64(int(seed) & 0xFFFFFFFFFFFFFFFF), C.byref(lp.handle)))
         return lp
 
-    def distmult_score(self, lp: LpBatch, h: torch.Tensor, rel_emb: torch.Tensor, corrupt: int = CORRUPT_BOTH):
+    def distmult_score(self, lp: LpBatch, h: torch.Tensor, rel_emb: torch.Tensor, corrupt: int = CORRUPT_BOTH,
+                       precision: int = GEMM_TF32):
         assert h.is_cuda and rel_emb.is_cuda and h.dtype == torch.float32 and rel_emb.dtype == torch.float32
         h, rel_emb = h.contiguous(), rel_emb.contiguous()
         pos = torch.empty(lp.n_edges, dtype=torch.float32, device=self.device)
         nd = torch.empty((lp.n_edges, lp.negs), dtype=torch.float32, device=self.device) if corrupt & CORRUPT_DST else None
         ns = torch.empty((lp.n_edges, lp.negs), dtype=torch.float32, device=self.device) if corrupt & CORRUPT_SRC else None
         self._check(self.lib.mg_distmult_score(self.handle, lp.handle, _ptr(h), C.c_int32(h.shape[1]), _ptr(rel_emb),
-                                               C.c_int32(rel_emb.shape[0]), C.c_int(corrupt), _ptr(pos), _ptr(nd), _ptr(ns)))
+                                               C.c_int32(rel_emb.shape[0]), C.c_int(corrupt), C.c_int(precision), _ptr(pos), _ptr(nd), _ptr(ns)))
         return pos, nd, ns

@@ -4,7 +4,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-#define MG_SLOT_BITS 21  // per-batch id-table slots are addressed with 21 bits (<= 2M slots)
+#define MG_SLOT_BITS 24  // per-batch id-table slots are addressed with 24 bits (<= 16M slots)
 
 // Philox4x32-10 (Salmon et al., SC'11); the draw of (seed, node, hop, slot) is word slot % 4
 // of the block with counter (node, 0, hop, slot / 4) and key (seed low, seed high).

@@ -5,6 +5,7 @@
 
 #include "mg_device.cuh"
 #include "mg_internal.cuh"
+#include "mg_tcgen05.cuh"
 
 namespace {
 
@@ -153,6 +154,134 @@ __global__ void __launch_bounds__(256) k_distmult_neg(NegArgs a) {
     }
 }
 
+// ---- tensor-core negative scoring ------------------------------------------------------------
+// One CTA owns 128 edges of one chunk and one corrupted side.  The left operand rows
+// h[keep] (*) rel[r] are formed on the fly, rounded to TF32 and written K-major with the 128-byte
+// swizzle; for each block of up to 256 negatives the right operand rows h[neg] are gathered the same
+// way, one thread issues the tcgen05 MMAs (fp32 accumulator in tensor memory) and four warps store
+// the block of scores with coalesced row segments.  The score matrix (4 bytes per (edge, negative))
+// is the bulk of the traffic; the contraction itself is small.
+constexpr int kTcThreads = 256;
+constexpr int kTcMaxSlices = 4;   // dim <= 128
+
+struct NegTcArgs {
+    NegArgs base;
+    int32_t n_slices, bn_max, tmem_cols;
+    uint32_t* error;
+};
+
+__device__ __forceinline__ size_t swz_off(int row, int slot) {   // 16-byte slot of a 128-byte row, 8-row groups
+    return (size_t)(row >> 3) * 1024 + (size_t)(row & 7) * 128 + (size_t)((slot ^ (row & 7)) << 4);
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1) k_distmult_neg_tc(NegTcArgs ta) {
+    using namespace tc;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t mma_done;
+    __shared__ uint32_t tmem_slot;
+    __shared__ int32_t a_row[128], a_rel[128], b_row[256];
+    __shared__ float out_stage[4][32 * 33];
+    const NegArgs& a = ta.base;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t* a_smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);   // n_slices x 16 KiB
+    uint8_t* b_smem = a_smem + (size_t)ta.n_slices * 16384;                          // n_slices x bn_max x 128 B
+    const size_t b_slice_bytes = (size_t)ta.bn_max * 128;
+
+    const int c = blockIdx.x / a.tiles_per_chunk, tile = blockIdx.x % a.tiles_per_chunk;
+    const int64_t lo = ((int64_t)c * a.E + a.n_chunks - 1) / a.n_chunks;
+    const int64_t hi = ((int64_t)(c + 1) * a.E + a.n_chunks - 1) / a.n_chunks;
+    const int64_t m0 = lo + (int64_t)tile * 128;
+
+    if (threadIdx.x == 0) {
+        mbar_init(&mma_done, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"((uint32_t)ta.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (threadIdx.x < 128) {
+        const int64_t i = m0 + threadIdx.x;
+        a_row[threadIdx.x] = i < hi ? a.keep_idx[i] : -1;
+        a_rel[threadIdx.x] = i < hi ? a.rel[i] : 0;
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_slot;
+    const int n_slots = ta.n_slices * 8;                  // 16-byte slots per operand row
+    // left operand: (row, slot) pairs over all threads
+    for (int i = threadIdx.x; i < 128 * n_slots; i += kTcThreads) {
+        const int r = i / n_slots, q = i % n_slots;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (a_row[r] >= 0 && q * 4 < a.dim) {
+            const float4 hv = __ldg(reinterpret_cast<const float4*>(a.h + (int64_t)a_row[r] * a.dim) + q);
+            const float4 rv = __ldg(reinterpret_cast<const float4*>(a.rel_emb + (int64_t)a_rel[r] * a.dim) + q);
+            v = make_float4(to_tf32(hv.x * rv.x), to_tf32(hv.y * rv.y), to_tf32(hv.z * rv.z), to_tf32(hv.w * rv.w));
+        }
+        *reinterpret_cast<float4*>(a_smem + (size_t)(q >> 3) * 16384 + swz_off(r, q & 7)) = v;
+    }
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int n0 = 0; n0 < a.negs; n0 += ta.bn_max) {
+        const int bn = min(ta.bn_max, (a.negs - n0 + 15) / 16 * 16);   // MMA N of this block
+        for (int t = threadIdx.x; t < bn; t += kTcThreads)
+            b_row[t] = (n0 + t < a.negs) ? a.neg_idx[(int64_t)c * a.negs + n0 + t] : -1;
+        __syncthreads();   // also: the previous block's epilogue has drained tensor memory reads
+        for (int i = threadIdx.x; i < bn * n_slots; i += kTcThreads) {
+            const int r = i / n_slots, q = i % n_slots;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (b_row[r] >= 0 && q * 4 < a.dim) {
+                const float4 hv = __ldg(reinterpret_cast<const float4*>(a.h + (int64_t)b_row[r] * a.dim) + q);
+                v = make_float4(to_tf32(hv.x), to_tf32(hv.y), to_tf32(hv.z), to_tf32(hv.w));
+            }
+            *reinterpret_cast<float4*>(b_smem + (size_t)(q >> 3) * b_slice_bytes + swz_off(r, q & 7)) = v;
+        }
+        fence_async_smem();
+        tc_fence_before();
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            tc_fence_after();
+            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+            for (int sl = 0; sl < ta.n_slices; ++sl) {
+                const uint64_t da = smem_desc_sw128(smem_u32(a_smem + (size_t)sl * 16384));
+                const uint64_t db = smem_desc_sw128(smem_u32(b_smem + (size_t)sl * b_slice_bytes));
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) mma_tf32(tmem_base, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (sl | kk) ? 1u : 0u);
+            }
+            mma_commit(&mma_done);
+        }
+        if (ok && !mbar_wait(&mma_done, phase)) { if (lane == 0) atomicExch(ta.error, 21u); ok = false; }
+        phase ^= 1;
+        tc_fence_after();
+        if (ok && warp < 4) {
+            const int64_t row0 = m0 + warp * 32;
+            for (int c0 = 0; c0 < bn; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld_32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (row0 < hi) {
+                    float* st = out_stage[warp];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) st[lane * 33 + j] = __uint_as_float(v[j]);
+                    __syncwarp();
+                    const int n = n0 + c0 + lane;
+                    const int rows = (int)min((int64_t)32, hi - row0);
+                    if (n < a.negs)
+                        for (int rr = 0; rr < rows; ++rr) a.out[(row0 + rr) * a.negs + n] = st[rr * 33 + lane];
+                    __syncwarp();
+                }
+            }
+        }
+        tc_fence_before();
+    }
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)ta.tmem_cols) : "memory");
+    }
+}
+
 }  // namespace
 
 extern "C" int mg_lp_free(mg_lp_batch* lp) {
@@ -245,10 +374,11 @@ extern "C" int mg_lp_view(const mg_lp_batch* lp, int32_t* n_targets, const int32
 }
 
 extern "C" int mg_distmult_score(mg_ctx* ctx, const mg_lp_batch* lp, const float* h_dev, int32_t dim, const float* rel_emb_dev,
-                                 int32_t n_relations, int corrupt, float* pos_out, float* neg_dst_out, float* neg_src_out) {
+                                 int32_t n_relations, int corrupt, int gemm_precision, float* pos_out, float* neg_dst_out, float* neg_src_out) {
     if (!ctx) return MG_ERR_ARG;
     if (!lp || !h_dev || !rel_emb_dev || !pos_out) return mg_fail(ctx, MG_ERR_ARG, "null argument");
     if (dim <= 0 || n_relations <= 0) return mg_fail(ctx, MG_ERR_ARG, "dim and n_relations must be positive");
+    if (gemm_precision != MG_GEMM_TF32 && gemm_precision != MG_GEMM_FP32) return mg_fail(ctx, MG_ERR_ARG, "unknown gemm precision");
     if ((corrupt & MG_CORRUPT_DST) && lp->negs > 0 && !neg_dst_out) return mg_fail(ctx, MG_ERR_ARG, "null neg_dst_out");
     if ((corrupt & MG_CORRUPT_SRC) && lp->negs > 0 && !neg_src_out) return mg_fail(ctx, MG_ERR_ARG, "null neg_src_out");
     MG_CUDA(ctx, cudaSetDevice(ctx->device));
@@ -262,6 +392,30 @@ extern "C" int mg_distmult_score(mg_ctx* ctx, const mg_lp_batch* lp, const float
         a.h = h_dev; a.rel_emb = rel_emb_dev; a.rel = lp->rel; a.neg_idx = lp->neg_idx; a.E = lp->n_edges;
         a.n_chunks = lp->n_chunks; a.negs = lp->negs; a.dim = dim;
         a.tiles_per_chunk = (int32_t)((max_chunk + 63) / 64);
+        const bool tensor = gemm_precision == MG_GEMM_TF32 && dim % 4 == 0 && dim <= 32 * kTcMaxSlices;
+        if (tensor) {
+            NegTcArgs ta;
+            ta.n_slices = (dim + 31) / 32;
+            ta.bn_max = std::min(256, (lp->negs + 15) / 16 * 16);
+            int cols = 32;
+            while (cols < ta.bn_max) cols <<= 1;
+            ta.tmem_cols = cols;
+            ta.error = ctx->d_flags;
+            a.tiles_per_chunk = (int32_t)((max_chunk + 127) / 128);
+            const size_t smem = (size_t)ta.n_slices * 16384 + (size_t)ta.n_slices * ta.bn_max * 128 + 1024;
+            MG_CUDA(ctx, cudaFuncSetAttribute(k_distmult_neg_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            const unsigned blocks = (unsigned)(a.tiles_per_chunk * lp->n_chunks);
+            if (corrupt & MG_CORRUPT_DST) {
+                a.keep_idx = lp->src_idx; a.out = neg_dst_out; ta.base = a;
+                k_distmult_neg_tc<<<blocks, kTcThreads, smem, st>>>(ta);
+                ctx->launches++;
+            }
+            if (corrupt & MG_CORRUPT_SRC) {
+                a.keep_idx = lp->dst_idx; a.out = neg_src_out; ta.base = a;
+                k_distmult_neg_tc<<<blocks, kTcThreads, smem, st>>>(ta);
+                ctx->launches++;
+            }
+        } else {
         dim3 grid((unsigned)(a.tiles_per_chunk * lp->n_chunks), (unsigned)((lp->negs + 63) / 64));
         if (corrupt & MG_CORRUPT_DST) {
             a.keep_idx = lp->src_idx; a.out = neg_dst_out;
@@ -272,6 +426,7 @@ extern "C" int mg_distmult_score(mg_ctx* ctx, const mg_lp_batch* lp, const float
             a.keep_idx = lp->dst_idx; a.out = neg_src_out;
             k_distmult_neg<<<grid, 256, 0, st>>>(a);
             ctx->launches++;
+        }
         }
     }
     MG_CUDA(ctx, cudaGetLastError());

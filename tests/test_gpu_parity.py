@@ -249,12 +249,39 @@ def test_link_prediction_distmult():
     ctx.forward(model, d, h)
     ref_h = O.forward(ref, emb.numpy()[ref["node_ids"]], [(w.numpy(), nn.numpy(), b.numpy()) for w, nn, b in layers])
     close(h.cpu().numpy(), ref_h, RTOL_AGG)
-    pos, nd, ns = ctx.distmult_score(lp, h, rel_emb.cuda())
-    torch.cuda.synchronize()
     rpos, rnd, rns = O.distmult_scores(ref_h, rel_emb.numpy(), prep, rel.tolist(), n_chunks)
+    for prec, rtol in ((mg.GEMM_FP32, RTOL_AGG), (mg.GEMM_TF32, RTOL_TC)):
+        pos, nd, ns = ctx.distmult_score(lp, h, rel_emb.cuda(), precision=prec)
+        torch.cuda.synchronize()
+        close(pos.cpu().numpy(), rpos, RTOL_AGG)      # positives are always fp32
+        close(nd.cpu().numpy(), rnd, rtol)
+        close(ns.cpu().numpy(), rns, rtol)
+    # one corrupted side only
+    pos, nd, ns = ctx.distmult_score(lp, h, rel_emb.cuda(), corrupt=mg.CORRUPT_DST)
+    assert ns is None
+    close(nd.cpu().numpy(), rnd, RTOL_TC)
+
+
+@pytest.mark.parametrize("dim,n_edges,n_chunks,negs", [(100, 700, 3, 1000), (32, 129, 1, 17), (128, 300, 7, 256)])
+def test_distmult_tensor_core_shapes(dim, n_edges, n_chunks, negs):
+    """DistMult negatives on the tensor cores: padded K, several blocks of negatives, ragged chunks."""
+    n = 30_000
+    g = inputs.rmat_graph(n, 300_000, seed=6, n_relations=11)
+    ctx = mg.Context(0)
+    ctx.load_graph(g.row_offsets.cuda(), g.nbrs.cuda())
+    src, rel, dst = inputs.lp_edges(g, None, n_edges, seed=2)
+    lp = ctx.lp_prepare(src, rel, dst, n_chunks, negs, seed=7)
+    view = oracle_view(g)
+    prep = O.lp_prepare(view, src.tolist(), dst.tolist(), n_chunks, negs, 7)
+    assert lp.view()["neg_idx"].cpu().tolist() == prep["neg_idx"]
+    h = inputs.normal_features(len(prep["targets"]), dim, seed=4)
+    rel_emb = inputs.normal_features(11, dim, seed=5)
+    pos, nd, ns = ctx.distmult_score(lp, h.cuda(), rel_emb.cuda())
+    torch.cuda.synchronize()
+    rpos, rnd, rns = O.distmult_scores(h.numpy(), rel_emb.numpy(), prep, rel.tolist(), n_chunks)
     close(pos.cpu().numpy(), rpos, RTOL_AGG)
-    close(nd.cpu().numpy(), rnd, RTOL_AGG)
-    close(ns.cpu().numpy(), rns, RTOL_AGG)
+    close(nd.cpu().numpy(), rnd, RTOL_TC)
+    close(ns.cpu().numpy(), rns, RTOL_TC)
 
 
 @pytest.mark.parametrize("d_in,d_out", [(100, 100), (256, 256), (128, 256), (768, 256), (16, 520), (36, 4)])
