@@ -408,3 +408,93 @@ def test_full_size_config3_in_bench_launch_configuration():
             seg = ids[nio[j]:nio[j + 1]]
             assert bool((seg[1:] > seg[:-1]).all())
         assert ids[nio[-2]:].cpu().tolist() == tg[b].tolist()
+
+
+def test_config4_shaped_out_of_core_fp16_swaps():
+    """Config 4's path at 1/10 of its node count (the full fp16 x 768 table is 187 GB of pinned host
+    memory; the test box has 196 GB of RAM): R-MAT 12.2M nodes / 130M edges, fp16 features of width 768
+    kept in pinned host memory, 32 partitions with a 10-partition HBM buffer, swaps prefetched on the
+    side stream while batches run on the current set, only resident edges sampled."""
+    n, m, parts, cap, dim = 12_200_000, 130_000_000, 32, 10, 768
+    g = inputs.rmat_graph(n, m, seed=41, device="cuda")
+    feats = torch.empty((n, dim), dtype=torch.float16).pin_memory()
+    gen = torch.Generator(device="cuda"); gen.manual_seed(42)
+    for lo in range(0, n, 1 << 20):
+        hi = min(n, lo + (1 << 20))
+        feats[lo:hi].copy_(torch.randn((hi - lo, dim), generator=gen, device="cuda").half())
+    ctx = mg.Context(0)
+    ctx.load_graph(g.row_offsets, g.nbrs)
+    g_host = (g.row_offsets.cpu().numpy(), g.nbrs.cpu().numpy())
+    del g
+    ctx.set_partitioning(parts)
+    ctx.load_features(feats, capacity_parts=cap, backing=mg.BACKING_HOST)
+    layers = inputs.glorot_layers([dim, 256, 256, 256], seed=43)
+    model = ctx.model(layers, mg.GEMM_TF32)
+    states = inputs.swap_order(parts, cap, seed=44)[:4]
+    ctx.set_resident(states[0])
+    np_layers = [(w.numpy(), nn.numpy(), b.numpy()) for w, nn, b in layers]
+    B, T = 8, 1000
+    offs = [T * i for i in range(B + 1)]
+    for step, resident in enumerate(states):
+        if step + 1 < len(states):
+            ctx.set_resident(states[step + 1], async_=True)      # prefetch the next set on the side stream
+        mask = inputs.resident_node_mask(n, parts, resident)
+        pool = torch.nonzero(mask).flatten()
+        tg = torch.stack([inputs.distinct_targets(pool, T, seed=100 * step + b) for b in range(B)])
+        seeds = [1000 * step + b for b in range(B)]
+        d = ctx.sample_many(tg.reshape(-1), offs, [15, 10, 5], seeds)
+        out = torch.empty((B * T, 256), dtype=torch.float32, device="cuda")
+        ctx.forward(model, d, out)
+        view = O.GraphView(g_host[0], g_host[1], parts, resident)
+        b = step % B
+        ref = O.sample_dense(view, tg[b].tolist(), [15, 10, 5], seeds[b])
+        assert_dense_equal(d.view(b), ref)
+        assert all(view.is_resident(u) for u in ref["node_ids"][::97])
+        want = O.forward(ref, feats[torch.as_tensor(ref["node_ids"])].float().numpy(), np_layers)
+        close(out[offs[b]:offs[b + 1]].cpu().numpy(), want, RTOL_TC)
+        if step + 1 < len(states):
+            ctx.commit_resident(60_000)
+
+
+def test_config5_shaped_link_prediction_full_graph():
+    """Config 5's graph at full size (R-MAT 86M nodes / 338M edges, 14,824 relations, embeddings of width
+    100 with std 0.001, 16 partitions with 8 resident), a batch of 5,000 edges in 2 chunks of 1,000 shared
+    negatives (a tenth of the configured batch so that the oracle finishes in seconds)."""
+    n, m, parts, cap, dim, nrel = 86_000_000, 338_000_000, 16, 8, 100, 14824
+    g = inputs.rmat_graph(n, m, seed=5, device="cuda", n_relations=nrel)
+    emb = inputs.normal_features(n, dim, seed=3, device="cuda", std=0.001)
+    rel_emb = inputs.normal_features(nrel, dim, seed=9, device="cuda")
+    ctx = mg.Context(0)
+    ctx.load_graph(g.row_offsets, g.nbrs)
+    ctx.set_partitioning(parts)
+    ctx.load_features(emb, capacity_parts=cap)
+    resident = [0, 2, 3, 5, 8, 9, 12, 15]
+    ctx.set_resident(resident)
+    mask = inputs.resident_node_mask(n, parts, resident)
+    src, rel, dst = inputs.lp_edges(g, mask, 5000, seed=1)
+    g_host = (g.row_offsets.cpu().numpy(), g.nbrs.cpu().numpy())
+    del g
+    n_chunks, negs = 2, 1000
+    lp = ctx.lp_prepare(src, rel, dst, n_chunks, negs, seed=2024)
+    view = O.GraphView(g_host[0], g_host[1], parts, resident)
+    prep = O.lp_prepare(view, src.tolist(), dst.tolist(), n_chunks, negs, 2024)
+    got = lp.view()
+    for key in ("targets", "src_idx", "dst_idx", "neg_ids", "neg_idx"):
+        assert got[key].cpu().tolist() == prep[key], key
+    layers = inputs.glorot_layers([dim, dim], seed=8)
+    model = ctx.model(layers, mg.GEMM_TF32)
+    d = ctx.sample(got["targets"], [20], seed=5)
+    ref = O.sample_dense(view, prep["targets"], [20], 5)
+    assert_dense_equal(d.view(0), ref)
+    h = torch.empty((len(prep["targets"]), dim), dtype=torch.float32, device="cuda")
+    ctx.forward(model, d, h)
+    ids = torch.as_tensor(ref["node_ids"], device="cuda")
+    ref_h = O.forward(ref, emb[ids].cpu().numpy(), [(w.numpy(), nn.numpy(), b.numpy()) for w, nn, b in layers])
+    close(h.cpu().numpy(), ref_h, RTOL_TC)
+    pos, nd, ns = ctx.distmult_score(lp, h, rel_emb)
+    torch.cuda.synchronize()
+    # scores are checked against the oracle fed the GPU's own H (isolates the decoder's rounding)
+    rpos, rnd, rns = O.distmult_scores(h.cpu().numpy(), rel_emb.cpu().numpy(), prep, rel.tolist(), n_chunks)
+    close(pos.cpu().numpy(), rpos, RTOL_AGG)
+    close(nd.cpu().numpy(), rnd, RTOL_TC)
+    close(ns.cpu().numpy(), rns, RTOL_TC)
