@@ -35,6 +35,8 @@ CONFIGS = {
 }
 DEFAULT_WORKLOAD = "config3_papers100m_shaped"
 HBM_NOMINAL_GBS = 8000.0
+# dram bytes (read + write) of one launch of the dominant kernel, measured with ncu (see profiles/)
+NCU_TRAFFIC_PER_LAUNCH = {("config3_papers100m_shaped", 128): 10.58e9}
 
 
 def measured_peaks():
@@ -126,8 +128,9 @@ def algorithmic_bytes(nodes, ents, cfg, feat_bytes=4):
     for l in range(1, k + 1):
         flops += 2 * nodes[:, :k - l + 1].sum() * 2 * dims[l - 1] * dims[l]
     agg_l1 = a_f + 4 * (ents.sum() + nodes[:, :k].sum())
+    flops_l1 = 2 * nodes[:, :k].sum() * 2 * dims[0] * dims[1]
     return {"sampling": int(a_s), "features": int(a_f), "agg_index": int(a_i), "output": int(a_o),
-            "a_min": int(a_s + a_f + a_i + a_o), "flops": int(flops), "agg_l1": int(agg_l1)}
+            "a_min": int(a_s + a_f + a_i + a_o), "flops": int(flops), "agg_l1": int(agg_l1), "flops_l1": int(flops_l1)}
 
 
 def oracle_time(g_host, feats, layers, cfg, target_rows, seeds, budget_s=20.0):
@@ -286,28 +289,33 @@ def main():
     e2e_value = n_batches / (ms_e2e / 1e3)
     sampled_edges = float(ents.sum()) * world
 
-    # ---- rooflines per phase (CUDA-event times of the library's own kernels) --------------
+    # ---- rooflines (CUDA-event times of the library's own kernels, second pass) -----------------
+    # The dominant kernel is the fused layer-1 kernel (k_sage_layer_fused<first>): it gathers the base
+    # representations (the bulk of A_min), reduces them and runs the layer's GEMM on the tensor cores.
+    # It is HBM-bound: achieved = its algorithmic bytes (V d0 s + 4 (E_1 + N_1)) over its event time.
     sample_ms = sum(v["ms"] for name, v in phases.items() if name.startswith("sample_"))
     agg1 = phases["aggregate_l1"]
+    rest = phases["aggregate_rest"]
     gemm = phases["gemm"]
     tf32_peak = peaks["bf16_tflops_sustained"] * 0.5     # nominal TF32 : bf16 dense ratio is 1 : 2
-    rl_agg = {"kernel": "k_aggregate (layer 1: feature gather + segment mean)", "bound": "hbm",
-              "achieved": alg["agg_l1"] / (agg1["ms"] / 1e3) / 1e9 if agg1["ms"] else None,
-              "peak": peaks["hbm_gbs"], "unit": "GB/s",
-              "bytes_per_launch": alg["agg_l1"] / max(1, agg1["launches"]),
-              "ms_per_launch": agg1["ms"] / max(1, agg1["launches"]), "launches": agg1["launches"]}
-    rl_agg["frac"] = rl_agg["achieved"] / rl_agg["peak"] if rl_agg["achieved"] else None
-    rl_gemm = {"kernel": "k_gemm_tf32 (tcgen05)", "bound": "tensor",
-               "achieved": alg["flops"] / (gemm["ms"] / 1e3) / 1e12 if gemm["ms"] else None,
-               "peak": tf32_peak, "unit": "TFLOP/s", "launches": gemm["launches"],
-               "ms_per_launch": gemm["ms"] / max(1, gemm["launches"])}
-    rl_gemm["frac"] = rl_gemm["achieved"] / rl_gemm["peak"] if rl_gemm["achieved"] else None
-    mem_ms = sample_ms + agg1["ms"] + phases["aggregate_rest"]["ms"]
+    fused = gemm["launches"] == 0
+    n_l1 = max(1, agg1["launches"])
+    roofline = {"kernel": "k_sage_layer_fused<layer 1> (feature gather + segment mean + tcgen05 TF32 GEMM)" if fused
+                else "k_aggregate<layer 1> (feature gather + segment mean)",
+                "bound": "hbm", "achieved": alg["agg_l1"] / (agg1["ms"] / 1e3) / 1e9 if agg1["ms"] else None,
+                "peak": peaks["hbm_gbs"], "unit": "GB/s", "bytes_per_launch": alg["agg_l1"] / n_l1,
+                "ms_per_launch": agg1["ms"] / n_l1, "launches": agg1["launches"], "peak_source": peaks["source"]}
+    roofline["frac"] = roofline["achieved"] / roofline["peak"] if roofline["achieved"] else None
+    # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the single-pass ncu capture of this very
+    # command (profiles/): only known for the default workload and group size
+    roofline["traffic"] = NCU_TRAFFIC_PER_LAUNCH.get((args.workload, G))
+    flops_l1 = alg["flops_l1"]
+    tensor = {"what": "layer GEMM work inside the fused kernels (all layers)", "bound": "tensor",
+              "achieved": alg["flops"] / ((agg1["ms"] + rest["ms"] + gemm["ms"]) / 1e3) / 1e12, "peak": tf32_peak,
+              "unit": "TFLOP/s", "layer1_tflops": flops_l1 / (agg1["ms"] / 1e3) / 1e12 if agg1["ms"] else None}
+    tensor["frac"] = tensor["achieved"] / tensor["peak"]
+    mem_ms = sample_ms + agg1["ms"] + rest["ms"]
     path_gbs = alg["a_min"] / (mem_ms / 1e3) / 1e9 if mem_ms else None
-    dominant = rl_agg if agg1["ms"] >= gemm["ms"] else rl_gemm
-    roofline = dict(dominant)
-    roofline["traffic"] = None
-    roofline["peak_source"] = peaks["source"]
 
     line = {
         "metric": "DENSE sample+aggregate mini-batches/s", "value": value, "unit": "mini-batches/s",
@@ -328,9 +336,8 @@ def main():
         "gpu_launches": int(launches),
         "clocks": clocks,
         "roofline": roofline,
-        "roofline_gemm": rl_gemm,
-        "roofline_aggregate_l1": rl_agg,
-        "path_hbm": {"what": "A_min over the sampling + aggregation kernel time (GEMMs excluded)",
+        "tensor": tensor,
+        "path_hbm": {"what": "A_min over the time of all sampling and layer kernels (the layer GEMMs run inside them)",
                      "achieved_gbs": path_gbs, "frac_of_measured": path_gbs / peaks["hbm_gbs"] if path_gbs else None,
                      "frac_of_8tbs": path_gbs / HBM_NOMINAL_GBS if path_gbs else None, "kernel_ms": mem_ms},
         "phases_ms_per_step": {name: round(v["ms"] / args.steps, 4) for name, v in phases.items() if v["launches"]},

@@ -305,8 +305,12 @@ static int upload_slot_map(mg_ctx* c) {
 }
 
 static int rebuild_view(mg_ctx* c) {
-    bool all = true;
-    for (int p = 0; p < c->n_parts; ++p) all = all && c->slot_of_part[p] >= 0;
+    bool all = true, any = false;
+    for (int p = 0; p < c->n_parts; ++p) { all = all && c->slot_of_part[p] >= 0; any = any || c->slot_of_part[p] >= 0; }
+    if (!any) {   // nothing in the buffer: there is no view, and sampling refuses to run
+        free_view(c);
+        return MG_OK;
+    }
     if (all) {
         free_view(c);
         c->view_off = c->row_off; c->view_nbrs = c->nbrs; c->view_edges = c->n_edges; c->view_owned = false;

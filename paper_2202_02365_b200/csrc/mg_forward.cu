@@ -399,7 +399,9 @@ extern "C" int mg_forward(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* ou
     }
     {
         size_t have = ctx->ws_h_bytes[0] / sizeof(float);
-        if ((rc = mg_ensure(ctx, &ctx->ws_h[0], &have, total))) return rc;
+        // a quarter of headroom: the row counts of consecutive calls differ slightly, and growing means a
+        // device-wide synchronising free + malloc
+        if (have < total && (rc = mg_ensure(ctx, &ctx->ws_h[0], &have, total + total / 4))) return rc;
         ctx->ws_h_bytes[0] = have * sizeof(float);
     }
     int64_t max_x = 0;

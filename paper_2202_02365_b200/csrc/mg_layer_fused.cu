@@ -465,7 +465,7 @@ int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_ou
     {
         size_t have = ctx->ws_x_bytes / sizeof(int4);
         int4* buf = reinterpret_cast<int4*>(ctx->ws_x);
-        int rc = mg_ensure(ctx, &buf, &have, (size_t)M);
+        int rc = have >= (size_t)M ? MG_OK : mg_ensure(ctx, &buf, &have, (size_t)M + (size_t)M / 4);
         ctx->ws_x = reinterpret_cast<float*>(buf);
         ctx->ws_x_bytes = have * sizeof(int4);
         if (rc) return rc;

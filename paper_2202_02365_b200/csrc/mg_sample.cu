@@ -816,6 +816,7 @@ extern "C" int mg_sample_many(mg_ctx* ctx, const int32_t* targets, int targets_o
     for (int h = 0; h < k; ++h)
         if (fanouts[h] <= 0 || fanouts[h] > MG_MAX_FANOUT) return mg_fail(ctx, MG_ERR_ARG, "fanouts must be in [1, %d]", MG_MAX_FANOUT);
     if (!ctx->row_off) return mg_fail(ctx, MG_ERR_STATE, "no graph loaded");
+    if (!ctx->view_off) return mg_fail(ctx, MG_ERR_NONRESIDENT, "no partition is resident");
     if (target_offsets[0] != 0) return mg_fail(ctx, MG_ERR_ARG, "target_offsets[0] must be 0");
     for (int b = 0; b < n_batches; ++b)
         if (target_offsets[b + 1] < target_offsets[b]) return mg_fail(ctx, MG_ERR_ARG, "target_offsets must be non-decreasing");
