@@ -196,6 +196,17 @@ int mg_model_free(mg_model* m);
  * depths differ / feature dim != dims[0]), MG_ERR_OOM. */
 int mg_forward(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out, int out_on_device);
 
+/* mg_forward with a HOST output whose device-to-host copy does not block the caller: the kernels are
+ * queued on the context's stream, the copy follows them on the library's side stream, and the call
+ * returns at once.  out_host should be pinned memory (a pageable buffer makes the copy synchronous)
+ * and holds H^k only after mg_wait_output returns MG_OK.  Calls made in between (sampling the next
+ * group into another mg_dense) overlap the copy; the next forward on this context waits for it before
+ * it reuses the layer workspace. */
+int mg_forward_host_async(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out_host);
+/* Block until the output copy of the last mg_forward_host_async has finished; reports a tensor-core
+ * barrier time-out of that forward as MG_ERR_TIMEOUT. */
+int mg_wait_output(mg_ctx* ctx);
+
 /* H^0 of one batch: base representations of its node_ids, rows in the order of
  * mg_dense_view's node_ids, widened to fp32.  out_dev: DEVICE [n_nodes, feature dim]. */
 int mg_gather_h0(mg_ctx* ctx, mg_dense* d, int32_t batch, float* out_dev);

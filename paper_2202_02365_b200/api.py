@@ -30,7 +30,7 @@ EXPORTS = [
     "mg_create", "mg_destroy", "mg_last_error", "mg_load_graph", "mg_set_partitioning",
     "mg_load_features", "mg_set_resident", "mg_commit_resident", "mg_sample_many", "mg_sample",
     "mg_dense_counts", "mg_dense_view", "mg_dense_free", "mg_model_create", "mg_model_free",
-    "mg_forward", "mg_forward_noalloc", "mg_gather_h0", "mg_layer_output", "mg_lp_prepare", "mg_lp_view", "mg_lp_free",
+    "mg_forward", "mg_forward_host_async", "mg_wait_output", "mg_forward_noalloc", "mg_gather_h0", "mg_layer_output", "mg_lp_prepare", "mg_lp_view", "mg_lp_free",
     "mg_distmult_score", "mg_kernel_launches", "mg_profile", "mg_profile_read",
 ]
 
@@ -319,6 +319,15 @@ class Context:
         assert out.dtype == torch.float32 and out.is_contiguous()
         self._check(self.lib.mg_forward(self.handle, model.handle, dense.handle, _ptr(out), C.c_int(out.is_cuda)))
         return out
+
+    def forward_host_async(self, model: Model, dense: Dense, out: torch.Tensor) -> torch.Tensor:
+        """mg_forward_host_async: `out` (pinned CPU tensor) is valid after wait_output()."""
+        assert out.dtype == torch.float32 and out.is_contiguous() and not out.is_cuda
+        self._check(self.lib.mg_forward_host_async(self.handle, model.handle, dense.handle, _ptr(out)))
+        return out
+
+    def wait_output(self):
+        self._check(self.lib.mg_wait_output(self.handle))
 
     def forward_noalloc(self, model: Model, dense: Dense, out: torch.Tensor) -> torch.Tensor:
         """mg_forward_noalloc: same result as forward(), all temporaries in the library's built-in

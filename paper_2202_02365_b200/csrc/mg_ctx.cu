@@ -217,6 +217,8 @@ extern "C" int mg_create(mg_ctx** out, int device, void* stream) {
     if (c->n_sms <= 0) c->n_sms = 148;
     for (int i = 0; i < PH_COUNT; ++i) c->prof[i] = ProfPhase{kPhaseNames[i], 0.0, 0};
     if (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->ev_fwd_done, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->ev_out_done, cudaEventDisableTiming) != cudaSuccess ||
         cudaMalloc((void**)&c->d_slot_of_part, sizeof(int32_t) * MG_MAX_PARTS) != cudaSuccess ||
         cudaMalloc((void**)&c->d_res_prefix, sizeof(int64_t) * (MG_MAX_PARTS + 1)) != cudaSuccess ||
         cudaMalloc((void**)&c->d_flags, sizeof(uint32_t)) != cudaSuccess ||
@@ -250,6 +252,7 @@ extern "C" int mg_destroy(mg_ctx* c) {
     free_features(c);
     cudaFree(c->row_off); cudaFree(c->nbrs); cudaFree(c->d_slot_of_part); cudaFree(c->d_res_prefix); cudaFree(c->d_flags);
     cudaFree(c->ws_x); cudaFree(c->ws_h[0]); cudaFree(c->ws_h[1]);
+    cudaEventDestroy(c->ev_fwd_done); cudaEventDestroy(c->ev_out_done);
     cudaStreamDestroy(c->side);
     delete c;
     return MG_OK;

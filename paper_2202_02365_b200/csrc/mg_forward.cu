@@ -381,7 +381,9 @@ static int64_t chunk_rows_for(int d_in) {
     return rows;
 }
 
-extern "C" int mg_forward(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out, int out_on_device) {
+enum { OUT_DEVICE = 0, OUT_HOST = 1, OUT_HOST_ASYNC = 2 };
+
+static int forward_impl(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out, int out_mode) {
     if (!ctx) return MG_ERR_ARG;
     int rc = forward_checks(ctx, m, d);
     if (rc) return rc;
@@ -389,6 +391,10 @@ extern "C" int mg_forward(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* ou
     MG_CUDA(ctx, cudaSetDevice(ctx->device));
     const int k = d->k, B = d->n_batches;
     cudaStream_t st = ctx->stream;
+    if (ctx->out_copy_pending) {   // the previous asynchronous output copy still reads the layer workspace
+        MG_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_out_done, 0));
+        ctx->out_copy_pending = false;
+    }
 
     // per-layer outputs H^1..H^k live in one workspace (kept for mg_layer_output)
     size_t total = 0;
@@ -468,9 +474,36 @@ extern "C" int mg_forward(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* ou
     }
     MG_CUDA(ctx, cudaGetLastError());
     const size_t out_bytes = (size_t)d->h_hdr.rows_total[k] * m->dims[k] * sizeof(float);
-    MG_CUDA(ctx, cudaMemcpyAsync(out, ctx->ws_h[0] + off[k], out_bytes, out_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, st));
+    if (out_mode == OUT_HOST_ASYNC) {
+        // the copy to the host runs on the side stream behind the last layer kernel; the caller's next
+        // calls (sampling the next group) overlap it
+        MG_CUDA(ctx, cudaEventRecord(ctx->ev_fwd_done, st));
+        MG_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_fwd_done, 0));
+        MG_CUDA(ctx, cudaMemcpyAsync(out, ctx->ws_h[0] + off[k], out_bytes, cudaMemcpyDeviceToHost, ctx->side));
+        MG_CUDA(ctx, cudaEventRecord(ctx->ev_out_done, ctx->side));
+        ctx->out_copy_pending = true;
+        ctx->out_check_gemm = m->precision == MG_GEMM_TF32;
+        return MG_OK;
+    }
+    MG_CUDA(ctx, cudaMemcpyAsync(out, ctx->ws_h[0] + off[k], out_bytes, out_mode == OUT_DEVICE ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, st));
     MG_CUDA(ctx, cudaStreamSynchronize(st));
     if (m->precision == MG_GEMM_TF32) return mg_gemm_tf32_status(ctx);
+    return MG_OK;
+}
+
+extern "C" int mg_forward(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out, int out_on_device) {
+    return forward_impl(ctx, m, d, out, out_on_device ? OUT_DEVICE : OUT_HOST);
+}
+
+extern "C" int mg_forward_host_async(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out_host) {
+    return forward_impl(ctx, m, d, out_host, OUT_HOST_ASYNC);
+}
+
+extern "C" int mg_wait_output(mg_ctx* ctx) {
+    if (!ctx) return MG_ERR_ARG;
+    MG_CUDA(ctx, cudaSetDevice(ctx->device));
+    MG_CUDA(ctx, cudaEventSynchronize(ctx->ev_out_done));   // completes at once when nothing was recorded
+    if (ctx->out_check_gemm) { ctx->out_check_gemm = false; return mg_gemm_tf32_status(ctx); }
     return MG_OK;
 }
 

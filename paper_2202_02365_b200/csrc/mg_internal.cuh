@@ -103,6 +103,10 @@ struct mg_ctx {
     float* ws_h[2] = {nullptr, nullptr}; size_t ws_h_bytes[2] = {0, 0};
     float** ws_layer = nullptr;
 
+    // asynchronous output copy of mg_forward_host_async
+    cudaEvent_t ev_fwd_done = nullptr, ev_out_done = nullptr;
+    bool out_copy_pending = false, out_check_gemm = false;
+
     // profiling
     bool prof_on = false;
     ProfPhase prof[PH_COUNT];

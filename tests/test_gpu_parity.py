@@ -498,3 +498,25 @@ def test_config5_shaped_link_prediction_full_graph():
     close(pos.cpu().numpy(), rpos, RTOL_AGG)
     close(nd.cpu().numpy(), rnd, RTOL_TC)
     close(ns.cpu().numpy(), rns, RTOL_TC)
+
+
+def test_async_host_output_equals_blocking_forward(tiny):
+    g, feats = tiny
+    ctx = make_ctx(g, feats)
+    layers = inputs.random_bias_layers([16, 32, 8], seed=3)
+    model = ctx.model(layers, mg.GEMM_TF32)
+    outs_async = [torch.empty((300, 8), dtype=torch.float32).pin_memory() for _ in range(2)]
+    want = []
+    denses = []
+    for i in range(2):
+        targets = inputs.distinct_targets(10_000, 300, seed=20 + i)
+        d = ctx.sample(targets, [6, 4], seed=i)
+        ref = torch.empty((300, 8), dtype=torch.float32)
+        ctx.forward(model, d, ref)
+        want.append(ref)
+        denses.append(d)
+    for i in range(2):      # two copies in flight back to back, then one wait
+        ctx.forward_host_async(model, denses[i], outs_async[i])
+    ctx.wait_output()
+    for i in range(2):
+        assert torch.equal(outs_async[i], want[i])
