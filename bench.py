@@ -160,6 +160,7 @@ def main():
     ap.add_argument("--impl", default="mgdense", choices=["mgdense", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(CONFIGS))
     ap.add_argument("--group", type=int, default=128, help="mini-batches per step")
+    ap.add_argument("--window", type=int, default=0, help="mini-batches per window of the layer schedule (0 = whole layers)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     args = ap.parse_args()
@@ -200,6 +201,7 @@ def main():
     else:
         ctx.load_features(feats)
     model = ctx.model(layers, mg.GEMM_TF32)
+    ctx.set_layer_window(args.window)
 
     G, T, k = args.group, cfg["batch"], len(cfg["fanouts"])
     n_steps_total = args.warmup + 2 * args.steps + 1
@@ -228,14 +230,29 @@ def main():
     host_targets = [step_targets(i).pin_memory() for i in range(n_steps_total)]
 
     out_hosts = [out_host, torch.empty_like(out_host).pin_memory()]
+    denses = [dense, ctx.sample_many(step_targets(0).to(device), offs, cfg["fanouts"], step_seeds(0), caps=caps)]
+
+    def begin(i, e2e):
+        tg = host_targets[i] if e2e else dev_targets[i]
+        ctx.sample_many_begin(tg, offs, cfg["fanouts"], step_seeds(i), caps=caps, out=denses[i & 1])
+
+    def run_steps(first, count, e2e):
+        """`count` steps, software-pipelined: group i+1 is sampled (sampling stream) while group i runs its
+        layers (context stream); with e2e the host H^k of group i is copied out during group i+1."""
+        begin(first, e2e)
+        for i in range(first, first + count):
+            ctx.sample_many_end(denses[i & 1])
+            if i + 1 < first + count:
+                begin(i + 1, e2e)
+            if e2e:
+                ctx.forward_host_async(model, denses[i & 1], out_hosts[i & 1])
+            else:
+                ctx.forward(model, denses[i & 1], out_dev)
+        if e2e:
+            ctx.wait_output()
 
     def run_step(i, e2e):
-        tg = host_targets[i] if e2e else dev_targets[i]
-        ctx.sample_many(tg, offs, cfg["fanouts"], step_seeds(i), caps=caps, out=dense)
-        if e2e:   # host H^k of step i is copied out while step i+1 samples (two pinned buffers alternate)
-            ctx.forward_host_async(model, dense, out_hosts[i & 1])
-        else:
-            ctx.forward(model, dense, out_dev)
+        run_steps(i, 1, e2e)
 
     def barrier():
         torch.cuda.synchronize()
@@ -253,8 +270,7 @@ def main():
     sampler.start()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
-    for s in range(args.steps):
-        run_step(args.warmup + s, False)
+    run_steps(args.warmup, args.steps, False)
     ev1.record()
     barrier()
     clocks = sampler.stop()
@@ -264,9 +280,9 @@ def main():
     # ---- the same steps again with per-phase CUDA events on the library's stream ---------------
     ctx.profile(True)
     ctx.profile_read(reset=True)
-    for s in range(args.steps):
+    for s in range(args.steps):          # one group at a time here, so that the phase events do not overlap
         run_step(args.warmup + s, False)
-        n_, e_ = dense.counts()
+        n_, e_ = denses[(args.warmup + s) & 1].counts()
         stats["nodes"].append(n_); stats["ents"].append(e_)
     phases = ctx.profile_read(reset=True)
     ctx.profile(False)
@@ -275,9 +291,7 @@ def main():
     barrier()
     ev2, ev3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev2.record()
-    for s in range(args.steps):
-        run_step(args.warmup + args.steps + s, True)
-    ctx.wait_output()          # the last step's H^k is on the host
+    run_steps(args.warmup + args.steps, args.steps, True)      # ends with the last H^k on the host
     ev3.record()
     barrier()
     ms_e2e = ev2.elapsed_time(ev3)

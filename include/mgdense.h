@@ -152,13 +152,27 @@ int mg_commit_resident(mg_ctx* ctx, int32_t timeout_ms);
  * `targets` is a host pointer, or a device pointer if targets_on_device; target_offsets,
  * fanouts and seeds are host pointers.  *out: NULL to allocate a new mg_dense, or an
  * existing one (of this context) to reuse its buffers.
- * The call is synchronous: on return the sample is complete and its status checked.
+ * The call is synchronous: on return the sample is complete and its status checked.  The kernels run
+ * on a library-owned sampling stream, ordered after the work queued on the context's stream so far.
  * Errors: MG_ERR_ARG, MG_ERR_STATE, MG_ERR_NONRESIDENT, MG_ERR_DUPLICATE, MG_ERR_CAPACITY,
  * MG_ERR_OOM. */
 int mg_sample_many(mg_ctx* ctx, const int32_t* targets, int targets_on_device,
                    const int64_t* target_offsets, int32_t n_batches, const int32_t* fanouts,
                    int32_t k, const uint64_t* seeds, const mg_sample_caps* caps /*nullable*/,
                    mg_dense** out);
+
+/* The two halves of mg_sample_many, for callers that overlap sampling with other work (the
+ * forward pass of the previous group, say).  mg_sample_many_begin queues the whole sample on the
+ * library's sampling stream and returns; target_offsets, fanouts and seeds may be reused at once, a
+ * device or pinned-host `targets` buffer must stay valid until mg_sample_many_end.  The mg_dense
+ * (*out, allocated or reused as in mg_sample_many) must not be used until mg_sample_many_end has
+ * waited for the sample and checked its status (same errors as mg_sample_many).  A sample begun into
+ * an mg_dense that a forward pass is still reading waits for that pass on the device. */
+int mg_sample_many_begin(mg_ctx* ctx, const int32_t* targets, int targets_on_device,
+                         const int64_t* target_offsets, int32_t n_batches, const int32_t* fanouts,
+                         int32_t k, const uint64_t* seeds, const mg_sample_caps* caps /*nullable*/,
+                         mg_dense** out);
+int mg_sample_many_end(mg_ctx* ctx, mg_dense* d);
 
 /* One batch: mg_sample_many with n_batches = 1. */
 int mg_sample(mg_ctx* ctx, const int32_t* targets, int targets_on_device, int32_t n_targets,
@@ -195,6 +209,15 @@ int mg_model_free(mg_model* m);
  * pointer if out_on_device = 0.  Errors: MG_ERR_STATE (no features / sample and model
  * depths differ / feature dim != dims[0]), MG_ERR_OOM. */
 int mg_forward(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out, int out_on_device);
+
+/* Schedule of the layers inside mg_forward.  mini_batches = 0: every layer runs over all mini-batches
+ * before the next starts, and H^1..H^{k-1} stay available for mg_layer_output.  mini_batches = w > 0: the
+ * layers run over windows of w consecutive mini-batches through small reused buffers, so that a layer's
+ * output is read back from L2 instead of DRAM; H^k is the same, the intermediate layers are not kept.
+ * Only the fused tensor-core layers (MG_GEMM_TF32, widths <= 256) use windows. */
+int mg_set_layer_window(mg_ctx* ctx, int32_t mini_batches);
+/* enable = 1 forces the whole-layer schedule whatever the window, so that mg_layer_output works. */
+int mg_keep_layer_outputs(mg_ctx* ctx, int enable);
 
 /* mg_forward with a HOST output whose device-to-host copy does not block the caller: the kernels are
  * queued on the context's stream, the copy follows them on the library's side stream, and the call

@@ -28,9 +28,9 @@ CORRUPT_DST, CORRUPT_SRC, CORRUPT_BOTH = 1, 2, 3
 # every symbol include/mgdense.h declares
 EXPORTS = [
     "mg_create", "mg_destroy", "mg_last_error", "mg_load_graph", "mg_set_partitioning",
-    "mg_load_features", "mg_set_resident", "mg_commit_resident", "mg_sample_many", "mg_sample",
+    "mg_load_features", "mg_set_resident", "mg_commit_resident", "mg_sample_many", "mg_sample_many_begin", "mg_sample_many_end", "mg_sample",
     "mg_dense_counts", "mg_dense_view", "mg_dense_free", "mg_model_create", "mg_model_free",
-    "mg_forward", "mg_forward_host_async", "mg_wait_output", "mg_forward_noalloc", "mg_gather_h0", "mg_layer_output", "mg_lp_prepare", "mg_lp_view", "mg_lp_free",
+    "mg_forward", "mg_set_layer_window", "mg_keep_layer_outputs", "mg_forward_host_async", "mg_wait_output", "mg_forward_noalloc", "mg_gather_h0", "mg_layer_output", "mg_lp_prepare", "mg_lp_view", "mg_lp_free",
     "mg_distmult_score", "mg_kernel_launches", "mg_profile", "mg_profile_read",
 ]
 
@@ -281,7 +281,7 @@ class Context:
         self._check(self.lib.mg_commit_resident(self.handle, C.c_int32(timeout_ms)))
 
     # -- sampling
-    def sample_many(self, targets: torch.Tensor, target_offsets, fanouts, seeds, caps=None, out: Dense | None = None) -> Dense:
+    def _sample_many_call(self, fn, targets, target_offsets, fanouts, seeds, caps, out):
         assert targets.dtype == torch.int32
         targets = targets.contiguous()
         offs = _host(target_offsets, torch.int64)
@@ -292,10 +292,21 @@ class Context:
         if caps is not None:
             cp = SampleCaps(int(caps.get("max_nodes_total", 0)), int(caps.get("max_entries_total", 0)),
                             int(caps.get("max_nodes_per_batch", 0)))
-        self._check(self.lib.mg_sample_many(self.handle, _ptr(targets), C.c_int(targets.is_cuda), _ptr(offs),
-                                            C.c_int32(offs.numel() - 1), _ptr(fo), C.c_int32(fo.numel()), C.c_void_p(sd.ctypes.data),
-                                            C.byref(cp) if cp is not None else None, C.byref(d.handle)))
+        self._check(fn(self.handle, _ptr(targets), C.c_int(targets.is_cuda), _ptr(offs),
+                       C.c_int32(offs.numel() - 1), _ptr(fo), C.c_int32(fo.numel()), C.c_void_p(sd.ctypes.data),
+                       C.byref(cp) if cp is not None else None, C.byref(d.handle)))
+        d._targets_keepalive = targets     # device targets must outlive the queued kernels
         return d
+
+    def sample_many(self, targets: torch.Tensor, target_offsets, fanouts, seeds, caps=None, out: Dense | None = None) -> Dense:
+        return self._sample_many_call(self.lib.mg_sample_many, targets, target_offsets, fanouts, seeds, caps, out)
+
+    def sample_many_begin(self, targets: torch.Tensor, target_offsets, fanouts, seeds, caps=None, out: Dense | None = None) -> Dense:
+        """Queue a sample on the sampling stream; finish it with sample_many_end(dense)."""
+        return self._sample_many_call(self.lib.mg_sample_many_begin, targets, target_offsets, fanouts, seeds, caps, out)
+
+    def sample_many_end(self, dense: Dense):
+        self._check(self.lib.mg_sample_many_end(self.handle, dense.handle))
 
     def sample(self, targets: torch.Tensor, fanouts, seed: int, caps=None, out: Dense | None = None) -> Dense:
         assert targets.dtype == torch.int32
@@ -319,6 +330,12 @@ class Context:
         assert out.dtype == torch.float32 and out.is_contiguous()
         self._check(self.lib.mg_forward(self.handle, model.handle, dense.handle, _ptr(out), C.c_int(out.is_cuda)))
         return out
+
+    def set_layer_window(self, mini_batches: int):
+        self._check(self.lib.mg_set_layer_window(self.handle, C.c_int32(mini_batches)))
+
+    def keep_layer_outputs(self, on: bool = True):
+        self._check(self.lib.mg_keep_layer_outputs(self.handle, C.c_int(1 if on else 0)))
 
     def forward_host_async(self, model: Model, dense: Dense, out: torch.Tensor) -> torch.Tensor:
         """mg_forward_host_async: `out` (pinned CPU tensor) is valid after wait_output()."""

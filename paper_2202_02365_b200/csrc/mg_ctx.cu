@@ -217,6 +217,8 @@ extern "C" int mg_create(mg_ctx** out, int device, void* stream) {
     if (c->n_sms <= 0) c->n_sms = 148;
     for (int i = 0; i < PH_COUNT; ++i) c->prof[i] = ProfPhase{kPhaseNames[i], 0.0, 0};
     if (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&c->sample_stream, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->ev_user, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&c->ev_fwd_done, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&c->ev_out_done, cudaEventDisableTiming) != cudaSuccess ||
         cudaMalloc((void**)&c->d_slot_of_part, sizeof(int32_t) * MG_MAX_PARTS) != cudaSuccess ||
@@ -246,13 +248,15 @@ extern "C" int mg_destroy(mg_ctx* c) {
     cudaSetDevice(c->device);
     cudaStreamSynchronize(c->stream);
     cudaStreamSynchronize(c->side);
+    cudaStreamSynchronize(c->sample_stream);
     for (auto ev : c->pending_events) cudaEventDestroy(ev);
     for (auto& p : c->prof_pending) { cudaEventDestroy(p.second.first); cudaEventDestroy(p.second.second); }
     free_view(c);
     free_features(c);
     cudaFree(c->row_off); cudaFree(c->nbrs); cudaFree(c->d_slot_of_part); cudaFree(c->d_res_prefix); cudaFree(c->d_flags);
     cudaFree(c->ws_x); cudaFree(c->ws_h[0]); cudaFree(c->ws_h[1]);
-    cudaEventDestroy(c->ev_fwd_done); cudaEventDestroy(c->ev_out_done);
+    cudaEventDestroy(c->ev_fwd_done); cudaEventDestroy(c->ev_out_done); cudaEventDestroy(c->ev_user);
+    cudaStreamDestroy(c->sample_stream);
     cudaStreamDestroy(c->side);
     delete c;
     return MG_OK;
@@ -271,6 +275,7 @@ extern "C" int mg_profile_read(mg_ctx* c, int32_t* n_phases, const char** names,
     if (!c) return MG_ERR_ARG;
     cudaSetDevice(c->device);
     cudaStreamSynchronize(c->stream);
+    cudaStreamSynchronize(c->sample_stream);
     for (auto& p : c->prof_pending) {
         float t = 0.f;
         if (cudaEventElapsedTime(&t, p.second.first, p.second.second) == cudaSuccess) c->prof[p.first].ms += t;
@@ -590,6 +595,7 @@ extern "C" int mg_commit_resident(mg_ctx* c, int32_t timeout_ms) {
     }
     for (auto ev : c->pending_events) cudaEventDestroy(ev);
     c->pending_events.clear();
+    MG_CUDA(c, cudaStreamSynchronize(c->sample_stream));   // samples in flight were drawn under the old set
     c->slot_of_part = c->pending_slot;
     c->has_pending = false;
     int rc = upload_slot_map(c);

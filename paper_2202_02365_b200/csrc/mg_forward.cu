@@ -19,8 +19,10 @@ int mg_gemm_tf32_status(mg_ctx* ctx);
 // mg_layer_fused.cu
 int mg_pack_layer_weights(mg_ctx* ctx, const float* w_cat_dev, float* w_pad_t_dev, int d_in, int N);
 bool mg_layer_fused_supported(int d_in, int d_out);
+int mg_layer_rows(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_out, int4* row_meta);
 int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_out, const float* w_pad_t, const float* bias,
-                   const float* h_prev, float* h_out, bool relu);
+                   const float* h_prev, float* h_out, bool relu, const int4* row_meta, int64_t row_lo, int64_t row_hi,
+                   int64_t safe_src_row);
 
 namespace {
 
@@ -364,6 +366,7 @@ extern "C" int mg_model_free(mg_model* m) {
 
 static int forward_checks(mg_ctx* ctx, const mg_model* m, const mg_dense* d) {
     if (!m || !d) return mg_fail(ctx, MG_ERR_ARG, "null argument");
+    if (d->pending) return mg_fail(ctx, MG_ERR_STATE, "a sample is in flight on this mg_dense: call mg_sample_many_end first");
     if (!d->valid) return mg_fail(ctx, MG_ERR_STATE, "mg_dense holds no completed sample");
     if (d->ctx != ctx || m->ctx != ctx) return mg_fail(ctx, MG_ERR_ARG, "handle belongs to another context");
     if (!ctx->slots || ctx->feat_dim <= 0) return mg_fail(ctx, MG_ERR_STATE, "no feature table loaded");
@@ -383,6 +386,30 @@ static int64_t chunk_rows_for(int d_in) {
 
 enum { OUT_DEVICE = 0, OUT_HOST = 1, OUT_HOST_ASYNC = 2 };
 
+// hands H^k (device, packed) to the caller: device or host copy, blocking or on the side stream
+static int finish_forward(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out, int out_mode, const float* hk) {
+    cudaStream_t st = ctx->stream;
+    if (!d->ev_read_done) MG_CUDA(ctx, cudaEventCreateWithFlags(&d->ev_read_done, cudaEventDisableTiming));
+    MG_CUDA(ctx, cudaEventRecord(d->ev_read_done, st));   // the next sample into d waits for this
+    const int k = d->k;
+    const size_t out_bytes = (size_t)d->h_hdr.rows_total[k] * m->dims[k] * sizeof(float);
+    if (out_mode == OUT_HOST_ASYNC) {
+        // the copy to the host runs on the side stream behind the last layer kernel; the caller's next
+        // calls (sampling the next group) overlap it
+        MG_CUDA(ctx, cudaEventRecord(ctx->ev_fwd_done, st));
+        MG_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_fwd_done, 0));
+        MG_CUDA(ctx, cudaMemcpyAsync(out, hk, out_bytes, cudaMemcpyDeviceToHost, ctx->side));
+        MG_CUDA(ctx, cudaEventRecord(ctx->ev_out_done, ctx->side));
+        ctx->out_copy_pending = true;
+        ctx->out_check_gemm = m->precision == MG_GEMM_TF32;
+        return MG_OK;
+    }
+    MG_CUDA(ctx, cudaMemcpyAsync(out, hk, out_bytes, out_mode == OUT_DEVICE ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, st));
+    MG_CUDA(ctx, cudaStreamSynchronize(st));
+    if (m->precision == MG_GEMM_TF32) return mg_gemm_tf32_status(ctx);
+    return MG_OK;
+}
+
 static int forward_impl(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out, int out_mode) {
     if (!ctx) return MG_ERR_ARG;
     int rc = forward_checks(ctx, m, d);
@@ -394,6 +421,68 @@ static int forward_impl(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out,
     if (ctx->out_copy_pending) {   // the previous asynchronous output copy still reads the layer workspace
         MG_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_out_done, 0));
         ctx->out_copy_pending = false;
+    }
+
+    // Windowed schedule: when every layer runs in the fused kernel and the intermediate layer outputs need not
+    // be kept, the layers are run over sub-groups of a few mini-batches at a time through small reused
+    // buffers.  H^l of a sub-group is then still in L2 when layer l+1 reads it, and is overwritten in L2 by the
+    // next sub-group before most of it is written back to DRAM.
+    bool all_fused = m->precision == MG_GEMM_TF32;
+    for (int l = 1; l <= k; ++l) all_fused = all_fused && mg_layer_fused_supported(m->dims[l - 1], m->dims[l]);
+    const int sub = ctx->layer_window_batches;
+    ctx->layers_kept = !(all_fused && sub > 0 && !ctx->keep_layers && k > 1);
+    if (!ctx->layers_kept) {
+        const int32_t* rb = d->h_rowbase.data();      // [(k+1)][B+1]
+        size_t ring_off[MG_MAX_HOPS + 1] = {0}, ring_total = 0, meta_off[MG_MAX_HOPS + 1] = {0}, meta_total = 0;
+        for (int l = 1; l <= k; ++l) {
+            meta_off[l] = meta_total;
+            meta_total += (size_t)d->h_hdr.rows_total[l];
+            ring_off[l] = ring_total;
+            if (l == k) { ring_total += (size_t)d->h_hdr.rows_total[k] * m->dims[k]; break; }
+            int64_t widest = 0;
+            for (int b0 = 0; b0 < B; b0 += sub) {
+                const int b1 = std::min(B, b0 + sub);
+                widest = std::max<int64_t>(widest, rb[(size_t)l * (B + 1) + b1] - rb[(size_t)l * (B + 1) + b0]);
+            }
+            ring_total += (size_t)widest * m->dims[l];
+        }
+        {
+            size_t have = ctx->ws_h_bytes[0] / sizeof(float);
+            if (have < ring_total && (rc = mg_ensure(ctx, &ctx->ws_h[0], &have, ring_total + ring_total / 4))) return rc;
+            ctx->ws_h_bytes[0] = have * sizeof(float);
+        }
+        int4* meta = reinterpret_cast<int4*>(ctx->ws_x);
+        {
+            size_t have = ctx->ws_x_bytes / sizeof(int4);
+            if (have < meta_total) {
+                rc = mg_ensure(ctx, &meta, &have, meta_total + meta_total / 4);
+                ctx->ws_x = reinterpret_cast<float*>(meta);
+                ctx->ws_x_bytes = have * sizeof(int4);
+                if (rc) return rc;
+            }
+        }
+        {
+            ProfScope ps(ctx, PH_OTHER, k);
+            for (int l = 1; l <= k; ++l)
+                if ((rc = mg_layer_rows(ctx, d, l, m->dims[l - 1], m->dims[l], meta + meta_off[l]))) return rc;
+        }
+        float* base = ctx->ws_h[0];
+        for (int b0 = 0; b0 < B; b0 += sub) {
+            const int b1 = std::min(B, b0 + sub);
+            for (int l = 1; l <= k; ++l) {
+                const int64_t lo = rb[(size_t)l * (B + 1) + b0], hi = rb[(size_t)l * (B + 1) + b1];
+                const int64_t lo_in = rb[(size_t)(l - 1) * (B + 1) + b0];
+                // pointers shifted so that the kernel's global packed row indices land inside the windows
+                const float* h_prev = l > 1 ? base + ring_off[l - 1] - lo_in * m->dims[l - 1] : nullptr;
+                float* h_out = l == k ? base + ring_off[k] : base + ring_off[l] - lo * m->dims[l];
+                ProfScope ps(ctx, l == 1 ? PH_AGG_L1 : PH_AGG_REST, 1);
+                rc = mg_layer_fused(ctx, d, l, m->dims[l - 1], m->dims[l], m->w_pad_t[l - 1], m->bias[l - 1], h_prev, h_out,
+                                    l < k, meta + meta_off[l], lo, hi, l > 1 ? lo_in : 0);
+                if (rc) return rc;
+            }
+        }
+        MG_CUDA(ctx, cudaGetLastError());
+        return finish_forward(ctx, m, d, out, out_mode, base + ring_off[k]);
     }
 
     // per-layer outputs H^1..H^k live in one workspace (kept for mg_layer_output)
@@ -429,8 +518,17 @@ static int forward_impl(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out,
         const float* h_prev = l > 1 ? ctx->ws_h[0] + off[l - 1] : nullptr;
         if (m->precision == MG_GEMM_TF32 && mg_layer_fused_supported(d_in, d_out)) {
             // gather + segment mean + both linear maps in one persistent tensor-core kernel
-            ProfScope ps(ctx, l == 1 ? PH_AGG_L1 : PH_AGG_REST, 1);
-            rc = mg_layer_fused(ctx, d, l, d_in, d_out, m->w_pad_t[l - 1], m->bias[l - 1], h_prev, h_out, l < k);
+            ProfScope ps(ctx, l == 1 ? PH_AGG_L1 : PH_AGG_REST, 2);
+            size_t have = ctx->ws_x_bytes / sizeof(int4);
+            int4* meta = reinterpret_cast<int4*>(ctx->ws_x);
+            if (have < (size_t)M) {
+                rc = mg_ensure(ctx, &meta, &have, (size_t)M + (size_t)M / 4);
+                ctx->ws_x = reinterpret_cast<float*>(meta);
+                ctx->ws_x_bytes = have * sizeof(int4);
+                if (rc) return rc;
+            }
+            if ((rc = mg_layer_rows(ctx, d, l, d_in, d_out, meta))) return rc;
+            rc = mg_layer_fused(ctx, d, l, d_in, d_out, m->w_pad_t[l - 1], m->bias[l - 1], h_prev, h_out, l < k, meta, 0, M, 0);
             if (rc) return rc;
             continue;
         }
@@ -473,22 +571,7 @@ static int forward_impl(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out,
         }
     }
     MG_CUDA(ctx, cudaGetLastError());
-    const size_t out_bytes = (size_t)d->h_hdr.rows_total[k] * m->dims[k] * sizeof(float);
-    if (out_mode == OUT_HOST_ASYNC) {
-        // the copy to the host runs on the side stream behind the last layer kernel; the caller's next
-        // calls (sampling the next group) overlap it
-        MG_CUDA(ctx, cudaEventRecord(ctx->ev_fwd_done, st));
-        MG_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_fwd_done, 0));
-        MG_CUDA(ctx, cudaMemcpyAsync(out, ctx->ws_h[0] + off[k], out_bytes, cudaMemcpyDeviceToHost, ctx->side));
-        MG_CUDA(ctx, cudaEventRecord(ctx->ev_out_done, ctx->side));
-        ctx->out_copy_pending = true;
-        ctx->out_check_gemm = m->precision == MG_GEMM_TF32;
-        return MG_OK;
-    }
-    MG_CUDA(ctx, cudaMemcpyAsync(out, ctx->ws_h[0] + off[k], out_bytes, out_mode == OUT_DEVICE ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, st));
-    MG_CUDA(ctx, cudaStreamSynchronize(st));
-    if (m->precision == MG_GEMM_TF32) return mg_gemm_tf32_status(ctx);
-    return MG_OK;
+    return finish_forward(ctx, m, d, out, out_mode, ctx->ws_h[0] + off[k]);
 }
 
 extern "C" int mg_forward(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out, int out_on_device) {
@@ -537,6 +620,7 @@ extern "C" int mg_layer_output(mg_ctx* ctx, const mg_model* m, mg_dense* d, int3
     if (layer < 1 || layer > d->k) return mg_fail(ctx, MG_ERR_ARG, "layer must be in [1, k]");
     if (batch < 0 || batch >= d->n_batches) return mg_fail(ctx, MG_ERR_ARG, "batch out of range");
     if (!ctx->ws_h[0]) return mg_fail(ctx, MG_ERR_STATE, "mg_forward has not run");
+    if (!ctx->layers_kept) return mg_fail(ctx, MG_ERR_STATE, "the last forward did not keep its intermediate layers: call mg_keep_layer_outputs(ctx, 1) first");
     MG_CUDA(ctx, cudaSetDevice(ctx->device));
     size_t off = 0;
     for (int l = 1; l < layer; ++l) off += (size_t)d->h_hdr.rows_total[l] * m->dims[l];
@@ -649,5 +733,18 @@ extern "C" int mg_forward_noalloc(mg_ctx* ctx, const mg_model* m, mg_dense* d, f
     MG_CUDA(ctx, cudaGetLastError());
     MG_CUDA(ctx, cudaStreamSynchronize(st));
     if (m->precision == MG_GEMM_TF32) return mg_gemm_tf32_status(ctx);
+    return MG_OK;
+}
+
+extern "C" int mg_keep_layer_outputs(mg_ctx* ctx, int enable) {
+    if (!ctx) return MG_ERR_ARG;
+    ctx->keep_layers = enable != 0;
+    return MG_OK;
+}
+
+extern "C" int mg_set_layer_window(mg_ctx* ctx, int32_t mini_batches) {
+    if (!ctx) return MG_ERR_ARG;
+    if (mini_batches < 0) return mg_fail(ctx, MG_ERR_ARG, "negative window");
+    ctx->layer_window_batches = mini_batches;
     return MG_OK;
 }

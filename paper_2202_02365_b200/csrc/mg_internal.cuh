@@ -59,7 +59,9 @@ enum {
 struct mg_ctx {
     int device = 0;
     cudaStream_t stream = nullptr;
-    cudaStream_t side = nullptr;  // partition swaps
+    cudaStream_t side = nullptr;  // partition swaps, asynchronous output copies
+    cudaStream_t sample_stream = nullptr;  // all sampling kernels
+    cudaEvent_t ev_user = nullptr;
     std::string err;
     int64_t launches = 0;
     int n_sms = 148;
@@ -102,6 +104,11 @@ struct mg_ctx {
     float* ws_x = nullptr; size_t ws_x_bytes = 0;
     float* ws_h[2] = {nullptr, nullptr}; size_t ws_h_bytes[2] = {0, 0};
     float** ws_layer = nullptr;
+
+    // forward schedule
+    int32_t layer_window_batches = 0;  // mini-batches per window of the layer schedule; 0 = whole layers
+    bool keep_layers = false;          // keep H^1..H^{k-1} for mg_layer_output (whole-layer schedule)
+    bool layers_kept = false;          // what the last forward did
 
     // asynchronous output copy of mg_forward_host_async
     cudaEvent_t ev_fwd_done = nullptr, ev_out_done = nullptr;
@@ -155,6 +162,11 @@ struct mg_dense {
     std::vector<int32_t> h_ent_hop;  // [k * (B+1)] arena entry index where batch b's hop-h entries start
     int32_t* d_ent_hop = nullptr;    // device copy of the same
     bool valid = false;
+    // asynchronous sampling: the summary lands in pinned memory, ev_sampled marks its arrival
+    int32_t* h_pinned = nullptr; size_t h_pinned_ints = 0;
+    cudaEvent_t ev_sampled = nullptr;
+    cudaEvent_t ev_read_done = nullptr;  // recorded after the last kernel that read this sample
+    bool pending = false;
 };
 
 struct mg_model {

@@ -58,11 +58,13 @@ struct FusedArgs {
     const int32_t* slot_of_part;
     int64_t slot_bytes, row_bytes;
     uint32_t part_size;
+    int32_t safe_src;            // a source row that is always valid to read (rows past the end load it)
     int32_t identity_rows;       // layer 1: slot == partition for every resident partition (whole table in HBM)
     // shapes
     int32_t d_in, d_in_pad;      // d_in_pad = d_in rounded up to 32; K = 2 * d_in_pad
     int32_t N, BN;               // output width and its MMA tile width (multiple of 16, <= 256)
-    int64_t M;                   // packed output rows of the layer
+    int64_t row_lo;              // first packed output row this launch computes
+    int64_t M;                   // one past its last packed output row
     int32_t sa, sb;              // A and B stages
     int32_t tmem_cols;
     int32_t relu;
@@ -122,7 +124,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, FusedArgs a) {
     uint8_t* a_base = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* b_base = a_base + (size_t)a.sa * kABytes;
     const int n_chunks = 2 * a.d_in_pad / KC;
-    const int64_t n_tiles = (a.M + BM - 1) / BM;
+    const int64_t n_tiles = (a.M - a.row_lo + BM - 1) / BM;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < a.sa; ++s) { mbar_init(&a_full[s], kProducerWarps); mbar_init(&a_empty[s], 1); }
@@ -194,7 +196,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, FusedArgs a) {
             const uint32_t buf = it & 1;
             if (!mbar_wait(&acc_full[buf], (it >> 1) & 1)) { if (lane == 0) atomicExch(a.error, 14u); ok = false; break; }
             tc_fence_after();
-            const int64_t row0 = t * BM + lane_group * 32;
+            const int64_t row0 = a.row_lo + t * BM + lane_group * 32;
             for (int c0 = 0; c0 < a.BN; c0 += 32) {
                 uint32_t v[32];
                 tmem_ld_32(tmem_base + buf * acc_stride + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)c0, v);
@@ -217,10 +219,10 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, FusedArgs a) {
             // row metadata of the tile and the source rows of all its entries, once per tile
             asm volatile("bar.sync 1, %0;" ::"r"(kProducerWarps * 32) : "memory");   // previous tile's readers are done
             RowMeta mm;
-            mm.self_src = 0; mm.e0 = 0; mm.cnt = -1; mm.koff = -1; mm.in_base = 0;
+            mm.self_src = a.safe_src; mm.e0 = 0; mm.cnt = -1; mm.koff = -1; mm.in_base = 0;
             uint32_t incl = 0;
             if (ptid < BM) {
-                const int64_t r = t * BM + ptid;
+                const int64_t r = a.row_lo + t * BM + ptid;
                 if (r < a.M) {
                     const int4 rm = __ldg(a.row_meta + r);   // (self_src, e0, cnt, in_base) from the pre-pass
                     mm.self_src = rm.x; mm.e0 = rm.y; mm.cnt = rm.z; mm.in_base = rm.w;
@@ -421,39 +423,64 @@ int mg_pack_layer_weights(mg_ctx* ctx, const float* w_cat_dev, float* w_pad_t_de
 
 bool mg_layer_fused_supported(int d_in, int d_out) { return d_out <= 256 && d_out % 4 == 0 && d_in % 4 == 0; }
 
-// Runs layer `layer` (1-based) of the model over all mini-batches of the sample.
-int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_out, const float* w_pad_t, const float* bias,
-                   const float* h_prev, float* h_out, bool relu) {
-    const int64_t M = d->h_hdr.rows_total[layer];
-    if (M <= 0) return MG_OK;
+static void fill_args(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_out, FusedArgs* pa) {
+    FusedArgs& a = *pa;
     const int B = d->n_batches;
-    FusedArgs a;
     a.B = B; a.k = d->k; a.layer = layer;
     a.rowbase_out = d->rowbase + (size_t)layer * (B + 1);
     a.rowbase_in = d->rowbase + (size_t)(layer - 1) * (B + 1);
     a.cum = d->cum; a.node_off = d->node_off; a.nodes = d->nodes;
     a.ent_off = d->ent_off; a.ent_nbrs = d->ent_nbrs; a.ent_repr = d->ent_repr;
-    a.h_prev = h_prev;
-    a.src_base = layer == 1 ? ctx->slots : reinterpret_cast<const char*>(h_prev);
-    a.src_row_bytes = layer == 1 ? ctx->row_bytes : (int64_t)d_in * 4;
+    a.slots = ctx->slots; a.slot_of_part = ctx->d_slot_of_part;
+    a.slot_bytes = ctx->slot_bytes; a.row_bytes = ctx->row_bytes; a.part_size = (uint32_t)ctx->part_size;
     a.identity_rows = 1;
     for (int p = 0; p < ctx->n_parts; ++p)
         if (ctx->slot_of_part[p] >= 0 && ctx->slot_of_part[p] != p) a.identity_rows = 0;
-    a.slots = ctx->slots; a.slot_of_part = ctx->d_slot_of_part;
-    a.slot_bytes = ctx->slot_bytes; a.row_bytes = ctx->row_bytes; a.part_size = (uint32_t)ctx->part_size;
     a.d_in = d_in;
     a.d_in_pad = (d_in + KC - 1) / KC * KC;
     a.N = d_out;
     a.BN = (d_out + 15) / 16 * 16;
-    a.M = M;
+    a.row_lo = 0;
+    a.M = d->h_hdr.rows_total[layer];
+    a.error = ctx->d_flags;
+}
+
+// Pre-pass of one layer: row_meta[r] for every packed output row r of the layer.
+int mg_layer_rows(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_out, int4* row_meta) {
+    FusedArgs a;
+    memset(&a, 0, sizeof(a));
+    fill_args(ctx, d, layer, d_in, d_out, &a);
+    if (a.M <= 0) return MG_OK;
+    if (layer == 1) k_layer_rows<true><<<mg_grid(ctx, 8), 256, 0, ctx->stream>>>(a, row_meta);
+    else k_layer_rows<false><<<mg_grid(ctx, 8), 256, 0, ctx->stream>>>(a, row_meta);
+    ctx->launches++;
+    return MG_OK;
+}
+
+// Runs layer `layer` (1-based) for the packed output rows [row_lo, row_hi).  h_prev and h_out are indexed by
+// GLOBAL packed row (callers that keep only a window of a layer pass pointers shifted accordingly).
+int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_out, const float* w_pad_t, const float* bias,
+                   const float* h_prev, float* h_out, bool relu, const int4* row_meta, int64_t row_lo, int64_t row_hi,
+                   int64_t safe_src_row) {
+    if (row_hi <= row_lo) return MG_OK;
+    FusedArgs a;
+    memset(&a, 0, sizeof(a));
+    fill_args(ctx, d, layer, d_in, d_out, &a);
+    a.row_lo = row_lo;
+    a.M = row_hi;
+    a.row_meta = row_meta;
+    a.safe_src = (int32_t)safe_src_row;
+    a.h_prev = h_prev;
+    a.src_base = layer == 1 ? ctx->slots : reinterpret_cast<const char*>(h_prev);
+    a.src_row_bytes = layer == 1 ? ctx->row_bytes : (int64_t)d_in * 4;
     a.relu = relu ? 1 : 0;
-    a.bias = bias; a.out = h_out; a.error = ctx->d_flags;
+    a.bias = bias; a.out = h_out;
     int stride = 32;
     while (stride < a.BN) stride <<= 1;
     a.tmem_cols = 2 * stride;   // two accumulator buffers, each a power of two >= 32 columns
     const int b_bytes = a.BN * KC * 4;
     const int n_chunks = 2 * a.d_in_pad / KC;
-    a.sa = std::min(8, n_chunks);   // two groups of (self, mean) slice pairs, 64 input columns each
+    a.sa = std::min(8, n_chunks);   // one group of (self, mean) slice pairs: 128 input columns
     a.sb = std::max(2, std::min({kMaxStages, n_chunks, (int)((194 * 1024 - a.sa * (int)kABytes) / b_bytes)}));
     const size_t smem = (size_t)a.sa * kABytes + (size_t)a.sb * b_bytes + 1024;
     CUtensorMap mw;
@@ -462,19 +489,7 @@ int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_ou
     const bool first = layer == 1, half = first && ctx->feat_dtype == MG_DTYPE_F16;
     auto kern = first ? (half ? k_sage_layer_fused<true, true> : k_sage_layer_fused<true, false>) : k_sage_layer_fused<false, false>;
     MG_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    {
-        size_t have = ctx->ws_x_bytes / sizeof(int4);
-        int4* buf = reinterpret_cast<int4*>(ctx->ws_x);
-        int rc = have >= (size_t)M ? MG_OK : mg_ensure(ctx, &buf, &have, (size_t)M + (size_t)M / 4);
-        ctx->ws_x = reinterpret_cast<float*>(buf);
-        ctx->ws_x_bytes = have * sizeof(int4);
-        if (rc) return rc;
-        a.row_meta = buf;
-        if (first) k_layer_rows<true><<<mg_grid(ctx, 8), 256, 0, ctx->stream>>>(a, buf);
-        else k_layer_rows<false><<<mg_grid(ctx, 8), 256, 0, ctx->stream>>>(a, buf);
-        ctx->launches++;
-    }
-    const int64_t n_tiles = (M + BM - 1) / BM;
+    const int64_t n_tiles = (row_hi - row_lo + BM - 1) / BM;
     const int grid = (int)std::min<int64_t>(n_tiles, ctx->n_sms);
     kern<<<grid, kFusedThreads, smem, ctx->stream>>>(mw, a);
     ctx->launches++;

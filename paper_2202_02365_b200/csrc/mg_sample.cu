@@ -806,9 +806,55 @@ static int status_code(uint32_t st) {
     return MG_ERR_CUDA;
 }
 
+// All sampling work is queued on the library's sampling stream, so that it can overlap a forward pass that is
+// running on the context's stream.  The sampling stream first waits for whatever the caller had queued on the
+// context's stream (e.g. the kernel that produced device-resident targets).
+static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on_device,
+                             const int64_t* target_offsets, int32_t n_batches, const int32_t* fanouts,
+                             int32_t k, const uint64_t* seeds, const mg_sample_caps* caps, mg_dense** out);
+
+extern "C" int mg_sample_many_begin(mg_ctx* ctx, const int32_t* targets, int targets_on_device,
+                                    const int64_t* target_offsets, int32_t n_batches, const int32_t* fanouts,
+                                    int32_t k, const uint64_t* seeds, const mg_sample_caps* caps, mg_dense** out) {
+    if (!ctx) return MG_ERR_ARG;
+    cudaStream_t user = ctx->stream;
+    if (cudaEventRecord(ctx->ev_user, user) == cudaSuccess) cudaStreamWaitEvent(ctx->sample_stream, ctx->ev_user, 0);
+    ctx->stream = ctx->sample_stream;     // every helper launches on ctx->stream
+    const int rc = sample_begin_impl(ctx, targets, targets_on_device, target_offsets, n_batches, fanouts, k, seeds, caps, out);
+    ctx->stream = user;
+    return rc;
+}
+
+extern "C" int mg_sample_many_end(mg_ctx* ctx, mg_dense* d) {
+    if (!ctx) return MG_ERR_ARG;
+    if (!d) return mg_fail(ctx, MG_ERR_ARG, "null mg_dense");
+    if (!d->pending) return mg_fail(ctx, MG_ERR_STATE, "no sample in flight on this mg_dense");
+    MG_CUDA(ctx, cudaSetDevice(ctx->device));
+    d->pending = false;
+    MG_CUDA(ctx, cudaEventSynchronize(d->ev_sampled));
+    const int B = d->n_batches, k = d->k;
+    const int32_t* p = d->h_pinned;
+    memcpy(&d->h_hdr, p, sizeof(DenseHeader)); p += (sizeof(DenseHeader) + 3) / 4;
+    d->h_cum.assign(p, p + (size_t)B * (k + 2)); p += (size_t)B * (k + 2);
+    d->h_node_off.assign(p, p + (size_t)(k + 1) * (B + 1)); p += (size_t)(k + 1) * (B + 1);
+    d->h_rowbase.assign(p, p + (size_t)(k + 1) * (B + 1)); p += (size_t)(k + 1) * (B + 1);
+    d->h_ent_hop.assign(p, p + (size_t)k * (B + 1));
+    if (d->h_hdr.status) return mg_fail(ctx, status_code(d->h_hdr.status), "%s", status_text(d->h_hdr.status));
+    d->valid = true;
+    return MG_OK;
+}
+
 extern "C" int mg_sample_many(mg_ctx* ctx, const int32_t* targets, int targets_on_device,
                               const int64_t* target_offsets, int32_t n_batches, const int32_t* fanouts,
                               int32_t k, const uint64_t* seeds, const mg_sample_caps* caps, mg_dense** out) {
+    const int rc = mg_sample_many_begin(ctx, targets, targets_on_device, target_offsets, n_batches, fanouts, k, seeds, caps, out);
+    if (rc) return rc;
+    return mg_sample_many_end(ctx, *out);
+}
+
+static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on_device,
+                             const int64_t* target_offsets, int32_t n_batches, const int32_t* fanouts,
+                             int32_t k, const uint64_t* seeds, const mg_sample_caps* caps, mg_dense** out) {
     if (!ctx) return MG_ERR_ARG;
     if (!out || !target_offsets || !fanouts || !seeds) return mg_fail(ctx, MG_ERR_ARG, "null argument");
     if (n_batches <= 0 || n_batches > MG_MAX_BATCHES) return mg_fail(ctx, MG_ERR_ARG, "n_batches must be in [1, %d]", MG_MAX_BATCHES);
@@ -864,6 +910,8 @@ extern "C" int mg_sample_many(mg_ctx* ctx, const int32_t* targets, int targets_o
     if (created) { d = new mg_dense(); d->ctx = ctx; d->device = ctx->device; }
     else if (d->ctx != ctx) return mg_fail(ctx, MG_ERR_ARG, "mg_dense belongs to another context");
     d->valid = false;
+    d->pending = false;
+    if (d->ev_read_done) MG_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, d->ev_read_done, 0));
     int rc = dense_alloc(ctx, d, n_batches, k, cap_nodes, std::max<int64_t>(cap_entries, 1), table_size);
     if (rc) { if (created) mg_dense_free(d); return rc; }
     *out = d;
@@ -960,19 +1008,28 @@ extern "C" int mg_sample_many(mg_ctx* ctx, const int32_t* targets, int targets_o
     }
     MG_CUDA(ctx, cudaGetLastError());
 
-    // read the summary back (the one host sync of a sample)
-    d->h_cum.resize((size_t)B * (k + 2));
-    d->h_node_off.resize((size_t)(k + 1) * (B + 1));
-    d->h_rowbase.resize((size_t)(k + 1) * (B + 1));
-    d->h_ent_hop.resize((size_t)k * (B + 1));
-    MG_CUDA(ctx, cudaMemcpyAsync(&d->h_hdr, d->hdr, sizeof(DenseHeader), cudaMemcpyDeviceToHost, st));
-    MG_CUDA(ctx, cudaMemcpyAsync(d->h_cum.data(), d->cum, sizeof(int32_t) * d->h_cum.size(), cudaMemcpyDeviceToHost, st));
-    MG_CUDA(ctx, cudaMemcpyAsync(d->h_node_off.data(), d->node_off, sizeof(int32_t) * d->h_node_off.size(), cudaMemcpyDeviceToHost, st));
-    MG_CUDA(ctx, cudaMemcpyAsync(d->h_rowbase.data(), d->rowbase, sizeof(int32_t) * d->h_rowbase.size(), cudaMemcpyDeviceToHost, st));
-    MG_CUDA(ctx, cudaMemcpyAsync(d->h_ent_hop.data(), d->d_ent_hop, sizeof(int32_t) * d->h_ent_hop.size(), cudaMemcpyDeviceToHost, st));
-    MG_CUDA(ctx, cudaStreamSynchronize(st));
-    if (d->h_hdr.status) return mg_fail(ctx, status_code(d->h_hdr.status), "%s", status_text(d->h_hdr.status));
-    d->valid = true;
+    // the summary goes to pinned host memory behind the kernels; mg_sample_many_end waits for it
+    {
+        const size_t n_ints = (sizeof(DenseHeader) + 3) / 4 + (size_t)B * (k + 2) + 2 * (size_t)(k + 1) * (B + 1) + (size_t)k * (B + 1);
+        if (d->h_pinned_ints < n_ints) {
+            if (d->h_pinned) cudaFreeHost(d->h_pinned);
+            d->h_pinned = nullptr; d->h_pinned_ints = 0;
+            if (cudaHostAlloc((void**)&d->h_pinned, n_ints * sizeof(int32_t), cudaHostAllocDefault) != cudaSuccess) {
+                cudaGetLastError();
+                return mg_fail(ctx, MG_ERR_OOM, "pinned host allocation failed");
+            }
+            d->h_pinned_ints = n_ints;
+        }
+        int32_t* p = d->h_pinned;
+        MG_CUDA(ctx, cudaMemcpyAsync(p, d->hdr, sizeof(DenseHeader), cudaMemcpyDeviceToHost, st)); p += (sizeof(DenseHeader) + 3) / 4;
+        MG_CUDA(ctx, cudaMemcpyAsync(p, d->cum, sizeof(int32_t) * (size_t)B * (k + 2), cudaMemcpyDeviceToHost, st)); p += (size_t)B * (k + 2);
+        MG_CUDA(ctx, cudaMemcpyAsync(p, d->node_off, sizeof(int32_t) * (size_t)(k + 1) * (B + 1), cudaMemcpyDeviceToHost, st)); p += (size_t)(k + 1) * (B + 1);
+        MG_CUDA(ctx, cudaMemcpyAsync(p, d->rowbase, sizeof(int32_t) * (size_t)(k + 1) * (B + 1), cudaMemcpyDeviceToHost, st)); p += (size_t)(k + 1) * (B + 1);
+        MG_CUDA(ctx, cudaMemcpyAsync(p, d->d_ent_hop, sizeof(int32_t) * (size_t)k * (B + 1), cudaMemcpyDeviceToHost, st));
+    }
+    if (!d->ev_sampled) MG_CUDA(ctx, cudaEventCreateWithFlags(&d->ev_sampled, cudaEventDisableTiming));
+    MG_CUDA(ctx, cudaEventRecord(d->ev_sampled, st));
+    d->pending = true;
     return MG_OK;
 }
 
@@ -1062,6 +1119,9 @@ extern "C" int mg_dense_free(mg_dense* d) {
     cudaFree(d->rowbase); cudaFree(d->hkeys); cudaFree(d->hvals); cudaFree(d->newlist[0]);
     cudaFree(d->newlist[1]); cudaFree(d->d_seeds); cudaFree(d->scan_tmp); cudaFree(d->sort_hist);
     cudaFree(d->exp_buf); cudaFree(d->d_ent_hop);
+    if (d->h_pinned) cudaFreeHost(d->h_pinned);
+    if (d->ev_sampled) cudaEventDestroy(d->ev_sampled);
+    if (d->ev_read_done) cudaEventDestroy(d->ev_read_done);
     delete d;
     return MG_OK;
 }

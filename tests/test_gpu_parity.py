@@ -520,3 +520,71 @@ def test_async_host_output_equals_blocking_forward(tiny):
     ctx.wait_output()
     for i in range(2):
         assert torch.equal(outs_async[i], want[i])
+
+
+@pytest.mark.parametrize("window", [1, 3, 16])
+def test_windowed_layer_schedule_gives_the_same_output(tiny, window):
+    g, feats = tiny
+    ctx = make_ctx(g, feats)
+    sizes = [200, 0, 13, 200, 1, 300, 64, 128, 5]
+    B = len(sizes)
+    tg = [inputs.distinct_targets(10_000, s, seed=30 + i) for i, s in enumerate(sizes)]
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    d = ctx.sample_many(torch.cat(tg), offs, [4, 3, 2], [500 + i for i in range(B)])
+    layers = inputs.random_bias_layers([16, 32, 64, 8], seed=9)
+    model = ctx.model(layers, mg.GEMM_TF32)
+    want = torch.empty((int(offs[-1]), 8), dtype=torch.float32, device="cuda")
+    ctx.forward(model, d, want)
+    ctx.set_layer_window(window)
+    got = torch.full_like(want, float("nan"))
+    ctx.forward(model, d, got)
+    assert torch.equal(got, want)
+    with pytest.raises(mg.MgError) as e:          # the windows do not keep H^1, H^2
+        ctx.layer_output(model, d, 1, 0, 10)
+    assert e.value.code == -2
+    ctx.keep_layer_outputs(True)
+    ctx.forward(model, d, got)
+    assert torch.equal(got, want)
+    nodes, _ = d.counts()
+    assert ctx.layer_output(model, d, 1, 0, int(nodes[0, :3].sum())).shape[1] == 32
+
+
+def test_sampling_overlapped_with_forward_matches_blocking_calls(tiny):
+    """mg_sample_many_begin / _end: group i+1 is sampled on the sampling stream while group i runs its
+    layers; results equal the blocking calls, and an unfinished sample cannot be used."""
+    g, feats = tiny
+    ctx = make_ctx(g, feats)
+    layers = inputs.random_bias_layers([16, 32, 8], seed=3)
+    model = ctx.model(layers, mg.GEMM_TF32)
+    B, T, steps = 4, 150, 5
+    offs = [T * i for i in range(B + 1)]
+    tgs = [torch.cat([inputs.distinct_targets(10_000, T, seed=1000 * s + b) for b in range(B)]).cuda() for s in range(steps)]
+    seeds = [[10 * s + b for b in range(B)] for s in range(steps)]
+    want = []
+    for s in range(steps):
+        d = ctx.sample_many(tgs[s], offs, [6, 4], seeds[s])
+        o = torch.empty((B * T, 8), dtype=torch.float32, device="cuda")
+        ctx.forward(model, d, o)
+        want.append((o, d.view(B - 1).node_ids.clone()))
+    denses = [None, None]
+    denses[0] = ctx.sample_many_begin(tgs[0], offs, [6, 4], seeds[0])
+    with pytest.raises(mg.MgError) as e:
+        ctx.forward(model, denses[0], torch.empty((B * T, 8), dtype=torch.float32, device="cuda"))
+    assert e.value.code == -2                       # still in flight
+    outs = [torch.empty((B * T, 8), dtype=torch.float32, device="cuda") for _ in range(steps)]
+    for s in range(steps):
+        ctx.sample_many_end(denses[s & 1])
+        if s + 1 < steps:
+            denses[(s + 1) & 1] = ctx.sample_many_begin(tgs[s + 1], offs, [6, 4], seeds[s + 1], out=denses[(s + 1) & 1])
+        ctx.forward(model, denses[s & 1], outs[s])
+        assert torch.equal(denses[s & 1].view(B - 1).node_ids, want[s][1])
+    for s in range(steps):
+        assert torch.equal(outs[s], want[s][0])
+    with pytest.raises(mg.MgError) as e:
+        ctx.sample_many_end(denses[0])
+    assert e.value.code == -2                       # nothing in flight
+    # errors of an asynchronous sample surface at its end
+    bad = ctx.sample_many_begin(torch.tensor([1, 1], dtype=torch.int32), [0, 2], [3], [0])
+    with pytest.raises(mg.MgError) as e:
+        ctx.sample_many_end(bad)
+    assert e.value.code == -4
