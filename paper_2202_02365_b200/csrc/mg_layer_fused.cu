@@ -108,7 +108,7 @@ __device__ __forceinline__ float4 load4(const char* p) {
 
 template <bool FIRST, bool HALF>
 __global__ void __launch_bounds__(kFusedThreads, 1)
-k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, FusedArgs a) {
+k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_out, FusedArgs a) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t a_full[kMaxStages], a_empty[kMaxStages], b_full[kMaxStages], b_empty[kMaxStages];
     __shared__ uint64_t acc_full[2], acc_empty[2];
@@ -117,7 +117,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, FusedArgs a) {
     __shared__ int32_t src_rows[kKeyCap];
     __shared__ uint32_t key_warp_sum[BM / 32];
     __shared__ int32_t key_end[BM];
-    __shared__ float out_stage[4][32 * 33];   // per epilogue warp: transpose buffer for coalesced stores
+    __shared__ __align__(1024) float out_stage[4][32 * 32];   // per epilogue warp: one 32 x 32 slice, 128-byte swizzled, for the TMA store
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t b_bytes = (uint32_t)a.BN * KC * 4;
@@ -132,6 +132,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, FusedArgs a) {
         for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out) : "memory");
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"((uint32_t)a.tmem_cols) : "memory");
@@ -197,11 +198,37 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, FusedArgs a) {
             if (!mbar_wait(&acc_full[buf], (it >> 1) & 1)) { if (lane == 0) atomicExch(a.error, 14u); ok = false; break; }
             tc_fence_after();
             const int64_t row0 = a.row_lo + t * BM + lane_group * 32;
+            uint8_t* stage = reinterpret_cast<uint8_t*>(out_stage[lane_group]);
             for (int c0 = 0; c0 < a.BN; c0 += 32) {
                 uint32_t v[32];
                 tmem_ld_32(tmem_base + buf * acc_stride + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)c0, v);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (row0 < a.M) store_slice_coalesced(v, out_stage[lane_group], a.bias, a.out, row0, a.M, a.N, c0, a.relu != 0);
+                if (row0 < a.M && c0 < a.N) {
+                    // the previous slice's TMA store must have read the staging tile before it is rewritten
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    __syncwarp();
+                    // lane = row of the slice; 16-byte piece c of the row goes to piece c ^ (row % 8) (128-byte swizzle)
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const int n = c0 + 4 * c;
+                        float4 o = make_float4(__uint_as_float(v[4 * c]), __uint_as_float(v[4 * c + 1]),
+                                               __uint_as_float(v[4 * c + 2]), __uint_as_float(v[4 * c + 3]));
+                        if (n < a.N) {
+                            const float4 bb = __ldg(reinterpret_cast<const float4*>(a.bias + n));
+                            o.x += bb.x; o.y += bb.y; o.z += bb.z; o.w += bb.w;
+                        }
+                        if (a.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f); }
+                        *reinterpret_cast<float4*>(stage + lane * 128 + ((c ^ (lane & 7)) << 4)) = o;
+                    }
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        // rows past the end of the layer and columns past its width are clipped by the tensor map
+                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                                     ::"l"(&map_out), "r"(smem_u32(stage)), "r"(c0), "r"((int)row0) : "memory");
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    }
+                }
             }
             tc_fence_before();
             __syncwarp();
@@ -368,6 +395,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, FusedArgs a) {
             }
         }
     }
+    if (warp >= 2 && warp < kFirstProducerWarp && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -486,12 +514,17 @@ int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_ou
     CUtensorMap mw;
     if (!make_map_f32(&mw, w_pad_t, d_out, 2 * a.d_in_pad, a.BN))
         return mg_fail(ctx, MG_ERR_CUDA, "cuTensorMapEncodeTiled failed for the layer weights");
+    // output [row_hi rows, d_out] fp32, 32 x 32 boxes, 128-byte swizzle; rows are global packed rows, so a window's
+    // shifted base pointer works unchanged (rows below row_lo are never stored)
+    CUtensorMap mo;
+    if (!make_map_f32(&mo, h_out, row_hi, d_out, 32))
+        return mg_fail(ctx, MG_ERR_CUDA, "cuTensorMapEncodeTiled failed for the layer output");
     const bool first = layer == 1, half = first && ctx->feat_dtype == MG_DTYPE_F16;
     auto kern = first ? (half ? k_sage_layer_fused<true, true> : k_sage_layer_fused<true, false>) : k_sage_layer_fused<false, false>;
     MG_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const int64_t n_tiles = (row_hi - row_lo + BM - 1) / BM;
     const int grid = (int)std::min<int64_t>(n_tiles, ctx->n_sms);
-    kern<<<grid, kFusedThreads, smem, ctx->stream>>>(mw, a);
+    kern<<<grid, kFusedThreads, smem, ctx->stream>>>(mw, mo, a);
     ctx->launches++;
     MG_CUDA(ctx, cudaGetLastError());
     return MG_OK;
