@@ -890,7 +890,7 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
     int64_t cap_nodes = (caps && caps->max_nodes_total > 0) ? caps->max_nodes_total : worst_nodes_total;
     int64_t cap_entries = (caps && caps->max_entries_total > 0) ? caps->max_entries_total : worst_entries_total;
     int64_t cap_batch = (caps && caps->max_nodes_per_batch > 0) ? caps->max_nodes_per_batch : worst_nodes_batch;
-    cap_nodes = std::max<int64_t>(cap_nodes, T);
+    cap_nodes = std::max<int64_t>({cap_nodes, T, 1});   // even an empty call needs its (one-element) arrays
     cap_batch = std::max<int64_t>(cap_batch, 1);
     for (int b = 0; b < n_batches; ++b) cap_batch = std::max<int64_t>(cap_batch, target_offsets[b + 1] - target_offsets[b]);
     if (cap_nodes >= (1ll << 31) - 1 || cap_entries >= (1ll << 31) - 1)
@@ -974,7 +974,11 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
             else if (f <= 8) k_pick<8><<<grid, kThreads, 0, st>>>(a);
             else if (f <= 16) k_pick<16><<<grid, kThreads, 0, st>>>(a);
             else if (f <= 32) k_pick<32><<<grid, kThreads, 0, st>>>(a);
-            else k_pick_wide<<<grid, kThreads, (size_t)(kThreads / 32) * 2 * f * sizeof(uint32_t), st>>>(a);
+            else {
+                const size_t wide_smem = (size_t)(kThreads / 32) * 2 * f * sizeof(uint32_t);   // 64 KiB at the largest fanout
+                MG_CUDA(ctx, cudaFuncSetAttribute(k_pick_wide, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)wide_smem));
+                k_pick_wide<<<grid, kThreads, wide_smem, st>>>(a);
+            }
             InsertArgs ia{d->hdr, h, d->ent_nbrs, d->ent_repr, d->hkeys, tg, d->newlist[0], d->cap_nodes, id_bits};
             k_insert<<<grid, kThreads, 0, st>>>(ia);
             ctx->launches++;

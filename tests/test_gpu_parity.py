@@ -588,3 +588,38 @@ def test_sampling_overlapped_with_forward_matches_blocking_calls(tiny):
     with pytest.raises(mg.MgError) as e:
         ctx.sample_many_end(bad)
     assert e.value.code == -4
+
+
+def test_extremes_largest_fanout_deepest_sample_all_nodes_empty_call():
+    # a hub with 3000 in-neighbours and the largest supported fanout (1024): Floyd over a wide row
+    n = 4000
+    hub_src = torch.arange(1, 3001)
+    src = torch.cat([hub_src, torch.randint(0, n, (20_000,), generator=torch.Generator().manual_seed(1))])
+    dst = torch.cat([torch.zeros(3000, dtype=torch.int64), torch.randint(0, n, (20_000,), generator=torch.Generator().manual_seed(2))])
+    g = inputs.build_csr(src, dst, n)
+    ctx = make_ctx(g)
+    view = oracle_view(g)
+    t = torch.tensor([0, 5, 9], dtype=torch.int32)
+    d = ctx.sample(t, [1024, 2], seed=3)
+    ref = O.sample_dense(view, t.tolist(), [1024, 2], 3)
+    assert_dense_equal(d.view(0), ref)
+    assert np.diff(ref["nbr_offsets"])[-3] == 1024          # the hub keeps exactly the largest fanout
+    with pytest.raises(mg.MgError) as e:
+        ctx.sample(t, [1025], seed=3)
+    assert e.value.code == -1
+    # the deepest sample the library takes (8 hops), fanout 1 and 2
+    d = ctx.sample(t, [2, 1, 2, 1, 2, 1, 2, 1], seed=4)
+    assert_dense_equal(d.view(0), O.sample_dense(view, t.tolist(), [2, 1, 2, 1, 2, 1, 2, 1], 4))
+    with pytest.raises(mg.MgError) as e:
+        ctx.sample(t, [1] * 9, seed=4)
+    assert e.value.code == -1
+    # every node of the graph as a target: nothing new can be found, all deltas but the targets are empty
+    allv = torch.arange(n, dtype=torch.int32)
+    d = ctx.sample(allv, [3, 3], seed=5)
+    ref = O.sample_dense(view, allv.tolist(), [3, 3], 5)
+    assert_dense_equal(d.view(0), ref)
+    assert ref["node_id_offsets"] == [0, 0, 0, n]
+    # no targets at all
+    d = ctx.sample(torch.empty(0, dtype=torch.int32), [3], seed=0)
+    v = d.view(0)
+    assert v.node_ids.numel() == 0 and v.nbrs.numel() == 0 and v.node_id_offsets.cpu().tolist() == [0, 0, 0]
