@@ -32,6 +32,10 @@ CONFIGS = {
                             batch=1000, parts=1, train=1_000_000),
     "config3_papers100m_shaped": dict(n=111_000_000, m=1_620_000_000, kind="rmat", dim=128, hidden=256,
                                       fanouts=[15, 10, 5], batch=1000, parts=16, train=1_100_000),
+    # config 4's shapes at a tenth of its node count, whole fp16 table in HBM (no swaps): a throughput probe of the
+    # wide fp16 layer-1 path, not the out-of-core configuration itself (that one is exercised by the tests)
+    "config4_tenth_fp16_768_in_hbm": dict(n=12_200_000, m=130_000_000, kind="rmat", dim=768, hidden=256,
+                                          fanouts=[15, 10, 5], batch=1000, parts=1, train=12_200_000, fp16=True),
 }
 DEFAULT_WORKLOAD = "config3_papers100m_shaped"
 HBM_NOMINAL_GBS = 8000.0
@@ -102,7 +106,8 @@ def build_workload(cfg, device, seed=0):
         g = inputs.rmat_graph(cfg["n"], cfg["m"], seed, device)
     torch.cuda.synchronize()
     t1 = time.time()
-    feats = inputs.normal_features(cfg["n"], cfg["dim"], seed + 1, device)
+    feats = inputs.normal_features(cfg["n"], cfg["dim"], seed + 1, device,
+                                   dtype=torch.float16 if cfg.get("fp16") else torch.float32)
     torch.cuda.synchronize()
     dims = [cfg["dim"]] + [cfg["hidden"]] * len(cfg["fanouts"])
     layers = inputs.glorot_layers(dims, seed + 2)
@@ -303,7 +308,7 @@ def main():
 
     nodes = torch.cat(stats["nodes"]).numpy()
     ents = torch.cat(stats["ents"]).numpy()
-    alg = algorithmic_bytes(nodes, ents, cfg)
+    alg = algorithmic_bytes(nodes, ents, cfg, feat_bytes=2 if cfg.get("fp16") else 4)
     n_batches = args.steps * G * world
     value = n_batches / (ms_dev / 1e3)
     e2e_value = n_batches / (ms_e2e / 1e3)
