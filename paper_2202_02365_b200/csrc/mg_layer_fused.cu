@@ -29,12 +29,15 @@ constexpr int BM = 128;               // output rows per tile
 constexpr int KC = 32;                // floats per K slice (one 128-byte swizzle row)
 constexpr int kProducerWarps = 16;
 constexpr int kFirstProducerWarp = 6; // warp 0 TMA, warp 1 MMA + tensor memory, warps 2..5 epilogue
-constexpr int kFusedThreads = (kFirstProducerWarp + kProducerWarps) * 32;  // 704
+constexpr int kPlannerWarps = 2;      // after the producers: they prepare the producers' row blocks ahead of time
+constexpr int kFirstPlannerWarp = kFirstProducerWarp + kProducerWarps;
+constexpr int kFusedThreads = (kFirstPlannerWarp + kPlannerWarps) * 32;  // 768
 constexpr int kMaxStages = 8;
 constexpr int kGroupCols = 128;                  // input columns whose (self, mean) slices the producers fill together
-constexpr int kLanesPerRow = kGroupCols / 4;     // lanes covering one row segment with 16-byte loads
-constexpr int kRowsPerInstr = 32 / kLanesPerRow; // rows one warp-wide load instruction covers
 constexpr int kRowsInFlight = 2;                 // rows a producer warp builds at the same time
+constexpr int kBlockRows = kProducerWarps * kRowsInFlight;   // 32: rows of a tile the producers build in one round
+constexpr int kBlocksPerTile = BM / kBlockRows;              // 4
+constexpr int kPlanSlots = kBlocksPerTile;                   // planned row blocks in shared memory (one tile's worth)
 constexpr int kUnroll = 5;                       // neighbour rows per output row fetched before the first add
 constexpr uint32_t kABytes = BM * KC * 4;  // 16 KiB per A stage
 
@@ -73,14 +76,13 @@ struct FusedArgs {
     uint32_t* error;
 };
 
-constexpr int kKeyCap = 2048;   // source-row indices of a tile's entries cached in shared memory
+constexpr int kKeyCap = 512;    // source-row indices of a row block's entries cached in shared memory (16 per row)
 
-struct RowMeta {      // what a producer needs to build one output row
-    int32_t self_src; // source row of the row's own representation
-    int32_t e0, cnt;  // its entries in the sample's entry arrays; cnt < 0: row past the end
-    int32_t koff;     // first cached source-row index of the row, or -1 when the tile's entries do not fit
-    int32_t in_base;  // layers >= 2: first row of the mini-batch in H^{l-1}
-};
+// What a producer needs to build one output row: x = source row of the row's own representation; y = first
+// entry and z = number of entries in the sample's entry arrays (z < 0: row past the end); w = first cached
+// source-row index of the row when the block's entries fit the cache, else (layers >= 2) the first row of the
+// mini-batch in H^{l-1}.
+typedef int4 RowMeta;
 
 // Source row of an entry.  Layer 1: the feature-buffer row of node `key` (its partition's slot);
 // later layers: row of H^{l-1}.  The address is src_base + row * src_row_bytes.
@@ -113,10 +115,10 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
     __shared__ uint64_t a_full[kMaxStages], a_empty[kMaxStages], b_full[kMaxStages], b_empty[kMaxStages];
     __shared__ uint64_t acc_full[2], acc_empty[2];
     __shared__ uint32_t tmem_slot;
-    __shared__ RowMeta meta[BM];
-    __shared__ int32_t src_rows[kKeyCap];
-    __shared__ uint32_t key_warp_sum[BM / 32];
-    __shared__ int32_t key_end[BM];
+    __shared__ uint64_t plan_full[kPlanSlots], plan_empty[kPlanSlots];
+    __shared__ RowMeta meta[kPlanSlots][kBlockRows];
+    __shared__ int32_t src_rows[kPlanSlots][kKeyCap];
+    __shared__ int32_t plan_total[kPlanSlots];   // entries of the block, or -1 when they do not fit the cache
     __shared__ __align__(1024) float out_stage[4][32 * 32];   // per epilogue warp: one 32 x 32 slice, 128-byte swizzled, for the TMA store
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -130,6 +132,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
         for (int s = 0; s < a.sa; ++s) { mbar_init(&a_full[s], kProducerWarps); mbar_init(&a_empty[s], 1); }
         for (int s = 0; s < a.sb; ++s) { mbar_init(&b_full[s], 1); mbar_init(&b_empty[s], 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4); }
+        for (int s = 0; s < kPlanSlots; ++s) { mbar_init(&plan_full[s], 1); mbar_init(&plan_empty[s], kProducerWarps); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out) : "memory");
@@ -234,89 +237,52 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[buf]);
         }
-    } else {
+    } else if (warp < kFirstPlannerWarp) {
         // ---------------- producers: gather + segment mean -> swizzled A slices ----------------
+        // K slices come in groups of eight: (self, mean) pairs for four consecutive 32-column blocks, i.e. 128
+        // columns of the input rows.  A tile is built in rounds of 32 rows (a row block, planned ahead by the
+        // planner warps): a warp builds two rows per round from whole 512-byte row segments (lane L owns columns
+        // 4L..4L+3 of the group) and keeps 2 x (1 + kUnroll) loads in flight per lane -- memory-level parallelism
+        // comes from registers.  Each lane scatters its 16-byte pieces into the group's stages: slice pair L / 8,
+        // slot L % 8.  Producer warps only meet at the mbarriers, never at a block-wide barrier.
         const int pw = warp - kFirstProducerWarp;     // 0 .. kProducerWarps-1
-        const int ptid = threadIdx.x - kFirstProducerWarp * 32;
         const int gl = lane & 7;                      // 16-byte slot inside a 128-byte slice row
-        constexpr int kRowsPerWarp = BM / kProducerWarps;  // 8
-        uint32_t cnt = 0;
+        const int n_groups = (a.d_in_pad + kGroupCols - 1) / kGroupCols;
+        uint32_t cnt = 0, it = 0;
         bool ok = true;
-        for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
-            // row metadata of the tile and the source rows of all its entries, once per tile
-            asm volatile("bar.sync 1, %0;" ::"r"(kProducerWarps * 32) : "memory");   // previous tile's readers are done
-            RowMeta mm;
-            mm.self_src = a.safe_src; mm.e0 = 0; mm.cnt = -1; mm.koff = -1; mm.in_base = 0;
-            uint32_t incl = 0;
-            if (ptid < BM) {
-                const int64_t r = a.row_lo + t * BM + ptid;
-                if (r < a.M) {
-                    const int4 rm = __ldg(a.row_meta + r);   // (self_src, e0, cnt, in_base) from the pre-pass
-                    mm.self_src = rm.x; mm.e0 = rm.y; mm.cnt = rm.z; mm.in_base = rm.w;
-                }
-                incl = warp_incl_scan((uint32_t)max(mm.cnt, 0));
-                if (lane == 31) key_warp_sum[pw] = incl;
-            }
-            asm volatile("bar.sync 1, %0;" ::"r"(kProducerWarps * 32) : "memory");
-            uint32_t total = 0;
-#pragma unroll
-            for (int w = 0; w < BM / 32; ++w) total += key_warp_sum[w];
-            const bool cached = total <= (uint32_t)kKeyCap;
-            if (ptid < BM) {
-                uint32_t before = 0;
-#pragma unroll
-                for (int w = 0; w < BM / 32; ++w)
-                    if (w < pw) before += key_warp_sum[w];
-                if (cached && mm.cnt >= 0) mm.koff = (int32_t)(before + incl) - mm.cnt;
-                meta[ptid] = mm;
-                key_end[ptid] = (int32_t)(before + incl);   // end of row ptid's cached entries
-            }
-            asm volatile("bar.sync 1, %0;" ::"r"(kProducerWarps * 32) : "memory");
-            if (cached) {
-                // all producer threads copy the tile's entries: entry j belongs to the first row whose end exceeds j
-                const int32_t* keys = FIRST ? a.ent_nbrs : a.ent_repr;
-                for (uint32_t j = ptid; j < total; j += kProducerWarps * 32) {
-                    int lo = 0, hi = BM - 1;
-                    while (lo < hi) {
-                        const int mid = (lo + hi) >> 1;
-                        if (key_end[mid] > (int32_t)j) hi = mid; else lo = mid + 1;
-                    }
-                    const RowMeta rm = meta[lo];
-                    src_rows[j] = source_row<FIRST>(a, rm.in_base, __ldg(keys + rm.e0 + ((int32_t)j - rm.koff)));
-                }
-            }
-            asm volatile("bar.sync 1, %0;" ::"r"(kProducerWarps * 32) : "memory");
-            // K slices come in groups of eight: (self, mean) pairs for four consecutive 32-column blocks, i.e.
-            // 128 columns of the input rows.  A warp builds output rows from whole 512-byte row segments (lane
-            // L owns columns 4L..4L+3 of the group) and keeps kRowsInFlight rows x (1 + kUnroll) loads in
-            // flight per lane -- the producers are few and fat on purpose: memory-level parallelism comes from
-            // registers, not from warps.  Each lane scatters its 16-byte pieces into the group's stages: slice
-            // pair L / 8, slot L % 8.
-            const int n_groups = (a.d_in_pad + kGroupCols - 1) / kGroupCols;
+        for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++it) {
             for (int grp = 0; grp < n_groups; ++grp) {
                 const int pairs = min(kGroupCols / KC, (a.d_in_pad - grp * kGroupCols) / KC);   // slice pairs in this group
-                const int sub = lane / kLanesPerRow, ll = lane % kLanesPerRow;
-                const int col = grp * kGroupCols + ll * 4;
-                const bool lane_on = (ll >> 3) < pairs;
+                const int col = grp * kGroupCols + lane * 4;
+                const bool lane_on = (lane >> 3) < pairs;
                 const bool col_ok = lane_on && col < a.d_in;
                 const char* src = a.src_base + (size_t)col * (HALF ? 2 : 4);
                 bool waited = false;
-                for (int rr = 0; rr < kRowsPerWarp; rr += kRowsInFlight * kRowsPerInstr) {
-                    const int row0 = pw * kRowsPerWarp + rr + sub;   // this lane's rows: row0 + q * kRowsPerInstr
+                for (int blk = 0; blk < kBlocksPerTile; ++blk) {
+                    const uint32_t q = it * kBlocksPerTile + blk;     // row block counter of this CTA
+                    const int slot = q % kPlanSlots;
+                    if (grp == 0 && ok && !mbar_wait(&plan_full[slot], (q / kPlanSlots) & 1)) {
+                        if (lane == 0) atomicExch(a.error, 16u);
+                        ok = false;
+                    }
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    const bool cached = plan_total[slot] >= 0;
+                    const int32_t* rows_of = src_rows[slot];
+                    const int brow = pw * kRowsInFlight;              // this warp's first row inside the block
                     RowMeta mq[kRowsInFlight];
                     float4 selfv[kRowsInFlight], acc[kRowsInFlight];
                     int top = 0;
 #pragma unroll
-                    for (int q = 0; q < kRowsInFlight; ++q) {
-                        mq[q] = meta[row0 + q * kRowsPerInstr];
-                        selfv[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        acc[q] = selfv[q];
-                        top = max(top, mq[q].cnt);
+                    for (int q2 = 0; q2 < kRowsInFlight; ++q2) {
+                        mq[q2] = meta[slot][brow + q2];
+                        selfv[q2] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        acc[q2] = selfv[q2];
+                        top = max(top, mq[q2].z);
                     }
-                    if (col_ok) {
+                    if (col_ok && ok) {
 #pragma unroll
-                        for (int q = 0; q < kRowsInFlight; ++q)
-                            selfv[q] = load4<HALF>(src + (size_t)(uint32_t)mq[q].self_src * a.src_row_bytes);
+                        for (int q2 = 0; q2 < kRowsInFlight; ++q2)
+                            selfv[q2] = load4<HALF>(src + (size_t)(uint32_t)mq[q2].x * a.src_row_bytes);
                         if (cached) {
                             // Every load is issued unconditionally: a slot past the end of a row's entries re-reads
                             // the row's own representation (a cache hit) and is added as an exact zero.  Branch-free
@@ -326,39 +292,44 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
 #pragma unroll
                                 for (int j = 0; j < kUnroll; ++j)
 #pragma unroll
-                                    for (int q = 0; q < kRowsInFlight; ++q) {
-                                        const bool live = e + j < mq[q].cnt;
-                                        const int32_t sr = src_rows[live ? mq[q].koff + e + j : 0];
-                                        v[q][j] = load4<HALF>(src + (size_t)(uint32_t)(live ? sr : mq[q].self_src) * a.src_row_bytes);
+                                    for (int q2 = 0; q2 < kRowsInFlight; ++q2) {
+                                        const bool live = e + j < mq[q2].z;
+                                        const int32_t sr = rows_of[live ? mq[q2].w + e + j : 0];
+                                        v[q2][j] = load4<HALF>(src + (size_t)(uint32_t)(live ? sr : mq[q2].x) * a.src_row_bytes);
                                     }
 #pragma unroll
                                 for (int j = 0; j < kUnroll; ++j)   // entry order
 #pragma unroll
-                                    for (int q = 0; q < kRowsInFlight; ++q) {
-                                        const bool live = e + j < mq[q].cnt;   // selects, not branches
-                                        acc[q].x += live ? v[q][j].x : 0.f; acc[q].y += live ? v[q][j].y : 0.f;
-                                        acc[q].z += live ? v[q][j].z : 0.f; acc[q].w += live ? v[q][j].w : 0.f;
+                                    for (int q2 = 0; q2 < kRowsInFlight; ++q2) {
+                                        const bool live = e + j < mq[q2].z;   // selects, not branches
+                                        acc[q2].x += live ? v[q2][j].x : 0.f; acc[q2].y += live ? v[q2][j].y : 0.f;
+                                        acc[q2].z += live ? v[q2][j].z : 0.f; acc[q2].w += live ? v[q2][j].w : 0.f;
                                     }
                             }
                         } else {
-                            // a tile with more entries than the shared-memory cache holds: plain per-entry loop
+                            // a row block with more entries than the shared-memory cache holds: plain per-entry loop
                             const int32_t* keys = FIRST ? a.ent_nbrs : a.ent_repr;
 #pragma unroll
-                            for (int q = 0; q < kRowsInFlight; ++q)
-                                for (int e = 0; e < mq[q].cnt; ++e) {
-                                    const int32_t sr = source_row<FIRST>(a, mq[q].in_base, __ldg(keys + mq[q].e0 + e));
+                            for (int q2 = 0; q2 < kRowsInFlight; ++q2)
+                                for (int e = 0; e < mq[q2].z; ++e) {
+                                    const int32_t sr = source_row<FIRST>(a, mq[q2].w, __ldg(keys + mq[q2].y + e));
                                     const float4 v = load4<HALF>(src + (size_t)(uint32_t)sr * a.src_row_bytes);
-                                    acc[q].x += v.x; acc[q].y += v.y; acc[q].z += v.z; acc[q].w += v.w;
+                                    acc[q2].x += v.x; acc[q2].y += v.y; acc[q2].z += v.z; acc[q2].w += v.w;
                                 }
                         }
 #pragma unroll
-                        for (int q = 0; q < kRowsInFlight; ++q) {
-                            const float inv = mq[q].cnt > 0 ? 1.f / (float)mq[q].cnt : 0.f;
-                            acc[q].x = to_tf32(acc[q].x * inv); acc[q].y = to_tf32(acc[q].y * inv);
-                            acc[q].z = to_tf32(acc[q].z * inv); acc[q].w = to_tf32(acc[q].w * inv);
-                            selfv[q].x = to_tf32(selfv[q].x); selfv[q].y = to_tf32(selfv[q].y);
-                            selfv[q].z = to_tf32(selfv[q].z); selfv[q].w = to_tf32(selfv[q].w);
+                        for (int q2 = 0; q2 < kRowsInFlight; ++q2) {
+                            const float inv = mq[q2].z > 0 ? 1.f / (float)mq[q2].z : 0.f;
+                            acc[q2].x = to_tf32(acc[q2].x * inv); acc[q2].y = to_tf32(acc[q2].y * inv);
+                            acc[q2].z = to_tf32(acc[q2].z * inv); acc[q2].w = to_tf32(acc[q2].w * inv);
+                            selfv[q2].x = to_tf32(selfv[q2].x); selfv[q2].y = to_tf32(selfv[q2].y);
+                            selfv[q2].z = to_tf32(selfv[q2].z); selfv[q2].w = to_tf32(selfv[q2].w);
                         }
+                    }
+                    if (grp == n_groups - 1) {
+                        // the block's plan has been read for the last time: its slot may be planned again
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&plan_empty[slot]);
                     }
                     if (!waited) {
                         // the group's stages must have been read by the MMAs of their previous use; the loads
@@ -375,15 +346,15 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     }
                     if (ok && lane_on) {
                         // K-major, 128-byte swizzle: 16-byte slot gl of row r lands in slot gl ^ (r % 8)
-                        const uint32_t s_self = (cnt + 2 * (ll >> 3)) % a.sa, s_mean = (cnt + 2 * (ll >> 3) + 1) % a.sa;
+                        const uint32_t s_self = (cnt + 2 * (lane >> 3)) % a.sa, s_mean = (cnt + 2 * (lane >> 3) + 1) % a.sa;
                         uint8_t* stage_self = a_base + (size_t)s_self * kABytes;
                         uint8_t* stage_mean = a_base + (size_t)s_mean * kABytes;
 #pragma unroll
-                        for (int q = 0; q < kRowsInFlight; ++q) {
-                            const int row = row0 + q * kRowsPerInstr;
+                        for (int q2 = 0; q2 < kRowsInFlight; ++q2) {
+                            const int row = blk * kBlockRows + brow + q2;
                             const size_t off = (size_t)(row >> 3) * 1024 + (size_t)(row & 7) * 128 + (size_t)((gl ^ (row & 7)) << 4);
-                            *reinterpret_cast<float4*>(stage_self + off) = selfv[q];
-                            *reinterpret_cast<float4*>(stage_mean + off) = acc[q];
+                            *reinterpret_cast<float4*>(stage_self + off) = selfv[q2];
+                            *reinterpret_cast<float4*>(stage_mean + off) = acc[q2];
                         }
                     }
                 }
@@ -393,6 +364,61 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     for (int j = 0; j < 2 * pairs; ++j) mbar_arrive(&a_full[(cnt + j) % a.sa]);
                 cnt += 2 * pairs;
             }
+        }
+    } else {
+        // ---------------- planners: row blocks of 32 rows, prepared ahead of the producers ----------------
+        // A planner warp takes every kPlannerWarps-th row block: lane = row.  It reads the rows' metadata, scans the
+        // entry counts, and translates the block's entries to source rows in shared memory, so that the producers'
+        // gathers depend on nothing but shared memory.
+        const int plw = warp - kFirstPlannerWarp;
+        const int32_t* keys = FIRST ? a.ent_nbrs : a.ent_repr;
+        bool ok = true;
+        for (uint32_t q = plw; ok; q += kPlannerWarps) {
+            const int64_t t = blockIdx.x + (int64_t)(q / kBlocksPerTile) * gridDim.x;
+            if (t >= n_tiles) break;
+            const int slot = q % kPlanSlots;
+            if (q >= (uint32_t)kPlanSlots && !mbar_wait(&plan_empty[slot], ((q / kPlanSlots) - 1) & 1)) {
+                if (lane == 0) atomicExch(a.error, 17u);
+                ok = false;
+            }
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            const int64_t r = a.row_lo + t * BM + (q % kBlocksPerTile) * kBlockRows + lane;
+            int4 rm = make_int4(a.safe_src, 0, -1, 0);
+            if (r < a.M) rm = __ldg(a.row_meta + r);   // (self source row, first entry, count, first H^{l-1} row of the batch)
+            const int32_t end = (int32_t)warp_incl_scan((uint32_t)max(rm.z, 0));   // end of the row's cached entries
+            const int32_t total = __shfl_sync(0xFFFFFFFFu, end, 31);
+            const bool cached = total <= kKeyCap;
+            const int32_t in_base = rm.w, koff = end - max(rm.z, 0);
+            meta[slot][lane] = make_int4(rm.x, rm.y, rm.z, cached ? koff : in_base);
+            if (cached) {
+                // entry j belongs to the first row whose end exceeds j
+                for (int32_t j0 = 0; j0 < total; j0 += 32 * 4) {
+                    int32_t key[4], base[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int32_t j = j0 + u * 32 + lane;
+                        int lo = 0, hi = 31;
+#pragma unroll
+                        for (int s = 0; s < 5; ++s) {
+                            const int mid = (lo + hi) >> 1;
+                            const int32_t e = __shfl_sync(0xFFFFFFFFu, end, mid);
+                            if (lo < hi) { if (e > j) hi = mid; else lo = mid + 1; }
+                        }
+                        const int32_t e0 = __shfl_sync(0xFFFFFFFFu, rm.y, lo), k0 = __shfl_sync(0xFFFFFFFFu, koff, lo);
+                        base[u] = __shfl_sync(0xFFFFFFFFu, in_base, lo);
+                        key[u] = j < total ? __ldg(keys + e0 + (j - k0)) : 0;
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int32_t j = j0 + u * 32 + lane;
+                        if (j < total) src_rows[slot][j] = source_row<FIRST>(a, base[u], key[u]);
+                    }
+                }
+            }
+            if (lane == 0) plan_total[slot] = cached ? total : -1;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&plan_full[slot]);
         }
     }
     if (warp >= 2 && warp < kFirstProducerWarp && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
