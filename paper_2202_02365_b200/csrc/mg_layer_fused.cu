@@ -109,10 +109,13 @@ __device__ __forceinline__ float4 load4(const char* p) {
 }
 
 template <bool FIRST, bool HALF>
-__global__ void __launch_bounds__(kFusedThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFusedThreads, 1)
 k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_out, FusedArgs a) {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t a_full[kMaxStages], a_empty[kMaxStages], b_full[kMaxStages], b_empty[kMaxStages];
+    // a_ready and acc_empty are used in the leader CTA only (both CTAs arrive there); a_free, b_empty and acc_full
+    // exist in both CTAs and are signalled in both by the leader's commits; b_full counts both halves' bytes in
+    // the leader.
+    __shared__ uint64_t a_ready[2], a_free[2], b_full[kMaxStages], b_empty[kMaxStages];
     __shared__ uint64_t acc_full[2], acc_empty[2];
     __shared__ uint32_t tmem_slot;
     __shared__ uint64_t plan_full[kPlanSlots], plan_empty[kPlanSlots];
@@ -122,81 +125,91 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
     __shared__ __align__(1024) float out_stage[4][32 * 32];   // per epilogue warp: one 32 x 32 slice, 128-byte swizzled, for the TMA store
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t b_bytes = (uint32_t)a.BN * KC * 4;
+    const uint32_t rank = cluster_ctarank();      // 0: leader of the pair (issues the MMAs), 1: its peer
+    const bool leader = rank == 0;
+    const uint32_t pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    const int half_n = a.BN / 2;                  // weight rows (output columns) this CTA stages
+    const uint32_t b_bytes = (uint32_t)half_n * KC * 4;
     uint8_t* a_base = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* b_base = a_base + (size_t)a.sa * kABytes;
     const int n_chunks = 2 * a.d_in_pad / KC;
     const int64_t n_tiles = (a.M - a.row_lo + BM - 1) / BM;
+    const int64_t n_tile_pairs = (n_tiles + 1) / 2;
+    // iteration `it` of this pair works on tile pair (pair + it * n_pairs): the leader on its even tile, the peer
+    // on the odd one (which may lie past the end: then all its rows are padding)
+    const uint32_t my_iters = pair < n_tile_pairs ? (uint32_t)((n_tile_pairs - pair + n_pairs - 1) / n_pairs) : 0u;
+    auto tile_of = [&](uint32_t it) -> int64_t { return 2 * ((int64_t)pair + (int64_t)it * n_pairs) + rank; };
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < a.sa; ++s) { mbar_init(&a_full[s], kProducerWarps); mbar_init(&a_empty[s], 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&a_ready[s], 2 * kProducerWarps); mbar_init(&a_free[s], 1); }
         for (int s = 0; s < a.sb; ++s) { mbar_init(&b_full[s], 1); mbar_init(&b_empty[s], 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 2 * 4); }
         for (int s = 0; s < kPlanSlots; ++s) { mbar_init(&plan_full[s], 1); mbar_init(&plan_empty[s], kProducerWarps); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out) : "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"((uint32_t)a.tmem_cols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        // the same warp of both CTAs allocates the pair's tensor memory
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"((uint32_t)a.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
-    __syncthreads();
+    cluster_sync_all();       // barriers of both CTAs are initialised before anyone arrives on a remote one
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
     const uint32_t acc_stride = (uint32_t)(a.tmem_cols / 2);  // columns per accumulator buffer (a multiple of 32)
 
     if (warp == 0) {
-        // ---------------- weight slices: TMA from L2 ----------------
+        // ---------------- weight slices: each CTA stages its half of the output columns (TMA from L2) ----------------
         if (lane == 0) {
             uint32_t cnt = 0;
             bool ok = true;
-            for (int64_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+            for (uint32_t it = 0; it < my_iters && ok; ++it) {
                 for (int c = 0; c < n_chunks; ++c, ++cnt) {
                     const int s = cnt % a.sb;
                     if (cnt >= (uint32_t)a.sb && !mbar_wait(&b_empty[s], ((cnt / a.sb) - 1) & 1)) { atomicExch(a.error, 11u); ok = false; break; }
-                    mbar_expect_tx(&b_full[s], b_bytes);
-                    tma_load_2d(b_base + (size_t)s * b_bytes, &map_w, &b_full[s], c * KC, 0);
+                    if (leader) mbar_expect_tx(&b_full[s], 2 * b_bytes);   // both halves are counted on the leader's barrier
+                    tma_load_2d_pair(b_base + (size_t)s * b_bytes, &map_w, mapa_u32(smem_u32(&b_full[s]), 0), c * KC, (int)rank * half_n);
                 }
             }
         }
         __syncwarp();
     } else if (warp == 1) {
-        // ---------------- MMA issue ----------------
-        if (lane == 0) {
-            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(a.BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-            uint32_t cnt = 0, it = 0;
+        // ---------------- MMA issue: one thread of the leader, for both CTAs ----------------
+        if (lane == 0 && leader) {
+            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(a.BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+            uint32_t cnt = 0, unit = 0;
             bool ok = true;
-            for (int64_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++it) {
+            for (uint32_t it = 0; it < my_iters && ok; ++it) {
                 const uint32_t buf = it & 1;
                 if (it >= 2 && !mbar_wait(&acc_empty[buf], ((it >> 1) - 1) & 1)) { atomicExch(a.error, 12u); ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * acc_stride;
                 for (int c = 0; c < n_chunks; ++c, ++cnt) {
+                    // a group of (up to) eight K slices is one unit: both CTAs' producers have filled it
+                    if ((c & 7) == 0 && !mbar_wait(&a_ready[unit & 1], (unit >> 1) & 1)) { atomicExch(a.error, 13u); ok = false; break; }
                     const int sa = cnt % a.sa, sb = cnt % a.sb;
-                    if (!mbar_wait(&a_full[sa], (cnt / a.sa) & 1) || !mbar_wait(&b_full[sb], (cnt / a.sb) & 1)) {
-                        atomicExch(a.error, 13u); ok = false; break;
-                    }
+                    if (!mbar_wait(&b_full[sb], (cnt / a.sb) & 1)) { atomicExch(a.error, 13u); ok = false; break; }
                     tc_fence_after();
                     const uint64_t da = smem_desc_sw128(smem_u32(a_base + (size_t)sa * kABytes));
                     const uint64_t db = smem_desc_sw128(smem_u32(b_base + (size_t)sb * b_bytes));
 #pragma unroll
                     for (int kk = 0; kk < KC / 8; ++kk)
-                        mma_tf32(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (c | kk) ? 1u : 0u);
-                    mma_commit(&a_empty[sa]);
-                    mma_commit(&b_empty[sb]);
+                        mma_tf32_pair(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (c | kk) ? 1u : 0u);
+                    mma_commit_pair(&b_empty[sb]);
+                    if ((c & 7) == 7 || c == n_chunks - 1) { mma_commit_pair(&a_free[unit & 1]); ++unit; }
                 }
-                mma_commit(&acc_full[buf]);
+                if (ok) mma_commit_pair(&acc_full[buf]);
             }
         }
         __syncwarp();
     } else if (warp < kFirstProducerWarp) {
         // ---------------- epilogue: tensor memory -> bias, ReLU -> global ----------------
         const int lane_group = warp & 3;
-        uint32_t it = 0;
         bool ok = true;
-        for (int64_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++it) {
+        for (uint32_t it = 0; it < my_iters && ok; ++it) {
+            const int64_t t = tile_of(it);
             const uint32_t buf = it & 1;
             if (!mbar_wait(&acc_full[buf], (it >> 1) & 1)) { if (lane == 0) atomicExch(a.error, 14u); ok = false; break; }
             tc_fence_after();
@@ -235,7 +248,10 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&acc_empty[buf]);
+            if (lane == 0) {   // this accumulator buffer of this CTA is drained: tell the leader's MMA thread
+                if (leader) mbar_arrive(&acc_empty[buf]);
+                else mbar_arrive_cluster(mapa_u32(smem_u32(&acc_empty[buf]), 0));
+            }
         }
     } else if (warp < kFirstPlannerWarp) {
         // ---------------- producers: gather + segment mean -> swizzled A slices ----------------
@@ -248,10 +264,11 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
         const int pw = warp - kFirstProducerWarp;     // 0 .. kProducerWarps-1
         const int gl = lane & 7;                      // 16-byte slot inside a 128-byte slice row
         const int n_groups = (a.d_in_pad + kGroupCols - 1) / kGroupCols;
-        uint32_t cnt = 0, it = 0;
         bool ok = true;
-        for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++it) {
+        for (uint32_t it = 0; it < my_iters; ++it) {
             for (int grp = 0; grp < n_groups; ++grp) {
+                const uint32_t u = it * (uint32_t)n_groups + (uint32_t)grp;   // (tile, group) unit of this pair
+                const uint32_t cnt = it * (uint32_t)n_chunks + (uint32_t)grp * (2 * kGroupCols / KC);   // its first K slice
                 const int pairs = min(kGroupCols / KC, (a.d_in_pad - grp * kGroupCols) / KC);   // slice pairs in this group
                 const int col = grp * kGroupCols + lane * 4;
                 const bool lane_on = (lane >> 3) < pairs;
@@ -332,14 +349,11 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                         if (lane == 0) mbar_arrive(&plan_empty[slot]);
                     }
                     if (!waited) {
-                        // the group's stages must have been read by the MMAs of their previous use; the loads
-                        // above are already in flight while this waits
-                        for (int j = 0; j < 2 * pairs; ++j) {
-                            const uint32_t cj = cnt + j;
-                            if (ok && cj >= (uint32_t)a.sa && !mbar_wait(&a_empty[cj % a.sa], ((cj / a.sa) - 1) & 1)) {
-                                if (lane == 0) atomicExch(a.error, 15u);
-                                ok = false;
-                            }
+                        // the stages must have been read by the MMAs of the previous unit (one commit frees them all);
+                        // the loads above are already in flight while this waits
+                        if (ok && u >= 1 && !mbar_wait(&a_free[(u - 1) & 1], ((u - 1) >> 1) & 1)) {
+                            if (lane == 0) atomicExch(a.error, 15u);
+                            ok = false;
                         }
                         ok = __all_sync(0xFFFFFFFFu, ok);
                         waited = true;
@@ -360,9 +374,10 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 }
                 fence_async_smem();
                 __syncwarp();
-                if (ok && lane == 0)
-                    for (int j = 0; j < 2 * pairs; ++j) mbar_arrive(&a_full[(cnt + j) % a.sa]);
-                cnt += 2 * pairs;
+                if (ok && lane == 0) {   // this warp's rows of the unit are in place: tell the leader's MMA thread
+                    if (leader) mbar_arrive(&a_ready[u & 1]);
+                    else mbar_arrive_cluster(mapa_u32(smem_u32(&a_ready[u & 1]), 0));
+                }
             }
         }
     } else {
@@ -374,8 +389,8 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
         const int32_t* keys = FIRST ? a.ent_nbrs : a.ent_repr;
         bool ok = true;
         for (uint32_t q = plw; ok; q += kPlannerWarps) {
-            const int64_t t = blockIdx.x + (int64_t)(q / kBlocksPerTile) * gridDim.x;
-            if (t >= n_tiles) break;
+            if (q / kBlocksPerTile >= my_iters) break;
+            const int64_t t = tile_of(q / kBlocksPerTile);   // past the end for the peer of an odd last tile: all padding
             const int slot = q % kPlanSlots;
             if (q >= (uint32_t)kPlanSlots && !mbar_wait(&plan_empty[slot], ((q / kPlanSlots) - 1) & 1)) {
                 if (lane == 0) atomicExch(a.error, 17u);
@@ -423,10 +438,10 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
     }
     if (warp >= 2 && warp < kFirstProducerWarp && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     tc_fence_before();
-    __syncthreads();
+    cluster_sync_all();   // neither CTA leaves (or frees tensor memory) while the other may still signal or read it
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)a.tmem_cols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)a.tmem_cols) : "memory");
     }
 }
 
@@ -532,13 +547,13 @@ int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_ou
     int stride = 32;
     while (stride < a.BN) stride <<= 1;
     a.tmem_cols = 2 * stride;   // two accumulator buffers, each a power of two >= 32 columns
-    const int b_bytes = a.BN * KC * 4;
+    const int b_bytes = (a.BN / 2) * KC * 4;    // each CTA of a pair stages half of the output columns
     const int n_chunks = 2 * a.d_in_pad / KC;
     a.sa = std::min(8, n_chunks);   // one group of (self, mean) slice pairs: 128 input columns
     a.sb = std::max(2, std::min({kMaxStages, n_chunks, (int)((194 * 1024 - a.sa * (int)kABytes) / b_bytes)}));
     const size_t smem = (size_t)a.sa * kABytes + (size_t)a.sb * b_bytes + 1024;
     CUtensorMap mw;
-    if (!make_map_f32(&mw, w_pad_t, d_out, 2 * a.d_in_pad, a.BN))
+    if (!make_map_f32(&mw, w_pad_t, d_out, 2 * a.d_in_pad, a.BN / 2))
         return mg_fail(ctx, MG_ERR_CUDA, "cuTensorMapEncodeTiled failed for the layer weights");
     // output [row_hi rows, d_out] fp32, 32 x 32 boxes, 128-byte swizzle; rows are global packed rows, so a window's
     // shifted base pointer works unchanged (rows below row_lo are never stored)
@@ -549,7 +564,7 @@ int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_ou
     auto kern = first ? (half ? k_sage_layer_fused<true, true> : k_sage_layer_fused<true, false>) : k_sage_layer_fused<false, false>;
     MG_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const int64_t n_tiles = (row_hi - row_lo + BM - 1) / BM;
-    const int grid = (int)std::min<int64_t>(n_tiles, ctx->n_sms);
+    const int grid = 2 * (int)std::min<int64_t>((n_tiles + 1) / 2, ctx->n_sms / 2);   // CTA pairs
     kern<<<grid, kFusedThreads, smem, ctx->stream>>>(mw, mo, a);
     ctx->launches++;
     MG_CUDA(ctx, cudaGetLastError());
