@@ -38,6 +38,10 @@ constexpr int kRowsInFlight = 2;                 // rows a producer warp builds 
 constexpr int kBlockRows = kProducerWarps * kRowsInFlight;   // 32: rows of a tile the producers build in one round
 constexpr int kBlocksPerTile = BM / kBlockRows;              // 4
 constexpr int kPlanSlots = kBlocksPerTile;                   // planned row blocks in shared memory (one tile's worth)
+constexpr int HM = BM / 2;                                   // rows of a half tile: the unit the MMAs work on
+constexpr int kBlocksPerHalf = kBlocksPerTile / 2;
+constexpr int kAccBufs = 4;                                  // accumulator buffers in tensor memory (two tiles' halves)
+constexpr int kSlicesPerGroup = 2 * kGroupCols / KC;         // 8 K slices: (self, mean) x four 32-column blocks
 constexpr int kUnroll = 5;                       // neighbour rows per output row fetched before the first add
 constexpr uint32_t kABytes = BM * KC * 4;  // 16 KiB per A stage
 
@@ -115,8 +119,8 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
     // a_ready and acc_empty are used in the leader CTA only (both CTAs arrive there); a_free, b_empty and acc_full
     // exist in both CTAs and are signalled in both by the leader's commits; b_full counts both halves' bytes in
     // the leader.
-    __shared__ uint64_t a_ready[2], a_free[2], b_full[kMaxStages], b_empty[kMaxStages];
-    __shared__ uint64_t acc_full[2], acc_empty[2];
+    __shared__ uint64_t a_ready[2], a_free[2], b_full[kMaxStages], b_empty[kMaxStages];   // a_*: one per half tile
+    __shared__ uint64_t acc_full[kAccBufs], acc_empty[kAccBufs];
     __shared__ uint32_t tmem_slot;
     __shared__ uint64_t plan_full[kPlanSlots], plan_empty[kPlanSlots];
     __shared__ RowMeta meta[kPlanSlots][kBlockRows];
@@ -143,7 +147,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
     if (threadIdx.x == 0) {
         for (int s = 0; s < 2; ++s) { mbar_init(&a_ready[s], 2 * kProducerWarps); mbar_init(&a_free[s], 1); }
         for (int s = 0; s < a.sb; ++s) { mbar_init(&b_full[s], 1); mbar_init(&b_empty[s], 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 2 * 4); }
+        for (int s = 0; s < kAccBufs; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 2 * 4); }
         for (int s = 0; s < kPlanSlots; ++s) { mbar_init(&plan_full[s], 1); mbar_init(&plan_empty[s], kProducerWarps); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
@@ -158,75 +162,95 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
     cluster_sync_all();       // barriers of both CTAs are initialised before anyone arrives on a remote one
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
-    const uint32_t acc_stride = (uint32_t)(a.tmem_cols / 2);  // columns per accumulator buffer (a multiple of 32)
+    const uint32_t acc_stride = (uint32_t)(a.tmem_cols / kAccBufs);  // columns per accumulator buffer (a multiple of 32)
+    const int n_groups = (a.d_in_pad + kGroupCols - 1) / kGroupCols;
 
     if (warp == 0) {
         // ---------------- weight slices: each CTA stages its half of the output columns (TMA from L2) ----------------
         if (lane == 0) {
             uint32_t cnt = 0;
             bool ok = true;
-            for (uint32_t it = 0; it < my_iters && ok; ++it) {
-                for (int c = 0; c < n_chunks; ++c, ++cnt) {
-                    const int s = cnt % a.sb;
-                    if (cnt >= (uint32_t)a.sb && !mbar_wait(&b_empty[s], ((cnt / a.sb) - 1) & 1)) { atomicExch(a.error, 11u); ok = false; break; }
-                    if (leader) mbar_expect_tx(&b_full[s], 2 * b_bytes);   // both halves are counted on the leader's barrier
-                    tma_load_2d_pair(b_base + (size_t)s * b_bytes, &map_w, mapa_u32(smem_u32(&b_full[s]), 0), c * KC, (int)rank * half_n);
-                }
-            }
+            // the weight slices of a group are streamed once per half tile, in the order the MMAs consume them
+            for (uint32_t it = 0; it < my_iters && ok; ++it)
+                for (int grp = 0; grp < n_groups && ok; ++grp)
+                    for (int h = 0; h < 2 && ok; ++h) {
+                        const int gch = min(kSlicesPerGroup, n_chunks - grp * kSlicesPerGroup);
+                        for (int c = 0; c < gch; ++c, ++cnt) {
+                            const int s = cnt % a.sb;
+                            if (cnt >= (uint32_t)a.sb && !mbar_wait(&b_empty[s], ((cnt / a.sb) - 1) & 1)) { atomicExch(a.error, 11u); ok = false; break; }
+                            if (leader) mbar_expect_tx(&b_full[s], 2 * b_bytes);   // both halves are counted on the leader's barrier
+                            tma_load_2d_pair(b_base + (size_t)s * b_bytes, &map_w, mapa_u32(smem_u32(&b_full[s]), 0),
+                                             (grp * kSlicesPerGroup + c) * KC, (int)rank * half_n);
+                        }
+                    }
         }
         __syncwarp();
     } else if (warp == 1) {
         // ---------------- MMA issue: one thread of the leader, for both CTAs ----------------
         if (lane == 0 && leader) {
-            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(a.BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
-            uint32_t cnt = 0, unit = 0;
+            // M = 128 over the pair: 64 rows (a half tile) of each CTA per instruction
+            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(a.BN >> 3) << 17) | ((uint32_t)((2 * HM) >> 4) << 24);
+            uint32_t cnt = 0;
             bool ok = true;
-            for (uint32_t it = 0; it < my_iters && ok; ++it) {
-                const uint32_t buf = it & 1;
-                if (it >= 2 && !mbar_wait(&acc_empty[buf], ((it >> 1) - 1) & 1)) { atomicExch(a.error, 12u); ok = false; break; }
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * acc_stride;
-                for (int c = 0; c < n_chunks; ++c, ++cnt) {
-                    // a group of (up to) eight K slices is one unit: both CTAs' producers have filled it
-                    if ((c & 7) == 0 && !mbar_wait(&a_ready[unit & 1], (unit >> 1) & 1)) { atomicExch(a.error, 13u); ok = false; break; }
-                    const int sa = cnt % a.sa, sb = cnt % a.sb;
-                    if (!mbar_wait(&b_full[sb], (cnt / a.sb) & 1)) { atomicExch(a.error, 13u); ok = false; break; }
-                    tc_fence_after();
-                    const uint64_t da = smem_desc_sw128(smem_u32(a_base + (size_t)sa * kABytes));
-                    const uint64_t db = smem_desc_sw128(smem_u32(b_base + (size_t)sb * b_bytes));
+            for (uint32_t it = 0; it < my_iters && ok; ++it)
+                for (int grp = 0; grp < n_groups && ok; ++grp)
+                    for (int h = 0; h < 2 && ok; ++h) {
+                        const uint32_t hu = it * 2 + h;                       // half tiles of this CTA, in order
+                        const uint32_t buf = hu % kAccBufs;
+                        const uint32_t s_h = it * (uint32_t)n_groups + grp;   // fills of half h's stage rows so far
+                        if (grp == 0) {
+                            if (hu >= (uint32_t)kAccBufs && !mbar_wait(&acc_empty[buf], ((hu / kAccBufs) - 1) & 1)) { atomicExch(a.error, 12u); ok = false; break; }
+                            tc_fence_after();
+                        }
+                        // both CTAs' producers have filled the half's rows of this group's K slices
+                        if (!mbar_wait(&a_ready[h], s_h & 1)) { atomicExch(a.error, 13u); ok = false; break; }
+                        const uint32_t d_tmem = tmem_base + buf * acc_stride;
+                        const int gch = min(kSlicesPerGroup, n_chunks - grp * kSlicesPerGroup);
+                        for (int c = 0; c < gch; ++c, ++cnt) {
+                            const int sb = cnt % a.sb;
+                            if (!mbar_wait(&b_full[sb], (cnt / a.sb) & 1)) { atomicExch(a.error, 13u); ok = false; break; }
+                            tc_fence_after();
+                            const uint64_t da = smem_desc_sw128(smem_u32(a_base + (size_t)c * kABytes + (size_t)h * (HM * KC * 4)));
+                            const uint64_t db = smem_desc_sw128(smem_u32(b_base + (size_t)sb * b_bytes));
 #pragma unroll
-                    for (int kk = 0; kk < KC / 8; ++kk)
-                        mma_tf32_pair(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (c | kk) ? 1u : 0u);
-                    mma_commit_pair(&b_empty[sb]);
-                    if ((c & 7) == 7 || c == n_chunks - 1) { mma_commit_pair(&a_free[unit & 1]); ++unit; }
-                }
-                if (ok) mma_commit_pair(&acc_full[buf]);
-            }
+                            for (int kk = 0; kk < KC / 8; ++kk)
+                                mma_tf32_pair(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (grp | c | kk) ? 1u : 0u);
+                            mma_commit_pair(&b_empty[sb]);
+                        }
+                        if (!ok) break;
+                        mma_commit_pair(&a_free[h]);    // one commit frees the half's rows of all the group's stages
+                        if (grp == n_groups - 1) mma_commit_pair(&acc_full[buf]);
+                    }
         }
         __syncwarp();
     } else if (warp < kFirstProducerWarp) {
         // ---------------- epilogue: tensor memory -> bias, ReLU -> global ----------------
+        // A half tile's accumulator: rows 0..63 of output columns [0, BN/2) in lanes 0..63, the same rows of columns
+        // [BN/2, BN) in lanes 64..127.  Warp quadrant q reads lanes 32q..32q+31.
         const int lane_group = warp & 3;
+        const int col_base = (lane_group >> 1) * half_n;
         bool ok = true;
-        for (uint32_t it = 0; it < my_iters && ok; ++it) {
-            const int64_t t = tile_of(it);
-            const uint32_t buf = it & 1;
-            if (!mbar_wait(&acc_full[buf], (it >> 1) & 1)) { if (lane == 0) atomicExch(a.error, 14u); ok = false; break; }
+        for (uint32_t hu = 0; hu < 2 * my_iters && ok; ++hu) {
+            const int64_t t = tile_of(hu >> 1);
+            const uint32_t buf = hu % kAccBufs;
+            if (!mbar_wait(&acc_full[buf], (hu / kAccBufs) & 1)) { if (lane == 0) atomicExch(a.error, 14u); ok = false; break; }
             tc_fence_after();
-            const int64_t row0 = a.row_lo + t * BM + lane_group * 32;
+            const int64_t row0 = a.row_lo + t * BM + (hu & 1) * HM + (lane_group & 1) * 32;
             uint8_t* stage = reinterpret_cast<uint8_t*>(out_stage[lane_group]);
-            for (int c0 = 0; c0 < a.BN; c0 += 32) {
+            for (int c0 = 0; c0 < half_n; c0 += 32) {
                 uint32_t v[32];
                 tmem_ld_32(tmem_base + buf * acc_stride + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)c0, v);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (row0 < a.M && c0 < a.N) {
+                const int ncol0 = col_base + c0;   // first output column of this slice
+                if (row0 >= a.M || ncol0 >= a.N) continue;
+                if (c0 + 32 <= half_n) {
                     // the previous slice's TMA store must have read the staging tile before it is rewritten
                     if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                     __syncwarp();
                     // lane = row of the slice; 16-byte piece c of the row goes to piece c ^ (row % 8) (128-byte swizzle)
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
-                        const int n = c0 + 4 * c;
+                        const int n = ncol0 + 4 * c;
                         float4 o = make_float4(__uint_as_float(v[4 * c]), __uint_as_float(v[4 * c + 1]),
                                                __uint_as_float(v[4 * c + 2]), __uint_as_float(v[4 * c + 3]));
                         if (n < a.N) {
@@ -241,8 +265,25 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     if (lane == 0) {
                         // rows past the end of the layer and columns past its width are clipped by the tensor map
                         asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                                     ::"l"(&map_out), "r"(smem_u32(stage)), "r"(c0), "r"((int)row0) : "memory");
+                                     ::"l"(&map_out), "r"(smem_u32(stage)), "r"(ncol0), "r"((int)row0) : "memory");
                         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    }
+                } else {
+                    // a ragged last slice of the half (BN / 2 is not a multiple of 32): lane = row, plain stores
+                    const int64_t row = row0 + lane;
+                    if (row < a.M) {
+                        float* orow = a.out + row * a.N;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            const int n = ncol0 + 4 * c;
+                            if (c0 + 4 * c < half_n && n < a.N) {
+                                const float4 bb = __ldg(reinterpret_cast<const float4*>(a.bias + n));
+                                float4 o = make_float4(__uint_as_float(v[4 * c]) + bb.x, __uint_as_float(v[4 * c + 1]) + bb.y,
+                                                       __uint_as_float(v[4 * c + 2]) + bb.z, __uint_as_float(v[4 * c + 3]) + bb.w);
+                                if (a.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f); }
+                                *reinterpret_cast<float4*>(orow + n) = o;
+                            }
+                        }
                     }
                 }
             }
@@ -263,19 +304,17 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
         // slot L % 8.  Producer warps only meet at the mbarriers, never at a block-wide barrier.
         const int pw = warp - kFirstProducerWarp;     // 0 .. kProducerWarps-1
         const int gl = lane & 7;                      // 16-byte slot inside a 128-byte slice row
-        const int n_groups = (a.d_in_pad + kGroupCols - 1) / kGroupCols;
         bool ok = true;
         for (uint32_t it = 0; it < my_iters; ++it) {
             for (int grp = 0; grp < n_groups; ++grp) {
-                const uint32_t u = it * (uint32_t)n_groups + (uint32_t)grp;   // (tile, group) unit of this pair
-                const uint32_t cnt = it * (uint32_t)n_chunks + (uint32_t)grp * (2 * kGroupCols / KC);   // its first K slice
+                const uint32_t s_h = it * (uint32_t)n_groups + (uint32_t)grp;   // fills of each half's stage rows so far
                 const int pairs = min(kGroupCols / KC, (a.d_in_pad - grp * kGroupCols) / KC);   // slice pairs in this group
                 const int col = grp * kGroupCols + lane * 4;
                 const bool lane_on = (lane >> 3) < pairs;
                 const bool col_ok = lane_on && col < a.d_in;
                 const char* src = a.src_base + (size_t)col * (HALF ? 2 : 4);
-                bool waited = false;
                 for (int blk = 0; blk < kBlocksPerTile; ++blk) {
+                    const int h = blk / kBlocksPerHalf;               // the half tile this block belongs to
                     const uint32_t q = it * kBlocksPerTile + blk;     // row block counter of this CTA
                     const int slot = q % kPlanSlots;
                     if (grp == 0 && ok && !mbar_wait(&plan_full[slot], (q / kPlanSlots) & 1)) {
@@ -348,19 +387,19 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&plan_empty[slot]);
                     }
-                    if (!waited) {
-                        // the stages must have been read by the MMAs of the previous unit (one commit frees them all);
-                        // the loads above are already in flight while this waits
-                        if (ok && u >= 1 && !mbar_wait(&a_free[(u - 1) & 1], ((u - 1) >> 1) & 1)) {
+                    if (blk % kBlocksPerHalf == 0) {
+                        // the half's rows of the stages must have been read by the MMAs of their previous fill (one
+                        // commit frees them all); those MMAs ran while the other half was gathered, and the loads
+                        // above are already in flight while this waits
+                        if (ok && s_h >= 1 && !mbar_wait(&a_free[h], (s_h - 1) & 1)) {
                             if (lane == 0) atomicExch(a.error, 15u);
                             ok = false;
                         }
                         ok = __all_sync(0xFFFFFFFFu, ok);
-                        waited = true;
                     }
                     if (ok && lane_on) {
                         // K-major, 128-byte swizzle: 16-byte slot gl of row r lands in slot gl ^ (r % 8)
-                        const uint32_t s_self = (cnt + 2 * (lane >> 3)) % a.sa, s_mean = (cnt + 2 * (lane >> 3) + 1) % a.sa;
+                        const uint32_t s_self = 2 * (lane >> 3), s_mean = 2 * (lane >> 3) + 1;   // the group's slice = its stage
                         uint8_t* stage_self = a_base + (size_t)s_self * kABytes;
                         uint8_t* stage_mean = a_base + (size_t)s_mean * kABytes;
 #pragma unroll
@@ -371,12 +410,15 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                             *reinterpret_cast<float4*>(stage_mean + off) = acc[q2];
                         }
                     }
-                }
-                fence_async_smem();
-                __syncwarp();
-                if (ok && lane == 0) {   // this warp's rows of the unit are in place: tell the leader's MMA thread
-                    if (leader) mbar_arrive(&a_ready[u & 1]);
-                    else mbar_arrive_cluster(mapa_u32(smem_u32(&a_ready[u & 1]), 0));
+                    if (blk % kBlocksPerHalf == kBlocksPerHalf - 1) {
+                        // this warp's rows of the half are in place: tell the leader's MMA thread
+                        fence_async_smem();
+                        __syncwarp();
+                        if (ok && lane == 0) {
+                            if (leader) mbar_arrive(&a_ready[h]);
+                            else mbar_arrive_cluster(mapa_u32(smem_u32(&a_ready[h]), 0));
+                        }
+                    }
                 }
             }
         }
@@ -545,8 +587,8 @@ int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_ou
     a.relu = relu ? 1 : 0;
     a.bias = bias; a.out = h_out;
     int stride = 32;
-    while (stride < a.BN) stride <<= 1;
-    a.tmem_cols = 2 * stride;   // two accumulator buffers, each a power of two >= 32 columns
+    while (stride < a.BN / 2) stride <<= 1;
+    a.tmem_cols = kAccBufs * stride;   // accumulator buffers of half tiles: BN / 2 columns each, a power of two >= 32
     const int b_bytes = (a.BN / 2) * KC * 4;    // each CTA of a pair stages half of the output columns
     const int n_chunks = 2 * a.d_in_pad / KC;
     a.sa = std::min(8, n_chunks);   // one group of (self, mean) slice pairs: 128 input columns
