@@ -357,9 +357,10 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                                 for (int j = 0; j < kUnroll; ++j)   // entry order
 #pragma unroll
                                     for (int q2 = 0; q2 < kRowsInFlight; ++q2) {
-                                        const bool live = e + j < mq[q2].z;   // selects, not branches
-                                        acc[q2].x += live ? v[q2][j].x : 0.f; acc[q2].y += live ? v[q2][j].y : 0.f;
-                                        acc[q2].z += live ? v[q2][j].z : 0.f; acc[q2].w += live ? v[q2][j].w : 0.f;
+                                        if (e + j < mq[q2].z) {   // warp-uniform: a predicated add, not a branch around a load
+                                            acc[q2].x += v[q2][j].x; acc[q2].y += v[q2][j].y;
+                                            acc[q2].z += v[q2][j].z; acc[q2].w += v[q2][j].w;
+                                        }
                                     }
                             }
                         } else {
