@@ -40,7 +40,7 @@ CONFIGS = {
 DEFAULT_WORKLOAD = "config3_papers100m_shaped"
 HBM_NOMINAL_GBS = 8000.0
 # dram bytes (read + write) of one launch of the dominant kernel, measured with ncu (see profiles/)
-NCU_TRAFFIC_PER_LAUNCH = {("config3_papers100m_shaped", 128): 10.58e9}
+NCU_TRAFFIC_PER_LAUNCH = {("config3_papers100m_shaped", 128): 10.70e9}
 
 
 def measured_peaks():
