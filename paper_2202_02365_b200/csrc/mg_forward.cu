@@ -597,6 +597,10 @@ extern "C" int mg_gather_h0(mg_ctx* ctx, mg_dense* d, int32_t batch, float* out_
     if (!ctx->slots || ctx->feat_dim <= 0) return mg_fail(ctx, MG_ERR_STATE, "no feature table loaded");
     if (batch < 0 || batch >= d->n_batches) return mg_fail(ctx, MG_ERR_ARG, "batch out of range");
     MG_CUDA(ctx, cudaSetDevice(ctx->device));
+    {
+        const int rc0 = mg_dense_canonicalize(ctx, d);   // rows come in the paper's order
+        if (rc0) return rc0;
+    }
     H0Args a;
     fill_row_export(d, batch, 0, ctx->feat_dim, &a.r);
     for (int h = 0; h <= d->k; ++h) a.node_off[h] = d->h_node_off[(size_t)h * (d->n_batches + 1) + batch];

@@ -625,6 +625,47 @@ k_finalize(DenseHeader* hdr, int32_t B, int32_t k, const int32_t* __restrict__ c
             ent_hop[h * (B + 1) + b] = ent_off[node_off[h * (B + 1) + b]];
 }
 
+
+// -------------------------------------------------------------------------------------
+// ascending id order for the outermost delta (on demand)
+// -------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+k_canon_keys(const int32_t* __restrict__ nodes, const int32_t* __restrict__ node_batch, const int32_t* __restrict__ node_off_k,
+             int32_t start, int32_t n, int id_bits, uint64_t* keys) {
+    for (int32_t j = blockIdx.x * blockDim.x + threadIdx.x; j < n; j += gridDim.x * blockDim.x) {
+        const int32_t b = node_batch[start + j];
+        const uint64_t local = (uint64_t)(start + j - node_off_k[b]);   // position inside the mini-batch's delta
+        keys[j] = ((uint64_t)b << (MG_SLOT_BITS + id_bits)) | ((uint64_t)(uint32_t)nodes[start + j] << MG_SLOT_BITS) | local;
+    }
+}
+
+// sorted position p of the hop -> the node id goes to its place, and the old position learns its new one
+__global__ void __launch_bounds__(kThreads)
+k_canon_place(const uint64_t* __restrict__ sorted, const int32_t* __restrict__ node_off_k, int32_t start, int32_t n, int id_bits,
+              int32_t* nodes, int32_t* new_local) {
+    const uint64_t id_mask = (1ull << id_bits) - 1ull;
+    for (int32_t p = blockIdx.x * blockDim.x + threadIdx.x; p < n; p += gridDim.x * blockDim.x) {
+        const uint64_t key = sorted[p];
+        const int32_t b = (int32_t)(key >> (MG_SLOT_BITS + id_bits));
+        const int32_t old_local = (int32_t)(key & ((1u << MG_SLOT_BITS) - 1u));
+        nodes[start + p] = (int32_t)((key >> MG_SLOT_BITS) & id_mask);
+        new_local[node_off_k[b] - start + old_local] = start + p - node_off_k[b];
+    }
+}
+
+// entries of the last sampling round that point into the outermost delta follow their node
+__global__ void __launch_bounds__(kThreads)
+k_canon_relabel(int32_t e_lo, int32_t e_hi, const int32_t* __restrict__ ent_hop_last, int32_t B, int32_t k,
+                const int32_t* __restrict__ cum, const int32_t* __restrict__ node_off_k, int32_t start,
+                const int32_t* __restrict__ new_local, int32_t* ent_repr) {
+    for (int32_t e = e_lo + blockIdx.x * blockDim.x + threadIdx.x; e < e_hi; e += gridDim.x * blockDim.x) {
+        const int b = upper_segment(ent_hop_last, B + 1, e);
+        const int32_t base = cum[b * (k + 2) + k];      // first local row of the outermost delta in this mini-batch
+        const int32_t l = ent_repr[e];
+        if (l >= base) ent_repr[e] = base + new_local[node_off_k[b] - start + (l - base)];
+    }
+}
+
 // -------------------------------------------------------------------------------------
 // export to the paper's layout (mg_dense_view)
 // -------------------------------------------------------------------------------------
@@ -841,6 +882,7 @@ extern "C" int mg_sample_many_end(mg_ctx* ctx, mg_dense* d) {
     d->h_ent_hop.assign(p, p + (size_t)k * (B + 1));
     if (d->h_hdr.status) return mg_fail(ctx, status_code(d->h_hdr.status), "%s", status_text(d->h_hdr.status));
     d->valid = true;
+    d->canonical = d->k == 0;
     return MG_OK;
 }
 
@@ -985,11 +1027,17 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
         }
         int res_buf = 0;
         {
-            const int key_bits = id_bits + b_bits;
+            // Inner deltas are sorted by (mini-batch, id): ascending ids inside a mini-batch.  The outermost delta is
+            // only grouped by mini-batch here: nothing on the path depends on the order of its ids (no later round
+            // samples from it, layer 1 reads its representations by global id), so it stays in discovery order until
+            // someone asks for the paper's arrays (mg_dense_canonicalize).
+            const bool outermost = h == k - 1;
+            const int lo_bit = outermost ? MG_SLOT_BITS + id_bits : MG_SLOT_BITS;
+            const int key_bits = outermost ? b_bits : id_bits + b_bits;
             const int passes = (key_bits + kRadixBits - 1) / kRadixBits;
             ProfScope ps(ctx, PH_SAMPLE_SORT, 1 + passes * 5);
             k_sort_setup<<<1, 1, 0, st>>>(d->hdr, sp);
-            mg_sort_u64(ctx, d->newlist, sp, MG_SLOT_BITS, key_bits, d->sort_hist, (uint32_t*)d->scan_tmp, &res_buf);
+            mg_sort_u64(ctx, d->newlist, sp, lo_bit, key_bits, d->sort_hist, (uint32_t*)d->scan_tmp, &res_buf);
         }
         {
             ProfScope ps(ctx, PH_SAMPLE_PLACE, 3);
@@ -1063,12 +1111,46 @@ extern "C" int mg_dense_counts(const mg_dense* d, int32_t* n_batches, int32_t* k
     return MG_OK;
 }
 
+
+int mg_dense_canonicalize(mg_ctx* ctx, mg_dense* d) {
+    if (d->canonical) return MG_OK;
+    const int k = d->k, B = d->n_batches;
+    const int32_t start = d->h_hdr.hop_base[k], n = d->h_hdr.hop_base[k + 1] - start;
+    if (k == 0 || n <= 0) { d->canonical = true; return MG_OK; }
+    cudaStream_t st = ctx->stream;
+    const int id_bits = std::max(1, ilog2_ceil(ctx->n_nodes)), b_bits = std::max(1, ilog2_ceil(B));
+    const int32_t* node_off_k = d->node_off + (size_t)k * (B + 1);
+    SortParams* sp = (SortParams*)(d->scan_tmp + d->scan_tmp_elems - 8);   // tail of the scratch block, as in the sampler
+    SortParams h_sp;
+    mg_sort_params_host(&h_sp, n);
+    MG_CUDA(ctx, cudaMemcpyAsync(sp, &h_sp, sizeof(h_sp), cudaMemcpyHostToDevice, st));
+    const int grid = mg_grid(ctx, 8);
+    k_canon_keys<<<grid, kThreads, 0, st>>>(d->nodes, d->node_batch, node_off_k, start, n, id_bits, d->newlist[0]);
+    int res = 0;
+    mg_sort_u64(ctx, d->newlist, sp, MG_SLOT_BITS, id_bits + b_bits, d->sort_hist, (uint32_t*)d->scan_tmp, &res);
+    int32_t* new_local = reinterpret_cast<int32_t*>(d->node_r0);   // per-node scratch of the sampler, free by now
+    k_canon_place<<<grid, kThreads, 0, st>>>(d->newlist[res], node_off_k, start, n, id_bits, d->nodes, new_local);
+    const int32_t e_lo = d->h_hdr.ent_base[k - 1], e_hi = d->h_hdr.ent_base[k];
+    if (e_hi > e_lo)
+        k_canon_relabel<<<grid, kThreads, 0, st>>>(e_lo, e_hi, d->d_ent_hop + (size_t)(k - 1) * (B + 1), B, k, d->cum, node_off_k,
+                                                   start, new_local, d->ent_repr);
+    ctx->launches += 3;
+    MG_CUDA(ctx, cudaGetLastError());
+    MG_CUDA(ctx, cudaStreamSynchronize(st));   // h_sp is a stack variable
+    d->canonical = true;
+    return MG_OK;
+}
+
 extern "C" int mg_dense_view(mg_ctx* ctx, mg_dense* d, int32_t batch, mg_dense_arrays* out) {
     if (!ctx) return MG_ERR_ARG;
     if (!d || !out) return mg_fail(ctx, MG_ERR_ARG, "null argument");
     if (!d->valid) return mg_fail(ctx, MG_ERR_STATE, "mg_dense holds no completed sample");
     if (batch < 0 || batch >= d->n_batches) return mg_fail(ctx, MG_ERR_ARG, "batch out of range");
     MG_CUDA(ctx, cudaSetDevice(ctx->device));
+    {
+        const int rc0 = mg_dense_canonicalize(ctx, d);
+        if (rc0) return rc0;
+    }
     const int k = d->k, B = d->n_batches, b = batch;
     ExportArgs a;
     memset(&a, 0, sizeof(a));
