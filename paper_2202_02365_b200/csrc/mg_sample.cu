@@ -333,13 +333,27 @@ struct InsertArgs {
     uint64_t* newlist;
     int64_t cap_new;
     int id_bits;
+    // outermost hop only: rows are handed out at insert time
+    int32_t k;
+    const int32_t* cum;          // [B][k+2]
+    int32_t* hvals;
+    uint32_t* batch_cnt;         // [B] new nodes of the hop per mini-batch, zero before the launch
+    int32_t max_nodes_per_batch;
 };
 
 constexpr int kInsertPerThread = 8;
+constexpr int kInsertSpan = 16;   // mini-batches a block's chunk of entries may touch on the fast path
 
+// OUTER = the last sampling round.  Its new nodes are not sorted (nothing depends on their order, see
+// mg_dense_canonicalize): a new node takes the next free row of its mini-batch right here -- a count per
+// mini-batch in shared memory, one global atomic per (block, mini-batch) -- its table value is written at once, and
+// the list entry carries (mini-batch, id, rank) instead of (mini-batch, id, table slot).
+template <bool OUTER>
 __global__ void __launch_bounds__(kThreads) k_insert(InsertArgs a) {
     __shared__ uint32_t warp_tot[kThreads / 32 + 1];
     __shared__ uint32_t block_base;
+    __shared__ uint32_t span_cnt[kInsertSpan], span_base[kInsertSpan];
+    __shared__ int32_t first_batch;
     if (a.hdr->status) return;
     const int32_t lo = a.hdr->ent_base[a.hop], hi = a.hdr->ent_base[a.hop + 1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -390,10 +404,39 @@ __global__ void __launch_bounds__(kThreads) k_insert(InsertArgs a) {
         }
         __syncthreads();
         int64_t pos = (int64_t)block_base + warp_tot[warp] + inc - n_mine;
+        uint32_t rank[kInsertPerThread];
+        if (OUTER) {
+            // entries are ordered by mini-batch, so a chunk touches a short run of them
+            if (threadIdx.x == 0) first_batch = b[0];   // thread 0's first item is the chunk's first entry
+            if (threadIdx.x < kInsertSpan) span_cnt[threadIdx.x] = 0;
+            __syncthreads();
+            const int32_t b0 = first_batch;
+#pragma unroll
+            for (int j = 0; j < kInsertPerThread; ++j) {
+                rank[j] = 0;
+                if (new_bits & (1u << j)) {
+                    const int32_t bb = b[j] - b0;
+                    rank[j] = bb < kInsertSpan ? atomicAdd(&span_cnt[bb], 1u) : atomicAdd(&a.batch_cnt[b[j]], 1u);
+                }
+            }
+            __syncthreads();
+            if (threadIdx.x < kInsertSpan && span_cnt[threadIdx.x])
+                span_base[threadIdx.x] = atomicAdd(&a.batch_cnt[b0 + threadIdx.x], span_cnt[threadIdx.x]);
+            __syncthreads();
+#pragma unroll
+            for (int j = 0; j < kInsertPerThread; ++j)
+                if (new_bits & (1u << j)) {
+                    const int32_t bb = b[j] - b0;
+                    if (bb < kInsertSpan) rank[j] += span_base[bb];
+                    const int64_t row = (int64_t)a.cum[b[j] * (a.k + 2) + a.k] + rank[j];
+                    if (row < a.max_nodes_per_batch) a.hvals[(int64_t)b[j] * a.tg.size + slot[j]] = (int32_t)row;
+                    else atomicOr(&a.hdr->status, ST_CAP_TABLE);
+                }
+        }
 #pragma unroll
         for (int j = 0; j < kInsertPerThread; ++j)
             if (new_bits & (1u << j)) {
-                const uint64_t key = (uint64_t)slot[j] | ((uint64_t)(uint32_t)u[j] << MG_SLOT_BITS) |
+                const uint64_t key = (uint64_t)(OUTER ? rank[j] : slot[j]) | ((uint64_t)(uint32_t)u[j] << MG_SLOT_BITS) |
                                      ((uint64_t)(uint32_t)b[j] << (MG_SLOT_BITS + a.id_bits));
                 if (pos < a.cap_new) a.newlist[pos] = key;
                 else atomicOr(&a.hdr->status, ST_CAP_NODES);
@@ -587,6 +630,56 @@ k_relabel(const DenseHeader* hdr, int hop, const int32_t* __restrict__ hvals, in
     const int32_t lo = hdr->ent_base[hop], hi = hdr->ent_base[hop + 1];
     for (int32_t e = lo + blockIdx.x * blockDim.x + threadIdx.x; e < hi; e += gridDim.x * blockDim.x)
         ent_repr[e] = hvals[ent_repr[e]];
+}
+
+// Outermost hop: per-batch counts -> node offsets of the hop and the batches' row totals (one block)
+__global__ void __launch_bounds__(1024)
+k_outer_offsets(DenseHeader* hdr, int hop, int32_t B, int32_t k, const uint32_t* __restrict__ batch_cnt, int32_t* node_off_next,
+                int32_t* cum, int32_t max_nodes_per_batch) {
+    __shared__ uint32_t warp_tot[33];
+    if (hdr->status) return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int32_t start = hdr->hop_base[hop + 1];
+    uint32_t carry = 0;
+    for (int s0 = 0; s0 < B; s0 += 1024) {
+        const int b = s0 + threadIdx.x;
+        const uint32_t v = b < B ? batch_cnt[b] : 0u;
+        const uint32_t inc = warp_incl_scan(v);
+        if (lane == 31) warp_tot[warp] = inc;
+        __syncthreads();
+        if (warp == 0) {
+            const uint32_t w = warp_tot[lane];
+            const uint32_t wi = warp_incl_scan(w);
+            warp_tot[lane] = wi - w;
+            if (lane == 31) warp_tot[32] = wi;
+        }
+        __syncthreads();
+        if (b < B) {
+            node_off_next[b] = start + (int32_t)(carry + warp_tot[warp] + inc - v);
+            const int32_t rows = cum[b * (k + 2) + hop + 1] + (int32_t)v;
+            cum[b * (k + 2) + hop + 2] = rows;
+            if (rows > max_nodes_per_batch) atomicOr(&hdr->status, ST_CAP_TABLE);
+        }
+        carry += warp_tot[32];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) node_off_next[B] = start + (int32_t)carry;
+}
+
+// Outermost hop: list entry (mini-batch, id, rank) -> the node's place in its mini-batch's run
+__global__ void __launch_bounds__(kThreads)
+k_place_nodes_outer(const DenseHeader* hdr, const uint64_t* __restrict__ list, int id_bits, const int32_t* __restrict__ node_off_next,
+                    int32_t* nodes, int32_t* node_batch) {
+    if (hdr->status) return;
+    const int32_t n = (int32_t)hdr->n_new;
+    const uint64_t id_mask = (1ull << id_bits) - 1ull;
+    for (int32_t j = blockIdx.x * blockDim.x + threadIdx.x; j < n; j += gridDim.x * blockDim.x) {
+        const uint64_t key = list[j];
+        const int32_t b = (int32_t)(key >> (MG_SLOT_BITS + id_bits));
+        const int32_t at = node_off_next[b] + (int32_t)(key & ((1u << MG_SLOT_BITS) - 1u));
+        nodes[at] = (int32_t)((key >> MG_SLOT_BITS) & id_mask);
+        node_batch[at] = b;
+    }
 }
 
 // one block: packed row bases of every layer and the per-batch entry bounds of every hop
@@ -994,6 +1087,9 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
     }
 
     SortParams* sp = (SortParams*)(d->scan_tmp + d->scan_tmp_elems - 8);  // tail of the scratch block
+    // new nodes of the outermost hop per mini-batch: the unused last block of the row-base array
+    uint32_t* batch_cnt = reinterpret_cast<uint32_t*>(d->rowbase + (size_t)(MG_MAX_HOPS + 1) * (B + 1));
+    MG_CUDA(ctx, cudaMemsetAsync(batch_cnt, 0, sizeof(uint32_t) * B, st));
     uint32_t* scan_total = (uint32_t*)(d->scan_tmp + d->scan_tmp_elems - 4);
     const int grid = mg_grid(ctx, 8);
     for (int h = 0; h < k; ++h) {
@@ -1021,37 +1117,46 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
                 MG_CUDA(ctx, cudaFuncSetAttribute(k_pick_wide, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)wide_smem));
                 k_pick_wide<<<grid, kThreads, wide_smem, st>>>(a);
             }
-            InsertArgs ia{d->hdr, h, d->ent_nbrs, d->ent_repr, d->hkeys, tg, d->newlist[0], d->cap_nodes, id_bits};
-            k_insert<<<grid, kThreads, 0, st>>>(ia);
+            InsertArgs ia{d->hdr, h, d->ent_nbrs, d->ent_repr, d->hkeys, tg, d->newlist[0], d->cap_nodes, id_bits,
+                          k, d->cum, d->hvals, batch_cnt, (int32_t)cap_batch};
+            if (h == k - 1) k_insert<true><<<grid, kThreads, 0, st>>>(ia);
+            else k_insert<false><<<grid, kThreads, 0, st>>>(ia);
             ctx->launches++;
         }
-        int res_buf = 0;
-        {
-            // Inner deltas are sorted by (mini-batch, id): ascending ids inside a mini-batch.  The outermost delta is
-            // only grouped by mini-batch here: nothing on the path depends on the order of its ids (no later round
-            // samples from it, layer 1 reads its representations by global id), so it stays in discovery order until
-            // someone asks for the paper's arrays (mg_dense_canonicalize).
-            const bool outermost = h == k - 1;
-            const int lo_bit = outermost ? MG_SLOT_BITS + id_bits : MG_SLOT_BITS;
-            const int key_bits = outermost ? b_bits : id_bits + b_bits;
-            const int passes = (key_bits + kRadixBits - 1) / kRadixBits;
-            ProfScope ps(ctx, PH_SAMPLE_SORT, 1 + passes * 5);
-            k_sort_setup<<<1, 1, 0, st>>>(d->hdr, sp);
-            mg_sort_u64(ctx, d->newlist, sp, lo_bit, key_bits, d->sort_hist, (uint32_t*)d->scan_tmp, &res_buf);
-        }
-        {
+        if (h == k - 1) {
+            // The outermost delta: rows were handed out at insert time, in discovery order (nothing on the path
+            // depends on the order of its ids; mg_dense_canonicalize sorts it on demand).  No sort, no table pass.
             ProfScope ps(ctx, PH_SAMPLE_PLACE, 3);
             int32_t* off_next = d->node_off + (size_t)(h + 1) * (B + 1);
             k_hop_advance<<<1, 256, 0, st>>>(d->hdr, h, B, off_next, d->cap_nodes);
-            k_place_nodes<<<grid, kThreads, 0, st>>>(d->hdr, h, B, d->newlist[res_buf], id_bits, d->nodes, d->node_batch, off_next);
-            k_place_rows<<<grid, kThreads, 0, st>>>(d->hdr, h, B, k, d->newlist[res_buf], id_bits, off_next, d->cum, d->hvals, tg,
-                                                    (int32_t)cap_batch);
+            k_outer_offsets<<<1, 1024, 0, st>>>(d->hdr, h, B, k, batch_cnt, off_next, d->cum, (int32_t)cap_batch);
+            k_place_nodes_outer<<<grid, kThreads, 0, st>>>(d->hdr, d->newlist[0], id_bits, off_next, d->nodes, d->node_batch);
+            ctx->launches += 3;
+        } else {
+            int res_buf = 0;
+            {
+                // inner deltas are sorted by (mini-batch, id): ascending ids inside a mini-batch
+                const int key_bits = id_bits + b_bits;
+                const int passes = (key_bits + kRadixBits - 1) / kRadixBits;
+                ProfScope ps(ctx, PH_SAMPLE_SORT, 1 + passes * 5);
+                k_sort_setup<<<1, 1, 0, st>>>(d->hdr, sp);
+                mg_sort_u64(ctx, d->newlist, sp, MG_SLOT_BITS, key_bits, d->sort_hist, (uint32_t*)d->scan_tmp, &res_buf);
+            }
+            {
+                ProfScope ps(ctx, PH_SAMPLE_PLACE, 3);
+                int32_t* off_next = d->node_off + (size_t)(h + 1) * (B + 1);
+                k_hop_advance<<<1, 256, 0, st>>>(d->hdr, h, B, off_next, d->cap_nodes);
+                k_place_nodes<<<grid, kThreads, 0, st>>>(d->hdr, h, B, d->newlist[res_buf], id_bits, d->nodes, d->node_batch, off_next);
+                k_place_rows<<<grid, kThreads, 0, st>>>(d->hdr, h, B, k, d->newlist[res_buf], id_bits, off_next, d->cum, d->hvals, tg,
+                                                        (int32_t)cap_batch);
+            }
+            ctx->launches += 1 + 3;   // sort_setup, place x3
         }
         {
             ProfScope ps(ctx, PH_SAMPLE_RELABEL, 1);
             k_relabel<<<grid, kThreads, 0, st>>>(d->hdr, h, d->hvals, d->ent_repr);
         }
-        ctx->launches += 1 + 1 + 1 + 1 + 3 + 1;  // count, entries_done, pick, sort_setup, place x3, relabel
+        ctx->launches += 1 + 1 + 1 + 1;  // count, entries_done, pick, relabel
     }
     {
         ProfScope ps(ctx, PH_SAMPLE_FINAL, 1);
