@@ -400,7 +400,8 @@ static int finish_forward(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* ou
         MG_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_fwd_done, 0));
         MG_CUDA(ctx, cudaMemcpyAsync(out, hk, out_bytes, cudaMemcpyDeviceToHost, ctx->side));
         MG_CUDA(ctx, cudaEventRecord(ctx->ev_out_done, ctx->side));
-        ctx->out_copy_pending = true;
+        MG_CUDA(ctx, cudaEventRecord(ctx->ev_hk_done[ctx->hk_cur], ctx->side));   // this H^k buffer is free again after the copy
+        ctx->hk_pending[ctx->hk_cur] = true;
         ctx->out_check_gemm = m->precision == MG_GEMM_TF32;
         return MG_OK;
     }
@@ -418,9 +419,20 @@ static int forward_impl(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out,
     MG_CUDA(ctx, cudaSetDevice(ctx->device));
     const int k = d->k, B = d->n_batches;
     cudaStream_t st = ctx->stream;
-    if (ctx->out_copy_pending) {   // the previous asynchronous output copy still reads the layer workspace
-        MG_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_out_done, 0));
-        ctx->out_copy_pending = false;
+    // H^k of this pass goes to the buffer the pass before last used; an output copy of that pass to the host (side
+    // stream) may still read it.  The copy of the previous pass reads the other buffer and is not waited for.
+    float* hk = nullptr;
+    {
+        const int hi = ctx->hk_cur ^= 1;
+        if (!ctx->ev_hk_done[hi]) MG_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_hk_done[hi], cudaEventDisableTiming));
+        if (ctx->hk_pending[hi]) {
+            MG_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_hk_done[hi], 0));
+            ctx->hk_pending[hi] = false;
+        }
+        const size_t need = (size_t)d->h_hdr.rows_total[k] * m->dims[k];
+        if (ctx->hk_elems[hi] < need && (rc = mg_ensure(ctx, &ctx->hk_buf[hi], &ctx->hk_elems[hi], need + need / 4 + 4))) return rc;
+        hk = ctx->hk_buf[hi];
+        ctx->last_hk = hk;
     }
 
     // Windowed schedule: when every layer runs in the fused kernel and the intermediate layer outputs need not
@@ -438,7 +450,7 @@ static int forward_impl(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out,
             meta_off[l] = meta_total;
             meta_total += (size_t)d->h_hdr.rows_total[l];
             ring_off[l] = ring_total;
-            if (l == k) { ring_total += (size_t)d->h_hdr.rows_total[k] * m->dims[k]; break; }
+            if (l == k) break;
             int64_t widest = 0;
             for (int b0 = 0; b0 < B; b0 += sub) {
                 const int b1 = std::min(B, b0 + sub);
@@ -474,7 +486,7 @@ static int forward_impl(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out,
                 const int64_t lo_in = rb[(size_t)(l - 1) * (B + 1) + b0];
                 // pointers shifted so that the kernel's global packed row indices land inside the windows
                 const float* h_prev = l > 1 ? base + ring_off[l - 1] - lo_in * m->dims[l - 1] : nullptr;
-                float* h_out = l == k ? base + ring_off[k] : base + ring_off[l] - lo * m->dims[l];
+                float* h_out = l == k ? hk : base + ring_off[l] - lo * m->dims[l];
                 ProfScope ps(ctx, l == 1 ? PH_AGG_L1 : PH_AGG_REST, 1);
                 rc = mg_layer_fused(ctx, d, l, m->dims[l - 1], m->dims[l], m->w_pad_t[l - 1], m->bias[l - 1], h_prev, h_out,
                                     l < k, meta + meta_off[l], lo, hi, l > 1 ? lo_in : 0);
@@ -482,16 +494,17 @@ static int forward_impl(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out,
             }
         }
         MG_CUDA(ctx, cudaGetLastError());
-        return finish_forward(ctx, m, d, out, out_mode, base + ring_off[k]);
+        return finish_forward(ctx, m, d, out, out_mode, hk);
     }
 
     // per-layer outputs H^1..H^k live in one workspace (kept for mg_layer_output)
     size_t total = 0;
     size_t off[MG_MAX_HOPS + 1];
-    for (int l = 1; l <= k; ++l) {
+    for (int l = 1; l < k; ++l) {
         off[l] = total;
         total += (size_t)d->h_hdr.rows_total[l] * m->dims[l];
     }
+    off[k] = 0;   // H^k has buffers of its own
     {
         size_t have = ctx->ws_h_bytes[0] / sizeof(float);
         // a quarter of headroom: the row counts of consecutive calls differ slightly, and growing means a
@@ -514,7 +527,7 @@ static int forward_impl(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out,
     for (int l = 1; l <= k; ++l) {
         const int d_in = m->dims[l - 1], d_out = m->dims[l];
         const int64_t M = d->h_hdr.rows_total[l];
-        float* h_out = ctx->ws_h[0] + off[l];
+        float* h_out = l == k ? hk : ctx->ws_h[0] + off[l];
         const float* h_prev = l > 1 ? ctx->ws_h[0] + off[l - 1] : nullptr;
         if (m->precision == MG_GEMM_TF32 && mg_layer_fused_supported(d_in, d_out)) {
             // gather + segment mean + both linear maps in one persistent tensor-core kernel
@@ -571,7 +584,7 @@ static int forward_impl(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out,
         }
     }
     MG_CUDA(ctx, cudaGetLastError());
-    return finish_forward(ctx, m, d, out, out_mode, ctx->ws_h[0] + off[k]);
+    return finish_forward(ctx, m, d, out, out_mode, hk);
 }
 
 extern "C" int mg_forward(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out, int out_on_device) {
@@ -623,13 +636,15 @@ extern "C" int mg_layer_output(mg_ctx* ctx, const mg_model* m, mg_dense* d, int3
     if (!out_dev) return mg_fail(ctx, MG_ERR_ARG, "null output");
     if (layer < 1 || layer > d->k) return mg_fail(ctx, MG_ERR_ARG, "layer must be in [1, k]");
     if (batch < 0 || batch >= d->n_batches) return mg_fail(ctx, MG_ERR_ARG, "batch out of range");
-    if (!ctx->ws_h[0]) return mg_fail(ctx, MG_ERR_STATE, "mg_forward has not run");
+    if (!ctx->last_hk) return mg_fail(ctx, MG_ERR_STATE, "mg_forward has not run");
     if (!ctx->layers_kept) return mg_fail(ctx, MG_ERR_STATE, "the last forward did not keep its intermediate layers: call mg_keep_layer_outputs(ctx, 1) first");
     MG_CUDA(ctx, cudaSetDevice(ctx->device));
     size_t off = 0;
     for (int l = 1; l < layer; ++l) off += (size_t)d->h_hdr.rows_total[l] * m->dims[l];
     const int B = d->n_batches;
-    const float* src = ctx->ws_h[0] + off + (size_t)d->h_rowbase[(size_t)layer * (B + 1) + batch] * m->dims[layer];
+    const float* layer_base = layer == d->k ? ctx->last_hk : ctx->ws_h[0] + off;
+    if (!layer_base) return mg_fail(ctx, MG_ERR_STATE, "mg_forward has not run");
+    const float* src = layer_base + (size_t)d->h_rowbase[(size_t)layer * (B + 1) + batch] * m->dims[layer];
     RowExportArgs r;
     fill_row_export(d, batch, layer, m->dims[layer], &r);
     if (r.n_rows > 0) {

@@ -112,7 +112,15 @@ struct mg_ctx {
 
     // asynchronous output copy of mg_forward_host_async
     cudaEvent_t ev_fwd_done = nullptr, ev_out_done = nullptr;
-    bool out_copy_pending = false, out_check_gemm = false;
+    bool out_check_gemm = false;
+    // H^k goes to one of two buffers in turn, so that a forward pass need not wait for the copy of the previous
+    // pass's output to the host
+    float* hk_buf[2] = {nullptr, nullptr};
+    size_t hk_elems[2] = {0, 0};
+    cudaEvent_t ev_hk_done[2] = {nullptr, nullptr};
+    bool hk_pending[2] = {false, false};
+    int hk_cur = 0;
+    const float* last_hk = nullptr;
 
     // profiling
     bool prof_on = false;
