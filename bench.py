@@ -235,24 +235,30 @@ def main():
     host_targets = [step_targets(i).pin_memory() for i in range(n_steps_total)]
 
     out_hosts = [out_host, torch.empty_like(out_host).pin_memory()]
-    denses = [dense, ctx.sample_many(step_targets(0).to(device), offs, cfg["fanouts"], step_seeds(0), caps=caps)]
+    # three sample handles: two groups are always queued ahead of the one whose layers run, so that the GPU has
+    # work while the host reads a finished sample's sizes and queues the next calls
+    denses = [dense] + [ctx.sample_many(step_targets(0).to(device), offs, cfg["fanouts"], step_seeds(0), caps=caps)
+                        for _ in range(2)]
 
     def begin(i, e2e):
         tg = host_targets[i] if e2e else dev_targets[i]
-        ctx.sample_many_begin(tg, offs, cfg["fanouts"], step_seeds(i), caps=caps, out=denses[i & 1])
+        ctx.sample_many_begin(tg, offs, cfg["fanouts"], step_seeds(i), caps=caps, out=denses[i % 3])
 
     def run_steps(first, count, e2e):
-        """`count` steps, software-pipelined: group i+1 is sampled (sampling stream) while group i runs its
-        layers (context stream); with e2e the host H^k of group i is copied out during group i+1."""
+        """`count` steps, software-pipelined: groups i+1 and i+2 are sampled (sampling stream) while group i runs
+        its layers (context stream); with e2e the host H^k of group i is copied out during group i+1."""
+        last = first + count
         begin(first, e2e)
-        for i in range(first, first + count):
-            ctx.sample_many_end(denses[i & 1])
-            if i + 1 < first + count:
-                begin(i + 1, e2e)
+        if first + 1 < last:
+            begin(first + 1, e2e)
+        for i in range(first, last):
+            ctx.sample_many_end(denses[i % 3])
+            if i + 2 < last:
+                begin(i + 2, e2e)
             if e2e:
-                ctx.forward_host_async(model, denses[i & 1], out_hosts[i & 1])
+                ctx.forward_host_async(model, denses[i % 3], out_hosts[i & 1])
             else:
-                ctx.forward(model, denses[i & 1], out_dev)
+                ctx.forward(model, denses[i % 3], out_dev)
         if e2e:
             ctx.wait_output()
 
@@ -287,7 +293,7 @@ def main():
     ctx.profile_read(reset=True)
     for s in range(args.steps):          # one group at a time here, so that the phase events do not overlap
         run_step(args.warmup + s, False)
-        n_, e_ = denses[(args.warmup + s) & 1].counts()
+        n_, e_ = denses[(args.warmup + s) % 3].counts()
         stats["nodes"].append(n_); stats["ents"].append(e_)
     phases = ctx.profile_read(reset=True)
     ctx.profile(False)

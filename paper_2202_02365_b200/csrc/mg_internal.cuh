@@ -173,6 +173,7 @@ struct mg_dense {
     bool canonical = false;          // the outermost delta has been put in ascending id order (mg_dense_canonicalize)
     // asynchronous sampling: the summary lands in pinned memory, ev_sampled marks its arrival
     int32_t* h_pinned = nullptr; size_t h_pinned_ints = 0;
+    int32_t* h_pinned_dev = nullptr; // the same memory as the device sees it
     cudaEvent_t ev_sampled = nullptr;
     cudaEvent_t ev_read_done = nullptr;  // recorded after the last kernel that read this sample
     bool pending = false;

@@ -719,6 +719,26 @@ k_finalize(DenseHeader* hdr, int32_t B, int32_t k, const int32_t* __restrict__ c
 }
 
 
+// The sample's summary (header, per-batch tables) for the host: stored straight into mapped pinned memory.  A copy
+// engine is not used on purpose: a large output copy of a forward pass may be queued on it, and the host would wait
+// for that copy before it learned the sample's sizes.
+__global__ void __launch_bounds__(kThreads)
+k_summary(const DenseHeader* hdr, const int32_t* __restrict__ cum, const int32_t* __restrict__ node_off,
+          const int32_t* __restrict__ rowbase, const int32_t* __restrict__ ent_hop, int32_t n_hdr, int32_t n_cum, int32_t n_off,
+          int32_t n_ent, int32_t* out) {
+    const int32_t total = n_hdr + n_cum + 2 * n_off + n_ent;
+    const int32_t* h = reinterpret_cast<const int32_t*>(hdr);
+    for (int32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+        int32_t j = i, v;
+        if (j < n_hdr) v = j < (int32_t)(sizeof(DenseHeader) / 4) ? h[j] : 0;
+        else if ((j -= n_hdr) < n_cum) v = cum[j];
+        else if ((j -= n_cum) < n_off) v = node_off[j];
+        else if ((j -= n_off) < n_off) v = rowbase[j];
+        else v = ent_hop[j - n_off];
+        out[i] = v;
+    }
+}
+
 // -------------------------------------------------------------------------------------
 // ascending id order for the outermost delta (on demand)
 // -------------------------------------------------------------------------------------
@@ -1171,18 +1191,18 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
         if (d->h_pinned_ints < n_ints) {
             if (d->h_pinned) cudaFreeHost(d->h_pinned);
             d->h_pinned = nullptr; d->h_pinned_ints = 0;
-            if (cudaHostAlloc((void**)&d->h_pinned, n_ints * sizeof(int32_t), cudaHostAllocDefault) != cudaSuccess) {
+            if (cudaHostAlloc((void**)&d->h_pinned, n_ints * sizeof(int32_t), cudaHostAllocMapped) != cudaSuccess ||
+                cudaHostGetDevicePointer((void**)&d->h_pinned_dev, d->h_pinned, 0) != cudaSuccess) {
                 cudaGetLastError();
                 return mg_fail(ctx, MG_ERR_OOM, "pinned host allocation failed");
             }
             d->h_pinned_ints = n_ints;
         }
-        int32_t* p = d->h_pinned;
-        MG_CUDA(ctx, cudaMemcpyAsync(p, d->hdr, sizeof(DenseHeader), cudaMemcpyDeviceToHost, st)); p += (sizeof(DenseHeader) + 3) / 4;
-        MG_CUDA(ctx, cudaMemcpyAsync(p, d->cum, sizeof(int32_t) * (size_t)B * (k + 2), cudaMemcpyDeviceToHost, st)); p += (size_t)B * (k + 2);
-        MG_CUDA(ctx, cudaMemcpyAsync(p, d->node_off, sizeof(int32_t) * (size_t)(k + 1) * (B + 1), cudaMemcpyDeviceToHost, st)); p += (size_t)(k + 1) * (B + 1);
-        MG_CUDA(ctx, cudaMemcpyAsync(p, d->rowbase, sizeof(int32_t) * (size_t)(k + 1) * (B + 1), cudaMemcpyDeviceToHost, st)); p += (size_t)(k + 1) * (B + 1);
-        MG_CUDA(ctx, cudaMemcpyAsync(p, d->d_ent_hop, sizeof(int32_t) * (size_t)k * (B + 1), cudaMemcpyDeviceToHost, st));
+        static_assert(sizeof(DenseHeader) % 4 == 0, "the header is copied as 32-bit words");
+        k_summary<<<8, kThreads, 0, st>>>(d->hdr, d->cum, d->node_off, d->rowbase, d->d_ent_hop, (int32_t)((sizeof(DenseHeader) + 3) / 4),
+                                         B * (k + 2), (k + 1) * (B + 1), k * (B + 1), d->h_pinned_dev);
+        ctx->launches++;
+        MG_CUDA(ctx, cudaGetLastError());
     }
     if (!d->ev_sampled) MG_CUDA(ctx, cudaEventCreateWithFlags(&d->ev_sampled, cudaEventDisableTiming));
     MG_CUDA(ctx, cudaEventRecord(d->ev_sampled, st));
