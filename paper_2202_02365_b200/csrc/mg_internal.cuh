@@ -124,8 +124,16 @@ struct mg_ctx {
 
     // profiling
     bool prof_on = false;
+    bool sample_graphs = true;   // replay the sampler's launches from a CUDA graph
     ProfPhase prof[PH_COUNT];
     std::vector<std::pair<int, std::pair<cudaEvent_t, cudaEvent_t>>> prof_pending;
+};
+
+// everything the sampler's captured device work depends on
+struct SampleSignature {
+    int32_t B, k, table_size, fanouts[MG_MAX_HOPS];
+    int64_t T, cap_batch, cap_nodes, cap_entries, n_nodes, part_size;
+    const void* ptrs[32];
 };
 
 struct mg_dense {
@@ -174,6 +182,10 @@ struct mg_dense {
     // asynchronous sampling: the summary lands in pinned memory, ev_sampled marks its arrival
     int32_t* h_pinned = nullptr; size_t h_pinned_ints = 0;
     int32_t* h_pinned_dev = nullptr; // the same memory as the device sees it
+    int32_t* h_stage = nullptr; size_t h_stage_ints = 0;   // pinned: header, offsets, seeds of the call being queued
+    cudaGraphExec_t graph_exec = nullptr;                 // the sampler's device work for graph_sig
+    SampleSignature graph_sig;
+    int64_t graph_launches = 0;
     cudaEvent_t ev_sampled = nullptr;
     cudaEvent_t ev_read_done = nullptr;  // recorded after the last kernel that read this sample
     bool pending = false;

@@ -16,6 +16,7 @@
 #include <stdarg.h>
 
 #include <algorithm>
+#include <cstdlib>
 
 #include "mg_device.cuh"
 #include "mg_internal.cuh"
@@ -835,6 +836,8 @@ void mg_sort_params_host(SortParams* sp, int64_t n) {
 }
 size_t mg_scan_tmp_elems(int64_t max_elems) { return (size_t)((max_elems + kScanTile - 1) / kScanTile) + 16; }
 
+static void sample_kernel_attributes();
+
 // LSD radix sort of 64-bit keys on bits [lo_bit, lo_bit + bits); sp (device) holds the key count.
 // Keys start in buf[0]; *res_buf tells which buffer holds the result.
 void mg_sort_u64(mg_ctx* ctx, uint64_t* const buf[2], const SortParams* sp, int lo_bit, int bits, uint32_t* hist,
@@ -843,11 +846,7 @@ void mg_sort_u64(mg_ctx* ctx, uint64_t* const buf[2], const SortParams* sp, int 
     const int grid = mg_grid(ctx, 8);
     const int passes = (bits + kRadixBits - 1) / kRadixBits;
     ScanRange r{&sp->zero, &sp->hist_len, nullptr};
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaFuncSetAttribute(k_radix_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScatterSmem);
-        attr_set = true;
-    }
+    sample_kernel_attributes();
     int cur = 0;
     for (int p = 0; p < passes; ++p) {
         const int shift = lo_bit + kRadixBits * p;
@@ -1007,6 +1006,17 @@ extern "C" int mg_sample_many(mg_ctx* ctx, const int32_t* targets, int targets_o
     return mg_sample_many_end(ctx, *out);
 }
 
+
+// dynamic shared-memory limits of the sampler's kernels, set once (not inside a stream capture)
+static void sample_kernel_attributes() {
+    static bool done = false;
+    if (done) return;
+    cudaFuncSetAttribute(k_radix_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScatterSmem);
+    cudaFuncSetAttribute(k_pick_wide, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         (int)((size_t)(kThreads / 32) * 2 * MG_MAX_FANOUT * sizeof(uint32_t)));
+    done = true;
+}
+
 static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on_device,
                              const int64_t* target_offsets, int32_t n_batches, const int32_t* fanouts,
                              int32_t k, const uint64_t* seeds, const mg_sample_caps* caps, mg_dense** out) {
@@ -1077,27 +1087,60 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
     const int B = n_batches;
     const TableGeom tg{table_size, d->table_shift};
 
-    // host-known part of the header and per-batch tables
-    DenseHeader hh;
-    memset(&hh, 0, sizeof(hh));
-    hh.hop_base[0] = 0;
-    hh.hop_base[1] = (int32_t)T;
-    std::vector<int32_t> off32(B + 1), cum0((size_t)B * (k + 2), 0);
-    for (int b = 0; b <= B; ++b) off32[b] = (int32_t)target_offsets[b];
-    for (int b = 0; b < B; ++b) cum0[(size_t)b * (k + 2) + 1] = off32[b + 1] - off32[b];
+    // Host-known part of the header, the per-batch tables and the seeds go through a pinned staging block of the
+    // sample handle, so that the device work below reads nothing but fixed addresses: it can then be captured once
+    // in a CUDA graph and replayed for every later call with the same shape.
+    const size_t n_stage_ints = (sizeof(DenseHeader) + 3) / 4 + (size_t)(B + 1) + (size_t)B * (k + 2) + 2 * (size_t)B + 2;
+    if (d->h_stage_ints < n_stage_ints) {
+        if (d->h_stage) cudaFreeHost(d->h_stage);
+        d->h_stage = nullptr; d->h_stage_ints = 0;
+        if (cudaHostAlloc((void**)&d->h_stage, n_stage_ints * sizeof(int32_t), cudaHostAllocDefault) != cudaSuccess) {
+            cudaGetLastError();
+            return mg_fail(ctx, MG_ERR_OOM, "pinned host allocation failed");
+        }
+        d->h_stage_ints = n_stage_ints;
+    }
+    DenseHeader* st_hdr = reinterpret_cast<DenseHeader*>(d->h_stage);
+    int32_t* st_off = d->h_stage + (sizeof(DenseHeader) + 3) / 4;
+    int32_t* st_cum = st_off + (B + 1);
+    uint64_t* st_seeds = reinterpret_cast<uint64_t*>(d->h_stage + (((sizeof(DenseHeader) + 3) / 4 + (size_t)(B + 1) + (size_t)B * (k + 2) + 1) & ~(size_t)1));
+    memset(st_hdr, 0, sizeof(DenseHeader));
+    st_hdr->hop_base[0] = 0;
+    st_hdr->hop_base[1] = (int32_t)T;
+    memset(st_cum, 0, sizeof(int32_t) * (size_t)B * (k + 2));
+    for (int b = 0; b <= B; ++b) st_off[b] = (int32_t)target_offsets[b];
+    for (int b = 0; b < B; ++b) st_cum[(size_t)b * (k + 2) + 1] = st_off[b + 1] - st_off[b];
+    memcpy(st_seeds, seeds, sizeof(uint64_t) * B);
+
+    // the summary's landing place (mapped pinned memory)
+    const size_t n_ints = (sizeof(DenseHeader) + 3) / 4 + (size_t)B * (k + 2) + 2 * (size_t)(k + 1) * (B + 1) + (size_t)k * (B + 1);
+    if (d->h_pinned_ints < n_ints) {
+        if (d->h_pinned) cudaFreeHost(d->h_pinned);
+        d->h_pinned = nullptr; d->h_pinned_ints = 0;
+        if (cudaHostAlloc((void**)&d->h_pinned, n_ints * sizeof(int32_t), cudaHostAllocMapped) != cudaSuccess ||
+            cudaHostGetDevicePointer((void**)&d->h_pinned_dev, d->h_pinned, 0) != cudaSuccess) {
+            cudaGetLastError();
+            return mg_fail(ctx, MG_ERR_OOM, "pinned host allocation failed");
+        }
+        d->h_pinned_ints = n_ints;
+    }
+    sample_kernel_attributes();
+
+    // the targets are staged in newlist[1] (outside the graph: their source changes from call to call)
+    if (T > 0)
+        MG_CUDA(ctx, cudaMemcpyAsync(d->newlist[1], targets, sizeof(int32_t) * T,
+                                     targets_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, st));
+    const int32_t* tgt_dev = (const int32_t*)d->newlist[1];
+
+    // ---- everything the device does for this sample ----
+    auto enqueue = [&]() -> int {
     {
         ProfScope ps(ctx, PH_SAMPLE_INIT, 1);
-        MG_CUDA(ctx, cudaMemcpyAsync(d->hdr, &hh, sizeof(hh), cudaMemcpyHostToDevice, st));
-        MG_CUDA(ctx, cudaMemcpyAsync(d->node_off, off32.data(), sizeof(int32_t) * (B + 1), cudaMemcpyHostToDevice, st));
-        MG_CUDA(ctx, cudaMemcpyAsync(d->cum, cum0.data(), sizeof(int32_t) * cum0.size(), cudaMemcpyHostToDevice, st));
-        MG_CUDA(ctx, cudaMemcpyAsync(d->d_seeds, seeds, sizeof(uint64_t) * B, cudaMemcpyHostToDevice, st));
+        MG_CUDA(ctx, cudaMemcpyAsync(d->hdr, st_hdr, sizeof(DenseHeader), cudaMemcpyHostToDevice, st));
+        MG_CUDA(ctx, cudaMemcpyAsync(d->node_off, st_off, sizeof(int32_t) * (B + 1), cudaMemcpyHostToDevice, st));
+        MG_CUDA(ctx, cudaMemcpyAsync(d->cum, st_cum, sizeof(int32_t) * (size_t)B * (k + 2), cudaMemcpyHostToDevice, st));
+        MG_CUDA(ctx, cudaMemcpyAsync(d->d_seeds, st_seeds, sizeof(uint64_t) * B, cudaMemcpyHostToDevice, st));
         MG_CUDA(ctx, cudaMemsetAsync(d->hkeys, 0xFF, sizeof(int32_t) * (size_t)B * table_size, st));
-        // the targets are staged in newlist[1] when they come from the host
-        const int32_t* tgt_dev = targets;
-        if (!targets_on_device && T > 0) {
-            MG_CUDA(ctx, cudaMemcpyAsync(d->newlist[1], targets, sizeof(int32_t) * T, cudaMemcpyHostToDevice, st));
-            tgt_dev = (const int32_t*)d->newlist[1];
-        }
         if (T > 0) {
             k_init_targets<<<mg_grid(ctx, 4), kThreads, 0, st>>>(d->hdr, tgt_dev, (int32_t)T, d->node_off, B, d->nodes,
                                                                d->node_batch, d->hkeys, d->hvals, tg, ctx->n_nodes,
@@ -1134,7 +1177,6 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
             else if (f <= 32) k_pick<32><<<grid, kThreads, 0, st>>>(a);
             else {
                 const size_t wide_smem = (size_t)(kThreads / 32) * 2 * f * sizeof(uint32_t);   // 64 KiB at the largest fanout
-                MG_CUDA(ctx, cudaFuncSetAttribute(k_pick_wide, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)wide_smem));
                 k_pick_wide<<<grid, kThreads, wide_smem, st>>>(a);
             }
             InsertArgs ia{d->hdr, h, d->ent_nbrs, d->ent_repr, d->hkeys, tg, d->newlist[0], d->cap_nodes, id_bits,
@@ -1183,26 +1225,53 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
         k_finalize<<<1, 1024, 0, st>>>(d->hdr, B, k, d->cum, d->node_off, d->ent_off, d->rowbase, d->d_ent_hop);
         ctx->launches++;
     }
-    MG_CUDA(ctx, cudaGetLastError());
-
     // the summary goes to pinned host memory behind the kernels; mg_sample_many_end waits for it
-    {
-        const size_t n_ints = (sizeof(DenseHeader) + 3) / 4 + (size_t)B * (k + 2) + 2 * (size_t)(k + 1) * (B + 1) + (size_t)k * (B + 1);
-        if (d->h_pinned_ints < n_ints) {
-            if (d->h_pinned) cudaFreeHost(d->h_pinned);
-            d->h_pinned = nullptr; d->h_pinned_ints = 0;
-            if (cudaHostAlloc((void**)&d->h_pinned, n_ints * sizeof(int32_t), cudaHostAllocMapped) != cudaSuccess ||
-                cudaHostGetDevicePointer((void**)&d->h_pinned_dev, d->h_pinned, 0) != cudaSuccess) {
+    static_assert(sizeof(DenseHeader) % 4 == 0, "the header is copied as 32-bit words");
+    k_summary<<<8, kThreads, 0, st>>>(d->hdr, d->cum, d->node_off, d->rowbase, d->d_ent_hop, (int32_t)((sizeof(DenseHeader) + 3) / 4),
+                                     B * (k + 2), (k + 1) * (B + 1), k * (B + 1), d->h_pinned_dev);
+    ctx->launches++;
+    MG_CUDA(ctx, cudaGetLastError());
+    return MG_OK;
+    };   // enqueue
+
+    // Replay the captured graph when nothing that the device work depends on has changed since it was captured;
+    // capture it (again) otherwise.  Profiling runs the launches one by one (its events do not belong in a graph).
+    SampleSignature sig;
+    memset(&sig, 0, sizeof(sig));
+    sig.B = B; sig.k = k; sig.T = T; sig.table_size = table_size; sig.cap_batch = cap_batch;
+    sig.cap_nodes = d->cap_nodes; sig.cap_entries = d->cap_entries; sig.n_nodes = ctx->n_nodes; sig.part_size = ctx->part_size;
+    for (int h = 0; h < k; ++h) sig.fanouts[h] = fanouts[h];
+    const void* ptrs[] = {d->hdr, d->nodes, d->node_batch, d->ent_off, d->node_r0, d->node_deg, d->newlist[0], d->newlist[1],
+                          d->scan_tmp, d->sort_hist, d->ent_nbrs, d->ent_repr, d->hkeys, d->hvals, d->node_off, d->cum, d->rowbase,
+                          d->d_ent_hop, d->d_seeds, d->h_stage, d->h_pinned_dev, ctx->view_off, ctx->view_nbrs, ctx->d_slot_of_part, st};
+    static_assert(sizeof(ptrs) <= sizeof(sig.ptrs), "signature too small");
+    memcpy(sig.ptrs, ptrs, sizeof(ptrs));
+    const bool use_graph = ctx->sample_graphs && !ctx->prof_on && !getenv("MG_NO_SAMPLE_GRAPH");
+    if (use_graph) {
+        if (!d->graph_exec || memcmp(&sig, &d->graph_sig, sizeof(sig)) != 0) {
+            if (d->graph_exec) { cudaGraphExecDestroy(d->graph_exec); d->graph_exec = nullptr; }
+            const int64_t launches0 = ctx->launches;
+            MG_CUDA(ctx, cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+            const int erc = enqueue();
+            cudaGraph_t graph = nullptr;
+            const cudaError_t ce = cudaStreamEndCapture(st, &graph);
+            d->graph_launches = ctx->launches - launches0;
+            ctx->launches = launches0;
+            if (erc || ce != cudaSuccess || !graph) {
+                if (graph) cudaGraphDestroy(graph);
                 cudaGetLastError();
-                return mg_fail(ctx, MG_ERR_OOM, "pinned host allocation failed");
+                return erc ? erc : mg_fail(ctx, MG_ERR_CUDA, "capture of the sampler failed: %s", cudaGetErrorString(ce));
             }
-            d->h_pinned_ints = n_ints;
+            const cudaError_t ie = cudaGraphInstantiate(&d->graph_exec, graph, 0);
+            cudaGraphDestroy(graph);
+            if (ie != cudaSuccess) { d->graph_exec = nullptr; cudaGetLastError(); return mg_fail(ctx, MG_ERR_CUDA, "cudaGraphInstantiate: %s", cudaGetErrorString(ie)); }
+            d->graph_sig = sig;
         }
-        static_assert(sizeof(DenseHeader) % 4 == 0, "the header is copied as 32-bit words");
-        k_summary<<<8, kThreads, 0, st>>>(d->hdr, d->cum, d->node_off, d->rowbase, d->d_ent_hop, (int32_t)((sizeof(DenseHeader) + 3) / 4),
-                                         B * (k + 2), (k + 1) * (B + 1), k * (B + 1), d->h_pinned_dev);
-        ctx->launches++;
-        MG_CUDA(ctx, cudaGetLastError());
+        MG_CUDA(ctx, cudaGraphLaunch(d->graph_exec, st));
+        ctx->launches += d->graph_launches;
+    } else {
+        const int erc = enqueue();
+        if (erc) return erc;
     }
     if (!d->ev_sampled) MG_CUDA(ctx, cudaEventCreateWithFlags(&d->ev_sampled, cudaEventDisableTiming));
     MG_CUDA(ctx, cudaEventRecord(d->ev_sampled, st));
@@ -1331,6 +1400,8 @@ extern "C" int mg_dense_free(mg_dense* d) {
     cudaFree(d->newlist[1]); cudaFree(d->d_seeds); cudaFree(d->scan_tmp); cudaFree(d->sort_hist);
     cudaFree(d->exp_buf); cudaFree(d->d_ent_hop);
     if (d->h_pinned) cudaFreeHost(d->h_pinned);
+    if (d->h_stage) cudaFreeHost(d->h_stage);
+    if (d->graph_exec) cudaGraphExecDestroy(d->graph_exec);
     if (d->ev_sampled) cudaEventDestroy(d->ev_sampled);
     if (d->ev_read_done) cudaEventDestroy(d->ev_read_done);
     delete d;

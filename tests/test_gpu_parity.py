@@ -631,3 +631,21 @@ def test_extremes_largest_fanout_deepest_sample_all_nodes_empty_call():
     d = ctx.sample(torch.empty(0, dtype=torch.int32), [3], seed=0)
     v = d.view(0)
     assert v.node_ids.numel() == 0 and v.nbrs.numel() == 0 and v.node_id_offsets.cpu().tolist() == [0, 0, 0]
+
+
+def test_sample_handle_reuse_replays_and_recaptures(tiny):
+    """The sampler's device work is captured in a CUDA graph per sample handle and replayed while the call's shape
+    stays the same; targets, seeds and offsets of every call still take effect, and a new shape is captured anew."""
+    g, feats = tiny
+    ctx = make_ctx(g, feats)
+    view = oracle_view(g)
+    d = None
+    for step, (fanouts, n) in enumerate([([6, 3], 200), ([6, 3], 200), ([6, 3], 200), ([4, 2, 2], 200), ([6, 3], 150)]):
+        targets = inputs.distinct_targets(10_000, n, seed=40 + step)
+        tg = targets.cuda() if step % 2 else targets
+        offs = np.array([0, n // 2, n], dtype=np.int64)
+        seeds = [7 * step + 1, 7 * step + 2]
+        d = ctx.sample_many(tg, offs, fanouts, seeds, out=d)
+        for b in range(2):
+            ref = O.sample_dense(view, targets[offs[b]:offs[b + 1]].tolist(), fanouts, seeds[b])
+            assert_dense_equal(d.view(b), ref)
