@@ -186,11 +186,10 @@ int mg_dense_counts(const mg_dense* d, int32_t* n_batches, int32_t* k, int64_t* 
                     int64_t* entries_per_hop);
 
 /* Materialise batch `batch` in the paper's array layout (Section 4.1 plus repr_map,
- * Section 4.2) into a device buffer owned by `d`.  Ids inside a delta ascend.  The sampler keeps the outermost
- * delta (the last hop's new nodes) in discovery order, since nothing on the sample / forward path depends on its
- * order; the first mg_dense_view or mg_gather_h0 on a sample sorts it and re-labels the repr_map entries that
- * point into it (all mini-batches at once; later calls find it done).  mg_forward gives the same H^k, bit for
- * bit, before and after. */
+ * Section 4.2) into a device buffer owned by `d`.  Ids inside a delta ascend; targets keep the caller's order.
+ * On the device a delta is kept in the order in which its nodes were found (nothing on the sample / forward path
+ * depends on that order); this call, mg_gather_h0 and mg_layer_output sort the mini-batch's ids (one radix sort per
+ * call, on the context's stream, synchronous) and translate rows and repr_map entries. */
 int mg_dense_view(mg_ctx* ctx, mg_dense* d, int32_t batch, mg_dense_arrays* out);
 
 int mg_dense_free(mg_dense* d);

@@ -224,6 +224,7 @@ struct RowExportArgs {
     int32_t nio[MG_MAX_HOPS + 2];    // canonical offsets of the deltas of this batch
     int32_t cum[MG_MAX_HOPS + 2];
     int32_t dim;
+    const int32_t* perm;             // local row of every canonical row of the mini-batch (mg_dense_batch_perm)
 };
 
 // out[c, :] = src[local(c), :] where c runs over the paper's row order
@@ -233,9 +234,7 @@ __global__ void __launch_bounds__(kThreads) k_export_rows(RowExportArgs a, const
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
         const int32_t c = (int32_t)(i / vec) + a.nio[a.first_delta];
         const int q = (int)(i % vec);
-        int j = a.first_delta;
-        while (j < a.k && c >= a.nio[j + 1]) ++j;
-        const int32_t l = a.cum[a.k - j] + (c - a.nio[j]);
+        const int32_t l = a.perm[c];
         reinterpret_cast<float4*>(out)[i] = reinterpret_cast<const float4*>(src + (int64_t)l * a.dim)[q];
     }
 }
@@ -258,10 +257,10 @@ __global__ void __launch_bounds__(kThreads) k_gather_h0(H0Args a, float* __restr
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
         const int32_t c = (int32_t)(i / n_chunks);
         const int q = (int)(i % n_chunks);
-        int j = 0;
-        while (j < a.r.k && c >= a.r.nio[j + 1]) ++j;
-        const int h = a.r.k - j;
-        const int32_t node = a.nodes[a.node_off[h] + (c - a.r.nio[j])];
+        const int32_t l = a.r.perm[c];
+        int h = 0;
+        while (h < a.r.k && l >= a.r.cum[h + 1]) ++h;
+        const int32_t node = a.nodes[a.node_off[h] + (l - a.r.cum[h])];
         const uint32_t p = (uint32_t)node / a.part_size;
         const char* row = a.slots + (int64_t)a.slot_of_part[p] * a.slot_bytes + (int64_t)((uint32_t)node - p * a.part_size) * a.row_bytes;
         C v;
@@ -611,12 +610,13 @@ extern "C" int mg_gather_h0(mg_ctx* ctx, mg_dense* d, int32_t batch, float* out_
     if (!ctx->slots || ctx->feat_dim <= 0) return mg_fail(ctx, MG_ERR_STATE, "no feature table loaded");
     if (batch < 0 || batch >= d->n_batches) return mg_fail(ctx, MG_ERR_ARG, "batch out of range");
     MG_CUDA(ctx, cudaSetDevice(ctx->device));
-    {
-        const int rc0 = mg_dense_canonicalize(ctx, d);   // rows come in the paper's order
-        if (rc0) return rc0;
-    }
     H0Args a;
     fill_row_export(d, batch, 0, ctx->feat_dim, &a.r);
+    {
+        const int32_t* inv_unused;
+        const int rc0 = mg_dense_batch_perm(ctx, d, batch, &a.r.perm, &inv_unused);   // rows come in the paper's order
+        if (rc0) return rc0;
+    }
     for (int h = 0; h <= d->k; ++h) a.node_off[h] = d->h_node_off[(size_t)h * (d->n_batches + 1) + batch];
     a.nodes = d->nodes; a.slots = ctx->slots; a.slot_of_part = ctx->d_slot_of_part;
     a.slot_bytes = ctx->slot_bytes; a.row_bytes = ctx->row_bytes; a.part_size = (uint32_t)ctx->part_size;
@@ -648,6 +648,10 @@ extern "C" int mg_layer_output(mg_ctx* ctx, const mg_model* m, mg_dense* d, int3
     const float* src = layer_base + (size_t)d->h_rowbase[(size_t)layer * (B + 1) + batch] * m->dims[layer];
     RowExportArgs r;
     fill_row_export(d, batch, layer, m->dims[layer], &r);
+    {
+        const int32_t* inv_unused;
+        if ((rc = mg_dense_batch_perm(ctx, d, batch, &r.perm, &inv_unused))) return rc;
+    }
     if (r.n_rows > 0) {
         k_export_rows<<<mg_grid(ctx, 4), kThreads, 0, ctx->stream>>>(r, src, out_dev);
         ctx->launches++;

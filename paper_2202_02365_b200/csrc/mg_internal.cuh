@@ -178,7 +178,9 @@ struct mg_dense {
     std::vector<int32_t> h_ent_hop;  // [k * (B+1)] arena entry index where batch b's hop-h entries start
     int32_t* d_ent_hop = nullptr;    // device copy of the same
     bool valid = false;
-    bool canonical = false;          // the outermost delta has been put in ascending id order (mg_dense_canonicalize)
+    int32_t* perm_buf = nullptr; size_t perm_elems = 0;   // perm | inv of mini-batch perm_batch (mg_dense_batch_perm)
+    int perm_batch = -1;
+    uint32_t* batch_cnt = nullptr;   // [k][B] new nodes per hop and mini-batch
     // asynchronous sampling: the summary lands in pinned memory, ev_sampled marks its arrival
     int32_t* h_pinned = nullptr; size_t h_pinned_ints = 0;
     int32_t* h_pinned_dev = nullptr; // the same memory as the device sees it
@@ -265,9 +267,10 @@ struct SortParams {   // device-resident
 };
 size_t mg_sort_hist_elems(int64_t max_keys);
 void mg_sort_params_host(SortParams* sp, int64_t n);
-// Puts the outermost delta of every mini-batch in ascending id order (the sampler leaves it in discovery order) and
-// re-labels the entries that point into it; idempotent, on ctx->stream, off the hot path.
-int mg_dense_canonicalize(mg_ctx* ctx, mg_dense* d);
+// The device keeps every delta in discovery order; exports go through a permutation of the mini-batch's local rows
+// (perm[c] = local row of canonical row c: deltas in the paper's order, ids ascending inside a delta, targets in the
+// caller's order; inv = its inverse).  Device arrays owned by d; on ctx->stream, synchronous, off the hot path.
+int mg_dense_batch_perm(mg_ctx* ctx, mg_dense* d, int b, const int32_t** perm, const int32_t** inv);
 size_t mg_scan_tmp_elems(int64_t max_elems);
 void mg_sort_u64(mg_ctx* ctx, uint64_t* const buf[2], const SortParams* sp, int lo_bit, int bits, uint32_t* hist,
                  uint32_t* scan_tmp, int* res_buf);

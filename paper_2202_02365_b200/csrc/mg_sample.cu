@@ -345,12 +345,12 @@ struct InsertArgs {
 constexpr int kInsertPerThread = 8;
 constexpr int kInsertSpan = 16;   // mini-batches a block's chunk of entries may touch on the fast path
 
-// OUTER = the last sampling round.  Its new nodes are not sorted (nothing depends on their order, see
-// mg_dense_canonicalize): a new node takes the next free row of its mini-batch right here -- a count per
-// mini-batch in shared memory, one global atomic per (block, mini-batch) -- its table value is written at once, and
-// the list entry carries (mini-batch, id, rank) instead of (mini-batch, id, table slot).
-template <bool OUTER>
+// New nodes are not sorted on the device: nothing the path computes depends on the order of ids inside a delta (the
+// paper's arrays, with ascending ids, are an export: mg_dense_batch_perm).  A new node takes the next free row of its
+// mini-batch right here -- a count per mini-batch in shared memory, one global atomic per (block, mini-batch) --,
+// its table value is written at once, and its list entry carries (mini-batch, id, rank in the hop).
 __global__ void __launch_bounds__(kThreads) k_insert(InsertArgs a) {
+    constexpr bool OUTER = true;
     __shared__ uint32_t warp_tot[kThreads / 32 + 1];
     __shared__ uint32_t block_base;
     __shared__ uint32_t span_cnt[kInsertSpan], span_base[kInsertSpan];
@@ -429,7 +429,7 @@ __global__ void __launch_bounds__(kThreads) k_insert(InsertArgs a) {
                 if (new_bits & (1u << j)) {
                     const int32_t bb = b[j] - b0;
                     if (bb < kInsertSpan) rank[j] += span_base[bb];
-                    const int64_t row = (int64_t)a.cum[b[j] * (a.k + 2) + a.k] + rank[j];
+                    const int64_t row = (int64_t)a.cum[b[j] * (a.k + 2) + a.hop + 1] + rank[j];
                     if (row < a.max_nodes_per_batch) a.hvals[(int64_t)b[j] * a.tg.size + slot[j]] = (int32_t)row;
                     else atomicOr(&a.hdr->status, ST_CAP_TABLE);
                 }
@@ -456,13 +456,6 @@ constexpr int kRadixBits = 9;                              // 34 key bits (27 id
 constexpr int kBins = 1 << kRadixBits;
 constexpr int kBinsPerThread = kBins / kThreads;
 
-__global__ void k_sort_setup(const DenseHeader* hdr, SortParams* sp) {
-    const int32_t n = hdr->status ? 0 : (int32_t)hdr->n_new;
-    sp->zero = 0;
-    sp->n = n;
-    sp->ntiles = (n + kSortTile - 1) / kSortTile;
-    sp->hist_len = kBins * sp->ntiles;
-}
 
 __global__ void __launch_bounds__(kThreads)
 k_radix_hist(const uint64_t* __restrict__ keys, const SortParams* sp, int shift, uint32_t* hist) {
@@ -588,44 +581,6 @@ __global__ void k_hop_advance(DenseHeader* hdr, int hop, int32_t B, int32_t* nod
 }
 
 __global__ void __launch_bounds__(kThreads)
-k_place_nodes(const DenseHeader* hdr, int hop, int32_t B, const uint64_t* __restrict__ sorted, int id_bits,
-              int32_t* nodes, int32_t* node_batch, int32_t* node_off_next) {
-    if (hdr->status) return;
-    const int32_t n = (int32_t)hdr->n_new, start = hdr->hop_base[hop + 1];
-    const uint64_t id_mask = (1ull << id_bits) - 1ull;
-    for (int32_t j = blockIdx.x * blockDim.x + threadIdx.x; j < n; j += gridDim.x * blockDim.x) {
-        const uint64_t key = sorted[j];
-        const int32_t b = (int32_t)(key >> (MG_SLOT_BITS + id_bits));
-        nodes[start + j] = (int32_t)((key >> MG_SLOT_BITS) & id_mask);
-        node_batch[start + j] = b;
-        const int32_t prev_b = j == 0 ? -1 : (int32_t)(sorted[j - 1] >> (MG_SLOT_BITS + id_bits));
-        for (int bb = prev_b + 1; bb <= b; ++bb) node_off_next[bb] = start + j;
-        if (j == n - 1)
-            for (int bb = b + 1; bb <= B; ++bb) node_off_next[bb] = start + n;
-    }
-}
-
-__global__ void __launch_bounds__(kThreads)
-k_place_rows(DenseHeader* hdr, int hop, int32_t B, int32_t k, const uint64_t* __restrict__ sorted, int id_bits,
-             const int32_t* __restrict__ node_off_next, int32_t* cum, int32_t* hvals, TableGeom tg,
-             int32_t max_nodes_per_batch) {
-    if (hdr->status) return;
-    const int32_t n = (int32_t)hdr->n_new, start = hdr->hop_base[hop + 1];
-    const int32_t tid = blockIdx.x * blockDim.x + threadIdx.x;
-    for (int32_t j = tid; j < n; j += gridDim.x * blockDim.x) {
-        const uint64_t key = sorted[j];
-        const int32_t b = (int32_t)(key >> (MG_SLOT_BITS + id_bits));
-        const int32_t slot = (int32_t)(key & ((1u << MG_SLOT_BITS) - 1u));
-        hvals[(int64_t)b * tg.size + slot] = cum[b * (k + 2) + hop + 1] + (start + j - node_off_next[b]);
-    }
-    for (int32_t b = tid; b < B; b += gridDim.x * blockDim.x) {
-        const int32_t v = cum[b * (k + 2) + hop + 1] + (node_off_next[b + 1] - node_off_next[b]);
-        cum[b * (k + 2) + hop + 2] = v;
-        if (v > max_nodes_per_batch) atomicOr(&hdr->status, ST_CAP_TABLE);
-    }
-}
-
-__global__ void __launch_bounds__(kThreads)
 k_relabel(const DenseHeader* hdr, int hop, const int32_t* __restrict__ hvals, int32_t* ent_repr) {
     if (hdr->status) return;
     const int32_t lo = hdr->ent_base[hop], hi = hdr->ent_base[hop + 1];
@@ -741,80 +696,103 @@ k_summary(const DenseHeader* hdr, const int32_t* __restrict__ cum, const int32_t
 }
 
 // -------------------------------------------------------------------------------------
-// ascending id order for the outermost delta (on demand)
-// -------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads)
-k_canon_keys(const int32_t* __restrict__ nodes, const int32_t* __restrict__ node_batch, const int32_t* __restrict__ node_off_k,
-             int32_t start, int32_t n, int id_bits, uint64_t* keys) {
-    for (int32_t j = blockIdx.x * blockDim.x + threadIdx.x; j < n; j += gridDim.x * blockDim.x) {
-        const int32_t b = node_batch[start + j];
-        const uint64_t local = (uint64_t)(start + j - node_off_k[b]);   // position inside the mini-batch's delta
-        keys[j] = ((uint64_t)b << (MG_SLOT_BITS + id_bits)) | ((uint64_t)(uint32_t)nodes[start + j] << MG_SLOT_BITS) | local;
-    }
-}
-
-// sorted position p of the hop -> the node id goes to its place, and the old position learns its new one
-__global__ void __launch_bounds__(kThreads)
-k_canon_place(const uint64_t* __restrict__ sorted, const int32_t* __restrict__ node_off_k, int32_t start, int32_t n, int id_bits,
-              int32_t* nodes, int32_t* new_local) {
-    const uint64_t id_mask = (1ull << id_bits) - 1ull;
-    for (int32_t p = blockIdx.x * blockDim.x + threadIdx.x; p < n; p += gridDim.x * blockDim.x) {
-        const uint64_t key = sorted[p];
-        const int32_t b = (int32_t)(key >> (MG_SLOT_BITS + id_bits));
-        const int32_t old_local = (int32_t)(key & ((1u << MG_SLOT_BITS) - 1u));
-        nodes[start + p] = (int32_t)((key >> MG_SLOT_BITS) & id_mask);
-        new_local[node_off_k[b] - start + old_local] = start + p - node_off_k[b];
-    }
-}
-
-// entries of the last sampling round that point into the outermost delta follow their node
-__global__ void __launch_bounds__(kThreads)
-k_canon_relabel(int32_t e_lo, int32_t e_hi, const int32_t* __restrict__ ent_hop_last, int32_t B, int32_t k,
-                const int32_t* __restrict__ cum, const int32_t* __restrict__ node_off_k, int32_t start,
-                const int32_t* __restrict__ new_local, int32_t* ent_repr) {
-    for (int32_t e = e_lo + blockIdx.x * blockDim.x + threadIdx.x; e < e_hi; e += gridDim.x * blockDim.x) {
-        const int b = upper_segment(ent_hop_last, B + 1, e);
-        const int32_t base = cum[b * (k + 2) + k];      // first local row of the outermost delta in this mini-batch
-        const int32_t l = ent_repr[e];
-        if (l >= base) ent_repr[e] = base + new_local[node_off_k[b] - start + (l - base)];
-    }
-}
-
-// -------------------------------------------------------------------------------------
 // export to the paper's layout (mg_dense_view)
 // -------------------------------------------------------------------------------------
+// The device keeps every delta in discovery order.  The paper's arrays list the ids of a delta in ascending order
+// (targets in the caller's order), so an export goes through a permutation of the mini-batch's local rows:
+// perm[c] = local row of canonical row c, inv[l] = canonical row of local row l.
+struct BatchGeom {
+    int32_t k, V, n_targets;
+    int32_t cum[MG_MAX_HOPS + 2];      // local row base per hop
+    int32_t node_off[MG_MAX_HOPS + 1]; // first node of the mini-batch's run in each hop
+};
+
+__device__ __forceinline__ int hop_of_row(const BatchGeom& g, int32_t l) {
+    int h = 0;
+    while (h < g.k && l >= g.cum[h + 1]) ++h;
+    return h;
+}
+
+// keys (canonical delta, id, local row) of the rows of hops >= 1
+__global__ void __launch_bounds__(kThreads)
+k_perm_keys(BatchGeom g, const int32_t* __restrict__ nodes, int id_bits, uint64_t* keys) {
+    const int32_t n = g.V - g.n_targets;
+    for (int32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        const int32_t l = g.n_targets + i;
+        const int h = hop_of_row(g, l);
+        const int32_t id = nodes[g.node_off[h] + (l - g.cum[h])];
+        keys[i] = ((uint64_t)(g.k - h) << (MG_SLOT_BITS + id_bits)) | ((uint64_t)(uint32_t)id << MG_SLOT_BITS) | (uint64_t)l;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_perm_fill(BatchGeom g, const uint64_t* __restrict__ sorted, int32_t* perm, int32_t* inv) {
+    const int32_t n = g.V - g.n_targets;
+    for (int32_t c = blockIdx.x * blockDim.x + threadIdx.x; c < g.V; c += gridDim.x * blockDim.x) {
+        // deltas k-1 .. 0 (hops >= 1) come first in the sorted keys; the targets keep the caller's order at the end
+        const int32_t l = c < n ? (int32_t)(sorted[c] & ((1u << MG_SLOT_BITS) - 1u)) : c - n;
+        perm[c] = l;
+        inv[l] = c;
+    }
+}
+
 struct ExportArgs {
-    int32_t k, b, B;
-    int32_t V, n0, E;
+    BatchGeom g;
+    int32_t n0;                       // |Delta_0|: canonical rows below n0 have no sampled neighbours
     int32_t nio[MG_MAX_HOPS + 2];     // canonical node_id_offsets
-    int32_t ebase[MG_MAX_HOPS + 1];   // canonical first entry of Delta_j's neighbours, j = 1..k
-    int32_t cum[MG_MAX_HOPS + 2];     // local row base per hop
-    int32_t node_off[MG_MAX_HOPS + 1];
-    int32_t ent_hop[MG_MAX_HOPS + 1];
-    const int32_t *nodes, *ent_off, *ent_nbrs, *ent_repr;
+    const int32_t *nodes, *ent_off, *ent_nbrs, *ent_repr, *perm, *inv;
     int32_t *o_node_ids, *o_nio, *o_nbrs, *o_nbr_off, *o_repr;
 };
 
-__global__ void __launch_bounds__(kThreads) k_export(ExportArgs a) {
+// node ids in canonical order; the sampled nodes' entry counts go to o_nbr_off (scanned next)
+__global__ void __launch_bounds__(kThreads) k_export_nodes(ExportArgs a) {
     const int32_t tid = blockIdx.x * blockDim.x + threadIdx.x;
-    if (tid <= a.k + 1) a.o_nio[tid] = a.nio[tid];
-    if (tid == 0) a.o_nbr_off[a.V - a.n0] = a.E;
-    for (int32_t c = tid; c < a.V; c += gridDim.x * blockDim.x) {
-        int j = 0;
-        while (j < a.k && c >= a.nio[j + 1]) ++j;
-        const int h = a.k - j;
-        const int32_t idx = a.node_off[h] + (c - a.nio[j]);
+    if (tid <= a.g.k + 1) a.o_nio[tid] = a.nio[tid];
+    for (int32_t c = tid; c < a.g.V; c += gridDim.x * blockDim.x) {
+        const int32_t l = a.perm[c];
+        const int h = hop_of_row(a.g, l);
+        const int32_t idx = a.g.node_off[h] + (l - a.g.cum[h]);
         a.o_node_ids[c] = a.nodes[idx];
-        if (j == 0) continue;
+        if (c >= a.n0) a.o_nbr_off[c - a.n0] = a.ent_off[idx + 1] - a.ent_off[idx];
+    }
+}
+
+// in-place exclusive scan of data[0, n), total to data[n] (one block)
+__global__ void __launch_bounds__(1024) k_export_scan(int32_t* data, int32_t n) {
+    __shared__ uint32_t warp_tot[33];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t carry = 0;
+    for (int s0 = 0; s0 < n; s0 += 1024) {
+        const int i = s0 + threadIdx.x;
+        const uint32_t v = i < n ? (uint32_t)data[i] : 0u;
+        const uint32_t inc = warp_incl_scan(v);
+        if (lane == 31) warp_tot[warp] = inc;
+        __syncthreads();
+        if (warp == 0) {
+            const uint32_t w = warp_tot[lane];
+            const uint32_t wi = warp_incl_scan(w);
+            warp_tot[lane] = wi - w;
+            if (lane == 31) warp_tot[32] = wi;
+        }
+        __syncthreads();
+        if (i < n) data[i] = (int32_t)(carry + warp_tot[warp] + inc - v);
+        carry += warp_tot[32];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) data[n] = (int32_t)carry;
+}
+
+// nbrs and repr_map: the entries of canonical node c start at o_nbr_off[c - n0]
+__global__ void __launch_bounds__(kThreads) k_export_entries(ExportArgs a) {
+    for (int32_t c = a.n0 + blockIdx.x * blockDim.x + threadIdx.x; c < a.g.V; c += gridDim.x * blockDim.x) {
+        const int32_t l = a.perm[c];
+        const int h = hop_of_row(a.g, l);
+        const int32_t idx = a.g.node_off[h] + (l - a.g.cum[h]);
         const int32_t e0 = a.ent_off[idx], e1 = a.ent_off[idx + 1];
-        const int32_t o0 = a.ebase[j] + (e0 - a.ent_hop[h]);
-        a.o_nbr_off[c - a.n0] = o0;
+        const int32_t o0 = a.o_nbr_off[c - a.n0];
         for (int32_t e = e0; e < e1; ++e) {
             a.o_nbrs[o0 + (e - e0)] = a.ent_nbrs[e];
-            const int32_t l = a.ent_repr[e];
-            int hh = 0;
-            while (hh < a.k && l >= a.cum[hh + 1]) ++hh;
-            a.o_repr[o0 + (e - e0)] = a.nio[a.k - hh] + (l - a.cum[hh]);
+            a.o_repr[o0 + (e - e0)] = a.inv[a.ent_repr[e]];
         }
     }
 }
@@ -932,6 +910,7 @@ static int dense_alloc(mg_ctx* ctx, mg_dense* d, int32_t B, int32_t k, int64_t c
         if ((rc = dev_realloc(ctx, &d->rowbase, (size_t)need_b))) return rc;
         if ((rc = dev_realloc(ctx, &d->d_ent_hop, (size_t)need_b))) return rc;
         if ((rc = dev_realloc(ctx, &d->d_seeds, (size_t)need_b))) return rc;
+        if ((rc = dev_realloc(ctx, &d->batch_cnt, (size_t)need_b))) return rc;
         d->alloc_batches = need_b;
     }
     d->k = k;
@@ -994,7 +973,7 @@ extern "C" int mg_sample_many_end(mg_ctx* ctx, mg_dense* d) {
     d->h_ent_hop.assign(p, p + (size_t)k * (B + 1));
     if (d->h_hdr.status) return mg_fail(ctx, status_code(d->h_hdr.status), "%s", status_text(d->h_hdr.status));
     d->valid = true;
-    d->canonical = d->k == 0;
+    d->perm_batch = -1;
     return MG_OK;
 }
 
@@ -1149,10 +1128,9 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
         }
     }
 
-    SortParams* sp = (SortParams*)(d->scan_tmp + d->scan_tmp_elems - 8);  // tail of the scratch block
-    // new nodes of the outermost hop per mini-batch: the unused last block of the row-base array
-    uint32_t* batch_cnt = reinterpret_cast<uint32_t*>(d->rowbase + (size_t)(MG_MAX_HOPS + 1) * (B + 1));
-    MG_CUDA(ctx, cudaMemsetAsync(batch_cnt, 0, sizeof(uint32_t) * B, st));
+    // new nodes per (hop, mini-batch)
+    uint32_t* batch_cnt = d->batch_cnt;
+    MG_CUDA(ctx, cudaMemsetAsync(batch_cnt, 0, sizeof(uint32_t) * (size_t)k * B, st));
     uint32_t* scan_total = (uint32_t*)(d->scan_tmp + d->scan_tmp_elems - 4);
     const int grid = mg_grid(ctx, 8);
     for (int h = 0; h < k; ++h) {
@@ -1180,42 +1158,22 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
                 k_pick_wide<<<grid, kThreads, wide_smem, st>>>(a);
             }
             InsertArgs ia{d->hdr, h, d->ent_nbrs, d->ent_repr, d->hkeys, tg, d->newlist[0], d->cap_nodes, id_bits,
-                          k, d->cum, d->hvals, batch_cnt, (int32_t)cap_batch};
+                          k, d->cum, d->hvals, batch_cnt + (size_t)h * B, (int32_t)cap_batch};
             // many short blocks: measured on the bench's last hop, 0.94 ms at 32 blocks per SM against 1.08 ms at 8
             // (blocks past the end of the entries return at once)
             const int igrid = mg_grid(ctx, 32);
-            if (h == k - 1) k_insert<true><<<igrid, kThreads, 0, st>>>(ia);
-            else k_insert<false><<<igrid, kThreads, 0, st>>>(ia);
+            k_insert<<<igrid, kThreads, 0, st>>>(ia);
             ctx->launches++;
         }
-        if (h == k - 1) {
-            // The outermost delta: rows were handed out at insert time, in discovery order (nothing on the path
-            // depends on the order of its ids; mg_dense_canonicalize sorts it on demand).  No sort, no table pass.
+        {
+            // rows were handed out at insert time, in discovery order: per-batch counts -> offsets, then every list
+            // entry (mini-batch, id, rank) goes to its place.  No sort, no second pass over the id tables.
             ProfScope ps(ctx, PH_SAMPLE_PLACE, 3);
             int32_t* off_next = d->node_off + (size_t)(h + 1) * (B + 1);
             k_hop_advance<<<1, 256, 0, st>>>(d->hdr, h, B, off_next, d->cap_nodes);
-            k_outer_offsets<<<1, 1024, 0, st>>>(d->hdr, h, B, k, batch_cnt, off_next, d->cum, (int32_t)cap_batch);
+            k_outer_offsets<<<1, 1024, 0, st>>>(d->hdr, h, B, k, batch_cnt + (size_t)h * B, off_next, d->cum, (int32_t)cap_batch);
             k_place_nodes_outer<<<grid, kThreads, 0, st>>>(d->hdr, d->newlist[0], id_bits, off_next, d->nodes, d->node_batch);
             ctx->launches += 3;
-        } else {
-            int res_buf = 0;
-            {
-                // inner deltas are sorted by (mini-batch, id): ascending ids inside a mini-batch
-                const int key_bits = id_bits + b_bits;
-                const int passes = (key_bits + kRadixBits - 1) / kRadixBits;
-                ProfScope ps(ctx, PH_SAMPLE_SORT, 1 + passes * 5);
-                k_sort_setup<<<1, 1, 0, st>>>(d->hdr, sp);
-                mg_sort_u64(ctx, d->newlist, sp, MG_SLOT_BITS, key_bits, d->sort_hist, (uint32_t*)d->scan_tmp, &res_buf);
-            }
-            {
-                ProfScope ps(ctx, PH_SAMPLE_PLACE, 3);
-                int32_t* off_next = d->node_off + (size_t)(h + 1) * (B + 1);
-                k_hop_advance<<<1, 256, 0, st>>>(d->hdr, h, B, off_next, d->cap_nodes);
-                k_place_nodes<<<grid, kThreads, 0, st>>>(d->hdr, h, B, d->newlist[res_buf], id_bits, d->nodes, d->node_batch, off_next);
-                k_place_rows<<<grid, kThreads, 0, st>>>(d->hdr, h, B, k, d->newlist[res_buf], id_bits, off_next, d->cum, d->hvals, tg,
-                                                        (int32_t)cap_batch);
-            }
-            ctx->launches += 1 + 3;   // sort_setup, place x3
         }
         {
             ProfScope ps(ctx, PH_SAMPLE_RELABEL, 1);
@@ -1309,32 +1267,47 @@ extern "C" int mg_dense_counts(const mg_dense* d, int32_t* n_batches, int32_t* k
 }
 
 
-int mg_dense_canonicalize(mg_ctx* ctx, mg_dense* d) {
-    if (d->canonical) return MG_OK;
+static void batch_geom(const mg_dense* d, int b, BatchGeom* g) {
     const int k = d->k, B = d->n_batches;
-    const int32_t start = d->h_hdr.hop_base[k], n = d->h_hdr.hop_base[k + 1] - start;
-    if (k == 0 || n <= 0) { d->canonical = true; return MG_OK; }
+    memset(g, 0, sizeof(*g));
+    g->k = k;
+    for (int h = 0; h <= k + 1; ++h) g->cum[h] = d->h_cum[(size_t)b * (k + 2) + h];
+    for (int h = 0; h <= k; ++h) g->node_off[h] = d->h_node_off[(size_t)h * (B + 1) + b];
+    g->V = g->cum[k + 1];
+    g->n_targets = g->cum[1];
+}
+
+// perm / inv of mini-batch b (device arrays owned by d, valid until the next call for another batch or sample)
+int mg_dense_batch_perm(mg_ctx* ctx, mg_dense* d, int b, const int32_t** perm, const int32_t** inv) {
+    BatchGeom g;
+    batch_geom(d, b, &g);
+    int rc = mg_ensure(ctx, &d->perm_buf, &d->perm_elems, 2 * (size_t)g.V + 8);
+    if (rc) return rc;
+    *perm = d->perm_buf;
+    *inv = d->perm_buf + g.V;
+    if (d->perm_batch == b) return MG_OK;
+    d->perm_batch = -1;
     cudaStream_t st = ctx->stream;
-    const int id_bits = std::max(1, ilog2_ceil(ctx->n_nodes)), b_bits = std::max(1, ilog2_ceil(B));
-    const int32_t* node_off_k = d->node_off + (size_t)k * (B + 1);
-    SortParams* sp = (SortParams*)(d->scan_tmp + d->scan_tmp_elems - 8);   // tail of the scratch block, as in the sampler
-    SortParams h_sp;
-    mg_sort_params_host(&h_sp, n);
-    MG_CUDA(ctx, cudaMemcpyAsync(sp, &h_sp, sizeof(h_sp), cudaMemcpyHostToDevice, st));
-    const int grid = mg_grid(ctx, 8);
-    k_canon_keys<<<grid, kThreads, 0, st>>>(d->nodes, d->node_batch, node_off_k, start, n, id_bits, d->newlist[0]);
+    const int32_t n = g.V - g.n_targets;
+    const int id_bits = std::max(1, ilog2_ceil(ctx->n_nodes)), hop_bits = std::max(1, ilog2_ceil(g.k + 1));
+    const int grid = std::max(1, std::min(mg_grid(ctx, 4), (g.V + kThreads - 1) / kThreads));
     int res = 0;
-    mg_sort_u64(ctx, d->newlist, sp, MG_SLOT_BITS, id_bits + b_bits, d->sort_hist, (uint32_t*)d->scan_tmp, &res);
-    int32_t* new_local = reinterpret_cast<int32_t*>(d->node_r0);   // per-node scratch of the sampler, free by now
-    k_canon_place<<<grid, kThreads, 0, st>>>(d->newlist[res], node_off_k, start, n, id_bits, d->nodes, new_local);
-    const int32_t e_lo = d->h_hdr.ent_base[k - 1], e_hi = d->h_hdr.ent_base[k];
-    if (e_hi > e_lo)
-        k_canon_relabel<<<grid, kThreads, 0, st>>>(e_lo, e_hi, d->d_ent_hop + (size_t)(k - 1) * (B + 1), B, k, d->cum, node_off_k,
-                                                   start, new_local, d->ent_repr);
-    ctx->launches += 3;
+    if (n > 0) {
+        SortParams* sp = (SortParams*)(d->scan_tmp + d->scan_tmp_elems - 8);   // tail of the scratch block, as in the sampler
+        SortParams h_sp;
+        mg_sort_params_host(&h_sp, n);
+        MG_CUDA(ctx, cudaMemcpyAsync(sp, &h_sp, sizeof(h_sp), cudaMemcpyHostToDevice, st));
+        k_perm_keys<<<grid, kThreads, 0, st>>>(g, d->nodes, id_bits, d->newlist[0]);
+        mg_sort_u64(ctx, d->newlist, sp, MG_SLOT_BITS, id_bits + hop_bits, d->sort_hist, (uint32_t*)d->scan_tmp, &res);
+        ctx->launches++;
+    }
+    if (g.V > 0) {
+        k_perm_fill<<<grid, kThreads, 0, st>>>(g, d->newlist[res], d->perm_buf, d->perm_buf + g.V);
+        ctx->launches++;
+    }
     MG_CUDA(ctx, cudaGetLastError());
     MG_CUDA(ctx, cudaStreamSynchronize(st));   // h_sp is a stack variable
-    d->canonical = true;
+    d->perm_batch = b;
     return MG_OK;
 }
 
@@ -1344,48 +1317,39 @@ extern "C" int mg_dense_view(mg_ctx* ctx, mg_dense* d, int32_t batch, mg_dense_a
     if (!d->valid) return mg_fail(ctx, MG_ERR_STATE, "mg_dense holds no completed sample");
     if (batch < 0 || batch >= d->n_batches) return mg_fail(ctx, MG_ERR_ARG, "batch out of range");
     MG_CUDA(ctx, cudaSetDevice(ctx->device));
-    {
-        const int rc0 = mg_dense_canonicalize(ctx, d);
-        if (rc0) return rc0;
-    }
     const int k = d->k, B = d->n_batches, b = batch;
     ExportArgs a;
     memset(&a, 0, sizeof(a));
-    a.k = k; a.b = b; a.B = B;
-    for (int h = 0; h <= k + 1; ++h) a.cum[h] = d->h_cum[(size_t)b * (k + 2) + h];
-    a.V = a.cum[k + 1];
+    batch_geom(d, b, &a.g);
+    int rc = mg_dense_batch_perm(ctx, d, b, &a.perm, &a.inv);
+    if (rc) return rc;
     // canonical Delta_j = hop k - j
     a.nio[0] = 0;
-    for (int j = 0; j <= k; ++j) a.nio[j + 1] = a.nio[j] + (a.cum[k - j + 1] - a.cum[k - j]);
+    for (int j = 0; j <= k; ++j) a.nio[j + 1] = a.nio[j] + (a.g.cum[k - j + 1] - a.g.cum[k - j]);
     a.n0 = a.nio[1];
-    for (int h = 0; h <= k; ++h) a.node_off[h] = d->h_node_off[(size_t)h * (B + 1) + b];
-    int32_t e_run = 0;
-    for (int j = 1; j <= k; ++j) {
-        const int h = k - j;
-        a.ebase[j] = e_run;
-        a.ent_hop[h] = d->h_ent_hop[(size_t)h * (B + 1) + b];
-        e_run += d->h_ent_hop[(size_t)h * (B + 1) + b + 1] - a.ent_hop[h];
-    }
-    a.E = e_run;
-    const int32_t n_s = a.V - a.n0;
-    const size_t need = (size_t)a.V + (k + 2) + 2 * (size_t)a.E + (size_t)n_s + 1 + 16;
-    int rc = mg_ensure(ctx, &d->exp_buf, &d->exp_elems, need);
+    int32_t n_entries = 0;
+    for (int h = 0; h < k; ++h) n_entries += d->h_ent_hop[(size_t)h * (B + 1) + b + 1] - d->h_ent_hop[(size_t)h * (B + 1) + b];
+    const int32_t n_s = a.g.V - a.n0;
+    const size_t need = (size_t)a.g.V + (k + 2) + 2 * (size_t)n_entries + (size_t)n_s + 1 + 16;
+    rc = mg_ensure(ctx, &d->exp_buf, &d->exp_elems, need);
     if (rc) return rc;
     a.nodes = d->nodes; a.ent_off = d->ent_off; a.ent_nbrs = d->ent_nbrs; a.ent_repr = d->ent_repr;
     a.o_node_ids = d->exp_buf;
-    a.o_nio = a.o_node_ids + a.V;
+    a.o_nio = a.o_node_ids + a.g.V;
     a.o_nbrs = a.o_nio + (k + 2);
-    a.o_nbr_off = a.o_nbrs + a.E;
+    a.o_nbr_off = a.o_nbrs + n_entries;
     a.o_repr = a.o_nbr_off + n_s + 1;
-    const int grid = std::max(1, std::min(mg_grid(ctx, 4), (a.V + kThreads - 1) / kThreads));
-    k_export<<<grid, kThreads, 0, ctx->stream>>>(a);
-    ctx->launches++;
+    const int grid = std::max(1, std::min(mg_grid(ctx, 4), (a.g.V + kThreads - 1) / kThreads));
+    k_export_nodes<<<grid, kThreads, 0, ctx->stream>>>(a);
+    k_export_scan<<<1, 1024, 0, ctx->stream>>>(a.o_nbr_off, n_s);
+    if (n_s > 0) k_export_entries<<<grid, kThreads, 0, ctx->stream>>>(a);
+    ctx->launches += 3;
     MG_CUDA(ctx, cudaGetLastError());
     MG_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     out->k = k;
-    out->n_nodes = a.V;
+    out->n_nodes = a.g.V;
     out->n_sampled = n_s;
-    out->n_entries = a.E;
+    out->n_entries = n_entries;
     out->node_ids = a.o_node_ids;
     out->node_id_offsets = a.o_nio;
     out->nbrs = a.o_nbrs;
@@ -1400,8 +1364,8 @@ extern "C" int mg_dense_free(mg_dense* d) {
     cudaFree(d->hdr); cudaFree(d->nodes); cudaFree(d->node_batch); cudaFree(d->ent_off); cudaFree(d->node_r0); cudaFree(d->node_deg);
     cudaFree(d->ent_nbrs); cudaFree(d->ent_repr); cudaFree(d->node_off); cudaFree(d->cum);
     cudaFree(d->rowbase); cudaFree(d->hkeys); cudaFree(d->hvals); cudaFree(d->newlist[0]);
-    cudaFree(d->newlist[1]); cudaFree(d->d_seeds); cudaFree(d->scan_tmp); cudaFree(d->sort_hist);
-    cudaFree(d->exp_buf); cudaFree(d->d_ent_hop);
+    cudaFree(d->newlist[1]); cudaFree(d->d_seeds); cudaFree(d->batch_cnt); cudaFree(d->scan_tmp); cudaFree(d->sort_hist);
+    cudaFree(d->exp_buf); cudaFree(d->perm_buf); cudaFree(d->d_ent_hop);
     if (d->h_pinned) cudaFreeHost(d->h_pinned);
     if (d->h_stage) cudaFreeHost(d->h_stage);
     if (d->graph_exec) cudaGraphExecDestroy(d->graph_exec);

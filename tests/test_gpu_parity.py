@@ -111,8 +111,8 @@ def test_many_batches_match_single_and_oracle(tiny):
     # device-resident targets give the same sample; so does reusing the handle
     d2 = ctx.sample_many(torch.cat(tg).cuda(), offs, [4, 3, 2], seeds, out=d)
     assert d2 is d
-    # the sampler leaves the outermost delta in discovery order; the first view puts it in ascending order and
-    # re-labels the entries that point into it.  The forward pass does not depend on that order, bit for bit.
+    # the device keeps a delta in discovery order and the views translate to ascending ids; the forward pass does
+    # not depend on the order, bit for bit, and viewing a mini-batch changes nothing on the device
     before = torch.empty_like(out)
     ctx.forward(model, d, before)
     assert_dense_equal(d.view(3), O.sample_dense(view, tg[3].tolist(), [4, 3, 2], seeds[3]))
