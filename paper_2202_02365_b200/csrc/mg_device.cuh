@@ -28,35 +28,33 @@ __device__ __forceinline__ uint32_t draw_word(uint64_t seed, uint32_t node, uint
     return s == 0 ? o[0] : (s == 1 ? o[1] : (s == 2 ? o[2] : o[3]));
 }
 
-__device__ __forceinline__ uint32_t table_hash(int32_t id, int shift) {
-    return ((uint32_t)id * 0x9E3779B1u) >> shift;
+// first probe slot of `id` in a table of `size` slots (any size: multiplicative hash, then multiply-high)
+__device__ __forceinline__ uint32_t table_hash(int32_t id, int32_t size) {
+    return __umulhi((uint32_t)id * 0x9E3779B1u, (uint32_t)size);
 }
 
 // Insert `id` into the open-addressing table `keys` (table_size slots, -1 = empty).
 // Returns the slot; *is_new tells whether this call created the entry.  Returns -1 when the
 // table is full (the caller raises ST_CAP_TABLE).
-__device__ __forceinline__ int32_t table_insert(int32_t* keys, int32_t table_size, int shift,
-                                                int32_t id, bool* is_new) {
-    uint32_t slot = table_hash(id, shift);
-    const uint32_t mask = (uint32_t)table_size - 1u;
+__device__ __forceinline__ int32_t table_insert(int32_t* keys, int32_t table_size, int32_t id, bool* is_new) {
+    uint32_t slot = table_hash(id, table_size);
     for (int32_t probe = 0; probe < table_size; ++probe) {
         const int32_t old = atomicCAS(&keys[slot], -1, id);
         if (old == -1) { *is_new = true; return (int32_t)slot; }
         if (old == id) { *is_new = false; return (int32_t)slot; }
-        slot = (slot + 1u) & mask;
+        slot = slot + 1u == (uint32_t)table_size ? 0u : slot + 1u;
     }
     *is_new = false;
     return -1;
 }
 
-__device__ __forceinline__ int32_t table_find(const int32_t* keys, int32_t table_size, int shift, int32_t id) {
-    uint32_t slot = table_hash(id, shift);
-    const uint32_t mask = (uint32_t)table_size - 1u;
+__device__ __forceinline__ int32_t table_find(const int32_t* keys, int32_t table_size, int32_t id) {
+    uint32_t slot = table_hash(id, table_size);
     for (int32_t probe = 0; probe < table_size; ++probe) {
         const int32_t cur = keys[slot];
         if (cur == id) return (int32_t)slot;
         if (cur == -1) return -1;
-        slot = (slot + 1u) & mask;
+        slot = slot + 1u == (uint32_t)table_size ? 0u : slot + 1u;
     }
     return -1;
 }

@@ -143,7 +143,6 @@ struct mg_dense {
     int32_t fanouts[MG_MAX_HOPS] = {0};
     int64_t cap_nodes = 0, cap_entries = 0;
     int32_t table_size = 0;  // slots per batch, power of two
-    int32_t table_shift = 0; // 32 - log2(table_size)
     int64_t n_targets_total = 0;
 
     // device arrays

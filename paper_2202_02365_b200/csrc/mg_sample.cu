@@ -124,8 +124,7 @@ __global__ void __launch_bounds__(kThreads) k_scan_down(uint32_t* data, ScanRang
 // hop 0: targets
 // -------------------------------------------------------------------------------------
 struct TableGeom {
-    int32_t size;   // slots per batch
-    int32_t shift;  // 32 - log2(size)
+    int32_t size;   // slots per batch (any size)
 };
 
 __global__ void __launch_bounds__(kThreads)
@@ -141,7 +140,7 @@ k_init_targets(DenseHeader* hdr, const int32_t* __restrict__ targets, int32_t n_
         if (v < 0 || (int64_t)v >= n_nodes) { atomicOr(&hdr->status, ST_RANGE); continue; }
         if (slot_of_part[(int64_t)v / part_size] < 0) { atomicOr(&hdr->status, ST_NONRESIDENT); continue; }
         bool is_new;
-        const int32_t slot = table_insert(hkeys + (int64_t)b * tg.size, tg.size, tg.shift, v, &is_new);
+        const int32_t slot = table_insert(hkeys + (int64_t)b * tg.size, tg.size, v, &is_new);
         if (slot < 0) { atomicOr(&hdr->status, ST_CAP_TABLE); continue; }
         if (!is_new) { atomicOr(&hdr->status, ST_DUPLICATE); continue; }
         hvals[(int64_t)b * tg.size + slot] = i - tgt_off[b];
@@ -359,7 +358,6 @@ __global__ void __launch_bounds__(kThreads) k_insert(InsertArgs a) {
     const int32_t lo = a.hdr->ent_base[a.hop], hi = a.hdr->ent_base[a.hop + 1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int kChunk = kThreads * kInsertPerThread;
-    const uint32_t mask = (uint32_t)a.tg.size - 1u;
     for (int32_t base = lo + blockIdx.x * kChunk; base < hi; base += gridDim.x * kChunk) {
         int32_t u[kInsertPerThread], b[kInsertPerThread], old[kInsertPerThread];
         uint32_t slot[kInsertPerThread];
@@ -372,7 +370,7 @@ __global__ void __launch_bounds__(kThreads) k_insert(InsertArgs a) {
 #pragma unroll
         for (int j = 0; j < kInsertPerThread; ++j)
             if (u[j] >= 0) {
-                slot[j] = table_hash(u[j], a.tg.shift);
+                slot[j] = table_hash(u[j], a.tg.size);
                 old[j] = atomicCAS(&a.hkeys[(int64_t)b[j] * a.tg.size + slot[j]], -1, u[j]);
             }
         uint32_t n_mine = 0, new_bits = 0;
@@ -384,7 +382,7 @@ __global__ void __launch_bounds__(kThreads) k_insert(InsertArgs a) {
                 int32_t* keys = a.hkeys + (int64_t)b[j] * a.tg.size;
                 int32_t probe = 1;
                 for (; probe < a.tg.size; ++probe) {
-                    slot[j] = (slot[j] + 1u) & mask;
+                    slot[j] = slot[j] + 1u == (uint32_t)a.tg.size ? 0u : slot[j] + 1u;
                     const int32_t o = atomicCAS(&keys[slot[j]], -1, u[j]);
                     if (o == -1) { fresh = true; break; }
                     if (o == u[j]) break;
@@ -916,7 +914,6 @@ static int dense_alloc(mg_ctx* ctx, mg_dense* d, int32_t B, int32_t k, int64_t c
     d->k = k;
     d->n_batches = B;
     d->table_size = table_size;
-    d->table_shift = 32 - ilog2_ceil(table_size);
     return MG_OK;
 }
 
@@ -1040,9 +1037,11 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
     if (cap_nodes >= (1ll << 31) - 1 || cap_entries >= (1ll << 31) - 1)
         return mg_fail(ctx, MG_ERR_CAPACITY, "capacities must stay below 2^31 (nodes %lld, entries %lld): pass tighter mg_sample_caps or fewer batches",
                        (long long)cap_nodes, (long long)cap_entries);
-    const int tbits = std::max(4, ilog2_ceil(cap_batch * 2));
-    if (tbits > MG_SLOT_BITS) return mg_fail(ctx, MG_ERR_CAPACITY, "max_nodes_per_batch above %d", 1 << (MG_SLOT_BITS - 1));
-    const int32_t table_size = 1 << tbits;
+    // id table of a mini-batch: 1.625 slots per node it may hold (load factor <= 0.62 for linear probing), any size:
+    // its traffic is random 32-byte sectors, so every slot that is not needed costs DRAM bandwidth
+    const int64_t want_slots = std::max<int64_t>(16, (cap_batch + cap_batch / 2 + cap_batch / 8 + 7) / 8 * 8);
+    if (want_slots > (1ll << MG_SLOT_BITS)) return mg_fail(ctx, MG_ERR_CAPACITY, "max_nodes_per_batch above %d", (int)((1ll << MG_SLOT_BITS) * 8 / 13));
+    const int32_t table_size = (int32_t)want_slots;
     if ((int64_t)table_size * n_batches >= (1ll << 31))
         return mg_fail(ctx, MG_ERR_CAPACITY, "n_batches x id-table size must stay below 2^31: pass a smaller max_nodes_per_batch or fewer batches");
     const int id_bits = std::max(1, ilog2_ceil(N));
@@ -1064,7 +1063,7 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
 
     cudaStream_t st = ctx->stream;
     const int B = n_batches;
-    const TableGeom tg{table_size, d->table_shift};
+    const TableGeom tg{table_size};
 
     // Host-known part of the header, the per-batch tables and the seeds go through a pinned staging block of the
     // sample handle, so that the device work below reads nothing but fixed addresses: it can then be captured once
