@@ -327,7 +327,7 @@ struct InsertArgs {
     DenseHeader* hdr;
     int hop;
     const int32_t* ent_nbrs;
-    int32_t* ent_repr;   // in: batch id; out: batch * table_size + slot
+    int32_t* ent_repr;   // in: batch id; out: the node's row (new node) or -1 - (batch * table_size + slot)
     int32_t* hkeys;
     TableGeom tg;
     uint64_t* newlist;
@@ -389,8 +389,10 @@ __global__ void __launch_bounds__(kThreads) k_insert(InsertArgs a) {
                 }
                 if (probe >= a.tg.size) { atomicOr(&a.hdr->status, ST_CAP_TABLE); slot[j] = 0; }
             }
-            a.ent_repr[base + j * kThreads + threadIdx.x] = b[j] * a.tg.size + (int32_t)slot[j];
+            // an entry that found its node already in the table gets the node's row later (k_relabel): it leaves
+            // -1 - (table index) behind; the entry of a new node gets its row below
             if (fresh) { new_bits |= 1u << j; ++n_mine; }
+            else a.ent_repr[base + j * kThreads + threadIdx.x] = -1 - (b[j] * a.tg.size + (int32_t)slot[j]);
         }
         // block-wide exclusive scan of the per-thread counts, one global atomic for the block
         const uint32_t inc = warp_incl_scan(n_mine);
@@ -430,6 +432,7 @@ __global__ void __launch_bounds__(kThreads) k_insert(InsertArgs a) {
                     const int64_t row = (int64_t)a.cum[b[j] * (a.k + 2) + a.hop + 1] + rank[j];
                     if (row < a.max_nodes_per_batch) a.hvals[(int64_t)b[j] * a.tg.size + slot[j]] = (int32_t)row;
                     else atomicOr(&a.hdr->status, ST_CAP_TABLE);
+                    a.ent_repr[base + j * kThreads + threadIdx.x] = (int32_t)row;   // final: no table read for this entry
                 }
         }
 #pragma unroll
@@ -582,8 +585,10 @@ __global__ void __launch_bounds__(kThreads)
 k_relabel(const DenseHeader* hdr, int hop, const int32_t* __restrict__ hvals, int32_t* ent_repr) {
     if (hdr->status) return;
     const int32_t lo = hdr->ent_base[hop], hi = hdr->ent_base[hop + 1];
-    for (int32_t e = lo + blockIdx.x * blockDim.x + threadIdx.x; e < hi; e += gridDim.x * blockDim.x)
-        ent_repr[e] = hvals[ent_repr[e]];
+    for (int32_t e = lo + blockIdx.x * blockDim.x + threadIdx.x; e < hi; e += gridDim.x * blockDim.x) {
+        const int32_t v = ent_repr[e];
+        if (v < 0) ent_repr[e] = hvals[-1 - v];   // entries of nodes that were new got their row at insert time
+    }
 }
 
 // Outermost hop: per-batch counts -> node offsets of the hop and the batches' row totals (one block)
