@@ -341,7 +341,7 @@ struct InsertArgs {
     int32_t max_nodes_per_batch;
 };
 
-constexpr int kInsertPerThread = 8;
+constexpr int kInsertPerThread = 4;
 constexpr int kInsertSpan = 16;   // mini-batches a block's chunk of entries may touch on the fast path
 
 // New nodes are not sorted on the device: nothing the path computes depends on the order of ids inside a delta (the
