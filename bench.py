@@ -345,7 +345,7 @@ def main():
               "achieved": alg["flops"] / ((agg1["ms"] + rest["ms"] + gemm["ms"]) / 1e3) / 1e12, "peak": tf32_peak,
               "unit": "TFLOP/s", "layer1_tflops": flops_l1 / (agg1["ms"] / 1e3) / 1e12 if agg1["ms"] else None}
     tensor["frac"] = tensor["achieved"] / tensor["peak"]
-    mem_ms = sample_ms + agg1["ms"] + rest["ms"]
+    mem_ms = sample_ms + agg1["ms"] + rest["ms"] + phases.get("other", {"ms": 0.0})["ms"]   # "other": the layers' row pre-pass
     path_gbs = alg["a_min"] / (mem_ms / 1e3) / 1e9 if mem_ms else None
 
     line = {

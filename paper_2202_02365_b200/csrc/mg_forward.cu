@@ -530,8 +530,8 @@ static int forward_impl(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out,
         float* h_out = l == k ? hk : ctx->ws_h[0] + off[l];
         const float* h_prev = l > 1 ? ctx->ws_h[0] + off[l - 1] : nullptr;
         if (m->precision == MG_GEMM_TF32 && mg_layer_fused_supported(d_in, d_out)) {
-            // gather + segment mean + both linear maps in one persistent tensor-core kernel
-            ProfScope ps(ctx, l == 1 ? PH_AGG_L1 : PH_AGG_REST, 2);
+            // gather + segment mean + both linear maps in one persistent tensor-core kernel (after a small
+            // pre-pass that resolves every output row's sources)
             size_t have = ctx->ws_x_bytes / sizeof(int4);
             int4* meta = reinterpret_cast<int4*>(ctx->ws_x);
             if (have < (size_t)M) {
@@ -540,8 +540,14 @@ static int forward_impl(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out,
                 ctx->ws_x_bytes = have * sizeof(int4);
                 if (rc) return rc;
             }
-            if ((rc = mg_layer_rows(ctx, d, l, d_in, d_out, meta))) return rc;
-            rc = mg_layer_fused(ctx, d, l, d_in, d_out, m->w_pad_t[l - 1], m->bias[l - 1], h_prev, h_out, l < k, meta, 0, M, 0);
+            {
+                ProfScope ps(ctx, PH_OTHER, 1);
+                if ((rc = mg_layer_rows(ctx, d, l, d_in, d_out, meta))) return rc;
+            }
+            {
+                ProfScope ps(ctx, l == 1 ? PH_AGG_L1 : PH_AGG_REST, 1);
+                rc = mg_layer_fused(ctx, d, l, d_in, d_out, m->w_pad_t[l - 1], m->bias[l - 1], h_prev, h_out, l < k, meta, 0, M, 0);
+            }
             if (rc) return rc;
             continue;
         }
