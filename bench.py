@@ -37,6 +37,10 @@ CONFIGS = {
     "config4_tenth_fp16_768_in_hbm": dict(n=12_200_000, m=130_000_000, kind="rmat", dim=768, hidden=256,
                                           fanouts=[15, 10, 5], batch=1000, parts=1, train=12_200_000, fp16=True),
 }
+# link prediction (config 5: Freebase86M-shaped), measured by run_lp: a step = one batch of 50,000 edges
+LP_CONFIG = dict(n=86_000_000, m=338_000_000, dim=100, n_rel=14_824, parts=16, resident=8, edges=50_000, chunks=10,
+                 negs=1000, fanout=20)
+LP_WORKLOAD = "config5_freebase86m_shaped_lp"
 DEFAULT_WORKLOAD = "config3_papers100m_shaped"
 HBM_NOMINAL_GBS = 8000.0
 # dram bytes (read + write) of one launch of the dominant kernel, measured with ncu (see profiles/)
@@ -163,7 +167,7 @@ def main():
     ap.add_argument("--steps", type=int, default=8)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="mgdense", choices=["mgdense", "reference"])
-    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(CONFIGS))
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(CONFIGS) + [LP_WORKLOAD])
     ap.add_argument("--group", type=int, default=128, help="mini-batches per step")
     ap.add_argument("--window", type=int, default=0, help="mini-batches per window of the layer schedule (0 = whole layers)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -174,8 +178,15 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    cfg = CONFIGS[args.workload]
     peaks = measured_peaks()
+    if args.workload == LP_WORKLOAD:
+        if args.impl == "reference":
+            if rank == 0:
+                print(json.dumps({"impl": "reference", "unavailable": "the reference arm times the oracle on the default workload only"}))
+            return
+        run_lp(args, peaks, rank, local_rank, world)
+        return
+    cfg = CONFIGS[args.workload]
 
     if args.impl == "reference":
         if rank != 0:
@@ -383,6 +394,118 @@ def main():
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+
+def run_lp(args, peaks, rank, local_rank, world):
+    """Link-prediction step at config 5's sizes: negatives + target union (mg_lp_prepare), a one-hop DENSE sample with
+    fanout 20, one GraphSage layer 100 -> 100, DistMult scores of the positives and of both corrupted sides."""
+    import paper_2202_02365_b200 as mg
+    c = LP_CONFIG
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    t0 = time.time()
+    g = inputs.rmat_graph(c["n"], c["m"], seed=5, device=device, n_relations=c["n_rel"])
+    emb = inputs.normal_features(c["n"], c["dim"], seed=3, device=device, std=0.001)
+    rel_emb = inputs.normal_features(c["n_rel"], c["dim"], seed=9, device=device)
+    setup_s = round(time.time() - t0, 1)
+    ctx = mg.Context(local_rank)
+    ctx.load_graph(g.row_offsets, g.nbrs)
+    ctx.set_partitioning(c["parts"])
+    ctx.load_features(emb, capacity_parts=c["resident"])
+    resident = [0, 2, 3, 5, 8, 9, 12, 15]
+    ctx.set_resident(resident)
+    mask = inputs.resident_node_mask(c["n"], c["parts"], resident)
+    n_total = args.warmup + 2 * args.steps
+    batches = [inputs.lp_edges(g, mask, c["edges"], seed=1000 * rank + i) for i in range(n_total)]
+    n_edges_graph = g.n_edges
+    del g, mask
+    torch.cuda.empty_cache()
+    layers = inputs.glorot_layers([c["dim"], c["dim"]], seed=8)
+    model = ctx.model(layers, mg.GEMM_TF32)
+    dense = None
+    h = None
+    stats = {"targets": [], "entries": []}
+
+    def step(i, record=False):
+        nonlocal dense, h
+        src, rel, dst = batches[i]
+        lp = ctx.lp_prepare(src, rel, dst, c["chunks"], c["negs"], seed=77 + i)
+        targets = lp.view()["targets"]
+        dense = ctx.sample(targets, [c["fanout"]], seed=i, out=dense)
+        if h is None or h.shape[0] < targets.numel():
+            h = torch.empty((int(targets.numel() * 1.2) + 16, c["dim"]), dtype=torch.float32, device=device)
+        ctx.forward(model, dense, h[:targets.numel()])
+        scores = ctx.distmult_score(lp, h[:targets.numel()], rel_emb)
+        if record:
+            n_, e_ = dense.counts()
+            stats["targets"].append(int(targets.numel())); stats["entries"].append(int(e_.sum()))
+        lp.free()
+        return scores
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+
+    for i in range(args.warmup):
+        step(i)
+    sampler = ClockSampler(local_rank)
+    launches0 = ctx.kernel_launches()
+    barrier()
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for i in range(args.warmup, args.warmup + args.steps):
+        step(i)
+    ev1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms = ev0.elapsed_time(ev1)
+    launches = ctx.kernel_launches() - launches0
+    # the same steps with the library's phase events: DistMult kernel time
+    ctx.profile(True)
+    ctx.profile_read(reset=True)
+    for i in range(args.warmup + args.steps, args.warmup + 2 * args.steps):
+        step(i, record=True)
+    phases = ctx.profile_read(reset=True)
+    ctx.profile(False)
+    if world > 1:
+        tt = torch.tensor([ms], device=device, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms = float(tt[0])
+    B, negs, dim = c["edges"], c["negs"], c["dim"]
+    dm_ms = phases["distmult"]["ms"] / args.steps
+    score_bytes = 4.0 * B * (1 + 2 * negs)                       # compulsory score writes, both corrupted sides
+    operand_bytes = 4.0 * (3 * B * dim + 2 * c["chunks"] * negs * dim)
+    flops = 2.0 * B * negs * dim * 2 + 3.0 * B * dim
+    line = {
+        "metric": "link-prediction steps/s (negatives + DENSE sample + GraphSage layer + DistMult, 50,000 edges per step)",
+        "value": args.steps * world / (ms / 1e3), "unit": "steps/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32 (TF32 tensor-core GEMM)", "data": "synthetic",
+        "config": {"workload": LP_WORKLOAD, "nodes": c["n"], "edges": n_edges_graph, "embedding_dim": dim,
+                   "relations": c["n_rel"], "partitions": c["parts"], "resident": len(resident), "edges_per_step": B,
+                   "chunks": c["chunks"], "negatives_per_chunk": negs, "fanouts": [c["fanout"]],
+                   "l2": "inputs larger than L2 (embedding table 34 GB, scores 400 MB per step; no flush)",
+                   "setup_s": {"graph_and_embeddings_s": setup_s}},
+        "scored_pairs_per_s": args.steps * world * B * (1 + 2 * negs) / (ms / 1e3),
+        "per_step": {"targets": float(np.mean(stats["targets"])), "sampled_edges": float(np.mean(stats["entries"]))},
+        "gpu_launches": int(launches), "clocks": clocks,
+        "roofline": {"kernel": "k_distmult_neg_tc (both corrupted sides) + k_distmult_pos", "bound": "hbm",
+                     "achieved": (score_bytes + operand_bytes) / (dm_ms / 1e3) / 1e9 if dm_ms else None,
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "bytes_per_step": score_bytes + operand_bytes,
+                     "ms_per_step": dm_ms, "peak_source": peaks["source"], "traffic": None,
+                     "tensor_tflops": flops / (dm_ms / 1e3) / 1e12 if dm_ms else None},
+        "phases_ms_per_step": {k2: round(v2["ms"] / args.steps, 4) for k2, v2 in phases.items() if v2["ms"] > 0},
+    }
+    if line["roofline"]["achieved"]:
+        line["roofline"]["frac"] = line["roofline"]["achieved"] / peaks["hbm_gbs"]
+    if rank == 0:
+        print(json.dumps(line))
 
 
 def run_reference(args, cfg):

@@ -123,6 +123,10 @@ struct mg_ctx {
     const float* last_hk = nullptr;
 
     // profiling
+    // link-prediction batches: scratch of mg_lp_prepare (grows, never shrinks) and one spare result block, so that a
+    // loop of prepare / free allocates nothing
+    char* lp_ws = nullptr; size_t lp_ws_bytes = 0;
+    char* lp_spare = nullptr; size_t lp_spare_bytes = 0;
     bool prof_on = false;
     bool sample_graphs = true;   // replay the sampler's launches from a CUDA graph
     ProfPhase prof[PH_COUNT];
@@ -215,6 +219,8 @@ struct mg_lp_batch {
     int32_t* rel = nullptr;
     int32_t* neg_ids = nullptr;
     int32_t* neg_idx = nullptr;
+    char* block = nullptr;       // the one device allocation the six arrays above live in
+    size_t block_bytes = 0;
 };
 
 // ---------------------------------------------------------------------------------------

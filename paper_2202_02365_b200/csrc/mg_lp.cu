@@ -2,6 +2,7 @@
 // scoring (the decoder of the paper's link-prediction configuration, Section 7.1).
 
 #include <algorithm>
+#include <cstdlib>
 
 #include "mg_device.cuh"
 #include "mg_internal.cuh"
@@ -211,15 +212,30 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_distmult_neg_tc(NegTcArgs ta)
     const uint32_t tmem_base = tmem_slot;
     const int n_slots = ta.n_slices * 8;                  // 16-byte slots per operand row
     // left operand: (row, slot) pairs over all threads
-    for (int i = threadIdx.x; i < 128 * n_slots; i += kTcThreads) {
-        const int r = i / n_slots, q = i % n_slots;
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (a_row[r] >= 0 && q * 4 < a.dim) {
-            const float4 hv = __ldg(reinterpret_cast<const float4*>(a.h + (int64_t)a_row[r] * a.dim) + q);
-            const float4 rv = __ldg(reinterpret_cast<const float4*>(a.rel_emb + (int64_t)a_rel[r] * a.dim) + q);
-            v = make_float4(to_tf32(hv.x * rv.x), to_tf32(hv.y * rv.y), to_tf32(hv.z * rv.z), to_tf32(hv.w * rv.w));
+    // (all loads of a round are issued before the first use: the gathers are latency-bound otherwise)
+    constexpr int kGatherUnroll = 8;
+    for (int i0 = threadIdx.x; i0 < 128 * n_slots; i0 += kTcThreads * kGatherUnroll) {
+        float4 hv[kGatherUnroll], rv[kGatherUnroll];
+#pragma unroll
+        for (int u = 0; u < kGatherUnroll; ++u) {
+            const int i = i0 + u * kTcThreads;
+            const int r = min(i, 128 * n_slots - 1) / n_slots, q = min(i, 128 * n_slots - 1) % n_slots;
+            const bool on = i < 128 * n_slots && a_row[r] >= 0 && q * 4 < a.dim;
+            // an absent row reads row 0 (always valid) and is zeroed below: no branch around the loads
+            hv[u] = __ldg(reinterpret_cast<const float4*>(a.h + (int64_t)(on ? a_row[r] : 0) * a.dim) + (on ? q : 0));
+            rv[u] = __ldg(reinterpret_cast<const float4*>(a.rel_emb + (int64_t)(on ? a_rel[r] : 0) * a.dim) + (on ? q : 0));
         }
-        *reinterpret_cast<float4*>(a_smem + (size_t)(q >> 3) * 16384 + swz_off(r, q & 7)) = v;
+#pragma unroll
+        for (int u = 0; u < kGatherUnroll; ++u) {
+            const int i = i0 + u * kTcThreads;
+            if (i >= 128 * n_slots) continue;
+            const int r = i / n_slots, q = i % n_slots;
+            const bool on = a_row[r] >= 0 && q * 4 < a.dim;
+            const float4 v = on ? make_float4(to_tf32(hv[u].x * rv[u].x), to_tf32(hv[u].y * rv[u].y), to_tf32(hv[u].z * rv[u].z),
+                                              to_tf32(hv[u].w * rv[u].w))
+                                : make_float4(0.f, 0.f, 0.f, 0.f);
+            *reinterpret_cast<float4*>(a_smem + (size_t)(q >> 3) * 16384 + swz_off(r, q & 7)) = v;
+        }
     }
     uint32_t phase = 0;
     bool ok = true;
@@ -228,14 +244,25 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_distmult_neg_tc(NegTcArgs ta)
         for (int t = threadIdx.x; t < bn; t += kTcThreads)
             b_row[t] = (n0 + t < a.negs) ? a.neg_idx[(int64_t)c * a.negs + n0 + t] : -1;
         __syncthreads();   // also: the previous block's epilogue has drained tensor memory reads
-        for (int i = threadIdx.x; i < bn * n_slots; i += kTcThreads) {
-            const int r = i / n_slots, q = i % n_slots;
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (b_row[r] >= 0 && q * 4 < a.dim) {
-                const float4 hv = __ldg(reinterpret_cast<const float4*>(a.h + (int64_t)b_row[r] * a.dim) + q);
-                v = make_float4(to_tf32(hv.x), to_tf32(hv.y), to_tf32(hv.z), to_tf32(hv.w));
+        for (int i0 = threadIdx.x; i0 < bn * n_slots; i0 += kTcThreads * kGatherUnroll) {
+            float4 hv[kGatherUnroll];
+#pragma unroll
+            for (int u = 0; u < kGatherUnroll; ++u) {
+                const int i = i0 + u * kTcThreads;
+                const int r = min(i, bn * n_slots - 1) / n_slots, q = min(i, bn * n_slots - 1) % n_slots;
+                const bool on = i < bn * n_slots && b_row[r] >= 0 && q * 4 < a.dim;
+                hv[u] = __ldg(reinterpret_cast<const float4*>(a.h + (int64_t)(on ? b_row[r] : 0) * a.dim) + (on ? q : 0));
             }
-            *reinterpret_cast<float4*>(b_smem + (size_t)(q >> 3) * b_slice_bytes + swz_off(r, q & 7)) = v;
+#pragma unroll
+            for (int u = 0; u < kGatherUnroll; ++u) {
+                const int i = i0 + u * kTcThreads;
+                if (i >= bn * n_slots) continue;
+                const int r = i / n_slots, q = i % n_slots;
+                const bool on = b_row[r] >= 0 && q * 4 < a.dim;
+                const float4 v = on ? make_float4(to_tf32(hv[u].x), to_tf32(hv[u].y), to_tf32(hv[u].z), to_tf32(hv[u].w))
+                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+                *reinterpret_cast<float4*>(b_smem + (size_t)(q >> 3) * b_slice_bytes + swz_off(r, q & 7)) = v;
+            }
         }
         fence_async_smem();
         tc_fence_before();
@@ -287,8 +314,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_distmult_neg_tc(NegTcArgs ta)
 extern "C" int mg_lp_free(mg_lp_batch* lp) {
     if (!lp) return MG_OK;
     cudaSetDevice(lp->device);
-    cudaFree(lp->targets); cudaFree(lp->src_idx); cudaFree(lp->dst_idx); cudaFree(lp->rel);
-    cudaFree(lp->neg_ids); cudaFree(lp->neg_idx);
+    mg_ctx* ctx = lp->ctx;
+    // the block becomes the context's spare (the next mg_lp_prepare takes it) unless the spare is already larger
+    if (ctx && lp->block && lp->block_bytes > ctx->lp_spare_bytes) {
+        cudaFree(ctx->lp_spare);
+        ctx->lp_spare = lp->block; ctx->lp_spare_bytes = lp->block_bytes;
+    } else {
+        cudaFree(lp->block);
+    }
     delete lp;
     return MG_OK;
 }
@@ -307,26 +340,54 @@ extern "C" int mg_lp_prepare(mg_ctx* ctx, const int32_t* src, const int32_t* rel
     mg_lp_batch* lp = new mg_lp_batch();
     lp->ctx = ctx; lp->device = ctx->device; lp->n_edges = n_edges; lp->n_chunks = n_chunks; lp->negs = negs;
 
-    int32_t *d_src = nullptr, *d_dst = nullptr, *d_nt = nullptr;
-    uint64_t* keys[2] = {nullptr, nullptr};
-    uint32_t *heads = nullptr, *hist = nullptr, *scan_tmp = nullptr, *d_status = nullptr;
-    SortParams* sp = nullptr;
     const size_t n_neg = (size_t)std::max<int64_t>((int64_t)n_chunks * negs, 1);
-    auto cleanup = [&]() {
-        cudaFree(d_src); cudaFree(d_dst); cudaFree(d_nt); cudaFree(keys[0]); cudaFree(keys[1]);
-        cudaFree(heads); cudaFree(hist); cudaFree(scan_tmp); cudaFree(d_status); cudaFree(sp);
-    };
     const size_t hist_elems = mg_sort_hist_elems(total);
     const size_t scan_elems = std::max(mg_scan_tmp_elems(total), mg_scan_tmp_elems((int64_t)hist_elems));
-    bool ok = cudaMalloc((void**)&d_src, 4 * n_edges) == cudaSuccess && cudaMalloc((void**)&d_dst, 4 * n_edges) == cudaSuccess &&
-              cudaMalloc((void**)&d_nt, 4) == cudaSuccess && cudaMalloc((void**)&keys[0], 8 * total) == cudaSuccess &&
-              cudaMalloc((void**)&keys[1], 8 * total) == cudaSuccess && cudaMalloc((void**)&heads, 4 * total) == cudaSuccess &&
-              cudaMalloc((void**)&hist, 4 * hist_elems) == cudaSuccess && cudaMalloc((void**)&scan_tmp, 4 * scan_elems) == cudaSuccess &&
-              cudaMalloc((void**)&d_status, 4) == cudaSuccess && cudaMalloc((void**)&sp, sizeof(SortParams)) == cudaSuccess &&
-              cudaMalloc((void**)&lp->targets, 4 * total) == cudaSuccess && cudaMalloc((void**)&lp->src_idx, 4 * n_edges) == cudaSuccess &&
-              cudaMalloc((void**)&lp->dst_idx, 4 * n_edges) == cudaSuccess && cudaMalloc((void**)&lp->rel, 4 * n_edges) == cudaSuccess &&
-              cudaMalloc((void**)&lp->neg_ids, 4 * n_neg) == cudaSuccess && cudaMalloc((void**)&lp->neg_idx, 4 * n_neg) == cudaSuccess;
-    if (!ok) { cudaGetLastError(); cleanup(); mg_lp_free(lp); return mg_fail(ctx, MG_ERR_OOM, "allocation of the link-prediction batch failed"); }
+    auto up = [](size_t b) { return (b + 255) / 256 * 256; };
+    // scratch: one block of the context that only grows
+    const size_t ws_bytes = 2 * up(4 * (size_t)n_edges) + 2 * up(8 * (size_t)total) + up(4 * (size_t)total) + up(4 * hist_elems) +
+                            up(4 * scan_elems) + 3 * 256;
+    if (ctx->lp_ws_bytes < ws_bytes) {
+        cudaFree(ctx->lp_ws);
+        ctx->lp_ws = nullptr; ctx->lp_ws_bytes = 0;
+        if (cudaMalloc((void**)&ctx->lp_ws, ws_bytes + ws_bytes / 4) != cudaSuccess) {
+            cudaGetLastError(); delete lp;
+            return mg_fail(ctx, MG_ERR_OOM, "allocation of the link-prediction scratch failed");
+        }
+        ctx->lp_ws_bytes = ws_bytes + ws_bytes / 4;
+    }
+    char* w = ctx->lp_ws;
+    auto take = [&](size_t b) { char* p = w; w += up(b); return p; };
+    int32_t* d_src = (int32_t*)take(4 * (size_t)n_edges);
+    int32_t* d_dst = (int32_t*)take(4 * (size_t)n_edges);
+    uint64_t* keys[2];
+    keys[0] = (uint64_t*)take(8 * (size_t)total);
+    keys[1] = (uint64_t*)take(8 * (size_t)total);
+    uint32_t* heads = (uint32_t*)take(4 * (size_t)total);
+    uint32_t* hist = (uint32_t*)take(4 * hist_elems);
+    uint32_t* scan_tmp = (uint32_t*)take(4 * scan_elems);
+    uint32_t* d_status = (uint32_t*)take(4);
+    int32_t* d_nt = (int32_t*)take(4);
+    SortParams* sp = (SortParams*)take(sizeof(SortParams));
+    // results: one block, taken from the context's spare when that is large enough
+    const size_t blk_bytes = up(4 * (size_t)total) + 3 * up(4 * (size_t)n_edges) + 2 * up(4 * n_neg);
+    if (ctx->lp_spare && ctx->lp_spare_bytes >= blk_bytes) {
+        lp->block = ctx->lp_spare; lp->block_bytes = ctx->lp_spare_bytes;
+        ctx->lp_spare = nullptr; ctx->lp_spare_bytes = 0;
+    } else if (cudaMalloc((void**)&lp->block, blk_bytes) != cudaSuccess) {
+        cudaGetLastError(); delete lp;
+        return mg_fail(ctx, MG_ERR_OOM, "allocation of the link-prediction batch failed");
+    } else {
+        lp->block_bytes = blk_bytes;
+    }
+    w = lp->block;
+    lp->targets = (int32_t*)take(4 * (size_t)total);
+    lp->src_idx = (int32_t*)take(4 * (size_t)n_edges);
+    lp->dst_idx = (int32_t*)take(4 * (size_t)n_edges);
+    lp->rel = (int32_t*)take(4 * (size_t)n_edges);
+    lp->neg_ids = (int32_t*)take(4 * n_neg);
+    lp->neg_idx = (int32_t*)take(4 * n_neg);
+    auto cleanup = [&]() {};
 
     SortParams h_sp;
     mg_sort_params_host(&h_sp, total);

@@ -128,10 +128,11 @@ struct TableGeom {
 };
 
 __global__ void __launch_bounds__(kThreads)
-k_init_targets(DenseHeader* hdr, const int32_t* __restrict__ targets, int32_t n_total,
+k_init_targets(DenseHeader* hdr, const int32_t* __restrict__ targets,
                const int32_t* __restrict__ tgt_off, int32_t B, int32_t* nodes, int32_t* node_batch,
                int32_t* hkeys, int32_t* hvals, TableGeom tg, int64_t n_nodes, int64_t part_size,
                const int32_t* __restrict__ slot_of_part) {
+    const int32_t n_total = hdr->hop_base[1];   // read on the device: the launch does not depend on the number of targets
     for (int32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n_total; i += gridDim.x * blockDim.x) {
         const int b = upper_segment(tgt_off, B + 1, i);
         const int32_t v = targets[i];
@@ -1033,9 +1034,17 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
         worst_entries_total += (int64_t)std::min(entries, 4.0e18);
         worst_nodes_batch = std::max(worst_nodes_batch, nb);
     }
-    int64_t cap_nodes = (caps && caps->max_nodes_total > 0) ? caps->max_nodes_total : worst_nodes_total;
-    int64_t cap_entries = (caps && caps->max_entries_total > 0) ? caps->max_entries_total : worst_entries_total;
+    // Worst-case bounds follow the number of targets: they are rounded up on a geometric grid (steps of 1/8), so
+    // that calls of similar size share allocations, table size and the captured graph.
+    auto grid_up = [](int64_t v) {
+        int64_t q = 1024;
+        while (q < v) q += std::max<int64_t>(q / 8, 1);
+        return q >= (1ll << 31) - 1 ? v : q;   // never round a legal bound out of range
+    };
+    int64_t cap_nodes = (caps && caps->max_nodes_total > 0) ? caps->max_nodes_total : grid_up(worst_nodes_total);
+    int64_t cap_entries = (caps && caps->max_entries_total > 0) ? caps->max_entries_total : grid_up(worst_entries_total);
     int64_t cap_batch = (caps && caps->max_nodes_per_batch > 0) ? caps->max_nodes_per_batch : worst_nodes_batch;
+    if (!(caps && caps->max_nodes_per_batch > 0)) cap_batch = std::min<int64_t>(grid_up(cap_batch), std::max<int64_t>(N, 1));
     cap_nodes = std::max<int64_t>({cap_nodes, T, 1});   // even an empty call needs its (one-element) arrays
     cap_batch = std::max<int64_t>(cap_batch, 1);
     for (int b = 0; b < n_batches; ++b) cap_batch = std::max<int64_t>(cap_batch, target_offsets[b + 1] - target_offsets[b]);
@@ -1124,8 +1133,8 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
         MG_CUDA(ctx, cudaMemcpyAsync(d->cum, st_cum, sizeof(int32_t) * (size_t)B * (k + 2), cudaMemcpyHostToDevice, st));
         MG_CUDA(ctx, cudaMemcpyAsync(d->d_seeds, st_seeds, sizeof(uint64_t) * B, cudaMemcpyHostToDevice, st));
         MG_CUDA(ctx, cudaMemsetAsync(d->hkeys, 0xFF, sizeof(int32_t) * (size_t)B * table_size, st));
-        if (T > 0) {
-            k_init_targets<<<mg_grid(ctx, 4), kThreads, 0, st>>>(d->hdr, tgt_dev, (int32_t)T, d->node_off, B, d->nodes,
+        {
+            k_init_targets<<<mg_grid(ctx, 4), kThreads, 0, st>>>(d->hdr, tgt_dev, d->node_off, B, d->nodes,
                                                                d->node_batch, d->hkeys, d->hvals, tg, ctx->n_nodes,
                                                                ctx->part_size, ctx->d_slot_of_part);
             ctx->launches++;
@@ -1203,7 +1212,7 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
     // capture it (again) otherwise.  Profiling runs the launches one by one (its events do not belong in a graph).
     SampleSignature sig;
     memset(&sig, 0, sizeof(sig));
-    sig.B = B; sig.k = k; sig.T = T; sig.table_size = table_size; sig.cap_batch = cap_batch;
+    sig.B = B; sig.k = k; sig.T = 0; sig.table_size = table_size; sig.cap_batch = cap_batch;   // (the device work does not depend on T)
     sig.cap_nodes = d->cap_nodes; sig.cap_entries = d->cap_entries; sig.n_nodes = ctx->n_nodes; sig.part_size = ctx->part_size;
     for (int h = 0; h < k; ++h) sig.fanouts[h] = fanouts[h];
     const void* ptrs[] = {d->hdr, d->nodes, d->node_batch, d->ent_off, d->node_r0, d->node_deg, d->newlist[0], d->newlist[1],
