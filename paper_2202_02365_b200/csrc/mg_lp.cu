@@ -156,14 +156,17 @@ __global__ void __launch_bounds__(256) k_distmult_neg(NegArgs a) {
 }
 
 // ---- tensor-core negative scoring ------------------------------------------------------------
-// One CTA owns 128 edges of one chunk and one corrupted side.  The left operand rows
-// h[keep] (*) rel[r] are formed on the fly, rounded to TF32 and written K-major with the 128-byte
-// swizzle; for each block of up to 256 negatives the right operand rows h[neg] are gathered the same
-// way, one thread issues the tcgen05 MMAs (fp32 accumulator in tensor memory) and four warps store
-// the block of scores with coalesced row segments.  The score matrix (4 bytes per (edge, negative))
-// is the bulk of the traffic; the contraction itself is small.
-constexpr int kTcThreads = 256;
+// One CTA owns 128 edges of one chunk and one corrupted side.  The left operand rows h[keep] (*) rel[r] are formed
+// once, rounded to TF32 and written K-major with the 128-byte swizzle.  The chunk's negatives are scored in blocks of
+// up to 128: four gather warps fill the right operand rows h[neg] of block j+1 (two buffers) while one thread issues the
+// tcgen05 MMAs of block j (fp32 accumulator in tensor memory, two buffers) and four epilogue warps store block j-1's
+// scores as coalesced row segments.  The score matrix (4 bytes per (edge, negative)) is the bulk of the traffic; the
+// contraction itself is small.  Every wait is bounded.
+constexpr int kTcGatherWarps = 8, kTcEpilogueWarps = 4;
+constexpr int kTcMmaWarp = kTcEpilogueWarps + kTcGatherWarps;
+constexpr int kTcThreads = (kTcMmaWarp + 1) * 32;   // 416: epilogue 0..3, gather 4..11, MMA 12
 constexpr int kTcMaxSlices = 4;   // dim <= 128
+constexpr int kTcBlockN = 128;    // negatives per block
 
 struct NegTcArgs {
     NegArgs base;
@@ -178,26 +181,34 @@ __device__ __forceinline__ size_t swz_off(int row, int slot) {   // 16-byte slot
 __global__ void __launch_bounds__(kTcThreads, 1) k_distmult_neg_tc(NegTcArgs ta) {
     using namespace tc;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t mma_done;
+    __shared__ uint64_t a_full, b_full[2], b_empty[2], acc_full[2], acc_empty[2];
     __shared__ uint32_t tmem_slot;
-    __shared__ int32_t a_row[128], a_rel[128], b_row[256];
-    __shared__ float out_stage[4][32 * 33];
+    __shared__ int32_t a_row[128], a_rel[128];
+    __shared__ __align__(16) float out_stage[kTcEpilogueWarps][32 * 33];
     const NegArgs& a = ta.base;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint8_t* a_smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);   // n_slices x 16 KiB
-    uint8_t* b_smem = a_smem + (size_t)ta.n_slices * 16384;                          // n_slices x bn_max x 128 B
     const size_t b_slice_bytes = (size_t)ta.bn_max * 128;
+    const size_t b_buf_bytes = (size_t)ta.n_slices * b_slice_bytes;
+    uint8_t* b_smem = a_smem + (size_t)ta.n_slices * 16384;                          // 2 x n_slices x bn_max x 128 B
 
     const int c = blockIdx.x / a.tiles_per_chunk, tile = blockIdx.x % a.tiles_per_chunk;
     const int64_t lo = ((int64_t)c * a.E + a.n_chunks - 1) / a.n_chunks;
     const int64_t hi = ((int64_t)(c + 1) * a.E + a.n_chunks - 1) / a.n_chunks;
     const int64_t m0 = lo + (int64_t)tile * 128;
+    const int n_blocks = (a.negs + ta.bn_max - 1) / ta.bn_max;
+    const int n_slots = ta.n_slices * 8;                  // 16-byte slots per operand row
+    constexpr int kGatherThreads = kTcGatherWarps * 32, kGatherUnroll = 8;
 
     if (threadIdx.x == 0) {
-        mbar_init(&mma_done, 1);
+        mbar_init(&a_full, kTcGatherWarps);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&b_full[s], kTcGatherWarps); mbar_init(&b_empty[s], 1);
+            mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], kTcEpilogueWarps);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {
+    if (warp == kTcMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"((uint32_t)ta.tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -210,100 +221,161 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_distmult_neg_tc(NegTcArgs ta)
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
-    const int n_slots = ta.n_slices * 8;                  // 16-byte slots per operand row
-    // left operand: (row, slot) pairs over all threads
-    // (all loads of a round are issued before the first use: the gathers are latency-bound otherwise)
-    constexpr int kGatherUnroll = 8;
-    for (int i0 = threadIdx.x; i0 < 128 * n_slots; i0 += kTcThreads * kGatherUnroll) {
-        float4 hv[kGatherUnroll], rv[kGatherUnroll];
-#pragma unroll
-        for (int u = 0; u < kGatherUnroll; ++u) {
-            const int i = i0 + u * kTcThreads;
-            const int r = min(i, 128 * n_slots - 1) / n_slots, q = min(i, 128 * n_slots - 1) % n_slots;
-            const bool on = i < 128 * n_slots && a_row[r] >= 0 && q * 4 < a.dim;
-            // an absent row reads row 0 (always valid) and is zeroed below: no branch around the loads
-            hv[u] = __ldg(reinterpret_cast<const float4*>(a.h + (int64_t)(on ? a_row[r] : 0) * a.dim) + (on ? q : 0));
-            rv[u] = __ldg(reinterpret_cast<const float4*>(a.rel_emb + (int64_t)(on ? a_rel[r] : 0) * a.dim) + (on ? q : 0));
-        }
-#pragma unroll
-        for (int u = 0; u < kGatherUnroll; ++u) {
-            const int i = i0 + u * kTcThreads;
-            if (i >= 128 * n_slots) continue;
-            const int r = i / n_slots, q = i % n_slots;
-            const bool on = a_row[r] >= 0 && q * 4 < a.dim;
-            const float4 v = on ? make_float4(to_tf32(hv[u].x * rv[u].x), to_tf32(hv[u].y * rv[u].y), to_tf32(hv[u].z * rv[u].z),
-                                              to_tf32(hv[u].w * rv[u].w))
-                                : make_float4(0.f, 0.f, 0.f, 0.f);
-            *reinterpret_cast<float4*>(a_smem + (size_t)(q >> 3) * 16384 + swz_off(r, q & 7)) = v;
-        }
-    }
-    uint32_t phase = 0;
-    bool ok = true;
-    for (int n0 = 0; n0 < a.negs; n0 += ta.bn_max) {
-        const int bn = min(ta.bn_max, (a.negs - n0 + 15) / 16 * 16);   // MMA N of this block
-        for (int t = threadIdx.x; t < bn; t += kTcThreads)
-            b_row[t] = (n0 + t < a.negs) ? a.neg_idx[(int64_t)c * a.negs + n0 + t] : -1;
-        __syncthreads();   // also: the previous block's epilogue has drained tensor memory reads
-        for (int i0 = threadIdx.x; i0 < bn * n_slots; i0 += kTcThreads * kGatherUnroll) {
-            float4 hv[kGatherUnroll];
-#pragma unroll
-            for (int u = 0; u < kGatherUnroll; ++u) {
-                const int i = i0 + u * kTcThreads;
-                const int r = min(i, bn * n_slots - 1) / n_slots, q = min(i, bn * n_slots - 1) % n_slots;
-                const bool on = i < bn * n_slots && b_row[r] >= 0 && q * 4 < a.dim;
-                hv[u] = __ldg(reinterpret_cast<const float4*>(a.h + (int64_t)(on ? b_row[r] : 0) * a.dim) + (on ? q : 0));
-            }
-#pragma unroll
-            for (int u = 0; u < kGatherUnroll; ++u) {
-                const int i = i0 + u * kTcThreads;
-                if (i >= bn * n_slots) continue;
-                const int r = i / n_slots, q = i % n_slots;
-                const bool on = b_row[r] >= 0 && q * 4 < a.dim;
-                const float4 v = on ? make_float4(to_tf32(hv[u].x), to_tf32(hv[u].y), to_tf32(hv[u].z), to_tf32(hv[u].w))
-                                    : make_float4(0.f, 0.f, 0.f, 0.f);
-                *reinterpret_cast<float4*>(b_smem + (size_t)(q >> 3) * b_slice_bytes + swz_off(r, q & 7)) = v;
-            }
-        }
-        fence_async_smem();
-        tc_fence_before();
-        __syncthreads();
-        if (threadIdx.x == 0) {
+    const uint32_t acc_stride = (uint32_t)(ta.tmem_cols / 2);
+
+    if (warp < kTcEpilogueWarps) {
+        // ---------------- epilogue: tensor memory -> coalesced row segments of the score matrix ----------------
+        bool ok = true;
+        const int64_t row0 = m0 + warp * 32;
+        const bool vec4 = a.negs % 4 == 0 && (reinterpret_cast<uintptr_t>(a.out) & 15) == 0;   // rows start 16-byte aligned
+        for (int j = 0; j < n_blocks && ok; ++j) {
+            const int buf = j & 1;
+            const int n0 = j * ta.bn_max;
+            const int bn = min(ta.bn_max, (a.negs - n0 + 15) / 16 * 16);
+            if (!mbar_wait(&acc_full[buf], (j >> 1) & 1)) { if (lane == 0) atomicExch(ta.error, 21u); ok = false; break; }
             tc_fence_after();
-            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-            for (int sl = 0; sl < ta.n_slices; ++sl) {
-                const uint64_t da = smem_desc_sw128(smem_u32(a_smem + (size_t)sl * 16384));
-                const uint64_t db = smem_desc_sw128(smem_u32(b_smem + (size_t)sl * b_slice_bytes));
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) mma_tf32(tmem_base, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (sl | kk) ? 1u : 0u);
-            }
-            mma_commit(&mma_done);
-        }
-        if (ok && !mbar_wait(&mma_done, phase)) { if (lane == 0) atomicExch(ta.error, 21u); ok = false; }
-        phase ^= 1;
-        tc_fence_after();
-        if (ok && warp < 4) {
-            const int64_t row0 = m0 + warp * 32;
             for (int c0 = 0; c0 < bn; c0 += 32) {
                 uint32_t v[32];
-                tmem_ld_32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
+                tmem_ld_32(tmem_base + buf * acc_stride + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 if (row0 < hi) {
                     float* st = out_stage[warp];
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) st[lane * 33 + j] = __uint_as_float(v[j]);
-                    __syncwarp();
-                    const int n = n0 + c0 + lane;
                     const int rows = (int)min((int64_t)32, hi - row0);
-                    if (n < a.negs)
-                        for (int rr = 0; rr < rows; ++rr) a.out[(row0 + rr) * a.negs + n] = st[rr * 33 + lane];
+                    if (vec4) {
+                        // lane = row: its 8 16-byte pieces go to slots piece ^ (row % 8) of a 128-byte row; then 8 lanes
+                        // store one row's 128 bytes, 4 rows per instruction
+                        uint8_t* sb = reinterpret_cast<uint8_t*>(st);
+#pragma unroll
+                        for (int p = 0; p < 8; ++p)
+                            *reinterpret_cast<float4*>(sb + lane * 128 + ((p ^ (lane & 7)) << 4)) =
+                                make_float4(__uint_as_float(v[4 * p]), __uint_as_float(v[4 * p + 1]), __uint_as_float(v[4 * p + 2]),
+                                            __uint_as_float(v[4 * p + 3]));
+                        __syncwarp();
+                        const int p = lane & 7;
+                        const int n = n0 + c0 + 4 * p;
+#pragma unroll
+                        for (int r4 = 0; r4 < 32; r4 += 4) {
+                            const int rr = r4 + (lane >> 3);
+                            if (rr < rows && n < a.negs)
+                                *reinterpret_cast<float4*>(a.out + (row0 + rr) * a.negs + n) =
+                                    *reinterpret_cast<const float4*>(sb + rr * 128 + ((p ^ (rr & 7)) << 4));
+                        }
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < 32; ++q) st[lane * 33 + q] = __uint_as_float(v[q]);
+                        __syncwarp();
+                        const int n = n0 + c0 + lane;
+                        if (n < a.negs)
+                            for (int rr = 0; rr < rows; ++rr) a.out[(row0 + rr) * a.negs + n] = st[rr * 33 + lane];
+                    }
                     __syncwarp();
                 }
             }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[buf]);
         }
-        tc_fence_before();
+    } else if (warp < kTcEpilogueWarps + kTcGatherWarps) {
+        // ---------------- gather warps: left operand once, then the negatives block by block ----------------
+        const int gt = threadIdx.x - kTcEpilogueWarps * 32;
+        // (all loads of a round are issued before the first use: the gathers are latency-bound otherwise)
+        for (int i0 = gt; i0 < 128 * n_slots; i0 += kGatherThreads * kGatherUnroll) {
+            float4 hv[kGatherUnroll], rv[kGatherUnroll];
+#pragma unroll
+            for (int u = 0; u < kGatherUnroll; ++u) {
+                const int i = min(i0 + u * kGatherThreads, 128 * n_slots - 1);
+                const int r = i / n_slots, q = i % n_slots;
+                const bool on = a_row[r] >= 0 && q * 4 < a.dim;
+                // an absent row reads row 0 (always valid) and is zeroed below: no branch around the loads
+                hv[u] = __ldg(reinterpret_cast<const float4*>(a.h + (int64_t)(on ? a_row[r] : 0) * a.dim) + (on ? q : 0));
+                rv[u] = __ldg(reinterpret_cast<const float4*>(a.rel_emb + (int64_t)(on ? a_rel[r] : 0) * a.dim) + (on ? q : 0));
+            }
+#pragma unroll
+            for (int u = 0; u < kGatherUnroll; ++u) {
+                const int i = i0 + u * kGatherThreads;
+                if (i >= 128 * n_slots) continue;
+                const int r = i / n_slots, q = i % n_slots;
+                const bool on = a_row[r] >= 0 && q * 4 < a.dim;
+                const float4 v = on ? make_float4(to_tf32(hv[u].x * rv[u].x), to_tf32(hv[u].y * rv[u].y), to_tf32(hv[u].z * rv[u].z),
+                                                  to_tf32(hv[u].w * rv[u].w))
+                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+                *reinterpret_cast<float4*>(a_smem + (size_t)(q >> 3) * 16384 + swz_off(r, q & 7)) = v;
+            }
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&a_full);
+        bool ok = true;
+        for (int j = 0; j < n_blocks; ++j) {
+            const int buf = j & 1;
+            const int n0 = j * ta.bn_max;
+            const int bn = min(ta.bn_max, (a.negs - n0 + 15) / 16 * 16);   // MMA N of this block
+            uint8_t* bb = b_smem + (size_t)buf * b_buf_bytes;
+            if (ok && j >= 2 && !mbar_wait(&b_empty[buf], ((j >> 1) - 1) & 1)) { if (lane == 0) atomicExch(ta.error, 22u); ok = false; }
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            const int32_t* neg_idx = a.neg_idx + (int64_t)c * a.negs + n0;
+            for (int i0 = gt; i0 < bn * n_slots; i0 += kGatherThreads * kGatherUnroll) {
+                float4 hv[kGatherUnroll];
+                int32_t src[kGatherUnroll];
+#pragma unroll
+                for (int u = 0; u < kGatherUnroll; ++u) {
+                    const int i = min(i0 + u * kGatherThreads, bn * n_slots - 1);
+                    const int r = i / n_slots;
+                    src[u] = n0 + r < a.negs ? __ldg(neg_idx + r) : -1;
+                }
+#pragma unroll
+                for (int u = 0; u < kGatherUnroll; ++u) {
+                    const int i = min(i0 + u * kGatherThreads, bn * n_slots - 1);
+                    const int q = i % n_slots;
+                    const bool on = src[u] >= 0 && q * 4 < a.dim;
+                    hv[u] = __ldg(reinterpret_cast<const float4*>(a.h + (int64_t)(on ? src[u] : 0) * a.dim) + (on ? q : 0));
+                }
+#pragma unroll
+                for (int u = 0; u < kGatherUnroll; ++u) {
+                    const int i = i0 + u * kGatherThreads;
+                    if (i >= bn * n_slots) continue;
+                    const int r = i / n_slots, q = i % n_slots;
+                    const bool on = src[u] >= 0 && q * 4 < a.dim;
+                    const float4 v = on ? make_float4(to_tf32(hv[u].x), to_tf32(hv[u].y), to_tf32(hv[u].z), to_tf32(hv[u].w))
+                                        : make_float4(0.f, 0.f, 0.f, 0.f);
+                    *reinterpret_cast<float4*>(bb + (size_t)(q >> 3) * b_slice_bytes + swz_off(r, q & 7)) = v;
+                }
+            }
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&b_full[buf]);
+        }
+    } else {
+        // ---------------- MMA issue ----------------
+        if (lane == 0) {
+            bool ok = mbar_wait(&a_full, 0);
+            if (!ok) atomicExch(ta.error, 23u);
+            for (int j = 0; j < n_blocks && ok; ++j) {
+                const int buf = j & 1;
+                const int n0 = j * ta.bn_max;
+                const int bn = min(ta.bn_max, (a.negs - n0 + 15) / 16 * 16);
+                if (!mbar_wait(&b_full[buf], (j >> 1) & 1)) { atomicExch(ta.error, 24u); ok = false; break; }
+                if (j >= 2 && !mbar_wait(&acc_empty[buf], ((j >> 1) - 1) & 1)) { atomicExch(ta.error, 25u); ok = false; break; }
+                tc_fence_after();
+                const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+                const uint8_t* bb = b_smem + (size_t)buf * b_buf_bytes;
+                for (int sl = 0; sl < ta.n_slices; ++sl) {
+                    const uint64_t da = smem_desc_sw128(smem_u32(a_smem + (size_t)sl * 16384));
+                    const uint64_t db = smem_desc_sw128(smem_u32(bb + (size_t)sl * b_slice_bytes));
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        mma_tf32(tmem_base + buf * acc_stride, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (sl | kk) ? 1u : 0u);
+                }
+                mma_commit(&b_empty[buf]);
+                mma_commit(&acc_full[buf]);
+            }
+        }
+        __syncwarp();
     }
+    tc_fence_before();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == kTcMmaWarp) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)ta.tmem_cols) : "memory");
     }
@@ -457,13 +529,13 @@ extern "C" int mg_distmult_score(mg_ctx* ctx, const mg_lp_batch* lp, const float
         if (tensor) {
             NegTcArgs ta;
             ta.n_slices = (dim + 31) / 32;
-            ta.bn_max = std::min(256, (lp->negs + 15) / 16 * 16);
+            ta.bn_max = std::min(kTcBlockN, (lp->negs + 15) / 16 * 16);
             int cols = 32;
             while (cols < ta.bn_max) cols <<= 1;
-            ta.tmem_cols = cols;
+            ta.tmem_cols = 2 * cols;   // two accumulator buffers
             ta.error = ctx->d_flags;
             a.tiles_per_chunk = (int32_t)((max_chunk + 127) / 128);
-            const size_t smem = (size_t)ta.n_slices * 16384 + (size_t)ta.n_slices * ta.bn_max * 128 + 1024;
+            const size_t smem = (size_t)ta.n_slices * 16384 + 2 * (size_t)ta.n_slices * ta.bn_max * 128 + 1024;
             MG_CUDA(ctx, cudaFuncSetAttribute(k_distmult_neg_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
             const unsigned blocks = (unsigned)(a.tiles_per_chunk * lp->n_chunks);
             if (corrupt & MG_CORRUPT_DST) {
