@@ -318,6 +318,20 @@ def main():
     barrier()
     ms_e2e = ev2.elapsed_time(ev3)
 
+    # ---- latency of a single mini-batch (sample + all layers, device-resident, one call after the other) ----
+    lat_dense = None
+    lat_out = torch.empty((T, cfg["hidden"]), dtype=torch.float32, device=device)
+    lat_targets = dev_targets[0][:T].contiguous()
+    lat_ms = []
+    for rep in range(3 + 20):
+        torch.cuda.synchronize()
+        t_lat = time.perf_counter()
+        lat_dense = ctx.sample(lat_targets, cfg["fanouts"], seed=rep, out=lat_dense)
+        ctx.forward(model, lat_dense, lat_out)      # synchronous: returns when H^k is in lat_out
+        if rep >= 3:
+            lat_ms.append((time.perf_counter() - t_lat) * 1e3)
+    single_batch_latency_ms = float(np.median(lat_ms))
+
     if world > 1:
         t = torch.tensor([ms_dev, ms_e2e], device=device, dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -376,6 +390,7 @@ def main():
         "e2e": {"value": e2e_value, "unit": "mini-batches/s", "h2d_bytes_per_step": int(G * T * 4),
                 "d2h_bytes_per_step": int(G * T * cfg["hidden"] * 4), "ms_per_step": ms_e2e / args.steps},
         "gpu_launches": int(launches),
+        "single_batch_latency_ms": single_batch_latency_ms,
         "clocks": clocks,
         "roofline": roofline,
         "tensor": tensor,
