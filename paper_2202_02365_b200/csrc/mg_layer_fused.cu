@@ -60,7 +60,7 @@ struct FusedArgs {
     // input rows
     const float* h_prev;         // layers >= 2: [rows of layer l-1, d_in]
     const char* src_base;        // layer 1: the feature buffer; later layers: h_prev
-    int64_t src_row_bytes;
+    uint32_t src_row_bytes;      // (32-bit: the row address is then one wide multiply-add)
     const char* slots;           // layer 1: partition buffer
     const int32_t* slot_of_part;
     int64_t slot_bytes, row_bytes;
@@ -338,7 +338,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     if (col_ok && ok) {
 #pragma unroll
                         for (int q2 = 0; q2 < kRowsInFlight; ++q2)
-                            selfv[q2] = load4<HALF>(src + (size_t)(uint32_t)mq[q2].x * a.src_row_bytes);
+                            selfv[q2] = load4<HALF>(src + (size_t)(uint32_t)mq[q2].x * (size_t)a.src_row_bytes);
                         if (cached) {
                             // Every load is issued unconditionally: a slot past the end of a row's entries re-reads
                             // the row's own representation (a cache hit) and is added as an exact zero.  Branch-free
@@ -351,7 +351,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                                     for (int q2 = 0; q2 < kRowsInFlight; ++q2) {
                                         const bool live = e + j < mq[q2].z;
                                         const int32_t sr = rows_of[live ? mq[q2].w + e + j : 0];
-                                        v[q2][j] = load4<HALF>(src + (size_t)(uint32_t)(live ? sr : mq[q2].x) * a.src_row_bytes);
+                                        v[q2][j] = load4<HALF>(src + (size_t)(uint32_t)(live ? sr : mq[q2].x) * (size_t)a.src_row_bytes);
                                     }
 #pragma unroll
                                 for (int j = 0; j < kUnroll; ++j)   // entry order
@@ -370,7 +370,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                             for (int q2 = 0; q2 < kRowsInFlight; ++q2)
                                 for (int e = 0; e < mq[q2].z; ++e) {
                                     const int32_t sr = source_row<FIRST>(a, mq[q2].w, __ldg(keys + mq[q2].y + e));
-                                    const float4 v = load4<HALF>(src + (size_t)(uint32_t)sr * a.src_row_bytes);
+                                    const float4 v = load4<HALF>(src + (size_t)(uint32_t)sr * (size_t)a.src_row_bytes);
                                     acc[q2].x += v.x; acc[q2].y += v.y; acc[q2].z += v.z; acc[q2].w += v.w;
                                 }
                         }
@@ -584,7 +584,7 @@ int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_ou
     a.safe_src = (int32_t)safe_src_row;
     a.h_prev = h_prev;
     a.src_base = layer == 1 ? ctx->slots : reinterpret_cast<const char*>(h_prev);
-    a.src_row_bytes = layer == 1 ? ctx->row_bytes : (int64_t)d_in * 4;
+    a.src_row_bytes = layer == 1 ? (uint32_t)ctx->row_bytes : (uint32_t)d_in * 4u;
     a.relu = relu ? 1 : 0;
     a.bias = bias; a.out = h_out;
     int stride = 32;
