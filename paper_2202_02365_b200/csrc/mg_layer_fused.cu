@@ -43,6 +43,7 @@ constexpr int kBlocksPerHalf = kBlocksPerTile / 2;
 constexpr int kAccBufs = 4;                                  // accumulator buffers in tensor memory (two tiles' halves)
 constexpr int kSlicesPerGroup = 2 * kGroupCols / KC;         // 8 K slices: (self, mean) x four 32-column blocks
 constexpr int kUnroll = 5;                       // neighbour rows per output row fetched before the first add
+static_assert(kUnroll == 5, "the first-round table is read as four + one source rows");
 constexpr uint32_t kABytes = BM * KC * 4;  // 16 KiB per A stage
 
 struct FusedArgs {
@@ -126,6 +127,9 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
     __shared__ RowMeta meta[kPlanSlots][kBlockRows];
     __shared__ int32_t src_rows[kPlanSlots][kKeyCap];
     __shared__ int32_t plan_total[kPlanSlots];   // entries of the block, or -1 when they do not fit the cache
+    // source rows of each row's first kUnroll entries, padded with the row's own source row: the first round of
+    // gathers then needs no selects
+    __shared__ __align__(16) int32_t first_rows[kPlanSlots][kBlockRows][8];
     __shared__ __align__(1024) float out_stage[4][32 * 32];   // per epilogue warp: one 32 x 32 slice, 128-byte swizzled, for the TMA store
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -341,9 +345,31 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                             selfv[q2] = load4<HALF>(src + (size_t)(uint32_t)mq[q2].x * (size_t)a.src_row_bytes);
                         if (cached) {
                             // Every load is issued unconditionally: a slot past the end of a row's entries re-reads
-                            // the row's own representation (a cache hit) and is added as an exact zero.  Branch-free
-                            // code is what lets all loads of a round be in flight together.
-                            for (int e = 0; e < top; e += kUnroll) {
+                            // the row's own representation (a cache hit) and is not added.  Branch-free code is what
+                            // lets all loads of a round be in flight together.  First round: the planner has laid
+                            // out the kUnroll source rows per row, padding included.
+                            {
+                                float4 v[kRowsInFlight][kUnroll];
+#pragma unroll
+                                for (int q2 = 0; q2 < kRowsInFlight; ++q2) {
+                                    const int4 f4 = *reinterpret_cast<const int4*>(first_rows[slot][brow + q2]);
+                                    const int32_t f5 = first_rows[slot][brow + q2][4];
+                                    v[q2][0] = load4<HALF>(src + (size_t)(uint32_t)f4.x * (size_t)a.src_row_bytes);
+                                    v[q2][1] = load4<HALF>(src + (size_t)(uint32_t)f4.y * (size_t)a.src_row_bytes);
+                                    v[q2][2] = load4<HALF>(src + (size_t)(uint32_t)f4.z * (size_t)a.src_row_bytes);
+                                    v[q2][3] = load4<HALF>(src + (size_t)(uint32_t)f4.w * (size_t)a.src_row_bytes);
+                                    v[q2][4] = load4<HALF>(src + (size_t)(uint32_t)f5 * (size_t)a.src_row_bytes);
+                                }
+#pragma unroll
+                                for (int j = 0; j < kUnroll; ++j)   // entry order
+#pragma unroll
+                                    for (int q2 = 0; q2 < kRowsInFlight; ++q2)
+                                        if (j < mq[q2].z) {
+                                            acc[q2].x += v[q2][j].x; acc[q2].y += v[q2][j].y;
+                                            acc[q2].z += v[q2][j].z; acc[q2].w += v[q2][j].w;
+                                        }
+                            }
+                            for (int e = kUnroll; e < top; e += kUnroll) {
                                 float4 v[kRowsInFlight][kUnroll];
 #pragma unroll
                                 for (int j = 0; j < kUnroll; ++j)
@@ -476,6 +502,15 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
             }
             if (lane == 0) plan_total[slot] = cached ? total : -1;
             __syncwarp();
+            if (cached) {
+                // lane = row: its first kUnroll source rows, padded with its own source row
+                int32_t fr[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) fr[j] = (j < kUnroll && j < rm.z) ? src_rows[slot][koff + j] : rm.x;
+                *reinterpret_cast<int4*>(&first_rows[slot][lane][0]) = make_int4(fr[0], fr[1], fr[2], fr[3]);
+                *reinterpret_cast<int4*>(&first_rows[slot][lane][4]) = make_int4(fr[4], fr[5], fr[6], fr[7]);
+                __syncwarp();
+            }
             if (lane == 0) mbar_arrive(&plan_full[slot]);
         }
     }
