@@ -402,7 +402,8 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                         }
 #pragma unroll
                         for (int q2 = 0; q2 < kRowsInFlight; ++q2) {
-                            const float inv = mq[q2].z > 0 ? 1.f / (float)mq[q2].z : 0.f;
+                            const float inv = cached ? __int_as_float(first_rows[slot][brow + q2][5])
+                                                     : (mq[q2].z > 0 ? 1.f / (float)mq[q2].z : 0.f);
                             acc[q2].x = to_tf32(acc[q2].x * inv); acc[q2].y = to_tf32(acc[q2].y * inv);
                             acc[q2].z = to_tf32(acc[q2].z * inv); acc[q2].w = to_tf32(acc[q2].w * inv);
                             selfv[q2].x = to_tf32(selfv[q2].x); selfv[q2].y = to_tf32(selfv[q2].y);
@@ -507,6 +508,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 int32_t fr[8];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) fr[j] = (j < kUnroll && j < rm.z) ? src_rows[slot][koff + j] : rm.x;
+                fr[5] = __float_as_int(rm.z > 0 ? 1.f / (float)rm.z : 0.f);   // the mean's factor
                 *reinterpret_cast<int4*>(&first_rows[slot][lane][0]) = make_int4(fr[0], fr[1], fr[2], fr[3]);
                 *reinterpret_cast<int4*>(&first_rows[slot][lane][4]) = make_int4(fr[4], fr[5], fr[6], fr[7]);
                 __syncwarp();
