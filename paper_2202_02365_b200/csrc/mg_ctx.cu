@@ -257,7 +257,7 @@ extern "C" int mg_destroy(mg_ctx* c) {
     cudaFree(c->ws_x); cudaFree(c->ws_h[0]); cudaFree(c->ws_h[1]);
     cudaEventDestroy(c->ev_fwd_done); cudaEventDestroy(c->ev_out_done); cudaEventDestroy(c->ev_user);
     for (int i = 0; i < 2; ++i) { if (c->ev_hk_done[i]) cudaEventDestroy(c->ev_hk_done[i]); cudaFree(c->hk_buf[i]); }
-    cudaFree(c->lp_ws); cudaFree(c->lp_spare);
+    cudaFree(c->lp_ws); cudaFree(c->lp_spare); cudaFree(c->dm_images);
     cudaStreamDestroy(c->sample_stream);
     cudaStreamDestroy(c->side);
     delete c;

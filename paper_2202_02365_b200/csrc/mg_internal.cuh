@@ -127,6 +127,7 @@ struct mg_ctx {
     // loop of prepare / free allocates nothing
     char* lp_ws = nullptr; size_t lp_ws_bytes = 0;
     char* lp_spare = nullptr; size_t lp_spare_bytes = 0;
+    char* dm_images = nullptr; size_t dm_images_bytes = 0;   // TF32 operand images of the negatives (mg_distmult_score)
     bool prof_on = false;
     bool sample_graphs = true;   // replay the sampler's launches from a CUDA graph
     ProfPhase prof[PH_COUNT];

@@ -156,26 +156,56 @@ __global__ void __launch_bounds__(256) k_distmult_neg(NegArgs a) {
 }
 
 // ---- tensor-core negative scoring ------------------------------------------------------------
-// One CTA owns 128 edges of one chunk and one corrupted side.  The left operand rows h[keep] (*) rel[r] are formed
-// once, rounded to TF32 and written K-major with the 128-byte swizzle.  The chunk's negatives are scored in blocks of
-// up to 128: four gather warps fill the right operand rows h[neg] of block j+1 (two buffers) while one thread issues the
-// tcgen05 MMAs of block j (fp32 accumulator in tensor memory, two buffers) and four epilogue warps store block j-1's
-// scores as coalesced row segments.  The score matrix (4 bytes per (edge, negative)) is the bulk of the traffic; the
-// contraction itself is small.  Every wait is bounded.
-constexpr int kTcGatherWarps = 8, kTcEpilogueWarps = 4;
-constexpr int kTcMmaWarp = kTcEpilogueWarps + kTcGatherWarps;
-constexpr int kTcThreads = (kTcMmaWarp + 1) * 32;   // 416: epilogue 0..3, gather 4..11, MMA 12
+// The right operand -- the chunk's negatives h[neg], rounded to TF32 -- is the same for every 128-edge tile of a chunk:
+// k_stage_negs writes it once per call as ready-made operand images (blocks of up to 128 negatives, K-major slices of
+// 32 columns, 128-byte swizzle), a few MB that stay in L2, and the scoring kernel fetches a block with one bulk copy
+// per slice.
+// One CTA of the scoring kernel owns 128 edges of one chunk and one corrupted side.  The left operand rows
+// h[keep] (*) rel[r] are gathered once (eight warps), rounded to TF32 and written K-major with the 128-byte swizzle.
+// Then, block by block: one thread streams the operand images (two buffers), one thread issues the tcgen05 MMAs (fp32
+// accumulator in tensor memory, two buffers), and eight epilogue warps -- four from the start, four more once the left
+// operand is in place -- store the scores as coalesced row segments.  The score matrix (4 bytes per (edge, negative))
+// is the bulk of the traffic; the contraction itself is small.  Every wait is bounded.
+constexpr int kTcGatherWarps = 8, kTcEpilogueWarps = 8;   // warps 4..7 gather first and store afterwards
+constexpr int kTcFirstGatherWarp = 4;
+constexpr int kTcMmaWarp = kTcFirstGatherWarp + kTcGatherWarps;   // 12
+constexpr int kTcCopyWarp = kTcMmaWarp + 1;                       // 13
+constexpr int kTcThreads = (kTcCopyWarp + 1) * 32;                // 448
 constexpr int kTcMaxSlices = 4;   // dim <= 128
 constexpr int kTcBlockN = 128;    // negatives per block
 
 struct NegTcArgs {
     NegArgs base;
     int32_t n_slices, bn_max, tmem_cols;
+    const uint8_t* b_images;   // [n_chunks][n_blocks][n_slices][bn_max x 128 bytes]
     uint32_t* error;
 };
 
 __device__ __forceinline__ size_t swz_off(int row, int slot) {   // 16-byte slot of a 128-byte row, 8-row groups
     return (size_t)(row >> 3) * 1024 + (size_t)(row & 7) * 128 + (size_t)((slot ^ (row & 7)) << 4);
+}
+
+// operand images of the negatives: item = (chunk, block, row of the block, 16-byte slot of the row)
+__global__ void __launch_bounds__(kThreads)
+k_stage_negs(const float* __restrict__ h, const int32_t* __restrict__ neg_idx, int32_t n_chunks, int32_t negs, int32_t dim,
+             int32_t n_slices, int32_t bn_max, uint8_t* images) {
+    const int n_slots = n_slices * 8;
+    const int n_blocks = (negs + bn_max - 1) / bn_max;
+    const int64_t total = (int64_t)n_chunks * n_blocks * bn_max * n_slots;
+    const size_t slice_bytes = (size_t)bn_max * 128;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int q = (int)(i % n_slots);
+        const int r = (int)((i / n_slots) % bn_max);
+        const int64_t cb = i / ((int64_t)n_slots * bn_max);   // chunk * n_blocks + block
+        const int n = (int)(cb % n_blocks) * bn_max + r;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (n < negs && q * 4 < dim) {
+            const int32_t src = neg_idx[(cb / n_blocks) * negs + n];
+            const float4 x = __ldg(reinterpret_cast<const float4*>(h + (int64_t)src * dim) + q);
+            v = make_float4(tc::to_tf32(x.x), tc::to_tf32(x.y), tc::to_tf32(x.z), tc::to_tf32(x.w));
+        }
+        *reinterpret_cast<float4*>(images + ((size_t)cb * n_slices + (q >> 3)) * slice_bytes + swz_off(r, q & 7)) = v;
+    }
 }
 
 __global__ void __launch_bounds__(kTcThreads, 1) k_distmult_neg_tc(NegTcArgs ta) {
@@ -184,7 +214,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_distmult_neg_tc(NegTcArgs ta)
     __shared__ uint64_t a_full, b_full[2], b_empty[2], acc_full[2], acc_empty[2];
     __shared__ uint32_t tmem_slot;
     __shared__ int32_t a_row[128], a_rel[128];
-    __shared__ __align__(16) float out_stage[kTcEpilogueWarps][32 * 33];
+    __shared__ __align__(16) float out_stage[kTcEpilogueWarps][32 * 32];
     const NegArgs& a = ta.base;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint8_t* a_smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);   // n_slices x 16 KiB
@@ -203,7 +233,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_distmult_neg_tc(NegTcArgs ta)
     if (threadIdx.x == 0) {
         mbar_init(&a_full, kTcGatherWarps);
         for (int s = 0; s < 2; ++s) {
-            mbar_init(&b_full[s], kTcGatherWarps); mbar_init(&b_empty[s], 1);
+            mbar_init(&b_full[s], 1); mbar_init(&b_empty[s], 1);
             mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], kTcEpilogueWarps);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -223,61 +253,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_distmult_neg_tc(NegTcArgs ta)
     const uint32_t tmem_base = tmem_slot;
     const uint32_t acc_stride = (uint32_t)(ta.tmem_cols / 2);
 
-    if (warp < kTcEpilogueWarps) {
-        // ---------------- epilogue: tensor memory -> coalesced row segments of the score matrix ----------------
-        bool ok = true;
-        const int64_t row0 = m0 + warp * 32;
-        const bool vec4 = a.negs % 4 == 0 && (reinterpret_cast<uintptr_t>(a.out) & 15) == 0;   // rows start 16-byte aligned
-        for (int j = 0; j < n_blocks && ok; ++j) {
-            const int buf = j & 1;
-            const int n0 = j * ta.bn_max;
-            const int bn = min(ta.bn_max, (a.negs - n0 + 15) / 16 * 16);
-            if (!mbar_wait(&acc_full[buf], (j >> 1) & 1)) { if (lane == 0) atomicExch(ta.error, 21u); ok = false; break; }
-            tc_fence_after();
-            for (int c0 = 0; c0 < bn; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld_32(tmem_base + buf * acc_stride + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (row0 < hi) {
-                    float* st = out_stage[warp];
-                    const int rows = (int)min((int64_t)32, hi - row0);
-                    if (vec4) {
-                        // lane = row: its 8 16-byte pieces go to slots piece ^ (row % 8) of a 128-byte row; then 8 lanes
-                        // store one row's 128 bytes, 4 rows per instruction
-                        uint8_t* sb = reinterpret_cast<uint8_t*>(st);
-#pragma unroll
-                        for (int p = 0; p < 8; ++p)
-                            *reinterpret_cast<float4*>(sb + lane * 128 + ((p ^ (lane & 7)) << 4)) =
-                                make_float4(__uint_as_float(v[4 * p]), __uint_as_float(v[4 * p + 1]), __uint_as_float(v[4 * p + 2]),
-                                            __uint_as_float(v[4 * p + 3]));
-                        __syncwarp();
-                        const int p = lane & 7;
-                        const int n = n0 + c0 + 4 * p;
-#pragma unroll
-                        for (int r4 = 0; r4 < 32; r4 += 4) {
-                            const int rr = r4 + (lane >> 3);
-                            if (rr < rows && n < a.negs)
-                                *reinterpret_cast<float4*>(a.out + (row0 + rr) * a.negs + n) =
-                                    *reinterpret_cast<const float4*>(sb + rr * 128 + ((p ^ (rr & 7)) << 4));
-                        }
-                    } else {
-#pragma unroll
-                        for (int q = 0; q < 32; ++q) st[lane * 33 + q] = __uint_as_float(v[q]);
-                        __syncwarp();
-                        const int n = n0 + c0 + lane;
-                        if (n < a.negs)
-                            for (int rr = 0; rr < rows; ++rr) a.out[(row0 + rr) * a.negs + n] = st[rr * 33 + lane];
-                    }
-                    __syncwarp();
-                }
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&acc_empty[buf]);
-        }
-    } else if (warp < kTcEpilogueWarps + kTcGatherWarps) {
-        // ---------------- gather warps: left operand once, then the negatives block by block ----------------
-        const int gt = threadIdx.x - kTcEpilogueWarps * 32;
+    if (warp >= kTcFirstGatherWarp && warp < kTcMmaWarp) {
+        // ---------------- gather warps: the left operand, once ----------------
+        const int gt = threadIdx.x - kTcFirstGatherWarp * 32;
         // (all loads of a round are issued before the first use: the gathers are latency-bound otherwise)
         for (int i0 = gt; i0 < 128 * n_slots; i0 += kGatherThreads * kGatherUnroll) {
             float4 hv[kGatherUnroll], rv[kGatherUnroll];
@@ -305,48 +283,85 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_distmult_neg_tc(NegTcArgs ta)
         fence_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(&a_full);
+    }
+    if (warp < kTcEpilogueWarps) {
+        // ---------------- epilogue: tensor memory -> coalesced row segments of the score matrix ----------------
+        // warp w reads the accumulator rows 32 (w % 4) .. + 31 (its quarter of tensor memory) and takes every second
+        // 32-column slice of them
         bool ok = true;
-        for (int j = 0; j < n_blocks; ++j) {
+        const int quarter = warp & 3, half = warp >> 2;
+        const int64_t row0 = m0 + quarter * 32;
+        const bool vec4 = a.negs % 4 == 0 && (reinterpret_cast<uintptr_t>(a.out) & 15) == 0;   // rows start 16-byte aligned
+        for (int j = 0; j < n_blocks && ok; ++j) {
             const int buf = j & 1;
             const int n0 = j * ta.bn_max;
-            const int bn = min(ta.bn_max, (a.negs - n0 + 15) / 16 * 16);   // MMA N of this block
-            uint8_t* bb = b_smem + (size_t)buf * b_buf_bytes;
-            if (ok && j >= 2 && !mbar_wait(&b_empty[buf], ((j >> 1) - 1) & 1)) { if (lane == 0) atomicExch(ta.error, 22u); ok = false; }
-            ok = __all_sync(0xFFFFFFFFu, ok);
-            if (!ok) break;
-            const int32_t* neg_idx = a.neg_idx + (int64_t)c * a.negs + n0;
-            for (int i0 = gt; i0 < bn * n_slots; i0 += kGatherThreads * kGatherUnroll) {
-                float4 hv[kGatherUnroll];
-                int32_t src[kGatherUnroll];
+            const int bn = min(ta.bn_max, (a.negs - n0 + 15) / 16 * 16);
+            if (!mbar_wait(&acc_full[buf], (j >> 1) & 1)) { if (lane == 0) atomicExch(ta.error, 21u); ok = false; break; }
+            tc_fence_after();
+            for (int c0 = 32 * half; c0 < bn; c0 += 64) {
+                uint32_t v[32];
+                tmem_ld_32(tmem_base + buf * acc_stride + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, v);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (row0 < hi) {
+                    float* st = out_stage[warp];
+                    const int rows = (int)min((int64_t)32, hi - row0);
+                    if (vec4) {
+                        // lane = row: its 8 16-byte pieces go to slots piece ^ (row % 8) of a 128-byte row; then 8 lanes
+                        // store one row's 128 bytes, 4 rows per instruction
+                        uint8_t* sb = reinterpret_cast<uint8_t*>(st);
 #pragma unroll
-                for (int u = 0; u < kGatherUnroll; ++u) {
-                    const int i = min(i0 + u * kGatherThreads, bn * n_slots - 1);
-                    const int r = i / n_slots;
-                    src[u] = n0 + r < a.negs ? __ldg(neg_idx + r) : -1;
-                }
+                        for (int p = 0; p < 8; ++p)
+                            *reinterpret_cast<float4*>(sb + lane * 128 + ((p ^ (lane & 7)) << 4)) =
+                                make_float4(__uint_as_float(v[4 * p]), __uint_as_float(v[4 * p + 1]), __uint_as_float(v[4 * p + 2]),
+                                            __uint_as_float(v[4 * p + 3]));
+                        __syncwarp();
+                        const int p = lane & 7;
+                        const int n = n0 + c0 + 4 * p;
 #pragma unroll
-                for (int u = 0; u < kGatherUnroll; ++u) {
-                    const int i = min(i0 + u * kGatherThreads, bn * n_slots - 1);
-                    const int q = i % n_slots;
-                    const bool on = src[u] >= 0 && q * 4 < a.dim;
-                    hv[u] = __ldg(reinterpret_cast<const float4*>(a.h + (int64_t)(on ? src[u] : 0) * a.dim) + (on ? q : 0));
-                }
+                        for (int r4 = 0; r4 < 32; r4 += 4) {
+                            const int rr = r4 + (lane >> 3);
+                            if (rr < rows && n < a.negs)
+                                *reinterpret_cast<float4*>(a.out + (row0 + rr) * a.negs + n) =
+                                    *reinterpret_cast<const float4*>(sb + rr * 128 + ((p ^ (rr & 7)) << 4));
+                        }
+                    } else {
+                        // lane = row: column q of the row goes to word q ^ row, so that writes (one column, 32 rows) and
+                        // reads (one row, 32 columns) both touch 32 banks
 #pragma unroll
-                for (int u = 0; u < kGatherUnroll; ++u) {
-                    const int i = i0 + u * kGatherThreads;
-                    if (i >= bn * n_slots) continue;
-                    const int r = i / n_slots, q = i % n_slots;
-                    const bool on = src[u] >= 0 && q * 4 < a.dim;
-                    const float4 v = on ? make_float4(to_tf32(hv[u].x), to_tf32(hv[u].y), to_tf32(hv[u].z), to_tf32(hv[u].w))
-                                        : make_float4(0.f, 0.f, 0.f, 0.f);
-                    *reinterpret_cast<float4*>(bb + (size_t)(q >> 3) * b_slice_bytes + swz_off(r, q & 7)) = v;
+                        for (int q = 0; q < 32; ++q) st[lane * 32 + (q ^ lane)] = __uint_as_float(v[q]);
+                        __syncwarp();
+                        const int n = n0 + c0 + lane;
+                        if (n < a.negs)
+                            for (int rr = 0; rr < rows; ++rr) a.out[(row0 + rr) * a.negs + n] = st[rr * 32 + (lane ^ rr)];
+                    }
+                    __syncwarp();
                 }
             }
-            fence_async_smem();
+            tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&b_full[buf]);
+            if (lane == 0) mbar_arrive(&acc_empty[buf]);
         }
-    } else {
+    } else if (warp == kTcCopyWarp) {
+        // ---------------- operand images of the negatives: one bulk copy per slice ----------------
+        if (lane == 0) {
+            bool ok = true;
+            const uint8_t* images = ta.b_images + (size_t)c * n_blocks * b_buf_bytes;
+            int issued = 0;
+            for (int j = 0; j < n_blocks && ok; ++j) {
+                const int buf = j & 1;
+                if (j >= 2 && !mbar_wait(&b_empty[buf], ((j >> 1) - 1) & 1)) { atomicExch(ta.error, 22u); ok = false; break; }
+                mbar_expect_tx(&b_full[buf], (uint32_t)b_buf_bytes);
+                for (int sl = 0; sl < ta.n_slices; ++sl)
+                    bulk_load(b_smem + (size_t)buf * b_buf_bytes + (size_t)sl * b_slice_bytes,
+                              images + (size_t)j * b_buf_bytes + (size_t)sl * b_slice_bytes, (uint32_t)b_slice_bytes, &b_full[buf]);
+                issued = j + 1;
+            }
+            // nothing of this CTA's may be in flight when it ends: the last copy into each buffer has landed
+            for (int j = max(0, issued - 2); j < issued; ++j)
+                if (!mbar_wait(&b_full[j & 1], (j >> 1) & 1)) atomicExch(ta.error, 26u);
+        }
+        __syncwarp();
+    } else if (warp == kTcMmaWarp) {
         // ---------------- MMA issue ----------------
         if (lane == 0) {
             bool ok = mbar_wait(&a_full, 0);
@@ -363,8 +378,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_distmult_neg_tc(NegTcArgs ta)
                 for (int sl = 0; sl < ta.n_slices; ++sl) {
                     const uint64_t da = smem_desc_sw128(smem_u32(a_smem + (size_t)sl * 16384));
                     const uint64_t db = smem_desc_sw128(smem_u32(bb + (size_t)sl * b_slice_bytes));
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)
+                    const int k_steps = min(4, (a.dim - 32 * sl + 7) / 8);   // columns past dim are zero: skipped
+                    for (int kk = 0; kk < k_steps; ++kk)
                         mma_tf32(tmem_base + buf * acc_stride, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (sl | kk) ? 1u : 0u);
                 }
                 mma_commit(&b_empty[buf]);
@@ -535,6 +550,22 @@ extern "C" int mg_distmult_score(mg_ctx* ctx, const mg_lp_batch* lp, const float
             ta.tmem_cols = 2 * cols;   // two accumulator buffers
             ta.error = ctx->d_flags;
             a.tiles_per_chunk = (int32_t)((max_chunk + 127) / 128);
+            // operand images of the negatives (context scratch, grow-only)
+            const int n_blocks = (lp->negs + ta.bn_max - 1) / ta.bn_max;
+            const size_t image_bytes = (size_t)lp->n_chunks * n_blocks * ta.n_slices * ta.bn_max * 128;
+            if (ctx->dm_images_bytes < image_bytes) {
+                cudaFree(ctx->dm_images);
+                ctx->dm_images = nullptr; ctx->dm_images_bytes = 0;
+                if (cudaMalloc((void**)&ctx->dm_images, image_bytes) != cudaSuccess) {
+                    cudaGetLastError();
+                    return mg_fail(ctx, MG_ERR_OOM, "device allocation of %zu bytes failed", image_bytes);
+                }
+                ctx->dm_images_bytes = image_bytes;
+            }
+            k_stage_negs<<<mg_grid(ctx, 8), kThreads, 0, st>>>(h_dev, lp->neg_idx, lp->n_chunks, lp->negs, dim, ta.n_slices, ta.bn_max,
+                                                             (uint8_t*)ctx->dm_images);
+            ctx->launches++;
+            ta.b_images = (const uint8_t*)ctx->dm_images;
             const size_t smem = (size_t)ta.n_slices * 16384 + 2 * (size_t)ta.n_slices * ta.bn_max * 128 + 1024;
             MG_CUDA(ctx, cudaFuncSetAttribute(k_distmult_neg_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
             const unsigned blocks = (unsigned)(a.tiles_per_chunk * lp->n_chunks);
