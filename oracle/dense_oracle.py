@@ -26,6 +26,13 @@ Points the paper leaves open, and the reading taken here:
     len(node_ids)), nbr_offsets has one entry per sampled node plus one (last =
     len(nbrs)); Algorithm 2 indexes one past the end on the last layer without
     them.
+  * sampling direction: the rows handed to GraphView are what is sampled (the
+    harness builds them by destination: incoming neighbours, Figure 1).  With a
+    second set of rows by source (Section 4.1 keeps both sorted edge lists) and
+    direction "inout", a node gets up to f incoming neighbours followed by up to
+    f outgoing ones (Section 7.1 samples from both incoming and outgoing
+    edges); the outgoing draws use slots 65536 + t, so the two directions of a
+    node never share a random word.
   * fanouts are given ordered away from the targets (Section 7.1): api
     fanouts[h] is Algorithm 1's fanouts[k - h]; hop h = 0 samples the targets.
   * GraphSage layer: act(self . W_self + mean(neighbours) . W_nbr + b), the mean
@@ -89,9 +96,13 @@ class GraphView:
     Partitions are contiguous id ranges of `part_size` nodes.
     """
 
-    def __init__(self, row_offsets, nbrs, n_parts: int = 1, resident_parts=None):
+    def __init__(self, row_offsets, nbrs, n_parts: int = 1, resident_parts=None,
+                 out_row_offsets=None, out_nbrs=None):
         self.row_offsets = np.asarray(row_offsets, dtype=np.int64)
         self.nbrs = np.asarray(nbrs)
+        # optional second edge list, sorted by source: row v = destinations of v's outgoing edges
+        self.out_row_offsets = None if out_row_offsets is None else np.asarray(out_row_offsets, dtype=np.int64)
+        self.out_nbrs = None if out_nbrs is None else np.asarray(out_nbrs)
         self.n_nodes = len(self.row_offsets) - 1
         self.n_parts = int(n_parts)
         self.part_size = (self.n_nodes + self.n_parts - 1) // self.n_parts
@@ -106,6 +117,16 @@ class GraphView:
     def row(self, v: int):
         """R(v): the stored row of v, in stored order, resident neighbours only."""
         r = self.nbrs[self.row_offsets[v]:self.row_offsets[v + 1]]
+        if len(self._res) == self.n_parts:
+            return r
+        keep = np.isin(r // self.part_size, self.resident_parts)
+        return r[keep]
+
+    def out_row(self, v: int):
+        """The outgoing row of v (second edge list), resident neighbours only."""
+        if self.out_row_offsets is None:
+            raise ValueError("no outgoing edge list")
+        r = self.out_nbrs[self.out_row_offsets[v]:self.out_row_offsets[v + 1]]
         if len(self._res) == self.n_parts:
             return r
         keep = np.isin(r // self.part_size, self.resident_parts)
@@ -133,7 +154,10 @@ class GraphView:
         raise IndexError(idx)
 
 
-def one_hop_sample(row, f: int, seed: int, node: int, hop: int):
+OUT_SLOT_BASE = 65536   # first slot of the outgoing direction's draws
+
+
+def one_hop_sample(row, f: int, seed: int, node: int, hop: int, slot_base: int = 0):
     """Up to f neighbours of one node (Section 4.1): the whole row when it has at
     most f entries, otherwise f distinct positions (Floyd's subset algorithm,
     slot t drawing from [0, d - f + t]), returned in ascending position."""
@@ -143,17 +167,22 @@ def one_hop_sample(row, f: int, seed: int, node: int, hop: int):
     chosen = set()
     for t in range(f):
         j = d - f + t
-        x = to_range(draw_word(seed, node, hop, t), j + 1)
+        x = to_range(draw_word(seed, node, hop, slot_base + t), j + 1)
         chosen.add(j if x in chosen else x)
     return [int(row[p]) for p in sorted(chosen)]
 
 
-def one_hop_sample_all(view: GraphView, delta, f: int, seed: int, hop: int):
-    """oneHopSample(delta, f): concatenated neighbours and each node's start."""
+def one_hop_sample_all(view: GraphView, delta, f: int, seed: int, hop: int, direction: str = "in"):
+    """oneHopSample(delta, f): concatenated neighbours and each node's start.
+    direction "inout": up to f incoming, then up to f outgoing neighbours per node."""
+    if direction not in ("in", "inout"):
+        raise ValueError("direction must be 'in' or 'inout'")
     d_nbrs, d_offsets = [], []
     for v in delta:
         d_offsets.append(len(d_nbrs))
         d_nbrs.extend(one_hop_sample(view.row(v), f, seed, v, hop))
+        if direction == "inout":
+            d_nbrs.extend(one_hop_sample(view.out_row(v), f, seed, v, hop, OUT_SLOT_BASE))
     return d_nbrs, d_offsets
 
 
@@ -163,8 +192,9 @@ def compute_next_delta(d_nbrs, node_ids):
     return sorted(set(d_nbrs) - set(node_ids))
 
 
-def sample_dense(view: GraphView, target_nodes, fanouts, seed: int):
-    """Algorithm 1.  `fanouts` is ordered away from the targets.
+def sample_dense(view: GraphView, target_nodes, fanouts, seed: int, direction: str = "in"):
+    """Algorithm 1.  `fanouts` is ordered away from the targets (per direction
+    when direction is "inout").
 
     Returns a dict with node_ids, node_id_offsets (k+2 entries), nbrs,
     nbr_offsets (sampled nodes + 1 entries) and repr_map.
@@ -187,7 +217,7 @@ def sample_dense(view: GraphView, target_nodes, fanouts, seed: int):
     for i in range(k, 0, -1):
         hop = k - i
         f = fanouts[hop]                                 # Algorithm 1's fanouts[i]
-        d_nbrs, d_offsets = one_hop_sample_all(view, delta, f, seed, hop)
+        d_nbrs, d_offsets = one_hop_sample_all(view, delta, f, seed, hop, direction)
         nbr_offsets = d_offsets + [o + len(d_nbrs) for o in nbr_offsets]
         nbrs = d_nbrs + nbrs
         delta = compute_next_delta(d_nbrs, node_ids)     # Delta_{i-1}

@@ -418,3 +418,133 @@ def test_distmult_closed_forms():
     pos2, nd2, ns2 = O.distmult_scores(h, rel_emb, prep2, rel, chunks)
     np.testing.assert_allclose(pos2, pos, rtol=1e-12)
     np.testing.assert_allclose(nd2, ns, rtol=1e-12)
+
+
+# ---------------------------------------------------------------- incoming + outgoing sampling (Section 4.1, Section 7.1)
+def _out_csr(n, off, nb):
+    """Rows by source, built edge by edge from the rows by destination."""
+    rows = [[] for _ in range(n)]
+    for d in range(n):
+        for s in nb[off[d]:off[d + 1]]:
+            rows[int(s)].append(d)
+    o, out = [0], []
+    for r in rows:
+        out.extend(sorted(r))
+        o.append(len(out))
+    return np.array(o), np.array(out, dtype=np.int64)
+
+
+def _undirected_bfs_levels(off, nb, ooff, onb, targets, k):
+    seen = set(targets)
+    frontier = list(targets)
+    levels = [list(targets)]
+    for _ in range(k):
+        nxt = set()
+        for v in frontier:
+            for u in list(nb[off[v]:off[v + 1]]) + list(onb[ooff[v]:ooff[v + 1]]):
+                if int(u) not in seen:
+                    nxt.add(int(u))
+        seen |= nxt
+        frontier = sorted(nxt)
+        levels.append(frontier)
+    return levels
+
+
+@pytest.mark.parametrize("seed", [0, 1])
+def test_inout_full_fanout_gives_undirected_bfs_levels(seed):
+    off, nb = _random_graph(70, 160, seed)
+    ooff, onb = _out_csr(70, off, nb)
+    assert ooff[-1] == off[-1]
+    f = int(max(np.diff(off).max(), np.diff(ooff).max()))
+    targets = [2, 41, 9]
+    k = 3
+    view = O.GraphView(off, nb, out_row_offsets=ooff, out_nbrs=onb)
+    d = O.sample_dense(view, targets, [f] * k, seed=8, direction="inout")
+    levels = _undirected_bfs_levels(off, nb, ooff, onb, targets, k)
+    nio = d["node_id_offsets"]
+    for j in range(k + 1):
+        i = k - j
+        assert d["node_ids"][nio[i]:nio[i + 1]] == levels[j]
+    sampled = d["node_ids"][nio[1]:]
+    for r, v in enumerate(sampled):              # incoming row, then outgoing row
+        got = d["nbrs"][d["nbr_offsets"][r]:d["nbr_offsets"][r + 1]]
+        assert got == [int(u) for u in nb[off[v]:off[v + 1]]] + [int(u) for u in onb[ooff[v]:ooff[v + 1]]]
+    for e, r in enumerate(d["repr_map"]):
+        assert d["node_ids"][r] == d["nbrs"][e]
+
+
+def test_inout_segments_and_reductions():
+    off, nb = _random_graph(150, 1500, 5)
+    ooff, onb = _out_csr(150, off, nb)
+    view = O.GraphView(off, nb, out_row_offsets=ooff, out_nbrs=onb)
+    targets = [3, 77, 140, 21]
+    fanouts = [3, 2]
+    d = O.sample_dense(view, targets, fanouts, seed=13, direction="inout")
+    d_in = O.sample_dense(view, targets, fanouts, seed=13, direction="in")
+    nio = d["node_id_offsets"]
+    k = len(fanouts)
+    sampled = d["node_ids"][nio[1]:]
+    for i in range(1, k + 1):
+        f = fanouts[k - i]
+        for r in range(nio[i] - nio[1], nio[i + 1] - nio[1]):
+            v = sampled[r]
+            seg = d["nbrs"][d["nbr_offsets"][r]:d["nbr_offsets"][r + 1]]
+            din, dout = int(off[v + 1] - off[v]), int(ooff[v + 1] - ooff[v])
+            assert len(seg) == min(din, f) + min(dout, f)
+            head, tail = seg[:min(din, f)], seg[min(din, f):]
+            in_row = [int(u) for u in nb[off[v]:off[v + 1]]]
+            out_row = [int(u) for u in onb[ooff[v]:ooff[v + 1]]]
+            # each part is a sub-sequence of its row (ascending positions, distinct slots)
+            it = iter(in_row)
+            assert all(any(u == w for w in it) for u in head)
+            it = iter(out_row)
+            assert all(any(u == w for w in it) for u in tail)
+            # the incoming part is exactly what incoming-only sampling of the same node at the same hop gives
+            assert head == O.one_hop_sample(view.row(v), f, 13, v, k - i)
+    # the targets' incoming parts coincide with incoming-only sampling of the same call
+    for r in range(len(targets)):
+        a = d["nbrs"][d["nbr_offsets"][nio[k] - nio[1] + r]:d["nbr_offsets"][nio[k] - nio[1] + r + 1]]
+        b = d_in["nbrs"][d_in["nbr_offsets"][d_in["node_id_offsets"][k] - d_in["node_id_offsets"][1] + r]:
+                         d_in["nbr_offsets"][d_in["node_id_offsets"][k] - d_in["node_id_offsets"][1] + r + 1]]
+        v = targets[r]
+        assert a[:len(b)] == b or int(off[v + 1] - off[v]) == 0
+    # no outgoing edges at all: "inout" is incoming-only sampling, bit for bit
+    empty = O.GraphView(off, nb, out_row_offsets=np.zeros(151, dtype=np.int64), out_nbrs=np.zeros(0, dtype=np.int64))
+    assert O.sample_dense(empty, targets, fanouts, 13, direction="inout") == d_in
+    # no incoming edges and a full fanout: "inout" over (nothing, A) is incoming-only sampling over A
+    full = int(np.diff(off).max())
+    swapped = O.GraphView(np.zeros(151, dtype=np.int64), np.zeros(0, dtype=np.int64), out_row_offsets=off, out_nbrs=nb)
+    assert O.sample_dense(swapped, targets, [full, full], 13, direction="inout") == \
+        O.sample_dense(O.GraphView(off, nb), targets, [full, full], 13, direction="in")
+
+
+def test_inout_directions_use_different_random_words():
+    # a node whose incoming and outgoing rows are the same list must not get the same subset twice by construction:
+    # over many seeds the two parts differ, and each direction's inclusion is uniform
+    row = np.arange(100, 140)
+    off = np.array([0, 40] + [40] * 140)
+    view = O.GraphView(off, row, out_row_offsets=off, out_nbrs=row)
+    same = 0
+    hits_out = np.zeros(40)
+    n_seeds = 1500
+    for s in range(n_seeds):
+        d = O.sample_dense(view, [0], [8], seed=s, direction="inout")
+        seg = d["nbrs"][:16]
+        assert len(seg) == 16
+        head, tail = seg[:8], seg[8:]
+        same += head == tail
+        assert tail == O.one_hop_sample(row, 8, s, 0, 0, O.OUT_SLOT_BASE)
+        for u in tail:
+            hits_out[u - 100] += 1
+    assert same <= 2
+    expect = n_seeds * 8 / 40
+    chi2 = ((hits_out - expect) ** 2 / expect).sum()
+    assert chi2 < 75.0      # 39 degrees of freedom: P(chi2 > 75) < 1e-3
+
+
+def test_inout_input_errors():
+    off, nb = _random_graph(30, 60, 0)
+    with pytest.raises(ValueError):
+        O.sample_dense(O.GraphView(off, nb), [1], [2], 0, direction="inout")     # no outgoing edge list
+    with pytest.raises(ValueError):
+        O.sample_dense(O.GraphView(off, nb), [1], [2], 0, direction="out")
