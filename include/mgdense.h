@@ -108,6 +108,24 @@ const char* mg_last_error(const mg_ctx* ctx);
 int mg_load_graph(mg_ctx* ctx, int64_t n_nodes, int64_t n_edges, const void* row_offsets,
                   int offsets_are_i64, const int32_t* nbrs, int ptrs_are_device);
 
+/* Load the second edge list of Section 4.1 as CSR over the same nodes: row v lists the
+ * destinations of v's outgoing edges, each row sorted by neighbour id; same array
+ * conventions as mg_load_graph, which must have been called before (a new mg_load_graph
+ * drops this list).  Needed by mg_set_sample_direction(MG_SAMPLE_INOUT).  The in-buffer
+ * filter applies to it as to the first list.  Errors: MG_ERR_STATE without a graph,
+ * MG_ERR_ARG on a malformed CSR, MG_ERR_OOM. */
+int mg_load_out_graph(mg_ctx* ctx, int64_t n_edges, const void* row_offsets, int offsets_are_i64,
+                      const int32_t* nbrs, int ptrs_are_device);
+
+/* Which edges one-hop sampling draws from (Section 4.1, Section 7.1): MG_SAMPLE_IN (default) =
+ * the rows given to mg_load_graph; MG_SAMPLE_INOUT = per node up to f of those followed by
+ * up to f rows of mg_load_out_graph (f = the hop's fanout, applied per direction; the
+ * outgoing draws are keyed by slots 65536 + t).  Errors: MG_ERR_ARG on an unknown value,
+ * MG_ERR_STATE for MG_SAMPLE_INOUT without an outgoing list. */
+#define MG_SAMPLE_IN 0
+#define MG_SAMPLE_INOUT 1
+int mg_set_sample_direction(mg_ctx* ctx, int direction);
+
 /* Split the nodes into n_parts physical partitions of ceil(n_nodes / n_parts) contiguous
  * ids (the last one short) — the sequential lookup table of Section 3.  All partitions
  * start non-resident except when n_parts == 1.  Drops any loaded feature table. */

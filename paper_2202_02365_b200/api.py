@@ -27,7 +27,7 @@ CORRUPT_DST, CORRUPT_SRC, CORRUPT_BOTH = 1, 2, 3
 
 # every symbol include/mgdense.h declares
 EXPORTS = [
-    "mg_create", "mg_destroy", "mg_last_error", "mg_load_graph", "mg_set_partitioning",
+    "mg_create", "mg_destroy", "mg_last_error", "mg_load_graph", "mg_load_out_graph", "mg_set_sample_direction", "mg_set_partitioning",
     "mg_load_features", "mg_set_resident", "mg_commit_resident", "mg_sample_many", "mg_sample_many_begin", "mg_sample_many_end", "mg_sample",
     "mg_dense_counts", "mg_dense_view", "mg_dense_free", "mg_model_create", "mg_model_free",
     "mg_forward", "mg_set_layer_window", "mg_keep_layer_outputs", "mg_forward_host_async", "mg_wait_output", "mg_forward_noalloc", "mg_gather_h0", "mg_layer_output", "mg_lp_prepare", "mg_lp_view", "mg_lp_free",
@@ -262,6 +262,19 @@ class Context:
                                            C.c_int(row_offsets.dtype == torch.int64), _ptr(nbrs),
                                            C.c_int(row_offsets.is_cuda)))
         self.n_nodes = n_nodes
+
+    def load_out_graph(self, row_offsets: torch.Tensor, nbrs: torch.Tensor):
+        """Second edge list (rows by source) for incoming + outgoing sampling."""
+        assert row_offsets.dtype in (torch.int32, torch.int64) and nbrs.dtype == torch.int32
+        assert row_offsets.is_cuda == nbrs.is_cuda
+        row_offsets, nbrs = row_offsets.contiguous(), nbrs.contiguous()
+        assert row_offsets.numel() - 1 == self.n_nodes
+        self._check(self.lib.mg_load_out_graph(self.handle, C.c_int64(nbrs.numel()), _ptr(row_offsets),
+                                               C.c_int(row_offsets.dtype == torch.int64), _ptr(nbrs),
+                                               C.c_int(row_offsets.is_cuda)))
+
+    def set_sample_direction(self, direction: str):
+        self._check(self.lib.mg_set_sample_direction(self.handle, C.c_int({"in": 0, "inout": 1}[direction])))
 
     def set_partitioning(self, n_parts: int):
         self._check(self.lib.mg_set_partitioning(self.handle, C.c_int32(n_parts)))

@@ -236,6 +236,16 @@ extern "C" int mg_create(mg_ctx** out, int device, void* stream) {
 static void free_view(mg_ctx* c) {
     if (c->view_owned) { cudaFree(c->view_off); cudaFree(c->view_nbrs); }
     c->view_off = nullptr; c->view_nbrs = nullptr; c->view_owned = false; c->view_edges = 0;
+    if (c->view_out_owned) { cudaFree(c->view_off_out); cudaFree(c->view_nbrs_out); }
+    c->view_off_out = nullptr; c->view_nbrs_out = nullptr; c->view_out_owned = false; c->view_edges_out = 0;
+}
+
+static void free_out_graph(mg_ctx* c) {
+    if (c->view_out_owned) { cudaFree(c->view_off_out); cudaFree(c->view_nbrs_out); }
+    c->view_off_out = nullptr; c->view_nbrs_out = nullptr; c->view_out_owned = false; c->view_edges_out = 0;
+    cudaFree(c->row_off_out); cudaFree(c->nbrs_out);
+    c->row_off_out = nullptr; c->nbrs_out = nullptr; c->n_edges_out = 0;
+    c->sample_inout = false;
 }
 
 static void free_features(mg_ctx* c) {
@@ -253,6 +263,7 @@ extern "C" int mg_destroy(mg_ctx* c) {
     for (auto& p : c->prof_pending) { cudaEventDestroy(p.second.first); cudaEventDestroy(p.second.second); }
     free_view(c);
     free_features(c);
+    free_out_graph(c);
     cudaFree(c->row_off); cudaFree(c->nbrs); cudaFree(c->d_slot_of_part); cudaFree(c->d_res_prefix); cudaFree(c->d_flags);
     cudaFree(c->ws_x); cudaFree(c->ws_h[0]); cudaFree(c->ws_h[1]);
     cudaEventDestroy(c->ev_fwd_done); cudaEventDestroy(c->ev_out_done); cudaEventDestroy(c->ev_user);
@@ -314,28 +325,25 @@ static int upload_slot_map(mg_ctx* c) {
     return MG_OK;
 }
 
-static int rebuild_view(mg_ctx* c) {
-    bool all = true, any = false;
-    for (int p = 0; p < c->n_parts; ++p) { all = all && c->slot_of_part[p] >= 0; any = any || c->slot_of_part[p] >= 0; }
-    if (!any) {   // nothing in the buffer: there is no view, and sampling refuses to run
-        free_view(c);
-        return MG_OK;
-    }
+// One edge list's in-buffer view: the rows of resident nodes restricted to resident neighbours (the list itself when
+// every partition is resident).
+static int rebuild_one_view(mg_ctx* c, bool all, const int64_t* row_off, const int32_t* nbrs, int64_t n_edges,
+                            int64_t** view_off, int32_t** view_nbrs, bool* owned, int64_t* view_edges) {
     if (all) {
-        free_view(c);
-        c->view_off = c->row_off; c->view_nbrs = c->nbrs; c->view_edges = c->n_edges; c->view_owned = false;
+        if (*owned) { cudaFree(*view_off); cudaFree(*view_nbrs); }
+        *view_off = const_cast<int64_t*>(row_off); *view_nbrs = const_cast<int32_t*>(nbrs); *view_edges = n_edges; *owned = false;
         return MG_OK;
     }
-    if (!c->view_owned) {
-        c->view_off = nullptr; c->view_nbrs = nullptr;
-        if (cudaMalloc((void**)&c->view_off, sizeof(int64_t) * (c->n_nodes + 1)) != cudaSuccess ||
-            cudaMalloc((void**)&c->view_nbrs, sizeof(int32_t) * std::max<int64_t>(c->n_edges, 1)) != cudaSuccess) {
+    if (!*owned) {
+        *view_off = nullptr; *view_nbrs = nullptr;
+        if (cudaMalloc((void**)view_off, sizeof(int64_t) * (c->n_nodes + 1)) != cudaSuccess ||
+            cudaMalloc((void**)view_nbrs, sizeof(int32_t) * std::max<int64_t>(n_edges, 1)) != cudaSuccess) {
             cudaGetLastError();
-            cudaFree(c->view_off);
-            c->view_off = nullptr; c->view_nbrs = nullptr;
+            cudaFree(*view_off);
+            *view_off = nullptr; *view_nbrs = nullptr;
             return mg_fail(c, MG_ERR_OOM, "allocation of the in-buffer graph view failed");
         }
-        c->view_owned = true;
+        *owned = true;
     }
     const int64_t n = c->n_nodes;
     const int64_t ntiles = (n + kTile - 1) / kTile;
@@ -351,11 +359,11 @@ static int rebuild_view(mg_ctx* c) {
     }
     const int grid = mg_grid(c, 8);
     cudaStream_t st = c->stream;
-    k_view_count<<<grid, kThreads, 0, st>>>(c->row_off, c->nbrs, n, (uint32_t)c->part_size, c->d_slot_of_part, cnt);
+    k_view_count<<<grid, kThreads, 0, st>>>(row_off, nbrs, n, (uint32_t)c->part_size, c->d_slot_of_part, cnt);
     k_scan64_reduce<<<grid, kThreads, 0, st>>>(cnt, n, tiles);
     k_scan64_tiles<<<1, kThreads, 0, st>>>(tiles, ntiles, d_total);
-    k_scan64_down<<<grid, kThreads, 0, st>>>(cnt, n, tiles, c->view_off);
-    k_view_fill<<<grid, kThreads, 0, st>>>(c->row_off, c->nbrs, n, (uint32_t)c->part_size, c->d_slot_of_part, c->view_off, c->view_nbrs);
+    k_scan64_down<<<grid, kThreads, 0, st>>>(cnt, n, tiles, *view_off);
+    k_view_fill<<<grid, kThreads, 0, st>>>(row_off, nbrs, n, (uint32_t)c->part_size, c->d_slot_of_part, *view_off, *view_nbrs);
     c->launches += 5;
     int64_t total = 0;
     cudaError_t e = cudaMemcpyAsync(&total, d_total, sizeof(int64_t), cudaMemcpyDeviceToHost, st);
@@ -363,7 +371,73 @@ static int rebuild_view(mg_ctx* c) {
     if (e == cudaSuccess) e = cudaGetLastError();
     cudaFree(cnt); cudaFree(tiles); cudaFree(d_total);
     if (e != cudaSuccess) return mg_cuda_fail(c, e, "rebuild of the in-buffer graph view");
-    c->view_edges = total;
+    *view_edges = total;
+    return MG_OK;
+}
+
+static int rebuild_view(mg_ctx* c) {
+    bool all = true, any = false;
+    for (int p = 0; p < c->n_parts; ++p) { all = all && c->slot_of_part[p] >= 0; any = any || c->slot_of_part[p] >= 0; }
+    if (!any) {   // nothing in the buffer: there is no view, and sampling refuses to run
+        free_view(c);
+        return MG_OK;
+    }
+    int rc = rebuild_one_view(c, all, c->row_off, c->nbrs, c->n_edges, &c->view_off, &c->view_nbrs, &c->view_owned, &c->view_edges);
+    if (rc == MG_OK && c->row_off_out)
+        rc = rebuild_one_view(c, all, c->row_off_out, c->nbrs_out, c->n_edges_out, &c->view_off_out, &c->view_nbrs_out,
+                              &c->view_out_owned, &c->view_edges_out);
+    return rc;
+}
+
+// Copy one CSR to the device and validate it there; *row_off_out / *nbrs_out own the copies.
+static int upload_csr(mg_ctx* c, int64_t n_nodes, int64_t n_edges, const void* row_offsets, int offsets_are_i64,
+                      const int32_t* nbrs, int ptrs_are_device, int64_t** d_row_off, int32_t** d_nbrs) {
+    const cudaMemcpyKind kind = ptrs_are_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+    *d_row_off = nullptr; *d_nbrs = nullptr;
+    if (cudaMalloc((void**)d_row_off, sizeof(int64_t) * (n_nodes + 1)) != cudaSuccess ||
+        cudaMalloc((void**)d_nbrs, sizeof(int32_t) * std::max<int64_t>(n_edges, 1)) != cudaSuccess) {
+        cudaGetLastError();
+        cudaFree(*d_row_off); *d_row_off = nullptr; *d_nbrs = nullptr;
+        return mg_fail(c, MG_ERR_OOM, "allocation of the graph store failed");
+    }
+    auto drop = [&]() { cudaFree(*d_row_off); cudaFree(*d_nbrs); *d_row_off = nullptr; *d_nbrs = nullptr; };
+    cudaStream_t st = c->stream;
+    cudaError_t e = cudaSuccess;
+    if (offsets_are_i64) {
+        e = cudaMemcpyAsync(*d_row_off, row_offsets, sizeof(int64_t) * (n_nodes + 1), kind, st);
+    } else {
+        int32_t* tmp = nullptr;
+        e = cudaMalloc((void**)&tmp, sizeof(int32_t) * (n_nodes + 1));
+        if (e == cudaSuccess) e = cudaMemcpyAsync(tmp, row_offsets, sizeof(int32_t) * (n_nodes + 1), kind, st);
+        if (e == cudaSuccess) {
+            k_widen_offsets<<<mg_grid(c, 4), kThreads, 0, st>>>(tmp, *d_row_off, n_nodes + 1);
+            c->launches++;
+            e = cudaStreamSynchronize(st);
+        }
+        cudaFree(tmp);
+    }
+    if (e == cudaSuccess && n_edges > 0) e = cudaMemcpyAsync(*d_nbrs, nbrs, sizeof(int32_t) * n_edges, kind, st);
+    // validate on the device; only the two end offsets come back
+    uint32_t* flags = nullptr;
+    if (e == cudaSuccess) e = cudaMalloc((void**)&flags, sizeof(uint32_t));
+    if (e != cudaSuccess) { cudaGetLastError(); drop(); return mg_cuda_fail(c, e, "graph upload"); }
+    cudaMemsetAsync(flags, 0, sizeof(uint32_t), st);
+    k_check_graph<<<mg_grid(c, 8), kThreads, 0, st>>>(*d_row_off, n_nodes, *d_nbrs, n_edges, flags);
+    c->launches++;
+    uint32_t h_flags = 0;
+    int64_t ends[2] = {0, 0};
+    cudaMemcpyAsync(&h_flags, flags, sizeof(uint32_t), cudaMemcpyDeviceToHost, st);
+    cudaMemcpyAsync(&ends[0], *d_row_off, sizeof(int64_t), cudaMemcpyDeviceToHost, st);
+    cudaMemcpyAsync(&ends[1], *d_row_off + n_nodes, sizeof(int64_t), cudaMemcpyDeviceToHost, st);
+    e = cudaStreamSynchronize(st);
+    cudaFree(flags);
+    if (e != cudaSuccess) { drop(); return mg_cuda_fail(c, e, "graph upload"); }
+    if (h_flags || ends[0] != 0 || ends[1] != n_edges) {
+        drop();
+        return mg_fail(c, MG_ERR_ARG, "malformed CSR: %s", (h_flags & 2) ? "neighbour id out of range"
+                                                            : (h_flags & 1) ? "row offsets decrease"
+                                                                            : "row_offsets[0] != 0 or row_offsets[n_nodes] != n_edges");
+    }
     return MG_OK;
 }
 
@@ -376,55 +450,37 @@ extern "C" int mg_load_graph(mg_ctx* c, int64_t n_nodes, int64_t n_edges, const 
     MG_CUDA(c, cudaStreamSynchronize(c->stream));
     free_view(c);
     free_features(c);
+    free_out_graph(c);
     cudaFree(c->row_off); cudaFree(c->nbrs);
     c->row_off = nullptr; c->nbrs = nullptr; c->n_nodes = 0; c->n_edges = 0;
-    const cudaMemcpyKind kind = ptrs_are_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
-    if (cudaMalloc((void**)&c->row_off, sizeof(int64_t) * (n_nodes + 1)) != cudaSuccess ||
-        cudaMalloc((void**)&c->nbrs, sizeof(int32_t) * std::max<int64_t>(n_edges, 1)) != cudaSuccess) {
-        cudaGetLastError();
-        cudaFree(c->row_off); c->row_off = nullptr;
-        return mg_fail(c, MG_ERR_OOM, "allocation of the graph store failed");
-    }
-    cudaStream_t st = c->stream;
-    if (offsets_are_i64) {
-        MG_CUDA(c, cudaMemcpyAsync(c->row_off, row_offsets, sizeof(int64_t) * (n_nodes + 1), kind, st));
-    } else {
-        int32_t* tmp = nullptr;
-        MG_CUDA(c, cudaMalloc((void**)&tmp, sizeof(int32_t) * (n_nodes + 1)));
-        cudaError_t e = cudaMemcpyAsync(tmp, row_offsets, sizeof(int32_t) * (n_nodes + 1), kind, st);
-        if (e == cudaSuccess) {
-            k_widen_offsets<<<mg_grid(c, 4), kThreads, 0, st>>>(tmp, c->row_off, n_nodes + 1);
-            c->launches++;
-            e = cudaStreamSynchronize(st);
-        }
-        cudaFree(tmp);
-        if (e != cudaSuccess) return mg_cuda_fail(c, e, "offset upload");
-    }
-    if (n_edges > 0) MG_CUDA(c, cudaMemcpyAsync(c->nbrs, nbrs, sizeof(int32_t) * n_edges, kind, st));
-    // validate on the device; only the two end offsets come back
-    uint32_t* flags = nullptr;
-    MG_CUDA(c, cudaMalloc((void**)&flags, sizeof(uint32_t)));
-    cudaMemsetAsync(flags, 0, sizeof(uint32_t), st);
-    k_check_graph<<<mg_grid(c, 8), kThreads, 0, st>>>(c->row_off, n_nodes, c->nbrs, n_edges, flags);
-    c->launches++;
-    uint32_t h_flags = 0;
-    int64_t ends[2] = {0, 0};
-    cudaMemcpyAsync(&h_flags, flags, sizeof(uint32_t), cudaMemcpyDeviceToHost, st);
-    cudaMemcpyAsync(&ends[0], c->row_off, sizeof(int64_t), cudaMemcpyDeviceToHost, st);
-    cudaMemcpyAsync(&ends[1], c->row_off + n_nodes, sizeof(int64_t), cudaMemcpyDeviceToHost, st);
-    cudaError_t e = cudaStreamSynchronize(st);
-    cudaFree(flags);
-    if (e != cudaSuccess) return mg_cuda_fail(c, e, "graph upload");
-    if (h_flags || ends[0] != 0 || ends[1] != n_edges) {
-        cudaFree(c->row_off); cudaFree(c->nbrs);
-        c->row_off = nullptr; c->nbrs = nullptr;
-        return mg_fail(c, MG_ERR_ARG, "malformed CSR: %s", (h_flags & 2) ? "neighbour id out of range"
-                                                            : (h_flags & 1) ? "row offsets decrease"
-                                                                            : "row_offsets[0] != 0 or row_offsets[n_nodes] != n_edges");
-    }
+    const int rc = upload_csr(c, n_nodes, n_edges, row_offsets, offsets_are_i64, nbrs, ptrs_are_device, &c->row_off, &c->nbrs);
+    if (rc) return rc;
     c->n_nodes = n_nodes;
     c->n_edges = n_edges;
     return mg_set_partitioning(c, 1);
+}
+
+extern "C" int mg_load_out_graph(mg_ctx* c, int64_t n_edges, const void* row_offsets, int offsets_are_i64, const int32_t* nbrs,
+                                 int ptrs_are_device) {
+    if (!c) return MG_ERR_ARG;
+    if (!row_offsets || (n_edges > 0 && !nbrs)) return mg_fail(c, MG_ERR_ARG, "null argument");
+    if (n_edges < 0) return mg_fail(c, MG_ERR_ARG, "n_edges must not be negative");
+    if (!c->row_off) return mg_fail(c, MG_ERR_STATE, "no graph loaded");
+    MG_CUDA(c, cudaSetDevice(c->device));
+    MG_CUDA(c, cudaStreamSynchronize(c->stream));
+    free_out_graph(c);
+    const int rc = upload_csr(c, c->n_nodes, n_edges, row_offsets, offsets_are_i64, nbrs, ptrs_are_device, &c->row_off_out, &c->nbrs_out);
+    if (rc) return rc;
+    c->n_edges_out = n_edges;
+    return rebuild_view(c);   // the in-buffer filter of the current resident set
+}
+
+extern "C" int mg_set_sample_direction(mg_ctx* c, int direction) {
+    if (!c) return MG_ERR_ARG;
+    if (direction != MG_SAMPLE_IN && direction != MG_SAMPLE_INOUT) return mg_fail(c, MG_ERR_ARG, "unknown sampling direction");
+    if (direction == MG_SAMPLE_INOUT && !c->row_off_out) return mg_fail(c, MG_ERR_STATE, "no outgoing edge list loaded");
+    c->sample_inout = direction == MG_SAMPLE_INOUT;
+    return MG_OK;
 }
 
 extern "C" int mg_set_partitioning(mg_ctx* c, int32_t n_parts) {

@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#define MG_OUT_SLOT_BASE 65536  // first draw slot of the outgoing direction (incoming + outgoing sampling)
 #define MG_SLOT_BITS 24  // per-batch id-table slots are addressed with 24 bits (<= 16M slots)
 
 // Philox4x32-10 (Salmon et al., SC'11); the draw of (seed, node, hop, slot) is word slot % 4

@@ -76,6 +76,15 @@ struct mg_ctx {
     int32_t* view_nbrs = nullptr;
     int64_t view_edges = 0;
     bool view_owned = false;
+    // second edge list (rows by source) and its in-buffer view; sample_inout = draw from both lists
+    int64_t n_edges_out = 0;
+    int64_t* row_off_out = nullptr;
+    int32_t* nbrs_out = nullptr;
+    int64_t* view_off_out = nullptr;
+    int32_t* view_nbrs_out = nullptr;
+    int64_t view_edges_out = 0;
+    bool view_out_owned = false;
+    bool sample_inout = false;
 
     // partitioning and buffer
     int32_t n_parts = 1;
@@ -137,7 +146,7 @@ struct mg_ctx {
 // everything the sampler's captured device work depends on
 struct SampleSignature {
     int32_t B, k, table_size, fanouts[MG_MAX_HOPS];
-    int64_t T, cap_batch, cap_nodes, cap_entries, n_nodes, part_size;
+    int64_t T, cap_batch, cap_nodes, cap_entries, n_nodes, part_size, inout;
     const void* ptrs[32];
 };
 
@@ -157,6 +166,9 @@ struct mg_dense {
     int32_t* ent_off = nullptr;     // [cap_nodes + 1] start of each sampled node's entries
     int64_t* node_r0 = nullptr;     // [cap_nodes] start of the node's row in the in-buffer view
     uint32_t* node_deg = nullptr;   // [cap_nodes] its (resident) degree
+    int64_t* node_r0_out = nullptr; // the same for the outgoing edge list (incoming + outgoing sampling only)
+    uint32_t* node_deg_out = nullptr;
+    int64_t cap_nodes_out = 0;
     int32_t* ent_nbrs = nullptr;    // [cap_entries] neighbour ids
     int32_t* ent_repr = nullptr;    // [cap_entries] neighbour's local row in its batch
     int32_t* node_off = nullptr;    // [(k+1) * (B+1)] arena index where batch b's hop-h nodes start

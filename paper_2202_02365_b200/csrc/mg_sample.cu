@@ -153,16 +153,25 @@ k_init_targets(DenseHeader* hdr, const int32_t* __restrict__ targets,
 // -------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads)
 k_count(const DenseHeader* hdr, int hop, int32_t fanout, const int32_t* __restrict__ nodes,
-        const int64_t* __restrict__ row_off, int32_t* ent_off, int64_t* node_r0, uint32_t* node_deg) {
+        const int64_t* __restrict__ row_off, int32_t* ent_off, int64_t* node_r0, uint32_t* node_deg,
+        const int64_t* __restrict__ row_off_out, int64_t* node_r0_out, uint32_t* node_deg_out) {
     if (hdr->status) return;
     const int32_t lo = hdr->hop_base[hop], hi = hdr->hop_base[hop + 1];
     for (int32_t i = lo + blockIdx.x * blockDim.x + threadIdx.x; i < hi; i += gridDim.x * blockDim.x) {
         const int32_t v = nodes[i];
         const int64_t r0 = row_off[v];
         const int64_t d = row_off[v + 1] - r0;
-        ent_off[i] = (int32_t)(d < (int64_t)fanout ? d : (int64_t)fanout);
+        int32_t n = (int32_t)(d < (int64_t)fanout ? d : (int64_t)fanout);
         node_r0[i] = r0;        // the one random look-up of the row bounds; k_pick reads these coalesced
         node_deg[i] = (uint32_t)d;
+        if (row_off_out) {      // incoming + outgoing sampling: up to `fanout` of each list
+            const int64_t q0 = row_off_out[v];
+            const int64_t dq = row_off_out[v + 1] - q0;
+            n += (int32_t)(dq < (int64_t)fanout ? dq : (int64_t)fanout);
+            node_r0_out[i] = q0;
+            node_deg_out[i] = (uint32_t)dq;
+        }
+        ent_off[i] = n;
     }
 }
 
@@ -189,7 +198,21 @@ struct PickArgs {
     int32_t* ent_nbrs;
     int32_t* ent_repr;  // receives the batch id of the entry (k_insert turns it into the id-table slot)
     const uint64_t* seeds;
+    // second direction of incoming + outgoing sampling: its picks follow the first direction's min(degree, fanout)
+    // entries of the node and its draws use slots slot_base + t
+    const uint32_t* pre_deg;   // nullptr for the first (or only) direction
+    uint32_t slot_base;
 };
+
+// first entry of node i's picks in this launch's direction
+__device__ __forceinline__ int32_t pick_base(const PickArgs& a, int32_t i) {
+    int32_t out0 = a.ent_off[i];
+    if (a.pre_deg) {
+        const uint32_t d0 = a.pre_deg[i];
+        out0 += (int32_t)(d0 < (uint32_t)a.fanout ? d0 : (uint32_t)a.fanout);
+    }
+    return out0;
+}
 
 // A pick goes to its place in the entry arena; ent_repr carries the batch id until k_insert replaces it.
 __device__ __forceinline__ void store_pick(const PickArgs& a, bool valid, int32_t b, int32_t u, int32_t out_pos) {
@@ -217,7 +240,7 @@ __global__ void __launch_bounds__(kThreads) k_pick(PickArgs a) {
         if (node_ok) {
             v = a.nodes[i];
             b = a.node_batch[i];
-            out0 = a.ent_off[i];
+            out0 = pick_base(a, i);
             r0 = a.node_r0[i];
             d = (int64_t)a.node_deg[i];
         }
@@ -230,7 +253,7 @@ __global__ void __launch_bounds__(kThreads) k_pick(PickArgs a) {
         uint32_t x = 0xFFFFFFFFu, jt = 0, pick = 0xFFFFFFFFu;
         if (floyd && gl < f) {
             jt = (uint32_t)(d - f) + (uint32_t)gl;
-            x = __umulhi(draw_word(a.seeds[b], (uint32_t)v, (uint32_t)a.hop, (uint32_t)gl), jt + 1u);
+            x = __umulhi(draw_word(a.seeds[b], (uint32_t)v, (uint32_t)a.hop, a.slot_base + (uint32_t)gl), jt + 1u);
         }
         for (int t = 0; t < f; ++t) {
             const uint32_t xt = __shfl_sync(0xFFFFFFFFu, x, gshift + t);
@@ -278,7 +301,7 @@ __global__ void __launch_bounds__(kThreads) k_pick_wide(PickArgs a) {
         if (node_ok) {
             v = a.nodes[i];
             b = a.node_batch[i];
-            out0 = a.ent_off[i];
+            out0 = pick_base(a, i);
             r0 = a.node_r0[i];
             d = (int64_t)a.node_deg[i];
         }
@@ -286,7 +309,7 @@ __global__ void __launch_bounds__(kThreads) k_pick_wide(PickArgs a) {
         if (floyd) {
             for (int t = lane; t < f; t += 32) {
                 const uint32_t jt = (uint32_t)(d - f) + (uint32_t)t;
-                xs[t] = __umulhi(draw_word(a.seeds[b], (uint32_t)v, (uint32_t)a.hop, (uint32_t)t), jt + 1u);
+                xs[t] = __umulhi(draw_word(a.seeds[b], (uint32_t)v, (uint32_t)a.hop, a.slot_base + (uint32_t)t), jt + 1u);
             }
             __syncwarp();
             for (int t = 0; t < f; ++t) {
@@ -881,6 +904,7 @@ static int dense_alloc(mg_ctx* ctx, mg_dense* d, int32_t B, int32_t k, int64_t c
         if ((rc = dev_realloc(ctx, &d->ent_off, (size_t)cap_nodes + 1))) return rc;
         if ((rc = dev_realloc(ctx, &d->node_r0, (size_t)cap_nodes))) return rc;
         if ((rc = dev_realloc(ctx, &d->node_deg, (size_t)cap_nodes))) return rc;
+        d->cap_nodes_out = 0;
         if ((rc = dev_realloc(ctx, &d->newlist[0], (size_t)cap_nodes))) return rc;
         if ((rc = dev_realloc(ctx, &d->newlist[1], (size_t)cap_nodes))) return rc;
         const int64_t sort_tiles = (cap_nodes + kSortTile - 1) / kSortTile;
@@ -898,6 +922,12 @@ static int dense_alloc(mg_ctx* ctx, mg_dense* d, int32_t B, int32_t k, int64_t c
         if ((rc = dev_realloc(ctx, &d->ent_nbrs, (size_t)cap_entries))) return rc;
         if ((rc = dev_realloc(ctx, &d->ent_repr, (size_t)cap_entries))) return rc;
         d->cap_entries = cap_entries;
+    }
+    if (ctx->sample_inout && d->cap_nodes_out < d->cap_nodes) {
+        d->cap_nodes_out = 0;
+        if ((rc = dev_realloc(ctx, &d->node_r0_out, (size_t)d->cap_nodes))) return rc;
+        if ((rc = dev_realloc(ctx, &d->node_deg_out, (size_t)d->cap_nodes))) return rc;
+        d->cap_nodes_out = d->cap_nodes;
     }
     const int64_t need_table = (int64_t)B * table_size;
     if (d->alloc_table < need_table) {
@@ -1010,6 +1040,8 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
         if (fanouts[h] <= 0 || fanouts[h] > MG_MAX_FANOUT) return mg_fail(ctx, MG_ERR_ARG, "fanouts must be in [1, %d]", MG_MAX_FANOUT);
     if (!ctx->row_off) return mg_fail(ctx, MG_ERR_STATE, "no graph loaded");
     if (!ctx->view_off) return mg_fail(ctx, MG_ERR_NONRESIDENT, "no partition is resident");
+    const bool inout = ctx->sample_inout;
+    if (inout && !ctx->view_off_out) return mg_fail(ctx, MG_ERR_STATE, "no outgoing edge list loaded");
     if (target_offsets[0] != 0) return mg_fail(ctx, MG_ERR_ARG, "target_offsets[0] must be 0");
     for (int b = 0; b < n_batches; ++b)
         if (target_offsets[b + 1] < target_offsets[b]) return mg_fail(ctx, MG_ERR_ARG, "target_offsets must be non-decreasing");
@@ -1025,7 +1057,7 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
         double level = (double)(target_offsets[b + 1] - target_offsets[b]);  // nodes that can be new at this hop
         double nodes = level, entries = 0;
         for (int h = 0; h < k; ++h) {
-            level = std::min(level, (double)N) * fanouts[h];
+            level = std::min(level, (double)N) * fanouts[h] * (ctx->sample_inout ? 2 : 1);
             entries += level;
             nodes += level;
         }
@@ -1150,7 +1182,8 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
         const int32_t f = fanouts[h];
         {
             ProfScope ps(ctx, PH_SAMPLE_COUNT, 1);
-            k_count<<<grid, kThreads, 0, st>>>(d->hdr, h, f, d->nodes, ctx->view_off, d->ent_off, d->node_r0, d->node_deg);
+            k_count<<<grid, kThreads, 0, st>>>(d->hdr, h, f, d->nodes, ctx->view_off, d->ent_off, d->node_r0, d->node_deg,
+                                               inout ? ctx->view_off_out : nullptr, d->node_r0_out, d->node_deg_out);
         }
         {
             ProfScope ps(ctx, PH_SAMPLE_SCAN, 4);
@@ -1160,15 +1193,19 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
         }
         {
             ProfScope ps(ctx, PH_SAMPLE_PICK, 1);
-            PickArgs a{d->hdr, h, f, d->nodes, d->node_batch, d->node_r0, d->node_deg, ctx->view_nbrs, d->ent_off, d->ent_nbrs,
-                       d->ent_repr, d->d_seeds};
-            if (f <= 4) k_pick<4><<<grid, kThreads, 0, st>>>(a);
-            else if (f <= 8) k_pick<8><<<grid, kThreads, 0, st>>>(a);
-            else if (f <= 16) k_pick<16><<<grid, kThreads, 0, st>>>(a);
-            else if (f <= 32) k_pick<32><<<grid, kThreads, 0, st>>>(a);
-            else {
-                const size_t wide_smem = (size_t)(kThreads / 32) * 2 * f * sizeof(uint32_t);   // 64 KiB at the largest fanout
-                k_pick_wide<<<grid, kThreads, wide_smem, st>>>(a);
+            for (int dir = 0; dir < (inout ? 2 : 1); ++dir) {
+                PickArgs a{d->hdr, h, f, d->nodes, d->node_batch, dir ? d->node_r0_out : d->node_r0, dir ? d->node_deg_out : d->node_deg,
+                           dir ? ctx->view_nbrs_out : ctx->view_nbrs, d->ent_off, d->ent_nbrs, d->ent_repr, d->d_seeds,
+                           dir ? d->node_deg : nullptr, dir ? (uint32_t)MG_OUT_SLOT_BASE : 0u};
+                if (f <= 4) k_pick<4><<<grid, kThreads, 0, st>>>(a);
+                else if (f <= 8) k_pick<8><<<grid, kThreads, 0, st>>>(a);
+                else if (f <= 16) k_pick<16><<<grid, kThreads, 0, st>>>(a);
+                else if (f <= 32) k_pick<32><<<grid, kThreads, 0, st>>>(a);
+                else {
+                    const size_t wide_smem = (size_t)(kThreads / 32) * 2 * f * sizeof(uint32_t);   // 64 KiB at the largest fanout
+                    k_pick_wide<<<grid, kThreads, wide_smem, st>>>(a);
+                }
+                if (dir) ctx->launches++;
             }
             InsertArgs ia{d->hdr, h, d->ent_nbrs, d->ent_repr, d->hkeys, tg, d->newlist[0], d->cap_nodes, id_bits,
                           k, d->cum, d->hvals, batch_cnt + (size_t)h * B, (int32_t)cap_batch};
@@ -1214,10 +1251,13 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
     memset(&sig, 0, sizeof(sig));
     sig.B = B; sig.k = k; sig.T = 0; sig.table_size = table_size; sig.cap_batch = cap_batch;   // (the device work does not depend on T)
     sig.cap_nodes = d->cap_nodes; sig.cap_entries = d->cap_entries; sig.n_nodes = ctx->n_nodes; sig.part_size = ctx->part_size;
+    sig.inout = inout ? 1 : 0;
     for (int h = 0; h < k; ++h) sig.fanouts[h] = fanouts[h];
     const void* ptrs[] = {d->hdr, d->nodes, d->node_batch, d->ent_off, d->node_r0, d->node_deg, d->newlist[0], d->newlist[1],
                           d->scan_tmp, d->sort_hist, d->ent_nbrs, d->ent_repr, d->hkeys, d->hvals, d->node_off, d->cum, d->rowbase,
-                          d->d_ent_hop, d->d_seeds, d->h_stage, d->h_pinned_dev, ctx->view_off, ctx->view_nbrs, ctx->d_slot_of_part, st};
+                          d->d_ent_hop, d->d_seeds, d->h_stage, d->h_pinned_dev, ctx->view_off, ctx->view_nbrs, ctx->d_slot_of_part, st,
+                          inout ? (const void*)ctx->view_off_out : nullptr, inout ? (const void*)ctx->view_nbrs_out : nullptr,
+                          d->node_r0_out, d->node_deg_out};
     static_assert(sizeof(ptrs) <= sizeof(sig.ptrs), "signature too small");
     memcpy(sig.ptrs, ptrs, sizeof(ptrs));
     const bool use_graph = ctx->sample_graphs && !ctx->prof_on && !getenv("MG_NO_SAMPLE_GRAPH");
@@ -1374,7 +1414,7 @@ extern "C" int mg_dense_view(mg_ctx* ctx, mg_dense* d, int32_t batch, mg_dense_a
 extern "C" int mg_dense_free(mg_dense* d) {
     if (!d) return MG_OK;
     cudaSetDevice(d->device);
-    cudaFree(d->hdr); cudaFree(d->nodes); cudaFree(d->node_batch); cudaFree(d->ent_off); cudaFree(d->node_r0); cudaFree(d->node_deg);
+    cudaFree(d->hdr); cudaFree(d->nodes); cudaFree(d->node_batch); cudaFree(d->ent_off); cudaFree(d->node_r0); cudaFree(d->node_deg); cudaFree(d->node_r0_out); cudaFree(d->node_deg_out);
     cudaFree(d->ent_nbrs); cudaFree(d->ent_repr); cudaFree(d->node_off); cudaFree(d->cum);
     cudaFree(d->rowbase); cudaFree(d->hkeys); cudaFree(d->hvals); cudaFree(d->newlist[0]);
     cudaFree(d->newlist[1]); cudaFree(d->d_seeds); cudaFree(d->batch_cnt); cudaFree(d->scan_tmp); cudaFree(d->sort_hist);

@@ -116,6 +116,23 @@ def build_csr(src: torch.Tensor, dst: torch.Tensor, n_nodes: int,
     return Graph(n_nodes, offsets, nbrs, erel)
 
 
+def transpose_csr(graph: Graph) -> Graph:
+    """The second edge list of the same edges: row = source, neighbours = destinations ascending."""
+    n = graph.n_nodes
+    counts = graph.row_offsets[1:] - graph.row_offsets[:-1]
+    dst = torch.repeat_interleave(torch.arange(n, dtype=torch.int64, device=graph.nbrs.device), counts)
+    key = torch.sort(graph.nbrs.to(torch.int64) * n + dst).values
+    del dst
+    rows = torch.div(key, n, rounding_mode="floor")
+    nbrs = (key - rows * n).to(torch.int32)
+    del key
+    out_counts = torch.bincount(rows, minlength=n)
+    del rows
+    offsets = torch.zeros(n + 1, dtype=torch.int64, device=nbrs.device)
+    torch.cumsum(out_counts, 0, out=offsets[1:])
+    return Graph(n, offsets, nbrs, None)
+
+
 def erdos_renyi_graph(n_nodes, n_edges, seed=0, device="cpu") -> Graph:
     s, d = erdos_renyi_edges(n_nodes, n_edges, seed, device)
     return build_csr(s, d, n_nodes)

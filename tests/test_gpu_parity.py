@@ -649,3 +649,59 @@ def test_sample_handle_reuse_replays_and_recaptures(tiny):
         for b in range(2):
             ref = O.sample_dense(view, targets[offs[b]:offs[b + 1]].tolist(), fanouts, seeds[b])
             assert_dense_equal(d.view(b), ref)
+
+
+def test_incoming_and_outgoing_sampling(tiny):
+    """Section 4.1's second edge list: up to f incoming then up to f outgoing neighbours per node."""
+    g, feats = tiny
+    gt = inputs.transpose_csr(g)
+    ctx = make_ctx(g, feats)
+    with pytest.raises(mg.MgError) as e:
+        ctx.set_sample_direction("inout")             # no outgoing list yet
+    assert e.value.code == -2
+    ctx.load_out_graph(gt.row_offsets.cuda(), gt.nbrs.cuda())
+    ctx.set_sample_direction("inout")
+    view = O.GraphView(g.row_offsets.numpy(), g.nbrs.numpy(), out_row_offsets=gt.row_offsets.numpy(), out_nbrs=gt.nbrs.numpy())
+    layers = inputs.random_bias_layers([16, 16, 16, 8], seed=9)
+    model = ctx.model(layers, mg.GEMM_FP32)
+    sizes = [300, 1, 0, 257]
+    tg = [inputs.distinct_targets(10_000, s, seed=40 + i) for i, s in enumerate(sizes)]
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    seeds = [77, 78, 79, 80]
+    for fanouts in ([10, 5, 2], [40, 3, 1]):          # the second one takes the any-fanout pick kernel on the first hop
+        d = ctx.sample_many(torch.cat(tg), offs, fanouts, seeds)
+        out = torch.empty((int(offs[-1]), 8), dtype=torch.float32, device="cuda")
+        ctx.forward(model, d, out)
+        for b in range(len(sizes)):
+            ref = O.sample_dense(view, tg[b].tolist(), fanouts, seeds[b], direction="inout")
+            assert_dense_equal(d.view(b), ref)
+            if sizes[b]:
+                ref_out = O.forward(ref, feats.numpy()[ref["node_ids"]], [(w.numpy(), n.numpy(), bb.numpy()) for w, n, bb in layers])
+                close(out[offs[b]:offs[b + 1]].cpu().numpy(), ref_out, RTOL_AGG)
+    # back to incoming-only sampling on the same context and handle
+    ctx.set_sample_direction("in")
+    d = ctx.sample_many(torch.cat(tg), offs, [10, 5, 2], seeds, out=d)
+    assert_dense_equal(d.view(0), O.sample_dense(view, tg[0].tolist(), [10, 5, 2], seeds[0]))
+
+
+def test_incoming_and_outgoing_sampling_under_the_buffer():
+    n, parts = 6000, 6
+    g = inputs.rmat_graph(n, 90_000, seed=4)
+    gt = inputs.transpose_csr(g)
+    feats = inputs.normal_features(n, 8, seed=2)
+    ctx = mg.Context(0)
+    ctx.load_graph(g.row_offsets.cuda(), g.nbrs.cuda())
+    ctx.load_out_graph(gt.row_offsets.to(torch.int32).cuda(), gt.nbrs.cuda())
+    ctx.set_partitioning(parts)
+    ctx.load_features(feats.cuda(), capacity_parts=parts)
+    ctx.set_sample_direction("inout")
+    for resident in ([0, 2, 5], [1, 2, 3, 4], list(range(parts))):
+        ctx.set_resident(resident, async_=True)
+        ctx.commit_resident(10_000)
+        view = O.GraphView(g.row_offsets.numpy(), g.nbrs.numpy(), parts, resident, gt.row_offsets.numpy(), gt.nbrs.numpy())
+        pool = torch.nonzero(inputs.resident_node_mask(n, parts, resident)).flatten()
+        targets = inputs.distinct_targets(pool, 100, seed=len(resident))
+        d = ctx.sample(targets, [6, 4], seed=31)
+        ref = O.sample_dense(view, targets.tolist(), [6, 4], 31, direction="inout")
+        assert_dense_equal(d.view(0), ref)
+        assert all(view.is_resident(u) for u in ref["node_ids"])
