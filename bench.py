@@ -32,6 +32,11 @@ CONFIGS = {
                             batch=1000, parts=1, train=1_000_000),
     "config3_papers100m_shaped": dict(n=111_000_000, m=1_620_000_000, kind="rmat", dim=128, hidden=256,
                                       fanouts=[15, 10, 5], batch=1000, parts=16, train=1_100_000),
+    # config 3's graph sampled from incoming AND outgoing edges, 15 / 10 / 5 neighbours per direction (the paper's
+    # 30 / 20 / 10 over both directions, Section 7.1); mini-batches are ~20x larger, so a step takes 16 of them
+    "config3_papers100m_shaped_inout": dict(n=111_000_000, m=1_620_000_000, kind="rmat", dim=128, hidden=256,
+                                            fanouts=[15, 10, 5], batch=1000, parts=16, train=1_100_000, inout=True,
+                                            group=16),
     # config 4's shapes at a tenth of its node count, whole fp16 table in HBM (no swaps): a throughput probe of the
     # wide fp16 layer-1 path, not the out-of-core configuration itself (that one is exercised by the tests)
     "config4_tenth_fp16_768_in_hbm": dict(n=12_200_000, m=130_000_000, kind="rmat", dim=768, hidden=256,
@@ -145,11 +150,13 @@ def algorithmic_bytes(nodes, ents, cfg, feat_bytes=4):
 def oracle_time(g_host, feats, layers, cfg, target_rows, seeds, budget_s=20.0):
     """The CPU oracle as it stands on a bounded sample of the same mini-batches."""
     from oracle import dense_oracle as O
-    view = O.GraphView(g_host[0], g_host[1])
+    view = O.GraphView(g_host[0], g_host[1], out_row_offsets=g_host[2] if len(g_host) > 2 else None,
+                       out_nbrs=g_host[3] if len(g_host) > 2 else None)
+    direction = "inout" if len(g_host) > 2 else "in"
     np_layers = [(w.numpy(), n.numpy(), b.numpy()) for w, n, b in layers]
     done, edges, t0 = 0, 0, time.time()
     for tg, seed in zip(target_rows, seeds):
-        ref = O.sample_dense(view, tg.tolist(), cfg["fanouts"], int(seed))
+        ref = O.sample_dense(view, tg.tolist(), cfg["fanouts"], int(seed), direction)
         ids = torch.as_tensor(ref["node_ids"], dtype=torch.int64)
         h0 = feats[ids.to(feats.device)].float().cpu().numpy()
         O.forward(ref, h0, np_layers)
@@ -168,7 +175,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="mgdense", choices=["mgdense", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(CONFIGS) + [LP_WORKLOAD])
-    ap.add_argument("--group", type=int, default=128, help="mini-batches per step")
+    ap.add_argument("--group", type=int, default=0, help="mini-batches per step (default: 128, or the workload's own)")
     ap.add_argument("--window", type=int, default=0, help="mini-batches per window of the layer schedule (0 = whole layers)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
@@ -208,6 +215,13 @@ def main():
     if rank == 0 and not args.no_cpu_baseline:
         g_host = (g.row_offsets.cpu().numpy(), g.nbrs.cpu().numpy())
     n_edges = g.n_edges
+    if cfg.get("inout"):
+        gt = inputs.transpose_csr(g)
+        ctx.load_out_graph(gt.row_offsets, gt.nbrs)
+        ctx.set_sample_direction("inout")
+        if g_host is not None:
+            g_host = g_host + (gt.row_offsets.cpu().numpy(), gt.nbrs.cpu().numpy())
+        del gt
     del g
     torch.cuda.empty_cache()
     if cfg["parts"] > 1:
@@ -219,7 +233,7 @@ def main():
     model = ctx.model(layers, mg.GEMM_TF32)
     ctx.set_layer_window(args.window)
 
-    G, T, k = args.group, cfg["batch"], len(cfg["fanouts"])
+    G, T, k = (args.group or cfg.get("group", 128)), cfg["batch"], len(cfg["fanouts"])
     n_steps_total = args.warmup + 2 * args.steps + 1
     # every rank draws its own mini-batches from the shuffled train set
     all_targets = inputs.train_set_batches(cfg["n"], cfg["train"], T, G * n_steps_total, seed=100 + rank)
@@ -233,7 +247,7 @@ def main():
 
     # capacities from a probe group (worst-case bounds would waste memory by ~10x)
     probe = ctx.sample_many(step_targets(0).to(device), offs, cfg["fanouts"], step_seeds(0),
-                            caps=None if cfg["n"] < 2_000_000 else {"max_nodes_per_batch": 1 << 19})
+                            caps=None if cfg["n"] < 2_000_000 else {"max_nodes_per_batch": 1 << (23 if cfg.get("inout") else 19)})
     nodes, ents = probe.counts()
     caps = {"max_nodes_total": int(nodes.sum() * 1.3) + 1024, "max_entries_total": int(ents.sum() * 1.3) + 1024,
             "max_nodes_per_batch": int(nodes.sum(1).max() * 1.5) + 64}
@@ -530,6 +544,10 @@ def run_reference(args, cfg):
     g, feats, layers, _ = build_workload(cfg, device, seed=0)
     g_host = (g.row_offsets.cpu().numpy(), g.nbrs.cpu().numpy())
     n_edges = g.n_edges
+    if cfg.get("inout"):
+        gt = inputs.transpose_csr(g)
+        g_host = g_host + (gt.row_offsets.cpu().numpy(), gt.nbrs.cpu().numpy())
+        del gt
     del g
     per_step = 1
     total = (args.warmup + args.steps) * per_step

@@ -341,10 +341,11 @@ def test_config2_shaped_power_law_three_layers():
 
 
 def _check_batches_against_oracle(g_host, feats, layers, fanouts, targets_by_batch, seeds, dense, out, offs, batches, rtol):
-    view = O.GraphView(g_host[0], g_host[1])
+    inout = len(g_host) > 2
+    view = O.GraphView(g_host[0], g_host[1], out_row_offsets=g_host[2] if inout else None, out_nbrs=g_host[3] if inout else None)
     np_layers = [(w.numpy(), nn.numpy(), b.numpy()) for w, nn, b in layers]
     for b in batches:
-        ref = O.sample_dense(view, targets_by_batch[b].tolist(), fanouts, seeds[b])
+        ref = O.sample_dense(view, targets_by_batch[b].tolist(), fanouts, seeds[b], "inout" if inout else "in")
         assert_dense_equal(dense.view(b), ref)
         ids = torch.as_tensor(ref["node_ids"], dtype=torch.int64, device=feats.device)
         want = O.forward(ref, feats[ids].float().cpu().numpy(), np_layers)
@@ -384,6 +385,7 @@ def test_full_size_config3_in_bench_launch_configuration():
     ctx = mg.Context(0)
     ctx.load_graph(g.row_offsets, g.nbrs)
     g_host = (g.row_offsets.cpu().numpy(), g.nbrs.cpu().numpy())
+    gt = inputs.transpose_csr(g)          # the second edge list, for the incoming + outgoing part below
     del g
     torch.cuda.empty_cache()
     ctx.set_partitioning(cfg["parts"])
@@ -416,6 +418,26 @@ def test_full_size_config3_in_bench_launch_configuration():
             seg = ids[nio[j]:nio[j + 1]]
             assert bool((seg[1:] > seg[:-1]).all())
         assert ids[nio[-2]:].cpu().tolist() == tg[b].tolist()
+    # the same graph sampled from incoming and outgoing edges (15 / 10 / 5 per direction), 16 mini-batches per pass as
+    # bench.py's config3_papers100m_shaped_inout runs it; one mini-batch (about 600k nodes) checked against the oracle
+    d.free()
+    ctx.load_out_graph(gt.row_offsets, gt.nbrs)
+    g_host = g_host + (gt.row_offsets.cpu().numpy(), gt.nbrs.cpu().numpy())
+    del gt
+    torch.cuda.empty_cache()
+    ctx.set_sample_direction("inout")
+    G2 = bench.CONFIGS["config3_papers100m_shaped_inout"]["group"]
+    offs2 = offs[:G2 + 1]
+    tg2 = tg[:G2].reshape(-1).cuda()
+    probe = ctx.sample_many(tg2, offs2, cfg["fanouts"], seeds[:G2], caps={"max_nodes_per_batch": 1 << 23})
+    nodes, ents = probe.counts()
+    caps = {"max_nodes_total": int(nodes.sum() * 1.3) + 1024, "max_entries_total": int(ents.sum() * 1.3) + 1024,
+            "max_nodes_per_batch": int(nodes.sum(1).max() * 1.5) + 64}
+    probe.free()
+    d = ctx.sample_many(tg2, offs2, cfg["fanouts"], seeds[:G2], caps=caps)
+    out2 = torch.empty((G2 * T, cfg["hidden"]), dtype=torch.float32, device="cuda")
+    ctx.forward(model, d, out2)
+    _check_batches_against_oracle(g_host, feats, layers, cfg["fanouts"], tg, seeds, d, out2, offs2, [G2 - 1], RTOL_TC)
 
 
 def test_config4_shaped_out_of_core_fp16_swaps():
