@@ -221,6 +221,12 @@ int mg_dense_free(mg_dense* d);
 int mg_model_create(mg_ctx* ctx, int32_t k, const int32_t* dims, const float* const* w_self,
                     const float* const* w_nbr, const float* const* bias, int gemm_precision,
                     mg_model** out);
+/* Neighbour aggregator of every layer of the model: MG_AGGR_MEAN (default; GraphSage's mean over the sampled
+ * neighbours) or MG_AGGR_SUM (their sum: Algorithm 3 as printed is this layer with identity weights, no bias and no
+ * activation).  Takes effect from the next forward call.  Errors: MG_ERR_ARG. */
+#define MG_AGGR_MEAN 0
+#define MG_AGGR_SUM 1
+int mg_model_set_aggregator(mg_model* m, int aggregator);
 int mg_model_free(mg_model* m);
 
 /* Forward pass for every batch of `d`.  H^0 is read straight from the feature buffer (rows

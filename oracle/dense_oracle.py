@@ -282,12 +282,15 @@ def additive_layer(dense, h_prev):
     return nbr_aggr + self_repr
 
 
-def sage_layer(dense, h_prev, w_self, w_nbr, bias, relu: bool):
-    """Algorithm 3 with GraphSage's mean aggregator and self/neighbour linears."""
+def sage_layer(dense, h_prev, w_self, w_nbr, bias, relu: bool, aggregator: str = "mean"):
+    """Algorithm 3 with self/neighbour linears; the neighbour term is GraphSage's mean over
+    the sampled neighbours ("mean") or their sum ("sum", the aggregation Algorithm 3 prints)."""
+    if aggregator not in ("mean", "sum"):
+        raise ValueError("aggregator must be 'mean' or 'sum'")
     h_prev = np.asarray(h_prev, dtype=np.float64)
     n_rows = len(dense["node_ids"]) - dense["node_id_offsets"][1]
     nbr_repr = h_prev[np.asarray(dense["repr_map"], dtype=np.int64)]
-    nbr_aggr = _segment_reduce(nbr_repr, dense["nbr_offsets"], n_rows, mean=True)
+    nbr_aggr = _segment_reduce(nbr_repr, dense["nbr_offsets"], n_rows, mean=(aggregator == "mean"))
     self_repr = h_prev[dense["node_id_offsets"][1]:]
     out = (self_repr @ np.asarray(w_self, dtype=np.float64)
            + nbr_aggr @ np.asarray(w_nbr, dtype=np.float64)
@@ -295,7 +298,7 @@ def sage_layer(dense, h_prev, w_self, w_nbr, bias, relu: bool):
     return np.maximum(out, 0.0) if relu else out
 
 
-def forward(dense, h0, layers, return_all: bool = False):
+def forward(dense, h0, layers, return_all: bool = False, aggregator: str = "mean"):
     """k layers: Step 1 (layer output) then Step 2 (Algorithm 2), Section 4.2.
 
     h0: [len(node_ids), d0] base representations aligned with node_ids.
@@ -307,7 +310,7 @@ def forward(dense, h0, layers, return_all: bool = False):
     cur = {key: list(val) for key, val in dense.items()}
     outs = []
     for i, (w_self, w_nbr, bias) in enumerate(layers):
-        h = sage_layer(cur, h, w_self, w_nbr, bias, relu=(i + 1 < len(layers)))
+        h = sage_layer(cur, h, w_self, w_nbr, bias, relu=(i + 1 < len(layers)), aggregator=aggregator)
         outs.append(h)
         cur = update_dense(cur)
     return outs if return_all else h

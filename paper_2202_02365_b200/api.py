@@ -29,7 +29,7 @@ CORRUPT_DST, CORRUPT_SRC, CORRUPT_BOTH = 1, 2, 3
 EXPORTS = [
     "mg_create", "mg_destroy", "mg_last_error", "mg_load_graph", "mg_load_out_graph", "mg_set_sample_direction", "mg_set_partitioning",
     "mg_load_features", "mg_set_resident", "mg_commit_resident", "mg_sample_many", "mg_sample_many_begin", "mg_sample_many_end", "mg_sample",
-    "mg_dense_counts", "mg_dense_view", "mg_dense_free", "mg_model_create", "mg_model_free",
+    "mg_dense_counts", "mg_dense_view", "mg_dense_free", "mg_model_create", "mg_model_set_aggregator", "mg_model_free",
     "mg_forward", "mg_set_layer_window", "mg_keep_layer_outputs", "mg_forward_host_async", "mg_wait_output", "mg_forward_noalloc", "mg_gather_h0", "mg_layer_output", "mg_lp_prepare", "mg_lp_view", "mg_lp_free",
     "mg_distmult_score", "mg_kernel_launches", "mg_profile", "mg_profile_read",
 ]
@@ -156,6 +156,10 @@ class Model:
         dims = (C.c_int32 * (k + 1))(*self.dims)
         ctx._check(ctx.lib.mg_model_create(ctx.handle, C.c_int32(k), dims, arrs[0], arrs[1], arrs[2],
                                            C.c_int(precision), C.byref(self.handle)))
+
+    def set_aggregator(self, aggregator: str):
+        """"mean" (GraphSage's mean over the sampled neighbours, the default) or "sum"."""
+        self.ctx._check(self.ctx.lib.mg_model_set_aggregator(self.handle, C.c_int({"mean": 0, "sum": 1}[aggregator])))
 
     def free(self):
         if self.handle:

@@ -22,8 +22,8 @@ int mg_pack_layer_weights(mg_ctx* ctx, const float* w_cat_dev, float* w_pad_t_de
 bool mg_layer_fused_supported(int d_in, int d_out);
 int mg_layer_rows(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_out, int4* row_meta);
 int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_out, const float* w_pad_t, const float* bias,
-                   const float* h_prev, float* h_out, bool relu, const int4* row_meta, int64_t row_lo, int64_t row_hi,
-                   int64_t safe_src_row);
+                   const float* h_prev, float* h_out, int flags /* 1 = ReLU, 2 = sum instead of mean */, const int4* row_meta,
+                   int64_t row_lo, int64_t row_hi, int64_t safe_src_row);
 
 namespace {
 
@@ -49,6 +49,7 @@ struct AggArgs {
     uint32_t part_size;
     float* x;                    // [rows, 2 * d_in], row r of this launch at x + (r - row_lo) * 2 * d_in
     int round_tf32;
+    int sum_aggr;                // neighbour term = sum of the sampled neighbours instead of their mean
 };
 
 __device__ __forceinline__ float to_tf32(float v) {
@@ -161,7 +162,7 @@ __global__ void __launch_bounds__(kThreads) k_aggregate(AggArgs a) {
                 if (c < n_chunks) { C t; t.load(r0, c); acc[j].add(t); }
             }
         }
-        const float inv = e1 > e0 ? 1.f / (float)(e1 - e0) : 0.f;
+        const float inv = e1 > e0 ? (a.sum_aggr ? 1.f : 1.f / (float)(e1 - e0)) : 0.f;
 #pragma unroll
         for (int j = 0; j < NCH; ++j) {
             const int c = gl + j * G;
@@ -356,6 +357,13 @@ extern "C" int mg_model_create(mg_ctx* ctx, int32_t k, const int32_t* dims, cons
     return MG_OK;
 }
 
+extern "C" int mg_model_set_aggregator(mg_model* m, int aggregator) {
+    if (!m) return MG_ERR_ARG;
+    if (aggregator != MG_AGGR_MEAN && aggregator != MG_AGGR_SUM) return mg_fail(m->ctx, MG_ERR_ARG, "unknown aggregator");
+    m->sum_aggr = aggregator == MG_AGGR_SUM;
+    return MG_OK;
+}
+
 extern "C" int mg_model_free(mg_model* m) {
     if (!m) return MG_OK;
     cudaSetDevice(m->device);
@@ -489,7 +497,7 @@ static int forward_impl(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out,
                 float* h_out = l == k ? hk : base + ring_off[l] - lo * m->dims[l];
                 ProfScope ps(ctx, l == 1 ? PH_AGG_L1 : PH_AGG_REST, 1);
                 rc = mg_layer_fused(ctx, d, l, m->dims[l - 1], m->dims[l], m->w_pad_t[l - 1], m->bias[l - 1], h_prev, h_out,
-                                    l < k, meta + meta_off[l], lo, hi, l > 1 ? lo_in : 0);
+                                    (l < k ? 1 : 0) | (m->sum_aggr ? 2 : 0), meta + meta_off[l], lo, hi, l > 1 ? lo_in : 0);
                 if (rc) return rc;
             }
         }
@@ -546,7 +554,8 @@ static int forward_impl(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out,
             }
             {
                 ProfScope ps(ctx, l == 1 ? PH_AGG_L1 : PH_AGG_REST, 1);
-                rc = mg_layer_fused(ctx, d, l, d_in, d_out, m->w_pad_t[l - 1], m->bias[l - 1], h_prev, h_out, l < k, meta, 0, M, 0);
+                rc = mg_layer_fused(ctx, d, l, d_in, d_out, m->w_pad_t[l - 1], m->bias[l - 1], h_prev, h_out,
+                                    (l < k ? 1 : 0) | (m->sum_aggr ? 2 : 0), meta, 0, M, 0);
             }
             if (rc) return rc;
             continue;
@@ -566,6 +575,7 @@ static int forward_impl(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out,
             a.slot_bytes = ctx->slot_bytes; a.row_bytes = ctx->row_bytes; a.part_size = (uint32_t)ctx->part_size;
             a.x = ctx->ws_x;
             a.round_tf32 = m->precision == MG_GEMM_TF32;
+            a.sum_aggr = m->sum_aggr ? 1 : 0;
             {
                 ProfScope ps(ctx, l == 1 ? PH_AGG_L1 : PH_AGG_REST, 1);
                 const int grid = mg_grid(ctx, 8);
@@ -743,6 +753,7 @@ extern "C" int mg_forward_noalloc(mg_ctx* ctx, const mg_model* m, mg_dense* d, f
             a.slot_bytes = ctx->slot_bytes; a.row_bytes = ctx->row_bytes; a.part_size = (uint32_t)ctx->part_size;
             a.x = staging;
             a.round_tf32 = m->precision == MG_GEMM_TF32;
+            a.sum_aggr = m->sum_aggr ? 1 : 0;
             const int grid = mg_grid(ctx, 8);
             if (l == 1) { if (half) launch_aggregate<true, true>(a, grid, st); else launch_aggregate<true, false>(a, grid, st); }
             else launch_aggregate<false, false>(a, grid, st);

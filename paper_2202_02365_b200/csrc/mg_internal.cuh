@@ -215,6 +215,7 @@ struct mg_model {
     int32_t k = 0;
     int32_t dims[MG_MAX_HOPS + 1] = {0};
     int precision = MG_GEMM_TF32;
+    bool sum_aggr = false;   // neighbour term: sum instead of mean (Algorithm 3 as printed)
     float* w_cat[MG_MAX_HOPS] = {nullptr};  // device [2*d_in, d_out]: rows 0..d_in-1 self, then neighbour
     float* w_cat_t[MG_MAX_HOPS] = {nullptr}; // device [d_out, 2*d_in] (K-major copy for the tensor-core path)
     float* w_pad_t[MG_MAX_HOPS] = {nullptr}; // device [d_out, 2*roundup32(d_in)], zero padded, for the fused layer kernel

@@ -76,6 +76,7 @@ struct FusedArgs {
     int32_t sa, sb;              // A and B stages
     int32_t tmem_cols;
     int32_t relu;
+    int32_t sum_aggr;            // neighbour term = sum of the sampled neighbours instead of their mean
     const float* bias;
     float* out;                  // [M, N]
     uint32_t* error;
@@ -403,7 +404,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
 #pragma unroll
                         for (int q2 = 0; q2 < kRowsInFlight; ++q2) {
                             const float inv = cached ? __int_as_float(first_rows[slot][brow + q2][5])
-                                                     : (mq[q2].z > 0 ? 1.f / (float)mq[q2].z : 0.f);
+                                                     : (mq[q2].z > 0 ? (a.sum_aggr ? 1.f : 1.f / (float)mq[q2].z) : 0.f);
                             acc[q2].x = to_tf32(acc[q2].x * inv); acc[q2].y = to_tf32(acc[q2].y * inv);
                             acc[q2].z = to_tf32(acc[q2].z * inv); acc[q2].w = to_tf32(acc[q2].w * inv);
                             selfv[q2].x = to_tf32(selfv[q2].x); selfv[q2].y = to_tf32(selfv[q2].y);
@@ -508,7 +509,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 int32_t fr[8];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) fr[j] = (j < kUnroll && j < rm.z) ? src_rows[slot][koff + j] : rm.x;
-                fr[5] = __float_as_int(rm.z > 0 ? 1.f / (float)rm.z : 0.f);   // the mean's factor
+                fr[5] = __float_as_int(rm.z > 0 ? (a.sum_aggr ? 1.f : 1.f / (float)rm.z) : 0.f);   // the mean's factor (1 for a sum)
                 *reinterpret_cast<int4*>(&first_rows[slot][lane][0]) = make_int4(fr[0], fr[1], fr[2], fr[3]);
                 *reinterpret_cast<int4*>(&first_rows[slot][lane][4]) = make_int4(fr[4], fr[5], fr[6], fr[7]);
                 __syncwarp();
@@ -609,7 +610,7 @@ int mg_layer_rows(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_out
 // Runs layer `layer` (1-based) for the packed output rows [row_lo, row_hi).  h_prev and h_out are indexed by
 // GLOBAL packed row (callers that keep only a window of a layer pass pointers shifted accordingly).
 int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_out, const float* w_pad_t, const float* bias,
-                   const float* h_prev, float* h_out, bool relu, const int4* row_meta, int64_t row_lo, int64_t row_hi,
+                   const float* h_prev, float* h_out, int flags, const int4* row_meta, int64_t row_lo, int64_t row_hi,
                    int64_t safe_src_row) {
     if (row_hi <= row_lo) return MG_OK;
     FusedArgs a;
@@ -622,7 +623,8 @@ int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_ou
     a.h_prev = h_prev;
     a.src_base = layer == 1 ? ctx->slots : reinterpret_cast<const char*>(h_prev);
     a.src_row_bytes = layer == 1 ? (uint32_t)ctx->row_bytes : (uint32_t)d_in * 4u;
-    a.relu = relu ? 1 : 0;
+    a.relu = flags & 1;
+    a.sum_aggr = (flags >> 1) & 1;
     a.bias = bias; a.out = h_out;
     int stride = 32;
     while (stride < a.BN / 2) stride <<= 1;

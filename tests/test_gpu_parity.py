@@ -727,3 +727,37 @@ def test_incoming_and_outgoing_sampling_under_the_buffer():
         ref = O.sample_dense(view, targets.tolist(), [6, 4], 31, direction="inout")
         assert_dense_equal(d.view(0), ref)
         assert all(view.is_resident(u) for u in ref["node_ids"])
+
+
+def test_sum_aggregator(tiny):
+    """The neighbour term as a sum (Algorithm 3 as printed) instead of GraphSage's mean: fused TF32 layers, the
+    unfused fp32 path, and identity weights = the printed additive layer."""
+    g, feats = tiny
+    ctx = make_ctx(g, feats)
+    targets = inputs.distinct_targets(10_000, 300, seed=21)
+    d = ctx.sample(targets, [7, 3], seed=5)
+    ref = O.sample_dense(oracle_view(g), targets.tolist(), [7, 3], 5)
+    h0 = feats.numpy()[ref["node_ids"]]
+    layers = inputs.random_bias_layers([16, 32, 8], seed=3)
+    np_layers = [(w.numpy(), n.numpy(), b.numpy()) for w, n, b in layers]
+    want = O.forward(ref, h0, np_layers, aggregator="sum")
+    want_mean = O.forward(ref, h0, np_layers)
+    for prec, rtol in ((mg.GEMM_FP32, RTOL_AGG), (mg.GEMM_TF32, RTOL_TC)):
+        model = ctx.model(layers, prec)
+        out = torch.empty((300, 8), dtype=torch.float32, device="cuda")
+        ctx.forward(model, d, out)
+        close(out.cpu().numpy(), want_mean, rtol)
+        model.set_aggregator("sum")
+        ctx.forward(model, d, out)
+        close(out.cpu().numpy(), want, rtol)
+        model.set_aggregator("mean")
+        ctx.forward(model, d, out)
+        close(out.cpu().numpy(), want_mean, rtol)
+    eye = [(torch.eye(16), torch.eye(16), torch.zeros(16))]
+    d1 = ctx.sample(targets, [7], seed=5)
+    ref1 = O.sample_dense(oracle_view(g), targets.tolist(), [7], 5)
+    model = ctx.model(eye, mg.GEMM_FP32)
+    model.set_aggregator("sum")
+    out = torch.empty((300, 16), dtype=torch.float32, device="cuda")
+    ctx.forward(model, d1, out)
+    close(out.cpu().numpy(), O.additive_layer(ref1, feats.numpy()[ref1["node_ids"]]), RTOL_AGG)

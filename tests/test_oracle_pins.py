@@ -548,3 +548,37 @@ def test_inout_input_errors():
         O.sample_dense(O.GraphView(off, nb), [1], [2], 0, direction="inout")     # no outgoing edge list
     with pytest.raises(ValueError):
         O.sample_dense(O.GraphView(off, nb), [1], [2], 0, direction="out")
+
+
+def test_sum_aggregator_reduces_to_algorithm_3_and_to_count_times_mean():
+    off, nb = _random_graph(120, 900, 2)
+    view = O.GraphView(off, nb)
+    d = O.sample_dense(view, [4, 9, 100], [3, 2], seed=5)
+    rng = np.random.default_rng(0)
+    h0 = rng.standard_normal((len(d["node_ids"]), 6))
+    eye, zero = np.eye(6), np.zeros(6)
+    # identity weights, no bias, no activation: the printed Algorithm 3
+    np.testing.assert_allclose(O.sage_layer(d, h0, eye, eye, zero, relu=False, aggregator="sum"), O.additive_layer(d, h0),
+                               rtol=0, atol=1e-12)
+    # sum = count x mean, row by row, through arbitrary weights
+    w_s, w_n, b = rng.standard_normal((6, 5)), rng.standard_normal((6, 5)), rng.standard_normal(5)
+    n_rows = len(d["node_ids"]) - d["node_id_offsets"][1]
+    counts = np.diff(d["nbr_offsets"])[:n_rows, None]
+    mean_part = O.sage_layer(d, h0, np.zeros((6, 5)), w_n, zero[:5], relu=False)
+    sum_part = O.sage_layer(d, h0, np.zeros((6, 5)), w_n, zero[:5], relu=False, aggregator="sum")
+    np.testing.assert_allclose(sum_part, counts * mean_part, rtol=1e-12, atol=1e-12)
+    # the whole forward pass with the sum against per-layer index_add_ in torch
+    layers = [(w_s, w_n, b), (rng.standard_normal((5, 4)), rng.standard_normal((5, 4)), rng.standard_normal(4))]
+    got = O.forward(d, h0, layers, aggregator="sum")
+    cur, h = d, torch.tensor(h0)
+    for i, (ws, wn, bb) in enumerate(layers):
+        rows = len(cur["node_ids"]) - cur["node_id_offsets"][1]
+        seg = torch.repeat_interleave(torch.arange(rows), torch.tensor(np.diff(cur["nbr_offsets"])[:rows]))
+        agg = torch.zeros((rows, h.shape[1]), dtype=torch.float64).index_add_(0, seg, h[torch.tensor(cur["repr_map"], dtype=torch.int64)])
+        h = h[cur["node_id_offsets"][1]:] @ torch.tensor(ws) + agg @ torch.tensor(wn) + torch.tensor(bb)
+        if i == 0:
+            h = torch.relu(h)
+        cur = O.update_dense(cur)
+    np.testing.assert_allclose(got, h.numpy(), rtol=1e-12, atol=1e-12)
+    with pytest.raises(ValueError):
+        O.sage_layer(d, h0, eye, eye, zero, relu=False, aggregator="max")
