@@ -169,6 +169,9 @@ struct mg_dense {
     int64_t* node_r0_out = nullptr; // the same for the outgoing edge list (incoming + outgoing sampling only)
     uint32_t* node_deg_out = nullptr;
     int64_t cap_nodes_out = 0;
+    int2* pairs = nullptr;          // last hop, shared-memory deduplication: (id, entry) grouped by (batch, share, bucket)
+    int32_t* share_off = nullptr;   // its group bounds
+    int64_t cap_pairs = 0, cap_share = 0;
     int32_t* ent_nbrs = nullptr;    // [cap_entries] neighbour ids
     int32_t* ent_repr = nullptr;    // [cap_entries] neighbour's local row in its batch
     int32_t* node_off = nullptr;    // [(k+1) * (B+1)] arena index where batch b's hop-h nodes start

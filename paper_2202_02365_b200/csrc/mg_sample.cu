@@ -473,6 +473,256 @@ __global__ void __launch_bounds__(kThreads) k_insert(InsertArgs a) {
 }
 
 // -------------------------------------------------------------------------------------
+// Last hop: deduplication in shared memory
+// -------------------------------------------------------------------------------------
+// The last hop has most of the entries (12.9M of 16.6M on the bench) and its new nodes are never looked up again, so
+// it does not go through the id tables in global memory.  The ids of a mini-batch are split by hash into nb buckets.
+// k_bucket_entries: block (mini-batch, r) takes the r-th share of the mini-batch's entries and writes them grouped by
+// bucket (a counting sort inside the block) as (id, entry) pairs, with the groups' bounds.
+// k_dedupe_last: block (mini-batch, bucket) holds the bucket's id table (keys and rows, S slots) in shared memory.  It
+// enters the nodes the mini-batch already has (hops 0..hop, rows = positions; every block of the mini-batch reads all
+// of them and keeps its bucket's, compacted per warp so that the table code runs on full warps), then its bucket's
+// pairs from every share (dense), ranks its new nodes (a scan over the table, no atomics), takes a run of the
+// mini-batch's rows and of the list of new nodes with ONE global atomic each, and gives every entry its node's row.
+constexpr int kDedupThreads = 1024;
+constexpr int kDedupMaxSlots = 26624;    // 208 KiB of keys + rows per block
+constexpr int kDedupMaxBuckets = 32;
+constexpr int kDedupQueue = 64;          // per warp: up to 31 waiting + 32 new (id, row) pairs
+constexpr size_t kDedupQueueBytes = (size_t)(kDedupThreads / 32) * kDedupQueue * sizeof(uint2);
+constexpr int kBucketThreads = 512;
+
+struct DedupArgs {
+    DenseHeader* hdr;
+    int hop;
+    int32_t B, k, nb, S;
+    const int32_t* nodes;
+    const int32_t* node_off;    // [hop + 1][B + 1] valid
+    const int32_t* ent_off;
+    const int32_t* ent_nbrs;
+    int32_t* ent_repr;
+    int2* pairs;                // [entries of the hop] (id, entry), grouped by (mini-batch, share, bucket)
+    int32_t* share_off;         // [B][nb][nb + 1] group bounds (positions in pairs)
+    const int32_t* cum;         // [B][k + 2]
+    uint32_t* batch_cnt;        // [B] new nodes of the hop per mini-batch, zero before the launch
+    uint64_t* newlist;
+    int64_t cap_new;
+    int id_bits;
+    int32_t max_nodes_per_batch;
+};
+
+// bucket and first slot of an id: one multiplicative hash, the bucket from its top, the slot from what is left
+__device__ __forceinline__ uint32_t dedup_bucket(int32_t id, uint32_t nb) { return __umulhi((uint32_t)id * 0x9E3779B1u, nb); }
+__device__ __forceinline__ uint32_t dedup_slot(int32_t id, uint32_t nb, uint32_t S) {
+    return __umulhi((uint32_t)id * 0x9E3779B1u * nb, S);
+}
+
+__global__ void __launch_bounds__(kBucketThreads) k_bucket_entries(DedupArgs a) {
+    constexpr int kWarps = kBucketThreads / 32;
+    __shared__ uint32_t cnt[kWarps][kDedupMaxBuckets];
+    __shared__ uint32_t base[kDedupMaxBuckets + 1];
+    if (a.hdr->status) return;
+    const uint32_t nb = (uint32_t)a.nb;
+    const int32_t b = (int32_t)(blockIdx.x / nb);
+    const uint32_t r = blockIdx.x % nb;
+    const int warp = threadIdx.x >> 5;
+    const int32_t e_lo = a.ent_off[a.node_off[a.hop * (a.B + 1) + b]];
+    const int32_t e_hi = a.ent_off[a.node_off[a.hop * (a.B + 1) + b + 1]];
+    const int32_t len = (int32_t)(((int64_t)(e_hi - e_lo) + nb - 1) / nb);
+    const int32_t s_lo = (int32_t)min((int64_t)e_hi, (int64_t)e_lo + (int64_t)r * len);
+    const int32_t s_hi = (int32_t)min((int64_t)e_hi, (int64_t)s_lo + len);
+    for (int i = threadIdx.x; i < kWarps * kDedupMaxBuckets; i += kBucketThreads) (&cnt[0][0])[i] = 0;
+    __syncthreads();
+    // (four loads in flight per thread: the walk is latency-bound otherwise)
+    for (int32_t e0 = s_lo + (int32_t)threadIdx.x; e0 < s_hi; e0 += 4 * kBucketThreads) {
+        int32_t id[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) id[u] = e0 + u * kBucketThreads < s_hi ? a.ent_nbrs[e0 + u * kBucketThreads] : -1;
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (e0 + u * kBucketThreads < s_hi) atomicAdd(&cnt[warp][dedup_bucket(id[u], nb)], 1u);
+    }
+    __syncthreads();
+    if (threadIdx.x < nb) {   // this bucket's pairs of the share: warp after warp
+        uint32_t run = 0;
+        for (int w = 0; w < kWarps; ++w) { const uint32_t c = cnt[w][threadIdx.x]; cnt[w][threadIdx.x] = run; run += c; }
+        base[threadIdx.x] = run;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t run = 0;
+        for (uint32_t q = 0; q < nb; ++q) { const uint32_t c = base[q]; base[q] = run; run += c; }
+        base[nb] = run;
+    }
+    __syncthreads();
+    if (threadIdx.x <= nb) a.share_off[((int64_t)b * nb + r) * (nb + 1) + threadIdx.x] = s_lo + (int32_t)base[threadIdx.x];
+    for (int32_t e0 = s_lo + (int32_t)threadIdx.x; e0 < s_hi; e0 += 4 * kBucketThreads) {
+        int32_t id[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) id[u] = e0 + u * kBucketThreads < s_hi ? a.ent_nbrs[e0 + u * kBucketThreads] : -1;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int32_t e = e0 + u * kBucketThreads;
+            if (e >= s_hi) continue;
+            const uint32_t q = dedup_bucket(id[u], nb);
+            a.pairs[s_lo + base[q] + atomicAdd(&cnt[warp][q], 1u)] = make_int2(id[u], e);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kDedupThreads) k_dedupe_last(DedupArgs a) {
+    extern __shared__ int32_t dedup_sm[];
+    __shared__ uint32_t row_base, list_base, warp_tot[kDedupThreads / 32];
+    __shared__ int32_t run_lo[kDedupMaxBuckets], run_start[kDedupMaxBuckets + 1];
+    if (a.hdr->status) return;
+    const uint32_t S = (uint32_t)a.S, nb = (uint32_t)a.nb;
+    int32_t* keys = dedup_sm;
+    int32_t* vals = dedup_sm + S;
+    const int32_t b = (int32_t)(blockIdx.x / nb);
+    const uint32_t bucket = blockIdx.x % nb;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (uint32_t i = threadIdx.x; i < S; i += kDedupThreads) keys[i] = -1;
+    if (threadIdx.x < nb) {   // this bucket's runs of pairs, one per share ...
+        const int32_t* so = a.share_off + ((int64_t)b * nb + threadIdx.x) * (nb + 1) + bucket;
+        run_lo[threadIdx.x] = so[0];
+        run_start[threadIdx.x + 1] = so[1] - so[0];
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {   // ... and their lengths' prefix
+        int32_t run = 0;
+        for (uint32_t r = 0; r < nb; ++r) { const int32_t c = run_start[r + 1]; run_start[r] = run; run += c; }
+        run_start[nb] = run;
+    }
+    __syncthreads();
+    // the nodes the mini-batch already has: a warp compacts the ids of this bucket and enters 32 at a time
+    {
+        uint2* q = reinterpret_cast<uint2*>(dedup_sm + 2 * S) + warp * kDedupQueue;
+        const uint32_t lt = (1u << lane) - 1u;
+        uint32_t waiting = 0;
+        auto enter = [&](uint2 it) {
+            const int32_t u = (int32_t)it.x;
+            uint32_t s = dedup_slot(u, nb, S), probe = 0;
+            for (; probe < S; ++probe) {
+                const int32_t old = atomicCAS(&keys[s], -1, u);
+                if (old == -1) { vals[s] = (int32_t)it.y; break; }
+                if (old == u) { atomicOr(&a.hdr->status, ST_DUPLICATE); break; }   // only targets can repeat
+                s = s + 1u == S ? 0u : s + 1u;
+            }
+            if (probe >= S) atomicOr(&a.hdr->status, ST_CAP_TABLE);
+        };
+        for (int j = 0; j <= a.hop; ++j) {
+            const int32_t lo = a.node_off[j * (a.B + 1) + b], hi = a.node_off[j * (a.B + 1) + b + 1];
+            const int32_t row0 = a.cum[b * (a.k + 2) + j];
+            for (int32_t p0 = lo + warp * 32; p0 < hi; p0 += 4 * kDedupThreads) {
+                int32_t us[4];   // four loads in flight per lane
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int32_t p = p0 + c * kDedupThreads + lane;
+                    us[c] = p < hi ? a.nodes[p] : 0;
+                }
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int32_t p = p0 + c * kDedupThreads + lane;
+                    const bool m = p < hi && dedup_bucket(us[c], nb) == bucket;
+                    const uint32_t mask = __ballot_sync(0xFFFFFFFFu, m);
+                    if (m) q[waiting + __popc(mask & lt)] = make_uint2((uint32_t)us[c], (uint32_t)(row0 + (p - lo)));
+                    waiting += __popc(mask);
+                    __syncwarp();
+                    if (waiting >= 32) {
+                        enter(q[waiting - 32 + lane]);
+                        waiting -= 32;
+                    }
+                    __syncwarp();
+                }
+            }
+        }
+        if ((uint32_t)lane < waiting) enter(q[lane]);
+    }
+    __syncthreads();
+    // this bucket's pairs: enter the id, leave its slot in place of the id
+    const int32_t n_pairs = run_start[nb];
+    auto pair_at = [&](int32_t i) -> int2* {
+        uint32_t r = 0;
+        while (r + 1 < nb && run_start[r + 1] <= i) ++r;
+        return a.pairs + run_lo[r] + (i - run_start[r]);
+    };
+    for (int32_t i0 = threadIdx.x; i0 < n_pairs; i0 += 4 * kDedupThreads) {
+        int2* pp[4];
+        int32_t id[4], old[4];
+        uint32_t s[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {   // four loads, then four first-probe compare-and-swaps, in flight per thread
+            const int32_t i = i0 + u * kDedupThreads;
+            pp[u] = pair_at(min(i, n_pairs - 1));
+            id[u] = i < n_pairs ? pp[u]->x : -1;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            s[u] = dedup_slot(id[u], nb, S);
+            old[u] = id[u] >= 0 ? atomicCAS(&keys[s[u]], -1, id[u]) : id[u];
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (id[u] < 0) continue;
+            bool fresh = old[u] == -1;
+            if (!fresh && old[u] != id[u]) {   // first slot taken by another id: linear probing
+                uint32_t probe = 1;
+                for (; probe < S; ++probe) {
+                    s[u] = s[u] + 1u == S ? 0u : s[u] + 1u;
+                    const int32_t o = atomicCAS(&keys[s[u]], -1, id[u]);
+                    if (o == -1) { fresh = true; break; }
+                    if (o == id[u]) break;
+                }
+                if (probe >= S) { atomicOr(&a.hdr->status, ST_CAP_TABLE); s[u] = 0; fresh = false; }
+            }
+            if (fresh) vals[s[u]] = -1;   // new: ranked below
+            pp[u]->x = (int32_t)s[u];
+        }
+    }
+    __syncthreads();
+    // rank the new nodes of this block's table, take a run of the mini-batch's rows and of the list of new nodes
+    uint32_t mine = 0;
+    for (uint32_t i = threadIdx.x; i < S; i += kDedupThreads) mine += (keys[i] != -1 && vals[i] < 0) ? 1u : 0u;
+    const uint32_t inc = warp_incl_scan(mine);
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        const uint32_t w = warp_tot[lane];
+        const uint32_t wi = warp_incl_scan(w);
+        warp_tot[lane] = wi - w;
+        if (lane == 31) {
+            row_base = wi ? atomicAdd(&a.batch_cnt[b], wi) : 0u;
+            list_base = wi ? atomicAdd(&a.hdr->n_new, wi) : 0u;
+        }
+    }
+    __syncthreads();
+    const int32_t first_row = a.cum[b * (a.k + 2) + a.hop + 1];
+    uint32_t rk = warp_tot[warp] + inc - mine;
+    for (uint32_t i = threadIdx.x; i < S; i += kDedupThreads) {
+        if (keys[i] == -1 || vals[i] >= 0) continue;
+        const uint32_t rank = row_base + rk;
+        const int64_t row = (int64_t)first_row + rank;
+        if (row >= a.max_nodes_per_batch) atomicOr(&a.hdr->status, ST_CAP_TABLE);
+        vals[i] = (int32_t)row;
+        const int64_t pos = (int64_t)list_base + rk;
+        if (pos < a.cap_new)
+            a.newlist[pos] = (uint64_t)rank | ((uint64_t)(uint32_t)keys[i] << MG_SLOT_BITS) |
+                             ((uint64_t)(uint32_t)b << (MG_SLOT_BITS + a.id_bits));
+        else atomicOr(&a.hdr->status, ST_CAP_NODES);
+        ++rk;
+    }
+    __syncthreads();
+    // every entry of the bucket gets its node's row
+    for (int32_t i0 = threadIdx.x; i0 < n_pairs; i0 += 4 * kDedupThreads) {
+        int2 p[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) p[u] = *pair_at(min(i0 + u * kDedupThreads, n_pairs - 1));
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (i0 + u * kDedupThreads < n_pairs) a.ent_repr[p[u].y] = vals[p[u].x];
+    }
+}
+
+// -------------------------------------------------------------------------------------
 // radix sort of the new-node list on bits [lo_bit, lo_bit + bits) of the composite key
 // -------------------------------------------------------------------------------------
 constexpr int kSortKeysPerThread = 16;
@@ -894,7 +1144,7 @@ static int dev_realloc(mg_ctx* ctx, T** p, size_t elems) {
 }
 
 static int dense_alloc(mg_ctx* ctx, mg_dense* d, int32_t B, int32_t k, int64_t cap_nodes, int64_t cap_entries,
-                       int32_t table_size) {
+                       int32_t table_size, int32_t smem_nb) {
     int rc;
     if (!d->hdr && (rc = dev_realloc(ctx, &d->hdr, 1))) return rc;
     if (d->cap_nodes < cap_nodes) {
@@ -922,6 +1172,20 @@ static int dense_alloc(mg_ctx* ctx, mg_dense* d, int32_t B, int32_t k, int64_t c
         if ((rc = dev_realloc(ctx, &d->ent_nbrs, (size_t)cap_entries))) return rc;
         if ((rc = dev_realloc(ctx, &d->ent_repr, (size_t)cap_entries))) return rc;
         d->cap_entries = cap_entries;
+        d->cap_pairs = 0;
+    }
+    if (smem_nb > 0) {
+        if (d->cap_pairs < d->cap_entries) {
+            d->cap_pairs = 0;
+            if ((rc = dev_realloc(ctx, &d->pairs, (size_t)d->cap_entries))) return rc;
+            d->cap_pairs = d->cap_entries;
+        }
+        const int64_t need_share = (int64_t)B * smem_nb * (smem_nb + 1);
+        if (d->cap_share < need_share) {
+            d->cap_share = 0;
+            if ((rc = dev_realloc(ctx, &d->share_off, (size_t)need_share))) return rc;
+            d->cap_share = need_share;
+        }
     }
     if (ctx->sample_inout && d->cap_nodes_out < d->cap_nodes) {
         d->cap_nodes_out = 0;
@@ -1024,6 +1288,7 @@ static void sample_kernel_attributes() {
     static bool done = false;
     if (done) return;
     cudaFuncSetAttribute(k_radix_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScatterSmem);
+    cudaFuncSetAttribute(k_dedupe_last, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kDedupMaxSlots * 2 * sizeof(int32_t) + kDedupQueueBytes));
     cudaFuncSetAttribute(k_pick_wide, cudaFuncAttributeMaxDynamicSharedMemorySize,
                          (int)((size_t)(kThreads / 32) * 2 * MG_MAX_FANOUT * sizeof(uint32_t)));
     done = true;
@@ -1088,6 +1353,12 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
     const int64_t want_slots = std::max<int64_t>(16, (cap_batch + cap_batch / 2 + cap_batch / 8 + 7) / 8 * 8);
     if (want_slots > (1ll << MG_SLOT_BITS)) return mg_fail(ctx, MG_ERR_CAPACITY, "max_nodes_per_batch above %d", (int)((1ll << MG_SLOT_BITS) * 8 / 13));
     const int32_t table_size = (int32_t)want_slots;
+    // The last hop is deduplicated in shared memory (k_bucket_entries, k_dedupe_last) when a mini-batch's nodes fit the
+    // tables of a few blocks: S slots per block, filled to 92 % at most when the mini-batch is at its capacity (the
+    // buckets of a hash differ by a per cent or so at these sizes), nb blocks per mini-batch.
+    const int32_t dedup_slots = (int32_t)std::min<int64_t>(kDedupMaxSlots, (cap_batch + cap_batch / 4 + 64 + 1023) / 1024 * 1024);
+    const int64_t dedup_nb = (cap_batch + (cap_batch * 7 + 79) / 80 + dedup_slots - 1) / dedup_slots;
+    const bool smem_last = dedup_nb <= kDedupMaxBuckets && dedup_nb * n_batches < (1ll << 24) && !getenv("MG_GLOBAL_TABLES");
     if ((int64_t)table_size * n_batches >= (1ll << 31))
         return mg_fail(ctx, MG_ERR_CAPACITY, "n_batches x id-table size must stay below 2^31: pass a smaller max_nodes_per_batch or fewer batches");
     const int id_bits = std::max(1, ilog2_ceil(N));
@@ -1101,7 +1372,7 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
     d->valid = false;
     d->pending = false;
     if (d->ev_read_done) MG_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, d->ev_read_done, 0));
-    int rc = dense_alloc(ctx, d, n_batches, k, cap_nodes, std::max<int64_t>(cap_entries, 1), table_size);
+    int rc = dense_alloc(ctx, d, n_batches, k, cap_nodes, std::max<int64_t>(cap_entries, 1), table_size, smem_last ? (int32_t)dedup_nb : 0);
     if (rc) { if (created) mg_dense_free(d); return rc; }
     *out = d;
     for (int h = 0; h < k; ++h) d->fanouts[h] = fanouts[h];
@@ -1207,13 +1478,22 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
                 }
                 if (dir) ctx->launches++;
             }
-            InsertArgs ia{d->hdr, h, d->ent_nbrs, d->ent_repr, d->hkeys, tg, d->newlist[0], d->cap_nodes, id_bits,
-                          k, d->cum, d->hvals, batch_cnt + (size_t)h * B, (int32_t)cap_batch};
-            // many short blocks: measured on the bench's last hop, 0.94 ms at 32 blocks per SM against 1.08 ms at 8
-            // (blocks past the end of the entries return at once)
-            const int igrid = mg_grid(ctx, 32);
-            k_insert<<<igrid, kThreads, 0, st>>>(ia);
-            ctx->launches++;
+            if (smem_last && h == k - 1) {
+                DedupArgs da{d->hdr, h, B, k, (int32_t)dedup_nb, dedup_slots, d->nodes, d->node_off, d->ent_off, d->ent_nbrs,
+                             d->ent_repr, d->pairs, d->share_off, d->cum, batch_cnt + (size_t)h * B, d->newlist[0], d->cap_nodes,
+                             id_bits, (int32_t)cap_batch};
+                k_bucket_entries<<<(unsigned)(B * dedup_nb), kBucketThreads, 0, st>>>(da);
+                k_dedupe_last<<<(unsigned)(B * dedup_nb), kDedupThreads, (size_t)dedup_slots * 2 * sizeof(int32_t) + kDedupQueueBytes, st>>>(da);
+                ctx->launches += 2;
+            } else {
+                InsertArgs ia{d->hdr, h, d->ent_nbrs, d->ent_repr, d->hkeys, tg, d->newlist[0], d->cap_nodes, id_bits,
+                              k, d->cum, d->hvals, batch_cnt + (size_t)h * B, (int32_t)cap_batch};
+                // many short blocks: measured on the bench's last hop, 0.94 ms at 32 blocks per SM against 1.08 ms at 8
+                // (blocks past the end of the entries return at once)
+                const int igrid = mg_grid(ctx, 32);
+                k_insert<<<igrid, kThreads, 0, st>>>(ia);
+                ctx->launches++;
+            }
         }
         {
             // rows were handed out at insert time, in discovery order: per-batch counts -> offsets, then every list
@@ -1225,11 +1505,12 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
             k_place_nodes_outer<<<grid, kThreads, 0, st>>>(d->hdr, d->newlist[0], id_bits, off_next, d->nodes, d->node_batch);
             ctx->launches += 3;
         }
-        {
+        if (!(smem_last && h == k - 1)) {   // (the last hop's shared-memory kernel leaves final rows)
             ProfScope ps(ctx, PH_SAMPLE_RELABEL, 1);
             k_relabel<<<grid, kThreads, 0, st>>>(d->hdr, h, d->hvals, d->ent_repr);
+            ctx->launches++;
         }
-        ctx->launches += 1 + 1 + 1 + 1;  // count, entries_done, pick, relabel
+        ctx->launches += 1 + 1 + 1;  // count, entries_done, pick
     }
     {
         ProfScope ps(ctx, PH_SAMPLE_FINAL, 1);
@@ -1251,13 +1532,13 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
     memset(&sig, 0, sizeof(sig));
     sig.B = B; sig.k = k; sig.T = 0; sig.table_size = table_size; sig.cap_batch = cap_batch;   // (the device work does not depend on T)
     sig.cap_nodes = d->cap_nodes; sig.cap_entries = d->cap_entries; sig.n_nodes = ctx->n_nodes; sig.part_size = ctx->part_size;
-    sig.inout = inout ? 1 : 0;
+    sig.inout = (inout ? 1 : 0) | (smem_last ? 2 + 4 * dedup_nb : 0);
     for (int h = 0; h < k; ++h) sig.fanouts[h] = fanouts[h];
     const void* ptrs[] = {d->hdr, d->nodes, d->node_batch, d->ent_off, d->node_r0, d->node_deg, d->newlist[0], d->newlist[1],
                           d->scan_tmp, d->sort_hist, d->ent_nbrs, d->ent_repr, d->hkeys, d->hvals, d->node_off, d->cum, d->rowbase,
                           d->d_ent_hop, d->d_seeds, d->h_stage, d->h_pinned_dev, ctx->view_off, ctx->view_nbrs, ctx->d_slot_of_part, st,
                           inout ? (const void*)ctx->view_off_out : nullptr, inout ? (const void*)ctx->view_nbrs_out : nullptr,
-                          d->node_r0_out, d->node_deg_out};
+                          d->node_r0_out, d->node_deg_out, d->pairs, d->share_off};
     static_assert(sizeof(ptrs) <= sizeof(sig.ptrs), "signature too small");
     memcpy(sig.ptrs, ptrs, sizeof(ptrs));
     const bool use_graph = ctx->sample_graphs && !ctx->prof_on && !getenv("MG_NO_SAMPLE_GRAPH");
@@ -1414,7 +1695,7 @@ extern "C" int mg_dense_view(mg_ctx* ctx, mg_dense* d, int32_t batch, mg_dense_a
 extern "C" int mg_dense_free(mg_dense* d) {
     if (!d) return MG_OK;
     cudaSetDevice(d->device);
-    cudaFree(d->hdr); cudaFree(d->nodes); cudaFree(d->node_batch); cudaFree(d->ent_off); cudaFree(d->node_r0); cudaFree(d->node_deg); cudaFree(d->node_r0_out); cudaFree(d->node_deg_out);
+    cudaFree(d->hdr); cudaFree(d->nodes); cudaFree(d->node_batch); cudaFree(d->ent_off); cudaFree(d->node_r0); cudaFree(d->node_deg); cudaFree(d->node_r0_out); cudaFree(d->node_deg_out); cudaFree(d->pairs); cudaFree(d->share_off);
     cudaFree(d->ent_nbrs); cudaFree(d->ent_repr); cudaFree(d->node_off); cudaFree(d->cum);
     cudaFree(d->rowbase); cudaFree(d->hkeys); cudaFree(d->hvals); cudaFree(d->newlist[0]);
     cudaFree(d->newlist[1]); cudaFree(d->d_seeds); cudaFree(d->batch_cnt); cudaFree(d->scan_tmp); cudaFree(d->sort_hist);

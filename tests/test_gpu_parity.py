@@ -761,3 +761,26 @@ def test_sum_aggregator(tiny):
     out = torch.empty((300, 16), dtype=torch.float32, device="cuda")
     ctx.forward(model, d1, out)
     close(out.cpu().numpy(), O.additive_layer(ref1, feats.numpy()[ref1["node_ids"]]), RTOL_AGG)
+
+
+@pytest.mark.parametrize("cap_batch", [0, 60_000, 900_000])
+def test_last_hop_deduplication_paths(tiny, cap_batch):
+    """The last hop is deduplicated in shared memory when a mini-batch's node capacity fits a few table blocks
+    (one block per mini-batch by default here, three buckets at 60,000) and through the global id table otherwise
+    (900,000): the arrays are the oracle's either way."""
+    g, feats = tiny
+    ctx = make_ctx(g, feats)
+    sizes = [150, 0, 1, 400]
+    tg = [inputs.distinct_targets(10_000, s, seed=60 + i) for i, s in enumerate(sizes)]
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    seeds = [5, 6, 7, 8]
+    caps = {"max_nodes_per_batch": cap_batch} if cap_batch else None
+    view = oracle_view(g)
+    for fanouts in ([6], [5, 4], [3, 3, 3]):
+        d = ctx.sample_many(torch.cat(tg), offs, fanouts, seeds, caps=caps)
+        for b in range(len(sizes)):
+            assert_dense_equal(d.view(b), O.sample_dense(view, tg[b].tolist(), fanouts, seeds[b]))
+    # a repeated target is still refused on every path
+    with pytest.raises(mg.MgError) as e:
+        ctx.sample_many(torch.tensor([3, 9, 3], dtype=torch.int32), [0, 3], [2], [1], caps=caps)
+    assert e.value.code == -4
