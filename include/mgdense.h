@@ -336,6 +336,34 @@ int mg_profile(mg_ctx* ctx, int enable);
 int mg_profile_read(mg_ctx* ctx, int32_t* n_phases, const char** names, double* ms, int64_t* launches,
                     int reset);
 
+/* ---- COMET: partition replacement for link prediction out of core (Section 5.1, Section 6) ----
+ * Host-side planning only; no context, no device work.  Partition ids are the physical partitions of
+ * mg_set_partitioning; a plan's sets drive mg_set_resident, its bucket table says which set trains edge bucket
+ * (i, j) = the edges from physical partition i to physical partition j. */
+
+/* One epoch's plan.  p physical partitions are grouped at random into l logical ones (p a multiple of l):
+ * logical_of_physical[p] (out).  The sequence of resident sets swaps ONE logical partition at a time, greedily by the
+ * number of partition pairs that share a set for the first time, until every pair has: sets (out) holds n_sets rows
+ * of c_l logical ids in buffer-slot order (a swap puts the new partition into the slot of the one it replaces;
+ * row 0 = 0 .. c_l - 1), at most cap_sets rows.  bucket_set[p * p] (out): for each edge bucket a set chosen
+ * uniformly among those that hold both of its partitions (deferred, randomised processing of training examples).
+ * All randomness is Philox keyed by `seed`.  Errors: MG_ERR_ARG (null pointer, p not a positive multiple of l, not
+ * 2 <= c_l <= l), MG_ERR_CAPACITY (more than cap_sets sets; l * l rows always suffice). */
+int mg_comet_plan(int32_t p, int32_t l, int32_t c_l, uint64_t seed, int32_t cap_sets, int32_t* logical_of_physical,
+                  int32_t* n_sets, int32_t* sets, int32_t* bucket_set);
+
+/* Edge Permutation Bias B of a bucket assignment (Section 6) under the uniform-degree assumption: every node of a
+ * physical partition shares one tally, bucket (i, j) counts once for i and once for j, tallies are normalised by
+ * their final value; B = max over sets of (largest - smallest tally).  Errors: MG_ERR_ARG. */
+int mg_comet_bias(int32_t p, int32_t n_sets, const int32_t* bucket_set, double* bias);
+
+/* The rules of Section 6: p = floor(min(NO / D, sqrt(EO / D))) (NO = n_nodes * dim * 4, EO = n_edges *
+ * bytes_per_edge, D = block_bytes), clamped to [2, max_parts]; c = the largest even buffer capacity with
+ * c * NO / p + 2 * c^2 * EO / p^2 + fudge_bytes < cpu_bytes whose half divides p (two logical partitions fill the
+ * buffer); l = 2 p / c.  Errors: MG_ERR_ARG, MG_ERR_CAPACITY when no capacity fits. */
+int mg_comet_autotune(int64_t n_nodes, int32_t dim, int64_t n_edges, int32_t bytes_per_edge, int64_t cpu_bytes,
+                      int64_t block_bytes, int64_t fudge_bytes, int32_t max_parts, int32_t* p, int32_t* l, int32_t* c);
+
 #ifdef __cplusplus
 }
 #endif

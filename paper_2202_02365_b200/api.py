@@ -31,7 +31,7 @@ EXPORTS = [
     "mg_load_features", "mg_set_resident", "mg_commit_resident", "mg_sample_many", "mg_sample_many_begin", "mg_sample_many_end", "mg_sample",
     "mg_dense_counts", "mg_dense_view", "mg_dense_free", "mg_model_create", "mg_model_set_aggregator", "mg_model_free",
     "mg_forward", "mg_set_layer_window", "mg_keep_layer_outputs", "mg_forward_host_async", "mg_wait_output", "mg_forward_noalloc", "mg_gather_h0", "mg_layer_output", "mg_lp_prepare", "mg_lp_view", "mg_lp_free",
-    "mg_distmult_score", "mg_kernel_launches", "mg_profile", "mg_profile_read",
+    "mg_distmult_score", "mg_kernel_launches", "mg_profile", "mg_profile_read", "mg_comet_plan", "mg_comet_bias", "mg_comet_autotune",
 ]
 
 
@@ -75,6 +75,46 @@ def _ptr(t: torch.Tensor | None):
 def _host(x, dtype) -> torch.Tensor:
     t = torch.as_tensor(x, dtype=dtype)
     return t.cpu().contiguous()
+
+
+def comet_plan(p: int, l: int, c_l: int, seed: int):
+    """One epoch's COMET plan (host-side, no GPU needed): logical grouping, the sequence of resident sets of
+    logical partitions, the set that trains each edge bucket, and the resident physical partitions of each set."""
+    lib = load_library()
+    cap = max(1, l * l)
+    lop = np.zeros(p, dtype=np.int32)
+    sets = np.zeros((cap, c_l), dtype=np.int32)
+    buckets = np.zeros((p, p), dtype=np.int32)
+    n = C.c_int32(0)
+    rc = lib.mg_comet_plan(C.c_int32(p), C.c_int32(l), C.c_int32(c_l), C.c_uint64(int(seed) & 0xFFFFFFFFFFFFFFFF), C.c_int32(cap),
+                           C.c_void_p(lop.ctypes.data), C.byref(n), C.c_void_p(sets.ctypes.data), C.c_void_p(buckets.ctypes.data))
+    if rc != MG_OK:
+        raise MgError(rc, "mg_comet_plan")
+    sets = sets[:n.value].copy()
+    physical = [sorted(int(q) for q in range(p) if lop[q] in set(s.tolist())) for s in sets]
+    return {"logical_of_physical": lop, "sets": sets, "bucket_set": buckets, "physical_sets": physical}
+
+
+def comet_bias(bucket_set: np.ndarray, n_sets: int) -> float:
+    lib = load_library()
+    b = np.ascontiguousarray(bucket_set, dtype=np.int32)
+    out = C.c_double(0.0)
+    rc = lib.mg_comet_bias(C.c_int32(b.shape[0]), C.c_int32(n_sets), C.c_void_p(b.ctypes.data), C.byref(out))
+    if rc != MG_OK:
+        raise MgError(rc, "mg_comet_bias")
+    return out.value
+
+
+def comet_autotune(n_nodes: int, dim: int, n_edges: int, bytes_per_edge: int, cpu_bytes: int, block_bytes: int,
+                   fudge_bytes: int, max_parts: int):
+    lib = load_library()
+    p, l, c = C.c_int32(0), C.c_int32(0), C.c_int32(0)
+    rc = lib.mg_comet_autotune(C.c_int64(n_nodes), C.c_int32(dim), C.c_int64(n_edges), C.c_int32(bytes_per_edge),
+                               C.c_int64(cpu_bytes), C.c_int64(block_bytes), C.c_int64(fudge_bytes), C.c_int32(max_parts),
+                               C.byref(p), C.byref(l), C.byref(c))
+    if rc != MG_OK:
+        raise MgError(rc, "mg_comet_autotune")
+    return p.value, l.value, c.value
 
 
 class _DeviceInts:

@@ -784,3 +784,62 @@ def test_last_hop_deduplication_paths(tiny, cap_batch):
     with pytest.raises(mg.MgError) as e:
         ctx.sample_many(torch.tensor([3, 9, 3], dtype=torch.int32), [0, 3], [2], [1], caps=caps)
     assert e.value.code == -4
+
+
+def test_comet_epoch_drives_the_partition_buffer():
+    """One link-prediction epoch out of core under a COMET plan (Section 5.1): the plan's sets go through
+    mg_set_resident / mg_commit_resident with host-backed embeddings, every set trains the edges of the buckets it
+    was given, and every edge of the graph is trained exactly once; two of the sets are checked against the oracle
+    end to end (negatives, target union, DENSE sample, layer, DistMult)."""
+    n, p, l, c_l = 6000, 12, 6, 2
+    g = inputs.rmat_graph(n, 40_000, seed=8, n_relations=11)
+    emb = inputs.normal_features(n, 16, seed=4, std=0.01, pin=False).pin_memory()
+    rel_emb = inputs.normal_features(11, 8, seed=6)
+    plan = mg.comet_plan(p, l, c_l, seed=77)
+    cap = c_l * (p // l)
+    ctx = mg.Context(0)
+    ctx.load_graph(g.row_offsets.cuda(), g.nbrs.cuda())
+    ctx.set_partitioning(p)
+    ctx.load_features(emb, capacity_parts=cap, backing=mg.BACKING_HOST)
+    layers = inputs.random_bias_layers([16, 8], seed=2)
+    model = ctx.model(layers, mg.GEMM_FP32)
+    # every CSR slot is an edge dst <- src; its bucket is (partition of src, partition of dst)
+    part_size = (n + p - 1) // p
+    dst_all = torch.repeat_interleave(torch.arange(n), g.row_offsets[1:] - g.row_offsets[:-1])
+    src_all = g.nbrs.long()
+    set_of_edge = torch.as_tensor(plan["bucket_set"])[src_all // part_size, dst_all // part_size]
+    trained = torch.zeros(g.n_edges, dtype=torch.int32)
+    swaps = 0
+    prev = None
+    for k, resident in enumerate(plan["physical_sets"]):
+        assert len(resident) == cap
+        if prev is not None:
+            swaps += len(set(resident) - set(prev))
+        prev = resident
+        ctx.set_resident(resident, async_=True)
+        ctx.commit_resident(10_000)
+        mine = torch.nonzero(set_of_edge == k).flatten()
+        trained[mine] += 1
+        if mine.numel() == 0:
+            continue
+        src, dst, rel = src_all[mine].int(), dst_all[mine].int(), g.edge_rel[mine]
+        lp = ctx.lp_prepare(src, rel, dst, 2, 50, seed=900 + k)        # both endpoints resident by construction
+        got = lp.view()
+        d = ctx.sample(got["targets"], [8], seed=k)
+        h = torch.empty((got["targets"].numel(), 8), dtype=torch.float32, device="cuda")
+        ctx.forward(model, d, h)
+        pos, nd, ns = ctx.distmult_score(lp, h, rel_emb.cuda(), precision=mg.GEMM_FP32)
+        if k in (0, len(plan["physical_sets"]) - 1):
+            view = oracle_view(g, p, resident)
+            prep = O.lp_prepare(view, src.tolist(), dst.tolist(), 2, 50, 900 + k)
+            assert got["targets"].cpu().tolist() == prep["targets"]
+            ref = O.sample_dense(view, prep["targets"], [8], k)
+            assert_dense_equal(d.view(0), ref)
+            ref_h = O.forward(ref, emb.numpy()[ref["node_ids"]], [(w.numpy(), nn.numpy(), b.numpy()) for w, nn, b in layers])
+            close(h.cpu().numpy(), ref_h, RTOL_AGG)
+            rpos, rnd, rns = O.distmult_scores(ref_h, rel_emb.numpy(), prep, rel.tolist(), 2)
+            close(pos.cpu().numpy(), rpos, RTOL_AGG)
+            close(nd.cpu().numpy(), rnd, RTOL_AGG)
+            close(ns.cpu().numpy(), rns, RTOL_AGG)
+    assert bool((trained == 1).all())                                   # an epoch trains every edge once
+    assert swaps == (len(plan["physical_sets"]) - 1) * (p // l)         # one logical partition per step
