@@ -39,6 +39,9 @@ Points the paper leaves open, and the reading taken here:
     over the sampled neighbours (0 when there are none), ReLU between layers and
     none after the last.
   * DistMult: score(s, r, o) = sum_d h_s[d] * rel_r[d] * h_o[d].
+  * graph attention (the paper names GAT by citation only): one head, the node itself is
+    one of the attended rows, LeakyReLU slope 0.2, ReLU between layers and none after
+    the last, bias after the weighted sum.
 """
 from __future__ import annotations
 
@@ -296,6 +299,41 @@ def sage_layer(dense, h_prev, w_self, w_nbr, bias, relu: bool, aggregator: str =
            + nbr_aggr @ np.asarray(w_nbr, dtype=np.float64)
            + np.asarray(bias, dtype=np.float64))
     return np.maximum(out, 0.0) if relu else out
+
+
+def gat_layer(dense, h_prev, w, a_src, a_dst, bias, relu: bool, slope: float = 0.2):
+    """One graph-attention layer (the GAT of Velickovic et al., which Section 7.1 trains as the second model) over
+    DENSE, single head: z = h W for every input row; for output row i with sampled neighbours j (repeats count) and
+    itself, e_ij = LeakyReLU(a_dst . z_i + a_src . z_j), alpha = softmax over {i} + neighbours, h'_i = sum alpha_ij z_j
+    + bias.  A node without neighbours attends to itself only."""
+    h_prev = np.asarray(h_prev, dtype=np.float64)
+    z = h_prev @ np.asarray(w, dtype=np.float64)
+    s_src = z @ np.asarray(a_src, dtype=np.float64)
+    s_dst = z @ np.asarray(a_dst, dtype=np.float64)
+    first = dense["node_id_offsets"][1]
+    n_rows = len(dense["node_ids"]) - first
+    repr_map, nbr_offsets = dense["repr_map"], dense["nbr_offsets"]
+    out = np.zeros((n_rows, z.shape[1]), dtype=np.float64)
+    for r in range(n_rows):
+        me = first + r
+        src = [me] + [repr_map[e] for e in range(nbr_offsets[r], nbr_offsets[r + 1])]
+        e = np.array([s_dst[me] + s_src[j] for j in src])
+        e = np.where(e > 0, e, slope * e)
+        a = np.exp(e - e.max())
+        a /= a.sum()
+        out[r] = (a[:, None] * z[src]).sum(axis=0)
+    out = out + np.asarray(bias, dtype=np.float64)
+    return np.maximum(out, 0.0) if relu else out
+
+
+def gat_forward(dense, h0, layers, slope: float = 0.2):
+    """k attention layers with Algorithm 2 between them; layers: (w, a_src, a_dst, bias); ReLU on all but the last."""
+    h = np.asarray(h0, dtype=np.float64)
+    cur = {key: list(val) for key, val in dense.items()}
+    for i, (w, a_src, a_dst, bias) in enumerate(layers):
+        h = gat_layer(cur, h, w, a_src, a_dst, bias, relu=(i + 1 < len(layers)), slope=slope)
+        cur = update_dense(cur)
+    return h
 
 
 def forward(dense, h0, layers, return_all: bool = False, aggregator: str = "mean"):

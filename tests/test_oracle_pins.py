@@ -582,3 +582,87 @@ def test_sum_aggregator_reduces_to_algorithm_3_and_to_count_times_mean():
     np.testing.assert_allclose(got, h.numpy(), rtol=1e-12, atol=1e-12)
     with pytest.raises(ValueError):
         O.sage_layer(d, h0, eye, eye, zero, relu=False, aggregator="max")
+
+
+# ---------------------------------------------------------------- graph attention over DENSE
+def test_gat_uniform_attention_is_the_mean_over_self_and_neighbours():
+    off, nb = _random_graph(90, 700, 1)
+    d = O.sample_dense(O.GraphView(off, nb), [3, 30, 60, 7], [4, 2], seed=2)
+    rng = np.random.default_rng(1)
+    h0 = rng.standard_normal((len(d["node_ids"]), 5))
+    w, b = rng.standard_normal((5, 3)), rng.standard_normal(3)
+    got = O.gat_layer(d, h0, w, np.zeros(3), np.zeros(3), b, relu=False)
+    n_rows = len(d["node_ids"]) - d["node_id_offsets"][1]
+    counts = np.diff(d["nbr_offsets"])[:n_rows, None]
+    total = O.sage_layer(d, h0, w, w, np.zeros(3), relu=False, aggregator="sum")      # (self + sum of neighbours) W
+    np.testing.assert_allclose(got, total / (counts + 1) + b, rtol=1e-12, atol=1e-12)
+
+
+def test_gat_full_fanout_equals_dense_masked_softmax_algebra():
+    off, nb = _random_graph(50, 260, 4)
+    n = 50
+    maxdeg = int(np.diff(off).max())
+    targets = list(range(0, 50, 3))
+    d = O.sample_dense(O.GraphView(off, nb), targets, [maxdeg], seed=0)
+    rng = np.random.default_rng(3)
+    feats = rng.standard_normal((n, 6))
+    w, a_s, a_d, b = rng.standard_normal((6, 4)), rng.standard_normal(4), rng.standard_normal(4), rng.standard_normal(4)
+    got = O.gat_layer(d, feats[d["node_ids"]], w, a_s, a_d, b, relu=True)
+    # whole graph, dense: multiplicity matrix + identity, masked softmax row by row in torch
+    A = torch.zeros((n, n), dtype=torch.float64)
+    for v in range(n):
+        for u in nb[off[v]:off[v + 1]]:
+            A[v, int(u)] += 1
+    A += torch.eye(n, dtype=torch.float64)
+    Z = torch.tensor(feats) @ torch.tensor(w)
+    E = torch.nn.functional.leaky_relu((Z @ torch.tensor(a_d))[:, None] + (Z @ torch.tensor(a_s))[None, :], 0.2)
+    P = A * torch.exp(E - E.max())
+    P = P / P.sum(1, keepdim=True)
+    want = torch.relu(P @ Z + torch.tensor(b))[targets].numpy()
+    np.testing.assert_allclose(got, want, rtol=1e-10, atol=1e-12)
+
+
+def test_gat_sharp_attention_picks_the_best_scoring_row_and_isolated_nodes_keep_themselves():
+    # node 0 aggregates from 1, 2, 3; node 4 has no neighbours
+    off = np.array([0, 3, 3, 3, 3, 3])
+    nb = np.array([1, 2, 3])
+    d = O.sample_dense(O.GraphView(off, nb), [0, 4], [5], seed=0)
+    h0 = np.array([[0.0, 1.0], [1.0, 2.0], [3.0, 3.0], [2.0, 4.0], [5.0, 5.0]])[d["node_ids"]]
+    eye = np.eye(2)
+    out = O.gat_layer(d, h0, eye, np.array([50.0, 0.0]), np.zeros(2), np.zeros(2), relu=False)
+    rows = {v: out[i] for i, v in enumerate(d["node_ids"][d["node_id_offsets"][1]:])}
+    np.testing.assert_allclose(rows[0], [3.0, 3.0], atol=1e-12)      # neighbour 2 has the largest first coordinate
+    np.testing.assert_allclose(rows[4], [5.0, 5.0], atol=1e-12)      # attends to itself only
+    # hand-computed softmax: scores ln 1, ln 2, ln 3, ln 4 for (self, 1, 2, 3) -> weights 0.1 .. 0.4
+    h1 = np.array([[np.log(1.0)], [np.log(2.0)], [np.log(3.0)], [np.log(4.0)], [0.0]])[d["node_ids"]]
+    vals = O.gat_layer(d, h1, np.ones((1, 1)), np.ones(1), np.zeros(1), np.zeros(1), relu=False)
+    want = 0.1 * np.log(1.0) + 0.2 * np.log(2.0) + 0.3 * np.log(3.0) + 0.4 * np.log(4.0)
+    got0 = vals[[i for i, v in enumerate(d["node_ids"][d["node_id_offsets"][1]:]) if v == 0][0]]
+    np.testing.assert_allclose(got0, [want], rtol=1e-12)
+
+
+def test_gat_forward_two_layers_uses_algorithm_2_between_layers():
+    off, nb = _random_graph(80, 500, 6)
+    maxdeg = int(np.diff(off).max())
+    targets = [1, 11, 21]
+    d = O.sample_dense(O.GraphView(off, nb), targets, [maxdeg, maxdeg], seed=0)
+    rng = np.random.default_rng(5)
+    feats = rng.standard_normal((80, 4))
+    layers = [(rng.standard_normal((4, 3)), rng.standard_normal(3), rng.standard_normal(3), rng.standard_normal(3)),
+              (rng.standard_normal((3, 2)), rng.standard_normal(2), rng.standard_normal(2), rng.standard_normal(2))]
+    got = O.gat_forward(d, feats[d["node_ids"]], layers)
+    # with full fanouts the two layers are whole-graph attention layers on the 2-hop ball
+    A = torch.zeros((80, 80), dtype=torch.float64)
+    for v in range(80):
+        for u in nb[off[v]:off[v + 1]]:
+            A[v, int(u)] += 1
+    A += torch.eye(80, dtype=torch.float64)
+    H = torch.tensor(feats)
+    for i, (w, a_s, a_d, b) in enumerate(layers):
+        Z = H @ torch.tensor(w)
+        E = torch.nn.functional.leaky_relu((Z @ torch.tensor(a_d))[:, None] + (Z @ torch.tensor(a_s))[None, :], 0.2)
+        P = A * torch.exp(E - E.max())
+        H = (P / P.sum(1, keepdim=True)) @ Z + torch.tensor(b)
+        if i == 0:
+            H = torch.relu(H)
+    np.testing.assert_allclose(got, H[targets].numpy(), rtol=1e-9, atol=1e-11)
