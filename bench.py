@@ -177,6 +177,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(CONFIGS) + [LP_WORKLOAD])
     ap.add_argument("--group", type=int, default=0, help="mini-batches per step (default: 128, or the workload's own)")
     ap.add_argument("--window", type=int, default=0, help="mini-batches per window of the layer schedule (0 = whole layers)")
+    ap.add_argument("--lp-model", default="graphsage", choices=["graphsage", "gat"],
+                    help="link-prediction workload only: the encoder layer (GraphSage mean or single-head graph attention)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     args = ap.parse_args()
@@ -455,6 +457,12 @@ def run_lp(args, peaks, rank, local_rank, world):
     torch.cuda.empty_cache()
     layers = inputs.glorot_layers([c["dim"], c["dim"]], seed=8)
     model = ctx.model(layers, mg.GEMM_TF32)
+    gat = None
+    if args.lp_model == "gat":
+        gen = torch.Generator().manual_seed(9)
+        w = layers[0][0]
+        gat = ctx.gat_model([(w, torch.randn(c["dim"], generator=gen) * 0.1, torch.randn(c["dim"], generator=gen) * 0.1,
+                              torch.zeros(c["dim"]))], mg.GEMM_TF32)
     dense = None
     h = None
     stats = {"targets": [], "entries": []}
@@ -467,7 +475,10 @@ def run_lp(args, peaks, rank, local_rank, world):
         dense = ctx.sample(targets, [c["fanout"]], seed=i, out=dense)
         if h is None or h.shape[0] < targets.numel():
             h = torch.empty((int(targets.numel() * 1.2) + 16, c["dim"]), dtype=torch.float32, device=device)
-        ctx.forward(model, dense, h[:targets.numel()])
+        if gat is not None:
+            ctx.gat_forward(gat, dense, h[:targets.numel()])
+        else:
+            ctx.forward(model, dense, h[:targets.numel()])
         scores = ctx.distmult_score(lp, h[:targets.numel()], rel_emb)
         if record:
             n_, e_ = dense.counts()
@@ -518,7 +529,7 @@ def run_lp(args, peaks, rank, local_rank, world):
         "vs_baseline": None, "dtype": "f32 (TF32 tensor-core GEMM)", "data": "synthetic",
         "config": {"workload": LP_WORKLOAD, "nodes": c["n"], "edges": n_edges_graph, "embedding_dim": dim,
                    "relations": c["n_rel"], "partitions": c["parts"], "resident": len(resident), "edges_per_step": B,
-                   "chunks": c["chunks"], "negatives_per_chunk": negs, "fanouts": [c["fanout"]],
+                   "chunks": c["chunks"], "negatives_per_chunk": negs, "fanouts": [c["fanout"]], "encoder": args.lp_model,
                    "l2": "inputs larger than L2 (embedding table 34 GB, scores 400 MB per step; no flush)",
                    "setup_s": {"graph_and_embeddings_s": setup_s}},
         "scored_pairs_per_s": args.steps * world * B * (1 + 2 * negs) / (ms / 1e3),

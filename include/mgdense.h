@@ -336,6 +336,25 @@ int mg_profile(mg_ctx* ctx, int enable);
 int mg_profile_read(mg_ctx* ctx, int32_t* n_phases, const char** names, double* ms, int64_t* launches,
                     int reset);
 
+/* ---- graph attention over DENSE (the GAT model of Section 7.1) --------------------------- */
+
+typedef struct mg_gat_model mg_gat_model;
+
+/* k single-head attention layers of widths dims[0] -> ... -> dims[k] (multiples of 4; dims[1..k] <= 512).  Layer l + 1:
+ * z = h w[l] for every input row; for an output row i with sampled neighbours j (repeats count) and itself,
+ * e_ij = LeakyReLU(a_dst[l] . z_i + a_src[l] . z_j) with slope negative_slope, alpha = softmax over {i} + neighbours,
+ * h'_i = sum alpha_ij z_j + bias[l]; ReLU on all but the last layer; a node without neighbours attends to itself.
+ * w[l] HOST row-major [dims[l], dims[l+1]]; a_src[l], a_dst[l], bias[l] HOST [dims[l+1]] (all copied).
+ * gemm_precision as in mg_model_create.  Errors: MG_ERR_ARG, MG_ERR_OOM. */
+int mg_gat_model_create(mg_ctx* ctx, int32_t k, const int32_t* dims, const float* const* w, const float* const* a_src,
+                        const float* const* a_dst, const float* const* bias, float negative_slope, int gemm_precision,
+                        mg_gat_model** out);
+int mg_gat_model_free(mg_gat_model* m);
+
+/* Attention forward pass for every batch of `d`; out_dev (DEVICE) receives one row of dims[k] floats per target, batch
+ * after batch in the caller's target order.  Synchronous on the context's stream.  Errors as mg_forward. */
+int mg_gat_forward(mg_ctx* ctx, const mg_gat_model* m, mg_dense* d, float* out_dev);
+
 /* ---- COMET: partition replacement for link prediction out of core (Section 5.1, Section 6) ----
  * Host-side planning only; no context, no device work.  Partition ids are the physical partitions of
  * mg_set_partitioning; a plan's sets drive mg_set_resident, its bucket table says which set trains edge bucket

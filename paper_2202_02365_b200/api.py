@@ -31,7 +31,7 @@ EXPORTS = [
     "mg_load_features", "mg_set_resident", "mg_commit_resident", "mg_sample_many", "mg_sample_many_begin", "mg_sample_many_end", "mg_sample",
     "mg_dense_counts", "mg_dense_view", "mg_dense_free", "mg_model_create", "mg_model_set_aggregator", "mg_model_free",
     "mg_forward", "mg_set_layer_window", "mg_keep_layer_outputs", "mg_forward_host_async", "mg_wait_output", "mg_forward_noalloc", "mg_gather_h0", "mg_layer_output", "mg_lp_prepare", "mg_lp_view", "mg_lp_free",
-    "mg_distmult_score", "mg_kernel_launches", "mg_profile", "mg_profile_read", "mg_comet_plan", "mg_comet_bias", "mg_comet_autotune",
+    "mg_distmult_score", "mg_kernel_launches", "mg_profile", "mg_profile_read", "mg_comet_plan", "mg_comet_bias", "mg_comet_autotune", "mg_gat_model_create", "mg_gat_model_free", "mg_gat_forward",
 ]
 
 
@@ -213,6 +213,38 @@ class Model:
             pass
 
 
+class GatModel:
+    """layers: list of (w [d_in, d_out], a_src [d_out], a_dst [d_out], bias [d_out]) host tensors."""
+
+    def __init__(self, ctx: "Context", layers, precision: int = GEMM_TF32, negative_slope: float = 0.2):
+        self.ctx = ctx
+        self.handle = C.c_void_p(0)
+        k = len(layers)
+        self.dims = [int(layers[0][0].shape[0])] + [int(l[0].shape[1]) for l in layers]
+        keep, arrs = [], []
+        for idx in range(4):
+            ptrs = (C.c_void_p * k)()
+            for i, l in enumerate(layers):
+                t = _host(l[idx], torch.float32)
+                keep.append(t)
+                ptrs[i] = t.data_ptr()
+            arrs.append(ptrs)
+        dims = (C.c_int32 * (k + 1))(*self.dims)
+        ctx._check(ctx.lib.mg_gat_model_create(ctx.handle, C.c_int32(k), dims, arrs[0], arrs[1], arrs[2], arrs[3],
+                                               C.c_float(negative_slope), C.c_int(precision), C.byref(self.handle)))
+
+    def free(self):
+        if self.handle:
+            self.ctx.lib.mg_gat_model_free(self.handle)
+            self.handle = C.c_void_p(0)
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
 class LpBatch:
     def __init__(self, ctx: "Context"):
         self.ctx = ctx
@@ -336,6 +368,13 @@ class Context:
 
     def commit_resident(self, timeout_ms: int = 60000):
         self._check(self.lib.mg_commit_resident(self.handle, C.c_int32(timeout_ms)))
+
+    def gat_model(self, layers, precision: int = GEMM_TF32, negative_slope: float = 0.2) -> "GatModel":
+        return GatModel(self, layers, precision, negative_slope)
+
+    def gat_forward(self, model: "GatModel", dense: "Dense", out: torch.Tensor):
+        assert out.is_cuda and out.dtype == torch.float32 and out.is_contiguous()
+        self._check(self.lib.mg_gat_forward(self.handle, model.handle, dense.handle, _ptr(out)))
 
     # -- sampling
     def _sample_many_call(self, fn, targets, target_offsets, fanouts, seeds, caps, out):

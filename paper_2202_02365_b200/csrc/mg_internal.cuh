@@ -136,6 +136,8 @@ struct mg_ctx {
     // loop of prepare / free allocates nothing
     char* lp_ws = nullptr; size_t lp_ws_bytes = 0;
     char* lp_spare = nullptr; size_t lp_spare_bytes = 0;
+    float* gat_x = nullptr; float* gat_z = nullptr; float* gat_s = nullptr; float* gat_h[2] = {nullptr, nullptr};   // mg_gat_forward scratch
+    size_t gat_x_elems = 0, gat_z_elems = 0, gat_s_elems = 0, gat_h_elems[2] = {0, 0};
     char* dm_images = nullptr; size_t dm_images_bytes = 0;   // TF32 operand images of the negatives (mg_distmult_score)
     bool prof_on = false;
     bool sample_graphs = true;   // replay the sampler's launches from a CUDA graph

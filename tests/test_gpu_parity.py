@@ -843,3 +843,74 @@ def test_comet_epoch_drives_the_partition_buffer():
             close(ns.cpu().numpy(), rns, RTOL_AGG)
     assert bool((trained == 1).all())                                   # an epoch trains every edge once
     assert swaps == (len(plan["physical_sets"]) - 1) * (p // l)         # one logical partition per step
+
+
+def _gat_layers(dims, seed):
+    g = torch.Generator().manual_seed(seed)
+    out = []
+    for di, dn in zip(dims[:-1], dims[1:]):
+        bound = (6.0 / (di + dn)) ** 0.5
+        w = (torch.rand((di, dn), generator=g) * 2 - 1) * bound
+        a_s = torch.randn(dn, generator=g) * 0.5
+        a_d = torch.randn(dn, generator=g) * 0.5
+        b = torch.randn(dn, generator=g) * 0.1
+        out.append((w, a_s, a_d, b))
+    return out
+
+
+@pytest.mark.parametrize("dims,fanouts", [([16, 8], [6]), ([16, 32, 12], [5, 3]), ([16, 260, 64, 4], [4, 3, 2])])
+def test_graph_attention_forward(tiny, dims, fanouts):
+    """The attention layers over DENSE against the oracle: fp32 GEMM and TF32 tensor-core GEMM, several mini-batches
+    (one empty, one with a single target), in-only and incoming + outgoing samples."""
+    g, feats = tiny
+    ctx = make_ctx(g, feats)
+    sizes = [120, 0, 1, 300]
+    tg = [inputs.distinct_targets(10_000, s, seed=70 + i) for i, s in enumerate(sizes)]
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    seeds = [11, 12, 13, 14]
+    layers = _gat_layers(dims, seed=len(dims))
+    np_layers = [tuple(t.numpy() for t in l) for l in layers]
+    view = oracle_view(g)
+    d = ctx.sample_many(torch.cat(tg), offs, fanouts, seeds)
+    refs = [O.sample_dense(view, tg[b].tolist(), fanouts, seeds[b]) for b in range(len(sizes))]
+    wants = [O.gat_forward(r, feats.numpy()[r["node_ids"]], np_layers) if sizes[b] else None for b, r in enumerate(refs)]
+    for prec, rtol in ((mg.GEMM_FP32, 2e-5), (mg.GEMM_TF32, RTOL_TC)):
+        model = ctx.gat_model(layers, prec)
+        out = torch.full((int(offs[-1]), dims[-1]), float("nan"), dtype=torch.float32, device="cuda")
+        ctx.gat_forward(model, d, out)
+        for b in range(len(sizes)):
+            if sizes[b]:
+                close(out[offs[b]:offs[b + 1]].cpu().numpy(), wants[b], rtol)
+    # uniform attention (a = 0) is the mean over the node and its sampled neighbours of h W
+    flat = [(w, torch.zeros_like(a), torch.zeros_like(a), b) for w, a, _, b in layers[:1]]
+    if len(dims) == 2:
+        model = ctx.gat_model(flat, mg.GEMM_FP32)
+        out = torch.empty((int(offs[-1]), dims[-1]), dtype=torch.float32, device="cuda")
+        ctx.gat_forward(model, d, out)
+        r = refs[3]
+        h0 = feats.numpy()[r["node_ids"]].astype(np.float64)
+        total = O.sage_layer(r, h0, flat[0][0].numpy(), flat[0][0].numpy(), np.zeros(dims[1]), relu=False, aggregator="sum")
+        counts = np.diff(r["nbr_offsets"])[:sizes[3], None]
+        close(out[offs[3]:offs[4]].cpu().numpy(), total / (counts + 1) + flat[0][3].numpy(), 2e-5)
+
+
+def test_graph_attention_errors_and_fp16_features():
+    n = 3000
+    g = inputs.rmat_graph(n, 30_000, seed=3)
+    feats16 = inputs.normal_features(n, 24, seed=2, dtype=torch.float16)
+    ctx = make_ctx(g, feats16)
+    layers = _gat_layers([24, 8], seed=1)
+    targets = inputs.distinct_targets(n, 200, seed=5)
+    d = ctx.sample(targets, [7], seed=3)
+    ref = O.sample_dense(oracle_view(g), targets.tolist(), [7], 3)
+    want = O.gat_forward(ref, feats16.float().numpy()[ref["node_ids"]], [tuple(t.numpy() for t in l) for l in layers])
+    model = ctx.gat_model(layers, mg.GEMM_FP32)
+    out = torch.empty((200, 8), dtype=torch.float32, device="cuda")
+    ctx.gat_forward(model, d, out)
+    close(out.cpu().numpy(), want, 2e-5)
+    with pytest.raises(mg.MgError) as e:
+        ctx.gat_model(_gat_layers([24, 516], seed=1))           # wider than an attention row may be
+    assert e.value.code == -1
+    with pytest.raises(mg.MgError) as e:
+        ctx.gat_forward(ctx.gat_model(_gat_layers([24, 8, 8], seed=1)), d, out)     # two layers, one hop
+    assert e.value.code == -2
