@@ -354,6 +354,49 @@ def forward(dense, h0, layers, return_all: bool = False, aggregator: str = "mean
     return outs if return_all else h
 
 
+def backward(dense, h0, layers, d_out, aggregator: str = "mean"):
+    """Gradients of a scalar loss through forward(): d_out = dL/dH^k, one row per target.
+
+    The chain rule through Algorithm 3 (self and neighbour linears, mean or sum over the
+    sampled neighbours through repr_map, ReLU on all but the last layer) and Algorithm 2
+    (layer l's rows are the rows of layer l-1 without the outermost delta).  Returns
+    (grads, d_h0): grads[l] = (dW_self, dW_nbr, dbias) of layer l + 1, d_h0 = dL/dH^0 with one
+    row per entry of node_ids (the gradient of the base representations, Section 3)."""
+    h = np.asarray(h0, dtype=np.float64)
+    cur = {key: list(val) for key, val in dense.items()}
+    saved = []
+    for i, (w_self, w_nbr, bias) in enumerate(layers):
+        first = cur["node_id_offsets"][1]
+        n_rows = len(cur["node_ids"]) - first
+        nbr_repr = h[np.asarray(cur["repr_map"], dtype=np.int64)]
+        agg = _segment_reduce(nbr_repr, cur["nbr_offsets"], n_rows, mean=(aggregator == "mean"))
+        pre = (h[first:] @ np.asarray(w_self, dtype=np.float64) + agg @ np.asarray(w_nbr, dtype=np.float64)
+               + np.asarray(bias, dtype=np.float64))
+        saved.append((cur, h, agg, pre))
+        h = np.maximum(pre, 0.0) if i + 1 < len(layers) else pre
+        cur = update_dense(cur)
+    d_h = np.asarray(d_out, dtype=np.float64)
+    grads = [None] * len(layers)
+    for i in range(len(layers) - 1, -1, -1):
+        cur, h_in, agg, pre = saved[i]
+        w_self, w_nbr = (np.asarray(x, dtype=np.float64) for x in layers[i][:2])
+        d_pre = d_h * (pre > 0.0) if i + 1 < len(layers) else d_h
+        first = cur["node_id_offsets"][1]
+        n_rows = len(cur["node_ids"]) - first
+        grads[i] = (h_in[first:].T @ d_pre, agg.T @ d_pre, d_pre.sum(axis=0))
+        d_in = np.zeros_like(h_in)
+        d_in[first:] += d_pre @ w_self.T
+        d_agg = d_pre @ w_nbr.T
+        for r in range(n_rows):
+            lo, hi = cur["nbr_offsets"][r], cur["nbr_offsets"][r + 1]
+            if hi > lo:
+                share = d_agg[r] / (hi - lo) if aggregator == "mean" else d_agg[r]
+                for e in range(lo, hi):
+                    d_in[cur["repr_map"][e]] += share
+        d_h = d_in
+    return grads, d_h
+
+
 # ----------------------------------------------------------------------------
 # Link prediction: shared uniform negatives, target union, DistMult
 # ----------------------------------------------------------------------------

@@ -666,3 +666,79 @@ def test_gat_forward_two_layers_uses_algorithm_2_between_layers():
         if i == 0:
             H = torch.relu(H)
     np.testing.assert_allclose(got, H[targets].numpy(), rtol=1e-9, atol=1e-11)
+
+
+# ---------------------------------------------------------------- backward pass
+@pytest.mark.parametrize("aggregator", ["mean", "sum"])
+def test_backward_equals_central_finite_differences(aggregator):
+    off, nb = _random_graph(70, 420, 9)
+    d = O.sample_dense(O.GraphView(off, nb), [2, 33, 64, 8, 50], [3, 2], seed=1)
+    rng = np.random.default_rng(2)
+    h0 = rng.standard_normal((len(d["node_ids"]), 4))
+    layers = [(rng.standard_normal((4, 5)) * 0.7, rng.standard_normal((4, 5)) * 0.7, rng.standard_normal(5) * 0.3),
+              (rng.standard_normal((5, 3)) * 0.7, rng.standard_normal((5, 3)) * 0.7, rng.standard_normal(3) * 0.3)]
+    g_out = rng.standard_normal((5, 3))
+
+    def loss(h0_, layers_):
+        return float((O.forward(d, h0_, layers_, aggregator=aggregator) * g_out).sum())
+
+    grads, d_h0 = O.backward(d, h0, layers, g_out, aggregator=aggregator)
+    eps = 1e-6
+    checks = 0
+    for li in range(2):
+        for pi in range(3):
+            arr = layers[li][pi]
+            for idx in list(np.ndindex(arr.shape))[::3]:
+                plus = [tuple(np.array(x, copy=True) for x in l) for l in layers]
+                minus = [tuple(np.array(x, copy=True) for x in l) for l in layers]
+                plus[li][pi][idx] += eps
+                minus[li][pi][idx] -= eps
+                fd = (loss(h0, plus) - loss(h0, minus)) / (2 * eps)
+                assert abs(fd - grads[li][pi][idx]) <= 1e-6 * max(1.0, abs(fd))
+                checks += 1
+    for r in range(0, h0.shape[0], 2):
+        for c in range(4):
+            hp, hm = h0.copy(), h0.copy()
+            hp[r, c] += eps
+            hm[r, c] -= eps
+            fd = (loss(hp, layers) - loss(hm, layers)) / (2 * eps)
+            assert abs(fd - d_h0[r, c]) <= 1e-6 * max(1.0, abs(fd))
+            checks += 1
+    assert checks > 80
+    # rows of the outermost delta only receive gradient through the neighbour term; a node nobody sampled gets none
+    used = set(d["repr_map"]) | set(range(d["node_id_offsets"][1], len(d["node_ids"])))
+    for r in range(len(d["node_ids"])):
+        if r not in used:
+            assert not d_h0[r].any()
+
+
+def test_backward_against_torch_autograd():
+    off, nb = _random_graph(60, 500, 3)
+    d = O.sample_dense(O.GraphView(off, nb), [1, 2, 3, 40], [4, 3, 2], seed=4)
+    rng = np.random.default_rng(8)
+    h0 = rng.standard_normal((len(d["node_ids"]), 3))
+    dims = [3, 4, 4, 2]
+    layers = [(rng.standard_normal((a, b)), rng.standard_normal((a, b)), rng.standard_normal(b)) for a, b in zip(dims[:-1], dims[1:])]
+    g_out = rng.standard_normal((4, 2))
+    grads, d_h0 = O.backward(d, h0, layers, g_out)
+    # the same network in torch, built from index_select / index_add_ on the DENSE arrays
+    th0 = torch.tensor(h0, requires_grad=True)
+    tl = [tuple(torch.tensor(x, requires_grad=True) for x in l) for l in layers]
+    cur, h = d, th0
+    for i, (ws, wn, b) in enumerate(tl):
+        first = cur["node_id_offsets"][1]
+        rows = len(cur["node_ids"]) - first
+        counts = torch.tensor(np.diff(cur["nbr_offsets"])[:rows])
+        seg = torch.repeat_interleave(torch.arange(rows), counts)
+        agg = torch.zeros((rows, h.shape[1]), dtype=torch.float64).index_add(0, seg, h[torch.tensor(cur["repr_map"], dtype=torch.int64)])
+        agg = agg / counts.clamp(min=1)[:, None]
+        h = h[first:] @ ws + agg @ wn + b
+        if i + 1 < len(tl):
+            h = torch.relu(h)
+        cur = O.update_dense(cur)
+    (h * torch.tensor(g_out)).sum().backward()
+    np.testing.assert_allclose(d_h0, th0.grad.numpy(), rtol=1e-10, atol=1e-12)
+    for (gs, gn, gb), (ws, wn, b) in zip(grads, tl):
+        np.testing.assert_allclose(gs, ws.grad.numpy(), rtol=1e-10, atol=1e-12)
+        np.testing.assert_allclose(gn, wn.grad.numpy(), rtol=1e-10, atol=1e-12)
+        np.testing.assert_allclose(gb, b.grad.numpy(), rtol=1e-10, atol=1e-12)
