@@ -336,6 +336,31 @@ int mg_profile(mg_ctx* ctx, int enable);
 int mg_profile_read(mg_ctx* ctx, int32_t* n_phases, const char** names, double* ms, int64_t* launches,
                     int reset);
 
+/* ---- backward pass and optimiser step (Section 3: a mini-batch's gradients update the model and the base
+ * representations) ------------------------------------------------------------------------ */
+
+/* Gradients of a scalar loss through the last mg_forward of (m, d), which must have run with
+ * mg_keep_layer_outputs(ctx, 1).  d_out_dev (DEVICE): dL/dH^k, one row of dims[k] floats per target, laid out like
+ * mg_forward's output.  The weight and bias gradients of every layer are left in buffers owned by the model
+ * (mg_model_grads), overwriting those of the previous call.  d_h0_dev (DEVICE, nullable): receives dL/dH^0, one row
+ * of dims[0] floats per node of every mini-batch in the library's packed row order -- mg_dense_packed_ids gives the
+ * node id of each row -- i.e. the gradient rows of the base representations.  fp32 arithmetic; sums over rows use
+ * atomic adds (low-order bits vary from run to run).  Synchronous.  Errors: MG_ERR_ARG, MG_ERR_STATE (no matching
+ * forward pass, layers not kept), MG_ERR_OOM. */
+int mg_backward(mg_ctx* ctx, mg_model* m, mg_dense* d, const float* d_out_dev, float* d_h0_dev);
+
+/* DEVICE pointers to the gradients mg_backward left for layer `layer` (1..k): d_w_self and d_w_nbr row-major
+ * [dims[layer-1], dims[layer]], d_bias [dims[layer]].  Owned by the model.  Errors: MG_ERR_ARG, MG_ERR_STATE. */
+int mg_model_grads(const mg_model* m, int32_t layer, const float** d_w_self, const float** d_w_nbr, const float** d_bias);
+
+/* One step of stochastic gradient descent on every weight and bias of the model with the gradients of the last
+ * mg_backward: w -= lr * dw.  Refreshes the copies the forward kernels read.  Synchronous. */
+int mg_model_sgd_step(mg_ctx* ctx, mg_model* m, float lr);
+
+/* ids_dev (DEVICE, int32, one per node of every mini-batch = the rows of H^0 in the library's packed order: batch
+ * after batch, targets first, then delta after delta in the order the nodes were found): the node id of each row. */
+int mg_dense_packed_ids(mg_ctx* ctx, mg_dense* d, int32_t* ids_dev);
+
 /* ---- graph attention over DENSE (the GAT model of Section 7.1) --------------------------- */
 
 typedef struct mg_gat_model mg_gat_model;

@@ -31,7 +31,7 @@ EXPORTS = [
     "mg_load_features", "mg_set_resident", "mg_commit_resident", "mg_sample_many", "mg_sample_many_begin", "mg_sample_many_end", "mg_sample",
     "mg_dense_counts", "mg_dense_view", "mg_dense_free", "mg_model_create", "mg_model_set_aggregator", "mg_model_free",
     "mg_forward", "mg_set_layer_window", "mg_keep_layer_outputs", "mg_forward_host_async", "mg_wait_output", "mg_forward_noalloc", "mg_gather_h0", "mg_layer_output", "mg_lp_prepare", "mg_lp_view", "mg_lp_free",
-    "mg_distmult_score", "mg_kernel_launches", "mg_profile", "mg_profile_read", "mg_comet_plan", "mg_comet_bias", "mg_comet_autotune", "mg_gat_model_create", "mg_gat_model_free", "mg_gat_forward",
+    "mg_distmult_score", "mg_kernel_launches", "mg_profile", "mg_profile_read", "mg_comet_plan", "mg_comet_bias", "mg_comet_autotune", "mg_gat_model_create", "mg_gat_model_free", "mg_gat_forward", "mg_backward", "mg_model_grads", "mg_model_sgd_step", "mg_dense_packed_ids",
 ]
 
 
@@ -129,6 +129,18 @@ def _from_dev(ptr, n: int, device) -> torch.Tensor:
     if n == 0 or not ptr:
         return torch.empty(0, dtype=torch.int32, device=device)
     return torch.as_tensor(_DeviceInts(ptr, n), device=device).clone()
+
+
+class _DeviceFloats:
+    def __init__(self, ptr: int, n: int):
+        self.__cuda_array_interface__ = {"shape": (n,), "typestr": "<f4", "data": (int(ptr), False), "version": 2}
+
+
+def _from_dev_f32(ptr, n: int, device) -> torch.Tensor:
+    """View n float32 values of a library-owned device buffer (the caller clones what it keeps)."""
+    if n == 0 or not ptr:
+        return torch.empty(0, dtype=torch.float32, device=device)
+    return torch.as_tensor(_DeviceFloats(ptr, n), device=device)
 
 
 @dataclass
@@ -368,6 +380,31 @@ class Context:
 
     def commit_resident(self, timeout_ms: int = 60000):
         self._check(self.lib.mg_commit_resident(self.handle, C.c_int32(timeout_ms)))
+
+    def backward(self, model: "Model", dense: "Dense", d_out: torch.Tensor, want_h0_grad: bool = False):
+        """Gradients through the last forward(model, dense) (keep_layer_outputs(True) must be set).  Returns the list of
+        (dW_self, dW_nbr, dbias) device tensors per layer and, on request, (dH0 rows, their node ids)."""
+        assert d_out.is_cuda and d_out.dtype == torch.float32 and d_out.is_contiguous()
+        nodes, _ = dense.counts()
+        n_rows = int(nodes.sum())
+        g_h0 = torch.empty((n_rows, model.dims[0]), dtype=torch.float32, device=d_out.device) if want_h0_grad else None
+        self._check(self.lib.mg_backward(self.handle, model.handle, dense.handle, _ptr(d_out), _ptr(g_h0)))
+        grads = []
+        for l in range(1, len(model.dims)):
+            ps, pn, pb = C.c_void_p(0), C.c_void_p(0), C.c_void_p(0)
+            self._check(self.lib.mg_model_grads(model.handle, C.c_int32(l), C.byref(ps), C.byref(pn), C.byref(pb)))
+            di, dn = model.dims[l - 1], model.dims[l]
+            grads.append((_from_dev_f32(ps.value, di * dn, d_out.device).view(di, dn).clone(),
+                          _from_dev_f32(pn.value, di * dn, d_out.device).view(di, dn).clone(),
+                          _from_dev_f32(pb.value, dn, d_out.device).clone()))
+        if not want_h0_grad:
+            return grads
+        ids = torch.empty(n_rows, dtype=torch.int32, device=d_out.device)
+        self._check(self.lib.mg_dense_packed_ids(self.handle, dense.handle, _ptr(ids)))
+        return grads, g_h0, ids
+
+    def sgd_step(self, model: "Model", lr: float):
+        self._check(self.lib.mg_model_sgd_step(self.handle, model.handle, C.c_float(lr)))
 
     def gat_model(self, layers, precision: int = GEMM_TF32, negative_slope: float = 0.2) -> "GatModel":
         return GatModel(self, layers, precision, negative_slope)

@@ -12,6 +12,8 @@
 #include <cstdlib>
 
 #include "mg_device.cuh"
+#include <mma.h>
+
 #include "mg_internal.cuh"
 
 int mg_gemm_tf32(mg_ctx* ctx, const float* x, const float* w_t, const float* bias, float* out, int64_t M, int N, int K,
@@ -367,7 +369,12 @@ extern "C" int mg_model_set_aggregator(mg_model* m, int aggregator) {
 extern "C" int mg_model_free(mg_model* m) {
     if (!m) return MG_OK;
     cudaSetDevice(m->device);
-    for (int l = 0; l < MG_MAX_HOPS; ++l) { cudaFree(m->w_cat[l]); cudaFree(m->w_cat_t[l]); cudaFree(m->w_pad_t[l]); cudaFree(m->bias[l]); }
+    for (int l = 0; l < MG_MAX_HOPS; ++l) {
+        cudaFree(m->w_cat[l]); cudaFree(m->w_cat_t[l]); cudaFree(m->w_pad_t[l]); cudaFree(m->bias[l]);
+        cudaFree(m->g_w_cat[l]); cudaFree(m->g_bias[l]);
+    }
+    cudaFree(m->zeros);
+    if (m->ctx && m->ctx->last_fwd_model == m) m->ctx->last_fwd_model = nullptr;
     delete m;
     return MG_OK;
 }
@@ -427,6 +434,7 @@ static int forward_impl(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out,
     MG_CUDA(ctx, cudaSetDevice(ctx->device));
     const int k = d->k, B = d->n_batches;
     cudaStream_t st = ctx->stream;
+    ctx->last_fwd_model = m; ctx->last_fwd_dense = d;
     // H^k of this pass goes to the buffer the pass before last used; an output copy of that pass to the host (side
     // stream) may still read it.  The copy of the previous pass reads the other buffer and is not waited for.
     float* hk = nullptr;
@@ -670,6 +678,347 @@ extern "C" int mg_layer_output(mg_ctx* ctx, const mg_model* m, mg_dense* d, int3
     }
     if (r.n_rows > 0) {
         k_export_rows<<<mg_grid(ctx, 4), kThreads, 0, ctx->stream>>>(r, src, out_dev);
+        ctx->launches++;
+    }
+    MG_CUDA(ctx, cudaGetLastError());
+    MG_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return MG_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// Backward pass through the GraphSage layers (Section 3: the gradients of a mini-batch update the model and the
+// base representations).  Chain rule through Algorithm 3 and Algorithm 2, layer k down to layer 1, over the same
+// row chunks as the unfused forward path:
+//   X = [self | aggregate] of the chunk is recomputed from H^{l-1} (kept by the forward pass),
+//   dPre = dH^l (masked by H^l > 0 below the last layer),
+//   dW += X^T dPre, dbias += column sums of dPre, dX = dPre W^T,
+//   dH^{l-1}[self row] += dX[:, :d_in];  dH^{l-1}[source row of entry e] += dX[:, d_in:] / count (or x 1 for a sum).
+// All arithmetic is fp32 on CUDA cores; sums over rows use atomic adds, so low-order bits vary from run to run.
+// ---------------------------------------------------------------------------------------
+namespace {
+
+struct RowGeom {
+    int32_t B, k;
+    const int32_t* rowbase;   // [(k + 1)][B + 1]
+    const int32_t* cum;       // [B][k + 2]
+    const int32_t* node_off;  // [(k + 1)][B + 1]
+};
+
+// packed row of layer `layer` -> its mini-batch, its local row, its place in the hop-major node list
+__device__ __forceinline__ void locate_row(const RowGeom& g, int layer, int64_t row, int32_t* b_out, int32_t* local_out, int32_t* node_out) {
+    const int32_t* rb = g.rowbase + (int64_t)layer * (g.B + 1);
+    int lo = 0, hi = g.B;   // rb[lo] <= row < rb[hi]
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if ((int64_t)rb[mid] <= row) lo = mid; else hi = mid;
+    }
+    const int32_t local = (int32_t)(row - rb[lo]);
+    const int32_t* cum = g.cum + (int64_t)lo * (g.k + 2);
+    int j = 0;
+    while (j + 1 <= g.k && cum[j + 1] <= local) ++j;
+    *b_out = lo; *local_out = local;
+    *node_out = g.node_off[(int64_t)j * (g.B + 1) + lo] + (local - cum[j]);
+}
+
+__global__ void __launch_bounds__(kThreads) k_relu_mask(float* g, const float* __restrict__ y, int64_t n) {
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        if (!(y[i] > 0.f)) g[i] = 0.f;
+}
+
+// dW[Kx, N] += X[rows, Kx]^T dPre[rows, N]; a block owns a 64 x 64 tile of dW and a slice of the rows
+constexpr int kGradRowsPerBlock = 1024;
+__global__ void __launch_bounds__(256) k_grad_weights(const float* __restrict__ x, const float* __restrict__ dpre, float* dw,
+                                                      int64_t rows, int Kx, int N) {
+    constexpr int T = 64, BR = 16;
+    __shared__ float xs[BR][T + 4];
+    __shared__ float gs[BR][T + 4];
+    const int k0 = blockIdx.x * T, n0 = blockIdx.y * T;
+    const int64_t r_lo = (int64_t)blockIdx.z * kGradRowsPerBlock, r_hi = min(rows, r_lo + kGradRowsPerBlock);
+    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
+    float acc[4][4] = {};
+    for (int64_t r0 = r_lo; r0 < r_hi; r0 += BR) {
+        for (int i = threadIdx.x; i < BR * T; i += 256) {
+            const int rr = i / T, c = i % T;
+            const bool on = r0 + rr < r_hi;
+            xs[rr][c] = (on && k0 + c < Kx) ? x[(r0 + rr) * Kx + k0 + c] : 0.f;
+            gs[rr][c] = (on && n0 + c < N) ? dpre[(r0 + rr) * N + n0 + c] : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int rr = 0; rr < BR; ++rr) {
+            float xv[4], gv[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { xv[i] = xs[rr][ty * 4 + i]; gv[i] = gs[rr][tx * 4 + i]; }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(xv[i], gv[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+    for (int i = 0; i < 4; ++i)
+        for (int j = 0; j < 4; ++j) {
+            const int kk = k0 + ty * 4 + i, n = n0 + tx * 4 + j;
+            if (kk < Kx && n < N) atomicAdd(&dw[(int64_t)kk * N + n], acc[i][j]);
+        }
+}
+
+// The same on the (legacy, warp-level) tensor-core path in TF32: X^T is read as a column-major operand straight
+// from the row-major chunk, so nothing is transposed.  A block owns a 64 x 64 tile of dW and a slice of the rows; each
+// of its four warps a 32 x 32 quarter (2 x 2 fragments of 16 x 16, K = 8 rows per step).
+__global__ void __launch_bounds__(128) k_grad_weights_tf32(const float* __restrict__ x, const float* __restrict__ dpre, float* dw,
+                                                           int64_t rows, int Kx, int N) {
+    using namespace nvcuda;
+    const int warp = threadIdx.x >> 5;
+    const int k0 = blockIdx.x * 64 + (warp >> 1) * 32, n0 = blockIdx.y * 64 + (warp & 1) * 32;
+    const int64_t r_lo = (int64_t)blockIdx.z * kGradRowsPerBlock, r_hi = min(rows, r_lo + kGradRowsPerBlock);
+    if (k0 >= Kx || n0 >= N) return;   // (widths are multiples of 32 on this path)
+    wmma::fragment<wmma::accumulator, 16, 16, 8, float> acc[2][2];
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+        for (int j = 0; j < 2; ++j) wmma::fill_fragment(acc[i][j], 0.f);
+    for (int64_t r = r_lo; r + 8 <= r_hi; r += 8) {
+        wmma::fragment<wmma::matrix_a, 16, 16, 8, wmma::precision::tf32, wmma::col_major> fa[2];
+        wmma::fragment<wmma::matrix_b, 16, 16, 8, wmma::precision::tf32, wmma::row_major> fb[2];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            wmma::load_matrix_sync(fa[i], x + r * Kx + k0 + 16 * i, Kx);       // element (k, row) at x[row * Kx + k]
+            wmma::load_matrix_sync(fb[i], dpre + r * N + n0 + 16 * i, N);
+#pragma unroll
+            for (int q = 0; q < fa[i].num_elements; ++q) fa[i].x[q] = wmma::__float_to_tf32(fa[i].x[q]);
+#pragma unroll
+            for (int q = 0; q < fb[i].num_elements; ++q) fb[i].x[q] = wmma::__float_to_tf32(fb[i].x[q]);
+        }
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) wmma::mma_sync(acc[i][j], fa[i], fb[j], acc[i][j]);
+    }
+    // the slice's last rows (fewer than 8) in plain fp32, one output per lane and step
+    const int64_t tail = r_lo + (r_hi - r_lo) / 8 * 8;
+    __shared__ float stage[4][32 * 32];
+    float* st = stage[warp];
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+        for (int j = 0; j < 2; ++j) wmma::store_matrix_sync(st + (16 * i) * 32 + 16 * j, acc[i][j], 32, wmma::mem_row_major);
+    __syncwarp();
+    const int lane = threadIdx.x & 31;
+    for (int o = lane; o < 32 * 32; o += 32) {
+        const int kk = o / 32, nn = o % 32;
+        float v = st[o];
+        for (int64_t r = tail; r < r_hi; ++r) v = fmaf(x[r * Kx + k0 + kk], dpre[r * N + n0 + nn], v);
+        atomicAdd(&dw[(int64_t)(k0 + kk) * N + n0 + nn], v);
+    }
+}
+
+__global__ void __launch_bounds__(kThreads) k_grad_bias(const float* __restrict__ dpre, float* db, int64_t rows, int N) {
+    // a block sums a slice of the rows for every column, then one atomic add per column
+    const int64_t r_lo = (int64_t)blockIdx.x * kGradRowsPerBlock, r_hi = min(rows, r_lo + kGradRowsPerBlock);
+    for (int c = threadIdx.x; c < N; c += kThreads) {
+        float s = 0.f;
+        for (int64_t r = r_lo; r < r_hi; ++r) s += dpre[r * N + c];
+        atomicAdd(&db[c], s);
+    }
+}
+
+struct ScatterArgs {
+    RowGeom g;
+    int32_t layer;             // the layer whose inputs receive the gradient (1 .. k)
+    int64_t row_lo, row_hi;    // packed output rows of this chunk
+    const int32_t* ent_off;
+    const int32_t* ent_repr;
+    const float* dx;           // [row_hi - row_lo, 2 d_in]
+    int32_t d_in, sum_aggr;
+    float* g_in;               // [rows of layer - 1, d_in]
+};
+
+// one warp per output row: its self row and the source rows of its entries receive their share of dX
+__global__ void __launch_bounds__(kThreads) k_scatter_grad(ScatterArgs a) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warps = (int64_t)gridDim.x * (kThreads / 32);
+    const int32_t* rb_in = a.g.rowbase + (int64_t)(a.layer - 1) * (a.g.B + 1);
+    for (int64_t row = a.row_lo + blockIdx.x * (int64_t)(kThreads / 32) + (threadIdx.x >> 5); row < a.row_hi; row += warps) {
+        int32_t b, local, node;
+        locate_row(a.g, a.layer, row, &b, &local, &node);
+        const int64_t in0 = rb_in[b];
+        const float* dxr = a.dx + (row - a.row_lo) * 2 * a.d_in;
+        float* self = a.g_in + (in0 + local) * a.d_in;
+        for (int c = lane; c < a.d_in; c += 32) atomicAdd(&self[c], dxr[c]);
+        const int32_t e0 = a.ent_off[node], e1 = a.ent_off[node + 1];
+        if (e1 <= e0) continue;
+        const float scale = a.sum_aggr ? 1.f : 1.f / (float)(e1 - e0);
+        for (int32_t e = e0; e < e1; ++e) {
+            float* src = a.g_in + (in0 + a.ent_repr[e]) * a.d_in;
+            for (int c = lane; c < a.d_in; c += 32) atomicAdd(&src[c], dxr[a.d_in + c] * scale);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads) k_sgd(float* w, const float* __restrict__ g, float lr, int64_t n) {
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) w[i] -= lr * g[i];
+}
+
+struct PackedIdArgs {
+    RowGeom g;
+    const int32_t* nodes;
+    int64_t n_rows;
+    int32_t* ids;
+};
+
+__global__ void __launch_bounds__(kThreads) k_packed_ids(PackedIdArgs a) {
+    for (int64_t row = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; row < a.n_rows; row += (int64_t)gridDim.x * blockDim.x) {
+        int32_t b, local, node;
+        locate_row(a.g, 0, row, &b, &local, &node);
+        a.ids[row] = a.nodes[node];
+    }
+}
+
+}  // namespace
+
+extern "C" int mg_backward(mg_ctx* ctx, mg_model* m, mg_dense* d, const float* d_out_dev, float* d_h0_dev) {
+    if (!ctx) return MG_ERR_ARG;
+    int rc = forward_checks(ctx, m, d);
+    if (rc) return rc;
+    if (!d_out_dev) return mg_fail(ctx, MG_ERR_ARG, "null output gradient");
+    if (!ctx->last_hk || ctx->last_fwd_model != m || ctx->last_fwd_dense != d)
+        return mg_fail(ctx, MG_ERR_STATE, "mg_backward follows mg_forward of the same model and sample");
+    if (!ctx->layers_kept) return mg_fail(ctx, MG_ERR_STATE, "the forward pass did not keep its intermediate layers: call mg_keep_layer_outputs(ctx, 1) first");
+    MG_CUDA(ctx, cudaSetDevice(ctx->device));
+    const int k = d->k, B = d->n_batches;
+    cudaStream_t st = ctx->stream;
+    // gradient buffers of the model (allocated once), cleared for this pass
+    int widest2 = 8;
+    for (int l = 1; l <= k; ++l) widest2 = std::max(widest2, 2 * m->dims[l - 1]);
+    for (int l = 0; l < k; ++l) {
+        const size_t n_w = (size_t)2 * m->dims[l] * m->dims[l + 1], n_b = (size_t)m->dims[l + 1];
+        if (!m->g_w_cat[l] && cudaMalloc((void**)&m->g_w_cat[l], n_w * sizeof(float)) != cudaSuccess) { cudaGetLastError(); return mg_fail(ctx, MG_ERR_OOM, "gradient allocation failed"); }
+        if (!m->g_bias[l] && cudaMalloc((void**)&m->g_bias[l], n_b * sizeof(float)) != cudaSuccess) { cudaGetLastError(); return mg_fail(ctx, MG_ERR_OOM, "gradient allocation failed"); }
+        MG_CUDA(ctx, cudaMemsetAsync(m->g_w_cat[l], 0, n_w * sizeof(float), st));
+        MG_CUDA(ctx, cudaMemsetAsync(m->g_bias[l], 0, n_b * sizeof(float), st));
+    }
+    if (!m->zeros) {
+        if (cudaMalloc((void**)&m->zeros, sizeof(float) * 2 * 1024) != cudaSuccess) { cudaGetLastError(); return mg_fail(ctx, MG_ERR_OOM, "gradient allocation failed"); }
+        MG_CUDA(ctx, cudaMemsetAsync(m->zeros, 0, sizeof(float) * 2 * 1024, st));
+    }
+    // scratch: dH^1 .. dH^{k-1}, the X and dX rows of a chunk
+    size_t g_off[MG_MAX_HOPS + 1] = {0}, g_total = 0, h_off[MG_MAX_HOPS + 1] = {0}, h_total = 0;
+    for (int l = 1; l < k; ++l) {
+        g_off[l] = g_total; g_total += ((size_t)d->h_hdr.rows_total[l] * m->dims[l] + 7) / 8 * 8;   // (32-byte aligned starts)
+        h_off[l] = h_total; h_total += (size_t)d->h_hdr.rows_total[l] * m->dims[l];
+    }
+    int64_t max_x = 0;
+    for (int l = 1; l <= k; ++l)
+        max_x = std::max<int64_t>(max_x, std::min<int64_t>(chunk_rows_for(m->dims[l - 1]), d->h_hdr.rows_total[l]) * 2 * m->dims[l - 1]);
+    if (ctx->bw_g_elems < g_total && (rc = mg_ensure(ctx, &ctx->bw_g, &ctx->bw_g_elems, g_total + g_total / 4 + 16))) return rc;
+    if (ctx->bw_x_elems < (size_t)max_x && (rc = mg_ensure(ctx, &ctx->bw_x, &ctx->bw_x_elems, (size_t)max_x + 16))) return rc;
+    if (ctx->bw_dx_elems < (size_t)max_x && (rc = mg_ensure(ctx, &ctx->bw_dx, &ctx->bw_dx_elems, (size_t)max_x + 16))) return rc;
+    if (g_total) MG_CUDA(ctx, cudaMemsetAsync(ctx->bw_g, 0, g_total * sizeof(float), st));
+    if (d_h0_dev) MG_CUDA(ctx, cudaMemsetAsync(d_h0_dev, 0, (size_t)d->h_hdr.rows_total[0] * m->dims[0] * sizeof(float), st));
+    const RowGeom geom{B, k, d->rowbase, d->cum, d->node_off};
+    const bool half = ctx->feat_dtype == MG_DTYPE_F16;
+    const int grid = mg_grid(ctx, 8);
+    for (int l = k; l >= 1; --l) {
+        const int d_in = m->dims[l - 1], d_out = m->dims[l];
+        const int64_t M = d->h_hdr.rows_total[l];
+        if (M == 0) continue;
+        const float* dpre_all = l == k ? d_out_dev : ctx->bw_g + g_off[l];
+        if (l < k) {   // through the ReLU
+            k_relu_mask<<<grid, kThreads, 0, st>>>(ctx->bw_g + g_off[l], ctx->ws_h[0] + h_off[l], M * d_out);
+            ctx->launches++;
+        }
+        const float* h_prev = l > 1 ? ctx->ws_h[0] + h_off[l - 1] : nullptr;
+        float* g_in = l > 1 ? ctx->bw_g + g_off[l - 1] : d_h0_dev;
+        const int64_t chunk = chunk_rows_for(d_in);
+        for (int64_t r0 = 0; r0 < M; r0 += chunk) {
+            const int64_t r1 = std::min(M, r0 + chunk), rows = r1 - r0;
+            AggArgs a;
+            a.B = B; a.k = k; a.layer = l; a.d_in = d_in;
+            a.row_lo = (int32_t)r0; a.row_hi = (int32_t)r1;
+            a.rowbase_out = d->rowbase + (size_t)l * (B + 1);
+            a.rowbase_in = d->rowbase + (size_t)(l - 1) * (B + 1);
+            a.cum = d->cum; a.node_off = d->node_off; a.nodes = d->nodes;
+            a.ent_off = d->ent_off; a.ent_nbrs = d->ent_nbrs; a.ent_repr = d->ent_repr;
+            a.h_prev = h_prev;
+            a.slots = ctx->slots; a.slot_of_part = ctx->d_slot_of_part;
+            a.slot_bytes = ctx->slot_bytes; a.row_bytes = ctx->row_bytes; a.part_size = (uint32_t)ctx->part_size;
+            a.x = ctx->bw_x;
+            a.round_tf32 = 0;
+            a.sum_aggr = m->sum_aggr ? 1 : 0;
+            if (l == 1) { if (half) launch_aggregate<true, true>(a, grid, st); else launch_aggregate<true, false>(a, grid, st); }
+            else launch_aggregate<false, false>(a, grid, st);
+            const float* dpre = dpre_all + r0 * d_out;
+            const unsigned slices = (unsigned)((rows + kGradRowsPerBlock - 1) / kGradRowsPerBlock);
+            dim3 gw((unsigned)((2 * d_in + 63) / 64), (unsigned)((d_out + 63) / 64), slices);
+            if (m->precision == MG_GEMM_TF32 && d_in % 16 == 0 && d_out % 32 == 0)
+                k_grad_weights_tf32<<<gw, 128, 0, st>>>(ctx->bw_x, dpre, m->g_w_cat[l - 1], rows, 2 * d_in, d_out);
+            else
+                k_grad_weights<<<gw, 256, 0, st>>>(ctx->bw_x, dpre, m->g_w_cat[l - 1], rows, 2 * d_in, d_out);
+            k_grad_bias<<<slices, kThreads, 0, st>>>(dpre, m->g_bias[l - 1], rows, d_out);
+            ctx->launches += 3;
+            if (!g_in) continue;   // layer 1 without a gradient of the base representations
+            if (m->precision == MG_GEMM_TF32) {
+                // dX = dPre W^T on the tensor cores: the K-major operand the kernel wants is W itself ([2 d_in, d_out])
+                if ((rc = mg_gemm_tf32(ctx, dpre, m->w_cat[l - 1], m->zeros, ctx->bw_dx, rows, 2 * d_in, d_out, false))) return rc;
+                ctx->launches--;
+            } else {
+                dim3 gx((unsigned)((rows + 63) / 64), (unsigned)((2 * d_in + 63) / 64));
+                k_gemm_fp32<false><<<gx, 256, 0, st>>>(dpre, m->w_cat_t[l - 1], m->zeros, ctx->bw_dx, rows, 2 * d_in, d_out);
+            }
+            ScatterArgs s;
+            s.g = geom; s.layer = l; s.row_lo = r0; s.row_hi = r1; s.ent_off = d->ent_off; s.ent_repr = d->ent_repr;
+            s.dx = ctx->bw_dx; s.d_in = d_in; s.sum_aggr = m->sum_aggr ? 1 : 0; s.g_in = g_in;
+            k_scatter_grad<<<grid, kThreads, 0, st>>>(s);
+            ctx->launches += 2;
+        }
+    }
+    MG_CUDA(ctx, cudaGetLastError());
+    MG_CUDA(ctx, cudaStreamSynchronize(st));
+    return m->precision == MG_GEMM_TF32 ? mg_gemm_tf32_status(ctx) : MG_OK;
+}
+
+extern "C" int mg_model_grads(const mg_model* m, int32_t layer, const float** d_w_self, const float** d_w_nbr, const float** d_bias) {
+    if (!m) return MG_ERR_ARG;
+    if (layer < 1 || layer > m->k) return mg_fail(m->ctx, MG_ERR_ARG, "layer must be in [1, k]");
+    if (!m->g_w_cat[layer - 1]) return mg_fail(m->ctx, MG_ERR_STATE, "mg_backward has not run");
+    const size_t half_elems = (size_t)m->dims[layer - 1] * m->dims[layer];
+    if (d_w_self) *d_w_self = m->g_w_cat[layer - 1];
+    if (d_w_nbr) *d_w_nbr = m->g_w_cat[layer - 1] + half_elems;
+    if (d_bias) *d_bias = m->g_bias[layer - 1];
+    return MG_OK;
+}
+
+extern "C" int mg_model_sgd_step(mg_ctx* ctx, mg_model* m, float lr) {
+    if (!ctx) return MG_ERR_ARG;
+    if (!m || m->ctx != ctx) return mg_fail(ctx, MG_ERR_ARG, "bad model handle");
+    if (!m->g_w_cat[0]) return mg_fail(ctx, MG_ERR_STATE, "mg_backward has not run");
+    MG_CUDA(ctx, cudaSetDevice(ctx->device));
+    cudaStream_t st = ctx->stream;
+    for (int l = 0; l < m->k; ++l) {
+        const size_t di = m->dims[l], dn = m->dims[l + 1];
+        k_sgd<<<mg_grid(ctx, 2), kThreads, 0, st>>>(m->w_cat[l], m->g_w_cat[l], lr, (int64_t)(2 * di * dn));
+        k_sgd<<<1, kThreads, 0, st>>>(m->bias[l], m->g_bias[l], lr, (int64_t)dn);
+        // the copies the forward kernels read
+        k_transpose<<<mg_grid(ctx, 2), kThreads, 0, st>>>(m->w_cat[l], m->w_cat_t[l], (int)(2 * di), (int)dn, m->precision == MG_GEMM_TF32);
+        ctx->launches += 3;
+        const int rc = mg_pack_layer_weights(ctx, m->w_cat[l], m->w_pad_t[l], (int)di, (int)dn);
+        if (rc) return rc;
+    }
+    MG_CUDA(ctx, cudaGetLastError());
+    MG_CUDA(ctx, cudaStreamSynchronize(st));
+    return MG_OK;
+}
+
+extern "C" int mg_dense_packed_ids(mg_ctx* ctx, mg_dense* d, int32_t* ids_dev) {
+    if (!ctx) return MG_ERR_ARG;
+    if (!d || !ids_dev) return mg_fail(ctx, MG_ERR_ARG, "null argument");
+    if (d->pending) return mg_fail(ctx, MG_ERR_STATE, "a sample is in flight on this mg_dense: call mg_sample_many_end first");
+    if (!d->valid) return mg_fail(ctx, MG_ERR_STATE, "mg_dense holds no completed sample");
+    MG_CUDA(ctx, cudaSetDevice(ctx->device));
+    PackedIdArgs a{{d->n_batches, d->k, d->rowbase, d->cum, d->node_off}, d->nodes, d->h_hdr.rows_total[0], ids_dev};
+    if (a.n_rows > 0) {
+        k_packed_ids<<<mg_grid(ctx, 4), kThreads, 0, ctx->stream>>>(a);
         ctx->launches++;
     }
     MG_CUDA(ctx, cudaGetLastError());

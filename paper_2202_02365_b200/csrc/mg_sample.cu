@@ -1695,6 +1695,7 @@ extern "C" int mg_dense_view(mg_ctx* ctx, mg_dense* d, int32_t batch, mg_dense_a
 extern "C" int mg_dense_free(mg_dense* d) {
     if (!d) return MG_OK;
     cudaSetDevice(d->device);
+    if (d->ctx && d->ctx->last_fwd_dense == d) d->ctx->last_fwd_dense = nullptr;
     cudaFree(d->hdr); cudaFree(d->nodes); cudaFree(d->node_batch); cudaFree(d->ent_off); cudaFree(d->node_r0); cudaFree(d->node_deg); cudaFree(d->node_r0_out); cudaFree(d->node_deg_out); cudaFree(d->pairs); cudaFree(d->share_off);
     cudaFree(d->ent_nbrs); cudaFree(d->ent_repr); cudaFree(d->node_off); cudaFree(d->cum);
     cudaFree(d->rowbase); cudaFree(d->hkeys); cudaFree(d->hvals); cudaFree(d->newlist[0]);

@@ -914,3 +914,74 @@ def test_graph_attention_errors_and_fp16_features():
     with pytest.raises(mg.MgError) as e:
         ctx.gat_forward(ctx.gat_model(_gat_layers([24, 8, 8], seed=1)), d, out)     # two layers, one hop
     assert e.value.code == -2
+
+
+@pytest.mark.parametrize("aggregator,prec,dims", [("mean", "fp32", [16, 24, 8]), ("sum", "fp32", [16, 24, 8]), ("mean", "tf32", [16, 24, 8]),
+                                                  ("mean", "tf32", [16, 64, 32])])
+def test_backward_pass_and_sgd_step(tiny, aggregator, prec, dims):
+    """Gradients of a scalar loss through the GraphSage layers against the oracle's chain rule (itself pinned by
+    finite differences): weights, biases and the base representations' rows; then one SGD step."""
+    g, feats = tiny
+    ctx = make_ctx(g, feats)
+    ctx.keep_layer_outputs(True)
+    sizes = [150, 0, 1, 260]
+    tg = [inputs.distinct_targets(10_000, s, seed=90 + i) for i, s in enumerate(sizes)]
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    seeds = [3, 4, 5, 6]
+    fanouts = [5, 3]
+    layers = inputs.random_bias_layers(dims, seed=12)
+    np_layers = [(w.numpy(), n.numpy(), b.numpy()) for w, n, b in layers]
+    precision = mg.GEMM_FP32 if prec == "fp32" else mg.GEMM_TF32
+    rtol = 2e-4                                      # fp32 sums over thousands of rows, atomics in any order
+    if prec == "tf32":
+        # the forward pass ran on the tensor cores: a pre-activation within TF32 rounding of zero may sit on the other
+        # side of the ReLU than in the fp64 oracle, which changes single gradient entries by O(1); compare in norm
+        def close(got, ref, _rtol):                  # noqa: F811
+            got, ref = np.asarray(got, dtype=np.float64), np.asarray(ref, dtype=np.float64)
+            assert got.shape == ref.shape
+            assert np.linalg.norm(got - ref) <= 2e-2 * max(np.linalg.norm(ref), 1e-30)
+    else:
+        close = globals()["close"]
+    model = ctx.model(layers, precision)
+    model.set_aggregator(aggregator)
+    d = ctx.sample_many(torch.cat(tg), offs, fanouts, seeds)
+    out = torch.empty((int(offs[-1]), dims[-1]), dtype=torch.float32, device="cuda")
+    ctx.forward(model, d, out)
+    gen = torch.Generator().manual_seed(5)
+    g_out = torch.randn((int(offs[-1]), dims[-1]), generator=gen)
+    grads, g_h0, ids = ctx.backward(model, d, g_out.cuda(), want_h0_grad=True)
+    view = oracle_view(g)
+    want = [[np.zeros_like(x, dtype=np.float64) for x in l] for l in np_layers]
+    nodes, _ = d.counts()
+    row0 = np.concatenate([[0], np.cumsum(nodes.sum(1).cpu().numpy())])
+    ids_h, g_h0_h = ids.cpu().numpy(), g_h0.cpu().numpy()
+    for b in range(len(sizes)):
+        if not sizes[b]:
+            continue
+        ref = O.sample_dense(view, tg[b].tolist(), fanouts, seeds[b])
+        gr, d_h0 = O.backward(ref, feats.numpy()[ref["node_ids"]], np_layers, g_out[offs[b]:offs[b + 1]].numpy(), aggregator)
+        for l in range(len(np_layers)):
+            for p in range(3):
+                want[l][p] += gr[l][p]
+        # base-representation gradients: the library's packed rows carry their node ids
+        lo, hi = int(row0[b]), int(row0[b + 1])
+        assert sorted(ids_h[lo:hi].tolist()) == sorted(ref["node_ids"])
+        where = {v: r for r, v in enumerate(ref["node_ids"])}
+        close(g_h0_h[lo:hi], d_h0[[where[int(v)] for v in ids_h[lo:hi]]], rtol)
+    for l in range(len(np_layers)):
+        for p in range(3):
+            close(grads[l][p].cpu().numpy(), want[l][p], rtol)
+    # one SGD step: the next forward pass uses w - lr dw
+    lr = 0.05
+    ctx.sgd_step(model, lr)
+    stepped = [tuple(torch.from_numpy(x - lr * gw).float() for x, gw in zip(np_layers[l], want[l])) for l in range(len(np_layers))]
+    ctx.forward(model, d, out)
+    ref3 = O.sample_dense(view, tg[3].tolist(), fanouts, seeds[3])
+    want_out = O.forward(ref3, feats.numpy()[ref3["node_ids"]], [tuple(t.numpy() for t in l) for l in stepped], aggregator=aggregator)
+    close(out[offs[3]:offs[4]].cpu().numpy(), want_out, 1e-3)
+    # state errors
+    ctx.keep_layer_outputs(False)
+    other = ctx.model(layers, precision)
+    with pytest.raises(mg.MgError) as e:
+        ctx.backward(other, d, g_out.cuda())
+    assert e.value.code == -2
