@@ -270,9 +270,11 @@ def test_link_prediction_distmult():
     close(nd.cpu().numpy(), rnd, RTOL_TC)
 
 
-@pytest.mark.parametrize("dim,n_edges,n_chunks,negs", [(100, 700, 3, 1000), (32, 129, 1, 17), (128, 300, 7, 256)])
+@pytest.mark.parametrize("dim,n_edges,n_chunks,negs", [(100, 700, 3, 1000), (32, 129, 1, 17), (128, 300, 7, 256),
+                                                       (32, 60_000, 5, 72)])
 def test_distmult_tensor_core_shapes(dim, n_edges, n_chunks, negs):
-    """DistMult negatives on the tensor cores: padded K, several blocks of negatives, ragged chunks."""
+    """DistMult negatives on the tensor cores: padded K, several blocks of negatives, ragged chunks; the last case
+    has more than three tiles per SM."""
     n = 30_000
     g = inputs.rmat_graph(n, 300_000, seed=6, n_relations=11)
     ctx = mg.Context(0)
