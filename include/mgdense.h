@@ -173,7 +173,10 @@ int mg_commit_resident(mg_ctx* ctx, int32_t timeout_ms);
  * The call is synchronous: on return the sample is complete and its status checked.  The kernels run
  * on a library-owned sampling stream, ordered after the work queued on the context's stream so far.
  * Errors: MG_ERR_ARG, MG_ERR_STATE, MG_ERR_NONRESIDENT, MG_ERR_DUPLICATE, MG_ERR_CAPACITY,
- * MG_ERR_OOM. */
+ * MG_ERR_OOM.
+ * Two environment variables switch off a fast path, for diagnosis (the results are the same): MG_NO_SAMPLE_GRAPH
+ * (launch the sampler's kernels one by one instead of replaying the captured CUDA graph) and MG_GLOBAL_TABLES
+ * (deduplicate the last hop through the id tables in global memory instead of shared memory). */
 int mg_sample_many(mg_ctx* ctx, const int32_t* targets, int targets_on_device,
                    const int64_t* target_offsets, int32_t n_batches, const int32_t* fanouts,
                    int32_t k, const uint64_t* seeds, const mg_sample_caps* caps /*nullable*/,
