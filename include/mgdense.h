@@ -360,6 +360,14 @@ int mg_model_grads(const mg_model* m, int32_t layer, const float** d_w_self, con
  * mg_backward: w -= lr * dw.  Refreshes the copies the forward kernels read.  Synchronous. */
 int mg_model_sgd_step(mg_ctx* ctx, mg_model* m, float lr);
 
+/* One SGD step on the base representations of the sample's nodes, in the partition buffer: row(node) -= lr * its
+ * gradient row(s) of d_h0_dev (as written by mg_backward; a node of several mini-batches receives all of its rows).
+ * fp32 tables only.  With host backing the table handed to mg_load_features must be writable: a partition updated
+ * here is copied back to it when mg_set_resident evicts it (side stream, before its slot is reused); partitions
+ * still resident hold the only current copy.  With HBM backing the caller's device table is updated in place.
+ * Synchronous.  Errors: MG_ERR_ARG, MG_ERR_STATE. */
+int mg_apply_embedding_sgd(mg_ctx* ctx, mg_dense* d, const float* d_h0_dev, float lr);
+
 /* ids_dev (DEVICE, int32, one per node of every mini-batch = the rows of H^0 in the library's packed order: batch
  * after batch, targets first, then delta after delta in the order the nodes were found): the node id of each row. */
 int mg_dense_packed_ids(mg_ctx* ctx, mg_dense* d, int32_t* ids_dev);

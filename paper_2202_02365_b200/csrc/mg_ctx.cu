@@ -496,6 +496,7 @@ extern "C" int mg_set_partitioning(mg_ctx* c, int32_t n_parts) {
     c->part_size = (c->n_nodes + n_parts - 1) / n_parts;
     c->capacity = n_parts;
     c->slot_of_part.assign(n_parts, n_parts == 1 ? 0 : -1);
+    c->dirty_part.clear();
     c->pending_slot.clear();
     c->has_pending = false;
     int rc = upload_slot_map(c);
@@ -550,6 +551,7 @@ extern "C" int mg_load_features(mg_ctx* c, const void* table, int table_is_devic
         for (int p = 0; p < c->n_parts; ++p)
             if (c->slot_of_part[p] >= 0) keep.push_back(p);
         c->slot_of_part.assign(c->n_parts, -1);
+        c->dirty_part.clear();
         c->feat_dim = dim;
         if ((int)keep.size() > c->capacity) keep.resize(c->capacity);
         if (!keep.empty()) {
@@ -607,6 +609,24 @@ extern "C" int mg_set_resident(mg_ctx* c, const int32_t* part_ids, int32_t n, in
             (evicted_slot[s] ? free_later : free_now).push_back(s);
         }
         cudaEvent_t main_done = nullptr;
+        // evicted partitions whose rows were updated in the buffer go back to the host table first (side stream, after
+        // the work queued on the main stream; the copies into reused slots below are queued behind them)
+        for (int p = 0; p < c->n_parts; ++p) {
+            const int s = c->slot_of_part[p];
+            if (s < 0 || want[p] || p >= (int)c->dirty_part.size() || !c->dirty_part[p]) continue;
+            if (!main_done) {
+                MG_CUDA(c, cudaEventCreateWithFlags(&main_done, cudaEventDisableTiming));
+                MG_CUDA(c, cudaEventRecord(main_done, c->stream));
+                MG_CUDA(c, cudaStreamWaitEvent(c->side, main_done, 0));
+            }
+            const int64_t first = (int64_t)p * c->part_size;
+            const int64_t rows = std::min<int64_t>(c->part_size, c->n_nodes - first);
+            if (rows > 0)
+                MG_CUDA(c, cudaMemcpyAsync(const_cast<char*>(c->host_table) + (size_t)first * c->row_bytes,
+                                           c->slots + (size_t)s * c->slot_bytes, (size_t)rows * c->row_bytes,
+                                           cudaMemcpyDeviceToHost, c->side));
+            c->dirty_part[p] = 0;
+        }
         for (int p = 0; p < c->n_parts; ++p) {
             if (!want[p] || next[p] >= 0) continue;
             int s;

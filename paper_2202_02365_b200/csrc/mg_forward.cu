@@ -1010,6 +1010,64 @@ extern "C" int mg_model_sgd_step(mg_ctx* ctx, mg_model* m, float lr) {
     return MG_OK;
 }
 
+namespace {
+
+struct EmbSgdArgs {
+    RowGeom g;
+    const int32_t* nodes;
+    const float* grad;          // [n_rows, dim] packed like H^0
+    int64_t n_rows;
+    char* slots;
+    const int32_t* slot_of_part;
+    int64_t slot_bytes, row_bytes;
+    uint32_t part_size;
+    int32_t dim;
+    float lr;
+};
+
+// base representation of node(row) -= lr * grad[row]; a node of several mini-batches receives several updates
+__global__ void __launch_bounds__(kThreads) k_embedding_sgd(EmbSgdArgs a) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warps = (int64_t)gridDim.x * (kThreads / 32);
+    for (int64_t row = blockIdx.x * (int64_t)(kThreads / 32) + (threadIdx.x >> 5); row < a.n_rows; row += warps) {
+        int32_t b, local, node;
+        locate_row(a.g, 0, row, &b, &local, &node);
+        const uint32_t id = (uint32_t)a.nodes[node];
+        const uint32_t p = id / a.part_size;
+        float* dst = reinterpret_cast<float*>(a.slots + (int64_t)a.slot_of_part[p] * a.slot_bytes + (int64_t)(id - p * a.part_size) * a.row_bytes);
+        const float* g = a.grad + row * a.dim;
+        for (int c = lane; c < a.dim; c += 32) {
+            const float v = g[c];
+            if (v != 0.f) atomicAdd(&dst[c], -a.lr * v);
+        }
+    }
+}
+
+}  // namespace
+
+extern "C" int mg_apply_embedding_sgd(mg_ctx* ctx, mg_dense* d, const float* d_h0_dev, float lr) {
+    if (!ctx) return MG_ERR_ARG;
+    if (!d || !d_h0_dev) return mg_fail(ctx, MG_ERR_ARG, "null argument");
+    if (d->pending) return mg_fail(ctx, MG_ERR_STATE, "a sample is in flight on this mg_dense: call mg_sample_many_end first");
+    if (!d->valid) return mg_fail(ctx, MG_ERR_STATE, "mg_dense holds no completed sample");
+    if (d->ctx != ctx) return mg_fail(ctx, MG_ERR_ARG, "handle belongs to another context");
+    if (!ctx->slots || ctx->feat_dim <= 0) return mg_fail(ctx, MG_ERR_STATE, "no feature table loaded");
+    if (ctx->feat_dtype != MG_DTYPE_F32) return mg_fail(ctx, MG_ERR_ARG, "base representations are updated in fp32 tables only");
+    MG_CUDA(ctx, cudaSetDevice(ctx->device));
+    EmbSgdArgs a{{d->n_batches, d->k, d->rowbase, d->cum, d->node_off}, d->nodes, d_h0_dev, d->h_hdr.rows_total[0], ctx->slots,
+                 ctx->d_slot_of_part, ctx->slot_bytes, ctx->row_bytes, (uint32_t)ctx->part_size, ctx->feat_dim, lr};
+    if (a.n_rows > 0) {
+        k_embedding_sgd<<<mg_grid(ctx, 8), kThreads, 0, ctx->stream>>>(a);
+        ctx->launches++;
+    }
+    // with host backing the updated slots go back to the host table when their partitions are evicted
+    ctx->dirty_part.assign(ctx->n_parts, 0);
+    for (int p = 0; p < ctx->n_parts; ++p) ctx->dirty_part[p] = ctx->slot_of_part[p] >= 0 ? 1 : 0;
+    MG_CUDA(ctx, cudaGetLastError());
+    MG_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return MG_OK;
+}
+
 extern "C" int mg_dense_packed_ids(mg_ctx* ctx, mg_dense* d, int32_t* ids_dev) {
     if (!ctx) return MG_ERR_ARG;
     if (!d || !ids_dev) return mg_fail(ctx, MG_ERR_ARG, "null argument");

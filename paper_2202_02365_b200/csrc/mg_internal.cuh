@@ -94,6 +94,7 @@ struct mg_ctx {
     std::vector<int32_t> pending_slot;  // after set_resident, before commit
     bool has_pending = false;
     std::vector<cudaEvent_t> pending_events;
+    std::vector<char> dirty_part;       // host backing: the partition's slot was updated (mg_apply_embedding_sgd) and not written back yet
     int32_t* d_slot_of_part = nullptr;   // [MG_MAX_PARTS]
     int64_t* d_res_prefix = nullptr;     // [MG_MAX_PARTS + 1] resident-node prefix counts
     int64_t n_resident_nodes = 0;

@@ -987,3 +987,60 @@ def test_backward_pass_and_sgd_step(tiny, aggregator, prec, dims):
     with pytest.raises(mg.MgError) as e:
         ctx.backward(other, d, g_out.cuda())
     assert e.value.code == -2
+
+
+def test_embedding_update_and_write_back_of_evicted_partitions():
+    """A training step on the base representations out of core: gradients of H^0 from mg_backward, an SGD step on the
+    rows in the partition buffer, and the updated partitions written back to the host table when they are evicted."""
+    n, parts, cap = 6000, 6, 3
+    g = inputs.rmat_graph(n, 60_000, seed=9)
+    table = inputs.normal_features(n, 8, seed=3, pin=False).pin_memory()
+    before = table.clone()
+    ctx = mg.Context(0)
+    ctx.load_graph(g.row_offsets.cuda(), g.nbrs.cuda())
+    ctx.set_partitioning(parts)
+    ctx.load_features(table, capacity_parts=cap, backing=mg.BACKING_HOST)
+    ctx.keep_layer_outputs(True)
+    resident = [0, 2, 5]
+    ctx.set_resident(resident, async_=True)
+    ctx.commit_resident(10_000)
+    layers = inputs.random_bias_layers([8, 8, 4], seed=1)
+    np_layers = [(w.numpy(), nn.numpy(), b.numpy()) for w, nn, b in layers]
+    model = ctx.model(layers, mg.GEMM_FP32)
+    pool = torch.nonzero(inputs.resident_node_mask(n, parts, resident)).flatten()
+    sizes = [60, 80]
+    tg = [inputs.distinct_targets(pool, s, seed=7 + i) for i, s in enumerate(sizes)]
+    offs = [0, 60, 140]
+    seeds = [1, 2]
+    d = ctx.sample_many(torch.cat(tg), offs, [4, 3], seeds)
+    out = torch.empty((140, 4), dtype=torch.float32, device="cuda")
+    ctx.forward(model, d, out)
+    g_out = torch.randn((140, 4), generator=torch.Generator().manual_seed(3))
+    _, g_h0, ids = ctx.backward(model, d, g_out.cuda(), want_h0_grad=True)
+    lr = 0.1
+    ctx.apply_embedding_sgd(d, g_h0, lr)
+    # what the table must look like now: the oracle's gradient rows, summed per node over the two mini-batches
+    view = oracle_view(g, parts, resident)
+    want = before.numpy().astype(np.float64).copy()
+    for b in range(2):
+        ref = O.sample_dense(view, tg[b].tolist(), [4, 3], seeds[b])
+        _, d_h0 = O.backward(ref, before.numpy()[ref["node_ids"]], np_layers, g_out[offs[b]:offs[b + 1]].numpy())
+        np.subtract.at(want, np.asarray(ref["node_ids"]), lr * d_h0)
+    # the buffer holds the update (read back through a fresh sample's H^0 rows); the host table does not yet
+    probe = inputs.distinct_targets(pool, 300, seed=99)
+    dp = ctx.sample(probe, [2], seed=5)
+    refp = O.sample_dense(view, probe.tolist(), [2], 5)
+    close(ctx.gather_h0(dp, 0, len(refp["node_ids"]), 8).cpu().numpy(), want[refp["node_ids"]], 2e-5)
+    assert torch.equal(table, before)
+    # evict everything that was updated: the rows go back to the host table before their slots are reused
+    ctx.set_resident([1, 3, 4], async_=True)
+    ctx.commit_resident(10_000)
+    torch.cuda.synchronize()
+    close(table.numpy(), want, 2e-5)
+    changed = np.nonzero(np.abs(want - before.numpy()).sum(1))[0]
+    assert len(changed) > 100 and all(int(v) // ((n + parts - 1) // parts) in resident for v in changed)
+    # and come back from there when the partitions are loaded again
+    ctx.set_resident(resident, async_=True)
+    ctx.commit_resident(10_000)
+    dp = ctx.sample(probe, [2], seed=5)
+    close(ctx.gather_h0(dp, 0, len(refp["node_ids"]), 8).cpu().numpy(), want[refp["node_ids"]], 2e-5)
