@@ -360,6 +360,11 @@ int mg_model_grads(const mg_model* m, int32_t layer, const float** d_w_self, con
  * mg_backward: w -= lr * dw.  Refreshes the copies the forward kernels read.  Synchronous. */
 int mg_model_sgd_step(mg_ctx* ctx, mg_model* m, float lr);
 
+/* One Adagrad step with the gradients of the last mg_backward: state += g^2 (state starts at zero with the first
+ * call), w -= lr * g / (sqrt(state) + eps), for every weight and bias.  Synchronous.  Errors: MG_ERR_ARG, MG_ERR_STATE,
+ * MG_ERR_OOM. */
+int mg_model_adagrad_step(mg_ctx* ctx, mg_model* m, float lr, float eps);
+
 /* One SGD step on the base representations of the sample's nodes, in the partition buffer: row(node) -= lr * its
  * gradient row(s) of d_h0_dev (as written by mg_backward; a node of several mini-batches receives all of its rows).
  * fp32 tables only.  With host backing the table handed to mg_load_features must be writable: a partition updated

@@ -397,6 +397,14 @@ def backward(dense, h0, layers, d_out, aggregator: str = "mean"):
     return grads, d_h
 
 
+def adagrad_step(w, g, state, lr: float, eps: float):
+    """Adagrad (Duchi et al.), the optimiser the paper's system trains with besides SGD: the state accumulates squared
+    gradients, the step of every coordinate is scaled by the root of its state.  Returns (w', state')."""
+    g = np.asarray(g, dtype=np.float64)
+    state = np.asarray(state, dtype=np.float64) + g * g
+    return np.asarray(w, dtype=np.float64) - lr * g / (np.sqrt(state) + eps), state
+
+
 # ----------------------------------------------------------------------------
 # Link prediction: shared uniform negatives, target union, DistMult
 # ----------------------------------------------------------------------------

@@ -31,7 +31,7 @@ EXPORTS = [
     "mg_load_features", "mg_set_resident", "mg_commit_resident", "mg_sample_many", "mg_sample_many_begin", "mg_sample_many_end", "mg_sample",
     "mg_dense_counts", "mg_dense_view", "mg_dense_free", "mg_model_create", "mg_model_set_aggregator", "mg_model_free",
     "mg_forward", "mg_set_layer_window", "mg_keep_layer_outputs", "mg_forward_host_async", "mg_wait_output", "mg_forward_noalloc", "mg_gather_h0", "mg_layer_output", "mg_lp_prepare", "mg_lp_view", "mg_lp_free",
-    "mg_distmult_score", "mg_kernel_launches", "mg_profile", "mg_profile_read", "mg_comet_plan", "mg_comet_bias", "mg_comet_autotune", "mg_gat_model_create", "mg_gat_model_free", "mg_gat_forward", "mg_backward", "mg_model_grads", "mg_model_sgd_step", "mg_dense_packed_ids", "mg_apply_embedding_sgd",
+    "mg_distmult_score", "mg_kernel_launches", "mg_profile", "mg_profile_read", "mg_comet_plan", "mg_comet_bias", "mg_comet_autotune", "mg_gat_model_create", "mg_gat_model_free", "mg_gat_forward", "mg_backward", "mg_model_grads", "mg_model_sgd_step", "mg_model_adagrad_step", "mg_dense_packed_ids", "mg_apply_embedding_sgd",
 ]
 
 
@@ -406,6 +406,9 @@ class Context:
     def apply_embedding_sgd(self, dense: "Dense", g_h0: torch.Tensor, lr: float):
         assert g_h0.is_cuda and g_h0.dtype == torch.float32 and g_h0.is_contiguous()
         self._check(self.lib.mg_apply_embedding_sgd(self.handle, dense.handle, _ptr(g_h0), C.c_float(lr)))
+
+    def adagrad_step(self, model: "Model", lr: float, eps: float = 1e-10):
+        self._check(self.lib.mg_model_adagrad_step(self.handle, model.handle, C.c_float(lr), C.c_float(eps)))
 
     def sgd_step(self, model: "Model", lr: float):
         self._check(self.lib.mg_model_sgd_step(self.handle, model.handle, C.c_float(lr)))

@@ -371,7 +371,7 @@ extern "C" int mg_model_free(mg_model* m) {
     cudaSetDevice(m->device);
     for (int l = 0; l < MG_MAX_HOPS; ++l) {
         cudaFree(m->w_cat[l]); cudaFree(m->w_cat_t[l]); cudaFree(m->w_pad_t[l]); cudaFree(m->bias[l]);
-        cudaFree(m->g_w_cat[l]); cudaFree(m->g_bias[l]);
+        cudaFree(m->g_w_cat[l]); cudaFree(m->g_bias[l]); cudaFree(m->s_w_cat[l]); cudaFree(m->s_bias[l]);
     }
     cudaFree(m->zeros);
     if (m->ctx && m->ctx->last_fwd_model == m) m->ctx->last_fwd_model = nullptr;
@@ -989,6 +989,54 @@ extern "C" int mg_model_grads(const mg_model* m, int32_t layer, const float** d_
     return MG_OK;
 }
 
+namespace {
+// Adagrad: state += g^2; w -= lr * g / (sqrt(state) + eps)
+__global__ void __launch_bounds__(kThreads) k_adagrad(float* w, const float* __restrict__ g, float* state, float lr, float eps, int64_t n) {
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const float gi = g[i];
+        const float s = state[i] + gi * gi;
+        state[i] = s;
+        w[i] -= lr * gi / (sqrtf(s) + eps);
+    }
+}
+}  // namespace
+
+// the copies of a layer's weights that the forward kernels read
+static int refresh_weight_copies(mg_ctx* ctx, mg_model* m, int l) {
+    const size_t di = m->dims[l], dn = m->dims[l + 1];
+    k_transpose<<<mg_grid(ctx, 2), kThreads, 0, ctx->stream>>>(m->w_cat[l], m->w_cat_t[l], (int)(2 * di), (int)dn, m->precision == MG_GEMM_TF32);
+    ctx->launches++;
+    return mg_pack_layer_weights(ctx, m->w_cat[l], m->w_pad_t[l], (int)di, (int)dn);
+}
+
+extern "C" int mg_model_adagrad_step(mg_ctx* ctx, mg_model* m, float lr, float eps) {
+    if (!ctx) return MG_ERR_ARG;
+    if (!m || m->ctx != ctx) return mg_fail(ctx, MG_ERR_ARG, "bad model handle");
+    if (!m->g_w_cat[0]) return mg_fail(ctx, MG_ERR_STATE, "mg_backward has not run");
+    if (!(eps > 0.f)) return mg_fail(ctx, MG_ERR_ARG, "eps must be positive");
+    MG_CUDA(ctx, cudaSetDevice(ctx->device));
+    cudaStream_t st = ctx->stream;
+    for (int l = 0; l < m->k; ++l) {
+        const size_t n_w = (size_t)2 * m->dims[l] * m->dims[l + 1], n_b = (size_t)m->dims[l + 1];
+        if (!m->s_w_cat[l]) {   // accumulated squared gradients start at zero
+            if (cudaMalloc((void**)&m->s_w_cat[l], n_w * sizeof(float)) != cudaSuccess || cudaMalloc((void**)&m->s_bias[l], n_b * sizeof(float)) != cudaSuccess) {
+                cudaGetLastError();
+                return mg_fail(ctx, MG_ERR_OOM, "optimizer state allocation failed");
+            }
+            MG_CUDA(ctx, cudaMemsetAsync(m->s_w_cat[l], 0, n_w * sizeof(float), st));
+            MG_CUDA(ctx, cudaMemsetAsync(m->s_bias[l], 0, n_b * sizeof(float), st));
+        }
+        k_adagrad<<<mg_grid(ctx, 2), kThreads, 0, st>>>(m->w_cat[l], m->g_w_cat[l], m->s_w_cat[l], lr, eps, (int64_t)n_w);
+        k_adagrad<<<1, kThreads, 0, st>>>(m->bias[l], m->g_bias[l], m->s_bias[l], lr, eps, (int64_t)n_b);
+        ctx->launches += 2;
+        const int rc = refresh_weight_copies(ctx, m, l);
+        if (rc) return rc;
+    }
+    MG_CUDA(ctx, cudaGetLastError());
+    MG_CUDA(ctx, cudaStreamSynchronize(st));
+    return MG_OK;
+}
+
 extern "C" int mg_model_sgd_step(mg_ctx* ctx, mg_model* m, float lr) {
     if (!ctx) return MG_ERR_ARG;
     if (!m || m->ctx != ctx) return mg_fail(ctx, MG_ERR_ARG, "bad model handle");
@@ -999,10 +1047,8 @@ extern "C" int mg_model_sgd_step(mg_ctx* ctx, mg_model* m, float lr) {
         const size_t di = m->dims[l], dn = m->dims[l + 1];
         k_sgd<<<mg_grid(ctx, 2), kThreads, 0, st>>>(m->w_cat[l], m->g_w_cat[l], lr, (int64_t)(2 * di * dn));
         k_sgd<<<1, kThreads, 0, st>>>(m->bias[l], m->g_bias[l], lr, (int64_t)dn);
-        // the copies the forward kernels read
-        k_transpose<<<mg_grid(ctx, 2), kThreads, 0, st>>>(m->w_cat[l], m->w_cat_t[l], (int)(2 * di), (int)dn, m->precision == MG_GEMM_TF32);
-        ctx->launches += 3;
-        const int rc = mg_pack_layer_weights(ctx, m->w_cat[l], m->w_pad_t[l], (int)di, (int)dn);
+        ctx->launches += 2;
+        const int rc = refresh_weight_copies(ctx, m, l);
         if (rc) return rc;
     }
     MG_CUDA(ctx, cudaGetLastError());

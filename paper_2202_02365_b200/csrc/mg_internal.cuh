@@ -232,6 +232,8 @@ struct mg_model {
     // mg_backward: gradients of w_cat and bias (allocated by the first backward pass), a zero vector
     float* g_w_cat[MG_MAX_HOPS] = {nullptr};
     float* g_bias[MG_MAX_HOPS] = {nullptr};
+    float* s_w_cat[MG_MAX_HOPS] = {nullptr};   // Adagrad: accumulated squared gradients
+    float* s_bias[MG_MAX_HOPS] = {nullptr};
     float* zeros = nullptr;
 };
 

@@ -981,6 +981,24 @@ def test_backward_pass_and_sgd_step(tiny, aggregator, prec, dims):
     ref3 = O.sample_dense(view, tg[3].tolist(), fanouts, seeds[3])
     want_out = O.forward(ref3, feats.numpy()[ref3["node_ids"]], [tuple(t.numpy() for t in l) for l in stepped], aggregator=aggregator)
     close(out[offs[3]:offs[4]].cpu().numpy(), want_out, 1e-3)
+    # two Adagrad steps with the same gradients on a fresh copy of the weights
+    if prec == "fp32":
+        m2 = ctx.model(layers, precision)
+        m2.set_aggregator(aggregator)
+        ctx.forward(m2, d, out)
+        ctx.backward(m2, d, g_out.cuda())
+        ctx.adagrad_step(m2, 0.05, 1e-8)
+        ctx.adagrad_step(m2, 0.05, 1e-8)
+        ada = []
+        for l in range(len(np_layers)):
+            cur = []
+            for x, gw in zip(np_layers[l], want[l]):
+                w1, s1 = O.adagrad_step(x, gw, np.zeros_like(gw), 0.05, 1e-8)
+                w2, _ = O.adagrad_step(w1, gw, s1, 0.05, 1e-8)
+                cur.append(w2)
+            ada.append(tuple(cur))
+        ctx.forward(m2, d, out)
+        close(out[offs[3]:offs[4]].cpu().numpy(), O.forward(ref3, feats.numpy()[ref3["node_ids"]], ada, aggregator=aggregator), 1e-3)
     # state errors
     ctx.keep_layer_outputs(False)
     other = ctx.model(layers, precision)

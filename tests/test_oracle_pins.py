@@ -742,3 +742,26 @@ def test_backward_against_torch_autograd():
         np.testing.assert_allclose(gs, ws.grad.numpy(), rtol=1e-10, atol=1e-12)
         np.testing.assert_allclose(gn, wn.grad.numpy(), rtol=1e-10, atol=1e-12)
         np.testing.assert_allclose(gb, b.grad.numpy(), rtol=1e-10, atol=1e-12)
+
+
+def test_adagrad_closed_forms():
+    w = np.array([1.0, -2.0, 0.5, 3.0])
+    g = np.array([0.5, -4.0, 0.0, 2.0])
+    # first step from a zero state: every coordinate with a gradient moves by lr against its sign
+    w1, s1 = O.adagrad_step(w, g, np.zeros(4), lr=0.1, eps=1e-12)
+    np.testing.assert_allclose(w1, w - 0.1 * np.sign(g), atol=1e-9)
+    np.testing.assert_allclose(s1, g * g)
+    # the same gradient again: steps shrink like 1 / sqrt(t)
+    w2, s2 = O.adagrad_step(w1, g, s1, lr=0.1, eps=1e-12)
+    np.testing.assert_allclose(w2, w1 - 0.1 * np.sign(g) / np.sqrt(2.0), atol=1e-9)
+    # against torch's optimiser over five steps of changing gradients
+    rng = np.random.default_rng(0)
+    tw = torch.tensor(w, requires_grad=True)
+    opt = torch.optim.Adagrad([tw], lr=0.05, eps=1e-10)
+    cw, cs = w.copy(), np.zeros(4)
+    for _ in range(5):
+        gi = rng.standard_normal(4)
+        tw.grad = torch.tensor(gi)
+        opt.step()
+        cw, cs = O.adagrad_step(cw, gi, cs, 0.05, 1e-10)
+    np.testing.assert_allclose(cw, tw.detach().numpy(), rtol=1e-10)
