@@ -147,7 +147,7 @@ def algorithmic_bytes(nodes, ents, cfg, feat_bytes=4):
             "a_min": int(a_s + a_f + a_i + a_o), "flops": int(flops), "agg_l1": int(agg_l1), "flops_l1": int(flops_l1)}
 
 
-def oracle_time(g_host, feats, layers, cfg, target_rows, seeds, budget_s=20.0):
+def oracle_time(g_host, feats, layers, cfg, target_rows, seeds, limit_s=20.0):
     """The CPU oracle as it stands on a bounded sample of the same mini-batches."""
     from oracle import dense_oracle as O
     view = O.GraphView(g_host[0], g_host[1], out_row_offsets=g_host[2] if len(g_host) > 2 else None,
@@ -162,7 +162,7 @@ def oracle_time(g_host, feats, layers, cfg, target_rows, seeds, budget_s=20.0):
         O.forward(ref, h0, np_layers)
         done += 1
         edges += len(ref["nbrs"])
-        if time.time() - t0 > budget_s:
+        if time.time() - t0 > limit_s:
             break
     dt = time.time() - t0
     return {"batches": done, "seconds": dt, "batches_per_s": done / dt, "edges_per_s": edges / dt}
@@ -180,7 +180,7 @@ def main():
     ap.add_argument("--lp-model", default="graphsage", choices=["graphsage", "gat"],
                     help="link-prediction workload only: the encoder layer (GraphSage mean or single-head graph attention)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-budget", type=float, default=20.0)
+    ap.add_argument("--cpu-seconds", type=float, default=20.0)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "mgdense" else args.warmup
 
@@ -418,7 +418,7 @@ def main():
     if rank == 0:
         if g_host is not None:
             r = oracle_time(g_host, feats, layers, cfg, all_targets[args.warmup * G:], step_seeds(args.warmup),
-                            budget_s=args.cpu_budget)
+                            limit_s=args.cpu_seconds)
             line["cpu_baseline"] = {"value": r["batches_per_s"], "unit": "mini-batches/s", "cores": 1, "kind": "oracle",
                                     "sample": f"{r['batches']} mini-batches of the timed workload in {r['seconds']:.1f} s",
                                     "sampled_edges_per_s": r["edges_per_s"]}
@@ -565,8 +565,8 @@ def run_reference(args, cfg):
     targets = inputs.train_set_batches(cfg["n"], cfg["train"], cfg["batch"], max(total, 1), seed=100)
     seeds = list(range(total))
     if args.warmup:
-        oracle_time(g_host, feats, layers, cfg, targets[:args.warmup], seeds[:args.warmup], budget_s=1e9)
-    r = oracle_time(g_host, feats, layers, cfg, targets[args.warmup:], seeds[args.warmup:], budget_s=1e9)
+        oracle_time(g_host, feats, layers, cfg, targets[:args.warmup], seeds[:args.warmup], limit_s=1e9)
+    r = oracle_time(g_host, feats, layers, cfg, targets[args.warmup:], seeds[args.warmup:], limit_s=1e9)
     line = {
         "impl": "reference", "metric": "DENSE sample+aggregate mini-batches/s", "value": r["batches_per_s"],
         "unit": "mini-batches/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
