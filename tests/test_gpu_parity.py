@@ -373,6 +373,33 @@ def test_full_size_config2_in_bench_launch_configuration():
     ctx.forward(model, d, out)
     g_host = (g.row_offsets.cpu().numpy(), g.nbrs.cpu().numpy())
     _check_batches_against_oracle(g_host, feats, layers, cfg["fanouts"], tg, seeds, d, out, offs, [0, 77, G - 1], RTOL_TC)
+    # backward pass at the same size: a loss that only looks at mini-batch 77 leaves gradients the oracle can compute
+    # from that mini-batch alone (TF32 forward: compared in norm, see the small backward test)
+    ctx.keep_layer_outputs(True)
+    ctx.forward(model, d, out)
+    b = 77
+    g_out = torch.zeros_like(out)
+    g_out[offs[b]:offs[b + 1]] = torch.randn((T, cfg["hidden"]), generator=torch.Generator().manual_seed(1)).cuda()
+    grads, g_h0, ids = ctx.backward(model, d, g_out, want_h0_grad=True)
+    ref = O.sample_dense(O.GraphView(g_host[0], g_host[1]), tg[b].tolist(), cfg["fanouts"], seeds[b])
+    nid = torch.as_tensor(ref["node_ids"], dtype=torch.int64, device=feats.device)
+    np_layers = [(w.numpy(), nn.numpy(), bb.numpy()) for w, nn, bb in layers]
+    want, d_h0 = O.backward(ref, feats[nid].float().cpu().numpy(), np_layers, g_out[offs[b]:offs[b + 1]].cpu().numpy())
+
+    def near(got, refv):
+        got, refv = np.asarray(got, dtype=np.float64), np.asarray(refv, dtype=np.float64)
+        assert np.linalg.norm(got - refv) <= 2e-2 * np.linalg.norm(refv)
+
+    for l in range(len(np_layers)):
+        for p in range(3):
+            near(grads[l][p].cpu().numpy(), want[l][p])
+    nodes, _ = d.counts()
+    row0 = np.concatenate([[0], np.cumsum(nodes.sum(1).cpu().numpy())])
+    lo, hi = int(row0[b]), int(row0[b + 1])
+    where = {v: r for r, v in enumerate(ref["node_ids"])}
+    ids_b = ids[lo:hi].cpu().numpy()
+    near(g_h0[lo:hi].cpu().numpy(), d_h0[[where[int(v)] for v in ids_b]])
+    assert not bool(g_h0[:lo].any()) and not bool(g_h0[hi:].any())     # the other mini-batches receive nothing
 
 
 def test_full_size_config3_in_bench_launch_configuration():
