@@ -19,6 +19,7 @@
 int mg_gemm_tf32(mg_ctx* ctx, const float* x, const float* w_t, const float* bias, float* out, int64_t M, int N, int K,
                  bool relu);  // mg_gemm_tcgen05.cu
 int mg_gemm_tf32_status(mg_ctx* ctx);
+int mg_gemm_tf32_splitk_add(mg_ctx* ctx, const float* x, const float* w_t, float* out, int64_t M, int N, int K, int kt_per_slice);
 // mg_layer_fused.cu
 int mg_pack_layer_weights(mg_ctx* ctx, const float* w_cat_dev, float* w_pad_t_dev, int d_in, int N);
 bool mg_layer_fused_supported(int d_in, int d_out);
@@ -763,6 +764,25 @@ __global__ void __launch_bounds__(256) k_grad_weights(const float* __restrict__ 
         }
 }
 
+// dst[cols][ld] = src[rows][cols]^T through a 32 x 33 shared tile; columns rows .. ld - 1 of dst are zero-filled (the
+// contraction dimension of the split-K GEMM is padded to a multiple of 32)
+__global__ void __launch_bounds__(256) k_transpose_pad(const float* __restrict__ src, float* dst, int64_t rows, int cols, int64_t ld) {
+    __shared__ float tile[32][33];
+    const int64_t r0 = (int64_t)blockIdx.x * 32;
+    const int c0 = blockIdx.y * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;   // 8 rows of the tile per pass
+    for (int i = ty; i < 32; i += 8) {
+        const int64_t r = r0 + i;
+        tile[i][tx] = (r < rows && c0 + tx < cols) ? src[r * cols + c0 + tx] : 0.f;
+    }
+    __syncthreads();
+    for (int i = ty; i < 32; i += 8) {
+        const int c = c0 + i;
+        const int64_t r = r0 + tx;
+        if (c < cols && r < ld) dst[(int64_t)c * ld + r] = tile[tx][i];
+    }
+}
+
 // The same on the (legacy, warp-level) tensor-core path in TF32: X^T is read as a column-major operand straight
 // from the row-major chunk, so nothing is transposed.  A block owns a 64 x 64 tile of dW and a slice of the rows; each
 // of its four warps a 32 x 32 quarter (2 x 2 fragments of 16 x 16, K = 8 rows per step).
@@ -813,13 +833,18 @@ __global__ void __launch_bounds__(128) k_grad_weights_tf32(const float* __restri
     }
 }
 
+constexpr int kBiasRowsPerBlock = 128;
 __global__ void __launch_bounds__(kThreads) k_grad_bias(const float* __restrict__ dpre, float* db, int64_t rows, int N) {
-    // a block sums a slice of the rows for every column, then one atomic add per column
-    const int64_t r_lo = (int64_t)blockIdx.x * kGradRowsPerBlock, r_hi = min(rows, r_lo + kGradRowsPerBlock);
+    // a block sums a slice of the rows for every column (four rows in flight per thread), then one atomic add per column
+    const int64_t r_lo = (int64_t)blockIdx.x * kBiasRowsPerBlock, r_hi = min(rows, r_lo + kBiasRowsPerBlock);
     for (int c = threadIdx.x; c < N; c += kThreads) {
-        float s = 0.f;
-        for (int64_t r = r_lo; r < r_hi; ++r) s += dpre[r * N + c];
-        atomicAdd(&db[c], s);
+        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+        int64_t r = r_lo;
+        for (; r + 4 <= r_hi; r += 4) {
+            s0 += dpre[r * N + c]; s1 += dpre[(r + 1) * N + c]; s2 += dpre[(r + 2) * N + c]; s3 += dpre[(r + 3) * N + c];
+        }
+        for (; r < r_hi; ++r) s0 += dpre[r * N + c];
+        atomicAdd(&db[c], (s0 + s1) + (s2 + s3));
     }
 }
 
@@ -844,14 +869,20 @@ __global__ void __launch_bounds__(kThreads) k_scatter_grad(ScatterArgs a) {
         locate_row(a.g, a.layer, row, &b, &local, &node);
         const int64_t in0 = rb_in[b];
         const float* dxr = a.dx + (row - a.row_lo) * 2 * a.d_in;
-        float* self = a.g_in + (in0 + local) * a.d_in;
-        for (int c = lane; c < a.d_in; c += 32) atomicAdd(&self[c], dxr[c]);
+        // (16-byte vector atomics: widths are multiples of 4 and every row starts 16-byte aligned)
+        float4* self = reinterpret_cast<float4*>(a.g_in + (in0 + local) * a.d_in);
+        const float4* dx4 = reinterpret_cast<const float4*>(dxr);
+        const int n4 = a.d_in / 4;
+        for (int c = lane; c < n4; c += 32) atomicAdd(&self[c], dx4[c]);
         const int32_t e0 = a.ent_off[node], e1 = a.ent_off[node + 1];
         if (e1 <= e0) continue;
         const float scale = a.sum_aggr ? 1.f : 1.f / (float)(e1 - e0);
         for (int32_t e = e0; e < e1; ++e) {
-            float* src = a.g_in + (in0 + a.ent_repr[e]) * a.d_in;
-            for (int c = lane; c < a.d_in; c += 32) atomicAdd(&src[c], dxr[a.d_in + c] * scale);
+            float4* src = reinterpret_cast<float4*>(a.g_in + (in0 + a.ent_repr[e]) * a.d_in);
+            for (int c = lane; c < n4; c += 32) {
+                const float4 v = dx4[n4 + c];
+                atomicAdd(&src[c], make_float4(v.x * scale, v.y * scale, v.z * scale, v.w * scale));
+            }
         }
     }
 }
@@ -914,6 +945,14 @@ extern "C" int mg_backward(mg_ctx* ctx, mg_model* m, mg_dense* d, const float* d
     if (ctx->bw_g_elems < g_total && (rc = mg_ensure(ctx, &ctx->bw_g, &ctx->bw_g_elems, g_total + g_total / 4 + 16))) return rc;
     if (ctx->bw_x_elems < (size_t)max_x && (rc = mg_ensure(ctx, &ctx->bw_x, &ctx->bw_x_elems, (size_t)max_x + 16))) return rc;
     if (ctx->bw_dx_elems < (size_t)max_x && (rc = mg_ensure(ctx, &ctx->bw_dx, &ctx->bw_dx_elems, (size_t)max_x + 16))) return rc;
+    if (m->precision == MG_GEMM_TF32) {   // transposed copies of a chunk's X and dPre rows
+        size_t max_t = 0;
+        for (int l = 1; l <= k; ++l) {
+            const int64_t rows = std::min<int64_t>(chunk_rows_for(m->dims[l - 1]), d->h_hdr.rows_total[l]);
+            max_t = std::max(max_t, (size_t)((rows + 31) / 32 * 32) * (2 * m->dims[l - 1] + m->dims[l]));
+        }
+        if (ctx->bw_xt_elems < max_t && (rc = mg_ensure(ctx, &ctx->bw_xt, &ctx->bw_xt_elems, max_t + 16))) return rc;
+    }
     if (g_total) MG_CUDA(ctx, cudaMemsetAsync(ctx->bw_g, 0, g_total * sizeof(float), st));
     if (d_h0_dev) MG_CUDA(ctx, cudaMemsetAsync(d_h0_dev, 0, (size_t)d->h_hdr.rows_total[0] * m->dims[0] * sizeof(float), st));
     const RowGeom geom{B, k, d->rowbase, d->cum, d->node_off};
@@ -951,11 +990,22 @@ extern "C" int mg_backward(mg_ctx* ctx, mg_model* m, mg_dense* d, const float* d
             const float* dpre = dpre_all + r0 * d_out;
             const unsigned slices = (unsigned)((rows + kGradRowsPerBlock - 1) / kGradRowsPerBlock);
             dim3 gw((unsigned)((2 * d_in + 63) / 64), (unsigned)((d_out + 63) / 64), slices);
-            if (m->precision == MG_GEMM_TF32 && d_in % 16 == 0 && d_out % 32 == 0)
+            if (m->precision == MG_GEMM_TF32 && rows >= 4096) {
+                // dW += X^T dPre as a tcgen05 GEMM whose contraction runs over the chunk's rows: both operands are
+                // transposed (rows become the contiguous dimension, padded to 32), the contraction is split over CTAs
+                const int64_t ld = (rows + 31) / 32 * 32;
+                dim3 tx((unsigned)(ld / 32), (unsigned)((2 * d_in + 31) / 32)), tg((unsigned)(ld / 32), (unsigned)((d_out + 31) / 32));
+                k_transpose_pad<<<tx, 256, 0, st>>>(ctx->bw_x, ctx->bw_xt, rows, 2 * d_in, ld);
+                k_transpose_pad<<<tg, 256, 0, st>>>(dpre, ctx->bw_xt + (size_t)2 * d_in * ld, rows, d_out, ld);
+                ctx->launches += 2;
+                if ((rc = mg_gemm_tf32_splitk_add(ctx, ctx->bw_xt, ctx->bw_xt + (size_t)2 * d_in * ld, m->g_w_cat[l - 1], 2 * d_in, d_out,
+                                                  (int)ld, 16))) return rc;
+                ctx->launches--;
+            } else if (m->precision == MG_GEMM_TF32 && d_in % 16 == 0 && d_out % 32 == 0)
                 k_grad_weights_tf32<<<gw, 128, 0, st>>>(ctx->bw_x, dpre, m->g_w_cat[l - 1], rows, 2 * d_in, d_out);
             else
                 k_grad_weights<<<gw, 256, 0, st>>>(ctx->bw_x, dpre, m->g_w_cat[l - 1], rows, 2 * d_in, d_out);
-            k_grad_bias<<<slices, kThreads, 0, st>>>(dpre, m->g_bias[l - 1], rows, d_out);
+            k_grad_bias<<<(unsigned)((rows + kBiasRowsPerBlock - 1) / kBiasRowsPerBlock), kThreads, 0, st>>>(dpre, m->g_bias[l - 1], rows, d_out);
             ctx->launches += 3;
             if (!g_in) continue;   // layer 1 without a gradient of the base representations
             if (m->precision == MG_GEMM_TF32) {

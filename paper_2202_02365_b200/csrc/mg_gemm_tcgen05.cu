@@ -31,6 +31,7 @@ struct GemmParams {
     const float* bias;
     int64_t M;
     int32_t N, K, BN, stages, tmem_cols, relu;
+    int32_t kt_per_slice;   // split-K: blockIdx.z owns this many 32-wide K steps and ADDS its product to out (0 = whole K, plain store)
     uint32_t* error;  // device word: 0 = ok, else the role that gave up waiting
 };
 
@@ -43,7 +44,9 @@ k_gemm_tf32(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t m0 = (int64_t)blockIdx.x * BM;
     const int n0 = blockIdx.y * p.BN;
-    const int kt_total = (p.K + BK - 1) / BK;
+    const int kt_all = (p.K + BK - 1) / BK;
+    const int kt_first = p.kt_per_slice ? (int)blockIdx.z * p.kt_per_slice : 0;
+    const int kt_total = p.kt_per_slice ? min(p.kt_per_slice, kt_all - kt_first) : kt_all;   // K steps of this CTA
     const uint32_t a_bytes = BM * BK * 4, b_bytes = (uint32_t)p.BN * BK * 4;
     uint8_t* stage_base = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t stage_bytes = a_bytes + b_bytes;  // both multiples of 1024
@@ -71,8 +74,8 @@ k_gemm_tf32(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 if (kt >= p.stages && !mbar_wait(&empty_bar[s], ((kt / p.stages) - 1) & 1)) { atomicExch(p.error, 1u); break; }
                 uint8_t* sa = stage_base + (size_t)s * stage_bytes;
                 mbar_expect_tx(&full_bar[s], stage_bytes);
-                tma_load_2d(sa, &map_a, &full_bar[s], kt * BK, (int)m0);
-                tma_load_2d(sa + a_bytes, &map_b, &full_bar[s], kt * BK, n0);
+                tma_load_2d(sa, &map_a, &full_bar[s], (kt_first + kt) * BK, (int)m0);
+                tma_load_2d(sa + a_bytes, &map_b, &full_bar[s], (kt_first + kt) * BK, n0);
             }
         }
         __syncwarp();
@@ -109,7 +112,9 @@ k_gemm_tf32(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 uint32_t v[32];
                 tmem_ld_32(tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)c0, v);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (row0 < p.M) store_slice_coalesced(v, out_stage + lane_group * (32 * 33), p.bias, p.out, row0, p.M, p.N, n0 + c0, p.relu != 0);
+                if (row0 >= p.M) continue;
+                if (p.kt_per_slice) add_slice_coalesced(v, out_stage + lane_group * (32 * 33), p.out, row0, p.M, p.N, n0 + c0);
+                else store_slice_coalesced(v, out_stage + lane_group * (32 * 33), p.bias, p.out, row0, p.M, p.N, n0 + c0, p.relu != 0);
             }
         }
     }
@@ -123,17 +128,18 @@ k_gemm_tf32(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 
 }  // namespace
 
-int mg_gemm_tf32(mg_ctx* ctx, const float* x, const float* w_t, const float* bias, float* out, int64_t M, int N, int K,
-                 bool relu) {
+static int gemm_tf32_launch(mg_ctx* ctx, const float* x, const float* w_t, const float* bias, float* out, int64_t M, int N, int K,
+                            bool relu, int kt_per_slice) {
     if (M <= 0) return MG_OK;
     if (K % 4 != 0 || N % 4 != 0) return mg_fail(ctx, MG_ERR_ARG, "GEMM sizes must be multiples of 4");
     GemmParams p;
     p.out = out; p.bias = bias; p.M = M; p.N = N; p.K = K; p.relu = relu ? 1 : 0; p.error = ctx->d_flags;
+    p.kt_per_slice = kt_per_slice;
     p.BN = std::min(256, (N + 15) / 16 * 16);
     p.tmem_cols = 32;
     while (p.tmem_cols < p.BN) p.tmem_cols <<= 1;
     const int stage_bytes = BM * BK * 4 + p.BN * BK * 4;
-    const int kt = (K + BK - 1) / BK;
+    const int kt = kt_per_slice ? std::min(kt_per_slice, (K + BK - 1) / BK) : (K + BK - 1) / BK;
     p.stages = std::max(1, std::min({kt, 8, (96 * 1024) / stage_bytes}));
     const size_t smem = (size_t)p.stages * stage_bytes + 1024;
     CUtensorMap ma, mb;
@@ -144,11 +150,23 @@ int mg_gemm_tf32(mg_ctx* ctx, const float* x, const float* w_t, const float* bia
         MG_CUDA(ctx, cudaFuncSetAttribute(k_gemm_tf32, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
         attr_set = true;
     }
-    dim3 grid((unsigned)((M + BM - 1) / BM), (unsigned)((N + p.BN - 1) / p.BN));
+    dim3 grid((unsigned)((M + BM - 1) / BM), (unsigned)((N + p.BN - 1) / p.BN),
+              kt_per_slice ? (unsigned)(((K + BK - 1) / BK + kt_per_slice - 1) / kt_per_slice) : 1u);
     k_gemm_tf32<<<grid, kGemmThreads, smem, ctx->stream>>>(ma, mb, p);
     ctx->launches++;
     MG_CUDA(ctx, cudaGetLastError());
     return MG_OK;
+}
+
+int mg_gemm_tf32(mg_ctx* ctx, const float* x, const float* w_t, const float* bias, float* out, int64_t M, int N, int K,
+                 bool relu) {
+    return gemm_tf32_launch(ctx, x, w_t, bias, out, M, N, K, relu, 0);
+}
+
+// out[M, N] += x[M, K] . w_t[N, K]^T with the contraction split over CTAs (kt_per_slice steps of 32 each): for products
+// whose K is far longer than M and N (weight gradients: K = rows of a chunk).  Atomic adds: any order.
+int mg_gemm_tf32_splitk_add(mg_ctx* ctx, const float* x, const float* w_t, float* out, int64_t M, int N, int K, int kt_per_slice) {
+    return gemm_tf32_launch(ctx, x, w_t, nullptr, out, M, N, K, false, std::max(1, kt_per_slice));
 }
 
 // After the stream has drained: MG_ERR_TIMEOUT if a GEMM gave up on a barrier (the word is cleared).

@@ -173,6 +173,21 @@ __device__ __forceinline__ void store_slice_coalesced(const uint32_t* v, float* 
     __syncwarp();
 }
 
+// The same for a split-K partial product: the slice is ADDED to out (no bias, no activation).
+__device__ __forceinline__ void add_slice_coalesced(const uint32_t* v, float* stage, float* __restrict__ out, int64_t row0, int64_t M,
+                                                    int N, int c0) {
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) stage[lane * 33 + j] = __uint_as_float(v[j]);
+    __syncwarp();
+    const int n = c0 + lane;
+    if (n < N) {
+        const int rows = (int)min((int64_t)32, M - row0);
+        for (int rr = 0; rr < rows; ++rr) atomicAdd(&out[(row0 + rr) * N + n], stage[rr * 33 + lane]);
+    }
+    __syncwarp();
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
