@@ -21,6 +21,8 @@
 int mg_gemm_tf32(mg_ctx* ctx, const float* x, const float* w_t, const float* bias, float* out, int64_t M, int N, int K,
                  bool relu);
 int mg_gemm_tf32_status(mg_ctx* ctx);
+int mg_gemm_tf32_dots(mg_ctx* ctx, const float* x, const float* w_t, const float* zero_bias, float* out, int64_t M, int N, int K,
+                      const float* a, const float* b, float* s_a, float* s_b);
 
 struct mg_gat_model {
     mg_ctx* ctx = nullptr;
@@ -339,9 +341,15 @@ extern "C" int mg_gat_forward(mg_ctx* ctx, const mg_gat_model* m, mg_dense* d, f
     for (int l = 1; l <= k; ++l) {
         const int d_in = m->dims[l - 1], d_out = m->dims[l];
         const int64_t rows_in = d->h_hdr.rows_total[l - 1], rows_out = d->h_hdr.rows_total[l];
+        float* s_src = ctx->gat_s;
+        float* s_dst = ctx->gat_s + rows_in;
+        const bool fused_scores = tf32 && d_out <= 256;   // the GEMM's epilogue also leaves Z a_src and Z a_dst
         {
             ProfScope ps(ctx, PH_GEMM, 1);
-            if (tf32) {
+            if (fused_scores) {
+                if ((rc = mg_gemm_tf32_dots(ctx, h_prev, m->w_t[l - 1], m->zeros, ctx->gat_z, rows_in, d_out, d_in, m->a_src[l - 1],
+                                            m->a_dst[l - 1], s_src, s_dst))) return rc;
+            } else if (tf32) {
                 if ((rc = mg_gemm_tf32(ctx, h_prev, m->w_t[l - 1], m->zeros, ctx->gat_z, rows_in, d_out, d_in, false))) return rc;
             } else {
                 dim3 g2((unsigned)((rows_in + 63) / 64), (unsigned)((d_out + 63) / 64));
@@ -350,16 +358,14 @@ extern "C" int mg_gat_forward(mg_ctx* ctx, const mg_gat_model* m, mg_dense* d, f
             }
         }
         ProfScope ps(ctx, PH_AGG_REST, 2);
-        float* s_src = ctx->gat_s;
-        float* s_dst = ctx->gat_s + rows_in;
-        k_gat_scores<<<grid, kThreads, 0, st>>>(ctx->gat_z, m->a_src[l - 1], m->a_dst[l - 1], rows_in, d_out, s_src, s_dst);
+        if (!fused_scores) k_gat_scores<<<grid, kThreads, 0, st>>>(ctx->gat_z, m->a_src[l - 1], m->a_dst[l - 1], rows_in, d_out, s_src, s_dst);
         AttendArgs a;
         a.g = geom; a.layer = l; a.ent_off = d->ent_off; a.ent_repr = d->ent_repr; a.z = ctx->gat_z; a.s_src = s_src; a.s_dst = s_dst;
         a.bias = m->bias[l - 1]; a.n_rows = rows_out; a.dim = d_out; a.relu = l < k; a.round = (tf32 && l < k) ? 1 : 0;
         a.slope = m->slope;
         a.out = l == k ? out_dev : ctx->gat_h[l & 1];
         k_gat_attend<<<grid, kThreads, 0, st>>>(a);
-        ctx->launches += 2;
+        ctx->launches += fused_scores ? 1 : 2;
         h_prev = a.out;
     }
     MG_CUDA(ctx, cudaGetLastError());
