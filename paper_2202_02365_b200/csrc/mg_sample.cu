@@ -486,7 +486,7 @@ __global__ void __launch_bounds__(kThreads) k_insert(InsertArgs a) {
 // mini-batch's rows and of the list of new nodes with ONE global atomic each, and gives every entry its node's row.
 constexpr int kDedupThreads = 1024;
 constexpr int kDedupMaxSlots = 26624;    // 208 KiB of keys + rows per block
-constexpr int kDedupMaxBuckets = 32;
+constexpr int kDedupMaxBuckets = 16;      // every block of a mini-batch walks all of its earlier nodes: measured faster than the global tables at 9 buckets, slower at 37
 constexpr int kDedupQueue = 64;          // per warp: up to 31 waiting + 32 new (id, row) pairs
 constexpr size_t kDedupQueueBytes = (size_t)(kDedupThreads / 32) * kDedupQueue * sizeof(uint2);
 constexpr int kBucketThreads = 512;
@@ -640,10 +640,13 @@ __global__ void __launch_bounds__(kDedupThreads) k_dedupe_last(DedupArgs a) {
     __syncthreads();
     // this bucket's pairs: enter the id, leave its slot in place of the id
     const int32_t n_pairs = run_start[nb];
-    auto pair_at = [&](int32_t i) -> int2* {
-        uint32_t r = 0;
-        while (r + 1 < nb && run_start[r + 1] <= i) ++r;
-        return a.pairs + run_lo[r] + (i - run_start[r]);
+    auto pair_at = [&](int32_t i) -> int2* {   // i-th pair of the bucket: which share's run it falls in (run_start ascends)
+        uint32_t lo = 0, hi = nb;                // run_start[lo] <= i < run_start[hi]
+        while (hi - lo > 1) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (run_start[mid] <= i) lo = mid; else hi = mid;
+        }
+        return a.pairs + run_lo[lo] + (i - run_start[lo]);
     };
     for (int32_t i0 = threadIdx.x; i0 < n_pairs; i0 += 4 * kDedupThreads) {
         int2* pp[4];
