@@ -179,6 +179,8 @@ def main():
     ap.add_argument("--window", type=int, default=0, help="mini-batches per window of the layer schedule (0 = whole layers)")
     ap.add_argument("--lp-model", default="graphsage", choices=["graphsage", "gat"],
                     help="link-prediction workload only: the encoder layer (GraphSage mean or single-head graph attention)")
+    ap.add_argument("--backward", action="store_true",
+                    help="also time mg_backward (with base-representation gradients) on one group of mini-batches")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=20.0)
     args = ap.parse_args()
@@ -348,6 +350,23 @@ def main():
             lat_ms.append((time.perf_counter() - t_lat) * 1e3)
     single_batch_latency_ms = float(np.median(lat_ms))
 
+    # ---- optional: the backward pass of one group (not part of the timed path; `--backward`) ----
+    backward_ms = None
+    if args.backward:
+        ctx.keep_layer_outputs(True)
+        g_out = torch.randn_like(out_dev)
+        bw = []
+        for rep in range(4):
+            ctx.forward(model, denses[0], out_dev)
+            torch.cuda.synchronize()
+            t_bw = time.perf_counter()
+            ctx.backward(model, denses[0], g_out, want_h0_grad=True)
+            torch.cuda.synchronize()
+            if rep:
+                bw.append((time.perf_counter() - t_bw) * 1e3)
+        backward_ms = float(np.median(bw))
+        ctx.keep_layer_outputs(False)
+
     if world > 1:
         t = torch.tensor([ms_dev, ms_e2e], device=device, dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -407,6 +426,7 @@ def main():
                 "d2h_bytes_per_step": int(G * T * cfg["hidden"] * 4), "ms_per_step": ms_e2e / args.steps},
         "gpu_launches": int(launches),
         "single_batch_latency_ms": single_batch_latency_ms,
+        "backward_ms_per_group": backward_ms,
         "clocks": clocks,
         "roofline": roofline,
         "tensor": tensor,
