@@ -1089,3 +1089,66 @@ def test_embedding_update_and_write_back_of_evicted_partitions():
     ctx.commit_resident(10_000)
     dp = ctx.sample(probe, [2], seed=5)
     close(ctx.gather_h0(dp, 0, len(refp["node_ids"]), 8).cpu().numpy(), want[refp["node_ids"]], 2e-5)
+
+
+@pytest.mark.parametrize("case", range(24))
+def test_randomised_small_configurations(case):
+    """Seeded random shapes through the whole path against the oracle: graph size and kind, number and sizes of
+    mini-batches (empty ones included), depth, fanouts, sampling direction, capacities (default, tight, large: the
+    three deduplication paths), partitions with a partial resident set, aggregator, precision."""
+    rng = np.random.default_rng(1000 + case)
+    n = int(rng.integers(40, 2500))
+    m = int(rng.integers(n, 12 * n))
+    g = inputs.rmat_graph(n, m, seed=case) if case % 2 else inputs.erdos_renyi_graph(n, m, seed=case)
+    dim = int(rng.choice([4, 8, 20, 36]))
+    feats = inputs.normal_features(n, dim, seed=case + 1)
+    parts = int(rng.choice([1, 1, 3, 5]))
+    ctx = mg.Context(0)
+    ctx.load_graph(g.row_offsets.to(torch.int32 if case % 3 == 0 else torch.int64).cuda(), g.nbrs.cuda())
+    inout = bool(rng.integers(0, 2))
+    gt = inputs.transpose_csr(g) if inout else None
+    if inout:
+        ctx.load_out_graph(gt.row_offsets.cuda(), gt.nbrs.cuda())
+        ctx.set_sample_direction("inout")
+    resident = None
+    if parts > 1:
+        ctx.set_partitioning(parts)
+        ctx.load_features(feats.cuda(), capacity_parts=parts)
+        resident = sorted(rng.choice(parts, size=int(rng.integers(1, parts + 1)), replace=False).tolist())
+        ctx.set_resident(resident)
+    else:
+        ctx.load_features(feats.cuda())
+    view = O.GraphView(g.row_offsets.numpy(), g.nbrs.numpy(), parts, resident,
+                       gt.row_offsets.numpy() if inout else None, gt.nbrs.numpy() if inout else None)
+    pool = torch.nonzero(inputs.resident_node_mask(n, parts, resident if resident is not None else [0])).flatten()
+    k = int(rng.integers(1, 5))
+    fanouts = [int(rng.integers(1, 9)) if rng.random() < 0.8 else int(rng.integers(9, 41)) for _ in range(k)]
+    B = int(rng.integers(1, 6))
+    sizes = [int(rng.integers(0, min(40, pool.numel()) + 1)) for _ in range(B)]
+    tg = [inputs.distinct_targets(pool, s, seed=50 * case + i) for i, s in enumerate(sizes)]
+    offs = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    seeds = [int(rng.integers(0, 2**62)) for _ in range(B)]
+    direction = "inout" if inout else "in"
+    refs = [O.sample_dense(view, tg[b].tolist(), fanouts, seeds[b], direction) for b in range(B)]
+    most = max(len(r["node_ids"]) for r in refs)
+    caps = [None, {"max_nodes_per_batch": most}, {"max_nodes_per_batch": 40_000}, {"max_nodes_per_batch": 1_200_000}][case % 4]
+    all_targets = torch.cat(tg) if B else torch.empty(0, dtype=torch.int32)
+    d = ctx.sample_many(all_targets.to(torch.int32), offs, fanouts, seeds, caps=caps)
+    for b in range(B):
+        assert_dense_equal(d.view(b), refs[b])
+    dims = [dim] + [int(rng.choice([4, 8, 12, 32])) for _ in range(k)]
+    layers = inputs.random_bias_layers(dims, seed=case + 3)
+    np_layers = [(w.numpy(), nn.numpy(), bb.numpy()) for w, nn, bb in layers]
+    aggregator = "sum" if case % 5 == 0 else "mean"
+    prec, rtol = ((mg.GEMM_TF32, RTOL_TC) if case % 2 else (mg.GEMM_FP32, RTOL_AGG))
+    if aggregator == "sum":
+        rtol *= 4                       # sums of up to 2 x 40 rows per node and layer instead of means
+    model = ctx.model(layers, prec)
+    model.set_aggregator(aggregator)
+    out = torch.full((int(offs[-1]), dims[-1]), float("nan"), dtype=torch.float32, device="cuda")
+    if int(offs[-1]):
+        ctx.forward(model, d, out)
+    for b in range(B):
+        if sizes[b]:
+            want = O.forward(refs[b], feats.numpy()[refs[b]["node_ids"]], np_layers, aggregator=aggregator)
+            close(out[offs[b]:offs[b + 1]].cpu().numpy(), want, rtol)
