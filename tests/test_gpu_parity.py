@@ -1152,3 +1152,58 @@ def test_randomised_small_configurations(case):
         if sizes[b]:
             want = O.forward(refs[b], feats.numpy()[refs[b]["node_ids"]], np_layers, aggregator=aggregator)
             close(out[offs[b]:offs[b + 1]].cpu().numpy(), want, rtol)
+
+
+@pytest.mark.parametrize("case", range(10))
+def test_randomised_backward_and_attention(case):
+    """Seeded random shapes for the two widened model paths: gradients (fp32) and the attention layers (fp32)."""
+    rng = np.random.default_rng(5000 + case)
+    n = int(rng.integers(60, 1500))
+    g = inputs.rmat_graph(n, int(rng.integers(2 * n, 10 * n)), seed=case)
+    dim = int(rng.choice([4, 8, 16]))
+    feats = inputs.normal_features(n, dim, seed=case + 1)
+    ctx = make_ctx(g, feats)
+    ctx.keep_layer_outputs(True)
+    view = oracle_view(g)
+    k = int(rng.integers(1, 4))
+    fanouts = [int(rng.integers(1, 7)) for _ in range(k)]
+    B = int(rng.integers(1, 4))
+    sizes = [int(rng.integers(1, 30)) for _ in range(B)]
+    tg = [inputs.distinct_targets(n, s, seed=70 * case + i) for i, s in enumerate(sizes)]
+    offs = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    seeds = [int(rng.integers(0, 2**40)) for _ in range(B)]
+    d = ctx.sample_many(torch.cat(tg), offs, fanouts, seeds)
+    refs = [O.sample_dense(view, tg[b].tolist(), fanouts, seeds[b]) for b in range(B)]
+    dims = [dim] + [int(rng.choice([4, 8, 20])) for _ in range(k)]
+    # gradients
+    layers = inputs.random_bias_layers(dims, seed=case)
+    np_layers = [(w.numpy(), nn.numpy(), bb.numpy()) for w, nn, bb in layers]
+    aggregator = "sum" if case % 3 == 0 else "mean"
+    model = ctx.model(layers, mg.GEMM_FP32)
+    model.set_aggregator(aggregator)
+    out = torch.empty((int(offs[-1]), dims[-1]), dtype=torch.float32, device="cuda")
+    ctx.forward(model, d, out)
+    g_out = torch.randn((int(offs[-1]), dims[-1]), generator=torch.Generator().manual_seed(case))
+    grads, g_h0, ids = ctx.backward(model, d, g_out.cuda(), want_h0_grad=True)
+    want = [[np.zeros_like(x, dtype=np.float64) for x in l] for l in np_layers]
+    nodes, _ = d.counts()
+    row0 = np.concatenate([[0], np.cumsum(nodes.sum(1).cpu().numpy())])
+    for b in range(B):
+        gr, d_h0 = O.backward(refs[b], feats.numpy()[refs[b]["node_ids"]], np_layers, g_out[offs[b]:offs[b + 1]].numpy(), aggregator)
+        for l in range(k):
+            for p in range(3):
+                want[l][p] += gr[l][p]
+        lo, hi = int(row0[b]), int(row0[b + 1])
+        where = {v: r for r, v in enumerate(refs[b]["node_ids"])}
+        close(g_h0[lo:hi].cpu().numpy(), d_h0[[where[int(v)] for v in ids[lo:hi].cpu().numpy()]], 5e-4)
+    for l in range(k):
+        for p in range(3):
+            close(grads[l][p].cpu().numpy(), want[l][p], 5e-4)
+    # attention layers
+    gat_layers = _gat_layers(dims, seed=case + 9)
+    slope = float(rng.choice([0.0, 0.2, 0.5]))
+    gm = ctx.gat_model(gat_layers, mg.GEMM_FP32, negative_slope=slope)
+    ctx.gat_forward(gm, d, out)
+    for b in range(B):
+        want_out = O.gat_forward(refs[b], feats.numpy()[refs[b]["node_ids"]], [tuple(t.numpy() for t in l) for l in gat_layers], slope=slope)
+        close(out[offs[b]:offs[b + 1]].cpu().numpy(), want_out, 5e-5)
