@@ -103,10 +103,19 @@ __global__ void __launch_bounds__(kThreads) k_gat_gather0(GatherArgs a) {
         const uint32_t id = (uint32_t)a.nodes[node];
         const uint32_t p = id / a.part_size;
         const char* src = a.slots + (int64_t)a.slot_of_part[p] * a.slot_bytes + (int64_t)(id - p * a.part_size) * a.row_bytes;
-        float* dst = a.x + row * a.dim;
-        for (int c = lane; c < a.dim; c += 32) {
-            const float v = a.half ? __half2float(reinterpret_cast<const __half*>(src)[c]) : reinterpret_cast<const float*>(src)[c];
-            dst[c] = a.round ? round_tf32(v) : v;
+        float4* dst = reinterpret_cast<float4*>(a.x + row * a.dim);   // (rows are multiples of 16 bytes on both sides)
+        for (int c = lane; c < a.dim / 4; c += 32) {
+            float4 v;
+            if (a.half) {
+                const uint2 raw = reinterpret_cast<const uint2*>(src)[c];
+                const float2 lo = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
+                const float2 hi = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
+                v = make_float4(lo.x, lo.y, hi.x, hi.y);
+            } else {
+                v = reinterpret_cast<const float4*>(src)[c];
+            }
+            if (a.round) v = make_float4(round_tf32(v.x), round_tf32(v.y), round_tf32(v.z), round_tf32(v.w));
+            dst[c] = v;
         }
     }
 }
@@ -187,6 +196,7 @@ struct AttendArgs {
 __device__ __forceinline__ float leaky(float v, float slope) { return v > 0.f ? v : slope * v; }
 
 // one warp per output row: softmax over {self} + entries, then the weighted sum of their Z rows
+template <int W>   // W = 32-column slices a lane owns: the row is at most 32 W wide
 __global__ void __launch_bounds__(kThreads) k_gat_attend(AttendArgs a) {
     const int lane = threadIdx.x & 31;
     const int64_t warps = (int64_t)gridDim.x * (kThreads / 32);
@@ -208,23 +218,23 @@ __global__ void __launch_bounds__(kThreads) k_gat_attend(AttendArgs a) {
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xFFFFFFFFu, den, o);
         const float inv = 1.f / den;
-        float acc[kMaxWidthPerLane];
+        float acc[W];
         {
             const float w = __expf(self_score - mx) * inv;
             const float* zr = a.z + me * a.dim;
 #pragma unroll
-            for (int q = 0; q < kMaxWidthPerLane; ++q) { const int c = lane + 32 * q; acc[q] = c < a.dim ? w * zr[c] : 0.f; }
+            for (int q = 0; q < W; ++q) { const int c = lane + 32 * q; acc[q] = c < a.dim ? w * zr[c] : 0.f; }
         }
         for (int32_t e = e0; e < e1; ++e) {
             const int64_t src = in0 + a.ent_repr[e];
             const float w = __expf(leaky(sd + a.s_src[src], a.slope) - mx) * inv;
             const float* zr = a.z + src * a.dim;
 #pragma unroll
-            for (int q = 0; q < kMaxWidthPerLane; ++q) { const int c = lane + 32 * q; if (c < a.dim) acc[q] = fmaf(w, zr[c], acc[q]); }
+            for (int q = 0; q < W; ++q) { const int c = lane + 32 * q; if (c < a.dim) acc[q] = fmaf(w, zr[c], acc[q]); }
         }
         float* dst = a.out + row * a.dim;
 #pragma unroll
-        for (int q = 0; q < kMaxWidthPerLane; ++q) {
+        for (int q = 0; q < W; ++q) {
             const int c = lane + 32 * q;
             if (c >= a.dim) continue;
             float v = acc[q] + a.bias[c];
@@ -364,7 +374,12 @@ extern "C" int mg_gat_forward(mg_ctx* ctx, const mg_gat_model* m, mg_dense* d, f
         a.bias = m->bias[l - 1]; a.n_rows = rows_out; a.dim = d_out; a.relu = l < k; a.round = (tf32 && l < k) ? 1 : 0;
         a.slope = m->slope;
         a.out = l == k ? out_dev : ctx->gat_h[l & 1];
-        k_gat_attend<<<grid, kThreads, 0, st>>>(a);
+        const int slices = (d_out + 31) / 32;   // instantiations for rows of up to 32, 64, 128, 256, 512 floats
+        if (slices <= 1) k_gat_attend<1><<<grid, kThreads, 0, st>>>(a);
+        else if (slices <= 2) k_gat_attend<2><<<grid, kThreads, 0, st>>>(a);
+        else if (slices <= 4) k_gat_attend<4><<<grid, kThreads, 0, st>>>(a);
+        else if (slices <= 8) k_gat_attend<8><<<grid, kThreads, 0, st>>>(a);
+        else k_gat_attend<kMaxWidthPerLane><<<grid, kThreads, 0, st>>>(a);
         ctx->launches += fused_scores ? 1 : 2;
         h_prev = a.out;
     }
