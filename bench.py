@@ -37,6 +37,11 @@ CONFIGS = {
     "config3_papers100m_shaped_inout": dict(n=111_000_000, m=1_620_000_000, kind="rmat", dim=128, hidden=256,
                                             fanouts=[15, 10, 5], batch=1000, parts=16, train=1_100_000, inout=True,
                                             group=16),
+    # the setting of the paper's Table 6 at three layers: up to 10 incoming + 10 outgoing neighbours per node and layer
+    # (the paper does not state its mini-batch size; 1,000 targets give mini-batches of its reported order, ~1M nodes)
+    "table6_papers100m_shaped_3layers": dict(n=111_000_000, m=1_620_000_000, kind="rmat", dim=128, hidden=256,
+                                             fanouts=[10, 10, 10], batch=1000, parts=16, train=1_100_000, inout=True,
+                                             group=8),
     # config 4's shapes at a tenth of its node count, whole fp16 table in HBM (no swaps): a throughput probe of the
     # wide fp16 layer-1 path, not the out-of-core configuration itself (that one is exercised by the tests)
     "config4_tenth_fp16_768_in_hbm": dict(n=12_200_000, m=130_000_000, kind="rmat", dim=768, hidden=256,
