@@ -82,7 +82,7 @@ struct FusedArgs {
     uint32_t* error;
 };
 
-constexpr int kKeyCap = 512;    // source-row indices of a row block's entries cached in shared memory (16 per row)
+constexpr int kKeyCap = 704;    // source-row indices of a row block's entries cached in shared memory (22 per row: what still fits the 196 KB carve-out)
 
 // What a producer needs to build one output row: x = source row of the row's own representation; y = first
 // entry and z = number of entries in the sample's entry arrays (z < 0: row past the end); w = first cached
