@@ -1207,3 +1207,32 @@ def test_randomised_backward_and_attention(case):
     for b in range(B):
         want_out = O.gat_forward(refs[b], feats.numpy()[refs[b]["node_ids"]], [tuple(t.numpy() for t in l) for l in gat_layers], slope=slope)
         close(out[offs[b]:offs[b + 1]].cpu().numpy(), want_out, 5e-5)
+
+
+@pytest.mark.parametrize("fanouts", [[22], [21, 3], [23, 2], [16, 2], [40, 2]])
+def test_fused_layer_rows_around_the_entry_cache(tiny, fanouts):
+    """Rows whose 32-row blocks hold about as many entries as the fused kernel caches in shared memory (22 per row on
+    average): the graph's degrees spread around 20, so blocks fall on both sides of the limit, and a fanout of 40 puts
+    every block past it.  Both aggregators, two mini-batches with a ragged last block."""
+    g, feats = tiny
+    ctx = make_ctx(g, feats)
+    sizes = [301, 77]
+    tg = [inputs.distinct_targets(10_000, s, seed=40 + i) for i, s in enumerate(sizes)]
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    seeds = [321, 322]
+    d = ctx.sample_many(torch.cat(tg), offs, fanouts, seeds)
+    dims = [16] + [32] * (len(fanouts) - 1) + [24]
+    layers = inputs.random_bias_layers(dims, seed=12)
+    model = ctx.model(layers, mg.GEMM_TF32)
+    out = torch.empty((int(offs[-1]), dims[-1]), dtype=torch.float32, device="cuda")
+    view = oracle_view(g)
+    np_layers = [(w.numpy(), n.numpy(), b.numpy()) for w, n, b in layers]
+    for aggregator in ("mean", "sum"):
+        model.set_aggregator(aggregator)
+        out.fill_(float("nan"))
+        ctx.forward(model, d, out)
+        for b in range(2):
+            ref = O.sample_dense(view, tg[b].tolist(), fanouts, seeds[b])
+            assert_dense_equal(d.view(b), ref)
+            want = O.forward(ref, feats.numpy()[ref["node_ids"]], np_layers, aggregator=aggregator)
+            close(out[offs[b]:offs[b + 1]].cpu().numpy(), want, RTOL_TC)
