@@ -221,20 +221,23 @@ __device__ __forceinline__ void store_pick(const PickArgs& a, bool valid, int32_
     a.ent_repr[out_pos] = b;
 }
 
-// G lanes per node, fanout <= G <= 32.
+// G lanes per node, fanout <= G <= 32; a warp holds 32 / G nodes (G need not divide 32: the lanes left over idle, and
+// G = 5 or 10 keeps 30 lanes busy where the next power of two keeps 20).
 template <int G>
 __global__ void __launch_bounds__(kThreads) k_pick(PickArgs a) {
     if (a.hdr->status) return;
-    constexpr int kGroups = kThreads / G;
+    constexpr int kPerWarp = 32 / G;
+    constexpr int kGroups = (kThreads / 32) * kPerWarp;
     const int32_t lo = a.hdr->hop_base[a.hop], hi = a.hdr->hop_base[a.hop + 1];
     const int lane = threadIdx.x & 31;
-    const int gl = threadIdx.x % G;               // lane inside the group
-    const int gshift = lane - gl;                 // first warp lane of the group
+    const int grp = lane / G;                     // group inside the warp (== kPerWarp: a left-over lane)
+    const int gl = lane - grp * G;                // lane inside the group
+    const int gshift = grp * G;                   // first warp lane of the group
     const uint32_t gmask = (G == 32) ? 0xFFFFFFFFu : (((1u << G) - 1u) << gshift);
     const int32_t f = a.fanout;
     for (int32_t base = lo + blockIdx.x * kGroups; base < hi; base += gridDim.x * kGroups) {
-        const int32_t i = base + threadIdx.x / G;
-        const bool node_ok = i < hi;
+        const int32_t i = base + (threadIdx.x >> 5) * kPerWarp + grp;
+        const bool node_ok = grp < kPerWarp && i < hi;
         int32_t v = 0, b = 0, out0 = 0;
         int64_t r0 = 0, d = 0;
         if (node_ok) {
@@ -1471,8 +1474,14 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
                 PickArgs a{d->hdr, h, f, d->nodes, d->node_batch, dir ? d->node_r0_out : d->node_r0, dir ? d->node_deg_out : d->node_deg,
                            dir ? ctx->view_nbrs_out : ctx->view_nbrs, d->ent_off, d->ent_nbrs, d->ent_repr, d->d_seeds,
                            dir ? d->node_deg : nullptr, dir ? (uint32_t)MG_OUT_SLOT_BASE : 0u};
-                if (f <= 4) k_pick<4><<<grid, kThreads, 0, st>>>(a);
+                // the narrowest group that holds the fanout among those that waste at most two lanes of a warp
+                if (f <= 2) k_pick<2><<<grid, kThreads, 0, st>>>(a);
+                else if (f == 3) k_pick<3><<<grid, kThreads, 0, st>>>(a);
+                else if (f == 4) k_pick<4><<<grid, kThreads, 0, st>>>(a);
+                else if (f == 5) k_pick<5><<<grid, kThreads, 0, st>>>(a);
+                else if (f == 6) k_pick<6><<<grid, kThreads, 0, st>>>(a);
                 else if (f <= 8) k_pick<8><<<grid, kThreads, 0, st>>>(a);
+                else if (f <= 10) k_pick<10><<<grid, kThreads, 0, st>>>(a);
                 else if (f <= 16) k_pick<16><<<grid, kThreads, 0, st>>>(a);
                 else if (f <= 32) k_pick<32><<<grid, kThreads, 0, st>>>(a);
                 else {
