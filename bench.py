@@ -54,7 +54,7 @@ LP_WORKLOAD = "config5_freebase86m_shaped_lp"
 DEFAULT_WORKLOAD = "config3_papers100m_shaped"
 HBM_NOMINAL_GBS = 8000.0
 # dram bytes (read + write) of one launch of the dominant kernel, measured with ncu (see profiles/)
-NCU_TRAFFIC_PER_LAUNCH = {("config3_papers100m_shaped", 128): 10.70e9,
+NCU_TRAFFIC_PER_LAUNCH = {("config3_papers100m_shaped", 128): 10.87e9,
                           ("config3_papers100m_shaped_inout", 16): 7.57e9}
 
 
