@@ -5,13 +5,14 @@ statement of what the CUDA library must compute.  Only the test-suite, the
 smoke check and the benchmark's CPU-baseline leg may import it; the product
 package never does, and this file imports nothing from the product package.
 
-It follows the paper's algorithms in the paper's order and notation:
-  * Algorithm 1  (multi-hop neighbourhood sampling)      -> sample_dense
-  * Section 4.1  (oneHopSample, computeNextDelta)        -> one_hop_sample, compute_next_delta
-  * Section 4.2  (repr_map, Steps 1 and 2 of the forward)-> build_repr_map, forward
-  * Algorithm 2  (DENSE update after a layer)            -> update_dense
-  * Algorithm 3  (layer aggregation; mean instead of sum)-> sage_layer / additive_layer
-Floating point is fp64 throughout.
+What it computes, and where the paper defines it:
+  * Algorithm 1, Section 4.1 (multi-hop sampling of only the newly reached nodes; oneHopSample,
+    computeNextDelta): sample_levels keeps one sampled neighbour list per node in a dict and finds
+    each hop's new nodes with Python sets; emit_dense lays the result out as the DENSE arrays.
+  * Section 4.2 (repr_map; a layer's output, then the shortened DENSE): forward, sage_layer,
+    additive_layer (the example layer of Algorithm 3), update_dense (the result of Algorithm 2,
+    obtained by dropping the per-node data the next layer no longer needs and laying it out again).
+Floating point is fp64 throughout; nothing is blocked, fused or vectorised beyond one matmul per layer.
 
 Points the paper leaves open, and the reading taken here:
   * which f neighbours are kept when a node has more than f: f distinct
@@ -175,126 +176,134 @@ def one_hop_sample(row, f: int, seed: int, node: int, hop: int, slot_base: int =
     return [int(row[p]) for p in sorted(chosen)]
 
 
-def one_hop_sample_all(view: GraphView, delta, f: int, seed: int, hop: int, direction: str = "in"):
-    """oneHopSample(delta, f): concatenated neighbours and each node's start.
-    direction "inout": up to f incoming, then up to f outgoing neighbours per node."""
-    if direction not in ("in", "inout"):
-        raise ValueError("direction must be 'in' or 'inout'")
-    d_nbrs, d_offsets = [], []
-    for v in delta:
-        d_offsets.append(len(d_nbrs))
-        d_nbrs.extend(one_hop_sample(view.row(v), f, seed, v, hop))
-        if direction == "inout":
-            d_nbrs.extend(one_hop_sample(view.out_row(v), f, seed, v, hop, OUT_SLOT_BASE))
-    return d_nbrs, d_offsets
-
-
-def compute_next_delta(d_nbrs, node_ids):
-    """computeNextDelta: the unique nodes among the new neighbours that are not
-    in node_ids yet (Section 4.1), in ascending id."""
-    return sorted(set(d_nbrs) - set(node_ids))
-
-
-def sample_dense(view: GraphView, target_nodes, fanouts, seed: int, direction: str = "in"):
-    """Algorithm 1.  `fanouts` is ordered away from the targets (per direction
-    when direction is "inout").
-
-    Returns a dict with node_ids, node_id_offsets (k+2 entries), nbrs,
-    nbr_offsets (sampled nodes + 1 entries) and repr_map.
-    """
-    k = len(fanouts)
-    target_nodes = [int(t) for t in target_nodes]
+def _check_targets(view: GraphView, target_nodes):
+    """Algorithm 1 takes unique target ids; Section 3: a batch's targets lie in resident partitions."""
     if len(set(target_nodes)) != len(target_nodes):
-        raise ValueError("duplicate target")            # Algorithm 1: unique ids
+        raise ValueError("duplicate target")
     for t in target_nodes:
         if not (0 <= t < view.n_nodes):
             raise ValueError("target out of range")
         if not view.is_resident(t):
-            raise ValueError("target not resident")      # X_i is a subset of S_i
-
-    node_id_offsets = [0]
-    node_ids = list(target_nodes)
-    nbr_offsets = []
-    nbrs = []
-    delta = list(target_nodes)                           # Delta_k
-    for i in range(k, 0, -1):
-        hop = k - i
-        f = fanouts[hop]                                 # Algorithm 1's fanouts[i]
-        d_nbrs, d_offsets = one_hop_sample_all(view, delta, f, seed, hop, direction)
-        nbr_offsets = d_offsets + [o + len(d_nbrs) for o in nbr_offsets]
-        nbrs = d_nbrs + nbrs
-        delta = compute_next_delta(d_nbrs, node_ids)     # Delta_{i-1}
-        node_id_offsets = [0] + [o + len(delta) for o in node_id_offsets]
-        node_ids = delta + node_ids
-    dense = {
-        "node_ids": node_ids,
-        "node_id_offsets": node_id_offsets + [len(node_ids)],   # sentinel
-        "nbrs": nbrs,
-        "nbr_offsets": nbr_offsets + [len(nbrs)],               # sentinel
-    }
-    dense["repr_map"] = build_repr_map(dense)
-    return dense
+            raise ValueError("target not resident")
 
 
-def build_repr_map(dense):
-    """repr_map[e] = row of H^0 (aligned with node_ids) holding nbrs[e] (Section 4.2)."""
+def sample_levels(view: GraphView, target_nodes, fanouts, seed: int, direction: str = "in"):
+    """What Algorithm 1 / Section 4.1 computes, kept per node instead of in arrays.
+
+    levels[h] = the nodes first reached after h hops (levels[0] = the targets in the caller's
+    order; every later level in ascending id) -- the paper's Delta_{k-h}.  sampled[v] = the one-hop
+    sample of v, drawn exactly once, at the hop whose level v belongs to, with that hop's fanout
+    (`fanouts` is ordered away from the targets; per direction when direction is "inout": up to f
+    incoming neighbours followed by up to f outgoing ones).  The nodes of the last level are
+    reached but not sampled."""
+    if direction not in ("in", "inout"):
+        raise ValueError("direction must be 'in' or 'inout'")
+    target_nodes = [int(t) for t in target_nodes]
+    _check_targets(view, target_nodes)
+    seen = set(target_nodes)
+    levels = [list(target_nodes)]
+    sampled = {}
+    for hop, f in enumerate(fanouts):
+        reached = set()
+        for v in levels[hop]:                    # only the newly reached nodes are sampled
+            picks = one_hop_sample(view.row(v), f, seed, v, hop)
+            if direction == "inout":
+                picks = picks + one_hop_sample(view.out_row(v), f, seed, v, hop, OUT_SLOT_BASE)
+            sampled[v] = picks
+            reached.update(picks)
+        new = reached - seen                     # unique, and not in any earlier level
+        seen |= new
+        levels.append(sorted(new))
+    return levels, sampled
+
+
+def emit_dense(levels, sampled):
+    """The DENSE arrays of Section 4.1 for per-node samples: node_ids lists the levels from the farthest one to the
+    targets; nbrs lists the samples of the sampled nodes in node_ids order; the offsets carry a terminal entry;
+    repr_map[e] = position of nbrs[e] in node_ids (Section 4.2)."""
+    node_ids, node_id_offsets = [], []
+    for level in reversed(levels):
+        node_id_offsets.append(len(node_ids))
+        node_ids.extend(level)
+    node_id_offsets.append(len(node_ids))
     where = {}
-    for r, v in enumerate(dense["node_ids"]):
-        assert v not in where, "node_ids must be duplicate-free"
+    for r, v in enumerate(node_ids):
+        assert v not in where, "a node belongs to one level only"
         where[v] = r
-    return [where[u] for u in dense["nbrs"]]
+    nbrs, nbr_offsets = [], []
+    for v in node_ids[node_id_offsets[1]:]:      # the farthest level has no samples
+        nbr_offsets.append(len(nbrs))
+        nbrs.extend(sampled[v])
+    nbr_offsets.append(len(nbrs))
+    return {"node_ids": node_ids, "node_id_offsets": node_id_offsets, "nbrs": nbrs, "nbr_offsets": nbr_offsets,
+            "repr_map": [where[u] for u in nbrs]}
+
+
+def sample_dense(view: GraphView, target_nodes, fanouts, seed: int, direction: str = "in"):
+    """Multi-hop sampling into DENSE (Algorithm 1): node_ids, node_id_offsets (k+2 entries), nbrs, nbr_offsets
+    (sampled nodes + 1 entries) and repr_map."""
+    levels, sampled = sample_levels(view, target_nodes, fanouts, seed, direction)
+    return emit_dense(levels, sampled)
+
+
+def read_dense(dense):
+    """Back from the arrays to per-node form: (levels from the targets outwards, sampled)."""
+    nio, node_ids = dense["node_id_offsets"], dense["node_ids"]
+    levels = [list(node_ids[nio[j]:nio[j + 1]]) for j in range(len(nio) - 1)][::-1]
+    sampled = {}
+    for r, v in enumerate(node_ids[nio[1]:]):
+        sampled[v] = list(dense["nbrs"][dense["nbr_offsets"][r]:dense["nbr_offsets"][r + 1]])
+    return levels, sampled
 
 
 # ----------------------------------------------------------------------------
 # Section 4.2: forward pass over DENSE
 # ----------------------------------------------------------------------------
 def update_dense(dense):
-    """Algorithm 2: drop Delta_{i-1} and the neighbours of Delta_i."""
-    nio = dense["node_id_offsets"]
-    node_ids, nbr_offsets = dense["node_ids"], dense["nbr_offsets"]
-    nbrs, repr_map = dense["nbrs"], dense["repr_map"]
-    delta_prev = node_ids[:nio[1]]
-    delta_i = node_ids[nio[1]:nio[2]]
-    delta_i_nbrs = nbrs[:nbr_offsets[len(delta_i)]]
-    return {
-        "nbrs": nbrs[len(delta_i_nbrs):],
-        "repr_map": [r - len(delta_prev) for r in repr_map[len(delta_i_nbrs):]],
-        "nbr_offsets": [o - len(delta_i_nbrs) for o in nbr_offsets[len(delta_i):]],
-        "node_ids": node_ids[nio[1]:],
-        "node_id_offsets": [o - len(delta_prev) for o in nio[1:]],
-    }
+    """What DENSE looks like after a layer (Algorithm 2, Section 4.2): the farthest level has served as input for
+    the last time, and the samples of the level next to it were consumed by the layer, so both go; that level is
+    now the farthest one, without samples.  Positions (offsets, repr_map) are those of the shortened arrays."""
+    levels, sampled = read_dense(dense)
+    gone = levels.pop()                          # farthest level
+    assert not any(v in sampled for v in gone)
+    for v in levels[-1]:
+        del sampled[v]
+    return emit_dense(levels, sampled)
 
 
-def _segment_reduce(nbr_repr, nbr_offsets, n_rows, mean: bool):
-    out = np.zeros((n_rows, nbr_repr.shape[1]), dtype=np.float64)
+def _neighbour_rows(dense, r):
+    """Rows of the layer's input that output row r aggregates (through repr_map, repeats included)."""
+    return dense["repr_map"][dense["nbr_offsets"][r]:dense["nbr_offsets"][r + 1]]
+
+
+def _aggregate(dense, h_prev, mean: bool):
+    """Per output row the sum (or mean) of its sampled neighbours' input rows; zero for a row without any."""
+    first = dense["node_id_offsets"][1]          # input rows below `first` belong to the farthest level
+    n_rows = len(dense["node_ids"]) - first
+    out = np.zeros((n_rows, h_prev.shape[1]), dtype=np.float64)
     for r in range(n_rows):
-        lo, hi = nbr_offsets[r], nbr_offsets[r + 1]
-        if hi > lo:
-            s = nbr_repr[lo:hi].sum(axis=0)
-            out[r] = s / (hi - lo) if mean else s
+        rows = _neighbour_rows(dense, r)
+        if len(rows):
+            s = h_prev[np.asarray(rows, dtype=np.int64)].sum(axis=0)
+            out[r] = s / len(rows) if mean else s
     return out
 
 
 def additive_layer(dense, h_prev):
-    """Algorithm 3 as printed: H = segment_sum(H_prev[repr_map]) + self."""
+    """The example layer of Section 4.2 (Algorithm 3): every output row is its own input row plus the sum of its
+    sampled neighbours' input rows."""
     h_prev = np.asarray(h_prev, dtype=np.float64)
-    n_rows = len(dense["node_ids"]) - dense["node_id_offsets"][1]
-    nbr_repr = h_prev[np.asarray(dense["repr_map"], dtype=np.int64)]
-    nbr_aggr = _segment_reduce(nbr_repr, dense["nbr_offsets"], n_rows, mean=False)
-    self_repr = h_prev[dense["node_id_offsets"][1]:]
-    return nbr_aggr + self_repr
+    return h_prev[dense["node_id_offsets"][1]:] + _aggregate(dense, h_prev, mean=False)
 
 
 def sage_layer(dense, h_prev, w_self, w_nbr, bias, relu: bool, aggregator: str = "mean"):
-    """Algorithm 3 with self/neighbour linears; the neighbour term is GraphSage's mean over
-    the sampled neighbours ("mean") or their sum ("sum", the aggregation Algorithm 3 prints)."""
+    """GraphSage layer over DENSE: act(self . W_self + aggregate . W_nbr + bias); the aggregate is the mean over the
+    sampled neighbours ("mean") or their sum ("sum", the aggregation of Algorithm 3)."""
     if aggregator not in ("mean", "sum"):
         raise ValueError("aggregator must be 'mean' or 'sum'")
     h_prev = np.asarray(h_prev, dtype=np.float64)
-    n_rows = len(dense["node_ids"]) - dense["node_id_offsets"][1]
-    nbr_repr = h_prev[np.asarray(dense["repr_map"], dtype=np.int64)]
-    nbr_aggr = _segment_reduce(nbr_repr, dense["nbr_offsets"], n_rows, mean=(aggregator == "mean"))
     self_repr = h_prev[dense["node_id_offsets"][1]:]
+    nbr_aggr = _aggregate(dense, h_prev, mean=(aggregator == "mean"))
     out = (self_repr @ np.asarray(w_self, dtype=np.float64)
            + nbr_aggr @ np.asarray(w_nbr, dtype=np.float64)
            + np.asarray(bias, dtype=np.float64))
@@ -329,7 +338,7 @@ def gat_layer(dense, h_prev, w, a_src, a_dst, bias, relu: bool, slope: float = 0
 def gat_forward(dense, h0, layers, slope: float = 0.2):
     """k attention layers with Algorithm 2 between them; layers: (w, a_src, a_dst, bias); ReLU on all but the last."""
     h = np.asarray(h0, dtype=np.float64)
-    cur = {key: list(val) for key, val in dense.items()}
+    cur = dense
     for i, (w, a_src, a_dst, bias) in enumerate(layers):
         h = gat_layer(cur, h, w, a_src, a_dst, bias, relu=(i + 1 < len(layers)), slope=slope)
         cur = update_dense(cur)
@@ -345,7 +354,7 @@ def forward(dense, h0, layers, return_all: bool = False, aggregator: str = "mean
     """
     h = np.asarray(h0, dtype=np.float64)
     assert h.shape[0] == len(dense["node_ids"])
-    cur = {key: list(val) for key, val in dense.items()}
+    cur = dense
     outs = []
     for i, (w_self, w_nbr, bias) in enumerate(layers):
         h = sage_layer(cur, h, w_self, w_nbr, bias, relu=(i + 1 < len(layers)), aggregator=aggregator)
@@ -354,45 +363,50 @@ def forward(dense, h0, layers, return_all: bool = False, aggregator: str = "mean
     return outs if return_all else h
 
 
-def backward(dense, h0, layers, d_out, aggregator: str = "mean"):
+def backward(dense, h0, layers, d_out, aggregator: str = "mean", relu_masks=None):
     """Gradients of a scalar loss through forward(): d_out = dL/dH^k, one row per target.
 
-    The chain rule through Algorithm 3 (self and neighbour linears, mean or sum over the
-    sampled neighbours through repr_map, ReLU on all but the last layer) and Algorithm 2
-    (layer l's rows are the rows of layer l-1 without the outermost delta).  Returns
-    (grads, d_h0): grads[l] = (dW_self, dW_nbr, dbias) of layer l + 1, d_h0 = dL/dH^0 with one
-    row per entry of node_ids (the gradient of the base representations, Section 3)."""
+    The chain rule through the GraphSage layer (self and neighbour linears, mean or sum over the
+    sampled neighbours through repr_map, ReLU on all but the last layer) and through the shortening
+    of DENSE between layers (layer l's rows are the rows of layer l-1 without the farthest level).
+    Returns (grads, d_h0): grads[l] = (dW_self, dW_nbr, dbias) of layer l + 1, d_h0 = dL/dH^0 with
+    one row per entry of node_ids (the gradient of the base representations, Section 3).
+
+    relu_masks (optional): for each layer but the last a boolean array shaped like that layer's
+    output; the ReLU of that layer then passes the gradient where the mask is set instead of where
+    this function's own pre-activation is positive.  A test that compares against a forward pass
+    computed in lower precision hands over the branch that pass took, so that both sides
+    differentiate the same piecewise-linear function."""
     h = np.asarray(h0, dtype=np.float64)
-    cur = {key: list(val) for key, val in dense.items()}
+    cur = dense
     saved = []
     for i, (w_self, w_nbr, bias) in enumerate(layers):
         first = cur["node_id_offsets"][1]
-        n_rows = len(cur["node_ids"]) - first
-        nbr_repr = h[np.asarray(cur["repr_map"], dtype=np.int64)]
-        agg = _segment_reduce(nbr_repr, cur["nbr_offsets"], n_rows, mean=(aggregator == "mean"))
+        agg = _aggregate(cur, h, mean=(aggregator == "mean"))
         pre = (h[first:] @ np.asarray(w_self, dtype=np.float64) + agg @ np.asarray(w_nbr, dtype=np.float64)
                + np.asarray(bias, dtype=np.float64))
-        saved.append((cur, h, agg, pre))
-        h = np.maximum(pre, 0.0) if i + 1 < len(layers) else pre
+        last = i + 1 == len(layers)
+        passes = None if last else (pre > 0.0 if relu_masks is None else np.asarray(relu_masks[i], dtype=bool))
+        saved.append((cur, h, agg, passes))
+        h = pre if last else np.where(passes, pre, 0.0)
         cur = update_dense(cur)
     d_h = np.asarray(d_out, dtype=np.float64)
     grads = [None] * len(layers)
     for i in range(len(layers) - 1, -1, -1):
-        cur, h_in, agg, pre = saved[i]
+        cur, h_in, agg, passes = saved[i]
         w_self, w_nbr = (np.asarray(x, dtype=np.float64) for x in layers[i][:2])
-        d_pre = d_h * (pre > 0.0) if i + 1 < len(layers) else d_h
+        d_pre = d_h if passes is None else d_h * passes
         first = cur["node_id_offsets"][1]
-        n_rows = len(cur["node_ids"]) - first
         grads[i] = (h_in[first:].T @ d_pre, agg.T @ d_pre, d_pre.sum(axis=0))
         d_in = np.zeros_like(h_in)
         d_in[first:] += d_pre @ w_self.T
         d_agg = d_pre @ w_nbr.T
-        for r in range(n_rows):
-            lo, hi = cur["nbr_offsets"][r], cur["nbr_offsets"][r + 1]
-            if hi > lo:
-                share = d_agg[r] / (hi - lo) if aggregator == "mean" else d_agg[r]
-                for e in range(lo, hi):
-                    d_in[cur["repr_map"][e]] += share
+        for r in range(d_pre.shape[0]):
+            rows = _neighbour_rows(cur, r)
+            if len(rows):
+                share = d_agg[r] / len(rows) if aggregator == "mean" else d_agg[r]
+                for src in rows:                 # a repeated neighbour receives its share once per repeat
+                    d_in[src] += share
         d_h = d_in
     return grads, d_h
 

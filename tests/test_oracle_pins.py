@@ -744,6 +744,105 @@ def test_backward_against_torch_autograd():
         np.testing.assert_allclose(gb, b.grad.numpy(), rtol=1e-10, atol=1e-12)
 
 
+def test_backward_with_a_given_relu_branch():
+    """relu_masks: the ReLU passes the gradient where the mask says, not where the oracle's own pre-activation is
+    positive.  Pinned by (a) its own branch reproducing the default, (b) torch autograd on the same network with the
+    ReLU replaced by a multiplication with random masks, (c) central finite differences of that masked network."""
+    off, nb = _random_graph(60, 500, 13)
+    d = O.sample_dense(O.GraphView(off, nb), [5, 6, 7, 30], [3, 3, 2], seed=2)
+    rng = np.random.default_rng(4)
+    h0 = rng.standard_normal((len(d["node_ids"]), 3))
+    dims = [3, 4, 5, 2]
+    layers = [(rng.standard_normal((a, b)), rng.standard_normal((a, b)), rng.standard_normal(b)) for a, b in zip(dims[:-1], dims[1:])]
+    g_out = rng.standard_normal((4, 2))
+    outs = O.forward(d, h0, layers, return_all=True)
+    own = [o > 0 for o in outs[:-1]]
+    g_def, dh_def = O.backward(d, h0, layers, g_out)
+    g_own, dh_own = O.backward(d, h0, layers, g_out, relu_masks=own)
+    np.testing.assert_array_equal(dh_def, dh_own)
+    for a, b in zip(g_def, g_own):
+        for x, y in zip(a, b):
+            np.testing.assert_array_equal(x, y)
+    masks = [rng.random(o.shape) < 0.6 for o in outs[:-1]]
+    grads, d_h0 = O.backward(d, h0, layers, g_out, relu_masks=masks)
+
+    def masked_net(h, ls, lib):
+        cur = d
+        for i, (ws, wn, b) in enumerate(ls):
+            first = cur["node_id_offsets"][1]
+            rows = len(cur["node_ids"]) - first
+            counts = np.diff(cur["nbr_offsets"])[:rows]
+            if lib is torch:
+                seg = torch.repeat_interleave(torch.arange(rows), torch.tensor(counts))
+                agg = torch.zeros((rows, h.shape[1]), dtype=torch.float64).index_add(0, seg, h[torch.tensor(cur["repr_map"], dtype=torch.int64)])
+                agg = agg / torch.tensor(counts).clamp(min=1)[:, None]
+            else:
+                agg = np.zeros((rows, h.shape[1]))
+                np.add.at(agg, np.repeat(np.arange(rows), counts), h[np.asarray(cur["repr_map"], dtype=np.int64)])
+                agg = agg / np.maximum(counts, 1)[:, None]
+            h = h[first:] @ ws + agg @ wn + b
+            if i + 1 < len(ls):
+                h = h * (torch.tensor(masks[i], dtype=torch.float64) if lib is torch else masks[i])
+            cur = O.update_dense(cur)
+        return h
+
+    th0 = torch.tensor(h0, requires_grad=True)
+    tl = [tuple(torch.tensor(x, requires_grad=True) for x in l) for l in layers]
+    (masked_net(th0, tl, torch) * torch.tensor(g_out)).sum().backward()
+    np.testing.assert_allclose(d_h0, th0.grad.numpy(), rtol=1e-10, atol=1e-12)
+    for (gs, gn, gb), (ws, wn, b) in zip(grads, tl):
+        np.testing.assert_allclose(gs, ws.grad.numpy(), rtol=1e-10, atol=1e-12)
+        np.testing.assert_allclose(gn, wn.grad.numpy(), rtol=1e-10, atol=1e-12)
+        np.testing.assert_allclose(gb, b.grad.numpy(), rtol=1e-10, atol=1e-12)
+    eps = 1e-6
+    for li, pi, idx in [(0, 0, (1, 2)), (0, 1, (2, 0)), (1, 1, (3, 4)), (2, 0, (0, 1)), (1, 2, (2,))]:
+        plus = [tuple(np.array(x, copy=True) for x in l) for l in layers]
+        minus = [tuple(np.array(x, copy=True) for x in l) for l in layers]
+        plus[li][pi][idx] += eps
+        minus[li][pi][idx] -= eps
+        fd = float(((masked_net(h0, plus, np) - masked_net(h0, minus, np)) * g_out).sum()) / (2 * eps)
+        assert abs(fd - grads[li][pi][idx]) <= 1e-6 * max(1.0, abs(fd))
+
+
+def test_per_node_form_and_arrays_are_two_views_of_one_sample():
+    """sample_levels / emit_dense / read_dense: the arrays list exactly the per-node samples, level by level, and
+    reading them back gives the per-node form again; shortening DENSE (Algorithm 2) equals sampling one hop less
+    from the same levels."""
+    off, nb = _random_graph(150, 1300, 17)
+    view = O.GraphView(off, nb)
+    targets, fanouts = [9, 80, 3, 41], [4, 3, 2]
+    levels, sampled = O.sample_levels(view, targets, fanouts, seed=6)
+    d = O.emit_dense(levels, sampled)
+    assert d == O.sample_dense(view, targets, fanouts, seed=6)
+    lv2, sm2 = O.read_dense(d)
+    assert lv2 == levels and sm2 == sampled
+    assert levels[0] == targets and all(l == sorted(l) for l in levels[1:])
+    flat = [v for l in levels for v in l]
+    assert len(set(flat)) == len(flat)
+    assert set(sampled) == set(v for l in levels[:-1] for v in l)
+    for h, l in enumerate(levels[:-1]):
+        for v in l:
+            row = [int(u) for u in nb[off[v]:off[v + 1]]]
+            assert len(sampled[v]) == min(len(row), fanouts[h])
+            it = iter(row)
+            assert all(u in it for u in sampled[v])          # a sub-sequence of the stored row
+    # the node set of level h+1 is what level h's samples reach for the first time
+    seen = set(levels[0])
+    for h in range(len(fanouts)):
+        new = set(u for v in levels[h] for u in sampled[v]) - seen
+        assert sorted(new) == levels[h + 1]
+        seen |= new
+    # one layer later: the farthest level and the samples next to it are gone, nothing else moved
+    u = O.update_dense(d)
+    lv3, sm3 = O.read_dense(u)
+    assert lv3 == levels[:-1]
+    assert sm3 == {v: sampled[v] for l in levels[:-2] for v in l}
+    n_gone, e_gone = len(levels[-1]), sum(len(sampled[v]) for v in levels[-2])
+    assert u["node_ids"] == d["node_ids"][n_gone:]
+    assert u["nbrs"] == d["nbrs"][e_gone:]
+    assert u["repr_map"] == [r - n_gone for r in d["repr_map"][e_gone:]]
+
+
 def test_adagrad_closed_forms():
     w = np.array([1.0, -2.0, 0.5, 3.0])
     g = np.array([0.5, -4.0, 0.0, 2.0])
