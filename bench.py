@@ -153,25 +153,57 @@ def algorithmic_bytes(nodes, ents, cfg, feat_bytes=4):
             "a_min": int(a_s + a_f + a_i + a_o), "flops": int(flops), "agg_l1": int(agg_l1), "flops_l1": int(flops_l1)}
 
 
-def oracle_time(g_host, feats, layers, cfg, target_rows, seeds, limit_s=20.0):
-    """The CPU oracle as it stands on a bounded sample of the same mini-batches."""
+def _oracle_worker_init():
+    try:
+        from threadpoolctl import threadpool_limits
+        threadpool_limits(1)          # one core per worker: the oracle's matmul must not spread over the others' cores
+    except Exception:
+        pass
+
+
+def _oracle_sample(job):
     from oracle import dense_oracle as O
-    view = O.GraphView(g_host[0], g_host[1], out_row_offsets=g_host[2] if len(g_host) > 2 else None,
-                       out_nbrs=g_host[3] if len(g_host) > 2 else None)
-    direction = "inout" if len(g_host) > 2 else "in"
-    np_layers = [(w.numpy(), n.numpy(), b.numpy()) for w, n, b in layers]
-    done, edges, t0 = 0, 0, time.time()
-    for tg, seed in zip(target_rows, seeds):
-        ref = O.sample_dense(view, tg.tolist(), cfg["fanouts"], int(seed), direction)
-        ids = torch.as_tensor(ref["node_ids"], dtype=torch.int64)
-        h0 = feats[ids.to(feats.device)].float().cpu().numpy()
-        O.forward(ref, h0, np_layers)
-        done += 1
-        edges += len(ref["nbrs"])
-        if time.time() - t0 > limit_s:
-            break
-    dt = time.time() - t0
-    return {"batches": done, "seconds": dt, "batches_per_s": done / dt, "edges_per_s": edges / dt}
+    tg, seed = job
+    g_host, cfg = _ORACLE_SHARED["g_host"], _ORACLE_SHARED["cfg"]
+    inout = len(g_host) > 2
+    view = O.GraphView(g_host[0], g_host[1], out_row_offsets=g_host[2] if inout else None, out_nbrs=g_host[3] if inout else None)
+    return O.sample_dense(view, tg, cfg["fanouts"], int(seed), "inout" if inout else "in")
+
+
+def _oracle_forward(job):
+    from oracle import dense_oracle as O
+    ref, h0 = job
+    O.forward(ref, h0, _ORACLE_SHARED["np_layers"])
+    return len(ref["nbrs"])
+
+
+_ORACLE_SHARED = {}
+
+
+def oracle_time(g_host, feats, layers, cfg, target_rows, seeds, limit_s=20.0, workers=None):
+    """The CPU oracle as it stands on a bounded sample of the same mini-batches, one mini-batch per worker process
+    over the host cores this job may use.  Rounds of `workers` mini-batches until the time limit: the workers sample
+    (Algorithm 1), the parent hands each its H^0 rows (the feature table lives on the GPU), the workers run the layers.
+    The workers are forked, so they share the graph arrays with the parent and never touch CUDA."""
+    import multiprocessing as mp
+    cores = len(os.sched_getaffinity(0))
+    workers = max(1, min(workers or cores, len(target_rows)))
+    _ORACLE_SHARED.update(g_host=g_host, cfg=cfg, np_layers=[(w.numpy(), n.numpy(), b.numpy()) for w, n, b in layers])
+    jobs = [(tg.tolist(), int(seed)) for tg, seed in zip(target_rows, seeds)]
+    done, edges = 0, 0
+    with mp.get_context("fork").Pool(workers, initializer=_oracle_worker_init) as pool:
+        t0 = time.time()
+        while done < len(jobs):
+            chunk = jobs[done:done + workers]
+            refs = pool.map(_oracle_sample, chunk, chunksize=1)
+            h0s = [feats[torch.as_tensor(r["node_ids"], dtype=torch.int64).to(feats.device)].float().cpu().numpy() for r in refs]
+            edges += sum(pool.map(_oracle_forward, list(zip(refs, h0s)), chunksize=1))
+            done += len(chunk)
+            if time.time() - t0 > limit_s:
+                break
+        dt = time.time() - t0
+    return {"batches": done, "seconds": dt, "batches_per_s": done / dt, "edges_per_s": edges / dt, "workers": workers,
+            "cores_available": cores}
 
 
 def main():
@@ -279,15 +311,19 @@ def main():
         tg = host_targets[i] if e2e else dev_targets[i]
         ctx.sample_many_begin(tg, offs, cfg["fanouts"], step_seeds(i), caps=caps, out=denses[i % 3])
 
-    def run_steps(first, count, e2e):
+    def run_steps(first, count, e2e, export=False):
         """`count` steps, software-pipelined: groups i+1 and i+2 are sampled (sampling stream) while group i runs
-        its layers (context stream); with e2e the host H^k of group i is copied out during group i+1."""
+        its layers (context stream); with e2e the host H^k of group i is copied out during group i+1; with export
+        every group's DENSE is also laid out in the paper's canonical arrays (ascending ids inside each delta) for all
+        of its mini-batches, on the sampling stream, before the next sample is queued there."""
         last = first + count
         begin(first, e2e)
         if first + 1 < last:
             begin(first + 1, e2e)
         for i in range(first, last):
             ctx.sample_many_end(denses[i % 3])
+            if export:
+                denses[i % 3].export_many()
             if i + 2 < last:
                 begin(i + 2, e2e)
             if e2e:
@@ -323,11 +359,24 @@ def main():
     ms_dev = ev0.elapsed_time(ev1)
     launches = ctx.kernel_launches() - launches0
 
+    # ---- the same steps with the canonical export of every mini-batch inside the timed region -------------
+    for i in range(2):
+        run_steps(i, 1, False, export=True)      # allocates the export buffers
+    barrier()
+    ev4, ev5 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev4.record()
+    run_steps(args.warmup, args.steps, False, export=True)
+    torch.cuda.synchronize()                     # the last export ends on the sampling stream
+    ev5.record()
+    barrier()
+    ms_export = ev4.elapsed_time(ev5)
+
     # ---- the same steps again with per-phase CUDA events on the library's stream ---------------
     ctx.profile(True)
     ctx.profile_read(reset=True)
     for s in range(args.steps):          # one group at a time here, so that the phase events do not overlap
         run_step(args.warmup + s, False)
+        denses[(args.warmup + s) % 3].export_many()      # its kernels are the "sample_sort" phase
         n_, e_ = denses[(args.warmup + s) % 3].counts()
         stats["nodes"].append(n_); stats["ents"].append(e_)
     phases = ctx.profile_read(reset=True)
@@ -374,9 +423,9 @@ def main():
         ctx.keep_layer_outputs(False)
 
     if world > 1:
-        t = torch.tensor([ms_dev, ms_e2e], device=device, dtype=torch.float64)
+        t = torch.tensor([ms_dev, ms_e2e, ms_export], device=device, dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_dev, ms_e2e = float(t[0]), float(t[1])
+        ms_dev, ms_e2e, ms_export = float(t[0]), float(t[1]), float(t[2])
 
     nodes = torch.cat(stats["nodes"]).numpy()
     ents = torch.cat(stats["ents"]).numpy()
@@ -390,7 +439,8 @@ def main():
     # The dominant kernel is the fused layer-1 kernel (k_sage_layer_fused<first>): it gathers the base
     # representations (the bulk of A_min), reduces them and runs the layer's GEMM on the tensor cores.
     # It is HBM-bound: achieved = its algorithmic bytes (V d0 s + 4 (E_1 + N_1)) over its event time.
-    sample_ms = sum(v["ms"] for name, v in phases.items() if name.startswith("sample_"))
+    export_ms = phases["sample_sort"]["ms"]          # mg_dense_export_many's kernels; not part of sample_ms / path_hbm
+    sample_ms = sum(v["ms"] for name, v in phases.items() if name.startswith("sample_") and name != "sample_sort")
     agg1 = phases["aggregate_l1"]
     rest = phases["aggregate_rest"]
     gemm = phases["gemm"]
@@ -425,6 +475,11 @@ def main():
                    "l2": "inputs larger than L2 (feature table and CSR far exceed 126 MB; no flush)",
                    "setup_s": setup},
         "sampled_edges_per_s": sampled_edges / (ms_dev / 1e3),
+        # the same steps with mg_dense_export_many for every group inside the timed region: the paper's arrays
+        # (ascending ids inside each delta, repr_map in those rows) for all mini-batches of the group
+        "value_with_canonical_export": n_batches / (ms_export / 1e3),
+        "ms_per_step_with_canonical_export": ms_export / args.steps,
+        "export_ms_per_step": export_ms / args.steps,
         "per_batch": {"nodes": float(nodes.sum(1).mean()), "sampled_edges": float(ents.sum(1).mean()),
                       "algorithmic_bytes": alg["a_min"] / (args.steps * G),
                       "gemm_flops": alg["flops"] / (args.steps * G)},
@@ -445,8 +500,9 @@ def main():
         if g_host is not None:
             r = oracle_time(g_host, feats, layers, cfg, all_targets[args.warmup * G:], step_seeds(args.warmup),
                             limit_s=args.cpu_seconds)
-            line["cpu_baseline"] = {"value": r["batches_per_s"], "unit": "mini-batches/s", "cores": 1, "kind": "oracle",
-                                    "sample": f"{r['batches']} mini-batches of the timed workload in {r['seconds']:.1f} s",
+            line["cpu_baseline"] = {"value": r["batches_per_s"], "unit": "mini-batches/s", "cores": r["workers"], "kind": "oracle",
+                                    "sample": f"{r['batches']} mini-batches of the timed workload in {r['seconds']:.1f} s, one "
+                                              f"mini-batch per worker process ({r['cores_available']} cores available to the job)",
                                     "sampled_edges_per_s": r["edges_per_s"]}
         print(json.dumps(line))
     if world > 1:
@@ -586,23 +642,25 @@ def run_reference(args, cfg):
         g_host = g_host + (gt.row_offsets.cpu().numpy(), gt.nbrs.cpu().numpy())
         del gt
     del g
-    per_step = 1
+    cores = len(os.sched_getaffinity(0))
+    per_step = cores                      # a step = one round of mini-batches, one per host core
     total = (args.warmup + args.steps) * per_step
     targets = inputs.train_set_batches(cfg["n"], cfg["train"], cfg["batch"], max(total, 1), seed=100)
     seeds = list(range(total))
-    if args.warmup:
-        oracle_time(g_host, feats, layers, cfg, targets[:args.warmup], seeds[:args.warmup], limit_s=1e9)
-    r = oracle_time(g_host, feats, layers, cfg, targets[args.warmup:], seeds[args.warmup:], limit_s=1e9)
+    nw = args.warmup * per_step
+    if nw:
+        oracle_time(g_host, feats, layers, cfg, targets[:nw], seeds[:nw], limit_s=1e9)
+    r = oracle_time(g_host, feats, layers, cfg, targets[nw:], seeds[nw:], limit_s=1e9)
     line = {
         "impl": "reference", "metric": "DENSE sample+aggregate mini-batches/s", "value": r["batches_per_s"],
         "unit": "mini-batches/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": r["seconds"] / max(1, r["batches"]) * 1e3, "higher_is_better": True, "scaling": "weak",
+        "ms_per_step": r["seconds"] / max(1, args.steps) * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": args.workload, "nodes": cfg["n"], "edges": n_edges, "feature_dim": cfg["dim"],
                    "hidden": cfg["hidden"], "fanouts": cfg["fanouts"], "targets_per_batch": cfg["batch"],
                    "mini_batches_per_step": per_step},
-        "cpu_baseline": {"value": r["batches_per_s"], "unit": "mini-batches/s", "cores": 1, "kind": "oracle",
-                         "sample": f"{per_step} mini-batch per step, {r['batches']} steps"},
+        "cpu_baseline": {"value": r["batches_per_s"], "unit": "mini-batches/s", "cores": r["workers"], "kind": "oracle",
+                         "sample": f"{per_step} mini-batches per step (one per worker process), {args.steps} steps"},
         "e2e": {"value": r["batches_per_s"], "unit": "mini-batches/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "sampled_edges_per_s": r["edges_per_s"],
     }

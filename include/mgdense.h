@@ -154,7 +154,13 @@ int mg_set_resident(mg_ctx* ctx, const int32_t* part_ids /*host*/, int32_t n, in
 /* Wait at most timeout_ms for the pending copies (polling, never an unbounded wait), then
  * switch the slot map to the pending set and rebuild the in-buffer view of the graph: the
  * rows of resident nodes restricted to resident neighbours (sampling sees only in-memory
- * nodes and edges, Section 3).  MG_ERR_TIMEOUT leaves the pending set pending. */
+ * nodes and edges, Section 3).  timeout_ms <= 0 polls once.  MG_ERR_TIMEOUT leaves the pending set
+ * pending and the committed one in use: sampling and forward calls go on under the old set, and a
+ * later mg_commit_resident picks the pending set up.  A sample drawn under the old set stays usable
+ * after the commit only if every partition that was resident when it was drawn kept its slot (the
+ * new set contains the old one); otherwise calls that read feature rows through it (mg_forward,
+ * mg_backward, mg_gather_h0, mg_gat_forward, mg_apply_embedding_sgd ...) refuse it with
+ * MG_ERR_STATE -- run them before the commit, or sample again. */
 int mg_commit_resident(mg_ctx* ctx, int32_t timeout_ms);
 
 /* ---- DENSE sampling (Algorithm 1) ---------------------------------------------------- */
@@ -212,6 +218,20 @@ int mg_dense_counts(const mg_dense* d, int32_t* n_batches, int32_t* k, int64_t* 
  * depends on that order); this call, mg_gather_h0 and mg_layer_output sort the mini-batch's ids (one radix sort per
  * call, on the context's stream, synchronous) and translate rows and repr_map entries. */
 int mg_dense_view(mg_ctx* ctx, mg_dense* d, int32_t batch, mg_dense_arrays* out);
+
+/* The canonical DENSE ordering for the whole sample in one pass (Algorithm 1's computeNextDelta leaves every delta
+ * as the ascending list of its ids; on the device a delta is kept in the order its nodes were found).
+ * mg_dense_export_many queues, on the library's sampling stream, ONE sort of all nodes of all mini-batches by
+ * (mini-batch, delta, id) and the translation of every entry, and returns at once: no host synchronisation, no work
+ * per mini-batch.  It overlaps whatever runs on the context's stream (the layers of this or another sample); a later
+ * sample into `d` is ordered behind it.  mg_dense_export_view waits for that export (first call only) and hands out
+ * mini-batch `batch` of it: the same five arrays as mg_dense_view, bit for bit, as DEVICE pointers into a buffer owned
+ * by `d` that holds all mini-batches packed one after the other; valid until the next mg_dense_export_many or
+ * mg_sample* on `d`.  The buffer is sized from the sample's capacities (4 x max_nodes_total + 2 x max_entries_total
+ * int32) and allocated by the first export of a handle.  Errors: MG_ERR_ARG, MG_ERR_STATE (no completed sample / no
+ * export), MG_ERR_CAPACITY (mini-batch, delta, id and row index do not fit one 64-bit sort key), MG_ERR_OOM. */
+int mg_dense_export_many(mg_ctx* ctx, mg_dense* d);
+int mg_dense_export_view(mg_ctx* ctx, mg_dense* d, int32_t batch, mg_dense_arrays* out);
 
 int mg_dense_free(mg_dense* d);
 
@@ -280,14 +300,18 @@ int mg_layer_output(mg_ctx* ctx, const mg_model* m, mg_dense* d, int32_t layer, 
  * cannot afford the device-wide synchronisation an allocation or a free implies.  mg_forward
  * grows its workspaces with cudaMalloc when a sample is larger than any before it; this entry
  * point never calls cudaMalloc, cudaFree or any allocating routine.  It computes the same H^k
- * with the same kernels, keeping the [self | mean] staging rows (first 4 MiB) and the
- * intermediate layer outputs H^1..H^{k-1} (remaining 12 MiB) in a scratch array of
- * MG_NOALLOC_SCRATCH_BYTES that is part of the library image.
+ * with the separate aggregation and GEMM kernels (mg_forward's default for MG_GEMM_TF32 is one
+ * fused kernel, so the two agree to the tensor-core tolerance there, not bit for bit), keeping
+ * the [self | mean] staging rows (first 4 MiB) and the intermediate layer outputs H^1..H^{k-1}
+ * (remaining 12 MiB) in a scratch array of MG_NOALLOC_SCRATCH_BYTES that is part of the library
+ * image.  The call is synchronous: it waits for the context's stream before it returns.
  *  - out_dev: DEVICE pointer, one row of dims[k] fp32 per target, as mg_forward writes it.
  *  - Limit: sum over l < k of rows(H^l) * dims[l] * 4 bytes must fit in 12 MiB; larger samples
  *    get MG_ERR_CAPACITY (nothing is launched) — use mg_forward or fewer mini-batches per call.
  *  - The first call on a device looks up the array's device address (cudaGetSymbolAddress);
- *    make that first call before any stream capture begins.
+ *    make that first call before any stream capture begins.  The CUDA runtime may also load
+ *    the kernels' code on their first launch, which is memory management of its own: a caller
+ *    that needs a steady state free of it makes one warm-up call per model shape first.
  *  - All calls in the process share the one array, and it keeps the previous call's contents.
  *    Nothing in it needs clearing (every value read was written earlier in the same call), but
  *    two calls that overlap on the GPU — from two contexts or two host threads — race on it:

@@ -29,7 +29,7 @@ CORRUPT_DST, CORRUPT_SRC, CORRUPT_BOTH = 1, 2, 3
 EXPORTS = [
     "mg_create", "mg_destroy", "mg_last_error", "mg_load_graph", "mg_load_out_graph", "mg_set_sample_direction", "mg_set_partitioning",
     "mg_load_features", "mg_set_resident", "mg_commit_resident", "mg_sample_many", "mg_sample_many_begin", "mg_sample_many_end", "mg_sample",
-    "mg_dense_counts", "mg_dense_view", "mg_dense_free", "mg_model_create", "mg_model_set_aggregator", "mg_model_free",
+    "mg_dense_counts", "mg_dense_view", "mg_dense_export_many", "mg_dense_export_view", "mg_dense_free", "mg_model_create", "mg_model_set_aggregator", "mg_model_free",
     "mg_forward", "mg_set_layer_window", "mg_keep_layer_outputs", "mg_forward_host_async", "mg_wait_output", "mg_forward_noalloc", "mg_gather_h0", "mg_layer_output", "mg_lp_prepare", "mg_lp_view", "mg_lp_free",
     "mg_distmult_score", "mg_kernel_launches", "mg_profile", "mg_profile_read", "mg_comet_plan", "mg_comet_bias", "mg_comet_autotune", "mg_gat_model_create", "mg_gat_model_free", "mg_gat_forward", "mg_backward", "mg_model_grads", "mg_model_sgd_step", "mg_model_adagrad_step", "mg_dense_packed_ids", "mg_apply_embedding_sgd",
 ]
@@ -171,6 +171,20 @@ class Dense:
     def view(self, batch: int = 0) -> DenseView:
         arr = DenseArrays()
         self.ctx._check(self.ctx.lib.mg_dense_view(self.ctx.handle, self.handle, C.c_int32(batch), C.byref(arr)))
+        dev = self.ctx.device
+        return DenseView(
+            _from_dev(arr.node_ids, arr.n_nodes, dev), _from_dev(arr.node_id_offsets, arr.k + 2, dev),
+            _from_dev(arr.nbrs, arr.n_entries, dev), _from_dev(arr.nbr_offsets, arr.n_sampled + 1, dev),
+            _from_dev(arr.repr_map, arr.n_entries, dev))
+
+    def export_many(self):
+        """Queue the export of every mini-batch into the paper's arrays (asynchronous, on the sampling stream)."""
+        self.ctx._check(self.ctx.lib.mg_dense_export_many(self.ctx.handle, self.handle))
+
+    def export_view(self, batch: int = 0) -> DenseView:
+        """Mini-batch `batch` of the last export_many (waits for it the first time)."""
+        arr = DenseArrays()
+        self.ctx._check(self.ctx.lib.mg_dense_export_view(self.ctx.handle, self.handle, C.c_int32(batch), C.byref(arr)))
         dev = self.ctx.device
         return DenseView(
             _from_dev(arr.node_ids, arr.n_nodes, dev), _from_dev(arr.node_id_offsets, arr.k + 2, dev),

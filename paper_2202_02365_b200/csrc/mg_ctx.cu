@@ -33,6 +33,15 @@ int mg_cuda_fail(mg_ctx* ctx, cudaError_t e, const char* what) {
     return mg_fail(ctx, code, "%s: %s", what, cudaGetErrorString(e));
 }
 
+int mg_check_sample_residency(mg_ctx* ctx, const mg_dense* d) {
+    if (d->resident_serial == ctx->resident_serial) return MG_OK;
+    const std::vector<int32_t>& then = d->slot_of_part_at_sample;
+    bool ok = then.size() == ctx->slot_of_part.size();
+    for (size_t p = 0; ok && p < then.size(); ++p) ok = then[p] < 0 || then[p] == ctx->slot_of_part[p];
+    if (ok) return MG_OK;
+    return mg_fail(ctx, MG_ERR_STATE, "the resident set changed since this sample was drawn: a partition it uses was evicted or moved; sample again");
+}
+
 void mg_prof_begin(mg_ctx* ctx, int phase) {
     if (!ctx->prof_on) return;
     cudaEvent_t a, b;
@@ -311,6 +320,7 @@ extern "C" int mg_profile_read(mg_ctx* c, int32_t* n_phases, const char** names,
 
 // upload the committed slot map and the resident-node prefix counts
 static int upload_slot_map(mg_ctx* c) {
+    ++c->resident_serial;   // every change of the committed slot map (or of the slots behind it) comes through here
     int32_t slots[MG_MAX_PARTS];
     int64_t prefix[MG_MAX_PARTS + 1];
     prefix[0] = 0;
@@ -669,7 +679,7 @@ extern "C" int mg_commit_resident(mg_ctx* c, int32_t timeout_ms) {
             if (q == cudaSuccess) break;
             if (q != cudaErrorNotReady) return mg_cuda_fail(c, q, "waiting for a partition copy");
             const auto ms = std::chrono::duration_cast<std::chrono::milliseconds>(std::chrono::steady_clock::now() - t0).count();
-            if (ms > timeout_ms) return mg_fail(c, MG_ERR_TIMEOUT, "partition copies still running after %d ms", timeout_ms);
+            if (ms >= timeout_ms) return mg_fail(c, MG_ERR_TIMEOUT, "partition copies still running after %d ms", timeout_ms);
             std::this_thread::sleep_for(std::chrono::microseconds(200));
         }
     }

@@ -388,7 +388,7 @@ static int forward_checks(mg_ctx* ctx, const mg_model* m, const mg_dense* d) {
     if (!ctx->slots || ctx->feat_dim <= 0) return mg_fail(ctx, MG_ERR_STATE, "no feature table loaded");
     if (m->k != d->k) return mg_fail(ctx, MG_ERR_STATE, "model has %d layers, sample has %d hops", m->k, d->k);
     if (m->dims[0] != ctx->feat_dim) return mg_fail(ctx, MG_ERR_STATE, "model input width %d != feature dim %d", m->dims[0], ctx->feat_dim);
-    return MG_OK;
+    return mg_check_sample_residency(ctx, d);
 }
 
 // rows of a layer are processed in chunks small enough for the [self | mean] staging matrix to
@@ -634,6 +634,7 @@ extern "C" int mg_gather_h0(mg_ctx* ctx, mg_dense* d, int32_t batch, float* out_
     if (!d->valid) return mg_fail(ctx, MG_ERR_STATE, "mg_dense holds no completed sample");
     if (!ctx->slots || ctx->feat_dim <= 0) return mg_fail(ctx, MG_ERR_STATE, "no feature table loaded");
     if (batch < 0 || batch >= d->n_batches) return mg_fail(ctx, MG_ERR_ARG, "batch out of range");
+    if (int rs = mg_check_sample_residency(ctx, d)) return rs;
     MG_CUDA(ctx, cudaSetDevice(ctx->device));
     H0Args a;
     fill_row_export(d, batch, 0, ctx->feat_dim, &a.r);
@@ -1149,6 +1150,7 @@ extern "C" int mg_apply_embedding_sgd(mg_ctx* ctx, mg_dense* d, const float* d_h
     if (d->ctx != ctx) return mg_fail(ctx, MG_ERR_ARG, "handle belongs to another context");
     if (!ctx->slots || ctx->feat_dim <= 0) return mg_fail(ctx, MG_ERR_STATE, "no feature table loaded");
     if (ctx->feat_dtype != MG_DTYPE_F32) return mg_fail(ctx, MG_ERR_ARG, "base representations are updated in fp32 tables only");
+    if (int rs = mg_check_sample_residency(ctx, d)) return rs;
     MG_CUDA(ctx, cudaSetDevice(ctx->device));
     EmbSgdArgs a{{d->n_batches, d->k, d->rowbase, d->cum, d->node_off}, d->nodes, d_h0_dev, d->h_hdr.rows_total[0], ctx->slots,
                  ctx->d_slot_of_part, ctx->slot_bytes, ctx->row_bytes, (uint32_t)ctx->part_size, ctx->feat_dim, lr};

@@ -315,6 +315,7 @@ extern "C" int mg_gat_forward(mg_ctx* ctx, const mg_gat_model* m, mg_dense* d, f
     if (!ctx->slots || ctx->feat_dim <= 0) return mg_fail(ctx, MG_ERR_STATE, "no feature table loaded");
     if (m->k != d->k) return mg_fail(ctx, MG_ERR_STATE, "model has %d layers, sample has %d hops", m->k, d->k);
     if (m->dims[0] != ctx->feat_dim) return mg_fail(ctx, MG_ERR_STATE, "model input width %d != feature dim %d", m->dims[0], ctx->feat_dim);
+    if (int rs = mg_check_sample_residency(ctx, d)) return rs;
     MG_CUDA(ctx, cudaSetDevice(ctx->device));
     const int k = d->k, B = d->n_batches;
     cudaStream_t st = ctx->stream;

@@ -92,6 +92,7 @@ struct mg_ctx {
     int32_t capacity = 1;
     std::vector<int32_t> slot_of_part;  // committed; -1 = not resident
     std::vector<int32_t> pending_slot;  // after set_resident, before commit
+    uint64_t resident_serial = 0;       // bumped whenever the committed slot map or the slots themselves change
     bool has_pending = false;
     std::vector<cudaEvent_t> pending_events;
     std::vector<char> dirty_part;       // host backing: the partition's slot was updated (mg_apply_embedding_sgd) and not written back yet
@@ -203,6 +204,14 @@ struct mg_dense {
     std::vector<int32_t> h_ent_hop;  // [k * (B+1)] arena entry index where batch b's hop-h entries start
     int32_t* d_ent_hop = nullptr;    // device copy of the same
     bool valid = false;
+    // the slot map the sample was drawn under: its feature rows are addressed through it, so a later call may only
+    // use the sample while every partition resident then still sits in the same slot
+    uint64_t resident_serial = 0;
+    std::vector<int32_t> slot_of_part_at_sample;
+    // export of all mini-batches at once (mg_dense_export_many): one buffer, laid out by export_layout()
+    int32_t* expm_buf = nullptr; size_t expm_elems = 0;
+    cudaEvent_t ev_exported = nullptr;
+    bool export_valid = false, export_pending = false;
     int32_t* perm_buf = nullptr; size_t perm_elems = 0;   // perm | inv of mini-batch perm_batch (mg_dense_batch_perm)
     int perm_batch = -1;
     uint32_t* batch_cnt = nullptr;   // [k][B] new nodes per hop and mini-batch
@@ -256,6 +265,9 @@ struct mg_lp_batch {
 // host helpers
 // ---------------------------------------------------------------------------------------
 int mg_fail(mg_ctx* ctx, int code, const char* fmt, ...);
+// MG_OK when the partitions that were resident while `d` was sampled are still resident in the same slots (the
+// sample's feature rows are then where its ids say); MG_ERR_STATE otherwise.  Host-side check, no device work.
+int mg_check_sample_residency(mg_ctx* ctx, const mg_dense* d);
 int mg_cuda_fail(mg_ctx* ctx, cudaError_t e, const char* what);
 
 #define MG_CUDA(ctx, call)                                      \

@@ -1080,6 +1080,88 @@ __global__ void __launch_bounds__(kThreads) k_export_entries(ExportArgs a) {
     }
 }
 
+// -------------------------------------------------------------------------------------
+// export of every mini-batch at once (mg_dense_export_many): the canonical DENSE ordering for the whole sample
+// -------------------------------------------------------------------------------------
+// One sort orders all nodes of the sample by (mini-batch, delta, id); a node's position in that order is its row in
+// the packed canonical node list (mini-batch after mini-batch, each [Delta_0 .. Delta_k]).  Targets keep the caller's
+// order: their "id" field is their position.
+struct ExportManyArgs {
+    int32_t B, k, n_nodes_total, pay_bits, id_bits;
+    int32_t hop_base[MG_MAX_HOPS + 2];
+    const int32_t *nodes, *node_batch, *node_off, *cum, *rowbase0, *ent_off, *ent_nbrs, *ent_repr;
+    int32_t *o_node_ids, *o_nio, *o_nbrs, *o_repr, *o_nbr_off, *inv;
+    uint32_t* cnt;   // per canonical row: entry count, then (scanned) its first entry in the packed entry list
+};
+
+__device__ __forceinline__ int hop_of_arena(const ExportManyArgs& a, int32_t i) {
+    int h = 0;
+    while (h < a.k && i >= a.hop_base[h + 1]) ++h;
+    return h;
+}
+
+__global__ void k_export_params(SortParams* sp, int32_t* range, int32_t n) {
+    sp->zero = 0; sp->n = n; sp->ntiles = (n + kSortTile - 1) / kSortTile; sp->hist_len = kBins * sp->ntiles;
+    range[0] = 0; range[1] = n;
+}
+
+__global__ void __launch_bounds__(kThreads) k_export_keys(ExportManyArgs a, uint64_t* keys) {
+    for (int32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < a.n_nodes_total; i += gridDim.x * blockDim.x) {
+        const int h = hop_of_arena(a, i);
+        const int32_t b = a.node_batch[i];
+        const uint32_t id = h == 0 ? (uint32_t)(i - a.node_off[b]) : (uint32_t)a.nodes[i];
+        const uint64_t seg = (uint64_t)b * (a.k + 1) + (uint64_t)(a.k - h);
+        keys[i] = (seg << (a.id_bits + a.pay_bits)) | ((uint64_t)id << a.pay_bits) | (uint64_t)(uint32_t)i;
+    }
+    // node_id_offsets of every mini-batch
+    for (int32_t t = blockIdx.x * blockDim.x + threadIdx.x; t < a.B; t += gridDim.x * blockDim.x) {
+        const int32_t* cum = a.cum + (int64_t)t * (a.k + 2);
+        int32_t run = 0;
+        a.o_nio[(int64_t)t * (a.k + 2)] = 0;
+        a.o_nbr_off[a.rowbase0[t] + t] = 0;   // (an empty mini-batch has this terminal entry only)
+        for (int j = 0; j <= a.k; ++j) { run += cum[a.k - j + 1] - cum[a.k - j]; a.o_nio[(int64_t)t * (a.k + 2) + j + 1] = run; }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads) k_export_place(ExportManyArgs a, const uint64_t* __restrict__ sorted) {
+    const uint64_t pay_mask = (1ull << a.pay_bits) - 1ull;
+    for (int32_t c = blockIdx.x * blockDim.x + threadIdx.x; c < a.n_nodes_total; c += gridDim.x * blockDim.x) {
+        const int32_t i = (int32_t)(sorted[c] & pay_mask);
+        a.inv[i] = c;
+        a.o_node_ids[c] = a.nodes[i];
+        a.cnt[c] = i < a.hop_base[a.k] ? (uint32_t)(a.ent_off[i + 1] - a.ent_off[i]) : 0u;   // the farthest delta has no entries
+    }
+}
+
+// 8 lanes per sampled node: its entries go to their place in the packed canonical entry list, neighbours translated to
+// canonical rows of the mini-batch; the node's offset (relative to its mini-batch) goes to nbr_offsets
+__global__ void __launch_bounds__(kThreads) k_export_many_entries(ExportManyArgs a) {
+    const int gl = threadIdx.x & 7;
+    const int32_t n_sampled = a.hop_base[a.k];
+    for (int32_t i = (blockIdx.x * blockDim.x + threadIdx.x) >> 3; i < n_sampled; i += (gridDim.x * blockDim.x) >> 3) {
+        const int32_t b = a.node_batch[i];
+        const int32_t c = a.inv[i];
+        const int32_t row0 = a.rowbase0[b];                        // first packed row of the mini-batch
+        const int32_t* cum = a.cum + (int64_t)b * (a.k + 2);
+        const int32_t n0 = cum[a.k + 1] - cum[a.k];                // |Delta_0|
+        const uint32_t o0 = a.cnt[c], batch_e0 = a.cnt[row0];
+        const int32_t e0 = a.ent_off[i], n = a.ent_off[i + 1] - e0;
+        if (gl == 0) {
+            int32_t* off = a.o_nbr_off + row0 + b;                 // the mini-batch's nbr_offsets: |sampled| + 1 entries
+            off[c - row0 - n0] = (int32_t)(o0 - batch_e0);
+            if (c + 1 == a.rowbase0[b + 1]) off[c + 1 - row0 - n0] = (int32_t)(o0 - batch_e0) + n;   // terminal entry
+        }
+        for (int32_t j = gl; j < n; j += 8) {
+            const int32_t l = a.ent_repr[e0 + j];                  // the neighbour's local row in the mini-batch
+            int h = 0;
+            while (h < a.k && l >= cum[h + 1]) ++h;
+            const int32_t ai = a.node_off[h * (a.B + 1) + b] + (l - cum[h]);
+            a.o_nbrs[o0 + j] = a.ent_nbrs[e0 + j];
+            a.o_repr[o0 + j] = a.inv[ai] - row0;
+        }
+    }
+}
+
 int ilog2_ceil(int64_t x) {
     int b = 0;
     while (((int64_t)1 << b) < x) ++b;
@@ -1377,12 +1459,15 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
     else if (d->ctx != ctx) return mg_fail(ctx, MG_ERR_ARG, "mg_dense belongs to another context");
     d->valid = false;
     d->pending = false;
+    d->export_valid = false;
     if (d->ev_read_done) MG_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, d->ev_read_done, 0));
     int rc = dense_alloc(ctx, d, n_batches, k, cap_nodes, std::max<int64_t>(cap_entries, 1), table_size, smem_last ? (int32_t)dedup_nb : 0);
     if (rc) { if (created) mg_dense_free(d); return rc; }
     *out = d;
     for (int h = 0; h < k; ++h) d->fanouts[h] = fanouts[h];
     d->n_targets_total = T;
+    d->resident_serial = ctx->resident_serial;
+    d->slot_of_part_at_sample = ctx->slot_of_part;
 
     cudaStream_t st = ctx->stream;
     const int B = n_batches;
@@ -1634,6 +1719,7 @@ int mg_dense_batch_perm(mg_ctx* ctx, mg_dense* d, int b, const int32_t** perm, c
     if (d->perm_batch == b) return MG_OK;
     d->perm_batch = -1;
     cudaStream_t st = ctx->stream;
+    if (d->export_pending) MG_CUDA(ctx, cudaStreamWaitEvent(st, d->ev_exported, 0));   // the export uses the same sort scratch
     const int32_t n = g.V - g.n_targets;
     const int id_bits = std::max(1, ilog2_ceil(ctx->n_nodes)), hop_bits = std::max(1, ilog2_ceil(g.k + 1));
     const int grid = std::max(1, std::min(mg_grid(ctx, 4), (g.V + kThreads - 1) / kThreads));
@@ -1704,6 +1790,109 @@ extern "C" int mg_dense_view(mg_ctx* ctx, mg_dense* d, int32_t batch, mg_dense_a
     return MG_OK;
 }
 
+// Layout of the export buffer (int32 elements), from the sample's capacities so that it is allocated once per handle.
+struct ExportLayout { size_t node_ids, nio, nbrs, repr, nbr_off, inv, cnt, total; };
+static ExportLayout export_layout(const mg_dense* d) {
+    ExportLayout L;
+    const size_t cn = (size_t)d->cap_nodes, ce = (size_t)d->cap_entries, B = (size_t)d->n_batches;
+    size_t at = 0;
+    L.node_ids = at; at += cn;
+    L.nio = at; at += B * (MG_MAX_HOPS + 2);
+    L.nbrs = at; at += ce;
+    L.repr = at; at += ce;
+    L.nbr_off = at; at += cn + B + 1;
+    L.inv = at; at += cn;
+    L.cnt = at; at += cn + 1;
+    L.total = at + 16;
+    return L;
+}
+
+extern "C" int mg_dense_export_many(mg_ctx* ctx, mg_dense* d) {
+    if (!ctx) return MG_ERR_ARG;
+    if (!d) return mg_fail(ctx, MG_ERR_ARG, "null mg_dense");
+    if (d->ctx != ctx) return mg_fail(ctx, MG_ERR_ARG, "mg_dense belongs to another context");
+    if (d->pending) return mg_fail(ctx, MG_ERR_STATE, "a sample is in flight on this mg_dense: call mg_sample_many_end first");
+    if (!d->valid) return mg_fail(ctx, MG_ERR_STATE, "mg_dense holds no completed sample");
+    MG_CUDA(ctx, cudaSetDevice(ctx->device));
+    const int k = d->k, B = d->n_batches;
+    const int32_t n_total = d->h_hdr.hop_base[k + 1];
+    const int id_bits = std::max({1, ilog2_ceil(ctx->n_nodes), ilog2_ceil(d->n_targets_total + 1)});
+    const int pay_bits = std::max(1, ilog2_ceil((int64_t)n_total + 1));
+    const int seg_bits = std::max(1, ilog2_ceil((int64_t)B * (k + 1)));
+    if (id_bits + pay_bits + seg_bits > 64)
+        return mg_fail(ctx, MG_ERR_CAPACITY, "sample too large for a one-pass export (%d key bits): export fewer mini-batches per sample", id_bits + pay_bits + seg_bits);
+    const ExportLayout L = export_layout(d);
+    int rc = mg_ensure(ctx, &d->expm_buf, &d->expm_elems, L.total);
+    if (rc) return rc;
+    if (!d->ev_exported) MG_CUDA(ctx, cudaEventCreateWithFlags(&d->ev_exported, cudaEventDisableTiming));
+    // on the sampling stream: behind the sample (and a later sample into d behind this), beside the layers
+    cudaStream_t user = ctx->stream;
+    cudaStream_t st = ctx->sample_stream;
+    ExportManyArgs a;
+    memset(&a, 0, sizeof(a));
+    a.B = B; a.k = k; a.n_nodes_total = n_total; a.pay_bits = pay_bits; a.id_bits = id_bits;
+    for (int h = 0; h <= k + 1; ++h) a.hop_base[h] = d->h_hdr.hop_base[h];
+    a.nodes = d->nodes; a.node_batch = d->node_batch; a.node_off = d->node_off; a.cum = d->cum; a.rowbase0 = d->rowbase;
+    a.ent_off = d->ent_off; a.ent_nbrs = d->ent_nbrs; a.ent_repr = d->ent_repr;
+    a.o_node_ids = d->expm_buf + L.node_ids; a.o_nio = d->expm_buf + L.nio; a.o_nbrs = d->expm_buf + L.nbrs;
+    a.o_repr = d->expm_buf + L.repr; a.o_nbr_off = d->expm_buf + L.nbr_off; a.inv = d->expm_buf + L.inv;
+    a.cnt = reinterpret_cast<uint32_t*>(d->expm_buf + L.cnt);
+    d->export_valid = false;
+    if (n_total > 0) {
+        SortParams* sp = (SortParams*)(d->scan_tmp + d->scan_tmp_elems - 8);
+        int32_t* range = d->scan_tmp + d->scan_tmp_elems - 12;
+        const int grid = mg_grid(ctx, 8);
+        ctx->stream = st;   // the sort and scan helpers (and the phase events) use ctx->stream
+        {
+        ProfScope ps(ctx, PH_SAMPLE_SORT, 0);
+        k_export_params<<<1, 1, 0, st>>>(sp, range, n_total);
+        k_export_keys<<<grid, kThreads, 0, st>>>(a, d->newlist[0]);
+        int res = 0;
+        mg_sort_u64(ctx, d->newlist, sp, pay_bits, id_bits + seg_bits, d->sort_hist, (uint32_t*)d->scan_tmp, &res);
+        k_export_place<<<grid, kThreads, 0, st>>>(a, d->newlist[res]);
+        mg_scan_u32(ctx, a.cnt, &range[0], &range[1], nullptr, (uint32_t*)d->scan_tmp, nullptr);
+        k_export_many_entries<<<grid, kThreads, 0, st>>>(a);
+        }
+        ctx->stream = user;
+        ctx->launches += 4;
+    }
+    MG_CUDA(ctx, cudaGetLastError());
+    MG_CUDA(ctx, cudaEventRecord(d->ev_exported, st));
+    d->export_pending = true;
+    d->export_valid = true;
+    d->perm_batch = -1;   // the per-batch permutation shares the sort scratch
+    return MG_OK;
+}
+
+extern "C" int mg_dense_export_view(mg_ctx* ctx, mg_dense* d, int32_t batch, mg_dense_arrays* out) {
+    if (!ctx) return MG_ERR_ARG;
+    if (!d || !out) return mg_fail(ctx, MG_ERR_ARG, "null argument");
+    if (!d->valid || !d->export_valid) return mg_fail(ctx, MG_ERR_STATE, "no export of this sample: call mg_dense_export_many first");
+    if (batch < 0 || batch >= d->n_batches) return mg_fail(ctx, MG_ERR_ARG, "batch out of range");
+    MG_CUDA(ctx, cudaSetDevice(ctx->device));
+    if (d->export_pending) { MG_CUDA(ctx, cudaEventSynchronize(d->ev_exported)); d->export_pending = false; }
+    const int k = d->k, B = d->n_batches, b = batch;
+    const ExportLayout L = export_layout(d);
+    const int32_t row0 = d->h_rowbase[b], V = d->h_rowbase[b + 1] - row0;
+    const int32_t n0 = d->h_cum[(size_t)b * (k + 2) + k + 1] - d->h_cum[(size_t)b * (k + 2) + k];
+    int64_t e_before = 0, e_mine = 0;
+    for (int h = 0; h < k; ++h) {
+        // entries are packed mini-batch after mini-batch in the export
+        for (int bb = 0; bb < b; ++bb) e_before += d->h_ent_hop[(size_t)h * (B + 1) + bb + 1] - d->h_ent_hop[(size_t)h * (B + 1) + bb];
+        e_mine += d->h_ent_hop[(size_t)h * (B + 1) + b + 1] - d->h_ent_hop[(size_t)h * (B + 1) + b];
+    }
+    out->k = k;
+    out->n_nodes = V;
+    out->n_sampled = V - n0;
+    out->n_entries = (int32_t)e_mine;
+    out->node_ids = d->expm_buf + L.node_ids + row0;
+    out->node_id_offsets = d->expm_buf + L.nio + (size_t)b * (k + 2);
+    out->nbrs = d->expm_buf + L.nbrs + e_before;
+    out->repr_map = d->expm_buf + L.repr + e_before;
+    out->nbr_offsets = d->expm_buf + L.nbr_off + row0 + b;
+    return MG_OK;
+}
+
 extern "C" int mg_dense_free(mg_dense* d) {
     if (!d) return MG_OK;
     cudaSetDevice(d->device);
@@ -1712,7 +1901,8 @@ extern "C" int mg_dense_free(mg_dense* d) {
     cudaFree(d->ent_nbrs); cudaFree(d->ent_repr); cudaFree(d->node_off); cudaFree(d->cum);
     cudaFree(d->rowbase); cudaFree(d->hkeys); cudaFree(d->hvals); cudaFree(d->newlist[0]);
     cudaFree(d->newlist[1]); cudaFree(d->d_seeds); cudaFree(d->batch_cnt); cudaFree(d->scan_tmp); cudaFree(d->sort_hist);
-    cudaFree(d->exp_buf); cudaFree(d->perm_buf); cudaFree(d->d_ent_hop);
+    cudaFree(d->exp_buf); cudaFree(d->perm_buf); cudaFree(d->d_ent_hop); cudaFree(d->expm_buf);
+    if (d->ev_exported) cudaEventDestroy(d->ev_exported);
     if (d->h_pinned) cudaFreeHost(d->h_pinned);
     if (d->h_stage) cudaFreeHost(d->h_stage);
     if (d->graph_exec) cudaGraphExecDestroy(d->graph_exec);

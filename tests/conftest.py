@@ -24,3 +24,24 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+# Worst element-wise relative error |got - ref| / |ref| seen by the parity tests, per tolerance class, over the
+# elements that are not small (|ref| > rms(ref) / 100); the tests' own bound is |got - ref| <= rtol * max(|ref|, rms).
+PARITY_WORST = {}
+
+
+def note_relative_error(rtol, worst_rel, worst_vs_bound):
+    cur = PARITY_WORST.setdefault(rtol, [0.0, 0.0, 0])
+    cur[0] = max(cur[0], worst_rel)
+    cur[1] = max(cur[1], worst_vs_bound)
+    cur[2] += 1
+
+
+def pytest_terminal_summary(terminalreporter):
+    if not PARITY_WORST:
+        return
+    terminalreporter.write_line("parity: worst errors per tolerance class (comparisons; error / bound; pure relative error where |ref| > rms/100)")
+    for rtol in sorted(PARITY_WORST):
+        rel, vs_bound, count = PARITY_WORST[rtol]
+        terminalreporter.write_line(f"  rtol {rtol:g}: {count} comparisons, worst {vs_bound:.3f} x the bound, worst relative error {rel:.3g}")
