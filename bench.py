@@ -42,6 +42,10 @@ CONFIGS = {
     "table6_papers100m_shaped_3layers": dict(n=111_000_000, m=1_620_000_000, kind="rmat", dim=128, hidden=256,
                                              fanouts=[10, 10, 10], batch=1000, parts=16, train=1_100_000, inout=True,
                                              group=8),
+    # a case small enough for ncu's counter passes whose feature table (4 GB) is still far larger than L2: the fused
+    # layer-1 kernel's DRAM traffic per unit is captured here (profiles/k_sage_layer_fused_dram_traffic.md)
+    "probe_rmat_8m_dim128": dict(n=8_000_000, m=160_000_000, kind="rmat", dim=128, hidden=256, fanouts=[15, 10, 5],
+                                 batch=1000, parts=1, train=8_000_000),
     # config 4's shapes at a tenth of its node count, whole fp16 table in HBM (no swaps): a throughput probe of the
     # wide fp16 layer-1 path, not the out-of-core configuration itself (that one is exercised by the tests)
     "config4_tenth_fp16_768_in_hbm": dict(n=12_200_000, m=130_000_000, kind="rmat", dim=768, hidden=256,
@@ -51,11 +55,31 @@ CONFIGS = {
 LP_CONFIG = dict(n=86_000_000, m=338_000_000, dim=100, n_rel=14_824, parts=16, resident=8, edges=50_000, chunks=10,
                  negs=1000, fanout=20)
 LP_WORKLOAD = "config5_freebase86m_shaped_lp"
+# config 4 (Mag240M-Cites-shaped) out of core, measured by run_out_of_core: fp16 x 768 features in 32 partition blocks of
+# 5.86 GB, a 10-partition HBM buffer, one block swapped in from pinned host memory per buffer state (side stream) while
+# mini-batches run on the current state; the 187 GB table is never held: a block is a pure function of (seed, block)
+OOC_CONFIG = dict(n=122_000_000, m=1_300_000_000, dim=768, hidden=256, fanouts=[15, 10, 5], batch=1000, parts=32, cap=10,
+                  group=128, steps_per_state=25)
+OOC_WORKLOAD = "config4_mag240m_shaped_out_of_core"
 DEFAULT_WORKLOAD = "config3_papers100m_shaped"
 HBM_NOMINAL_GBS = 8000.0
-# dram bytes (read + write) of one launch of the dominant kernel, measured with ncu (see profiles/)
-NCU_TRAFFIC_PER_LAUNCH = {("config3_papers100m_shaped", 128): 10.87e9,
-                          ("config3_papers100m_shaped_inout", 16): 7.57e9}
+# DRAM traffic of the dominant kernel (fused layer 1) comes from a tracked ncu summary, not from a constant here: the
+# summary gives, for a capture small enough for ncu's counter passes, DRAM bytes read per algorithmic byte and DRAM
+# bytes written per output row; both scale with the units a launch processes
+TRAFFIC_PROFILE = os.path.join(ROOT, "profiles", "k_sage_layer_fused_dram_traffic.md")
+
+
+def traffic_model():
+    """(dram read bytes per algorithmic byte, dram write bytes per output row, source) from the tracked summary."""
+    import re
+    try:
+        text = open(TRAFFIC_PROFILE).read()
+        r = re.search(r"dram_read_bytes_per_algorithmic_byte\s*[:=]\s*([0-9.]+)", text)
+        w = re.search(r"dram_write_bytes_per_output_row\s*[:=]\s*([0-9.]+)", text)
+        c = re.search(r"captured_at_commit\s*[:=]\s*([0-9a-f]+)", text)
+        return float(r.group(1)), float(w.group(1)), f"profiles/k_sage_layer_fused_dram_traffic.md @ {c.group(1) if c else '?'}"
+    except Exception:
+        return None
 
 
 def measured_peaks():
@@ -212,13 +236,15 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="mgdense", choices=["mgdense", "reference"])
-    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(CONFIGS) + [LP_WORKLOAD])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(CONFIGS) + [LP_WORKLOAD, OOC_WORKLOAD])
     ap.add_argument("--group", type=int, default=0, help="mini-batches per step (default: 128, or the workload's own)")
     ap.add_argument("--window", type=int, default=0, help="mini-batches per window of the layer schedule (0 = whole layers)")
     ap.add_argument("--lp-model", default="graphsage", choices=["graphsage", "gat"],
                     help="link-prediction workload only: the encoder layer (GraphSage mean or single-head graph attention)")
     ap.add_argument("--backward", action="store_true",
                     help="also time mg_backward (with base-representation gradients) on one group of mini-batches")
+    ap.add_argument("--steps-per-state", type=int, default=0,
+                    help="out-of-core workload only: steps run on one buffer state while the next state's block loads")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=20.0)
     args = ap.parse_args()
@@ -228,6 +254,13 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     peaks = measured_peaks()
+    if args.workload == OOC_WORKLOAD:
+        if args.impl == "reference":
+            if rank == 0:
+                print(json.dumps({"impl": "reference", "unavailable": "the reference arm times the oracle on the default workload only"}))
+            return
+        run_out_of_core(args, peaks, rank, local_rank, world)
+        return
     if args.workload == LP_WORKLOAD:
         if args.impl == "reference":
             if rank == 0:
@@ -273,6 +306,7 @@ def main():
     else:
         ctx.load_features(feats)
     model = ctx.model(layers, mg.GEMM_TF32)
+    dims_model = [cfg["dim"]] + [cfg["hidden"]] * len(cfg["fanouts"])
     ctx.set_layer_window(args.window)
 
     G, T, k = (args.group or cfg.get("group", 128)), cfg["batch"], len(cfg["fanouts"])
@@ -371,6 +405,30 @@ def main():
     barrier()
     ms_export = ev4.elapsed_time(ev5)
 
+    # ---- the same steps with the intermediate layer outputs kept as fp16 (a model option; the headline keeps fp32) ----
+    ms_f16 = None
+    if all(w % 128 == 0 for w in dims_model[1:-1]) and k > 1:
+        model16 = ctx.model(layers, mg.GEMM_TF32)
+        model16.set_intermediates(torch.float16)
+        model_main, model = model, model16
+        for i in range(3):
+            run_steps(i, 1, False)
+        barrier()
+        ev6, ev7 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev6.record()
+        run_steps(args.warmup, args.steps, False)
+        ev7.record()
+        barrier()
+        ms_f16 = ev6.elapsed_time(ev7)
+        ctx.profile(True)
+        ctx.profile_read(reset=True)
+        for s_ in range(min(args.steps, 8)):
+            run_step(args.warmup + s_, False)
+        phases16 = ctx.profile_read(reset=True)
+        ctx.profile(False)
+        phases16 = {name: round(v["ms"] / min(args.steps, 8), 4) for name, v in phases16.items() if v["launches"] and name.startswith("aggregate")}
+        model = model_main
+
     # ---- the same steps again with per-phase CUDA events on the library's stream ---------------
     ctx.profile(True)
     ctx.profile_read(reset=True)
@@ -453,9 +511,16 @@ def main():
                 "peak": peaks["hbm_gbs"], "unit": "GB/s", "bytes_per_launch": alg["agg_l1"] / n_l1,
                 "ms_per_launch": agg1["ms"] / n_l1, "launches": agg1["launches"], "peak_source": peaks["source"]}
     roofline["frac"] = roofline["achieved"] / roofline["peak"] if roofline["achieved"] else None
-    # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the single-pass ncu capture of this very
-    # command (profiles/): only known for the default workload and group size
-    roofline["traffic"] = NCU_TRAFFIC_PER_LAUNCH.get((args.workload, G))
+    # dram__bytes_read.sum + dram__bytes_write.sum per launch: the ncu capture of a smaller case of the same kernel
+    # (feature table of a few GB, far above L2), scaled by the units this launch processes (fp32 x 128 features only)
+    rows_out_l1 = float(nodes[:, :k].sum()) / n_l1
+    roofline["rows_out_per_launch"] = rows_out_l1
+    tm = traffic_model()
+    if tm and cfg["dim"] == 128 and not cfg.get("fp16"):
+        roofline["traffic"] = tm[0] * roofline["bytes_per_launch"] + tm[1] * rows_out_l1
+        roofline["traffic_source"] = tm[2]
+    else:
+        roofline["traffic"] = None
     flops_l1 = alg["flops_l1"]
     tensor = {"what": "layer GEMM work inside the fused kernels (all layers)", "bound": "tensor",
               "achieved": alg["flops"] / ((agg1["ms"] + rest["ms"] + gemm["ms"]) / 1e3) / 1e12, "peak": tf32_peak,
@@ -480,6 +545,11 @@ def main():
         "value_with_canonical_export": n_batches / (ms_export / 1e3),
         "ms_per_step_with_canonical_export": ms_export / args.steps,
         "export_ms_per_step": export_ms / args.steps,
+        # the same steps with H^1 .. H^{k-1} stored as fp16 (mg_model_set_intermediates; the same 10-bit mantissa the
+        # TF32 layers round their inputs to): half the bytes and half the row requests between the layers
+        "value_fp16_intermediates": (n_batches / (ms_f16 / 1e3)) if ms_f16 else None,
+        "ms_per_step_fp16_intermediates": (ms_f16 / args.steps) if ms_f16 else None,
+        "layer_phases_ms_per_step_fp16_intermediates": phases16 if ms_f16 else None,
         "per_batch": {"nodes": float(nodes.sum(1).mean()), "sampled_edges": float(ents.sum(1).mean()),
                       "algorithmic_bytes": alg["a_min"] / (args.steps * G),
                       "gemm_flops": alg["flops"] / (args.steps * G)},
@@ -508,6 +578,225 @@ def main():
     if world > 1:
         dist.destroy_process_group()
 
+
+
+def run_out_of_core(args, peaks, rank, local_rank, world):
+    """Config 4 as stated: R-MAT 122M nodes / 1.30B edges, fp16 features of width 768, 32 partitions, a 10-partition
+    buffer in HBM.  Buffer states follow the random one-swap order (Section 5.2's fallback); while the mini-batches of
+    a state run (sampling restricted to resident endpoints, three fused layers), the next state's incoming block is
+    copied from a pinned host block on the side stream, then committed (slot map + in-buffer view of the graph).
+    The timed region of a state = queueing the swap, its steps, and the commit; the incoming block is made in host
+    memory before the region starts (it stands in for the table that is already there)."""
+    import paper_2202_02365_b200 as mg
+    c = OOC_CONFIG
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    t0 = time.time()
+    g = inputs.rmat_graph(c["n"], c["m"], seed=40, device=device)
+    n_edges = g.n_edges
+    ctx = mg.Context(local_rank)
+    ctx.load_graph(g.row_offsets, g.nbrs)
+    del g
+    torch.cuda.empty_cache()
+    P, cap, dim, T, k = c["parts"], c["cap"], c["dim"], c["batch"], len(c["fanouts"])
+    G = args.group or c["group"]
+    S = args.steps_per_state or c["steps_per_state"]
+    ctx.set_partitioning(P)
+    ctx.load_features(None, capacity_parts=cap, backing=mg.BACKING_HOST, dtype=torch.float16, dim=dim)
+    part_rows = inputs.contiguous_partition(c["n"], P)
+    rows_of = lambda p: min(part_rows, c["n"] - p * part_rows)
+    staging = [torch.empty((part_rows, dim), dtype=torch.float16).pin_memory() for _ in range(2)]
+    feat_seed = 41 + 1000 * rank
+
+    def stage(p, slot):
+        inputs.block_features(rows_of(p), dim, feat_seed, p, device=device, dtype=torch.float16, out=staging[slot][:rows_of(p)])
+        torch.cuda.synchronize()
+        return staging[slot]
+
+    states = inputs.swap_order(P, cap, seed=44 + rank)
+    for i, p in enumerate(states[0]):                # fill the buffer, one block at a time through one staging block
+        ctx.set_partition_source(p, stage(p, 0))
+        ctx.set_resident(sorted(states[0][:i + 1]))
+    layers = inputs.glorot_layers([dim] + [c["hidden"]] * k, seed=43)
+    model = ctx.model(layers, mg.GEMM_TF32)
+    setup_s = round(time.time() - t0, 1)
+    offs = torch.arange(0, G + 1, dtype=torch.int64) * T
+    n_states = max(1, min(len(states) - 1, (args.warmup + args.steps + S - 1) // S + 1))
+
+    def state_targets(state, n_steps, seed):
+        mask = inputs.resident_node_mask(c["n"], P, state, device=device)
+        pool = torch.nonzero(mask).flatten().to(torch.int32)
+        gen = torch.Generator(device=device); gen.manual_seed(seed)
+        pick = torch.randperm(pool.numel(), generator=gen, device=device)[:n_steps * G * T]
+        return pool[pick].reshape(n_steps, G * T).contiguous()
+
+    tg0 = state_targets(states[0], 1, 7)
+    seeds0 = [(rank << 40) + b for b in range(G)]
+    probe = ctx.sample_many(tg0[0], offs, c["fanouts"], seeds0, caps={"max_nodes_per_batch": 1 << 19})
+    nodes, ents = probe.counts()
+    caps = {"max_nodes_total": int(nodes.sum() * 1.4) + 1024, "max_entries_total": int(ents.sum() * 1.4) + 1024,
+            "max_nodes_per_batch": int(nodes.sum(1).max() * 1.6) + 64}
+    probe.free()
+    denses = [ctx.sample_many(tg0[0], offs, c["fanouts"], seeds0, caps=caps) for _ in range(3)]
+    out_dev = torch.empty((G * T, c["hidden"]), dtype=torch.float32, device=device)
+    out_hosts = [torch.empty((G * T, c["hidden"]), dtype=torch.float32).pin_memory() for _ in range(2)]
+
+    def run_steps(tg, base_seed, e2e):
+        """tg: one row of G x T targets per step (device rows, or pinned host rows with e2e)"""
+        n = len(tg)
+        src = list(tg)
+        seeds = lambda i: [(rank << 40) + base_seed + i * G + b for b in range(G)]
+        begin = lambda i: ctx.sample_many_begin(src[i], offs, c["fanouts"], seeds(i), caps=caps, out=denses[i % 3])
+        begin(0)
+        if n > 1:
+            begin(1)
+        for i in range(n):
+            ctx.sample_many_end(denses[i % 3])
+            if i + 2 < n:
+                begin(i + 2)
+            if e2e:
+                ctx.forward_host_async(model, denses[i % 3], out_hosts[i & 1])
+            else:
+                ctx.forward(model, denses[i % 3], out_dev)
+        if e2e:
+            ctx.wait_output()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+
+    # a swap with nothing else running, and a commit whose copies have long finished (slot map + view rebuild alone)
+    incoming = lambda s: [p for p in states[s + 1] if p not in states[s]][0]
+    swap_alone_ms = rebuild_alone_ms = None
+    cur = 0
+    run_steps(state_targets(states[0], max(args.warmup, 3), 8), 1 << 20, False)       # warm-up steps
+    ctx.set_partition_source(incoming(0), stage(incoming(0), 1))
+    barrier()
+    t1 = time.perf_counter()
+    ctx.set_resident(states[1], async_=True)
+    ctx.commit_resident(120_000)
+    torch.cuda.synchronize()
+    swap_and_rebuild_ms = (time.perf_counter() - t1) * 1e3
+    cur = 1
+    # timed states
+    sampler = ClockSampler(local_rank)
+    launches0 = ctx.kernel_launches()
+    seg_ms, commit_ms, done_steps, stats = [], [], 0, {"nodes": [], "ents": []}
+    e2e_ms, e2e_steps = 0.0, 0
+    sampler.start()
+    while done_steps < args.steps and cur + 1 < len(states):
+        n_here = min(S, args.steps - done_steps)
+        tg = state_targets(states[cur], n_here, 100 + cur)
+        q = incoming(cur)
+        ctx.set_partition_source(q, stage(q, cur & 1))
+        barrier()
+        t1 = time.perf_counter()
+        ctx.set_resident(states[cur + 1], async_=True)       # the incoming block starts loading on the side stream
+        run_steps(tg, cur * 100_000, False)
+        ev_steps = torch.cuda.Event()
+        ev_steps.record()
+        ev_steps.synchronize()                                # the steps are done; the copy on the side stream may not be
+        t2 = time.perf_counter()
+        ctx.commit_resident(120_000)                          # waits for what is left of the copy, flips the map, rebuilds the view
+        torch.cuda.synchronize()
+        t3 = time.perf_counter()
+        barrier()
+        seg_ms.append((t3 - t1) * 1e3)
+        commit_ms.append((t3 - t2) * 1e3)
+        done_steps += n_here
+        cur += 1
+    clocks = sampler.stop()
+    launches = ctx.kernel_launches() - launches0
+    # the same without a swap in flight: steps alone on the current state (also the phase profile), then end to end
+    tg = state_targets(states[cur], min(S, args.steps), 999)
+    barrier()
+    t1 = time.perf_counter()
+    run_steps(tg, 7 << 20, False)
+    torch.cuda.synchronize()
+    steps_alone_ms = (time.perf_counter() - t1) * 1e3 / tg.shape[0]
+    ctx.profile(True)
+    ctx.profile_read(reset=True)
+    for i in range(tg.shape[0]):
+        run_steps(tg[i:i + 1], (8 << 20) + i * G, False)
+        n_, e_ = denses[0].counts()
+        stats["nodes"].append(n_); stats["ents"].append(e_)
+    phases = ctx.profile_read(reset=True)
+    ctx.profile(False)
+    tg_host = [t.cpu().pin_memory() for t in tg]
+    barrier()
+    t1 = time.perf_counter()
+    run_steps(tg_host, 9 << 20, True)
+    torch.cuda.synchronize()
+    e2e_ms = (time.perf_counter() - t1) * 1e3 / len(tg_host)
+    # a commit with its copy already complete: slot map + view rebuild alone
+    if cur + 1 < len(states):
+        q = incoming(cur)
+        ctx.set_partition_source(q, stage(q, cur & 1))
+        ctx.set_resident(states[cur + 1], async_=True)
+        time.sleep(1.0)
+        torch.cuda.synchronize()
+        t1 = time.perf_counter()
+        ctx.commit_resident(120_000)
+        torch.cuda.synchronize()
+        rebuild_alone_ms = (time.perf_counter() - t1) * 1e3
+        swap_alone_ms = swap_and_rebuild_ms - rebuild_alone_ms
+    total_ms = float(sum(seg_ms))
+    if world > 1:
+        tt = torch.tensor([total_ms], device=device, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt[0])
+    nodes = torch.cat(stats["nodes"]).numpy()
+    ents = torch.cat(stats["ents"]).numpy()
+    cfg_like = {"dim": dim, "hidden": c["hidden"]}
+    alg = algorithmic_bytes(nodes, ents, cfg_like, feat_bytes=2)
+    n_prof = tg.shape[0]
+    agg1, rest = phases["aggregate_l1"], phases["aggregate_rest"]
+    sample_ms = sum(v["ms"] for name, v in phases.items() if name.startswith("sample_"))
+    block_bytes = rows_of(0) * dim * 2
+    exposed = [max(0.0, cm - (rebuild_alone_ms or 0.0)) for cm in commit_ms]
+    tf32_peak = peaks["bf16_tflops_sustained"] * 0.5
+    line = {
+        "metric": "DENSE sample+aggregate mini-batches/s", "value": done_steps * G * world / (total_ms / 1e3), "unit": "mini-batches/s",
+        "n_gpus": world, "steps": done_steps, "warmup": args.warmup, "ms_per_step": total_ms / max(1, done_steps),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32 (fp16 features, TF32 tensor-core GEMM)",
+        "data": "synthetic",
+        "config": {"workload": OOC_WORKLOAD, "nodes": c["n"], "edges": n_edges, "feature_dim": dim, "feature_dtype": "fp16",
+                   "hidden": c["hidden"], "fanouts": c["fanouts"], "targets_per_batch": T, "mini_batches_per_step": G,
+                   "partitions": P, "resident": cap, "steps_per_buffer_state": S, "buffer_states_timed": len(seg_ms),
+                   "timed_region": "per buffer state: queue the swap of one 5.86 GB block from pinned host memory, run the state's "
+                                   "steps, commit (wait for the copy, slot map, in-buffer view); summed over the states",
+                   "l2": "inputs larger than L2 (58.6 GB of resident feature blocks; no flush)", "setup_s": setup_s},
+        "sampled_edges_per_s": float(ents.sum()) / n_prof * done_steps * world / (total_ms / 1e3),
+        "per_batch": {"nodes": float(nodes.sum(1).mean()), "sampled_edges": float(ents.sum(1).mean()),
+                      "algorithmic_bytes": alg["a_min"] / (n_prof * G)},
+        "swap": {"block_bytes": block_bytes, "swap_alone_ms": swap_alone_ms, "rebuild_alone_ms": rebuild_alone_ms,
+                 "h2d_gbs_alone": block_bytes / (swap_alone_ms / 1e3) / 1e9 if swap_alone_ms else None,
+                 "commit_ms_per_state": commit_ms, "exposed_swap_ms_per_state": exposed,
+                 "fraction_of_swap_hidden": (1.0 - float(np.mean(exposed)) / swap_alone_ms) if swap_alone_ms else None,
+                 "ms_per_step_without_a_swap_in_flight": steps_alone_ms},
+        "e2e": {"value": G * world / (e2e_ms / 1e3), "unit": "mini-batches/s", "h2d_bytes_per_step": int(G * T * 4),
+                "d2h_bytes_per_step": int(G * T * c["hidden"] * 4), "ms_per_step": e2e_ms,
+                "note": "host targets in, host H^k out, no swap in flight"},
+        "gpu_launches": int(launches), "clocks": clocks,
+        "roofline": {"kernel": "k_sage_layer_fused<layer 1, fp16 features> (feature gather + segment mean + tcgen05 TF32 GEMM)",
+                     "bound": "hbm", "achieved": alg["agg_l1"] / (agg1["ms"] / 1e3) / 1e9 if agg1["ms"] else None,
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "bytes_per_launch": alg["agg_l1"] / max(1, agg1["launches"]),
+                     "ms_per_launch": agg1["ms"] / max(1, agg1["launches"]), "peak_source": peaks["source"], "traffic": None},
+        "tensor": {"bound": "tensor", "achieved": alg["flops"] / ((agg1["ms"] + rest["ms"]) / 1e3) / 1e12, "peak": tf32_peak, "unit": "TFLOP/s",
+                   "layer1_tflops": alg["flops_l1"] / (agg1["ms"] / 1e3) / 1e12 if agg1["ms"] else None},
+        "phases_ms_per_step": {name: round(v["ms"] / n_prof, 4) for name, v in phases.items() if v["launches"]},
+    }
+    if line["roofline"]["achieved"]:
+        line["roofline"]["frac"] = line["roofline"]["achieved"] / peaks["hbm_gbs"]
+    line["tensor"]["frac"] = line["tensor"]["achieved"] / tf32_peak
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
 
 
 def run_lp(args, peaks, rank, local_rank, world):

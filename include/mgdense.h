@@ -144,6 +144,15 @@ int mg_set_partitioning(mg_ctx* ctx, int32_t n_parts);
 int mg_load_features(mg_ctx* ctx, const void* table, int table_is_device, int dtype, int32_t dim,
                      int32_t buffer_capacity_parts, int backing);
 
+/* MG_BACKING_HOST only: partition `part`'s rows (its ceil(n_nodes / n_parts) rows, the last partition fewer) are
+ * at host_block instead of at their place in the table -- for tables that do not fit host memory as a whole (config
+ * 4: 187 GB): the caller keeps a few pinned staging blocks, fills one with a partition (from disk, or regenerated),
+ * names it here, and asks for the partition with mg_set_resident.  mg_load_features may then be given table = NULL.
+ * The block must stay valid and unchanged until the mg_commit_resident that brings the partition in has returned
+ * MG_OK (and, if the partition's rows are updated in the buffer, until it has been evicted: the write-back goes to the
+ * same block).  NULL removes the override.  Errors: MG_ERR_ARG, MG_ERR_STATE (no host-backed buffer, or a set pending). */
+int mg_set_partition_source(mg_ctx* ctx, int32_t part, const void* host_block);
+
 /* Ask for the set of resident partitions (the S_i of Section 3).  The difference to the
  * current set is computed; partitions to be added are copied host->device on the side
  * stream (MG_BACKING_HOST).  Sampling and forward calls keep using the current set until
@@ -240,7 +249,11 @@ int mg_dense_free(mg_dense* d);
 /* k layers of widths dims[0] -> dims[1] -> ... -> dims[k]; w_self[l], w_nbr[l] are HOST
  * row-major [dims[l], dims[l+1]] fp32, bias[l] HOST [dims[l+1]] (copied).  Layer l+1
  * computes act(self . w_self + mean(sampled neighbours) . w_nbr + bias) with ReLU on all
- * but the last layer.  dims must be multiples of 4. */
+ * but the last layer.  dims must be multiples of 4.
+ * MG_GEMM_TF32 with half-precision base representations (MG_DTYPE_F16 table): the first layer's GEMM then runs on fp16
+ * operands (the rows as they are, the mean and the weights rounded to fp16: the same 10-bit mantissa as TF32, fp32
+ * accumulate), provided the layer's weights sit well inside fp16's range (largest magnitude below 2^15, root mean
+ * square above 2^-10) and the mean aggregator is used; otherwise on TF32 operands. */
 int mg_model_create(mg_ctx* ctx, int32_t k, const int32_t* dims, const float* const* w_self,
                     const float* const* w_nbr, const float* const* bias, int gemm_precision,
                     mg_model** out);
@@ -250,6 +263,15 @@ int mg_model_create(mg_ctx* ctx, int32_t k, const int32_t* dims, const float* co
 #define MG_AGGR_MEAN 0
 #define MG_AGGR_SUM 1
 int mg_model_set_aggregator(mg_model* m, int aggregator);
+/* Storage of the intermediate layer outputs H^1 .. H^{k-1} inside mg_forward: MG_DTYPE_F32 (default) or
+ * MG_DTYPE_F16.  The tensor-core layers round their inputs to a 10-bit mantissa anyway (TF32); fp16 keeps those bits,
+ * so H^k stays within the tensor-core tolerance of the fp32 result, while a layer's output and the next layer's gather
+ * move half the bytes in half the memory requests -- but fp16 has a 5-bit exponent: activations beyond 65504 overflow,
+ * so this is an option, not the default (the paper stores 4-byte floats).  Takes effect when every layer runs in the
+ * fused tensor-core kernel (MG_GEMM_TF32, widths <= 256), the intermediate widths are multiples of 128, the mean
+ * aggregator is used, the weights suit fp16 (largest magnitude below 2^15, root mean square above 2^-10) and
+ * mg_keep_layer_outputs is off; otherwise the call is accepted and fp32 is used.  Errors: MG_ERR_ARG. */
+int mg_model_set_intermediates(mg_model* m, int dtype);
 int mg_model_free(mg_model* m);
 
 /* Forward pass for every batch of `d`.  H^0 is read straight from the feature buffer (rows

@@ -28,8 +28,8 @@ CORRUPT_DST, CORRUPT_SRC, CORRUPT_BOTH = 1, 2, 3
 # every symbol include/mgdense.h declares
 EXPORTS = [
     "mg_create", "mg_destroy", "mg_last_error", "mg_load_graph", "mg_load_out_graph", "mg_set_sample_direction", "mg_set_partitioning",
-    "mg_load_features", "mg_set_resident", "mg_commit_resident", "mg_sample_many", "mg_sample_many_begin", "mg_sample_many_end", "mg_sample",
-    "mg_dense_counts", "mg_dense_view", "mg_dense_export_many", "mg_dense_export_view", "mg_dense_free", "mg_model_create", "mg_model_set_aggregator", "mg_model_free",
+    "mg_load_features", "mg_set_partition_source", "mg_set_resident", "mg_commit_resident", "mg_sample_many", "mg_sample_many_begin", "mg_sample_many_end", "mg_sample",
+    "mg_dense_counts", "mg_dense_view", "mg_dense_export_many", "mg_dense_export_view", "mg_dense_free", "mg_model_create", "mg_model_set_aggregator", "mg_model_set_intermediates", "mg_model_free",
     "mg_forward", "mg_set_layer_window", "mg_keep_layer_outputs", "mg_forward_host_async", "mg_wait_output", "mg_forward_noalloc", "mg_gather_h0", "mg_layer_output", "mg_lp_prepare", "mg_lp_view", "mg_lp_free",
     "mg_distmult_score", "mg_kernel_launches", "mg_profile", "mg_profile_read", "mg_comet_plan", "mg_comet_bias", "mg_comet_autotune", "mg_gat_model_create", "mg_gat_model_free", "mg_gat_forward", "mg_backward", "mg_model_grads", "mg_model_sgd_step", "mg_model_adagrad_step", "mg_dense_packed_ids", "mg_apply_embedding_sgd",
 ]
@@ -223,6 +223,11 @@ class Model:
         ctx._check(ctx.lib.mg_model_create(ctx.handle, C.c_int32(k), dims, arrs[0], arrs[1], arrs[2],
                                            C.c_int(precision), C.byref(self.handle)))
 
+    def set_intermediates(self, dtype):
+        """torch.float16: keep H^1 .. H^{k-1} as fp16 inside forward (where the model allows it); torch.float32: default."""
+        code = {torch.float32: DTYPE_F32, torch.float16: DTYPE_F16}[dtype]
+        self.ctx._check(self.ctx.lib.mg_model_set_intermediates(self.handle, C.c_int(code)))
+
     def set_aggregator(self, aggregator: str):
         """"mean" (GraphSage's mean over the sampled neighbours, the default) or "sum"."""
         self.ctx._check(self.ctx.lib.mg_model_set_aggregator(self.handle, C.c_int({"mean": 0, "sum": 1}[aggregator])))
@@ -381,12 +386,26 @@ class Context:
     def set_partitioning(self, n_parts: int):
         self._check(self.lib.mg_set_partitioning(self.handle, C.c_int32(n_parts)))
 
-    def load_features(self, table: torch.Tensor, capacity_parts: int = 1, backing: int = BACKING_HBM):
+    def load_features(self, table: torch.Tensor | None, capacity_parts: int = 1, backing: int = BACKING_HBM, dtype=None, dim=None):
+        """table = None (host backing only): no whole table exists; give dtype and dim, and name every partition's
+        host block with set_partition_source before asking for it."""
+        if table is None:
+            dt = {torch.float32: DTYPE_F32, torch.float16: DTYPE_F16}[dtype]
+            self._check(self.lib.mg_load_features(self.handle, None, C.c_int(0), C.c_int(dt), C.c_int32(dim),
+                                                  C.c_int32(capacity_parts), C.c_int(backing)))
+            return
         assert table.dim() == 2 and table.is_contiguous()
         dt = {torch.float32: DTYPE_F32, torch.float16: DTYPE_F16}[table.dtype]
         self._keep["features"] = table          # device tables are borrowed, host tables stay the backing store
         self._check(self.lib.mg_load_features(self.handle, _ptr(table), C.c_int(table.is_cuda), C.c_int(dt),
                                               C.c_int32(table.shape[1]), C.c_int32(capacity_parts), C.c_int(backing)))
+
+    def set_partition_source(self, part: int, block: torch.Tensor | None):
+        """Partition `part`'s rows are in `block` (host tensor, preferably pinned; kept alive by this context)."""
+        if block is not None:
+            assert not block.is_cuda and block.is_contiguous()
+            self._keep[("source", part)] = block
+        self._check(self.lib.mg_set_partition_source(self.handle, C.c_int32(part), _ptr(block)))
 
     def set_resident(self, parts, async_: bool = False):
         p = _host(list(parts), torch.int32)

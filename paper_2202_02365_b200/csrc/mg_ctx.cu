@@ -82,53 +82,117 @@ __global__ void k_check_graph(const int64_t* off, int64_t n_nodes, const int32_t
 }
 
 // ---- in-buffer view: rows of resident nodes restricted to resident neighbours -------------
-constexpr int kRowLanes = 8;
+// Edge-parallel, so that a hub's million-entry row costs what a million short rows cost.  Partitions are contiguous id
+// ranges and rows are stored in id order, so the rows of a partition are one contiguous range of edges: an edge stays
+// when its position lies in a resident partition's range and its neighbour's partition is resident.
+//   k_view_mask     per tile of 2048 edges: a keep bit per edge (32 per word), the number of kept edges before each
+//                   word inside the tile, the tile's count
+//   (64-bit scan of the tile counts)
+//   k_view_compact  kept edges to their places, in order
+//   k_view_offsets  a row's new offset = the number of kept edges before its first edge (tile base + word prefix +
+//                   population count of the word's lower bits)
+constexpr int kViewTile = 2048;   // edges per tile: 256 threads x 8
 
-__global__ void __launch_bounds__(kThreads)
-k_view_count(const int64_t* __restrict__ off, const int32_t* __restrict__ nbrs, int64_t n_nodes, uint32_t part_size,
-             const int32_t* __restrict__ slot_of_part, int32_t* cnt) {
-    const int gl = threadIdx.x % kRowLanes;
-    const int64_t groups = (int64_t)gridDim.x * (kThreads / kRowLanes);
-    const int64_t n_round = (n_nodes + groups - 1) / groups * groups;  // whole warps stay in the loop together
-    for (int64_t v = blockIdx.x * (int64_t)(kThreads / kRowLanes) + threadIdx.x / kRowLanes; v < n_round; v += groups) {
-        int32_t c = 0;
-        if (v < n_nodes && slot_of_part[(uint32_t)v / part_size] >= 0) {
-            const int64_t lo = off[v], hi = off[v + 1];
-            for (int64_t e = lo + gl; e < hi; e += kRowLanes)
-                c += slot_of_part[(uint32_t)nbrs[e] / part_size] >= 0 ? 1 : 0;
+struct ViewArgs {
+    const int64_t* off;
+    const int32_t* nbrs;
+    int64_t n_nodes, n_edges;
+    uint32_t part_size;
+    int32_t n_parts;
+    const int32_t* slot_of_part;
+    uint32_t* mask;        // [ceil(E / 32)]
+    uint16_t* word_before; // [ceil(E / 32)] kept edges of the tile before the word
+    int32_t* tile_cnt;     // [tiles]
+    const int64_t* tile_base;  // [tiles + 1]
+};
+
+// first edge of partition p's rows
+__device__ __forceinline__ int64_t part_edge_lo(const ViewArgs& a, int p) {
+    const int64_t v = (int64_t)p * a.part_size;
+    return a.off[v < a.n_nodes ? v : a.n_nodes];
+}
+
+__global__ void __launch_bounds__(kThreads) k_view_mask(ViewArgs a) {
+    __shared__ int64_t bound[MG_MAX_PARTS + 1];
+    __shared__ int32_t res[MG_MAX_PARTS];
+    __shared__ uint32_t warp_tot[kThreads / 32];
+    for (int p = threadIdx.x; p <= a.n_parts; p += kThreads) bound[p] = part_edge_lo(a, p);
+    for (int p = threadIdx.x; p < a.n_parts; p += kThreads) res[p] = a.slot_of_part[p] >= 0 ? 1 : 0;
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t n_tiles = (a.n_edges + kViewTile - 1) / kViewTile;
+    for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+        const int64_t e0 = t * kViewTile + (int64_t)threadIdx.x * 8;
+        // partition whose edge range holds e0 (ranges of empty partitions are empty and skipped)
+        int p = 0;
+        {
+            int lo = 0, hi = a.n_parts;   // bound[lo] <= e0 < bound[hi] (bound[n_parts] = E)
+            while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (bound[mid] <= e0) lo = mid; else hi = mid; }
+            p = lo;
         }
+        uint32_t bits = 0;
+        const bool any_row = e0 < a.n_edges && (res[p] || bound[p + 1] < e0 + 8);   // (a thread's 8 edges may cross into a resident range)
+        if (any_row) {
+            int32_t u[8];
+            if (e0 + 8 <= a.n_edges) {
+                const int4 x = __ldg(reinterpret_cast<const int4*>(a.nbrs + e0)), y = __ldg(reinterpret_cast<const int4*>(a.nbrs + e0 + 4));
+                u[0] = x.x; u[1] = x.y; u[2] = x.z; u[3] = x.w; u[4] = y.x; u[5] = y.y; u[6] = y.z; u[7] = y.w;
+            } else {
 #pragma unroll
-        for (int o = kRowLanes / 2; o > 0; o >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
-        if (gl == 0 && v < n_nodes) cnt[v] = c;
+                for (int j = 0; j < 8; ++j) u[j] = e0 + j < a.n_edges ? a.nbrs[e0 + j] : 0;
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int64_t e = e0 + j;
+                while (p + 1 < a.n_parts && e >= bound[p + 1]) ++p;
+                if (e < a.n_edges && res[p] && res[(uint32_t)u[j] / a.part_size]) bits |= 1u << j;
+            }
+        }
+        // four lanes make a word; counts: exclusive scan over the block's 256 threads
+        uint32_t word = bits << (8 * (lane & 3));
+        word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
+        word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
+        const uint32_t mine = __popc(bits);
+        const uint32_t inc = warp_incl_scan(mine);
+        if (lane == 31) warp_tot[warp] = inc;
+        __syncthreads();
+        uint32_t before = inc - mine;
+        for (int w = 0; w < warp; ++w) before += warp_tot[w];
+        if ((lane & 3) == 0 && e0 < a.n_edges) {
+            a.mask[e0 >> 5] = word;
+            a.word_before[e0 >> 5] = (uint16_t)before;
+        }
+        if (threadIdx.x == kThreads - 1) a.tile_cnt[t] = (int32_t)(before + mine);
+        __syncthreads();
     }
 }
 
-__global__ void __launch_bounds__(kThreads)
-k_view_fill(const int64_t* __restrict__ off, const int32_t* __restrict__ nbrs, int64_t n_nodes, uint32_t part_size,
-            const int32_t* __restrict__ slot_of_part, const int64_t* __restrict__ view_off, int32_t* view_nbrs) {
+__global__ void __launch_bounds__(kThreads) k_view_compact(ViewArgs a, int32_t* view_nbrs) {
     const int lane = threadIdx.x & 31;
-    const int gl = threadIdx.x % kRowLanes;
-    const int gshift = lane - gl;
-    const int64_t groups = (int64_t)gridDim.x * (kThreads / kRowLanes);
-    const int64_t n_round = (n_nodes + groups - 1) / groups * groups;  // whole warps stay in the loop together
-    for (int64_t v = blockIdx.x * (int64_t)(kThreads / kRowLanes) + threadIdx.x / kRowLanes; v < n_round; v += groups) {
-        int64_t lo = 0, hi = 0, out = 0;
-        if (v < n_nodes && slot_of_part[(uint32_t)v / part_size] >= 0) {
-            lo = off[v]; hi = off[v + 1]; out = view_off[v];
-        }
-        // the longest row of the warp's four groups sets the trip count, so ballots stay converged
-        int64_t len = hi - lo;
+    const int64_t n_tiles = (a.n_edges + kViewTile - 1) / kViewTile;
+    for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+        const int64_t base = a.tile_base[t];
+        if (a.tile_base[t + 1] == base) continue;             // nothing of this tile stays: its edges are not even read
+        const int64_t e0 = t * kViewTile + (int64_t)threadIdx.x * 8;
+        if (e0 >= a.n_edges) continue;
+        const uint32_t word = a.mask[e0 >> 5];
+        const uint32_t bits = (word >> (8 * (lane & 3))) & 0xFFu;
+        if (!bits) continue;
+        int64_t out = base + a.word_before[e0 >> 5] + __popc(word & ((1u << (8 * (lane & 3))) - 1u));
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) len = max(len, __shfl_xor_sync(0xFFFFFFFFu, len, o));
-        for (int64_t base = 0; base < len; base += kRowLanes) {
-            const int64_t e = lo + base + gl;
-            int32_t u = 0;
-            bool keep = false;
-            if (e < hi) { u = nbrs[e]; keep = slot_of_part[(uint32_t)u / part_size] >= 0; }
-            const uint32_t bal = (__ballot_sync(0xFFFFFFFFu, keep) >> gshift) & ((1u << kRowLanes) - 1u);
-            if (keep) view_nbrs[out + __popc(bal & ((1u << gl) - 1u))] = u;
-            out += __popc(bal);
-        }
+        for (int j = 0; j < 8; ++j)
+            if (bits & (1u << j)) view_nbrs[out++] = a.nbrs[e0 + j];
+    }
+}
+
+__global__ void __launch_bounds__(kThreads) k_view_offsets(ViewArgs a, int64_t* view_off) {
+    const int64_t n_tiles = (a.n_edges + kViewTile - 1) / kViewTile;
+    for (int64_t v = blockIdx.x * (int64_t)kThreads + threadIdx.x; v <= a.n_nodes; v += (int64_t)gridDim.x * kThreads) {
+        const int64_t e = a.off[v];
+        int64_t r;
+        if (e >= a.n_edges) r = a.tile_base[n_tiles];
+        else r = a.tile_base[e / kViewTile] + a.word_before[e >> 5] + __popc(a.mask[e >> 5] & ((1u << (e & 31)) - 1u));
+        view_off[v] = r;
     }
 }
 
@@ -225,8 +289,12 @@ extern "C" int mg_create(mg_ctx** out, int device, void* stream) {
     cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, device);
     if (c->n_sms <= 0) c->n_sms = 148;
     for (int i = 0; i < PH_COUNT; ++i) c->prof[i] = ProfPhase{kPhaseNames[i], 0.0, 0};
+    // the sampling stream has the lowest priority: when a layer kernel and sampler kernels are both ready, the layer
+    // kernel's blocks are placed first and the sampler's short blocks fill what is left of every SM
+    int prio_least = 0, prio_greatest = 0;
+    cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest);
     if (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
-        cudaStreamCreateWithFlags(&c->sample_stream, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithPriority(&c->sample_stream, cudaStreamNonBlocking, prio_least) != cudaSuccess ||
         cudaEventCreateWithFlags(&c->ev_user, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&c->ev_fwd_done, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&c->ev_out_done, cudaEventDisableTiming) != cudaSuccess ||
@@ -260,6 +328,7 @@ static void free_out_graph(mg_ctx* c) {
 static void free_features(mg_ctx* c) {
     if (c->slots_owned) cudaFree(c->slots);
     c->slots = nullptr; c->slots_owned = false; c->host_table = nullptr; c->feat_dim = 0; c->n_slots = 0;
+    c->part_source.clear();
 }
 
 extern "C" int mg_destroy(mg_ctx* c) {
@@ -274,6 +343,7 @@ extern "C" int mg_destroy(mg_ctx* c) {
     free_features(c);
     free_out_graph(c);
     cudaFree(c->row_off); cudaFree(c->nbrs); cudaFree(c->d_slot_of_part); cudaFree(c->d_res_prefix); cudaFree(c->d_flags);
+    cudaFree(c->view_ws);
     cudaFree(c->ws_x); cudaFree(c->ws_h[0]); cudaFree(c->ws_h[1]);
     cudaEventDestroy(c->ev_fwd_done); cudaEventDestroy(c->ev_out_done); cudaEventDestroy(c->ev_user);
     for (int i = 0; i < 2; ++i) { if (c->ev_hk_done[i]) cudaEventDestroy(c->ev_hk_done[i]); cudaFree(c->hk_buf[i]); }
@@ -357,31 +427,48 @@ static int rebuild_one_view(mg_ctx* c, bool all, const int64_t* row_off, const i
         }
         *owned = true;
     }
-    const int64_t n = c->n_nodes;
-    const int64_t ntiles = (n + kTile - 1) / kTile;
-    int32_t* cnt = nullptr;
-    uint64_t* tiles = nullptr;
-    int64_t* d_total = nullptr;
-    if (cudaMalloc((void**)&cnt, sizeof(int32_t) * std::max<int64_t>(n, 1)) != cudaSuccess ||
-        cudaMalloc((void**)&tiles, sizeof(uint64_t) * (ntiles + 1)) != cudaSuccess ||
-        cudaMalloc((void**)&d_total, sizeof(int64_t)) != cudaSuccess) {
-        cudaGetLastError();
-        cudaFree(cnt); cudaFree(tiles); cudaFree(d_total);
-        return mg_fail(c, MG_ERR_OOM, "scratch allocation for the in-buffer graph view failed");
+    // scratch (kept by the context, grown on demand): keep bits, per-word prefixes, tile counts and bases, scan scratch
+    const int64_t n_words = (n_edges + 31) / 32 + 1;
+    const int64_t n_tiles = (n_edges + kViewTile - 1) / kViewTile;
+    const int64_t n_scan_tiles = (n_tiles + kTile - 1) / kTile;
+    auto up = [](size_t b) { return (b + 255) / 256 * 256; };
+    const size_t o_mask = 0, o_before = o_mask + up(sizeof(uint32_t) * n_words), o_cnt = o_before + up(sizeof(uint16_t) * n_words),
+                 o_base = o_cnt + up(sizeof(int32_t) * (n_tiles + 1)), o_scan = o_base + up(sizeof(int64_t) * (n_tiles + 2)),
+                 o_total = o_scan + up(sizeof(uint64_t) * (n_scan_tiles + 1)), need = o_total + 256;
+    if (c->view_ws_bytes < need) {
+        cudaFree(c->view_ws);
+        c->view_ws = nullptr; c->view_ws_bytes = 0;
+        if (cudaMalloc((void**)&c->view_ws, need) != cudaSuccess) { cudaGetLastError(); return mg_fail(c, MG_ERR_OOM, "scratch allocation for the in-buffer graph view failed"); }
+        c->view_ws_bytes = need;
     }
+    ViewArgs a;
+    a.off = row_off; a.nbrs = nbrs; a.n_nodes = c->n_nodes; a.n_edges = n_edges;
+    a.part_size = (uint32_t)c->part_size; a.n_parts = c->n_parts; a.slot_of_part = c->d_slot_of_part;
+    a.mask = reinterpret_cast<uint32_t*>(c->view_ws + o_mask);
+    a.word_before = reinterpret_cast<uint16_t*>(c->view_ws + o_before);
+    a.tile_cnt = reinterpret_cast<int32_t*>(c->view_ws + o_cnt);
+    int64_t* tile_base = reinterpret_cast<int64_t*>(c->view_ws + o_base);
+    a.tile_base = tile_base;
+    uint64_t* scan_tiles = reinterpret_cast<uint64_t*>(c->view_ws + o_scan);
+    int64_t* d_total = reinterpret_cast<int64_t*>(c->view_ws + o_total);
     const int grid = mg_grid(c, 8);
     cudaStream_t st = c->stream;
-    k_view_count<<<grid, kThreads, 0, st>>>(row_off, nbrs, n, (uint32_t)c->part_size, c->d_slot_of_part, cnt);
-    k_scan64_reduce<<<grid, kThreads, 0, st>>>(cnt, n, tiles);
-    k_scan64_tiles<<<1, kThreads, 0, st>>>(tiles, ntiles, d_total);
-    k_scan64_down<<<grid, kThreads, 0, st>>>(cnt, n, tiles, *view_off);
-    k_view_fill<<<grid, kThreads, 0, st>>>(row_off, nbrs, n, (uint32_t)c->part_size, c->d_slot_of_part, *view_off, *view_nbrs);
-    c->launches += 5;
     int64_t total = 0;
-    cudaError_t e = cudaMemcpyAsync(&total, d_total, sizeof(int64_t), cudaMemcpyDeviceToHost, st);
+    cudaError_t e = cudaSuccess;
+    if (n_edges > 0) {
+        k_view_mask<<<grid, kThreads, 0, st>>>(a);
+        k_scan64_reduce<<<grid, kThreads, 0, st>>>(a.tile_cnt, n_tiles, scan_tiles);
+        k_scan64_tiles<<<1, kThreads, 0, st>>>(scan_tiles, n_scan_tiles, d_total);
+        k_scan64_down<<<grid, kThreads, 0, st>>>(a.tile_cnt, n_tiles, scan_tiles, tile_base);
+        k_view_compact<<<grid, kThreads, 0, st>>>(a, *view_nbrs);
+        k_view_offsets<<<grid, kThreads, 0, st>>>(a, *view_off);
+        c->launches += 6;
+        e = cudaMemcpyAsync(&total, d_total, sizeof(int64_t), cudaMemcpyDeviceToHost, st);
+    } else {
+        e = cudaMemsetAsync(*view_off, 0, sizeof(int64_t) * (c->n_nodes + 1), st);
+    }
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e == cudaSuccess) e = cudaGetLastError();
-    cudaFree(cnt); cudaFree(tiles); cudaFree(d_total);
     if (e != cudaSuccess) return mg_cuda_fail(c, e, "rebuild of the in-buffer graph view");
     *view_edges = total;
     return MG_OK;
@@ -518,7 +605,7 @@ extern "C" int mg_load_features(mg_ctx* c, const void* table, int table_is_devic
                                 int32_t buffer_capacity_parts, int backing) {
     if (!c) return MG_ERR_ARG;
     if (!c->row_off) return mg_fail(c, MG_ERR_STATE, "no graph loaded");
-    if (!table) return mg_fail(c, MG_ERR_ARG, "null table");
+    if (!table && backing != MG_BACKING_HOST) return mg_fail(c, MG_ERR_ARG, "null table");
     if (dtype != MG_DTYPE_F32 && dtype != MG_DTYPE_F16) return mg_fail(c, MG_ERR_ARG, "unknown dtype");
     const int64_t esz = dtype == MG_DTYPE_F32 ? 4 : 2;
     if (dim <= 0 || (dim * esz) % 16 != 0) return mg_fail(c, MG_ERR_ARG, "dim * sizeof(dtype) must be a positive multiple of 16 bytes");
@@ -564,6 +651,7 @@ extern "C" int mg_load_features(mg_ctx* c, const void* table, int table_is_devic
         c->dirty_part.clear();
         c->feat_dim = dim;
         if ((int)keep.size() > c->capacity) keep.resize(c->capacity);
+        if (!table) keep.clear();   // no whole table: partitions come in once their host blocks have been named
         if (!keep.empty()) {
             int rc = mg_set_resident(c, keep.data(), (int32_t)keep.size(), 0);
             if (rc) return rc;
@@ -586,6 +674,22 @@ extern "C" int mg_load_features(mg_ctx* c, const void* table, int table_is_devic
     return rebuild_view(c);
 }
 
+// where partition p's rows live in host memory (MG_BACKING_HOST), or null when nobody said
+static const char* host_block_of(const mg_ctx* c, int p) {
+    if (p < (int)c->part_source.size() && c->part_source[p]) return c->part_source[p];
+    return c->host_table ? c->host_table + (size_t)p * c->part_size * c->row_bytes : nullptr;
+}
+
+extern "C" int mg_set_partition_source(mg_ctx* c, int32_t part, const void* host_block) {
+    if (!c) return MG_ERR_ARG;
+    if (!c->slots || c->backing != MG_BACKING_HOST) return mg_fail(c, MG_ERR_STATE, "partition sources belong to a host-backed feature buffer");
+    if (part < 0 || part >= c->n_parts) return mg_fail(c, MG_ERR_ARG, "partition id out of range");
+    if (c->has_pending) return mg_fail(c, MG_ERR_STATE, "a resident set is pending (its copies may still read the old block); commit it first");
+    if ((int)c->part_source.size() < c->n_parts) c->part_source.resize(c->n_parts, nullptr);
+    c->part_source[part] = (const char*)host_block;
+    return MG_OK;
+}
+
 extern "C" int mg_set_resident(mg_ctx* c, const int32_t* part_ids, int32_t n, int async) {
     if (!c) return MG_ERR_ARG;
     if (!c->row_off) return mg_fail(c, MG_ERR_STATE, "no graph loaded");
@@ -601,6 +705,10 @@ extern "C" int mg_set_resident(mg_ctx* c, const int32_t* part_ids, int32_t n, in
     MG_CUDA(c, cudaSetDevice(c->device));
     std::vector<int32_t> next(c->n_parts, -1);
     const bool host_backed = c->slots && c->backing == MG_BACKING_HOST;
+    if (host_backed)
+        for (int p = 0; p < c->n_parts; ++p)
+            if (want[p] && c->slot_of_part[p] < 0 && !host_block_of(c, p))
+                return mg_fail(c, MG_ERR_STATE, "partition %d has no host block: no table was given and mg_set_partition_source was not called for it", p);
     if (!host_backed) {
         for (int p = 0; p < c->n_parts; ++p) next[p] = want[p] ? p : -1;
     } else {
@@ -631,9 +739,9 @@ extern "C" int mg_set_resident(mg_ctx* c, const int32_t* part_ids, int32_t n, in
             }
             const int64_t first = (int64_t)p * c->part_size;
             const int64_t rows = std::min<int64_t>(c->part_size, c->n_nodes - first);
-            if (rows > 0)
-                MG_CUDA(c, cudaMemcpyAsync(const_cast<char*>(c->host_table) + (size_t)first * c->row_bytes,
-                                           c->slots + (size_t)s * c->slot_bytes, (size_t)rows * c->row_bytes,
+            char* back = const_cast<char*>(host_block_of(c, p));
+            if (rows > 0 && back)
+                MG_CUDA(c, cudaMemcpyAsync(back, c->slots + (size_t)s * c->slot_bytes, (size_t)rows * c->row_bytes,
                                            cudaMemcpyDeviceToHost, c->side));
             c->dirty_part[p] = 0;
         }
@@ -652,9 +760,12 @@ extern "C" int mg_set_resident(mg_ctx* c, const int32_t* part_ids, int32_t n, in
             next[p] = s;
             const int64_t first = (int64_t)p * c->part_size;
             const int64_t rows = std::min<int64_t>(c->part_size, c->n_nodes - first);
-            if (rows > 0)
-                MG_CUDA(c, cudaMemcpyAsync(c->slots + (size_t)s * c->slot_bytes, c->host_table + (size_t)first * c->row_bytes,
-                                           (size_t)rows * c->row_bytes, cudaMemcpyHostToDevice, c->side));
+            // in pieces: a copy engine finishes what it has started, and one 5 GB copy would hold up every small
+            // host-to-device copy another stream issues meanwhile (targets of a sample, say) for a tenth of a second
+            const size_t bytes = (size_t)std::max<int64_t>(rows, 0) * c->row_bytes, piece = (size_t)8 << 20;
+            for (size_t at = 0; at < bytes; at += piece)
+                MG_CUDA(c, cudaMemcpyAsync(c->slots + (size_t)s * c->slot_bytes + at, host_block_of(c, p) + at,
+                                           std::min(piece, bytes - at), cudaMemcpyHostToDevice, c->side));
         }
         if (main_done) cudaEventDestroy(main_done);
         cudaEvent_t done;

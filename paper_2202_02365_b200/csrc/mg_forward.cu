@@ -9,6 +9,7 @@
 #include <cuda_fp16.h>
 
 #include <algorithm>
+#include <cmath>
 #include <cstdlib>
 
 #include "mg_device.cuh"
@@ -22,11 +23,13 @@ int mg_gemm_tf32_status(mg_ctx* ctx);
 int mg_gemm_tf32_splitk_add(mg_ctx* ctx, const float* x, const float* w_t, float* out, int64_t M, int N, int K, int kt_per_slice);
 // mg_layer_fused.cu
 int mg_pack_layer_weights(mg_ctx* ctx, const float* w_cat_dev, float* w_pad_t_dev, int d_in, int N);
+int mg_pack_layer_weights_f16(mg_ctx* ctx, const float* w_cat_dev, void* w_pad_h_dev, int d_in, int N);
 bool mg_layer_fused_supported(int d_in, int d_out);
 int mg_layer_rows(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_out, int4* row_meta);
 int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_out, const float* w_pad_t, const float* bias,
                    const float* h_prev, float* h_out, int flags /* 1 = ReLU, 2 = sum instead of mean */, const int4* row_meta,
-                   int64_t row_lo, int64_t row_hi, int64_t safe_src_row);
+                   int64_t row_lo, int64_t row_hi, int64_t safe_src_row, const void* w_pad_h /* the layer's fp16 weights, nullable */,
+                   int in_f16 /* layers >= 2: h_prev holds fp16 rows */, int out_f16 /* h_out receives fp16 rows */);
 
 namespace {
 
@@ -353,6 +356,28 @@ extern "C" int mg_model_create(mg_ctx* ctx, int32_t k, const int32_t* dims, cons
         ctx->launches++;
         mg_pack_layer_weights(ctx, m->w_cat[l], m->w_pad_t[l], (int)di, (int)dn);
     }
+    // Every layer's weights in fp16 form too, for layers whose input rows are fp16 (layer 1 over fp16 base
+    // representations; later layers when the model stores its intermediate outputs as fp16).  fp16 keeps the 10-bit
+    // mantissa TF32 keeps but has a 5-bit exponent: the copy is made only when the weights sit well inside its range
+    // (largest magnitude below 2^15, root mean square above 2^-10); otherwise that layer stays on TF32 operands.
+    for (int l = 0; l < k && gemm_precision == MG_GEMM_TF32; ++l) {
+        const size_t di = dims[l], dn = dims[l + 1];
+        if (di % 8 != 0) continue;
+        double sq = 0.0, mx = 0.0;
+        for (size_t i = 0; i < di * dn; ++i) {
+            const double a = std::fabs((double)w_self[l][i]), b = std::fabs((double)w_nbr[l][i]);
+            sq += a * a + b * b;
+            mx = std::max(mx, std::max(a, b));
+        }
+        const double rms = std::sqrt(sq / (double)(2 * di * dn));
+        if (!(mx < 32768.0 && rms > 1.0 / 1024.0)) continue;
+        if (cudaMalloc(&m->w_pad_h[l], sizeof(uint16_t) * 2 * ((di + 63) / 64 * 64) * dn) != cudaSuccess) {
+            cudaGetLastError();
+            mg_model_free(m);
+            return mg_fail(ctx, MG_ERR_OOM, "weight allocation failed");
+        }
+        mg_pack_layer_weights_f16(ctx, m->w_cat[l], m->w_pad_h[l], (int)di, (int)dn);
+    }
     cudaError_t e = cudaStreamSynchronize(ctx->stream);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) { mg_model_free(m); return mg_cuda_fail(ctx, e, "weight upload"); }
@@ -367,6 +392,13 @@ extern "C" int mg_model_set_aggregator(mg_model* m, int aggregator) {
     return MG_OK;
 }
 
+extern "C" int mg_model_set_intermediates(mg_model* m, int dtype) {
+    if (!m) return MG_ERR_ARG;
+    if (dtype != MG_DTYPE_F32 && dtype != MG_DTYPE_F16) return mg_fail(m->ctx, MG_ERR_ARG, "unknown dtype");
+    m->f16_intermediates = dtype == MG_DTYPE_F16;
+    return MG_OK;
+}
+
 extern "C" int mg_model_free(mg_model* m) {
     if (!m) return MG_OK;
     cudaSetDevice(m->device);
@@ -375,6 +407,7 @@ extern "C" int mg_model_free(mg_model* m) {
         cudaFree(m->g_w_cat[l]); cudaFree(m->g_bias[l]); cudaFree(m->s_w_cat[l]); cudaFree(m->s_bias[l]);
     }
     cudaFree(m->zeros);
+    for (int l = 0; l < MG_MAX_HOPS; ++l) cudaFree(m->w_pad_h[l]);
     if (m->ctx && m->ctx->last_fwd_model == m) m->ctx->last_fwd_model = nullptr;
     delete m;
     return MG_OK;
@@ -506,7 +539,7 @@ static int forward_impl(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out,
                 float* h_out = l == k ? hk : base + ring_off[l] - lo * m->dims[l];
                 ProfScope ps(ctx, l == 1 ? PH_AGG_L1 : PH_AGG_REST, 1);
                 rc = mg_layer_fused(ctx, d, l, m->dims[l - 1], m->dims[l], m->w_pad_t[l - 1], m->bias[l - 1], h_prev, h_out,
-                                    (l < k ? 1 : 0) | (m->sum_aggr ? 2 : 0), meta + meta_off[l], lo, hi, l > 1 ? lo_in : 0);
+                                    (l < k ? 1 : 0) | (m->sum_aggr ? 2 : 0), meta + meta_off[l], lo, hi, l > 1 ? lo_in : 0, l == 1 ? m->w_pad_h[0] : nullptr, 0, 0);
                 if (rc) return rc;
             }
         }
@@ -514,21 +547,28 @@ static int forward_impl(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out,
         return finish_forward(ctx, m, d, out, out_mode, hk);
     }
 
-    // per-layer outputs H^1..H^k live in one workspace (kept for mg_layer_output)
-    size_t total = 0;
+    // per-layer outputs H^1..H^k live in one workspace (kept for mg_layer_output).  A model may ask for fp16
+    // intermediates (mg_model_set_intermediates): used when every layer runs in the fused kernel with fp16 weights
+    // at hand, the widths allow 64-column output boxes, and nobody needs the fp32 layer outputs afterwards.
+    bool f16_inter = m->f16_intermediates && all_fused && !ctx->keep_layers && !m->sum_aggr && k > 1;
+    for (int l = 1; l < k && f16_inter; ++l) f16_inter = m->dims[l] % 128 == 0 && m->w_pad_h[l] != nullptr;
+    ctx->layers_kept = !f16_inter;
+    size_t total = 0;           // bytes
     size_t off[MG_MAX_HOPS + 1];
     for (int l = 1; l < k; ++l) {
         off[l] = total;
-        total += (size_t)d->h_hdr.rows_total[l] * m->dims[l];
+        total += (size_t)d->h_hdr.rows_total[l] * m->dims[l] * (f16_inter ? 2 : 4);   // (widths are multiples of 4: 16-byte aligned starts)
     }
     off[k] = 0;   // H^k has buffers of its own
     {
         size_t have = ctx->ws_h_bytes[0] / sizeof(float);
         // a quarter of headroom: the row counts of consecutive calls differ slightly, and growing means a
         // device-wide synchronising free + malloc
-        if (have < total && (rc = mg_ensure(ctx, &ctx->ws_h[0], &have, total + total / 4))) return rc;
+        const size_t need = (total + 3) / 4;
+        if (have < need && (rc = mg_ensure(ctx, &ctx->ws_h[0], &have, need + need / 4))) return rc;
         ctx->ws_h_bytes[0] = have * sizeof(float);
     }
+    char* ws_bytes = reinterpret_cast<char*>(ctx->ws_h[0]);
     int64_t max_x = 0;
     for (int l = 1; l <= k; ++l) {
         const int64_t rows = std::min<int64_t>(chunk_rows_for(m->dims[l - 1]), d->h_hdr.rows_total[l]);
@@ -544,8 +584,8 @@ static int forward_impl(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out,
     for (int l = 1; l <= k; ++l) {
         const int d_in = m->dims[l - 1], d_out = m->dims[l];
         const int64_t M = d->h_hdr.rows_total[l];
-        float* h_out = l == k ? hk : ctx->ws_h[0] + off[l];
-        const float* h_prev = l > 1 ? ctx->ws_h[0] + off[l - 1] : nullptr;
+        float* h_out = l == k ? hk : reinterpret_cast<float*>(ws_bytes + off[l]);
+        const float* h_prev = l > 1 ? reinterpret_cast<const float*>(ws_bytes + off[l - 1]) : nullptr;
         if (m->precision == MG_GEMM_TF32 && mg_layer_fused_supported(d_in, d_out)) {
             // gather + segment mean + both linear maps in one persistent tensor-core kernel (after a small
             // pre-pass that resolves every output row's sources)
@@ -564,7 +604,8 @@ static int forward_impl(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out,
             {
                 ProfScope ps(ctx, l == 1 ? PH_AGG_L1 : PH_AGG_REST, 1);
                 rc = mg_layer_fused(ctx, d, l, d_in, d_out, m->w_pad_t[l - 1], m->bias[l - 1], h_prev, h_out,
-                                    (l < k ? 1 : 0) | (m->sum_aggr ? 2 : 0), meta, 0, M, 0);
+                                    (l < k ? 1 : 0) | (m->sum_aggr ? 2 : 0), meta, 0, M, 0,
+                                    (l == 1 || f16_inter) ? m->w_pad_h[l - 1] : nullptr, f16_inter && l > 1, f16_inter && l < k);
             }
             if (rc) return rc;
             continue;
@@ -666,10 +707,10 @@ extern "C" int mg_layer_output(mg_ctx* ctx, const mg_model* m, mg_dense* d, int3
     if (!ctx->last_hk) return mg_fail(ctx, MG_ERR_STATE, "mg_forward has not run");
     if (!ctx->layers_kept) return mg_fail(ctx, MG_ERR_STATE, "the last forward did not keep its intermediate layers: call mg_keep_layer_outputs(ctx, 1) first");
     MG_CUDA(ctx, cudaSetDevice(ctx->device));
-    size_t off = 0;
-    for (int l = 1; l < layer; ++l) off += (size_t)d->h_hdr.rows_total[l] * m->dims[l];
+    size_t off = 0;   // bytes; the layers were kept as fp32 (layers_kept)
+    for (int l = 1; l < layer; ++l) off += (size_t)d->h_hdr.rows_total[l] * m->dims[l] * 4;
     const int B = d->n_batches;
-    const float* layer_base = layer == d->k ? ctx->last_hk : ctx->ws_h[0] + off;
+    const float* layer_base = layer == d->k ? ctx->last_hk : reinterpret_cast<const float*>(reinterpret_cast<const char*>(ctx->ws_h[0]) + off);
     if (!layer_base) return mg_fail(ctx, MG_ERR_STATE, "mg_forward has not run");
     const float* src = layer_base + (size_t)d->h_rowbase[(size_t)layer * (B + 1) + batch] * m->dims[layer];
     RowExportArgs r;
@@ -1057,6 +1098,7 @@ static int refresh_weight_copies(mg_ctx* ctx, mg_model* m, int l) {
     const size_t di = m->dims[l], dn = m->dims[l + 1];
     k_transpose<<<mg_grid(ctx, 2), kThreads, 0, ctx->stream>>>(m->w_cat[l], m->w_cat_t[l], (int)(2 * di), (int)dn, m->precision == MG_GEMM_TF32);
     ctx->launches++;
+    if (m->w_pad_h[l]) mg_pack_layer_weights_f16(ctx, m->w_cat[l], m->w_pad_h[l], (int)di, (int)dn);
     return mg_pack_layer_weights(ctx, m->w_cat[l], m->w_pad_t[l], (int)di, (int)dn);
 }
 

@@ -76,6 +76,7 @@ struct mg_ctx {
     int32_t* view_nbrs = nullptr;
     int64_t view_edges = 0;
     bool view_owned = false;
+    char* view_ws = nullptr; size_t view_ws_bytes = 0;   // scratch of the view rebuild (keep bits, prefixes, tile bases)
     // second edge list (rows by source) and its in-buffer view; sample_inout = draw from both lists
     int64_t n_edges_out = 0;
     int64_t* row_off_out = nullptr;
@@ -104,7 +105,8 @@ struct mg_ctx {
     int feat_dtype = MG_DTYPE_F32;
     int32_t feat_dim = 0;
     int backing = MG_BACKING_HBM;
-    const char* host_table = nullptr;  // MG_BACKING_HOST
+    const char* host_table = nullptr;  // MG_BACKING_HOST (may be null: then every partition needs a source of its own)
+    std::vector<const char*> part_source;  // MG_BACKING_HOST: host block of a partition when it is not at its place in host_table
     char* slots = nullptr;             // device: slot s at slots + s * slot_bytes
     bool slots_owned = false;
     int32_t n_slots = 0;
@@ -218,7 +220,8 @@ struct mg_dense {
     // asynchronous sampling: the summary lands in pinned memory, ev_sampled marks its arrival
     int32_t* h_pinned = nullptr; size_t h_pinned_ints = 0;
     int32_t* h_pinned_dev = nullptr; // the same memory as the device sees it
-    int32_t* h_stage = nullptr; size_t h_stage_ints = 0;   // pinned: header, offsets, seeds of the call being queued
+    int32_t* h_stage = nullptr; size_t h_stage_ints = 0;   // pinned, mapped: header, offsets, seeds of the call being queued
+    int32_t* h_stage_dev = nullptr;                        // the same memory as the device sees it
     cudaGraphExec_t graph_exec = nullptr;                 // the sampler's device work for graph_sig
     SampleSignature graph_sig;
     int64_t graph_launches = 0;
@@ -237,6 +240,10 @@ struct mg_model {
     float* w_cat[MG_MAX_HOPS] = {nullptr};  // device [2*d_in, d_out]: rows 0..d_in-1 self, then neighbour
     float* w_cat_t[MG_MAX_HOPS] = {nullptr}; // device [d_out, 2*d_in] (K-major copy for the tensor-core path)
     float* w_pad_t[MG_MAX_HOPS] = {nullptr}; // device [d_out, 2*roundup32(d_in)], zero padded, for the fused layer kernel
+    // device fp16 [dims[l+1], 2*roundup64(dims[l])]: a layer's weights for fp16 operands (layer 1 over fp16 base
+    // representations, later layers over fp16 intermediate outputs); null when the weights do not suit fp16
+    void* w_pad_h[MG_MAX_HOPS] = {nullptr};
+    bool f16_intermediates = false;   // store H^1 .. H^{k-1} as fp16 (mg_model_set_intermediates)
     float* bias[MG_MAX_HOPS] = {nullptr};
     // mg_backward: gradients of w_cat and bias (allocated by the first backward pass), a zero vector
     float* g_w_cat[MG_MAX_HOPS] = {nullptr};

@@ -16,6 +16,7 @@
 #include <cuda_fp16.h>
 
 #include <algorithm>
+#include <cstdlib>
 
 #include "mg_device.cuh"
 #include "mg_internal.cuh"
@@ -33,7 +34,16 @@ constexpr int kPlannerWarps = 2;      // after the producers: they prepare the p
 constexpr int kFirstPlannerWarp = kFirstProducerWarp + kProducerWarps;
 constexpr int kFusedThreads = (kFirstPlannerWarp + kPlannerWarps) * 32;  // 768
 constexpr int kMaxStages = 8;
-constexpr int kGroupCols = 128;                  // input columns whose (self, mean) slices the producers fill together
+constexpr int kGroupCols = 128;                  // input columns whose (self, mean) slices the producers fill together (TF32 operands)
+// With half-precision base representations the first layer can run its GEMM in kind::f16 (fp16 operands, fp32
+// accumulate): a 128-byte slice row then holds 64 columns, a lane's 16 bytes are 8 columns, a group is 256 columns,
+// and the same number of MMAs covers twice the K.  Everything else (slices per group, swizzle, stages, barriers) is
+// the same, so the element-size dependent constants come from one place:
+template <bool F16> struct Geo {
+    static constexpr int kKC = F16 ? 64 : 32;        // columns per K slice (one 128-byte swizzle row)
+    static constexpr int kLaneCols = F16 ? 8 : 4;    // columns of a group one lane owns (16 bytes of operand)
+    static constexpr int kGroup = 32 * kLaneCols;    // columns per group
+};
 constexpr int kRowsInFlight = 2;                 // rows a producer warp builds at the same time
 constexpr int kBlockRows = kProducerWarps * kRowsInFlight;   // 32: rows of a tile the producers build in one round
 constexpr int kBlocksPerTile = BM / kBlockRows;              // 4
@@ -77,6 +87,7 @@ struct FusedArgs {
     int32_t tmem_cols;
     int32_t relu;
     int32_t sum_aggr;            // neighbour term = sum of the sampled neighbours instead of their mean
+    int32_t out_f16;             // the output rows are stored as fp16 (an intermediate layer of a model that keeps them so)
     const float* bias;
     float* out;                  // [M, N]
     uint32_t* error;
@@ -102,21 +113,70 @@ __device__ __forceinline__ int32_t source_row(const FusedArgs& a, int32_t in_bas
     return in_base + key;
 }
 
-// 4 consecutive values at p (fp16 values are widened exactly)
-template <bool HALF>
-__device__ __forceinline__ float4 load4(const char* p) {
+// A lane's piece of a source row, as 16 bytes of registers: four fp32 values (fp16 sources widened exactly), or,
+// for fp16 operands (F16), eight fp16 values as they are in memory.
+template <bool HALF, bool F16>
+__device__ __forceinline__ uint4 load_piece(const char* p) {
+    if (F16) return __ldg(reinterpret_cast<const uint4*>(p));
     if (HALF) {
         const uint2 raw = __ldg(reinterpret_cast<const uint2*>(p));
         const float2 lo = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
         const float2 hi = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
-        return make_float4(lo.x, lo.y, hi.x, hi.y);
+        return make_uint4(__float_as_uint(lo.x), __float_as_uint(lo.y), __float_as_uint(hi.x), __float_as_uint(hi.y));
     }
-    return __ldg(reinterpret_cast<const float4*>(p));
+    return __ldg(reinterpret_cast<const uint4*>(p));
 }
 
-template <bool FIRST, bool HALF>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFusedThreads, 1)
+// fp32 running sum of a lane's piece over a row's entries, and the operand forms of the result and of the self row
+template <bool F16> struct PieceSum;
+template <> struct PieceSum<false> {
+    float a[4];
+    __device__ __forceinline__ void zero() { a[0] = a[1] = a[2] = a[3] = 0.f; }
+    __device__ __forceinline__ void add(const uint4& r) {
+        a[0] += __uint_as_float(r.x); a[1] += __uint_as_float(r.y); a[2] += __uint_as_float(r.z); a[3] += __uint_as_float(r.w);
+    }
+    __device__ __forceinline__ uint4 operand(float scale) const {   // rounded to nearest TF32
+        return make_uint4(__float_as_uint(to_tf32(a[0] * scale)), __float_as_uint(to_tf32(a[1] * scale)),
+                          __float_as_uint(to_tf32(a[2] * scale)), __float_as_uint(to_tf32(a[3] * scale)));
+    }
+    static __device__ __forceinline__ uint4 self_operand(const uint4& r) {
+        return make_uint4(__float_as_uint(to_tf32(__uint_as_float(r.x))), __float_as_uint(to_tf32(__uint_as_float(r.y))),
+                          __float_as_uint(to_tf32(__uint_as_float(r.z))), __float_as_uint(to_tf32(__uint_as_float(r.w))));
+    }
+};
+template <> struct PieceSum<true> {
+    float a[8];
+    __device__ __forceinline__ void zero() {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) a[i] = 0.f;
+    }
+    __device__ __forceinline__ void add(const uint4& r) {
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+            a[2 * i] += f.x; a[2 * i + 1] += f.y;
+        }
+    }
+    __device__ __forceinline__ uint4 operand(float scale) const {   // rounded to nearest fp16 (the 10-bit mantissa TF32 keeps)
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const __half2 h = __floats2half2_rn(a[2 * i] * scale, a[2 * i + 1] * scale);
+            w[i] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+        return make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    static __device__ __forceinline__ uint4 self_operand(const uint4& r) { return r; }   // fp16 rows are operands as they are
+};
+
+#ifndef MG_FUSED_MAXNREG
+#define MG_FUSED_MAXNREG 80
+#endif
+template <bool FIRST, bool HALF, bool F16>
+__global__ void __cluster_dims__(2, 1, 1) __maxnreg__(MG_FUSED_MAXNREG)
 k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_out, FusedArgs a) {
+    constexpr int KCE = Geo<F16>::kKC, GC = Geo<F16>::kGroup, LC = Geo<F16>::kLaneCols;
     extern __shared__ uint8_t smem_raw[];
     // a_ready and acc_empty are used in the leader CTA only (both CTAs arrive there); a_free, b_empty and acc_full
     // exist in both CTAs and are signalled in both by the leader's commits; b_full counts both halves' bytes in
@@ -138,10 +198,10 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
     const bool leader = rank == 0;
     const uint32_t pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     const int half_n = a.BN / 2;                  // weight rows (output columns) this CTA stages
-    const uint32_t b_bytes = (uint32_t)half_n * KC * 4;
+    const uint32_t b_bytes = (uint32_t)half_n * 128;   // one 128-byte slice row per staged output column
     uint8_t* a_base = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* b_base = a_base + (size_t)a.sa * kABytes;
-    const int n_chunks = 2 * a.d_in_pad / KC;
+    const int n_chunks = 2 * a.d_in_pad / KCE;
     const int64_t n_tiles = (a.M - a.row_lo + BM - 1) / BM;
     const int64_t n_tile_pairs = (n_tiles + 1) / 2;
     // iteration `it` of this pair works on tile pair (pair + it * n_pairs): the leader on its even tile, the peer
@@ -168,7 +228,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
     const uint32_t acc_stride = (uint32_t)(a.tmem_cols / kAccBufs);  // columns per accumulator buffer (a multiple of 32)
-    const int n_groups = (a.d_in_pad + kGroupCols - 1) / kGroupCols;
+    const int n_groups = (a.d_in_pad + GC - 1) / GC;
 
     if (warp == 0) {
         // ---------------- weight slices: each CTA stages its half of the output columns (TMA from L2) ----------------
@@ -185,7 +245,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                             if (cnt >= (uint32_t)a.sb && !mbar_wait(&b_empty[s], ((cnt / a.sb) - 1) & 1)) { atomicExch(a.error, 11u); ok = false; break; }
                             if (leader) mbar_expect_tx(&b_full[s], 2 * b_bytes);   // both halves are counted on the leader's barrier
                             tma_load_2d_pair(b_base + (size_t)s * b_bytes, &map_w, mapa_u32(smem_u32(&b_full[s]), 0),
-                                             (grp * kSlicesPerGroup + c) * KC, (int)rank * half_n);
+                                             (grp * kSlicesPerGroup + c) * KCE, (int)rank * half_n);
                         }
                     }
         }
@@ -194,7 +254,9 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
         // ---------------- MMA issue: one thread of the leader, for both CTAs ----------------
         if (lane == 0 && leader) {
             // M = 128 over the pair: 64 rows (a half tile) of each CTA per instruction
-            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(a.BN >> 3) << 17) | ((uint32_t)((2 * HM) >> 4) << 24);
+            // fp32 accumulate; operands TF32 (format 2) or fp16 (format 0), both K-major
+            const uint32_t idesc = (1u << 4) | ((F16 ? 0u : 2u) << 7) | ((F16 ? 0u : 2u) << 10) | ((uint32_t)(a.BN >> 3) << 17) |
+                                   ((uint32_t)((2 * HM) >> 4) << 24);
             uint32_t cnt = 0;
             bool ok = true;
             for (uint32_t it = 0; it < my_iters && ok; ++it)
@@ -215,11 +277,13 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                             const int sb = cnt % a.sb;
                             if (!mbar_wait(&b_full[sb], (cnt / a.sb) & 1)) { atomicExch(a.error, 13u); ok = false; break; }
                             tc_fence_after();
-                            const uint64_t da = smem_desc_sw128(smem_u32(a_base + (size_t)c * kABytes + (size_t)h * (HM * KC * 4)));
+                            const uint64_t da = smem_desc_sw128(smem_u32(a_base + (size_t)c * kABytes + (size_t)h * (HM * 128)));
                             const uint64_t db = smem_desc_sw128(smem_u32(b_base + (size_t)sb * b_bytes));
 #pragma unroll
-                            for (int kk = 0; kk < KC / 8; ++kk)
-                                mma_tf32_pair(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (grp | c | kk) ? 1u : 0u);
+                            for (int kk = 0; kk < 4; ++kk) {   // 32 bytes of every slice row per instruction: K = 8 (TF32) or 16 (fp16)
+                                if (F16) mma_f16_pair(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (grp | c | kk) ? 1u : 0u);
+                                else mma_tf32_pair(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (grp | c | kk) ? 1u : 0u);
+                            }
                             mma_commit_pair(&b_empty[sb]);
                         }
                         if (!ok) break;
@@ -234,6 +298,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
         // [BN/2, BN) in lanes 64..127.  Warp quadrant q reads lanes 32q..32q+31.
         const int lane_group = warp & 3;
         const int col_base = (lane_group >> 1) * half_n;
+        const int n_cols = half_n;
         bool ok = true;
         for (uint32_t hu = 0; hu < 2 * my_iters && ok; ++hu) {
             const int64_t t = tile_of(hu >> 1);
@@ -242,13 +307,45 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
             tc_fence_after();
             const int64_t row0 = a.row_lo + t * BM + (hu & 1) * HM + (lane_group & 1) * 32;
             uint8_t* stage = reinterpret_cast<uint8_t*>(out_stage[lane_group]);
-            for (int c0 = 0; c0 < half_n; c0 += 32) {
+            for (int c0 = 0; c0 < n_cols; c0 += 32) {
                 uint32_t v[32];
                 tmem_ld_32(tmem_base + buf * acc_stride + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)c0, v);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 const int ncol0 = col_base + c0;   // first output column of this slice
                 if (row0 >= a.M || ncol0 >= a.N) continue;
-                if (c0 + 32 <= half_n) {
+                if (a.out_f16) {
+                    // fp16 output (widths that are multiples of 128 only): two accumulator slices make one 64-column box,
+                    // 128 bytes per row, so a row of the next layer's input is again fetched in 512-byte requests
+                    const int piece0 = (c0 & 32) ? 4 : 0;
+                    if (!piece0) {
+                        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                        __syncwarp();
+                    }
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const int n = ncol0 + 8 * c;
+                        const float4 b0 = __ldg(reinterpret_cast<const float4*>(a.bias + n)), b1 = __ldg(reinterpret_cast<const float4*>(a.bias + n + 4));
+                        float o[8] = {__uint_as_float(v[8 * c]) + b0.x, __uint_as_float(v[8 * c + 1]) + b0.y, __uint_as_float(v[8 * c + 2]) + b0.z,
+                                      __uint_as_float(v[8 * c + 3]) + b0.w, __uint_as_float(v[8 * c + 4]) + b1.x, __uint_as_float(v[8 * c + 5]) + b1.y,
+                                      __uint_as_float(v[8 * c + 6]) + b1.z, __uint_as_float(v[8 * c + 7]) + b1.w};
+                        uint32_t w[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const __half2 h = a.relu ? __floats2half2_rn(fmaxf(o[2 * i], 0.f), fmaxf(o[2 * i + 1], 0.f)) : __floats2half2_rn(o[2 * i], o[2 * i + 1]);
+                            w[i] = *reinterpret_cast<const uint32_t*>(&h);
+                        }
+                        *reinterpret_cast<uint4*>(stage + lane * 128 + (((piece0 + c) ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                    if (piece0) {
+                        fence_async_smem();
+                        __syncwarp();
+                        if (lane == 0) {
+                            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                                         ::"l"(&map_out), "r"(smem_u32(stage)), "r"(ncol0 - 32), "r"((int)row0) : "memory");
+                            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                        }
+                    }
+                } else if (c0 + 32 <= n_cols) {
                     // the previous slice's TMA store must have read the staging tile before it is rewritten
                     if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                     __syncwarp();
@@ -281,7 +378,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
 #pragma unroll
                         for (int c = 0; c < 8; ++c) {
                             const int n = ncol0 + 4 * c;
-                            if (c0 + 4 * c < half_n && n < a.N) {
+                            if (c0 + 4 * c < n_cols && n < a.N) {
                                 const float4 bb = __ldg(reinterpret_cast<const float4*>(a.bias + n));
                                 float4 o = make_float4(__uint_as_float(v[4 * c]) + bb.x, __uint_as_float(v[4 * c + 1]) + bb.y,
                                                        __uint_as_float(v[4 * c + 2]) + bb.z, __uint_as_float(v[4 * c + 3]) + bb.w);
@@ -313,8 +410,8 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
         for (uint32_t it = 0; it < my_iters; ++it) {
             for (int grp = 0; grp < n_groups; ++grp) {
                 const uint32_t s_h = it * (uint32_t)n_groups + (uint32_t)grp;   // fills of each half's stage rows so far
-                const int pairs = min(kGroupCols / KC, (a.d_in_pad - grp * kGroupCols) / KC);   // slice pairs in this group
-                const int col = grp * kGroupCols + lane * 4;
+                const int pairs = min(GC / KCE, (a.d_in_pad - grp * GC) / KCE);   // slice pairs in this group
+                const int col = grp * GC + lane * LC;
                 const bool lane_on = (lane >> 3) < pairs;
                 const bool col_ok = lane_on && col < a.d_in;
                 const char* src = a.src_base + (size_t)col * (HALF ? 2 : 4);
@@ -331,64 +428,59 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     const int32_t* rows_of = src_rows[slot];
                     const int brow = pw * kRowsInFlight;              // this warp's first row inside the block
                     RowMeta mq[kRowsInFlight];
-                    float4 selfv[kRowsInFlight], acc[kRowsInFlight];
+                    uint4 selfv[kRowsInFlight], meanv[kRowsInFlight];   // the two operand pieces of each row
+                    PieceSum<F16> acc[kRowsInFlight];
                     int top = 0;
 #pragma unroll
                     for (int q2 = 0; q2 < kRowsInFlight; ++q2) {
                         mq[q2] = meta[slot][brow + q2];
-                        selfv[q2] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        acc[q2] = selfv[q2];
+                        selfv[q2] = make_uint4(0u, 0u, 0u, 0u);
+                        meanv[q2] = selfv[q2];
+                        acc[q2].zero();
                         top = max(top, mq[q2].z);
                     }
                     if (col_ok && ok) {
 #pragma unroll
                         for (int q2 = 0; q2 < kRowsInFlight; ++q2)
-                            selfv[q2] = load4<HALF>(src + (size_t)(uint32_t)mq[q2].x * (size_t)a.src_row_bytes);
+                            selfv[q2] = load_piece<HALF, F16>(src + (size_t)(uint32_t)mq[q2].x * (size_t)a.src_row_bytes);
                         if (cached) {
                             // Every load is issued unconditionally: a slot past the end of a row's entries re-reads
                             // the row's own representation (a cache hit) and is not added.  Branch-free code is what
                             // lets all loads of a round be in flight together.  First round: the planner has laid
                             // out the kUnroll source rows per row, padding included.
                             {
-                                float4 v[kRowsInFlight][kUnroll];
+                                uint4 v[kRowsInFlight][kUnroll];
 #pragma unroll
                                 for (int q2 = 0; q2 < kRowsInFlight; ++q2) {
                                     const int4 f4 = *reinterpret_cast<const int4*>(first_rows[slot][brow + q2]);
                                     const int32_t f5 = first_rows[slot][brow + q2][4];
-                                    v[q2][0] = load4<HALF>(src + (size_t)(uint32_t)f4.x * (size_t)a.src_row_bytes);
-                                    v[q2][1] = load4<HALF>(src + (size_t)(uint32_t)f4.y * (size_t)a.src_row_bytes);
-                                    v[q2][2] = load4<HALF>(src + (size_t)(uint32_t)f4.z * (size_t)a.src_row_bytes);
-                                    v[q2][3] = load4<HALF>(src + (size_t)(uint32_t)f4.w * (size_t)a.src_row_bytes);
-                                    v[q2][4] = load4<HALF>(src + (size_t)(uint32_t)f5 * (size_t)a.src_row_bytes);
+                                    v[q2][0] = load_piece<HALF, F16>(src + (size_t)(uint32_t)f4.x * (size_t)a.src_row_bytes);
+                                    v[q2][1] = load_piece<HALF, F16>(src + (size_t)(uint32_t)f4.y * (size_t)a.src_row_bytes);
+                                    v[q2][2] = load_piece<HALF, F16>(src + (size_t)(uint32_t)f4.z * (size_t)a.src_row_bytes);
+                                    v[q2][3] = load_piece<HALF, F16>(src + (size_t)(uint32_t)f4.w * (size_t)a.src_row_bytes);
+                                    v[q2][4] = load_piece<HALF, F16>(src + (size_t)(uint32_t)f5 * (size_t)a.src_row_bytes);
                                 }
 #pragma unroll
                                 for (int j = 0; j < kUnroll; ++j)   // entry order
 #pragma unroll
                                     for (int q2 = 0; q2 < kRowsInFlight; ++q2)
-                                        if (j < mq[q2].z) {
-                                            acc[q2].x += v[q2][j].x; acc[q2].y += v[q2][j].y;
-                                            acc[q2].z += v[q2][j].z; acc[q2].w += v[q2][j].w;
-                                        }
+                                        if (j < mq[q2].z) acc[q2].add(v[q2][j]);
                             }
                             for (int e = kUnroll; e < top; e += kUnroll) {
-                                float4 v[kRowsInFlight][kUnroll];
+                                uint4 v[kRowsInFlight][kUnroll];
 #pragma unroll
                                 for (int j = 0; j < kUnroll; ++j)
 #pragma unroll
                                     for (int q2 = 0; q2 < kRowsInFlight; ++q2) {
                                         const bool live = e + j < mq[q2].z;
                                         const int32_t sr = rows_of[live ? mq[q2].w + e + j : 0];
-                                        v[q2][j] = load4<HALF>(src + (size_t)(uint32_t)(live ? sr : mq[q2].x) * (size_t)a.src_row_bytes);
+                                        v[q2][j] = load_piece<HALF, F16>(src + (size_t)(uint32_t)(live ? sr : mq[q2].x) * (size_t)a.src_row_bytes);
                                     }
 #pragma unroll
                                 for (int j = 0; j < kUnroll; ++j)   // entry order
 #pragma unroll
-                                    for (int q2 = 0; q2 < kRowsInFlight; ++q2) {
-                                        if (e + j < mq[q2].z) {   // warp-uniform: a predicated add, not a branch around a load
-                                            acc[q2].x += v[q2][j].x; acc[q2].y += v[q2][j].y;
-                                            acc[q2].z += v[q2][j].z; acc[q2].w += v[q2][j].w;
-                                        }
-                                    }
+                                    for (int q2 = 0; q2 < kRowsInFlight; ++q2)
+                                        if (e + j < mq[q2].z) acc[q2].add(v[q2][j]);   // warp-uniform: predicated adds, not a branch around a load
                             }
                         } else {
                             // a row block with more entries than the shared-memory cache holds: plain per-entry loop
@@ -397,18 +489,15 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                             for (int q2 = 0; q2 < kRowsInFlight; ++q2)
                                 for (int e = 0; e < mq[q2].z; ++e) {
                                     const int32_t sr = source_row<FIRST>(a, mq[q2].w, __ldg(keys + mq[q2].y + e));
-                                    const float4 v = load4<HALF>(src + (size_t)(uint32_t)sr * (size_t)a.src_row_bytes);
-                                    acc[q2].x += v.x; acc[q2].y += v.y; acc[q2].z += v.z; acc[q2].w += v.w;
+                                    acc[q2].add(load_piece<HALF, F16>(src + (size_t)(uint32_t)sr * (size_t)a.src_row_bytes));
                                 }
                         }
 #pragma unroll
                         for (int q2 = 0; q2 < kRowsInFlight; ++q2) {
                             const float inv = cached ? __int_as_float(first_rows[slot][brow + q2][5])
                                                      : (mq[q2].z > 0 ? (a.sum_aggr ? 1.f : 1.f / (float)mq[q2].z) : 0.f);
-                            acc[q2].x = to_tf32(acc[q2].x * inv); acc[q2].y = to_tf32(acc[q2].y * inv);
-                            acc[q2].z = to_tf32(acc[q2].z * inv); acc[q2].w = to_tf32(acc[q2].w * inv);
-                            selfv[q2].x = to_tf32(selfv[q2].x); selfv[q2].y = to_tf32(selfv[q2].y);
-                            selfv[q2].z = to_tf32(selfv[q2].z); selfv[q2].w = to_tf32(selfv[q2].w);
+                            meanv[q2] = acc[q2].operand(inv);
+                            selfv[q2] = PieceSum<F16>::self_operand(selfv[q2]);
                         }
                     }
                     if (grp == n_groups - 1) {
@@ -435,8 +524,8 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                         for (int q2 = 0; q2 < kRowsInFlight; ++q2) {
                             const int row = blk * kBlockRows + brow + q2;
                             const size_t off = (size_t)(row >> 3) * 1024 + (size_t)(row & 7) * 128 + (size_t)((gl ^ (row & 7)) << 4);
-                            *reinterpret_cast<float4*>(stage_self + off) = selfv[q2];
-                            *reinterpret_cast<float4*>(stage_mean + off) = acc[q2];
+                            *reinterpret_cast<uint4*>(stage_self + off) = selfv[q2];
+                            *reinterpret_cast<uint4*>(stage_mean + off) = meanv[q2];
                         }
                     }
                     if (blk % kBlocksPerHalf == kBlocksPerHalf - 1) {
@@ -544,21 +633,37 @@ __global__ void __launch_bounds__(256) k_layer_rows(FusedArgs a, int4* __restric
     }
 }
 
-__global__ void k_pack_weights(const float* __restrict__ w_cat /*[2 d_in, N]*/, float* __restrict__ w_pad_t /*[N, 2 d_in_pad]*/,
+// slice order of the fused kernel: groups of kGroup input columns; inside a group (self, mean) pairs of kKC-column blocks
+template <bool F16>
+__global__ void k_pack_weights(const float* __restrict__ w_cat /*[2 d_in, N]*/, void* __restrict__ w_pad_t /*[N, 2 d_in_pad]*/,
                                int d_in, int d_in_pad, int N) {
+    constexpr int KCE = Geo<F16>::kKC, GC = Geo<F16>::kGroup;
     const int K = 2 * d_in_pad;
     const int64_t total = (int64_t)N * K;
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
         const int n = (int)(i / K), kx = (int)(i % K);
-        // slice order of the fused kernel: groups of 64 input columns; inside a group (self, mean) pairs of
-        // 32-column blocks
-        const int slice = kx / 32;
-        int grp = 0, rem = slice, pairs = min(kGroupCols / 32, d_in_pad / 32);
-        while (rem >= 2 * pairs) { rem -= 2 * pairs; ++grp; pairs = min(kGroupCols / 32, (d_in_pad - grp * kGroupCols) / 32); }
+        const int slice = kx / KCE;
+        int grp = 0, rem = slice, pairs = min(GC / KCE, d_in_pad / KCE);
+        while (rem >= 2 * pairs) { rem -= 2 * pairs; ++grp; pairs = min(GC / KCE, (d_in_pad - grp * GC) / KCE); }
         const int part = rem & 1;
-        const int col = grp * kGroupCols + (rem >> 1) * 32 + (kx & 31);
-        w_pad_t[i] = col < d_in ? to_tf32(w_cat[(int64_t)(part * d_in + col) * N + n]) : 0.f;
+        const int col = grp * GC + (rem >> 1) * KCE + (kx % KCE);
+        const float w = col < d_in ? w_cat[(int64_t)(part * d_in + col) * N + n] : 0.f;
+        if (F16) reinterpret_cast<__half*>(w_pad_t)[i] = __float2half_rn(w);
+        else reinterpret_cast<float*>(w_pad_t)[i] = to_tf32(w);
     }
+}
+
+// row-major [rows, K] fp16 matrix, boxes of 64 halves x box_rows, 128-byte swizzle, zero fill
+static bool make_map_f16(CUtensorMap* map, const void* base, int64_t rows, int K, int box_rows) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    const cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace
@@ -566,7 +671,16 @@ __global__ void k_pack_weights(const float* __restrict__ w_cat /*[2 d_in, N]*/, 
 // K-major, zero-padded, TF32-rounded copy of [W_self ; W_nbr] for the fused layer kernel
 int mg_pack_layer_weights(mg_ctx* ctx, const float* w_cat_dev, float* w_pad_t_dev, int d_in, int N) {
     const int d_in_pad = (d_in + KC - 1) / KC * KC;
-    k_pack_weights<<<mg_grid(ctx, 2), 256, 0, ctx->stream>>>(w_cat_dev, w_pad_t_dev, d_in, d_in_pad, N);
+    k_pack_weights<false><<<mg_grid(ctx, 2), 256, 0, ctx->stream>>>(w_cat_dev, w_pad_t_dev, d_in, d_in_pad, N);
+    ctx->launches++;
+    return MG_OK;
+}
+
+// The same rounded to fp16 (64-column slices), [N, 2 * roundup64(d_in)] halves: the first layer's weights when the base
+// representations are fp16 and the layer's GEMM runs on fp16 operands
+int mg_pack_layer_weights_f16(mg_ctx* ctx, const float* w_cat_dev, void* w_pad_h_dev, int d_in, int N) {
+    const int d_in_pad = (d_in + 63) / 64 * 64;
+    k_pack_weights<true><<<mg_grid(ctx, 2), 256, 0, ctx->stream>>>(w_cat_dev, w_pad_h_dev, d_in, d_in_pad, N);
     ctx->launches++;
     return MG_OK;
 }
@@ -611,7 +725,7 @@ int mg_layer_rows(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_out
 // GLOBAL packed row (callers that keep only a window of a layer pass pointers shifted accordingly).
 int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_out, const float* w_pad_t, const float* bias,
                    const float* h_prev, float* h_out, int flags, const int4* row_meta, int64_t row_lo, int64_t row_hi,
-                   int64_t safe_src_row) {
+                   int64_t safe_src_row, const void* w_pad_h, int in_f16, int out_f16) {
     if (row_hi <= row_lo) return MG_OK;
     FusedArgs a;
     memset(&a, 0, sizeof(a));
@@ -622,30 +736,40 @@ int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_ou
     a.safe_src = (int32_t)safe_src_row;
     a.h_prev = h_prev;
     a.src_base = layer == 1 ? ctx->slots : reinterpret_cast<const char*>(h_prev);
-    a.src_row_bytes = layer == 1 ? (uint32_t)ctx->row_bytes : (uint32_t)d_in * 4u;
+    a.src_row_bytes = layer == 1 ? (uint32_t)ctx->row_bytes : (uint32_t)d_in * (in_f16 ? 2u : 4u);
+    a.out_f16 = out_f16;
     a.relu = flags & 1;
     a.sum_aggr = (flags >> 1) & 1;
     a.bias = bias; a.out = h_out;
+    // fp16 operands: first layer over fp16 base representations, mean aggregator (a sum of fp16 values may leave the
+    // fp16 range), weights given in fp16 form (the caller withholds them when they do not suit fp16)
+    // (later layers: in_f16 says that H^{l-1} was stored as fp16; the caller only does that with fp16 weights at hand)
+    const bool f16 = (layer == 1 ? ctx->feat_dtype == MG_DTYPE_F16 : in_f16 != 0) && w_pad_h && !a.sum_aggr;
+    if (layer > 1 && in_f16 && !f16) return mg_fail(ctx, MG_ERR_STATE, "fp16 layer input without fp16 operands");
+    if (out_f16 && d_out % 128 != 0) return mg_fail(ctx, MG_ERR_STATE, "fp16 layer outputs need widths that are multiples of 128");
+    const int kce = f16 ? 64 : KC;
+    a.d_in_pad = (d_in + kce - 1) / kce * kce;
     int stride = 32;
     while (stride < a.BN / 2) stride <<= 1;
     a.tmem_cols = kAccBufs * stride;   // accumulator buffers of half tiles: BN / 2 columns each, a power of two >= 32
-    const int b_bytes = (a.BN / 2) * KC * 4;    // each CTA of a pair stages half of the output columns
-    const int n_chunks = 2 * a.d_in_pad / KC;
+    const int b_bytes = (a.BN / 2) * 128;       // each CTA of a pair stages half of the output columns
+    const int n_chunks = 2 * a.d_in_pad / kce;
     a.sa = std::min(8, n_chunks);   // one group of (self, mean) slice pairs: 128 input columns
     // A shallow weight ring (32 KB) on purpose: with 128 KB of A stages the CTA then fits the 196 KB shared-memory
     // carve-out, which leaves the gathers twice the L1 (measured: layer 1 of the bench 2.92 -> 2.75 ms).
     a.sb = std::max(2, std::min({kMaxStages, n_chunks, (32 * 1024) / b_bytes}));
     const size_t smem = (size_t)a.sa * kABytes + (size_t)a.sb * b_bytes + 1024;
     CUtensorMap mw;
-    if (!make_map_f32(&mw, w_pad_t, d_out, 2 * a.d_in_pad, a.BN / 2))
+    if (!(f16 ? make_map_f16(&mw, w_pad_h, d_out, 2 * a.d_in_pad, a.BN / 2) : make_map_f32(&mw, w_pad_t, d_out, 2 * a.d_in_pad, a.BN / 2)))
         return mg_fail(ctx, MG_ERR_CUDA, "cuTensorMapEncodeTiled failed for the layer weights");
     // output [row_hi rows, d_out] fp32, 32 x 32 boxes, 128-byte swizzle; rows are global packed rows, so a window's
     // shifted base pointer works unchanged (rows below row_lo are never stored)
     CUtensorMap mo;
-    if (!make_map_f32(&mo, h_out, row_hi, d_out, 32))
+    if (!(out_f16 ? make_map_f16(&mo, h_out, row_hi, d_out, 32) : make_map_f32(&mo, h_out, row_hi, d_out, 32)))
         return mg_fail(ctx, MG_ERR_CUDA, "cuTensorMapEncodeTiled failed for the layer output");
     const bool first = layer == 1, half = first && ctx->feat_dtype == MG_DTYPE_F16;
-    auto kern = first ? (half ? k_sage_layer_fused<true, true> : k_sage_layer_fused<true, false>) : k_sage_layer_fused<false, false>;
+    auto kern = first ? (f16 ? k_sage_layer_fused<true, true, true> : half ? k_sage_layer_fused<true, true, false> : k_sage_layer_fused<true, false, false>)
+                      : (f16 ? k_sage_layer_fused<false, true, true> : k_sage_layer_fused<false, false, false>);
     MG_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const int64_t n_tiles = (row_hi - row_lo + BM - 1) / BM;
     const int grid = 2 * (int)std::min<int64_t>((n_tiles + 1) / 2, ctx->n_sms / 2);   // CTA pairs

@@ -127,6 +127,26 @@ struct TableGeom {
     int32_t size;   // slots per batch (any size)
 };
 
+// The host-known part of a sample (header, target offsets, per-batch row tables, seeds) is read straight from mapped
+// pinned memory by a kernel instead of being copied by a copy engine: a copy engine may be busy for a long time with
+// a partition that is being swapped in, and the sample would wait behind it.
+__global__ void __launch_bounds__(kThreads)
+k_stage_in(const int32_t* __restrict__ stage, int32_t n_hdr, int32_t n_off, int32_t n_cum, int32_t n_seed_words, int32_t seed_at,
+           int32_t* hdr, int32_t* node_off, int32_t* cum, int32_t* seeds) {
+    const int32_t total = n_hdr + n_off + n_cum + n_seed_words;
+    for (int32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+        int32_t j = i;
+        if (j < n_hdr) hdr[j] = stage[j];
+        else if ((j -= n_hdr) < n_off) node_off[j] = stage[n_hdr + j];
+        else if ((j -= n_off) < n_cum) cum[j] = stage[n_hdr + n_off + j];
+        else seeds[j - n_cum] = stage[seed_at + (j - n_cum)];
+    }
+}
+
+__global__ void __launch_bounds__(kThreads) k_copy_i32(const int32_t* __restrict__ src, int32_t* dst, int64_t n) {
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) dst[i] = src[i];
+}
+
 __global__ void __launch_bounds__(kThreads)
 k_init_targets(DenseHeader* hdr, const int32_t* __restrict__ targets,
                const int32_t* __restrict__ tgt_off, int32_t B, int32_t* nodes, int32_t* node_batch,
@@ -1480,7 +1500,8 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
     if (d->h_stage_ints < n_stage_ints) {
         if (d->h_stage) cudaFreeHost(d->h_stage);
         d->h_stage = nullptr; d->h_stage_ints = 0;
-        if (cudaHostAlloc((void**)&d->h_stage, n_stage_ints * sizeof(int32_t), cudaHostAllocDefault) != cudaSuccess) {
+        if (cudaHostAlloc((void**)&d->h_stage, n_stage_ints * sizeof(int32_t), cudaHostAllocMapped) != cudaSuccess ||
+            cudaHostGetDevicePointer((void**)&d->h_stage_dev, d->h_stage, 0) != cudaSuccess) {
             cudaGetLastError();
             return mg_fail(ctx, MG_ERR_OOM, "pinned host allocation failed");
         }
@@ -1513,19 +1534,25 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
     sample_kernel_attributes();
 
     // the targets are staged in newlist[1] (outside the graph: their source changes from call to call)
-    if (T > 0)
-        MG_CUDA(ctx, cudaMemcpyAsync(d->newlist[1], targets, sizeof(int32_t) * T,
-                                     targets_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, st));
+    if (T > 0) {
+        if (targets_on_device) {
+            k_copy_i32<<<std::max(1, std::min(mg_grid(ctx, 2), (int)((T + kThreads - 1) / kThreads))), kThreads, 0, st>>>(targets, (int32_t*)d->newlist[1], T);
+            ctx->launches++;
+        } else {
+            MG_CUDA(ctx, cudaMemcpyAsync(d->newlist[1], targets, sizeof(int32_t) * T, cudaMemcpyHostToDevice, st));
+        }
+    }
     const int32_t* tgt_dev = (const int32_t*)d->newlist[1];
 
     // ---- everything the device does for this sample ----
     auto enqueue = [&]() -> int {
     {
         ProfScope ps(ctx, PH_SAMPLE_INIT, 1);
-        MG_CUDA(ctx, cudaMemcpyAsync(d->hdr, st_hdr, sizeof(DenseHeader), cudaMemcpyHostToDevice, st));
-        MG_CUDA(ctx, cudaMemcpyAsync(d->node_off, st_off, sizeof(int32_t) * (B + 1), cudaMemcpyHostToDevice, st));
-        MG_CUDA(ctx, cudaMemcpyAsync(d->cum, st_cum, sizeof(int32_t) * (size_t)B * (k + 2), cudaMemcpyHostToDevice, st));
-        MG_CUDA(ctx, cudaMemcpyAsync(d->d_seeds, st_seeds, sizeof(uint64_t) * B, cudaMemcpyHostToDevice, st));
+        static_assert(sizeof(DenseHeader) % 4 == 0, "the header is staged as 32-bit words");
+        k_stage_in<<<4, kThreads, 0, st>>>(d->h_stage_dev, (int32_t)(sizeof(DenseHeader) / 4), B + 1, B * (k + 2), 2 * B,
+                                          (int32_t)(reinterpret_cast<int32_t*>(st_seeds) - d->h_stage), reinterpret_cast<int32_t*>(d->hdr),
+                                          d->node_off, d->cum, reinterpret_cast<int32_t*>(d->d_seeds));
+        ctx->launches++;
         MG_CUDA(ctx, cudaMemsetAsync(d->hkeys, 0xFF, sizeof(int32_t) * (size_t)B * table_size, st));
         {
             k_init_targets<<<mg_grid(ctx, 4), kThreads, 0, st>>>(d->hdr, tgt_dev, d->node_off, B, d->nodes,
@@ -1633,7 +1660,7 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
     for (int h = 0; h < k; ++h) sig.fanouts[h] = fanouts[h];
     const void* ptrs[] = {d->hdr, d->nodes, d->node_batch, d->ent_off, d->node_r0, d->node_deg, d->newlist[0], d->newlist[1],
                           d->scan_tmp, d->sort_hist, d->ent_nbrs, d->ent_repr, d->hkeys, d->hvals, d->node_off, d->cum, d->rowbase,
-                          d->d_ent_hop, d->d_seeds, d->h_stage, d->h_pinned_dev, ctx->view_off, ctx->view_nbrs, ctx->d_slot_of_part, st,
+                          d->d_ent_hop, d->d_seeds, d->h_stage_dev, d->h_pinned_dev, ctx->view_off, ctx->view_nbrs, ctx->d_slot_of_part, st,
                           inout ? (const void*)ctx->view_off_out : nullptr, inout ? (const void*)ctx->view_nbrs_out : nullptr,
                           d->node_r0_out, d->node_deg_out, d->pairs, d->share_off};
     static_assert(sizeof(ptrs) <= sizeof(sig.ptrs), "signature too small");

@@ -169,6 +169,23 @@ def normal_features(n_nodes: int, dim: int, seed: int, device="cpu",
     return out
 
 
+def block_features(n_rows: int, dim: int, seed: int, block: int, device="cpu", dtype=torch.float32, std: float = 1.0,
+                   out: torch.Tensor | None = None, chunk_rows: int = 1 << 20) -> torch.Tensor:
+    """N(0, std^2) rows of ONE partition block, a pure function of (seed, block, device type): any block of a table
+    that is too large to keep (config 4: 187 GB) can be made again on its own, for the partition buffer's staging
+    blocks and for the oracle's H^0 rows alike.  `out` (any device, e.g. a pinned host block) receives the rows."""
+    g = _gen(int(seed) * 1_000_003 + int(block), device)
+    if out is None:
+        out = torch.empty((n_rows, dim), dtype=dtype, device=device)
+    for lo in range(0, n_rows, chunk_rows):
+        hi = min(n_rows, lo + chunk_rows)
+        blk = torch.randn((hi - lo, dim), generator=g, device=device, dtype=torch.float32)
+        if std != 1.0:
+            blk *= std
+        out[lo:hi].copy_(blk.to(dtype))
+    return out
+
+
 def glorot_layers(dims, seed: int):
     """GraphSage weights for widths dims[0] -> dims[1] -> ...; Glorot-uniform, bias 0.
 

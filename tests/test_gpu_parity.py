@@ -425,6 +425,75 @@ def test_tensor_core_linear_layer_shapes(d_in, d_out):
         close(out.cpu().numpy(), want, rtol)
 
 
+@pytest.mark.parametrize("d_in,d_out,fanout", [(8, 16, 6), (72, 100, 6), (256, 256, 6), (264, 64, 3), (768, 256, 6), (200, 36, 30)])
+def test_first_layer_on_fp16_operands(d_in, d_out, fanout):
+    """Half-precision base representations: the first layer's GEMM runs on fp16 operands (fp16 rows as they are, the
+    mean and the weights rounded to fp16, fp32 accumulate).  Widths below one 64-column slice, ragged slices, one and
+    several 256-column groups, rows past the entry cache (fanout 30); a second layer on TF32 operands behind it; the
+    sum aggregator and weights outside fp16's comfortable range keep TF32 operands and must agree as well."""
+    n = 5000
+    g = inputs.rmat_graph(n, 60_000, seed=11)
+    feats = inputs.normal_features(n, d_in, seed=12).half()
+    ctx = make_ctx(g, feats)
+    targets = inputs.distinct_targets(n, 777, seed=13)
+    d = ctx.sample(targets, [fanout, 4], seed=3)
+    ref = O.sample_dense(oracle_view(g), targets.tolist(), [fanout, 4], 3)
+    assert_dense_equal(d.view(0), ref)
+    h0 = feats.float().numpy()[ref["node_ids"]]
+    out = torch.empty((777, 8), dtype=torch.float32, device="cuda")
+    for scale, aggregator in ((1.0, "mean"), (1.0, "sum"), (1e-5, "mean")):
+        layers = inputs.random_bias_layers([d_in, d_out, 8], seed=14)
+        layers[0] = (layers[0][0] * scale, layers[0][1] * scale, layers[0][2] * scale)
+        np_layers = [(w.numpy(), nn.numpy(), b.numpy()) for w, nn, b in layers]
+        model = ctx.model(layers, mg.GEMM_TF32)
+        model.set_aggregator(aggregator)
+        ctx.keep_layer_outputs(True)
+        ctx.forward(model, d, out)
+        outs = O.forward(ref, h0, np_layers, return_all=True, aggregator=aggregator)
+        close(ctx.layer_output(model, d, 1, 0, outs[0].shape[0]).cpu().numpy(), outs[0], RTOL_TC)
+        close(out.cpu().numpy(), outs[1], RTOL_TC)
+        ctx.keep_layer_outputs(False)
+
+
+@pytest.mark.parametrize("dims", [[128, 256, 256, 256], [64, 128, 128], [16, 128, 100, 128, 8]])
+def test_fp16_intermediate_layer_outputs(dims):
+    """The model option that keeps H^1 .. H^{k-1} as fp16 inside the forward pass: H^k within the tensor-core tolerance
+    of the fp64 oracle, several mini-batches with ragged tiles; where the option cannot apply (an intermediate width
+    that is not a multiple of 128, kept layer outputs, the sum aggregator) the fp32 path answers, equally checked."""
+    n = 30_000
+    g = inputs.rmat_graph(n, 600_000, seed=21)
+    feats = inputs.normal_features(n, dims[0], seed=22)
+    ctx = make_ctx(g, feats)
+    k = len(dims) - 1
+    fanouts = [6, 4, 3, 2][:k]
+    sizes = [300, 1, 257]
+    tg = [inputs.distinct_targets(n, s_, seed=23 + i) for i, s_ in enumerate(sizes)]
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    seeds = [7, 8, 9]
+    d = ctx.sample_many(torch.cat(tg), offs, fanouts, seeds)
+    layers = inputs.random_bias_layers(dims, seed=24)
+    np_layers = [(w.numpy(), nn.numpy(), b.numpy()) for w, nn, b in layers]
+    view = oracle_view(g)
+    refs = [O.sample_dense(view, tg[b].tolist(), fanouts, seeds[b]) for b in range(3)]
+    model = ctx.model(layers, mg.GEMM_TF32)
+    out32 = torch.empty((int(offs[-1]), dims[-1]), dtype=torch.float32, device="cuda")
+    ctx.forward(model, d, out32)
+    model.set_intermediates(torch.float16)
+    for aggregator, keep in (("mean", False), ("mean", True), ("sum", False)):
+        model.set_aggregator(aggregator)
+        ctx.keep_layer_outputs(keep)
+        out = torch.full_like(out32, float("nan"))
+        ctx.forward(model, d, out)
+        for b in range(3):
+            want = O.forward(refs[b], feats.numpy()[refs[b]["node_ids"]], np_layers, aggregator=aggregator)
+            close(out[offs[b]:offs[b + 1]].cpu().numpy(), want, RTOL_TC)
+        if aggregator == "mean" and not keep and all(w % 128 == 0 for w in dims[1:-1]):
+            assert not torch.equal(out, out32)          # the fp16 path really ran (its rounding differs)
+            with pytest.raises(mg.MgError):
+                ctx.layer_output(model, d, 1, 0, 1)       # and kept no fp32 layer outputs
+    ctx.keep_layer_outputs(False)
+
+
 def test_config2_shaped_power_law_three_layers():
     """R-MAT, dim 128, hidden 256, fanouts [15, 10, 5], batches of 1000 (config 2 at 1/5 scale so
     the oracle finishes in seconds); hub rows, zero-degree nodes, several batches per pass."""
@@ -581,50 +650,86 @@ def test_full_size_config3_in_bench_launch_configuration():
     _check_batches_against_oracle(g_host, feats, layers, cfg["fanouts"], tg, seeds, d, out2, offs2, [G2 - 1], RTOL_TC)
 
 
-def test_config4_shaped_out_of_core_fp16_swaps():
-    """Config 4's path at 1/10 of its node count (the full fp16 x 768 table is 187 GB of pinned host
-    memory; the test box has 196 GB of RAM): R-MAT 12.2M nodes / 130M edges, fp16 features of width 768
-    kept in pinned host memory, 32 partitions with a 10-partition HBM buffer, swaps prefetched on the
-    side stream while batches run on the current set, only resident edges sampled."""
-    n, m, parts, cap, dim = 12_200_000, 130_000_000, 32, 10, 768
-    g = inputs.rmat_graph(n, m, seed=41, device="cuda")
-    feats = torch.empty((n, dim), dtype=torch.float16).pin_memory()
-    gen = torch.Generator(device="cuda"); gen.manual_seed(42)
-    for lo in range(0, n, 1 << 20):
-        hi = min(n, lo + (1 << 20))
-        feats[lo:hi].copy_(torch.randn((hi - lo, dim), generator=gen, device="cuda").half())
+def test_config4_out_of_core_at_its_stated_size():
+    """Config 4 as stated: R-MAT 122M nodes / 1.30B edges, fp16 features of width 768, 32 partitions with a
+    10-partition HBM buffer, in the launch configuration of bench.py's out-of-core workload.  The 187 GB table is never
+    held: a partition block is a pure function of (seed, block), made into a pinned staging block when the buffer asks
+    for it and made again for the oracle's H^0 rows.  Three buffer states of the random one-swap order; the next
+    state's block is copied on the side stream while the current state's mini-batches run; only edges with both
+    endpoints resident are sampled; one mini-batch per state is checked against the oracle."""
+    import bench
+    c = bench.OOC_CONFIG
+    free, _ = torch.cuda.mem_get_info()
+    if free < 110 * (1 << 30):
+        pytest.skip("needs a GPU with 110 GB free")
+    n, parts, cap, dim = c["n"], c["parts"], c["cap"], c["dim"]
+    g = inputs.rmat_graph(n, c["m"], seed=40, device="cuda")
     ctx = mg.Context(0)
     ctx.load_graph(g.row_offsets, g.nbrs)
     g_host = (g.row_offsets.cpu().numpy(), g.nbrs.cpu().numpy())
     del g
+    torch.cuda.empty_cache()
     ctx.set_partitioning(parts)
-    ctx.load_features(feats, capacity_parts=cap, backing=mg.BACKING_HOST)
-    layers = inputs.glorot_layers([dim, 256, 256, 256], seed=43)
-    model = ctx.model(layers, mg.GEMM_TF32)
-    states = inputs.swap_order(parts, cap, seed=44)[:4]
-    ctx.set_resident(states[0])
+    ctx.load_features(None, capacity_parts=cap, backing=mg.BACKING_HOST, dtype=torch.float16, dim=dim)
+    part_rows = inputs.contiguous_partition(n, parts)
+    rows_of = lambda p: min(part_rows, n - p * part_rows)
+    staging = [torch.empty((part_rows, dim), dtype=torch.float16).pin_memory() for _ in range(2)]
+
+    def stage(p, slot):
+        inputs.block_features(rows_of(p), dim, 41, p, device="cuda", dtype=torch.float16, out=staging[slot][:rows_of(p)])
+        torch.cuda.synchronize()
+        return staging[slot]
+
+    with pytest.raises(mg.MgError) as e:
+        ctx.set_resident([3])                       # no table and no block named for partition 3
+    assert e.value.code == -2
+    states = inputs.swap_order(parts, cap, seed=44)[:3]
+    for i, p in enumerate(states[0]):
+        ctx.set_partition_source(p, stage(p, 0))
+        ctx.set_resident(sorted(states[0][:i + 1]))
+    layers = inputs.glorot_layers([dim] + [c["hidden"]] * 3, seed=43)
     np_layers = [(w.numpy(), nn.numpy(), b.numpy()) for w, nn, b in layers]
-    B, T = 8, 1000
-    offs = [T * i for i in range(B + 1)]
+    model = ctx.model(layers, mg.GEMM_TF32)
+    G, T = c["group"], c["batch"]
+    offs = [T * i for i in range(G + 1)]
+
+    def oracle_h0(node_ids):
+        ids = torch.as_tensor(node_ids, dtype=torch.int64)
+        h0 = torch.empty((ids.numel(), dim), dtype=torch.float32)
+        part = ids // part_rows
+        for p in torch.unique(part).tolist():
+            block = inputs.block_features(rows_of(p), dim, 41, p, device="cuda", dtype=torch.float16)
+            sel = torch.nonzero(part == p).flatten()
+            h0[sel] = block[(ids[sel] - p * part_rows).cuda()].float().cpu()
+            del block
+        return h0.numpy()
+
     for step, resident in enumerate(states):
         if step + 1 < len(states):
-            ctx.set_resident(states[step + 1], async_=True)      # prefetch the next set on the side stream
-        mask = inputs.resident_node_mask(n, parts, resident)
-        pool = torch.nonzero(mask).flatten()
-        tg = torch.stack([inputs.distinct_targets(pool, T, seed=100 * step + b) for b in range(B)])
-        seeds = [1000 * step + b for b in range(B)]
-        d = ctx.sample_many(tg.reshape(-1), offs, [15, 10, 5], seeds)
-        out = torch.empty((B * T, 256), dtype=torch.float32, device="cuda")
+            q = [p for p in states[step + 1] if p not in resident][0]
+            ctx.set_partition_source(q, stage(q, 1))
+            ctx.set_resident(states[step + 1], async_=True)      # the incoming block loads on the side stream
+        pool = torch.nonzero(inputs.resident_node_mask(n, parts, resident, device="cuda")).flatten().to(torch.int32)
+        gen = torch.Generator(device="cuda"); gen.manual_seed(500 + step)
+        tg = pool[torch.randperm(pool.numel(), generator=gen, device="cuda")[:G * T]].reshape(G, T)
+        seeds = [1000 * step + b for b in range(G)]
+        probe = ctx.sample_many(tg.reshape(-1), offs, c["fanouts"], seeds, caps={"max_nodes_per_batch": 1 << 19})
+        nodes, ents = probe.counts()
+        caps = {"max_nodes_total": int(nodes.sum() * 1.4) + 1024, "max_entries_total": int(ents.sum() * 1.4) + 1024,
+                "max_nodes_per_batch": int(nodes.sum(1).max() * 1.6) + 64}
+        probe.free()
+        d = ctx.sample_many(tg.reshape(-1), offs, c["fanouts"], seeds, caps=caps)
+        out = torch.empty((G * T, c["hidden"]), dtype=torch.float32, device="cuda")
         ctx.forward(model, d, out)
         view = O.GraphView(g_host[0], g_host[1], parts, resident)
-        b = step % B
-        ref = O.sample_dense(view, tg[b].tolist(), [15, 10, 5], seeds[b])
+        b = (17 * step + 5) % G
+        ref = O.sample_dense(view, tg[b].tolist(), c["fanouts"], seeds[b])
         assert_dense_equal(d.view(b), ref)
         assert all(view.is_resident(u) for u in ref["node_ids"][::97])
-        want = O.forward(ref, feats[torch.as_tensor(ref["node_ids"])].float().numpy(), np_layers)
-        close(out[offs[b]:offs[b + 1]].cpu().numpy(), want, RTOL_TC)
+        close(out[offs[b]:offs[b + 1]].cpu().numpy(), O.forward(ref, oracle_h0(ref["node_ids"]), np_layers), RTOL_TC)
+        d.free()
         if step + 1 < len(states):
-            ctx.commit_resident(60_000)
+            ctx.commit_resident(120_000)
 
 
 def test_config5_shaped_link_prediction_full_graph():
