@@ -46,6 +46,9 @@ CONFIGS = {
     # layer-1 kernel's DRAM traffic per unit is captured here (profiles/k_sage_layer_fused_dram_traffic.md)
     "probe_rmat_8m_dim128": dict(n=8_000_000, m=160_000_000, kind="rmat", dim=128, hidden=256, fanouts=[15, 10, 5],
                                  batch=1000, parts=1, train=8_000_000),
+    # the same idea for the fp16-operand variant of that kernel (half-precision rows of 1,536 bytes, 3 GB table)
+    "probe_rmat_2m_fp16_768": dict(n=2_000_000, m=40_000_000, kind="rmat", dim=768, hidden=256, fanouts=[15, 10, 5],
+                                   batch=1000, parts=1, train=2_000_000, fp16=True, group=32),
     # config 4's shapes at a tenth of its node count, whole fp16 table in HBM (no swaps): a throughput probe of the
     # wide fp16 layer-1 path, not the out-of-core configuration itself (that one is exercised by the tests)
     "config4_tenth_fp16_768_in_hbm": dict(n=12_200_000, m=130_000_000, kind="rmat", dim=768, hidden=256,

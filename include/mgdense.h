@@ -126,10 +126,17 @@ int mg_load_out_graph(mg_ctx* ctx, int64_t n_edges, const void* row_offsets, int
 #define MG_SAMPLE_INOUT 1
 int mg_set_sample_direction(mg_ctx* ctx, int direction);
 
-/* Split the nodes into n_parts physical partitions of ceil(n_nodes / n_parts) contiguous
- * ids (the last one short) — the sequential lookup table of Section 3.  All partitions
- * start non-resident except when n_parts == 1.  Drops any loaded feature table. */
-int mg_set_partitioning(mg_ctx* ctx, int32_t n_parts);
+/* Split the nodes into n_parts physical partitions (Section 3).  part_of_node = NULL: ceil(n_nodes / n_parts)
+ * contiguous ids each (the last one short) -- the sequential lookup table cut into pieces.  part_of_node != NULL: a
+ * HOST array of n_nodes partition ids (< n_parts), copied -- the partition-id array of the graph store; Section 5.2's
+ * policy (training nodes in the first partitions, the others assigned at random) is expressed this way.  A node's place
+ * inside its partition is its rank among the partition's nodes in ascending id.  With MG_BACKING_HOST the host table
+ * (or the blocks named by mg_set_partition_source) is then partition-major: partition 0's rows in that order, then
+ * partition 1's, ...; with MG_BACKING_HBM the table stays in node order.  Buffer slots hold the largest partition.
+ * Negatives of mg_lp_prepare count resident nodes partition after partition, ascending id inside a partition.
+ * All partitions start non-resident except when n_parts == 1.  Drops any loaded feature table.
+ * Errors: MG_ERR_ARG (n_parts outside [1, MG_MAX_PARTS], an id >= n_parts), MG_ERR_STATE, MG_ERR_OOM. */
+int mg_set_partitioning(mg_ctx* ctx, int32_t n_parts, const uint8_t* part_of_node);
 
 /* Attach the table of base representations (Section 2): n_nodes rows of `dim` values of
  * `dtype`, row-major.  dim * sizeof(dtype) must be a multiple of 16 bytes.

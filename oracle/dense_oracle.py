@@ -97,11 +97,13 @@ class GraphView:
     """The in-memory subgraph: CSR rows restricted to resident endpoints.
 
     Section 3: sampling sees only nodes and edges of partitions in the buffer.
-    Partitions are contiguous id ranges of `part_size` nodes.
+    Partitions are contiguous id ranges of `part_size` nodes, or, with `part_of_node`
+    (one partition id per node), whatever that array says -- Section 5.2 places the
+    training nodes in the first partitions and assigns the others at random.
     """
 
     def __init__(self, row_offsets, nbrs, n_parts: int = 1, resident_parts=None,
-                 out_row_offsets=None, out_nbrs=None):
+                 out_row_offsets=None, out_nbrs=None, part_of_node=None):
         self.row_offsets = np.asarray(row_offsets, dtype=np.int64)
         self.nbrs = np.asarray(nbrs)
         # optional second edge list, sorted by source: row v = destinations of v's outgoing edges
@@ -110,51 +112,64 @@ class GraphView:
         self.n_nodes = len(self.row_offsets) - 1
         self.n_parts = int(n_parts)
         self.part_size = (self.n_nodes + self.n_parts - 1) // self.n_parts
+        self.part_of_node = None if part_of_node is None else np.asarray(part_of_node, dtype=np.int64)
+        if self.part_of_node is not None:
+            assert len(self.part_of_node) == self.n_nodes and self.part_of_node.max(initial=0) < self.n_parts
         if resident_parts is None:
             resident_parts = range(self.n_parts)
         self.resident_parts = sorted(int(p) for p in resident_parts)
         self._res = set(self.resident_parts)
+        self._members = {}
+
+    def part(self, u):
+        """Partition of node u (or of every node of an array)."""
+        if self.part_of_node is not None:
+            return self.part_of_node[u]
+        return u // self.part_size
+
+    def nodes_of_part(self, p: int):
+        """Ids of partition p's nodes, ascending (a range for the contiguous split, else an array, made once)."""
+        if self.part_of_node is None:
+            return range(p * self.part_size, min((p + 1) * self.part_size, self.n_nodes))
+        if p not in self._members:
+            self._members[p] = np.nonzero(self.part_of_node == p)[0]
+        return self._members[p]
 
     def is_resident(self, u: int) -> bool:
-        return (int(u) // self.part_size) in self._res
+        return int(self.part(int(u))) in self._res
+
+    def _filter(self, r):
+        if len(self._res) == self.n_parts:
+            return r
+        return r[np.isin(self.part(r), self.resident_parts)]
 
     def row(self, v: int):
         """R(v): the stored row of v, in stored order, resident neighbours only."""
-        r = self.nbrs[self.row_offsets[v]:self.row_offsets[v + 1]]
-        if len(self._res) == self.n_parts:
-            return r
-        keep = np.isin(r // self.part_size, self.resident_parts)
-        return r[keep]
+        return self._filter(self.nbrs[self.row_offsets[v]:self.row_offsets[v + 1]])
 
     def out_row(self, v: int):
         """The outgoing row of v (second edge list), resident neighbours only."""
         if self.out_row_offsets is None:
             raise ValueError("no outgoing edge list")
-        r = self.out_nbrs[self.out_row_offsets[v]:self.out_row_offsets[v + 1]]
-        if len(self._res) == self.n_parts:
-            return r
-        keep = np.isin(r // self.part_size, self.resident_parts)
-        return r[keep]
+        return self._filter(self.out_nbrs[self.out_row_offsets[v]:self.out_row_offsets[v + 1]])
 
     def resident_nodes(self):
-        """Resident node ids in ascending partition order (= ascending id)."""
+        """Resident node ids in ascending partition order, ascending id inside a partition."""
         out = []
         for p in self.resident_parts:
-            out.extend(range(p * self.part_size, min((p + 1) * self.part_size, self.n_nodes)))
+            out.extend(int(v) for v in self.nodes_of_part(p))
         return out
 
     def n_resident_nodes(self) -> int:
-        return sum(min((p + 1) * self.part_size, self.n_nodes) - p * self.part_size
-                   for p in self.resident_parts)
+        return sum(len(self.nodes_of_part(p)) for p in self.resident_parts)
 
     def resident_node_at(self, idx: int) -> int:
-        """idx-th resident node without building the list."""
+        """idx-th resident node in that order."""
         for p in self.resident_parts:
-            lo = p * self.part_size
-            sz = min((p + 1) * self.part_size, self.n_nodes) - lo
-            if idx < sz:
-                return lo + idx
-            idx -= sz
+            ids = self.nodes_of_part(p)
+            if idx < len(ids):
+                return int(ids[idx])
+            idx -= len(ids)
         raise IndexError(idx)
 
 

@@ -383,8 +383,10 @@ class Context:
     def set_sample_direction(self, direction: str):
         self._check(self.lib.mg_set_sample_direction(self.handle, C.c_int({"in": 0, "inout": 1}[direction])))
 
-    def set_partitioning(self, n_parts: int):
-        self._check(self.lib.mg_set_partitioning(self.handle, C.c_int32(n_parts)))
+    def set_partitioning(self, n_parts: int, part_of_node: torch.Tensor | None = None):
+        """part_of_node: optional uint8 partition id per node (host); None = contiguous equal id ranges."""
+        pn = None if part_of_node is None else part_of_node.to(torch.uint8).cpu().contiguous()
+        self._check(self.lib.mg_set_partitioning(self.handle, C.c_int32(n_parts), _ptr(pn)))
 
     def load_features(self, table: torch.Tensor | None, capacity_parts: int = 1, backing: int = BACKING_HBM, dtype=None, dim=None):
         """table = None (host backing only): no whole table exists; give dtype and dim, and name every partition's

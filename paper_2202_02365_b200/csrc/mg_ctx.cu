@@ -100,6 +100,7 @@ struct ViewArgs {
     uint32_t part_size;
     int32_t n_parts;
     const int32_t* slot_of_part;
+    const uint8_t* part_of_node;   // null: partitions are contiguous id ranges
     uint32_t* mask;        // [ceil(E / 32)]
     uint16_t* word_before; // [ceil(E / 32)] kept edges of the tile before the word
     int32_t* tile_cnt;     // [tiles]
@@ -111,12 +112,16 @@ __device__ __forceinline__ int64_t part_edge_lo(const ViewArgs& a, int p) {
     const int64_t v = (int64_t)p * a.part_size;
     return a.off[v < a.n_nodes ? v : a.n_nodes];
 }
+// With a partition-id array the rows of a partition are not one range of edges.  The view then keeps every edge whose
+// NEIGHBOUR is resident, whatever its row: sampling only ever reads the rows of resident nodes (targets are checked,
+// neighbours were filtered), so the rows of the others are dead weight in the view, not an error.
 
 __global__ void __launch_bounds__(kThreads) k_view_mask(ViewArgs a) {
     __shared__ int64_t bound[MG_MAX_PARTS + 1];
     __shared__ int32_t res[MG_MAX_PARTS];
     __shared__ uint32_t warp_tot[kThreads / 32];
-    for (int p = threadIdx.x; p <= a.n_parts; p += kThreads) bound[p] = part_edge_lo(a, p);
+    const bool ranges = a.part_of_node == nullptr;
+    for (int p = threadIdx.x; p <= a.n_parts; p += kThreads) bound[p] = ranges ? part_edge_lo(a, p) : (p == 0 ? 0 : a.n_edges);
     for (int p = threadIdx.x; p < a.n_parts; p += kThreads) res[p] = a.slot_of_part[p] >= 0 ? 1 : 0;
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -131,7 +136,7 @@ __global__ void __launch_bounds__(kThreads) k_view_mask(ViewArgs a) {
             p = lo;
         }
         uint32_t bits = 0;
-        const bool any_row = e0 < a.n_edges && (res[p] || bound[p + 1] < e0 + 8);   // (a thread's 8 edges may cross into a resident range)
+        const bool any_row = e0 < a.n_edges && (!ranges || res[p] || bound[p + 1] < e0 + 8);   // (a thread's 8 edges may cross into a resident range)
         if (any_row) {
             int32_t u[8];
             if (e0 + 8 <= a.n_edges) {
@@ -144,8 +149,12 @@ __global__ void __launch_bounds__(kThreads) k_view_mask(ViewArgs a) {
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 const int64_t e = e0 + j;
-                while (p + 1 < a.n_parts && e >= bound[p + 1]) ++p;
-                if (e < a.n_edges && res[p] && res[(uint32_t)u[j] / a.part_size]) bits |= 1u << j;
+                if (ranges) {
+                    while (p + 1 < a.n_parts && e >= bound[p + 1]) ++p;
+                    if (e < a.n_edges && res[p] && res[(uint32_t)u[j] / a.part_size]) bits |= 1u << j;
+                } else if (e < a.n_edges && res[a.part_of_node[u[j]]]) {
+                    bits |= 1u << j;
+                }
             }
         }
         // four lanes make a word; counts: exclusive scan over the block's 256 threads
@@ -300,6 +309,7 @@ extern "C" int mg_create(mg_ctx** out, int device, void* stream) {
         cudaEventCreateWithFlags(&c->ev_out_done, cudaEventDisableTiming) != cudaSuccess ||
         cudaMalloc((void**)&c->d_slot_of_part, sizeof(int32_t) * MG_MAX_PARTS) != cudaSuccess ||
         cudaMalloc((void**)&c->d_res_prefix, sizeof(int64_t) * (MG_MAX_PARTS + 1)) != cudaSuccess ||
+        cudaMalloc((void**)&c->d_part_start, sizeof(int64_t) * (MG_MAX_PARTS + 1)) != cudaSuccess ||
         cudaMalloc((void**)&c->d_flags, sizeof(uint32_t)) != cudaSuccess ||
         cudaMemset(c->d_flags, 0, sizeof(uint32_t)) != cudaSuccess) {
         cudaGetLastError();
@@ -343,7 +353,7 @@ extern "C" int mg_destroy(mg_ctx* c) {
     free_features(c);
     free_out_graph(c);
     cudaFree(c->row_off); cudaFree(c->nbrs); cudaFree(c->d_slot_of_part); cudaFree(c->d_res_prefix); cudaFree(c->d_flags);
-    cudaFree(c->view_ws);
+    cudaFree(c->view_ws); cudaFree(c->d_part_start); cudaFree(c->d_part_of_node); cudaFree(c->d_local_of_node); cudaFree(c->d_nodes_by_part);
     cudaFree(c->ws_x); cudaFree(c->ws_h[0]); cudaFree(c->ws_h[1]);
     cudaEventDestroy(c->ev_fwd_done); cudaEventDestroy(c->ev_out_done); cudaEventDestroy(c->ev_user);
     for (int i = 0; i < 2; ++i) { if (c->ev_hk_done[i]) cudaEventDestroy(c->ev_hk_done[i]); cudaFree(c->hk_buf[i]); }
@@ -396,11 +406,13 @@ static int upload_slot_map(mg_ctx* c) {
     prefix[0] = 0;
     for (int p = 0; p < MG_MAX_PARTS; ++p) {
         slots[p] = p < c->n_parts ? c->slot_of_part[p] : -1;
-        int64_t sz = 0;
-        if (p < c->n_parts && slots[p] >= 0) sz = std::min<int64_t>(c->part_size, c->n_nodes - (int64_t)p * c->part_size);
-        prefix[p + 1] = prefix[p] + std::max<int64_t>(sz, 0);
+        const int64_t sz = (p < c->n_parts && slots[p] >= 0) ? c->part_count[p] : 0;
+        prefix[p + 1] = prefix[p] + sz;
     }
     c->n_resident_nodes = prefix[MG_MAX_PARTS];
+    int64_t starts[MG_MAX_PARTS + 1];
+    for (int p = 0; p <= MG_MAX_PARTS; ++p) starts[p] = p < c->n_parts ? c->part_start[p] : c->n_nodes;
+    MG_CUDA(c, cudaMemcpyAsync(c->d_part_start, starts, sizeof(starts), cudaMemcpyHostToDevice, c->stream));
     MG_CUDA(c, cudaMemcpyAsync(c->d_slot_of_part, slots, sizeof(slots), cudaMemcpyHostToDevice, c->stream));
     MG_CUDA(c, cudaMemcpyAsync(c->d_res_prefix, prefix, sizeof(prefix), cudaMemcpyHostToDevice, c->stream));
     MG_CUDA(c, cudaStreamSynchronize(c->stream));
@@ -444,6 +456,7 @@ static int rebuild_one_view(mg_ctx* c, bool all, const int64_t* row_off, const i
     ViewArgs a;
     a.off = row_off; a.nbrs = nbrs; a.n_nodes = c->n_nodes; a.n_edges = n_edges;
     a.part_size = (uint32_t)c->part_size; a.n_parts = c->n_parts; a.slot_of_part = c->d_slot_of_part;
+    a.part_of_node = c->d_part_of_node;
     a.mask = reinterpret_cast<uint32_t*>(c->view_ws + o_mask);
     a.word_before = reinterpret_cast<uint16_t*>(c->view_ws + o_before);
     a.tile_cnt = reinterpret_cast<int32_t*>(c->view_ws + o_cnt);
@@ -556,7 +569,7 @@ extern "C" int mg_load_graph(mg_ctx* c, int64_t n_nodes, int64_t n_edges, const 
     if (rc) return rc;
     c->n_nodes = n_nodes;
     c->n_edges = n_edges;
-    return mg_set_partitioning(c, 1);
+    return mg_set_partitioning(c, 1, nullptr);
 }
 
 extern "C" int mg_load_out_graph(mg_ctx* c, int64_t n_edges, const void* row_offsets, int offsets_are_i64, const int32_t* nbrs,
@@ -582,15 +595,56 @@ extern "C" int mg_set_sample_direction(mg_ctx* c, int direction) {
     return MG_OK;
 }
 
-extern "C" int mg_set_partitioning(mg_ctx* c, int32_t n_parts) {
+extern "C" int mg_set_partitioning(mg_ctx* c, int32_t n_parts, const uint8_t* part_of_node) {
     if (!c) return MG_ERR_ARG;
     if (!c->row_off) return mg_fail(c, MG_ERR_STATE, "no graph loaded");
     if (n_parts <= 0 || n_parts > MG_MAX_PARTS) return mg_fail(c, MG_ERR_ARG, "n_parts must be in [1, %d]", MG_MAX_PARTS);
     MG_CUDA(c, cudaSetDevice(c->device));
     MG_CUDA(c, cudaStreamSynchronize(c->stream));
+    MG_CUDA(c, cudaStreamSynchronize(c->sample_stream));
     free_features(c);
+    cudaFree(c->d_part_of_node); cudaFree(c->d_local_of_node); cudaFree(c->d_nodes_by_part);
+    c->d_part_of_node = nullptr; c->d_local_of_node = nullptr; c->d_nodes_by_part = nullptr;
+    c->part_count.assign(n_parts, 0);
+    c->part_start.assign(n_parts + 1, 0);
+    const int64_t N = c->n_nodes;
+    if (!part_of_node) {
+        // contiguous equal id ranges (the sequential lookup table of Section 3 cut into n_parts pieces)
+        c->part_size = (N + n_parts - 1) / n_parts;
+        for (int p = 0; p < n_parts; ++p) {
+            c->part_start[p] = std::min<int64_t>((int64_t)p * c->part_size, N);
+            c->part_count[p] = std::max<int64_t>(0, std::min<int64_t>(c->part_size, N - (int64_t)p * c->part_size));
+        }
+        c->part_start[n_parts] = N;
+    } else {
+        // a partition id per node: populations, each node's rank inside its partition and the partitions' node lists
+        for (int64_t v = 0; v < N; ++v) {
+            if (part_of_node[v] >= n_parts) return mg_fail(c, MG_ERR_ARG, "part_of_node[%lld] = %d is not below n_parts", (long long)v, (int)part_of_node[v]);
+            ++c->part_count[part_of_node[v]];
+        }
+        int64_t largest = 1;
+        for (int p = 0; p < n_parts; ++p) { c->part_start[p + 1] = c->part_start[p] + c->part_count[p]; largest = std::max(largest, c->part_count[p]); }
+        c->part_size = largest;
+        std::vector<int32_t> local((size_t)N), by_part((size_t)N);
+        std::vector<int64_t> next(c->part_start.begin(), c->part_start.end() - 1);
+        for (int64_t v = 0; v < N; ++v) {
+            const int p = part_of_node[v];
+            local[(size_t)v] = (int32_t)(next[p] - c->part_start[p]);
+            by_part[(size_t)next[p]++] = (int32_t)v;
+        }
+        if (cudaMalloc((void**)&c->d_part_of_node, (size_t)N) != cudaSuccess ||
+            cudaMalloc((void**)&c->d_local_of_node, sizeof(int32_t) * (size_t)N) != cudaSuccess ||
+            cudaMalloc((void**)&c->d_nodes_by_part, sizeof(int32_t) * (size_t)N) != cudaSuccess) {
+            cudaGetLastError();
+            cudaFree(c->d_part_of_node); cudaFree(c->d_local_of_node); cudaFree(c->d_nodes_by_part);
+            c->d_part_of_node = nullptr; c->d_local_of_node = nullptr; c->d_nodes_by_part = nullptr;
+            return mg_fail(c, MG_ERR_OOM, "allocation of the partition tables failed");
+        }
+        MG_CUDA(c, cudaMemcpy(c->d_part_of_node, part_of_node, (size_t)N, cudaMemcpyHostToDevice));
+        MG_CUDA(c, cudaMemcpy(c->d_local_of_node, local.data(), sizeof(int32_t) * (size_t)N, cudaMemcpyHostToDevice));
+        MG_CUDA(c, cudaMemcpy(c->d_nodes_by_part, by_part.data(), sizeof(int32_t) * (size_t)N, cudaMemcpyHostToDevice));
+    }
     c->n_parts = n_parts;
-    c->part_size = (c->n_nodes + n_parts - 1) / n_parts;
     c->capacity = n_parts;
     c->slot_of_part.assign(n_parts, n_parts == 1 ? 0 : -1);
     c->dirty_part.clear();
@@ -677,7 +731,7 @@ extern "C" int mg_load_features(mg_ctx* c, const void* table, int table_is_devic
 // where partition p's rows live in host memory (MG_BACKING_HOST), or null when nobody said
 static const char* host_block_of(const mg_ctx* c, int p) {
     if (p < (int)c->part_source.size() && c->part_source[p]) return c->part_source[p];
-    return c->host_table ? c->host_table + (size_t)p * c->part_size * c->row_bytes : nullptr;
+    return c->host_table ? c->host_table + (size_t)c->part_start[p] * c->row_bytes : nullptr;   // partition-major table
 }
 
 extern "C" int mg_set_partition_source(mg_ctx* c, int32_t part, const void* host_block) {
@@ -737,8 +791,7 @@ extern "C" int mg_set_resident(mg_ctx* c, const int32_t* part_ids, int32_t n, in
                 MG_CUDA(c, cudaEventRecord(main_done, c->stream));
                 MG_CUDA(c, cudaStreamWaitEvent(c->side, main_done, 0));
             }
-            const int64_t first = (int64_t)p * c->part_size;
-            const int64_t rows = std::min<int64_t>(c->part_size, c->n_nodes - first);
+            const int64_t rows = c->part_count[p];
             char* back = const_cast<char*>(host_block_of(c, p));
             if (rows > 0 && back)
                 MG_CUDA(c, cudaMemcpyAsync(back, c->slots + (size_t)s * c->slot_bytes, (size_t)rows * c->row_bytes,
@@ -758,8 +811,7 @@ extern "C" int mg_set_resident(mg_ctx* c, const int32_t* part_ids, int32_t n, in
                 }
             } else return mg_fail(c, MG_ERR_CAPACITY, "no free buffer slot");
             next[p] = s;
-            const int64_t first = (int64_t)p * c->part_size;
-            const int64_t rows = std::min<int64_t>(c->part_size, c->n_nodes - first);
+            const int64_t rows = c->part_count[p];
             // in pieces: a copy engine finishes what it has started, and one 5 GB copy would hold up every small
             // host-to-device copy another stream issues meanwhile (targets of a sample, say) for a tenth of a second
             const size_t bytes = (size_t)std::max<int64_t>(rows, 0) * c->row_bytes, piece = (size_t)8 << 20;

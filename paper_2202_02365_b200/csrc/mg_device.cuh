@@ -7,6 +7,28 @@
 #define MG_OUT_SLOT_BASE 65536  // first draw slot of the outgoing direction (incoming + outgoing sampling)
 #define MG_SLOT_BITS 24  // per-batch id-table slots are addressed with 24 bits (<= 16M slots)
 
+// Where a node's base representation lives: its partition, and its row in the feature buffer (rows of one node each,
+// slot after slot).  Partitions are contiguous equal id ranges unless a partition-id array was given.
+struct FeatGeom {
+    const int32_t* slot_of_part;    // device [n_parts]; -1 = not resident
+    const uint8_t* part_of_node;    // device [n_nodes], or null: partition = id / part_size
+    const int32_t* local_of_node;   // device [n_nodes], or null: the node's rank inside its partition (partition-id array given)
+    uint32_t part_size;             // rows per slot: ceil(n_nodes / n_parts), or the largest partition's population
+    int32_t identity;               // 1: the buffer is the whole table in node order, row = node id
+};
+
+__device__ __forceinline__ uint32_t feat_part(const FeatGeom& g, int32_t v) {
+    return g.part_of_node ? (uint32_t)g.part_of_node[v] : (uint32_t)v / g.part_size;
+}
+__device__ __forceinline__ bool feat_resident(const FeatGeom& g, int32_t v) { return g.slot_of_part[feat_part(g, v)] >= 0; }
+// row of node v in the buffer (v must be resident)
+__device__ __forceinline__ int64_t feat_row(const FeatGeom& g, int32_t v) {
+    if (g.identity) return v;
+    if (g.part_of_node) return (int64_t)g.slot_of_part[g.part_of_node[v]] * g.part_size + g.local_of_node[v];
+    const uint32_t p = (uint32_t)v / g.part_size;
+    return (int64_t)g.slot_of_part[p] * g.part_size + ((uint32_t)v - p * g.part_size);
+}
+
 // Philox4x32-10 (Salmon et al., SC'11); the draw of (seed, node, hop, slot) is word slot % 4
 // of the block with counter (node, 0, hop, slot / 4) and key (seed low, seed high).
 __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,

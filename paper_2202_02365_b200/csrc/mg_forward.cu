@@ -50,9 +50,8 @@ struct AggArgs {
     const float* h_prev;         // layers >= 2
     // layer 1: the partition buffer
     const char* slots;
-    const int32_t* slot_of_part;
-    int64_t slot_bytes, row_bytes;
-    uint32_t part_size;
+    FeatGeom feat;
+    int64_t row_bytes;
     float* x;                    // [rows, 2 * d_in], row r of this launch at x + (r - row_lo) * 2 * d_in
     int round_tf32;
     int sum_aggr;                // neighbour term = sum of the sampled neighbours instead of their mean
@@ -65,8 +64,7 @@ __device__ __forceinline__ float to_tf32(float v) {
 }
 
 __device__ __forceinline__ const char* feature_row(const AggArgs& a, int32_t node) {
-    const uint32_t p = (uint32_t)node / a.part_size;
-    return a.slots + (int64_t)a.slot_of_part[p] * a.slot_bytes + (int64_t)((uint32_t)node - p * a.part_size) * a.row_bytes;
+    return a.slots + feat_row(a.feat, node) * a.row_bytes;
 }
 
 // one 16-byte chunk -> 4 (fp32) or 8 (fp16) floats
@@ -251,9 +249,8 @@ struct H0Args {
     int32_t node_off[MG_MAX_HOPS + 1];
     const int32_t* nodes;
     const char* slots;
-    const int32_t* slot_of_part;
-    int64_t slot_bytes, row_bytes;
-    uint32_t part_size;
+    FeatGeom feat;
+    int64_t row_bytes;
 };
 
 template <bool HALF>
@@ -268,8 +265,7 @@ __global__ void __launch_bounds__(kThreads) k_gather_h0(H0Args a, float* __restr
         int h = 0;
         while (h < a.r.k && l >= a.r.cum[h + 1]) ++h;
         const int32_t node = a.nodes[a.node_off[h] + (l - a.r.cum[h])];
-        const uint32_t p = (uint32_t)node / a.part_size;
-        const char* row = a.slots + (int64_t)a.slot_of_part[p] * a.slot_bytes + (int64_t)((uint32_t)node - p * a.part_size) * a.row_bytes;
+        const char* row = a.slots + feat_row(a.feat, node) * a.row_bytes;
         C v;
         v.load(row, q);
         v.store(out + (int64_t)c * a.r.dim + q * C::kVals, 1.f, false);
@@ -621,8 +617,7 @@ static int forward_impl(mg_ctx* ctx, const mg_model* m, mg_dense* d, float* out,
             a.cum = d->cum; a.node_off = d->node_off; a.nodes = d->nodes;
             a.ent_off = d->ent_off; a.ent_nbrs = d->ent_nbrs; a.ent_repr = d->ent_repr;
             a.h_prev = h_prev;
-            a.slots = ctx->slots; a.slot_of_part = ctx->d_slot_of_part;
-            a.slot_bytes = ctx->slot_bytes; a.row_bytes = ctx->row_bytes; a.part_size = (uint32_t)ctx->part_size;
+            a.slots = ctx->slots; a.feat = mg_feat_geom(ctx); a.row_bytes = ctx->row_bytes;
             a.x = ctx->ws_x;
             a.round_tf32 = m->precision == MG_GEMM_TF32;
             a.sum_aggr = m->sum_aggr ? 1 : 0;
@@ -685,8 +680,7 @@ extern "C" int mg_gather_h0(mg_ctx* ctx, mg_dense* d, int32_t batch, float* out_
         if (rc0) return rc0;
     }
     for (int h = 0; h <= d->k; ++h) a.node_off[h] = d->h_node_off[(size_t)h * (d->n_batches + 1) + batch];
-    a.nodes = d->nodes; a.slots = ctx->slots; a.slot_of_part = ctx->d_slot_of_part;
-    a.slot_bytes = ctx->slot_bytes; a.row_bytes = ctx->row_bytes; a.part_size = (uint32_t)ctx->part_size;
+    a.nodes = d->nodes; a.slots = ctx->slots; a.feat = mg_feat_geom(ctx); a.row_bytes = ctx->row_bytes;
     if (a.r.n_rows > 0) {
         if (ctx->feat_dtype == MG_DTYPE_F16) k_gather_h0<true><<<mg_grid(ctx, 4), kThreads, 0, ctx->stream>>>(a, out_dev);
         else k_gather_h0<false><<<mg_grid(ctx, 4), kThreads, 0, ctx->stream>>>(a, out_dev);
@@ -1022,8 +1016,7 @@ extern "C" int mg_backward(mg_ctx* ctx, mg_model* m, mg_dense* d, const float* d
             a.cum = d->cum; a.node_off = d->node_off; a.nodes = d->nodes;
             a.ent_off = d->ent_off; a.ent_nbrs = d->ent_nbrs; a.ent_repr = d->ent_repr;
             a.h_prev = h_prev;
-            a.slots = ctx->slots; a.slot_of_part = ctx->d_slot_of_part;
-            a.slot_bytes = ctx->slot_bytes; a.row_bytes = ctx->row_bytes; a.part_size = (uint32_t)ctx->part_size;
+            a.slots = ctx->slots; a.feat = mg_feat_geom(ctx); a.row_bytes = ctx->row_bytes;
             a.x = ctx->bw_x;
             a.round_tf32 = 0;
             a.sum_aggr = m->sum_aggr ? 1 : 0;
@@ -1157,9 +1150,8 @@ struct EmbSgdArgs {
     const float* grad;          // [n_rows, dim] packed like H^0
     int64_t n_rows;
     char* slots;
-    const int32_t* slot_of_part;
-    int64_t slot_bytes, row_bytes;
-    uint32_t part_size;
+    FeatGeom feat;
+    int64_t row_bytes;
     int32_t dim;
     float lr;
 };
@@ -1171,9 +1163,7 @@ __global__ void __launch_bounds__(kThreads) k_embedding_sgd(EmbSgdArgs a) {
     for (int64_t row = blockIdx.x * (int64_t)(kThreads / 32) + (threadIdx.x >> 5); row < a.n_rows; row += warps) {
         int32_t b, local, node;
         locate_row(a.g, 0, row, &b, &local, &node);
-        const uint32_t id = (uint32_t)a.nodes[node];
-        const uint32_t p = id / a.part_size;
-        float* dst = reinterpret_cast<float*>(a.slots + (int64_t)a.slot_of_part[p] * a.slot_bytes + (int64_t)(id - p * a.part_size) * a.row_bytes);
+        float* dst = reinterpret_cast<float*>(a.slots + feat_row(a.feat, a.nodes[node]) * a.row_bytes);
         const float* g = a.grad + row * a.dim;
         for (int c = lane; c < a.dim; c += 32) {
             const float v = g[c];
@@ -1195,7 +1185,7 @@ extern "C" int mg_apply_embedding_sgd(mg_ctx* ctx, mg_dense* d, const float* d_h
     if (int rs = mg_check_sample_residency(ctx, d)) return rs;
     MG_CUDA(ctx, cudaSetDevice(ctx->device));
     EmbSgdArgs a{{d->n_batches, d->k, d->rowbase, d->cum, d->node_off}, d->nodes, d_h0_dev, d->h_hdr.rows_total[0], ctx->slots,
-                 ctx->d_slot_of_part, ctx->slot_bytes, ctx->row_bytes, (uint32_t)ctx->part_size, ctx->feat_dim, lr};
+                 mg_feat_geom(ctx), ctx->row_bytes, ctx->feat_dim, lr};
     if (a.n_rows > 0) {
         k_embedding_sgd<<<mg_grid(ctx, 8), kThreads, 0, ctx->stream>>>(a);
         ctx->launches++;
@@ -1296,8 +1286,7 @@ extern "C" int mg_forward_noalloc(mg_ctx* ctx, const mg_model* m, mg_dense* d, f
             a.cum = d->cum; a.node_off = d->node_off; a.nodes = d->nodes;
             a.ent_off = d->ent_off; a.ent_nbrs = d->ent_nbrs; a.ent_repr = d->ent_repr;
             a.h_prev = h_prev;
-            a.slots = ctx->slots; a.slot_of_part = ctx->d_slot_of_part;
-            a.slot_bytes = ctx->slot_bytes; a.row_bytes = ctx->row_bytes; a.part_size = (uint32_t)ctx->part_size;
+            a.slots = ctx->slots; a.feat = mg_feat_geom(ctx); a.row_bytes = ctx->row_bytes;
             a.x = staging;
             a.round_tf32 = m->precision == MG_GEMM_TF32;
             a.sum_aggr = m->sum_aggr ? 1 : 0;

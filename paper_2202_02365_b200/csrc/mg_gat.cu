@@ -86,9 +86,8 @@ struct GatherArgs {
     GatGeom g;
     const int32_t* nodes;
     const char* slots;
-    const int32_t* slot_of_part;
-    int64_t slot_bytes, row_bytes, n_rows;
-    uint32_t part_size;
+    FeatGeom feat;
+    int64_t row_bytes, n_rows;
     int32_t dim, half, round;
     float* x;   // [n_rows, dim]
 };
@@ -100,9 +99,7 @@ __global__ void __launch_bounds__(kThreads) k_gat_gather0(GatherArgs a) {
     for (int64_t row = blockIdx.x * (int64_t)(kThreads / 32) + (threadIdx.x >> 5); row < a.n_rows; row += warps) {
         int32_t b, local, node;
         locate(a.g, 0, row, &b, &local, &node);
-        const uint32_t id = (uint32_t)a.nodes[node];
-        const uint32_t p = id / a.part_size;
-        const char* src = a.slots + (int64_t)a.slot_of_part[p] * a.slot_bytes + (int64_t)(id - p * a.part_size) * a.row_bytes;
+        const char* src = a.slots + feat_row(a.feat, a.nodes[node]) * a.row_bytes;
         float4* dst = reinterpret_cast<float4*>(a.x + row * a.dim);   // (rows are multiples of 16 bytes on both sides)
         for (int c = lane; c < a.dim / 4; c += 32) {
             float4 v;
@@ -341,9 +338,9 @@ extern "C" int mg_gat_forward(mg_ctx* ctx, const mg_gat_model* m, mg_dense* d, f
     {
         ProfScope ps(ctx, PH_AGG_L1, 1);
         GatherArgs a;
-        a.g = geom; a.nodes = d->nodes; a.slots = ctx->slots; a.slot_of_part = ctx->d_slot_of_part;
-        a.slot_bytes = ctx->slot_bytes; a.row_bytes = ctx->row_bytes; a.n_rows = d->h_hdr.rows_total[0];
-        a.part_size = (uint32_t)ctx->part_size; a.dim = m->dims[0]; a.half = ctx->feat_dtype == MG_DTYPE_F16; a.round = tf32;
+        a.g = geom; a.nodes = d->nodes; a.slots = ctx->slots; a.feat = mg_feat_geom(ctx);
+        a.row_bytes = ctx->row_bytes; a.n_rows = d->h_hdr.rows_total[0];
+        a.dim = m->dims[0]; a.half = ctx->feat_dtype == MG_DTYPE_F16; a.round = tf32;
         a.x = ctx->gat_x;
         k_gat_gather0<<<grid, kThreads, 0, st>>>(a);
         ctx->launches++;

@@ -10,6 +10,7 @@
 #include <vector>
 
 #include "mgdense.h"
+#include "mg_device.cuh"
 
 // ---------------------------------------------------------------------------------------
 // status word written by kernels (never a trap): bit flags, read by the host after a call
@@ -97,8 +98,14 @@ struct mg_ctx {
     bool has_pending = false;
     std::vector<cudaEvent_t> pending_events;
     std::vector<char> dirty_part;       // host backing: the partition's slot was updated (mg_apply_embedding_sgd) and not written back yet
+    // partition-id array (mg_set_partitioning with part_of_node): null for contiguous equal ranges
+    uint8_t* d_part_of_node = nullptr;    // [n_nodes]
+    int32_t* d_local_of_node = nullptr;   // [n_nodes] rank of the node inside its partition (ascending id)
+    int32_t* d_nodes_by_part = nullptr;   // [n_nodes] node ids partition after partition, ascending inside a partition
+    std::vector<int64_t> part_count, part_start;   // population of each partition; first row of its block in a partition-major table
     int32_t* d_slot_of_part = nullptr;   // [MG_MAX_PARTS]
     int64_t* d_res_prefix = nullptr;     // [MG_MAX_PARTS + 1] resident-node prefix counts
+    int64_t* d_part_start = nullptr;     // [MG_MAX_PARTS + 1] first row of each partition's block (prefix of the populations)
     int64_t n_resident_nodes = 0;
 
     // features
@@ -310,6 +317,17 @@ struct ProfScope {
 };
 
 static inline int mg_grid(const mg_ctx* ctx, int ctas_per_sm) { return ctx->n_sms * ctas_per_sm; }
+
+// how kernels find a node's partition and its row in the feature buffer
+static inline FeatGeom mg_feat_geom(const mg_ctx* ctx) {
+    FeatGeom g;
+    g.slot_of_part = ctx->d_slot_of_part;
+    g.part_of_node = ctx->d_part_of_node;
+    g.local_of_node = ctx->d_local_of_node;
+    g.part_size = (uint32_t)ctx->part_size;
+    g.identity = ctx->backing == MG_BACKING_HBM ? 1 : 0;   // the whole table in device memory, in node order
+    return g;
+}
 
 // ---- generic device-sized scan and sort (mg_sample.cu) -------------------------------------
 struct SortParams {   // device-resident

@@ -72,12 +72,8 @@ struct FusedArgs {
     const float* h_prev;         // layers >= 2: [rows of layer l-1, d_in]
     const char* src_base;        // layer 1: the feature buffer; later layers: h_prev
     uint32_t src_row_bytes;      // (32-bit: the row address is then one wide multiply-add)
-    const char* slots;           // layer 1: partition buffer
-    const int32_t* slot_of_part;
-    int64_t slot_bytes, row_bytes;
-    uint32_t part_size;
+    FeatGeom feat;               // layer 1: where a node's row lives in the partition buffer
     int32_t safe_src;            // a source row that is always valid to read (rows past the end load it)
-    int32_t identity_rows;       // layer 1: slot == partition for every resident partition (whole table in HBM)
     // shapes
     int32_t d_in, d_in_pad;      // d_in_pad = d_in rounded up to 32; K = 2 * d_in_pad
     int32_t N, BN;               // output width and its MMA tile width (multiple of 16, <= 256)
@@ -105,11 +101,7 @@ typedef int4 RowMeta;
 // later layers: row of H^{l-1}.  The address is src_base + row * src_row_bytes.
 template <bool FIRST>
 __device__ __forceinline__ int32_t source_row(const FusedArgs& a, int32_t in_base, int32_t key) {
-    if (FIRST) {
-        if (a.identity_rows) return key;
-        const uint32_t p = (uint32_t)key / a.part_size;
-        return (int32_t)((uint32_t)a.slot_of_part[p] * a.part_size + ((uint32_t)key - p * a.part_size));
-    }
+    if (FIRST) return (int32_t)feat_row(a.feat, key);
     return in_base + key;
 }
 
@@ -695,11 +687,7 @@ static void fill_args(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d
     a.rowbase_in = d->rowbase + (size_t)(layer - 1) * (B + 1);
     a.cum = d->cum; a.node_off = d->node_off; a.nodes = d->nodes;
     a.ent_off = d->ent_off; a.ent_nbrs = d->ent_nbrs; a.ent_repr = d->ent_repr;
-    a.slots = ctx->slots; a.slot_of_part = ctx->d_slot_of_part;
-    a.slot_bytes = ctx->slot_bytes; a.row_bytes = ctx->row_bytes; a.part_size = (uint32_t)ctx->part_size;
-    a.identity_rows = 1;
-    for (int p = 0; p < ctx->n_parts; ++p)
-        if (ctx->slot_of_part[p] >= 0 && ctx->slot_of_part[p] != p) a.identity_rows = 0;
+    a.feat = mg_feat_geom(ctx);
     a.d_in = d_in;
     a.d_in_pad = (d_in + KC - 1) / KC * KC;
     a.N = d_out;

@@ -16,15 +16,16 @@ constexpr int kThreads = 256;
 // origin: [0, E) sources, [E, 2E) destinations, [2E, 2E + C * negs) negatives.
 __global__ void __launch_bounds__(kThreads)
 k_lp_keys(const int32_t* __restrict__ src, const int32_t* __restrict__ dst, int64_t E, int32_t n_chunks, int32_t negs,
-          uint64_t seed, const int64_t* __restrict__ res_prefix, int32_t n_parts, int64_t part_size, int64_t n_resident,
-          int64_t n_nodes, const int32_t* __restrict__ slot_of_part, int32_t* neg_ids, uint64_t* keys, uint32_t* status) {
+          uint64_t seed, const int64_t* __restrict__ res_prefix, int32_t n_parts, int64_t n_resident, int64_t n_nodes, FeatGeom feat,
+          const int64_t* __restrict__ part_start, const int32_t* __restrict__ nodes_by_part, int32_t* neg_ids, uint64_t* keys,
+          uint32_t* status) {
     const int64_t total = 2 * E + (int64_t)n_chunks * negs;
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
         int32_t id;
         if (i < 2 * E) {
             id = i < E ? src[i] : dst[i - E];
             if (id < 0 || (int64_t)id >= n_nodes) { atomicOr(status, ST_RANGE); id = 0; }
-            else if (slot_of_part[(int64_t)id / part_size] < 0) atomicOr(status, ST_NONRESIDENT);
+            else if (!feat_resident(feat, id)) atomicOr(status, ST_NONRESIDENT);
         } else {
             const int64_t j = i - 2 * E;
             const uint32_t c = (uint32_t)(j / negs), t = (uint32_t)(j % negs);
@@ -34,7 +35,8 @@ k_lp_keys(const int32_t* __restrict__ src, const int32_t* __restrict__ dst, int6
             const int64_t r = (int64_t)(((unsigned __int128)o[0] * (unsigned __int128)(uint64_t)n_resident) >> 32);
             int p = 0;
             while (p + 1 < n_parts && res_prefix[p + 1] <= r) ++p;
-            id = (int32_t)((int64_t)p * part_size + (r - res_prefix[p]));
+            // (partitions are id ranges, or, with a partition-id array, listed in nodes_by_part in ascending id)
+            id = nodes_by_part ? nodes_by_part[part_start[p] + (r - res_prefix[p])] : (int32_t)(part_start[p] + (r - res_prefix[p]));
             neg_ids[j] = id;
         }
         keys[i] = ((uint64_t)(uint32_t)id << 32) | (uint64_t)(uint32_t)i;
@@ -485,7 +487,7 @@ extern "C" int mg_lp_prepare(mg_ctx* ctx, const int32_t* src, const int32_t* rel
     cudaMemsetAsync(d_status, 0, 4, st);
     const int grid = mg_grid(ctx, 4);
     k_lp_keys<<<grid, kThreads, 0, st>>>(d_src, d_dst, n_edges, n_chunks, negs, seed, ctx->d_res_prefix, ctx->n_parts,
-                                         ctx->part_size, ctx->n_resident_nodes, ctx->n_nodes, ctx->d_slot_of_part,
+                                         ctx->n_resident_nodes, ctx->n_nodes, mg_feat_geom(ctx), ctx->d_part_start, ctx->d_nodes_by_part,
                                          lp->neg_ids, keys[0], d_status);
     int id_bits = 1;
     while ((1ll << id_bits) < ctx->n_nodes) ++id_bits;

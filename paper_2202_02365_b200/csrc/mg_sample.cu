@@ -150,8 +150,7 @@ __global__ void __launch_bounds__(kThreads) k_copy_i32(const int32_t* __restrict
 __global__ void __launch_bounds__(kThreads)
 k_init_targets(DenseHeader* hdr, const int32_t* __restrict__ targets,
                const int32_t* __restrict__ tgt_off, int32_t B, int32_t* nodes, int32_t* node_batch,
-               int32_t* hkeys, int32_t* hvals, TableGeom tg, int64_t n_nodes, int64_t part_size,
-               const int32_t* __restrict__ slot_of_part) {
+               int32_t* hkeys, int32_t* hvals, TableGeom tg, int64_t n_nodes, FeatGeom feat) {
     const int32_t n_total = hdr->hop_base[1];   // read on the device: the launch does not depend on the number of targets
     for (int32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n_total; i += gridDim.x * blockDim.x) {
         const int b = upper_segment(tgt_off, B + 1, i);
@@ -159,7 +158,7 @@ k_init_targets(DenseHeader* hdr, const int32_t* __restrict__ targets,
         nodes[i] = v;
         node_batch[i] = b;
         if (v < 0 || (int64_t)v >= n_nodes) { atomicOr(&hdr->status, ST_RANGE); continue; }
-        if (slot_of_part[(int64_t)v / part_size] < 0) { atomicOr(&hdr->status, ST_NONRESIDENT); continue; }
+        if (!feat_resident(feat, v)) { atomicOr(&hdr->status, ST_NONRESIDENT); continue; }
         bool is_new;
         const int32_t slot = table_insert(hkeys + (int64_t)b * tg.size, tg.size, v, &is_new);
         if (slot < 0) { atomicOr(&hdr->status, ST_CAP_TABLE); continue; }
@@ -1556,8 +1555,7 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
         MG_CUDA(ctx, cudaMemsetAsync(d->hkeys, 0xFF, sizeof(int32_t) * (size_t)B * table_size, st));
         {
             k_init_targets<<<mg_grid(ctx, 4), kThreads, 0, st>>>(d->hdr, tgt_dev, d->node_off, B, d->nodes,
-                                                               d->node_batch, d->hkeys, d->hvals, tg, ctx->n_nodes,
-                                                               ctx->part_size, ctx->d_slot_of_part);
+                                                               d->node_batch, d->hkeys, d->hvals, tg, ctx->n_nodes, mg_feat_geom(ctx));
             ctx->launches++;
         }
     }
@@ -1660,7 +1658,7 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
     for (int h = 0; h < k; ++h) sig.fanouts[h] = fanouts[h];
     const void* ptrs[] = {d->hdr, d->nodes, d->node_batch, d->ent_off, d->node_r0, d->node_deg, d->newlist[0], d->newlist[1],
                           d->scan_tmp, d->sort_hist, d->ent_nbrs, d->ent_repr, d->hkeys, d->hvals, d->node_off, d->cum, d->rowbase,
-                          d->d_ent_hop, d->d_seeds, d->h_stage_dev, d->h_pinned_dev, ctx->view_off, ctx->view_nbrs, ctx->d_slot_of_part, st,
+                          d->d_ent_hop, d->d_seeds, d->h_stage_dev, d->h_pinned_dev, ctx->view_off, ctx->view_nbrs, ctx->d_slot_of_part, st, ctx->d_part_of_node,
                           inout ? (const void*)ctx->view_off_out : nullptr, inout ? (const void*)ctx->view_nbrs_out : nullptr,
                           d->node_r0_out, d->node_deg_out, d->pairs, d->share_off};
     static_assert(sizeof(ptrs) <= sizeof(sig.ptrs), "signature too small");

@@ -268,9 +268,22 @@ def swap_order(n_parts: int, capacity: int, seed: int):
     return states
 
 
-def resident_node_mask(n_nodes: int, n_parts: int, resident_parts, device="cpu") -> torch.Tensor:
+def training_first_partitioning(n_nodes: int, n_parts: int, train_nodes: torch.Tensor, seed: int) -> torch.Tensor:
+    """A partition id per node (uint8) after Section 5.2's policy: the training nodes fill the first partitions in
+    order, every other node goes to a uniformly random one of the remaining partitions."""
+    g = _gen(seed, "cpu")
     size = contiguous_partition(n_nodes, n_parts)
-    part = torch.arange(n_nodes, device=device) // size
+    train_nodes = train_nodes.cpu().long()
+    n_train_parts = max(1, (train_nodes.numel() + size - 1) // size)
+    assert n_train_parts < n_parts
+    part = torch.randint(n_train_parts, n_parts, (n_nodes,), generator=g, dtype=torch.int64)
+    part[train_nodes] = torch.arange(train_nodes.numel()) // size
+    return part.to(torch.uint8)
+
+
+def resident_node_mask(n_nodes: int, n_parts: int, resident_parts, device="cpu", part_of_node: torch.Tensor | None = None) -> torch.Tensor:
+    size = contiguous_partition(n_nodes, n_parts)
+    part = torch.arange(n_nodes, device=device) // size if part_of_node is None else part_of_node.to(device).long()
     res = torch.zeros(n_parts, dtype=torch.bool, device=device)
     res[torch.as_tensor(list(resident_parts), device=device)] = True
     return res[part]

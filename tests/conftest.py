@@ -32,9 +32,11 @@ PARITY_WORST = {}
 
 
 def note_relative_error(rtol, worst_rel, worst_vs_bound):
-    cur = PARITY_WORST.setdefault(rtol, [0.0, 0.0, 0])
+    cur = PARITY_WORST.setdefault(rtol, [0.0, 0.0, 0, ""])
     cur[0] = max(cur[0], worst_rel)
-    cur[1] = max(cur[1], worst_vs_bound)
+    if worst_vs_bound > cur[1]:
+        cur[1] = worst_vs_bound
+        cur[3] = os.environ.get("PYTEST_CURRENT_TEST", "").split(" ")[0]
     cur[2] += 1
 
 
@@ -43,5 +45,5 @@ def pytest_terminal_summary(terminalreporter):
         return
     terminalreporter.write_line("parity: worst errors per tolerance class (comparisons; error / bound; pure relative error where |ref| > rms/100)")
     for rtol in sorted(PARITY_WORST):
-        rel, vs_bound, count = PARITY_WORST[rtol]
-        terminalreporter.write_line(f"  rtol {rtol:g}: {count} comparisons, worst {vs_bound:.3f} x the bound, worst relative error {rel:.3g}")
+        rel, vs_bound, count, where = PARITY_WORST[rtol]
+        terminalreporter.write_line(f"  rtol {rtol:g}: {count} comparisons, worst {vs_bound:.3f} x the bound ({where}), worst relative error {rel:.3g}")

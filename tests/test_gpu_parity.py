@@ -335,6 +335,61 @@ def test_commit_timeout_keeps_the_old_set_and_stale_samples_are_refused():
     assert torch.equal(again, out_small)
 
 
+@pytest.mark.parametrize("backing", ["hbm", "host"])
+def test_partition_id_array_with_training_nodes_in_the_first_partitions(backing):
+    """A partition id per node instead of contiguous ranges (Section 5.2's policy: the training nodes fill the first
+    partitions, every other node sits in a random one of the rest).  Sampling under the buffer, the forward pass, H^0
+    rows and link-prediction negatives against the oracle given the same array; host backing reads a partition-major
+    table (a partition's rows in ascending id) through the buffer's slots and swaps a partition in."""
+    n, parts, dim = 60_000, 8, 32
+    g = inputs.rmat_graph(n, 900_000, seed=71)
+    feats = inputs.normal_features(n, dim, seed=72)
+    train = torch.randperm(n, generator=torch.Generator().manual_seed(73))[:9000]
+    pn = inputs.training_first_partitioning(n, parts, train, seed=74)
+    assert int(pn[train].max()) == 1                         # 9,000 training nodes fill partitions 0 and 1 (7,500 each)
+    ctx = mg.Context(0)
+    ctx.load_graph(g.row_offsets.cuda(), g.nbrs.cuda())
+    ctx.set_partitioning(parts, pn)
+    if backing == "hbm":
+        ctx.load_features(feats.cuda(), capacity_parts=4)
+    else:
+        order = torch.argsort(pn.long() * n + torch.arange(n))                    # partition-major, ascending id inside
+        ctx.load_features(feats[order].contiguous().pin_memory(), capacity_parts=4, backing=mg.BACKING_HOST)
+    layers = inputs.random_bias_layers([dim, 16, 8], seed=75)
+    np_layers = [(w.numpy(), nn.numpy(), b.numpy()) for w, nn, b in layers]
+    model = ctx.model(layers, mg.GEMM_FP32)
+    g_host = (g.row_offsets.numpy(), g.nbrs.numpy())
+    for step, resident in enumerate([[0, 1, 5], [1, 0, 5, 6], [0, 1, 2, 6]]):
+        ctx.set_resident(resident)
+        view = O.GraphView(g_host[0], g_host[1], parts, resident, part_of_node=pn.numpy())
+        tg = train[torch.randperm(9000, generator=torch.Generator().manual_seed(80 + step))[:400]].to(torch.int32)
+        d = ctx.sample(tg, [6, 4], seed=90 + step)
+        ref = O.sample_dense(view, tg.tolist(), [6, 4], 90 + step)
+        assert_dense_equal(d.view(0), ref)
+        assert all(view.is_resident(u) for u in ref["node_ids"])
+        np.testing.assert_array_equal(ctx.gather_h0(d, 0, len(ref["node_ids"]), dim).cpu().numpy(), feats.numpy()[ref["node_ids"]])
+        out = torch.empty((400, 8), dtype=torch.float32, device="cuda")
+        ctx.forward(model, d, out)
+        close(out.cpu().numpy(), O.forward(ref, feats.numpy()[ref["node_ids"]], np_layers), RTOL_AGG)
+        model_tc = ctx.model(layers, mg.GEMM_TF32)
+        ctx.forward(model_tc, d, out)
+        close(out.cpu().numpy(), O.forward(ref, feats.numpy()[ref["node_ids"]], np_layers), RTOL_TC)
+        # link prediction: negatives are drawn among the resident nodes, partition after partition
+        mask = inputs.resident_node_mask(n, parts, resident, part_of_node=pn)
+        src, rel, dst = inputs.lp_edges(g, mask, 300, seed=step)
+        lp = ctx.lp_prepare(src, rel, dst, 3, 50, seed=7 + step)
+        prep = O.lp_prepare(view, src.tolist(), dst.tolist(), 3, 50, 7 + step)
+        got = lp.view()
+        for key in ("targets", "src_idx", "dst_idx", "neg_ids", "neg_idx"):
+            assert got[key].cpu().tolist() == prep[key], key
+    with pytest.raises(mg.MgError) as e:
+        ctx.sample(torch.tensor([int(torch.nonzero(pn == 7)[0])], dtype=torch.int32), [2], seed=0)   # partition 7 is not resident
+    assert e.value.code == -3
+    with pytest.raises(mg.MgError) as e:
+        ctx.set_partitioning(4, pn)                          # ids up to 7 do not fit 4 partitions
+    assert e.value.code == -1
+
+
 def test_link_prediction_distmult():
     n, parts, cap = 8000, 4, 2
     g = inputs.rmat_graph(n, 100_000, seed=5, n_relations=37)

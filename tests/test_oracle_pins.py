@@ -284,6 +284,54 @@ def test_buffer_filter_equals_sampling_the_induced_subgraph(resident):
     assert c["node_ids"][nio[0]:nio[1]] == lv[2] and c["node_ids"][nio[1]:nio[2]] == lv[1]
 
 
+def test_partition_id_array():
+    """GraphView with one partition id per node (Section 5.2: training nodes in the first partitions, the rest at
+    random): (a) the array that spells out the contiguous split changes nothing; (b) under any array the filter equals
+    sampling the explicitly induced subgraph; (c) resident nodes are counted partition after partition, ascending id
+    inside a partition, and negatives are drawn from exactly those; (d) the policy's array keeps every training node
+    resident while only the first partitions are in the buffer."""
+    n, parts = 120, 4
+    off, nb = _random_graph(n, 1500, 9)
+    size = (n + parts - 1) // parts
+    same = np.arange(n) // size
+    for resident in ([0, 2], [1, 2, 3]):
+        targets = [v for v in range(n) if v // size in resident][::7]
+        a = O.sample_dense(O.GraphView(off, nb, parts, resident), targets, [3, 2], seed=5)
+        b = O.sample_dense(O.GraphView(off, nb, parts, resident, part_of_node=same), targets, [3, 2], seed=5)
+        assert a == b
+        assert (O.lp_negatives(O.GraphView(off, nb, parts, resident), 2, 50, 3)
+                == O.lp_negatives(O.GraphView(off, nb, parts, resident, part_of_node=same), 2, 50, 3))
+    rng = np.random.default_rng(3)
+    pn = rng.integers(0, parts, n)
+    for resident in ([0, 2], [3], [0, 1, 3]):
+        res = lambda u: pn[u] in resident
+        edges = [(int(u), v) for v in range(n) for u in nb[off[v]:off[v + 1]] if res(int(u)) and res(v)]
+        off2, nb2 = _csr_from_edges(n, edges)
+        view = O.GraphView(off, nb, parts, resident, part_of_node=pn)
+        targets = [v for v in range(n) if res(v)][::5]
+        assert O.sample_dense(view, targets, [3, 2], seed=5) == O.sample_dense(O.GraphView(off2, nb2), targets, [3, 2], seed=5)
+        with pytest.raises(ValueError):
+            O.sample_dense(view, [next(v for v in range(n) if not res(v))], [2], 0)
+        want = [v for p in sorted(resident) for v in range(n) if pn[v] == p]
+        assert view.resident_nodes() == want and view.n_resident_nodes() == len(want)
+        assert [view.resident_node_at(i) for i in range(len(want))] == want
+        negs = O.lp_negatives(view, 3, 400, seed=8)
+        assert all(res(u) for row in negs for u in row)
+        counts = np.bincount([want.index(u) for row in negs for u in row], minlength=len(want))
+        expect = 1200 / len(want)
+        assert ((counts - expect) ** 2 / expect).sum() < 2.0 * len(want)          # uniform over the resident nodes
+    train = torch.randperm(n, generator=torch.Generator().manual_seed(1))[:50]
+    policy = inputs.training_first_partitioning(n, parts, train, seed=2).numpy()
+    k_train = (50 + size - 1) // size
+    assert set(policy[train.numpy()].tolist()) == set(range(k_train))
+    rest = np.setdiff1d(np.arange(n), train.numpy())
+    assert set(policy[rest].tolist()) <= set(range(k_train, parts)) and len(set(policy[rest].tolist())) == parts - k_train
+    view = O.GraphView(off, nb, parts, list(range(k_train)), part_of_node=policy)
+    assert all(view.is_resident(int(t)) for t in train)
+    d = O.sample_dense(view, train.tolist()[:10], [4, 4], seed=1)
+    assert all(policy[u] < k_train for u in d["node_ids"])
+
+
 # ---------------------------------------------------------------- forward
 def test_hand_computed_means():
     g = _fields(os.path.join(GOLD, "dense_worked_example.txt"))
