@@ -146,11 +146,12 @@ def build_workload(cfg, device, seed=0):
         g = inputs.erdos_renyi_graph(cfg["n"], cfg["m"], seed, device)
     else:
         g = inputs.rmat_graph(cfg["n"], cfg["m"], seed, device)
-    torch.cuda.synchronize()
+    sync = torch.cuda.synchronize if torch.device(device).type == "cuda" else (lambda: None)
+    sync()
     t1 = time.time()
     feats = inputs.normal_features(cfg["n"], cfg["dim"], seed + 1, device,
                                    dtype=torch.float16 if cfg.get("fp16") else torch.float32)
-    torch.cuda.synchronize()
+    sync()
     dims = [cfg["dim"]] + [cfg["hidden"]] * len(cfg["fanouts"])
     layers = inputs.glorot_layers(dims, seed + 2)
     return g, feats, layers, {"graph_s": round(t1 - t0, 1), "features_s": round(time.time() - t1, 1)}
@@ -180,12 +181,23 @@ def algorithmic_bytes(nodes, ents, cfg, feat_bytes=4):
             "a_min": int(a_s + a_f + a_i + a_o), "flops": int(flops), "agg_l1": int(agg_l1), "flops_l1": int(flops_l1)}
 
 
-def _oracle_worker_init():
+_ORACLE_SHARED = {}
+
+
+def _oracle_worker_init(folder, n_arrays, cfg, np_layers):
+    """Runs once in every worker process: the graph arrays are memory-mapped from files the parent wrote (shared through
+    the page cache), and the worker keeps to one core."""
     try:
         from threadpoolctl import threadpool_limits
-        threadpool_limits(1)          # one core per worker: the oracle's matmul must not spread over the others' cores
+        _ORACLE_SHARED["limit"] = threadpool_limits(1)   # the oracle's matmul must not spread over the other workers' cores
     except Exception:
         pass
+    _ORACLE_SHARED.update(g_host=[np.load(os.path.join(folder, f"g{i}.npy"), mmap_mode="r") for i in range(n_arrays)],
+                          cfg=cfg, np_layers=np_layers)
+
+
+def _oracle_ready(_):
+    return os.getpid()
 
 
 def _oracle_sample(job):
@@ -204,31 +216,42 @@ def _oracle_forward(job):
     return len(ref["nbrs"])
 
 
-_ORACLE_SHARED = {}
-
-
 def oracle_time(g_host, feats, layers, cfg, target_rows, seeds, limit_s=20.0, workers=None):
     """The CPU oracle as it stands on a bounded sample of the same mini-batches, one mini-batch per worker process
     over the host cores this job may use.  Rounds of `workers` mini-batches until the time limit: the workers sample
     (Algorithm 1), the parent hands each its H^0 rows (the feature table lives on the GPU), the workers run the layers.
-    The workers are forked, so they share the graph arrays with the parent and never touch CUDA."""
+    The workers are fresh processes (spawned, never forked from a process that holds a CUDA context); they map the graph
+    arrays from files written once before the clock starts."""
     import multiprocessing as mp
+    import shutil
+    import tempfile
     cores = len(os.sched_getaffinity(0))
     workers = max(1, min(workers or cores, len(target_rows)))
-    _ORACLE_SHARED.update(g_host=g_host, cfg=cfg, np_layers=[(w.numpy(), n.numpy(), b.numpy()) for w, n, b in layers])
-    jobs = [(tg.tolist(), int(seed)) for tg, seed in zip(target_rows, seeds)]
-    done, edges = 0, 0
-    with mp.get_context("fork").Pool(workers, initializer=_oracle_worker_init) as pool:
-        t0 = time.time()
-        while done < len(jobs):
-            chunk = jobs[done:done + workers]
-            refs = pool.map(_oracle_sample, chunk, chunksize=1)
-            h0s = [feats[torch.as_tensor(r["node_ids"], dtype=torch.int64).to(feats.device)].float().cpu().numpy() for r in refs]
-            edges += sum(pool.map(_oracle_forward, list(zip(refs, h0s)), chunksize=1))
-            done += len(chunk)
-            if time.time() - t0 > limit_s:
-                break
-        dt = time.time() - t0
+    need = sum(int(a.nbytes) for a in g_host)
+    base = "/dev/shm" if os.path.isdir("/dev/shm") and shutil.disk_usage("/dev/shm").free > 1.2 * need else None
+    folder = tempfile.mkdtemp(prefix="mg_oracle_", dir=base)
+    try:
+        for i, a in enumerate(g_host):
+            np.save(os.path.join(folder, f"g{i}.npy"), np.asarray(a))
+        np_layers = [(w.numpy(), n.numpy(), b.numpy()) for w, n, b in layers]
+        small_cfg = {"fanouts": list(cfg["fanouts"])}
+        jobs = [(tg.tolist(), int(seed)) for tg, seed in zip(target_rows, seeds)]
+        done, edges = 0, 0
+        with mp.get_context("spawn").Pool(workers, initializer=_oracle_worker_init,
+                                          initargs=(folder, len(g_host), small_cfg, np_layers)) as pool:
+            pool.map(_oracle_ready, range(4 * workers), chunksize=1)      # every worker is up before the clock starts
+            t0 = time.time()
+            while done < len(jobs):
+                chunk = jobs[done:done + workers]
+                refs = pool.map(_oracle_sample, chunk, chunksize=1)
+                h0s = [feats[torch.as_tensor(r["node_ids"], dtype=torch.int64).to(feats.device)].float().cpu().numpy() for r in refs]
+                edges += sum(pool.map(_oracle_forward, list(zip(refs, h0s)), chunksize=1))
+                done += len(chunk)
+                if time.time() - t0 > limit_s:
+                    break
+            dt = time.time() - t0
+    finally:
+        shutil.rmtree(folder, ignore_errors=True)
     return {"batches": done, "seconds": dt, "batches_per_s": done / dt, "edges_per_s": edges / dt, "workers": workers,
             "cores_available": cores}
 
@@ -329,7 +352,8 @@ def main():
                             caps=None if cfg["n"] < 2_000_000 else {"max_nodes_per_batch": 1 << (23 if cfg.get("inout") else 19)})
     nodes, ents = probe.counts()
     caps = {"max_nodes_total": int(nodes.sum() * 1.3) + 1024, "max_entries_total": int(ents.sum() * 1.3) + 1024,
-            "max_nodes_per_batch": int(nodes.sum(1).max() * 1.5) + 64}
+            "max_nodes_per_batch": int(nodes.sum(1).max() * 1.5) + 64,
+            "max_inner_nodes_per_batch": int(nodes[:, :-1].sum(1).max() * 1.5) + 64}
     probe.free()
     dense = ctx.sample_many(step_targets(0).to(device), offs, cfg["fanouts"], step_seeds(0), caps=caps)
 
@@ -641,7 +665,8 @@ def run_out_of_core(args, peaks, rank, local_rank, world):
     probe = ctx.sample_many(tg0[0], offs, c["fanouts"], seeds0, caps={"max_nodes_per_batch": 1 << 19})
     nodes, ents = probe.counts()
     caps = {"max_nodes_total": int(nodes.sum() * 1.4) + 1024, "max_entries_total": int(ents.sum() * 1.4) + 1024,
-            "max_nodes_per_batch": int(nodes.sum(1).max() * 1.6) + 64}
+            "max_nodes_per_batch": int(nodes.sum(1).max() * 1.6) + 64,
+            "max_inner_nodes_per_batch": int(nodes[:, :-1].sum(1).max() * 1.6) + 64}
     probe.free()
     denses = [ctx.sample_many(tg0[0], offs, c["fanouts"], seeds0, caps=caps) for _ in range(3)]
     out_dev = torch.empty((G * T, c["hidden"]), dtype=torch.float32, device=device)

@@ -67,6 +67,11 @@ typedef struct mg_sample_caps {
     int64_t max_nodes_total;     /* sum over batches of |node_ids| */
     int64_t max_entries_total;   /* sum over batches of |nbrs| */
     int32_t max_nodes_per_batch; /* |node_ids| of one batch; sizes the per-batch id table */
+    int32_t max_inner_nodes_per_batch; /* nodes of one batch WITHOUT its farthest delta (targets and the deltas that are
+                                          sampled from).  When the last hop is deduplicated in shared memory only these
+                                          go through the id tables in global memory, so a bound here makes the tables
+                                          several times smaller (L2-resident at the bench's sizes).  0 = as large as
+                                          max_nodes_per_batch. */
 } mg_sample_caps;
 
 /* One batch's DENSE in the paper's layout (Section 4.1): node_ids = [Delta_0 .. Delta_k],
@@ -443,6 +448,10 @@ typedef struct mg_gat_model mg_gat_model;
 int mg_gat_model_create(mg_ctx* ctx, int32_t k, const int32_t* dims, const float* const* w, const float* const* a_src,
                         const float* const* a_dst, const float* const* bias, float negative_slope, int gemm_precision,
                         mg_gat_model** out);
+/* Attention heads of every layer of the model (1 .. 8; default 1): the columns of z, a_src and a_dst are cut into
+ * `heads` equal blocks, every block attends on its own (its own scores and softmax), the blocks' results are
+ * concatenated, so a layer's width stays dims[l + 1], which must be a multiple of `heads`.  Errors: MG_ERR_ARG. */
+int mg_gat_model_set_heads(mg_gat_model* m, int32_t heads);
 int mg_gat_model_free(mg_gat_model* m);
 
 /* Attention forward pass for every batch of `d`; out_dev (DEVICE) receives one row of dims[k] floats per target, batch

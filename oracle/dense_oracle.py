@@ -325,37 +325,47 @@ def sage_layer(dense, h_prev, w_self, w_nbr, bias, relu: bool, aggregator: str =
     return np.maximum(out, 0.0) if relu else out
 
 
-def gat_layer(dense, h_prev, w, a_src, a_dst, bias, relu: bool, slope: float = 0.2):
+def gat_layer(dense, h_prev, w, a_src, a_dst, bias, relu: bool, slope: float = 0.2, heads: int = 1):
     """One graph-attention layer (the GAT of Velickovic et al., which Section 7.1 trains as the second model) over
-    DENSE, single head: z = h W for every input row; for output row i with sampled neighbours j (repeats count) and
-    itself, e_ij = LeakyReLU(a_dst . z_i + a_src . z_j), alpha = softmax over {i} + neighbours, h'_i = sum alpha_ij z_j
-    + bias.  A node without neighbours attends to itself only."""
+    DENSE: z = h W for every input row; for output row i with sampled neighbours j (repeats count) and itself,
+    e_ij = LeakyReLU(a_dst . z_i + a_src . z_j), alpha = softmax over {i} + neighbours, h'_i = sum alpha_ij z_j + bias.
+    A node without neighbours attends to itself only.  With `heads` > 1 the columns of z (and of a_src, a_dst) are cut
+    into that many equal blocks, every block attends on its own with its own scores, and the blocks' results are
+    concatenated (the width of the layer stays that of W)."""
     h_prev = np.asarray(h_prev, dtype=np.float64)
     z = h_prev @ np.asarray(w, dtype=np.float64)
-    s_src = z @ np.asarray(a_src, dtype=np.float64)
-    s_dst = z @ np.asarray(a_dst, dtype=np.float64)
+    a_src = np.asarray(a_src, dtype=np.float64)
+    a_dst = np.asarray(a_dst, dtype=np.float64)
+    width = z.shape[1]
+    if heads < 1 or width % heads:
+        raise ValueError("the layer's width must be a multiple of the number of heads")
+    dh = width // heads
     first = dense["node_id_offsets"][1]
     n_rows = len(dense["node_ids"]) - first
-    repr_map, nbr_offsets = dense["repr_map"], dense["nbr_offsets"]
-    out = np.zeros((n_rows, z.shape[1]), dtype=np.float64)
-    for r in range(n_rows):
-        me = first + r
-        src = [me] + [repr_map[e] for e in range(nbr_offsets[r], nbr_offsets[r + 1])]
-        e = np.array([s_dst[me] + s_src[j] for j in src])
-        e = np.where(e > 0, e, slope * e)
-        a = np.exp(e - e.max())
-        a /= a.sum()
-        out[r] = (a[:, None] * z[src]).sum(axis=0)
+    out = np.zeros((n_rows, width), dtype=np.float64)
+    for hd in range(heads):
+        cols = slice(hd * dh, (hd + 1) * dh)
+        zh = z[:, cols]
+        s_src = zh @ a_src[cols]
+        s_dst = zh @ a_dst[cols]
+        for r in range(n_rows):
+            me = first + r
+            src = [me] + list(_neighbour_rows(dense, r))
+            e = np.array([s_dst[me] + s_src[j] for j in src])
+            e = np.where(e > 0, e, slope * e)
+            a = np.exp(e - e.max())
+            a /= a.sum()
+            out[r, cols] = (a[:, None] * zh[src]).sum(axis=0)
     out = out + np.asarray(bias, dtype=np.float64)
     return np.maximum(out, 0.0) if relu else out
 
 
-def gat_forward(dense, h0, layers, slope: float = 0.2):
+def gat_forward(dense, h0, layers, slope: float = 0.2, heads: int = 1):
     """k attention layers with Algorithm 2 between them; layers: (w, a_src, a_dst, bias); ReLU on all but the last."""
     h = np.asarray(h0, dtype=np.float64)
     cur = dense
     for i, (w, a_src, a_dst, bias) in enumerate(layers):
-        h = gat_layer(cur, h, w, a_src, a_dst, bias, relu=(i + 1 < len(layers)), slope=slope)
+        h = gat_layer(cur, h, w, a_src, a_dst, bias, relu=(i + 1 < len(layers)), slope=slope, heads=heads)
         cur = update_dense(cur)
     return h
 

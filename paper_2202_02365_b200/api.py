@@ -31,7 +31,7 @@ EXPORTS = [
     "mg_load_features", "mg_set_partition_source", "mg_set_resident", "mg_commit_resident", "mg_sample_many", "mg_sample_many_begin", "mg_sample_many_end", "mg_sample",
     "mg_dense_counts", "mg_dense_view", "mg_dense_export_many", "mg_dense_export_view", "mg_dense_free", "mg_model_create", "mg_model_set_aggregator", "mg_model_set_intermediates", "mg_model_free",
     "mg_forward", "mg_set_layer_window", "mg_keep_layer_outputs", "mg_forward_host_async", "mg_wait_output", "mg_forward_noalloc", "mg_gather_h0", "mg_layer_output", "mg_lp_prepare", "mg_lp_view", "mg_lp_free",
-    "mg_distmult_score", "mg_kernel_launches", "mg_profile", "mg_profile_read", "mg_comet_plan", "mg_comet_bias", "mg_comet_autotune", "mg_gat_model_create", "mg_gat_model_free", "mg_gat_forward", "mg_backward", "mg_model_grads", "mg_model_sgd_step", "mg_model_adagrad_step", "mg_dense_packed_ids", "mg_apply_embedding_sgd",
+    "mg_distmult_score", "mg_kernel_launches", "mg_profile", "mg_profile_read", "mg_comet_plan", "mg_comet_bias", "mg_comet_autotune", "mg_gat_model_create", "mg_gat_model_set_heads", "mg_gat_model_free", "mg_gat_forward", "mg_backward", "mg_model_grads", "mg_model_sgd_step", "mg_model_adagrad_step", "mg_dense_packed_ids", "mg_apply_embedding_sgd",
 ]
 
 
@@ -43,7 +43,7 @@ class MgError(RuntimeError):
 
 class SampleCaps(C.Structure):
     _fields_ = [("max_nodes_total", C.c_int64), ("max_entries_total", C.c_int64),
-                ("max_nodes_per_batch", C.c_int32)]
+                ("max_nodes_per_batch", C.c_int32), ("max_inner_nodes_per_batch", C.c_int32)]
 
 
 class DenseArrays(C.Structure):
@@ -264,6 +264,10 @@ class GatModel:
         ctx._check(ctx.lib.mg_gat_model_create(ctx.handle, C.c_int32(k), dims, arrs[0], arrs[1], arrs[2], arrs[3],
                                                C.c_float(negative_slope), C.c_int(precision), C.byref(self.handle)))
 
+    def set_heads(self, heads: int):
+        """Attention heads per layer: equal column blocks of every layer's width, concatenated."""
+        self.ctx._check(self.ctx.lib.mg_gat_model_set_heads(self.handle, C.c_int32(heads)))
+
     def free(self):
         if self.handle:
             self.ctx.lib.mg_gat_model_free(self.handle)
@@ -466,7 +470,7 @@ class Context:
         cp = None
         if caps is not None:
             cp = SampleCaps(int(caps.get("max_nodes_total", 0)), int(caps.get("max_entries_total", 0)),
-                            int(caps.get("max_nodes_per_batch", 0)))
+                            int(caps.get("max_nodes_per_batch", 0)), int(caps.get("max_inner_nodes_per_batch", 0)))
         self._check(fn(self.handle, _ptr(targets), C.c_int(targets.is_cuda), _ptr(offs),
                        C.c_int32(offs.numel() - 1), _ptr(fo), C.c_int32(fo.numel()), C.c_void_p(sd.ctypes.data),
                        C.byref(cp) if cp is not None else None, C.byref(d.handle)))
@@ -491,7 +495,7 @@ class Context:
         cp = None
         if caps is not None:
             cp = SampleCaps(int(caps.get("max_nodes_total", 0)), int(caps.get("max_entries_total", 0)),
-                            int(caps.get("max_nodes_per_batch", 0)))
+                            int(caps.get("max_nodes_per_batch", 0)), int(caps.get("max_inner_nodes_per_batch", 0)))
         self._check(self.lib.mg_sample(self.handle, _ptr(targets), C.c_int(targets.is_cuda), C.c_int32(targets.numel()),
                                        _ptr(fo), C.c_int32(fo.numel()), C.c_uint64(int(seed) & 0xFFFFFFFFFFFFFFFF),
                                        C.byref(cp) if cp is not None else None, C.byref(d.handle)))

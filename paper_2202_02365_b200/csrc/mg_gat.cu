@@ -31,6 +31,7 @@ struct mg_gat_model {
     int32_t dims[MG_MAX_HOPS + 1] = {0};
     int precision = MG_GEMM_TF32;
     float slope = 0.2f;
+    int32_t heads = 1;                       // attention heads per layer: equal column blocks of Z, a_src, a_dst
     float* w[MG_MAX_HOPS] = {nullptr};       // device [d_in, d_out]
     float* w_t[MG_MAX_HOPS] = {nullptr};     // device [d_out, d_in], rounded to TF32 for the tensor-core path
     float* a_src[MG_MAX_HOPS] = {nullptr};   // device [d_out]
@@ -175,6 +176,25 @@ __global__ void __launch_bounds__(kThreads) k_gat_scores(const float* __restrict
     }
 }
 
+// the same per head: s[row * heads + h] over the head's columns [h * dh, (h + 1) * dh)
+__global__ void __launch_bounds__(kThreads) k_gat_scores_heads(const float* __restrict__ z, const float* __restrict__ a_src,
+                                                               const float* __restrict__ a_dst, int64_t n_rows, int dim, int heads,
+                                                               float* s_src, float* s_dst) {
+    const int lane = threadIdx.x & 31;
+    const int dh = dim / heads;
+    const int64_t warps = (int64_t)gridDim.x * (kThreads / 32);
+    for (int64_t row = blockIdx.x * (int64_t)(kThreads / 32) + (threadIdx.x >> 5); row < n_rows; row += warps) {
+        const float* zr = z + row * dim;
+        for (int h = 0; h < heads; ++h) {
+            float ps = 0.f, pd = 0.f;
+            for (int c = h * dh + lane; c < (h + 1) * dh; c += 32) { const float v = zr[c]; ps = fmaf(v, a_src[c], ps); pd = fmaf(v, a_dst[c], pd); }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) { ps += __shfl_xor_sync(0xFFFFFFFFu, ps, o); pd += __shfl_xor_sync(0xFFFFFFFFu, pd, o); }
+            if (lane == 0) { s_src[row * heads + h] = ps; s_dst[row * heads + h] = pd; }
+        }
+    }
+}
+
 struct AttendArgs {
     GatGeom g;
     int32_t layer;              // 1 .. k
@@ -188,6 +208,7 @@ struct AttendArgs {
     int32_t dim, relu, round;
     float slope;
     float* out;                 // [n_rows, dim]
+    int32_t heads;              // > 1: s_src / s_dst hold `heads` values per row (k_gat_attend_heads)
 };
 
 __device__ __forceinline__ float leaky(float v, float slope) { return v > 0.f ? v : slope * v; }
@@ -241,7 +262,80 @@ __global__ void __launch_bounds__(kThreads) k_gat_attend(AttendArgs a) {
     }
 }
 
+constexpr int kMaxHeads = 8;
+
+// several heads: one warp per output row; per head a softmax over {self} + entries with that head's scores, then the
+// weighted sums of the Z rows, every column with the weights of the head it belongs to
+template <int W>
+__global__ void __launch_bounds__(kThreads) k_gat_attend_heads(AttendArgs a) {
+    const int lane = threadIdx.x & 31;
+    const int H = a.heads, dh = a.dim / a.heads;
+    const int64_t warps = (int64_t)gridDim.x * (kThreads / 32);
+    const int32_t* rb_in = a.g.rowbase + (int64_t)(a.layer - 1) * (a.g.B + 1);
+    int head_of[W];
+#pragma unroll
+    for (int q = 0; q < W; ++q) head_of[q] = min((lane + 32 * q) / dh, H - 1);
+    for (int64_t row = blockIdx.x * (int64_t)(kThreads / 32) + (threadIdx.x >> 5); row < a.n_rows; row += warps) {
+        int32_t b, local, node;
+        locate(a.g, a.layer, row, &b, &local, &node);
+        const int64_t in0 = rb_in[b];
+        const int64_t me = in0 + local;
+        const int32_t e0 = a.ent_off[node], e1 = a.ent_off[node + 1];
+        float sd[kMaxHeads], mx[kMaxHeads], inv[kMaxHeads];
+        for (int h = 0; h < H; ++h) {
+            sd[h] = a.s_dst[me * H + h];
+            const float self_score = leaky(sd[h] + a.s_src[me * H + h], a.slope);
+            float m = self_score;
+            for (int32_t e = e0 + lane; e < e1; e += 32) m = fmaxf(m, leaky(sd[h] + a.s_src[(in0 + a.ent_repr[e]) * H + h], a.slope));
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+            float den = lane == 0 ? __expf(self_score - m) : 0.f;
+            for (int32_t e = e0 + lane; e < e1; e += 32) den += __expf(leaky(sd[h] + a.s_src[(in0 + a.ent_repr[e]) * H + h], a.slope) - m);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xFFFFFFFFu, den, o);
+            mx[h] = m;
+            inv[h] = 1.f / den;
+        }
+        float acc[W];
+        {
+            const float* zr = a.z + me * a.dim;
+#pragma unroll
+            for (int q = 0; q < W; ++q) {
+                const int c = lane + 32 * q, h = head_of[q];
+                acc[q] = c < a.dim ? __expf(leaky(sd[h] + a.s_src[me * H + h], a.slope) - mx[h]) * inv[h] * zr[c] : 0.f;
+            }
+        }
+        for (int32_t e = e0; e < e1; ++e) {
+            const int64_t src = in0 + a.ent_repr[e];
+            const float* zr = a.z + src * a.dim;
+#pragma unroll
+            for (int q = 0; q < W; ++q) {
+                const int c = lane + 32 * q, h = head_of[q];
+                if (c < a.dim) acc[q] = fmaf(__expf(leaky(sd[h] + a.s_src[src * H + h], a.slope) - mx[h]) * inv[h], zr[c], acc[q]);
+            }
+        }
+        float* dst = a.out + row * a.dim;
+#pragma unroll
+        for (int q = 0; q < W; ++q) {
+            const int c = lane + 32 * q;
+            if (c >= a.dim) continue;
+            float v = acc[q] + a.bias[c];
+            if (a.relu) v = fmaxf(v, 0.f);
+            dst[c] = a.round ? round_tf32(v) : v;
+        }
+    }
+}
+
 }  // namespace
+
+extern "C" int mg_gat_model_set_heads(mg_gat_model* m, int32_t heads) {
+    if (!m) return MG_ERR_ARG;
+    if (heads < 1 || heads > kMaxHeads) return mg_fail(m->ctx, MG_ERR_ARG, "heads must be in [1, %d]", kMaxHeads);
+    for (int l = 1; l <= m->k; ++l)
+        if (m->dims[l] % heads) return mg_fail(m->ctx, MG_ERR_ARG, "layer width %d is not a multiple of %d heads", m->dims[l], heads);
+    m->heads = heads;
+    return MG_OK;
+}
 
 extern "C" int mg_gat_model_free(mg_gat_model* m) {
     if (!m) return MG_OK;
@@ -321,7 +415,7 @@ extern "C" int mg_gat_forward(mg_ctx* ctx, const mg_gat_model* m, mg_dense* d, f
     size_t need_x = (size_t)d->h_hdr.rows_total[0] * m->dims[0], need_z = 0, need_s = 0, need_h = 0;
     for (int l = 1; l <= k; ++l) {
         need_z = std::max(need_z, (size_t)d->h_hdr.rows_total[l - 1] * m->dims[l]);
-        need_s = std::max(need_s, (size_t)d->h_hdr.rows_total[l - 1] * 2);
+        need_s = std::max(need_s, (size_t)d->h_hdr.rows_total[l - 1] * 2 * m->heads);
         if (l < k) need_h = std::max(need_h, (size_t)d->h_hdr.rows_total[l] * m->dims[l]);
     }
     int rc;
@@ -350,8 +444,9 @@ extern "C" int mg_gat_forward(mg_ctx* ctx, const mg_gat_model* m, mg_dense* d, f
         const int d_in = m->dims[l - 1], d_out = m->dims[l];
         const int64_t rows_in = d->h_hdr.rows_total[l - 1], rows_out = d->h_hdr.rows_total[l];
         float* s_src = ctx->gat_s;
-        float* s_dst = ctx->gat_s + rows_in;
-        const bool fused_scores = tf32 && d_out <= 256;   // the GEMM's epilogue also leaves Z a_src and Z a_dst
+        const int H = m->heads;
+        float* s_dst = ctx->gat_s + rows_in * H;
+        const bool fused_scores = tf32 && d_out <= 256 && H == 1;   // the GEMM's epilogue also leaves Z a_src and Z a_dst
         {
             ProfScope ps(ctx, PH_GEMM, 1);
             if (fused_scores) {
@@ -366,14 +461,22 @@ extern "C" int mg_gat_forward(mg_ctx* ctx, const mg_gat_model* m, mg_dense* d, f
             }
         }
         ProfScope ps(ctx, PH_AGG_REST, 2);
-        if (!fused_scores) k_gat_scores<<<grid, kThreads, 0, st>>>(ctx->gat_z, m->a_src[l - 1], m->a_dst[l - 1], rows_in, d_out, s_src, s_dst);
+        if (H > 1) k_gat_scores_heads<<<grid, kThreads, 0, st>>>(ctx->gat_z, m->a_src[l - 1], m->a_dst[l - 1], rows_in, d_out, H, s_src, s_dst);
+        else if (!fused_scores) k_gat_scores<<<grid, kThreads, 0, st>>>(ctx->gat_z, m->a_src[l - 1], m->a_dst[l - 1], rows_in, d_out, s_src, s_dst);
         AttendArgs a;
         a.g = geom; a.layer = l; a.ent_off = d->ent_off; a.ent_repr = d->ent_repr; a.z = ctx->gat_z; a.s_src = s_src; a.s_dst = s_dst;
         a.bias = m->bias[l - 1]; a.n_rows = rows_out; a.dim = d_out; a.relu = l < k; a.round = (tf32 && l < k) ? 1 : 0;
         a.slope = m->slope;
+        a.heads = H;
         a.out = l == k ? out_dev : ctx->gat_h[l & 1];
         const int slices = (d_out + 31) / 32;   // instantiations for rows of up to 32, 64, 128, 256, 512 floats
-        if (slices <= 1) k_gat_attend<1><<<grid, kThreads, 0, st>>>(a);
+        if (H > 1) {
+            if (slices <= 1) k_gat_attend_heads<1><<<grid, kThreads, 0, st>>>(a);
+            else if (slices <= 2) k_gat_attend_heads<2><<<grid, kThreads, 0, st>>>(a);
+            else if (slices <= 4) k_gat_attend_heads<4><<<grid, kThreads, 0, st>>>(a);
+            else if (slices <= 8) k_gat_attend_heads<8><<<grid, kThreads, 0, st>>>(a);
+            else k_gat_attend_heads<kMaxWidthPerLane><<<grid, kThreads, 0, st>>>(a);
+        } else if (slices <= 1) k_gat_attend<1><<<grid, kThreads, 0, st>>>(a);
         else if (slices <= 2) k_gat_attend<2><<<grid, kThreads, 0, st>>>(a);
         else if (slices <= 4) k_gat_attend<4><<<grid, kThreads, 0, st>>>(a);
         else if (slices <= 8) k_gat_attend<8><<<grid, kThreads, 0, st>>>(a);

@@ -1457,15 +1457,23 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
                        (long long)cap_nodes, (long long)cap_entries);
     // id table of a mini-batch: 1.625 slots per node it may hold (load factor <= 0.62 for linear probing), any size:
     // its traffic is random 32-byte sectors, so every slot that is not needed costs DRAM bandwidth
-    const int64_t want_slots = std::max<int64_t>(16, (cap_batch + cap_batch / 2 + cap_batch / 8 + 7) / 8 * 8);
-    if (want_slots > (1ll << MG_SLOT_BITS)) return mg_fail(ctx, MG_ERR_CAPACITY, "max_nodes_per_batch above %d", (int)((1ll << MG_SLOT_BITS) * 8 / 13));
-    const int32_t table_size = (int32_t)want_slots;
+    // (sized below, once it is known whether the last hop goes through it)
     // The last hop is deduplicated in shared memory (k_bucket_entries, k_dedupe_last) when a mini-batch's nodes fit the
     // tables of a few blocks: S slots per block, filled to 92 % at most when the mini-batch is at its capacity (the
     // buckets of a hash differ by a per cent or so at these sizes), nb blocks per mini-batch.
     const int32_t dedup_slots = (int32_t)std::min<int64_t>(kDedupMaxSlots, (cap_batch + cap_batch / 4 + 64 + 1023) / 1024 * 1024);
     const int64_t dedup_nb = (cap_batch + (cap_batch * 7 + 79) / 80 + dedup_slots - 1) / dedup_slots;
     const bool smem_last = dedup_nb <= kDedupMaxBuckets && dedup_nb * n_batches < (1ll << 24) && !getenv("MG_GLOBAL_TABLES");
+    // With the last hop deduplicated in shared memory the global tables only ever hold the nodes that are sampled from
+    // (targets and the inner deltas): a caller who bounds those gets tables several times smaller.
+    int64_t table_nodes = cap_batch;
+    if (smem_last && caps && caps->max_inner_nodes_per_batch > 0) {
+        table_nodes = std::min<int64_t>(cap_batch, caps->max_inner_nodes_per_batch);
+        for (int b = 0; b < n_batches; ++b) table_nodes = std::max<int64_t>(table_nodes, target_offsets[b + 1] - target_offsets[b]);
+    }
+    const int64_t want_slots = std::max<int64_t>(16, (table_nodes + table_nodes / 2 + table_nodes / 8 + 7) / 8 * 8);
+    if (want_slots > (1ll << MG_SLOT_BITS)) return mg_fail(ctx, MG_ERR_CAPACITY, "max_nodes_per_batch above %d", (int)((1ll << MG_SLOT_BITS) * 8 / 13));
+    const int32_t table_size = (int32_t)want_slots;
     if ((int64_t)table_size * n_batches >= (1ll << 31))
         return mg_fail(ctx, MG_ERR_CAPACITY, "n_batches x id-table size must stay below 2^31: pass a smaller max_nodes_per_batch or fewer batches");
     const int id_bits = std::max(1, ilog2_ceil(N));

@@ -293,22 +293,22 @@ def lp_edges(graph: Graph, resident_mask: torch.Tensor | None, n_edges: int, see
     """Training edges for link prediction: CSR slots drawn uniformly among those
     whose endpoints are both resident.  Returns (src, rel, dst) int32 CPU tensors.
     """
-    g = _gen(seed, "cpu")
-    off = graph.row_offsets.cpu()
-    nbrs = graph.nbrs.cpu()
+    g = _gen(seed, "cpu")                  # the draws come from the CPU generator whatever device holds the graph
+    off, nbrs = graph.row_offsets, graph.nbrs
+    dev = nbrs.device
+    rm = None if resident_mask is None else resident_mask.to(dev)
     n_slots = int(nbrs.numel())
     src_l, rel_l, dst_l = [], [], []
     have = 0
     while have < n_edges:
-        slots = torch.randint(0, n_slots, (int((n_edges - have) * 1.5) + 64,), generator=g)
+        slots = torch.randint(0, n_slots, (int((n_edges - have) * 1.5) + 64,), generator=g).to(dev)
         dst = torch.searchsorted(off, slots, right=True) - 1
         src = nbrs[slots].to(torch.int64)
-        if resident_mask is not None:
-            rm = resident_mask.cpu()
+        if rm is not None:
             keep = rm[dst] & rm[src]
             slots, dst, src = slots[keep], dst[keep], src[keep]
-        rel = graph.edge_rel.cpu()[slots] if graph.edge_rel is not None else torch.zeros_like(src)
-        src_l.append(src); rel_l.append(rel.to(torch.int64)); dst_l.append(dst)
+        rel = graph.edge_rel[slots] if graph.edge_rel is not None else torch.zeros_like(src)
+        src_l.append(src.cpu()); rel_l.append(rel.to(torch.int64).cpu()); dst_l.append(dst.cpu())
         have += int(src.numel())
     src = torch.cat(src_l)[:n_edges].to(torch.int32)
     rel = torch.cat(rel_l)[:n_edges].to(torch.int32)

@@ -663,7 +663,8 @@ def test_full_size_config3_in_bench_launch_configuration():
     probe = ctx.sample_many(tg.reshape(-1).cuda(), offs, cfg["fanouts"], seeds, caps={"max_nodes_per_batch": 1 << 19})
     nodes, ents = probe.counts()
     caps = {"max_nodes_total": int(nodes.sum() * 1.3) + 1024, "max_entries_total": int(ents.sum() * 1.3) + 1024,
-            "max_nodes_per_batch": int(nodes.sum(1).max() * 1.5) + 64}
+            "max_nodes_per_batch": int(nodes.sum(1).max() * 1.5) + 64,
+            "max_inner_nodes_per_batch": int(nodes[:, :-1].sum(1).max() * 1.5) + 64}
     probe.free()
     d = ctx.sample_many(tg.reshape(-1).cuda(), offs, cfg["fanouts"], seeds, caps=caps)
     model = ctx.model(layers, mg.GEMM_TF32)
@@ -697,7 +698,8 @@ def test_full_size_config3_in_bench_launch_configuration():
     probe = ctx.sample_many(tg2, offs2, cfg["fanouts"], seeds[:G2], caps={"max_nodes_per_batch": 1 << 23})
     nodes, ents = probe.counts()
     caps = {"max_nodes_total": int(nodes.sum() * 1.3) + 1024, "max_entries_total": int(ents.sum() * 1.3) + 1024,
-            "max_nodes_per_batch": int(nodes.sum(1).max() * 1.5) + 64}
+            "max_nodes_per_batch": int(nodes.sum(1).max() * 1.5) + 64,
+            "max_inner_nodes_per_batch": int(nodes[:, :-1].sum(1).max() * 1.5) + 64}
     probe.free()
     d = ctx.sample_many(tg2, offs2, cfg["fanouts"], seeds[:G2], caps=caps)
     out2 = torch.empty((G2 * T, cfg["hidden"]), dtype=torch.float32, device="cuda")
@@ -771,7 +773,8 @@ def test_config4_out_of_core_at_its_stated_size():
         probe = ctx.sample_many(tg.reshape(-1), offs, c["fanouts"], seeds, caps={"max_nodes_per_batch": 1 << 19})
         nodes, ents = probe.counts()
         caps = {"max_nodes_total": int(nodes.sum() * 1.4) + 1024, "max_entries_total": int(ents.sum() * 1.4) + 1024,
-                "max_nodes_per_batch": int(nodes.sum(1).max() * 1.6) + 64}
+                "max_nodes_per_batch": int(nodes.sum(1).max() * 1.6) + 64,
+                "max_inner_nodes_per_batch": int(nodes[:, :-1].sum(1).max() * 1.6) + 64}
         probe.free()
         d = ctx.sample_many(tg.reshape(-1), offs, c["fanouts"], seeds, caps=caps)
         out = torch.empty((G * T, c["hidden"]), dtype=torch.float32, device="cuda")
@@ -1094,6 +1097,20 @@ def test_last_hop_deduplication_paths(tiny, cap_batch):
     with pytest.raises(mg.MgError) as e:
         ctx.sample_many(torch.tensor([3, 9, 3], dtype=torch.int32), [0, 3], [2], [1], caps=caps)
     assert e.value.code == -4
+    # a bound on the nodes that are sampled from (all but the farthest delta) shrinks the global id tables where the
+    # last hop goes through shared memory: same arrays when the bound holds, a capacity error (nothing out of bounds)
+    # when it does not
+    if cap_batch != 900_000:
+        fanouts = [5, 4, 3]
+        refs = [O.sample_dense(view, tg[b].tolist(), fanouts, seeds[b]) for b in range(len(sizes))]
+        inner = max(len(r["node_ids"]) - r["node_id_offsets"][1] for r in refs)
+        tight = dict(caps or {"max_nodes_per_batch": 20_000}, max_inner_nodes_per_batch=inner)
+        d = ctx.sample_many(torch.cat(tg), offs, fanouts, seeds, caps=tight)
+        for b in range(len(sizes)):
+            assert_dense_equal(d.view(b), refs[b])
+        with pytest.raises(mg.MgError) as e:
+            ctx.sample_many(torch.cat(tg), offs, fanouts, seeds, caps=dict(tight, max_inner_nodes_per_batch=inner // 3))
+        assert e.value.code == -5
 
 
 def test_comet_epoch_drives_the_partition_buffer():
@@ -1202,6 +1219,35 @@ def test_graph_attention_forward(tiny, dims, fanouts):
         total = O.sage_layer(r, h0, flat[0][0].numpy(), flat[0][0].numpy(), np.zeros(dims[1]), relu=False, aggregator="sum")
         counts = np.diff(r["nbr_offsets"])[:sizes[3], None]
         close(out[offs[3]:offs[4]].cpu().numpy(), total / (counts + 1) + flat[0][3].numpy(), 2e-5)
+
+
+@pytest.mark.parametrize("dims,heads", [([16, 24, 8], 2), ([16, 32, 32], 8), ([16, 100], 4), ([16, 264, 12], 3)])
+def test_graph_attention_with_several_heads(tiny, dims, heads):
+    """Multi-head attention: every head attends on its own column block; fp32 and tensor-core paths against the oracle,
+    widths whose head blocks do and do not line up with the 32-column slices a lane owns."""
+    g, feats = tiny
+    ctx = make_ctx(g, feats)
+    sizes = [120, 1, 77]
+    tg = [inputs.distinct_targets(10_000, s_, seed=50 + i) for i, s_ in enumerate(sizes)]
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    seeds = [21, 22, 23]
+    fanouts = [5, 3][:len(dims) - 1]
+    d = ctx.sample_many(torch.cat(tg), offs, fanouts, seeds)
+    view = oracle_view(g)
+    layers = _gat_layers(dims, seed=heads)
+    np_layers = [tuple(t.numpy() for t in l) for l in layers]
+    for prec, rtol in ((mg.GEMM_FP32, 5e-5), (mg.GEMM_TF32, RTOL_TC)):
+        gm = ctx.gat_model(layers, prec)
+        gm.set_heads(heads)
+        out = torch.empty((int(offs[-1]), dims[-1]), dtype=torch.float32, device="cuda")
+        ctx.gat_forward(gm, d, out)
+        for b in range(3):
+            ref = O.sample_dense(view, tg[b].tolist(), fanouts, seeds[b])
+            want = O.gat_forward(ref, feats.numpy()[ref["node_ids"]], np_layers, heads=heads)
+            close(out[offs[b]:offs[b + 1]].cpu().numpy(), want, rtol)
+    with pytest.raises(mg.MgError) as e:
+        gm.set_heads(5)                              # no layer width here is a multiple of 5
+    assert e.value.code == -1
 
 
 def test_graph_attention_errors_and_fp16_features():

@@ -716,6 +716,32 @@ def test_gat_forward_two_layers_uses_algorithm_2_between_layers():
     np.testing.assert_allclose(got, H[targets].numpy(), rtol=1e-9, atol=1e-11)
 
 
+def test_gat_heads_are_independent_single_head_layers_on_column_blocks():
+    """Multi-head attention: one head reproduces the single-head layer; H heads equal H single-head layers run on the
+    column blocks of W, a_src, a_dst and concatenated; with zero attention vectors every head is the plain mean."""
+    off, nb = _random_graph(90, 700, 31)
+    d = O.sample_dense(O.GraphView(off, nb), [4, 40, 77, 12], [4, 3], seed=3)
+    rng = np.random.default_rng(6)
+    h0 = rng.standard_normal((len(d["node_ids"]), 6))
+    w, a_s, a_d, b = rng.standard_normal((6, 12)), rng.standard_normal(12), rng.standard_normal(12), rng.standard_normal(12)
+    np.testing.assert_array_equal(O.gat_layer(d, h0, w, a_s, a_d, b, relu=True), O.gat_layer(d, h0, w, a_s, a_d, b, relu=True, heads=1))
+    for heads in (2, 3, 4):
+        dh = 12 // heads
+        got = O.gat_layer(d, h0, w, a_s, a_d, b, relu=False, heads=heads)
+        blocks = [O.gat_layer(d, h0, w[:, i * dh:(i + 1) * dh], a_s[i * dh:(i + 1) * dh], a_d[i * dh:(i + 1) * dh],
+                              b[i * dh:(i + 1) * dh], relu=False) for i in range(heads)]
+        np.testing.assert_allclose(got, np.concatenate(blocks, axis=1), rtol=1e-13, atol=1e-13)
+        uniform = O.gat_layer(d, h0, w, 0 * a_s, 0 * a_d, b, relu=False, heads=heads)
+        np.testing.assert_allclose(uniform, O.gat_layer(d, h0, w, 0 * a_s, 0 * a_d, b, relu=False), rtol=1e-13, atol=1e-13)
+    with pytest.raises(ValueError):
+        O.gat_layer(d, h0, w, a_s, a_d, b, relu=False, heads=5)
+    # two layers: heads apply to every layer
+    layers = [(w, a_s, a_d, b), (rng.standard_normal((12, 4)), rng.standard_normal(4), rng.standard_normal(4), rng.standard_normal(4))]
+    two = O.gat_forward(d, h0, layers, heads=2)
+    h1 = O.gat_layer(d, h0, *layers[0], relu=True, heads=2)
+    np.testing.assert_allclose(two, O.gat_layer(O.update_dense(d), h1, *layers[1], relu=False, heads=2), rtol=1e-13, atol=1e-13)
+
+
 # ---------------------------------------------------------------- backward pass
 @pytest.mark.parametrize("aggregator", ["mean", "sum"])
 def test_backward_equals_central_finite_differences(aggregator):
