@@ -1246,7 +1246,7 @@ def test_graph_attention_with_several_heads(tiny, dims, heads):
             want = O.gat_forward(ref, feats.numpy()[ref["node_ids"]], np_layers, heads=heads)
             close(out[offs[b]:offs[b + 1]].cpu().numpy(), want, rtol)
     with pytest.raises(mg.MgError) as e:
-        gm.set_heads(5)                              # no layer width here is a multiple of 5
+        gm.set_heads(7)                              # no layer width here is a multiple of 7
     assert e.value.code == -1
 
 
