@@ -84,7 +84,6 @@ struct FusedArgs {
     int32_t relu;
     int32_t sum_aggr;            // neighbour term = sum of the sampled neighbours instead of their mean
     int32_t out_f16;             // the output rows are stored as fp16 (an intermediate layer of a model that keeps them so)
-    uint32_t prefetch_bytes;     // bytes of a source row the planner asks L2 for ahead of the gather (0 = no prefetch)
     const float* bias;
     float* out;                  // [M, N]
     uint32_t* error;
@@ -580,18 +579,11 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
                         const int32_t j = j0 + u * 32 + lane;
-                        if (j < total) {
-                            const int32_t sr = source_row<FIRST>(a, base[u], key[u]);
-                            src_rows[slot][j] = sr;
-                            // the planner runs up to four row blocks ahead of the gather warps: asking L2 for the row now
-                            // turns the gather's DRAM latency into an L2 hit, and holds no register while it is in flight
-                            if (a.prefetch_bytes) prefetch_l2(a.src_base + (size_t)(uint32_t)sr * (size_t)a.src_row_bytes, a.prefetch_bytes);
-                        }
+                        if (j < total) src_rows[slot][j] = source_row<FIRST>(a, base[u], key[u]);
                     }
                 }
             }
             if (lane == 0) plan_total[slot] = cached ? total : -1;
-            if (a.prefetch_bytes && rm.z >= 0) prefetch_l2(a.src_base + (size_t)(uint32_t)rm.x * (size_t)a.src_row_bytes, a.prefetch_bytes);   // the row's own representation
             __syncwarp();
             if (cached) {
                 // lane = row: its first kUnroll source rows, padded with its own source row
@@ -734,8 +726,6 @@ int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_ou
     a.src_base = layer == 1 ? ctx->slots : reinterpret_cast<const char*>(h_prev);
     a.src_row_bytes = layer == 1 ? (uint32_t)ctx->row_bytes : (uint32_t)d_in * (in_f16 ? 2u : 4u);
     a.out_f16 = out_f16;
-    // whole source rows (a multiple of 16 bytes); MG_NO_PREFETCH switches the hint off for measurements
-    a.prefetch_bytes = getenv("MG_NO_PREFETCH") ? 0u : (uint32_t)((size_t)d_in * (layer == 1 ? (ctx->feat_dtype == MG_DTYPE_F16 ? 2 : 4) : (in_f16 ? 2 : 4)));
     a.relu = flags & 1;
     a.sum_aggr = (flags >> 1) & 1;
     a.bias = bias; a.out = h_out;
