@@ -28,11 +28,27 @@ namespace {
 
 constexpr int BM = 128;               // output rows per tile
 constexpr int KC = 32;                // floats per K slice (one 128-byte swizzle row)
+// Warp roles, laid out so that every role fills whole warpgroups (four consecutive warps):
+//   warps 0..15   producers (gather + segment mean)         four warpgroups
+//   warps 16..19  epilogue (tensor memory -> global)        one warpgroup
+//   warp 20 TMA (weights), warp 21 MMA + tensor memory, warps 22..23 planners: one warpgroup
+// Every thread has 80 registers (768 x 80 = 61,440 of the SM's 65,536).  A build option moves registers between the
+// warpgroups with `setmaxnreg` (-DMG_FUSED_SETMAXNREG=1 -DMG_FUSED_MAXNREG=72 -DMG_REG_PROD=80 -DMG_REG_EPI=56
+// -DMG_REG_CTL=56: the CTA then leaves room for a 256-thread block of the sampler beside it); it is off because every
+// such configuration measured 15 % slower in the first layer than the plain one.
 constexpr int kProducerWarps = 16;
-constexpr int kFirstProducerWarp = 6; // warp 0 TMA, warp 1 MMA + tensor memory, warps 2..5 epilogue
-constexpr int kPlannerWarps = 2;      // after the producers: they prepare the producers' row blocks ahead of time
-constexpr int kFirstPlannerWarp = kFirstProducerWarp + kProducerWarps;
+constexpr int kFirstProducerWarp = 0;
+constexpr int kFirstEpilogueWarp = 16;
+constexpr int kTmaWarp = 20, kMmaWarp = 21;
+constexpr int kPlannerWarps = 2;
+constexpr int kFirstPlannerWarp = 22;
 constexpr int kFusedThreads = (kFirstPlannerWarp + kPlannerWarps) * 32;  // 768
+#ifndef MG_FUSED_MAXNREG
+#define MG_FUSED_MAXNREG 80
+#endif
+#ifndef MG_FUSED_SETMAXNREG
+#define MG_FUSED_SETMAXNREG 0
+#endif
 constexpr int kMaxStages = 8;
 constexpr int kGroupCols = 128;                  // input columns whose (self, mean) slices the producers fill together (TF32 operands)
 // With half-precision base representations the first layer can run its GEMM in kind::f16 (fp16 operands, fp32
@@ -162,9 +178,6 @@ template <> struct PieceSum<true> {
     static __device__ __forceinline__ uint4 self_operand(const uint4& r) { return r; }   // fp16 rows are operands as they are
 };
 
-#ifndef MG_FUSED_MAXNREG
-#define MG_FUSED_MAXNREG 80
-#endif
 template <bool FIRST, bool HALF, bool F16>
 __global__ void __cluster_dims__(2, 1, 1) __maxnreg__(MG_FUSED_MAXNREG)
 k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_out, FusedArgs a) {
@@ -210,7 +223,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out) : "memory");
     }
-    if (warp == 1) {
+    if (warp == kMmaWarp) {
         // the same warp of both CTAs allocates the pair's tensor memory
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"((uint32_t)a.tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
@@ -222,7 +235,27 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
     const uint32_t acc_stride = (uint32_t)(a.tmem_cols / kAccBufs);  // columns per accumulator buffer (a multiple of 32)
     const int n_groups = (a.d_in_pad + GC - 1) / GC;
 
-    if (warp == 0) {
+    // (Build option) registers move from the epilogue's and the control warpgroup to the producers': each warpgroup
+    // executes its one setmaxnreg at the head of its own branch, so that the compiler budgets the branch with it (the
+    // decreases never wait, the increases wait for them; the static_assert keeps the sum within the launch allocation).
+#define MG_STR2(x) #x
+#define MG_STR(x) MG_STR2(x)
+#if MG_FUSED_SETMAXNREG
+#define MG_REG_SET(n) do { if ((n) < MG_FUSED_MAXNREG) asm volatile("setmaxnreg.dec.sync.aligned.u32 " MG_STR(n) ";" ::: "memory"); \
+                           else if ((n) > MG_FUSED_MAXNREG) asm volatile("setmaxnreg.inc.sync.aligned.u32 " MG_STR(n) ";" ::: "memory"); } while (0)
+#else
+#define MG_REG_SET(n)
+#endif
+#ifndef MG_REG_PROD
+#define MG_REG_PROD 80
+#define MG_REG_EPI 56
+#define MG_REG_CTL 56
+#endif
+    static_assert(MG_FUSED_SETMAXNREG == 0 || 16 * MG_REG_PROD + 4 * MG_REG_EPI + 4 * MG_REG_CTL <= 24 * MG_FUSED_MAXNREG,
+                  "the warpgroups' registers must fit what the CTA was launched with");
+    if (warp >= kTmaWarp) {
+    MG_REG_SET(MG_REG_CTL);
+    if (warp == kTmaWarp) {
         // ---------------- weight slices: each CTA stages its half of the output columns (TMA from L2) ----------------
         if (lane == 0) {
             uint32_t cnt = 0;
@@ -242,7 +275,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     }
         }
         __syncwarp();
-    } else if (warp == 1) {
+    } else if (warp == kMmaWarp) {
         // ---------------- MMA issue: one thread of the leader, for both CTAs ----------------
         if (lane == 0 && leader) {
             // M = 128 over the pair: 64 rows (a half tile) of each CTA per instruction
@@ -284,7 +317,75 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     }
         }
         __syncwarp();
-    } else if (warp < kFirstProducerWarp) {
+    } else {
+        // ---------------- planners: row blocks of 32 rows, prepared ahead of the producers ----------------
+        // A planner warp takes every kPlannerWarps-th row block: lane = row.  It reads the rows' metadata, scans the
+        // entry counts, and translates the block's entries to source rows in shared memory, so that the producers'
+        // gathers depend on nothing but shared memory.
+        const int plw = warp - kFirstPlannerWarp;
+        const int32_t* keys = FIRST ? a.ent_nbrs : a.ent_repr;
+        bool ok = true;
+        for (uint32_t q = plw; ok; q += kPlannerWarps) {
+            if (q / kBlocksPerTile >= my_iters) break;
+            const int64_t t = tile_of(q / kBlocksPerTile);   // past the end for the peer of an odd last tile: all padding
+            const int slot = q % kPlanSlots;
+            if (q >= (uint32_t)kPlanSlots && !mbar_wait(&plan_empty[slot], ((q / kPlanSlots) - 1) & 1)) {
+                if (lane == 0) atomicExch(a.error, 17u);
+                ok = false;
+            }
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            const int64_t r = a.row_lo + t * BM + (q % kBlocksPerTile) * kBlockRows + lane;
+            int4 rm = make_int4(a.safe_src, 0, -1, 0);
+            if (r < a.M) rm = __ldg(a.row_meta + r);   // (self source row, first entry, count, first H^{l-1} row of the batch)
+            const int32_t end = (int32_t)warp_incl_scan((uint32_t)max(rm.z, 0));   // end of the row's cached entries
+            const int32_t total = __shfl_sync(0xFFFFFFFFu, end, 31);
+            const bool cached = total <= kKeyCap;
+            const int32_t in_base = rm.w, koff = end - max(rm.z, 0);
+            meta[slot][lane] = make_int4(rm.x, rm.y, rm.z, cached ? koff : in_base);
+            if (cached) {
+                // entry j belongs to the first row whose end exceeds j
+                for (int32_t j0 = 0; j0 < total; j0 += 32 * 4) {
+                    int32_t key[4], base[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int32_t j = j0 + u * 32 + lane;
+                        int lo = 0, hi = 31;
+#pragma unroll
+                        for (int s = 0; s < 5; ++s) {
+                            const int mid = (lo + hi) >> 1;
+                            const int32_t e = __shfl_sync(0xFFFFFFFFu, end, mid);
+                            if (lo < hi) { if (e > j) hi = mid; else lo = mid + 1; }
+                        }
+                        const int32_t e0 = __shfl_sync(0xFFFFFFFFu, rm.y, lo), k0 = __shfl_sync(0xFFFFFFFFu, koff, lo);
+                        base[u] = __shfl_sync(0xFFFFFFFFu, in_base, lo);
+                        key[u] = j < total ? __ldg(keys + e0 + (j - k0)) : 0;
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int32_t j = j0 + u * 32 + lane;
+                        if (j < total) src_rows[slot][j] = source_row<FIRST>(a, base[u], key[u]);
+                    }
+                }
+            }
+            if (lane == 0) plan_total[slot] = cached ? total : -1;
+            __syncwarp();
+            if (cached) {
+                // lane = row: its first kUnroll source rows, padded with its own source row
+                int32_t fr[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) fr[j] = (j < kUnroll && j < rm.z) ? src_rows[slot][koff + j] : rm.x;
+                fr[5] = __float_as_int(rm.z > 0 ? (a.sum_aggr ? 1.f : 1.f / (float)rm.z) : 0.f);   // the mean's factor (1 for a sum)
+                *reinterpret_cast<int4*>(&first_rows[slot][lane][0]) = make_int4(fr[0], fr[1], fr[2], fr[3]);
+                *reinterpret_cast<int4*>(&first_rows[slot][lane][4]) = make_int4(fr[4], fr[5], fr[6], fr[7]);
+                __syncwarp();
+            }
+            if (lane == 0) mbar_arrive(&plan_full[slot]);
+        }
+    }
+    } else if (warp >= kFirstEpilogueWarp) {
+    MG_REG_SET(MG_REG_EPI);
+    {
         // ---------------- epilogue: tensor memory -> bias, ReLU -> global ----------------
         // A half tile's accumulator: rows 0..63 of output columns [0, BN/2) in lanes 0..63, the same rows of columns
         // [BN/2, BN) in lanes 64..127.  Warp quadrant q reads lanes 32q..32q+31.
@@ -299,22 +400,25 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
             tc_fence_after();
             const int64_t row0 = a.row_lo + t * BM + (hu & 1) * HM + (lane_group & 1) * 32;
             uint8_t* stage = reinterpret_cast<uint8_t*>(out_stage[lane_group]);
-            for (int c0 = 0; c0 < n_cols; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld_32(tmem_base + buf * acc_stride + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)c0, v);
+            // 16 accumulator columns at a time (few registers); two such steps fill one 32-column fp32 box of the TMA
+            // store, four a 64-column fp16 box
+            for (int c0 = 0; c0 < n_cols; c0 += 16) {
+                uint32_t v[16];
+                tmem_ld_16(tmem_base + buf * acc_stride + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)c0, v);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                const int ncol0 = col_base + c0;   // first output column of this slice
+                const int ncol0 = col_base + c0;   // first output column of this step
                 if (row0 >= a.M || ncol0 >= a.N) continue;
                 if (a.out_f16) {
-                    // fp16 output (widths that are multiples of 128 only): two accumulator slices make one 64-column box,
-                    // 128 bytes per row, so a row of the next layer's input is again fetched in 512-byte requests
-                    const int piece0 = (c0 & 32) ? 4 : 0;
-                    if (!piece0) {
+                    // fp16 output (widths that are multiples of 128 only): 128 bytes per row and box, so a row of the next
+                    // layer's input is again fetched in 512-byte requests
+                    const int pbase = (c0 & 63) >> 3;    // first 16-byte piece (8 columns) of this step in the box's rows
+                    if (pbase == 0) {
+                        // the previous box's TMA store must have read the staging tile before it is rewritten
                         if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                         __syncwarp();
                     }
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
+                    for (int c = 0; c < 2; ++c) {
                         const int n = ncol0 + 8 * c;
                         const float4 b0 = __ldg(reinterpret_cast<const float4*>(a.bias + n)), b1 = __ldg(reinterpret_cast<const float4*>(a.bias + n + 4));
                         float o[8] = {__uint_as_float(v[8 * c]) + b0.x, __uint_as_float(v[8 * c + 1]) + b0.y, __uint_as_float(v[8 * c + 2]) + b0.z,
@@ -326,24 +430,26 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                             const __half2 h = a.relu ? __floats2half2_rn(fmaxf(o[2 * i], 0.f), fmaxf(o[2 * i + 1], 0.f)) : __floats2half2_rn(o[2 * i], o[2 * i + 1]);
                             w[i] = *reinterpret_cast<const uint32_t*>(&h);
                         }
-                        *reinterpret_cast<uint4*>(stage + lane * 128 + (((piece0 + c) ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                        *reinterpret_cast<uint4*>(stage + lane * 128 + (((pbase + c) ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
                     }
-                    if (piece0) {
+                    if (pbase == 6) {
                         fence_async_smem();
                         __syncwarp();
                         if (lane == 0) {
                             asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                                         ::"l"(&map_out), "r"(smem_u32(stage)), "r"(ncol0 - 32), "r"((int)row0) : "memory");
+                                         ::"l"(&map_out), "r"(smem_u32(stage)), "r"(ncol0 - 48), "r"((int)row0) : "memory");
                             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                         }
                     }
-                } else if (c0 + 32 <= n_cols) {
-                    // the previous slice's TMA store must have read the staging tile before it is rewritten
-                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-                    __syncwarp();
-                    // lane = row of the slice; 16-byte piece c of the row goes to piece c ^ (row % 8) (128-byte swizzle)
+                } else if ((c0 & ~31) + 32 <= n_cols) {
+                    const int pbase = (c0 & 31) >> 2;    // 0 or 4: first 16-byte piece (4 columns) of this step
+                    if (pbase == 0) {
+                        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                        __syncwarp();
+                    }
+                    // lane = row of the box; 16-byte piece c of the row goes to piece c ^ (row % 8) (128-byte swizzle)
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) {
+                    for (int c = 0; c < 4; ++c) {
                         const int n = ncol0 + 4 * c;
                         float4 o = make_float4(__uint_as_float(v[4 * c]), __uint_as_float(v[4 * c + 1]),
                                                __uint_as_float(v[4 * c + 2]), __uint_as_float(v[4 * c + 3]));
@@ -352,23 +458,25 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                             o.x += bb.x; o.y += bb.y; o.z += bb.z; o.w += bb.w;
                         }
                         if (a.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f); }
-                        *reinterpret_cast<float4*>(stage + lane * 128 + ((c ^ (lane & 7)) << 4)) = o;
+                        *reinterpret_cast<float4*>(stage + lane * 128 + (((pbase + c) ^ (lane & 7)) << 4)) = o;
                     }
-                    fence_async_smem();
-                    __syncwarp();
-                    if (lane == 0) {
-                        // rows past the end of the layer and columns past its width are clipped by the tensor map
-                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                                     ::"l"(&map_out), "r"(smem_u32(stage)), "r"(ncol0), "r"((int)row0) : "memory");
-                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    if (pbase == 4) {
+                        fence_async_smem();
+                        __syncwarp();
+                        if (lane == 0) {
+                            // rows past the end of the layer and columns past its width are clipped by the tensor map
+                            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                                         ::"l"(&map_out), "r"(smem_u32(stage)), "r"(ncol0 - 16), "r"((int)row0) : "memory");
+                            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                        }
                     }
                 } else {
-                    // a ragged last slice of the half (BN / 2 is not a multiple of 32): lane = row, plain stores
+                    // the ragged end of the half (BN / 2 is not a multiple of 32): lane = row, plain stores
                     const int64_t row = row0 + lane;
                     if (row < a.M) {
                         float* orow = a.out + row * a.N;
 #pragma unroll
-                        for (int c = 0; c < 8; ++c) {
+                        for (int c = 0; c < 4; ++c) {
                             const int n = ncol0 + 4 * c;
                             if (c0 + 4 * c < n_cols && n < a.N) {
                                 const float4 bb = __ldg(reinterpret_cast<const float4*>(a.bias + n));
@@ -388,7 +496,10 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 else mbar_arrive_cluster(mapa_u32(smem_u32(&acc_empty[buf]), 0));
             }
         }
-    } else if (warp < kFirstPlannerWarp) {
+    }
+    } else {
+    MG_REG_SET(MG_REG_PROD);
+    {
         // ---------------- producers: gather + segment mean -> swizzled A slices ----------------
         // K slices come in groups of eight: (self, mean) pairs for four consecutive 32-column blocks, i.e. 128
         // columns of the input rows.  A tile is built in rounds of 32 rows (a row block, planned ahead by the
@@ -532,76 +643,12 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 }
             }
         }
-    } else {
-        // ---------------- planners: row blocks of 32 rows, prepared ahead of the producers ----------------
-        // A planner warp takes every kPlannerWarps-th row block: lane = row.  It reads the rows' metadata, scans the
-        // entry counts, and translates the block's entries to source rows in shared memory, so that the producers'
-        // gathers depend on nothing but shared memory.
-        const int plw = warp - kFirstPlannerWarp;
-        const int32_t* keys = FIRST ? a.ent_nbrs : a.ent_repr;
-        bool ok = true;
-        for (uint32_t q = plw; ok; q += kPlannerWarps) {
-            if (q / kBlocksPerTile >= my_iters) break;
-            const int64_t t = tile_of(q / kBlocksPerTile);   // past the end for the peer of an odd last tile: all padding
-            const int slot = q % kPlanSlots;
-            if (q >= (uint32_t)kPlanSlots && !mbar_wait(&plan_empty[slot], ((q / kPlanSlots) - 1) & 1)) {
-                if (lane == 0) atomicExch(a.error, 17u);
-                ok = false;
-            }
-            ok = __all_sync(0xFFFFFFFFu, ok);
-            if (!ok) break;
-            const int64_t r = a.row_lo + t * BM + (q % kBlocksPerTile) * kBlockRows + lane;
-            int4 rm = make_int4(a.safe_src, 0, -1, 0);
-            if (r < a.M) rm = __ldg(a.row_meta + r);   // (self source row, first entry, count, first H^{l-1} row of the batch)
-            const int32_t end = (int32_t)warp_incl_scan((uint32_t)max(rm.z, 0));   // end of the row's cached entries
-            const int32_t total = __shfl_sync(0xFFFFFFFFu, end, 31);
-            const bool cached = total <= kKeyCap;
-            const int32_t in_base = rm.w, koff = end - max(rm.z, 0);
-            meta[slot][lane] = make_int4(rm.x, rm.y, rm.z, cached ? koff : in_base);
-            if (cached) {
-                // entry j belongs to the first row whose end exceeds j
-                for (int32_t j0 = 0; j0 < total; j0 += 32 * 4) {
-                    int32_t key[4], base[4];
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int32_t j = j0 + u * 32 + lane;
-                        int lo = 0, hi = 31;
-#pragma unroll
-                        for (int s = 0; s < 5; ++s) {
-                            const int mid = (lo + hi) >> 1;
-                            const int32_t e = __shfl_sync(0xFFFFFFFFu, end, mid);
-                            if (lo < hi) { if (e > j) hi = mid; else lo = mid + 1; }
-                        }
-                        const int32_t e0 = __shfl_sync(0xFFFFFFFFu, rm.y, lo), k0 = __shfl_sync(0xFFFFFFFFu, koff, lo);
-                        base[u] = __shfl_sync(0xFFFFFFFFu, in_base, lo);
-                        key[u] = j < total ? __ldg(keys + e0 + (j - k0)) : 0;
-                    }
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int32_t j = j0 + u * 32 + lane;
-                        if (j < total) src_rows[slot][j] = source_row<FIRST>(a, base[u], key[u]);
-                    }
-                }
-            }
-            if (lane == 0) plan_total[slot] = cached ? total : -1;
-            __syncwarp();
-            if (cached) {
-                // lane = row: its first kUnroll source rows, padded with its own source row
-                int32_t fr[8];
-#pragma unroll
-                for (int j = 0; j < 8; ++j) fr[j] = (j < kUnroll && j < rm.z) ? src_rows[slot][koff + j] : rm.x;
-                fr[5] = __float_as_int(rm.z > 0 ? (a.sum_aggr ? 1.f : 1.f / (float)rm.z) : 0.f);   // the mean's factor (1 for a sum)
-                *reinterpret_cast<int4*>(&first_rows[slot][lane][0]) = make_int4(fr[0], fr[1], fr[2], fr[3]);
-                *reinterpret_cast<int4*>(&first_rows[slot][lane][4]) = make_int4(fr[4], fr[5], fr[6], fr[7]);
-                __syncwarp();
-            }
-            if (lane == 0) mbar_arrive(&plan_full[slot]);
-        }
     }
-    if (warp >= 2 && warp < kFirstProducerWarp && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    }
+    if (warp >= kFirstEpilogueWarp && warp < kTmaWarp && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     tc_fence_before();
     cluster_sync_all();   // neither CTA leaves (or frees tensor memory) while the other may still signal or read it
-    if (warp == 1) {
+    if (warp == kMmaWarp) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)a.tmem_cols) : "memory");
     }
