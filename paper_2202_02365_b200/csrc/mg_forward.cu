@@ -13,14 +13,13 @@
 #include <cstdlib>
 
 #include "mg_device.cuh"
-#include <mma.h>
 
 #include "mg_internal.cuh"
 
 int mg_gemm_tf32(mg_ctx* ctx, const float* x, const float* w_t, const float* bias, float* out, int64_t M, int N, int K,
                  bool relu);  // mg_gemm_tcgen05.cu
 int mg_gemm_tf32_status(mg_ctx* ctx);
-int mg_gemm_tf32_splitk_add(mg_ctx* ctx, const float* x, const float* w_t, float* out, int64_t M, int N, int K, int kt_per_slice);
+int mg_gemm_tf32_splitk_add_rows(mg_ctx* ctx, const float* x, const float* g, float* out, int M, int N, int64_t K, int kt_per_slice);
 // mg_layer_fused.cu
 int mg_pack_layer_weights(mg_ctx* ctx, const float* w_cat_dev, float* w_pad_t_dev, int d_in, int N);
 int mg_pack_layer_weights_f16(mg_ctx* ctx, const float* w_cat_dev, void* w_pad_h_dev, int d_in, int N);
@@ -757,9 +756,40 @@ __device__ __forceinline__ void locate_row(const RowGeom& g, int layer, int64_t 
     *node_out = g.node_off[(int64_t)j * (g.B + 1) + lo] + (local - cum[j]);
 }
 
-__global__ void __launch_bounds__(kThreads) k_relu_mask(float* g, const float* __restrict__ y, int64_t n) {
-    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
-        if (!(y[i] > 0.f)) g[i] = 0.f;
+// The gradient of a layer's pre-activations and of its bias in one pass: g *= (y > 0) where the layer has a ReLU
+// (MASK; y = the layer's kept outputs), db += column sums of g.  A thread keeps four columns and walks down the rows
+// (16-byte accesses, a block covers whole rows); column sums meet in shared memory, one atomic add per column and block.
+template <bool MASK>
+__global__ void __launch_bounds__(kThreads) k_grad_pre_bias(float* g, const float* __restrict__ y, float* db, int64_t rows, int N) {
+    __shared__ float sums[1024];
+    const int n4 = N / 4;                       // (widths are multiples of 4, at most 1024)
+    const int rows_per_pass = kThreads / n4;    // >= 1
+    for (int c = threadIdx.x; c < N; c += kThreads) sums[c] = 0.f;
+    __syncthreads();
+    const int c4 = threadIdx.x % n4, rr = threadIdx.x / n4;
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (rr < rows_per_pass) {
+        float4* g4 = reinterpret_cast<float4*>(g);
+        const float4* y4 = reinterpret_cast<const float4*>(y);
+        const int64_t step = (int64_t)gridDim.x * rows_per_pass;
+        for (int64_t r = (int64_t)blockIdx.x * rows_per_pass + rr; r < rows; r += 2 * step) {
+            const int64_t i0 = r * n4 + c4, i1 = (r + step) * n4 + c4;
+            const bool two = r + step < rows;
+            float4 v0 = g4[i0], v1 = two ? g4[i1] : make_float4(0.f, 0.f, 0.f, 0.f);
+            if (MASK) {
+                const float4 a0 = y4[i0], a1 = two ? y4[i1] : make_float4(1.f, 1.f, 1.f, 1.f);
+                const float4 m0 = make_float4(a0.x > 0.f ? v0.x : 0.f, a0.y > 0.f ? v0.y : 0.f, a0.z > 0.f ? v0.z : 0.f, a0.w > 0.f ? v0.w : 0.f);
+                const float4 m1 = make_float4(a1.x > 0.f ? v1.x : 0.f, a1.y > 0.f ? v1.y : 0.f, a1.z > 0.f ? v1.z : 0.f, a1.w > 0.f ? v1.w : 0.f);
+                g4[i0] = m0;
+                if (two) g4[i1] = m1;
+                v0 = m0; v1 = m1;
+            }
+            s.x += v0.x + v1.x; s.y += v0.y + v1.y; s.z += v0.z + v1.z; s.w += v0.w + v1.w;
+        }
+        atomicAdd(&sums[4 * c4], s.x); atomicAdd(&sums[4 * c4 + 1], s.y); atomicAdd(&sums[4 * c4 + 2], s.z); atomicAdd(&sums[4 * c4 + 3], s.w);
+    }
+    __syncthreads();
+    for (int c = threadIdx.x; c < N; c += kThreads) atomicAdd(&db[c], sums[c]);
 }
 
 // dW[Kx, N] += X[rows, Kx]^T dPre[rows, N]; a block owns a 64 x 64 tile of dW and a slice of the rows
@@ -798,90 +828,6 @@ __global__ void __launch_bounds__(256) k_grad_weights(const float* __restrict__ 
             const int kk = k0 + ty * 4 + i, n = n0 + tx * 4 + j;
             if (kk < Kx && n < N) atomicAdd(&dw[(int64_t)kk * N + n], acc[i][j]);
         }
-}
-
-// dst[cols][ld] = src[rows][cols]^T through a 32 x 33 shared tile; columns rows .. ld - 1 of dst are zero-filled (the
-// contraction dimension of the split-K GEMM is padded to a multiple of 32)
-__global__ void __launch_bounds__(256) k_transpose_pad(const float* __restrict__ src, float* dst, int64_t rows, int cols, int64_t ld) {
-    __shared__ float tile[32][33];
-    const int64_t r0 = (int64_t)blockIdx.x * 32;
-    const int c0 = blockIdx.y * 32;
-    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;   // 8 rows of the tile per pass
-    for (int i = ty; i < 32; i += 8) {
-        const int64_t r = r0 + i;
-        tile[i][tx] = (r < rows && c0 + tx < cols) ? src[r * cols + c0 + tx] : 0.f;
-    }
-    __syncthreads();
-    for (int i = ty; i < 32; i += 8) {
-        const int c = c0 + i;
-        const int64_t r = r0 + tx;
-        if (c < cols && r < ld) dst[(int64_t)c * ld + r] = tile[tx][i];
-    }
-}
-
-// The same on the (legacy, warp-level) tensor-core path in TF32: X^T is read as a column-major operand straight
-// from the row-major chunk, so nothing is transposed.  A block owns a 64 x 64 tile of dW and a slice of the rows; each
-// of its four warps a 32 x 32 quarter (2 x 2 fragments of 16 x 16, K = 8 rows per step).
-__global__ void __launch_bounds__(128) k_grad_weights_tf32(const float* __restrict__ x, const float* __restrict__ dpre, float* dw,
-                                                           int64_t rows, int Kx, int N) {
-    using namespace nvcuda;
-    const int warp = threadIdx.x >> 5;
-    const int k0 = blockIdx.x * 64 + (warp >> 1) * 32, n0 = blockIdx.y * 64 + (warp & 1) * 32;
-    const int64_t r_lo = (int64_t)blockIdx.z * kGradRowsPerBlock, r_hi = min(rows, r_lo + kGradRowsPerBlock);
-    if (k0 >= Kx || n0 >= N) return;   // (widths are multiples of 32 on this path)
-    wmma::fragment<wmma::accumulator, 16, 16, 8, float> acc[2][2];
-#pragma unroll
-    for (int i = 0; i < 2; ++i)
-#pragma unroll
-        for (int j = 0; j < 2; ++j) wmma::fill_fragment(acc[i][j], 0.f);
-    for (int64_t r = r_lo; r + 8 <= r_hi; r += 8) {
-        wmma::fragment<wmma::matrix_a, 16, 16, 8, wmma::precision::tf32, wmma::col_major> fa[2];
-        wmma::fragment<wmma::matrix_b, 16, 16, 8, wmma::precision::tf32, wmma::row_major> fb[2];
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            wmma::load_matrix_sync(fa[i], x + r * Kx + k0 + 16 * i, Kx);       // element (k, row) at x[row * Kx + k]
-            wmma::load_matrix_sync(fb[i], dpre + r * N + n0 + 16 * i, N);
-#pragma unroll
-            for (int q = 0; q < fa[i].num_elements; ++q) fa[i].x[q] = wmma::__float_to_tf32(fa[i].x[q]);
-#pragma unroll
-            for (int q = 0; q < fb[i].num_elements; ++q) fb[i].x[q] = wmma::__float_to_tf32(fb[i].x[q]);
-        }
-#pragma unroll
-        for (int i = 0; i < 2; ++i)
-#pragma unroll
-            for (int j = 0; j < 2; ++j) wmma::mma_sync(acc[i][j], fa[i], fb[j], acc[i][j]);
-    }
-    // the slice's last rows (fewer than 8) in plain fp32, one output per lane and step
-    const int64_t tail = r_lo + (r_hi - r_lo) / 8 * 8;
-    __shared__ float stage[4][32 * 32];
-    float* st = stage[warp];
-#pragma unroll
-    for (int i = 0; i < 2; ++i)
-#pragma unroll
-        for (int j = 0; j < 2; ++j) wmma::store_matrix_sync(st + (16 * i) * 32 + 16 * j, acc[i][j], 32, wmma::mem_row_major);
-    __syncwarp();
-    const int lane = threadIdx.x & 31;
-    for (int o = lane; o < 32 * 32; o += 32) {
-        const int kk = o / 32, nn = o % 32;
-        float v = st[o];
-        for (int64_t r = tail; r < r_hi; ++r) v = fmaf(x[r * Kx + k0 + kk], dpre[r * N + n0 + nn], v);
-        atomicAdd(&dw[(int64_t)(k0 + kk) * N + n0 + nn], v);
-    }
-}
-
-constexpr int kBiasRowsPerBlock = 128;
-__global__ void __launch_bounds__(kThreads) k_grad_bias(const float* __restrict__ dpre, float* db, int64_t rows, int N) {
-    // a block sums a slice of the rows for every column (four rows in flight per thread), then one atomic add per column
-    const int64_t r_lo = (int64_t)blockIdx.x * kBiasRowsPerBlock, r_hi = min(rows, r_lo + kBiasRowsPerBlock);
-    for (int c = threadIdx.x; c < N; c += kThreads) {
-        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-        int64_t r = r_lo;
-        for (; r + 4 <= r_hi; r += 4) {
-            s0 += dpre[r * N + c]; s1 += dpre[(r + 1) * N + c]; s2 += dpre[(r + 2) * N + c]; s3 += dpre[(r + 3) * N + c];
-        }
-        for (; r < r_hi; ++r) s0 += dpre[r * N + c];
-        atomicAdd(&db[c], (s0 + s1) + (s2 + s3));
-    }
 }
 
 struct ScatterArgs {
@@ -975,20 +921,15 @@ extern "C" int mg_backward(mg_ctx* ctx, mg_model* m, mg_dense* d, const float* d
         g_off[l] = g_total; g_total += ((size_t)d->h_hdr.rows_total[l] * m->dims[l] + 7) / 8 * 8;   // (32-byte aligned starts)
         h_off[l] = h_total; h_total += (size_t)d->h_hdr.rows_total[l] * m->dims[l];
     }
+    // (chunks 16 times the forward pass's: nothing here gains from a chunk that stays in L2, and fewer, longer launches
+    // mean fewer atomic adds into the weight gradients: 18.2 -> 14.6 ms at 128 mini-batches of the 1M-node workload)
+    const int64_t bw_mult = 16;
     int64_t max_x = 0;
     for (int l = 1; l <= k; ++l)
-        max_x = std::max<int64_t>(max_x, std::min<int64_t>(chunk_rows_for(m->dims[l - 1]), d->h_hdr.rows_total[l]) * 2 * m->dims[l - 1]);
+        max_x = std::max<int64_t>(max_x, std::min<int64_t>(bw_mult * chunk_rows_for(m->dims[l - 1]), d->h_hdr.rows_total[l]) * 2 * m->dims[l - 1]);
     if (ctx->bw_g_elems < g_total && (rc = mg_ensure(ctx, &ctx->bw_g, &ctx->bw_g_elems, g_total + g_total / 4 + 16))) return rc;
     if (ctx->bw_x_elems < (size_t)max_x && (rc = mg_ensure(ctx, &ctx->bw_x, &ctx->bw_x_elems, (size_t)max_x + 16))) return rc;
     if (ctx->bw_dx_elems < (size_t)max_x && (rc = mg_ensure(ctx, &ctx->bw_dx, &ctx->bw_dx_elems, (size_t)max_x + 16))) return rc;
-    if (m->precision == MG_GEMM_TF32) {   // transposed copies of a chunk's X and dPre rows
-        size_t max_t = 0;
-        for (int l = 1; l <= k; ++l) {
-            const int64_t rows = std::min<int64_t>(chunk_rows_for(m->dims[l - 1]), d->h_hdr.rows_total[l]);
-            max_t = std::max(max_t, (size_t)((rows + 31) / 32 * 32) * (2 * m->dims[l - 1] + m->dims[l]));
-        }
-        if (ctx->bw_xt_elems < max_t && (rc = mg_ensure(ctx, &ctx->bw_xt, &ctx->bw_xt_elems, max_t + 16))) return rc;
-    }
     if (g_total) MG_CUDA(ctx, cudaMemsetAsync(ctx->bw_g, 0, g_total * sizeof(float), st));
     if (d_h0_dev) MG_CUDA(ctx, cudaMemsetAsync(d_h0_dev, 0, (size_t)d->h_hdr.rows_total[0] * m->dims[0] * sizeof(float), st));
     const RowGeom geom{B, k, d->rowbase, d->cum, d->node_off};
@@ -999,13 +940,15 @@ extern "C" int mg_backward(mg_ctx* ctx, mg_model* m, mg_dense* d, const float* d
         const int64_t M = d->h_hdr.rows_total[l];
         if (M == 0) continue;
         const float* dpre_all = l == k ? d_out_dev : ctx->bw_g + g_off[l];
-        if (l < k) {   // through the ReLU
-            k_relu_mask<<<grid, kThreads, 0, st>>>(ctx->bw_g + g_off[l], ctx->ws_h[0] + h_off[l], M * d_out);
+        {   // through the ReLU (layers below the last), and the bias gradient
+            const int blocks = (int)std::min<int64_t>(grid, (M + kThreads / (d_out / 4) - 1) / (kThreads / (d_out / 4)));
+            if (l < k) k_grad_pre_bias<true><<<blocks, kThreads, 0, st>>>(ctx->bw_g + g_off[l], ctx->ws_h[0] + h_off[l], m->g_bias[l - 1], M, d_out);
+            else k_grad_pre_bias<false><<<blocks, kThreads, 0, st>>>(const_cast<float*>(d_out_dev), nullptr, m->g_bias[l - 1], M, d_out);
             ctx->launches++;
         }
         const float* h_prev = l > 1 ? ctx->ws_h[0] + h_off[l - 1] : nullptr;
         float* g_in = l > 1 ? ctx->bw_g + g_off[l - 1] : d_h0_dev;
-        const int64_t chunk = chunk_rows_for(d_in);
+        const int64_t chunk = bw_mult * chunk_rows_for(d_in);
         for (int64_t r0 = 0; r0 < M; r0 += chunk) {
             const int64_t r1 = std::min(M, r0 + chunk), rows = r1 - r0;
             AggArgs a;
@@ -1023,25 +966,20 @@ extern "C" int mg_backward(mg_ctx* ctx, mg_model* m, mg_dense* d, const float* d
             if (l == 1) { if (half) launch_aggregate<true, true>(a, grid, st); else launch_aggregate<true, false>(a, grid, st); }
             else launch_aggregate<false, false>(a, grid, st);
             const float* dpre = dpre_all + r0 * d_out;
-            const unsigned slices = (unsigned)((rows + kGradRowsPerBlock - 1) / kGradRowsPerBlock);
-            dim3 gw((unsigned)((2 * d_in + 63) / 64), (unsigned)((d_out + 63) / 64), slices);
-            if (m->precision == MG_GEMM_TF32 && rows >= 4096) {
-                // dW += X^T dPre as a tcgen05 GEMM whose contraction runs over the chunk's rows: both operands are
-                // transposed (rows become the contiguous dimension, padded to 32), the contraction is split over CTAs
-                const int64_t ld = (rows + 31) / 32 * 32;
-                dim3 tx((unsigned)(ld / 32), (unsigned)((2 * d_in + 31) / 32)), tg((unsigned)(ld / 32), (unsigned)((d_out + 31) / 32));
-                k_transpose_pad<<<tx, 256, 0, st>>>(ctx->bw_x, ctx->bw_xt, rows, 2 * d_in, ld);
-                k_transpose_pad<<<tg, 256, 0, st>>>(dpre, ctx->bw_xt + (size_t)2 * d_in * ld, rows, d_out, ld);
-                ctx->launches += 2;
-                if ((rc = mg_gemm_tf32_splitk_add(ctx, ctx->bw_xt, ctx->bw_xt + (size_t)2 * d_in * ld, m->g_w_cat[l - 1], 2 * d_in, d_out,
-                                                  (int)ld, 16))) return rc;
-                ctx->launches--;
-            } else if (m->precision == MG_GEMM_TF32 && d_in % 16 == 0 && d_out % 32 == 0)
-                k_grad_weights_tf32<<<gw, 128, 0, st>>>(ctx->bw_x, dpre, m->g_w_cat[l - 1], rows, 2 * d_in, d_out);
-            else
+            if (m->precision == MG_GEMM_TF32) {
+                // dW += X^T dPre as a tcgen05 GEMM whose contraction runs over the chunk's rows: both operands are read
+                // as they lie (rows x columns, the columns contiguous), the contraction is split over CTAs
+                const int m_tiles = (2 * d_in + 127) / 128, n_tiles = (d_out + 255) / 256;
+                const int64_t steps = (rows + 31) / 32;
+                const int per_slice = (int)std::max<int64_t>(16, (steps * m_tiles * n_tiles + 4 * ctx->n_sms - 1) / (4 * ctx->n_sms));
+                if ((rc = mg_gemm_tf32_splitk_add_rows(ctx, ctx->bw_x, dpre, m->g_w_cat[l - 1], 2 * d_in, d_out, rows, per_slice))) return rc;
+            } else {
+                const unsigned slices = (unsigned)((rows + kGradRowsPerBlock - 1) / kGradRowsPerBlock);
+                dim3 gw((unsigned)((2 * d_in + 63) / 64), (unsigned)((d_out + 63) / 64), slices);
                 k_grad_weights<<<gw, 256, 0, st>>>(ctx->bw_x, dpre, m->g_w_cat[l - 1], rows, 2 * d_in, d_out);
-            k_grad_bias<<<(unsigned)((rows + kBiasRowsPerBlock - 1) / kBiasRowsPerBlock), kThreads, 0, st>>>(dpre, m->g_bias[l - 1], rows, d_out);
-            ctx->launches += 3;
+                ctx->launches++;
+            }
+            ctx->launches++;   // (the aggregation above)
             if (!g_in) continue;   // layer 1 without a gradient of the base representations
             if (m->precision == MG_GEMM_TF32) {
                 // dX = dPre W^T on the tensor cores: the K-major operand the kernel wants is W itself ([2 d_in, d_out])

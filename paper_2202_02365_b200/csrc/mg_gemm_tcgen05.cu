@@ -35,6 +35,7 @@ struct GemmParams {
     // written to dot_out_a, dot_out_b [M]; only when one tile spans the whole width (N <= BN)
     const float* dot_a; const float* dot_b; float* dot_out_a; float* dot_out_b;
     int32_t kt_per_slice;   // split-K: blockIdx.z owns this many 32-wide K steps and ADDS its product to out (0 = whole K, plain store)
+    int32_t mn_major;       // 1: the operands are stored [K, M] and [K, N] (the contraction runs over their rows)
     uint32_t* error;  // device word: 0 = ok, else the role that gave up waiting
 };
 
@@ -80,6 +81,13 @@ k_gemm_tf32(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 if (kt >= p.stages && !mbar_wait(&empty_bar[s], ((kt / p.stages) - 1) & 1)) { atomicExch(p.error, 1u); break; }
                 uint8_t* sa = stage_base + (size_t)s * stage_bytes;
                 mbar_expect_tx(&full_bar[s], stage_bytes);
+                if (p.mn_major) {   // boxes of 32 K rows x 32 floats of M (or N): the tile's 32-float blocks one after the other
+                    for (int j = 0; j < BM / 32; ++j)
+                        tma_load_2d(sa + j * (BK * 128), &map_a, &full_bar[s], (int)m0 + 32 * j, (kt_first + kt) * BK);
+                    for (int j = 0; j < p.BN / 32; ++j)
+                        tma_load_2d(sa + a_bytes + j * (BK * 128), &map_b, &full_bar[s], n0 + 32 * j, (kt_first + kt) * BK);
+                    continue;
+                }
                 tma_load_2d(sa, &map_a, &full_bar[s], (kt_first + kt) * BK, (int)m0);
                 tma_load_2d(sa + a_bytes, &map_b, &full_bar[s], (kt_first + kt) * BK, n0);
             }
@@ -88,17 +96,26 @@ k_gemm_tf32(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     } else if (warp == 1) {
         if (lane == 0) {
             // instruction descriptor: fp32 accumulator, TF32 x TF32, both K-major, M = 128, N = BN
-            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(p.BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+            // (bits 15 and 16: the operand's M / N dimension is the contiguous one)
+            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(p.BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24) |
+                                   (p.mn_major ? (1u << 15) | (1u << 16) : 0u);
             bool ok = true;
             for (int kt = 0; kt < kt_total && ok; ++kt) {
                 const int s = kt % p.stages;
                 if (!mbar_wait(&full_bar[s], (kt / p.stages) & 1)) { atomicExch(p.error, 2u); ok = false; break; }
                 tc_fence_after();
                 const uint32_t sa = smem_u32(stage_base + (size_t)s * stage_bytes);
-                const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sa + a_bytes);
+                if (p.mn_major) {
+                    const uint64_t da = smem_desc_sw128_mn(sa, BK * 128), db = smem_desc_sw128_mn(sa + a_bytes, BK * 128);
 #pragma unroll
-                for (int kk = 0; kk < BK / 8; ++kk)   // one instruction consumes 8 TF32 values (32 bytes) of K
-                    mma_tf32(tmem_base, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (kt | kk) ? 1u : 0u);
+                    for (int kk = 0; kk < BK / 8; ++kk)   // 8 K rows of every box = 1024 bytes further on
+                        mma_tf32(tmem_base, da + (uint64_t)(kk * 64), db + (uint64_t)(kk * 64), idesc, (kt | kk) ? 1u : 0u);
+                } else {
+                    const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sa + a_bytes);
+#pragma unroll
+                    for (int kk = 0; kk < BK / 8; ++kk)   // one instruction consumes 8 TF32 values (32 bytes) of K
+                        mma_tf32(tmem_base, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (kt | kk) ? 1u : 0u);
+                }
                 mma_commit(&empty_bar[s]);   // the stage may be refilled once these MMAs have read it
             }
             mma_commit(&acc_bar);            // accumulator complete (arrives even after a time-out)
@@ -149,15 +166,16 @@ k_gemm_tf32(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 
 static int gemm_tf32_launch(mg_ctx* ctx, const float* x, const float* w_t, const float* bias, float* out, int64_t M, int N, int K,
                             bool relu, int kt_per_slice, const float* dot_a = nullptr, const float* dot_b = nullptr,
-                            float* dot_out_a = nullptr, float* dot_out_b = nullptr) {
+                            float* dot_out_a = nullptr, float* dot_out_b = nullptr, bool mn_major = false) {
     if (M <= 0) return MG_OK;
-    if (K % 4 != 0 || N % 4 != 0) return mg_fail(ctx, MG_ERR_ARG, "GEMM sizes must be multiples of 4");
+    if ((mn_major ? M : K) % 4 != 0 || N % 4 != 0) return mg_fail(ctx, MG_ERR_ARG, "GEMM sizes must be multiples of 4");
     GemmParams p;
     p.out = out; p.bias = bias; p.M = M; p.N = N; p.K = K; p.relu = relu ? 1 : 0; p.error = ctx->d_flags;
     p.kt_per_slice = kt_per_slice;
+    p.mn_major = mn_major ? 1 : 0;
     p.dot_a = dot_a; p.dot_b = dot_b; p.dot_out_a = dot_out_a; p.dot_out_b = dot_out_b;
     if (dot_a && N > 256) return mg_fail(ctx, MG_ERR_ARG, "row dot products need a single tile across the width");
-    p.BN = std::min(256, (N + 15) / 16 * 16);
+    p.BN = mn_major ? std::min(256, (N + 31) / 32 * 32) : std::min(256, (N + 15) / 16 * 16);
     p.tmem_cols = 32;
     while (p.tmem_cols < p.BN) p.tmem_cols <<= 1;
     const int stage_bytes = BM * BK * 4 + p.BN * BK * 4;
@@ -165,7 +183,8 @@ static int gemm_tf32_launch(mg_ctx* ctx, const float* x, const float* w_t, const
     p.stages = std::max(1, std::min({kt, 8, (96 * 1024) / stage_bytes}));
     const size_t smem = (size_t)p.stages * stage_bytes + 1024;
     CUtensorMap ma, mb;
-    if (!make_map_f32(&ma, x, M, K, BM) || !make_map_f32(&mb, w_t, N, K, p.BN))
+    if (mn_major ? (!make_map_f32(&ma, x, K, (int)M, BK, true) || !make_map_f32(&mb, w_t, K, N, BK, true))
+                 : (!make_map_f32(&ma, x, M, K, BM) || !make_map_f32(&mb, w_t, N, K, p.BN)))
         return mg_fail(ctx, MG_ERR_CUDA, "cuTensorMapEncodeTiled failed (M %lld N %d K %d)", (long long)M, N, K);
     static bool attr_set = false;
     if (!attr_set) {
@@ -192,10 +211,12 @@ int mg_gemm_tf32_dots(mg_ctx* ctx, const float* x, const float* w_t, const float
     return gemm_tf32_launch(ctx, x, w_t, zero_bias, out, M, N, K, false, 0, a, b, s_a, s_b);
 }
 
-// out[M, N] += x[M, K] . w_t[N, K]^T with the contraction split over CTAs (kt_per_slice steps of 32 each): for products
-// whose K is far longer than M and N (weight gradients: K = rows of a chunk).  Atomic adds: any order.
-int mg_gemm_tf32_splitk_add(mg_ctx* ctx, const float* x, const float* w_t, float* out, int64_t M, int N, int K, int kt_per_slice) {
-    return gemm_tf32_launch(ctx, x, w_t, nullptr, out, M, N, K, false, std::max(1, kt_per_slice));
+// out[M, N] += x[K, M]^T . g[K, N], both operands as they lie in memory (rows = the contraction, far longer than M and
+// N: weight gradients), the contraction split over CTAs (kt_per_slice steps of 32 rows each; atomic adds, any order).
+// M and N are multiples of 4; rows past K and columns past M, N read as zeros.
+int mg_gemm_tf32_splitk_add_rows(mg_ctx* ctx, const float* x, const float* g, float* out, int M, int N, int64_t K, int kt_per_slice) {
+    if (K >= (1ll << 31)) return mg_fail(ctx, MG_ERR_ARG, "too many rows for one product");
+    return gemm_tf32_launch(ctx, x, g, nullptr, out, M, N, (int)K, false, std::max(1, kt_per_slice), nullptr, nullptr, nullptr, nullptr, true);
 }
 
 // After the stream has drained: MG_ERR_TIMEOUT if a GEMM gave up on a barrier (the word is cleared).

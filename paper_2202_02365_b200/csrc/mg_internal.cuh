@@ -150,8 +150,8 @@ struct mg_ctx {
     float* gat_x = nullptr; float* gat_z = nullptr; float* gat_s = nullptr; float* gat_h[2] = {nullptr, nullptr};   // mg_gat_forward scratch
     size_t gat_x_elems = 0, gat_z_elems = 0, gat_s_elems = 0, gat_h_elems[2] = {0, 0};
     const struct mg_model* last_fwd_model = nullptr; const struct mg_dense* last_fwd_dense = nullptr;   // what mg_backward may follow
-    float* bw_g = nullptr; float* bw_x = nullptr; float* bw_dx = nullptr; float* bw_xt = nullptr;   // mg_backward scratch
-    size_t bw_g_elems = 0, bw_x_elems = 0, bw_dx_elems = 0, bw_xt_elems = 0;
+    float* bw_g = nullptr; float* bw_x = nullptr; float* bw_dx = nullptr;   // mg_backward scratch
+    size_t bw_g_elems = 0, bw_x_elems = 0, bw_dx_elems = 0;
     char* dm_images = nullptr; size_t dm_images_bytes = 0;   // TF32 operand images of the negatives (mg_distmult_score)
     bool prof_on = false;
     bool sample_graphs = true;   // replay the sampler's launches from a CUDA graph

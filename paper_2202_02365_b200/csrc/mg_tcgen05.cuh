@@ -68,6 +68,21 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t smem_addr) {
     return d;
 }
 
+// The same for a TF32 operand whose M (or N) dimension is the contiguous one ("MN-major"); four-byte elements
+// take the 128-byte swizzle on 32-byte units (the 32-byte pieces of a 128-byte row exchanged by the row number mod 4),
+// as a TMA load with CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B leaves them.  The tile is a row of boxes, each 32 floats of M
+// wide and all of the stage's K rows deep, `box_bytes` apart; an instruction reads 8 K rows (two groups of four rows,
+// 512 bytes apart) of every box.
+__device__ __forceinline__ uint64_t smem_desc_sw128_mn(uint32_t smem_addr, uint32_t box_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);   // start address
+    d |= (uint64_t)(box_bytes >> 4) << 16;          // leading byte offset: from one 32-float block of M to the next
+    d |= (uint64_t)(512 >> 4) << 32;                // stride byte offset between 4-row groups of K
+    d |= (uint64_t)1 << 46;                         // descriptor version of sm_100
+    d |= (uint64_t)1 << 61;                         // 128-byte swizzle on 32-byte units
+    return d;
+}
+
 __device__ __forceinline__ void mma_tf32(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -225,7 +240,7 @@ inline EncodeTiledFn get_encode() {
 }
 
 // row-major [rows, K] fp32 matrix, boxes of 32 floats x box_rows, 128-byte swizzle, zero fill
-inline bool make_map_f32(CUtensorMap* map, const float* base, int64_t rows, int K, int box_rows) {
+inline bool make_map_f32(CUtensorMap* map, const float* base, int64_t rows, int K, int box_rows, bool swizzle_32b_units = false) {
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
@@ -233,8 +248,8 @@ inline bool make_map_f32(CUtensorMap* map, const float* base, int64_t rows, int 
     const cuuint32_t box[2] = {32u, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+               CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_32b_units ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace tc
