@@ -499,18 +499,17 @@ __global__ void __launch_bounds__(kThreads) k_insert(InsertArgs a) {
 // -------------------------------------------------------------------------------------
 // The last hop has most of the entries (12.9M of 16.6M on the bench) and its new nodes are never looked up again, so
 // it does not go through the id tables in global memory.  The ids of a mini-batch are split by hash into nb buckets.
-// k_bucket_entries: block (mini-batch, r) takes the r-th share of the mini-batch's entries and writes them grouped by
-// bucket (a counting sort inside the block) as (id, entry) pairs, with the groups' bounds.
+// k_bucket_entries: block (mini-batch, r) takes the r-th share of the mini-batch's entries and the r-th share of the
+// nodes it already has (hops 0..hop) and writes both grouped by bucket (a counting sort inside the block): (id, entry)
+// pairs and (id, row) pairs, with the groups' bounds.
 // k_dedupe_last: block (mini-batch, bucket) holds the bucket's id table (keys and rows, S slots) in shared memory.  It
-// enters the nodes the mini-batch already has (hops 0..hop, rows = positions; every block of the mini-batch reads all
-// of them and keeps its bucket's, compacted per warp so that the table code runs on full warps), then its bucket's
-// pairs from every share (dense), ranks its new nodes (a scan over the table, no atomics), takes a run of the
-// mini-batch's rows and of the list of new nodes with ONE global atomic each, and gives every entry its node's row.
+// enters its bucket's earlier nodes, then its bucket's entries from every share (dense), ranks its new nodes (a scan over
+// the table, no atomics), takes a run of the mini-batch's rows and of the list of new nodes with ONE global atomic
+// each, and gives every entry its node's row.
+// (measured on the bench's last hop: 512 threads x 13,312 slots x 32 buckets and 512 x 6,656 x 64 take the same time)
 constexpr int kDedupThreads = 1024;
 constexpr int kDedupMaxSlots = 26624;    // 208 KiB of keys + rows per block
-constexpr int kDedupMaxBuckets = 16;      // every block of a mini-batch walks all of its earlier nodes: measured faster than the global tables at 9 buckets, slower at 37
-constexpr int kDedupQueue = 64;          // per warp: up to 31 waiting + 32 new (id, row) pairs
-constexpr size_t kDedupQueueBytes = (size_t)(kDedupThreads / 32) * kDedupQueue * sizeof(uint2);
+constexpr int kDedupMaxBuckets = 16;
 constexpr int kBucketThreads = 512;
 
 struct DedupArgs {
@@ -522,14 +521,16 @@ struct DedupArgs {
     const int32_t* ent_off;
     const int32_t* ent_nbrs;
     int32_t* ent_repr;
-    int2* pairs;                // [entries of the hop] (id, entry), grouped by (mini-batch, share, bucket)
-    int32_t* share_off;         // [B][nb][nb + 1] group bounds (positions in pairs)
+    int2* pairs;                // [entries of the hop] (id, entry), grouped by (mini-batch, share, bucket); from
+                                // node_pairs0 on: (id, row) of the earlier nodes, grouped the same way
+    int32_t* share_off;         // [2][B][nb][nb + 1] group bounds (positions in pairs): entries, then earlier nodes
     const int32_t* cum;         // [B][k + 2]
     uint32_t* batch_cnt;        // [B] new nodes of the hop per mini-batch, zero before the launch
     uint64_t* newlist;
     int64_t cap_new;
     int id_bits;
     int32_t max_nodes_per_batch;
+    int64_t node_pairs0;
 };
 
 // bucket and first slot of an id: one multiplicative hash, the bucket from its top, the slot from what is left
@@ -542,59 +543,84 @@ __global__ void __launch_bounds__(kBucketThreads) k_bucket_entries(DedupArgs a) 
     constexpr int kWarps = kBucketThreads / 32;
     __shared__ uint32_t cnt[kWarps][kDedupMaxBuckets];
     __shared__ uint32_t base[kDedupMaxBuckets + 1];
+    __shared__ int32_t hop_lo[MG_MAX_HOPS + 1], hop_row0[MG_MAX_HOPS + 2];
     if (a.hdr->status) return;
     const uint32_t nb = (uint32_t)a.nb;
     const int32_t b = (int32_t)(blockIdx.x / nb);
     const uint32_t r = blockIdx.x % nb;
     const int warp = threadIdx.x >> 5;
-    const int32_t e_lo = a.ent_off[a.node_off[a.hop * (a.B + 1) + b]];
-    const int32_t e_hi = a.ent_off[a.node_off[a.hop * (a.B + 1) + b + 1]];
-    const int32_t len = (int32_t)(((int64_t)(e_hi - e_lo) + nb - 1) / nb);
-    const int32_t s_lo = (int32_t)min((int64_t)e_hi, (int64_t)e_lo + (int64_t)r * len);
-    const int32_t s_hi = (int32_t)min((int64_t)e_hi, (int64_t)s_lo + len);
-    for (int i = threadIdx.x; i < kWarps * kDedupMaxBuckets; i += kBucketThreads) (&cnt[0][0])[i] = 0;
+    if (threadIdx.x <= (unsigned)a.hop) hop_lo[threadIdx.x] = a.node_off[threadIdx.x * (a.B + 1) + b];
+    if (threadIdx.x <= (unsigned)a.hop + 1) hop_row0[threadIdx.x] = a.cum[b * (a.k + 2) + threadIdx.x];
     __syncthreads();
-    // (four loads in flight per thread: the walk is latency-bound otherwise)
-    for (int32_t e0 = s_lo + (int32_t)threadIdx.x; e0 < s_hi; e0 += 4 * kBucketThreads) {
-        int32_t id[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) id[u] = e0 + u * kBucketThreads < s_hi ? a.ent_nbrs[e0 + u * kBucketThreads] : -1;
-#pragma unroll
-        for (int u = 0; u < 4; ++u)
-            if (e0 + u * kBucketThreads < s_hi) atomicAdd(&cnt[warp][dedup_bucket(id[u], nb)], 1u);
-    }
-    __syncthreads();
-    if (threadIdx.x < nb) {   // this bucket's pairs of the share: warp after warp
-        uint32_t run = 0;
-        for (int w = 0; w < kWarps; ++w) { const uint32_t c = cnt[w][threadIdx.x]; cnt[w][threadIdx.x] = run; run += c; }
-        base[threadIdx.x] = run;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        uint32_t run = 0;
-        for (uint32_t q = 0; q < nb; ++q) { const uint32_t c = base[q]; base[q] = run; run += c; }
-        base[nb] = run;
-    }
-    __syncthreads();
-    if (threadIdx.x <= nb) a.share_off[((int64_t)b * nb + r) * (nb + 1) + threadIdx.x] = s_lo + (int32_t)base[threadIdx.x];
-    for (int32_t e0 = s_lo + (int32_t)threadIdx.x; e0 < s_hi; e0 += 4 * kBucketThreads) {
-        int32_t id[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) id[u] = e0 + u * kBucketThreads < s_hi ? a.ent_nbrs[e0 + u * kBucketThreads] : -1;
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int32_t e = e0 + u * kBucketThreads;
-            if (e >= s_hi) continue;
-            const uint32_t q = dedup_bucket(id[u], nb);
-            a.pairs[s_lo + base[q] + atomicAdd(&cnt[warp][q], 1u)] = make_int2(id[u], e);
+    // pass 0: the entries of the hop; pass 1: the nodes the mini-batch already has, item t = the node of row t
+    for (int pass = 0; pass < 2; ++pass) {
+        int64_t first, last, out0;
+        if (pass == 0) {
+            first = a.ent_off[a.node_off[a.hop * (a.B + 1) + b]];
+            last = a.ent_off[a.node_off[a.hop * (a.B + 1) + b + 1]];
+            out0 = first;
+        } else {
+            first = 0;
+            last = hop_row0[a.hop + 1];
+            out0 = a.node_pairs0;   // this mini-batch's node pairs follow those of the mini-batches before it
+            for (int j = 0; j <= a.hop; ++j) out0 += hop_lo[j] - a.node_off[j * (a.B + 1)];
         }
+        const int32_t len = (int32_t)((last - first + nb - 1) / nb);
+        const int32_t s_lo = (int32_t)min(last, first + (int64_t)r * len);
+        const int32_t s_hi = (int32_t)min(last, (int64_t)s_lo + len);
+        auto id_at = [&](int32_t i) -> int32_t {
+            if (pass == 0) return a.ent_nbrs[i];
+            int j = 0;
+            while (j < a.hop && hop_row0[j + 1] <= i) ++j;
+            return a.nodes[hop_lo[j] + (i - hop_row0[j])];
+        };
+        for (int i = threadIdx.x; i < kWarps * kDedupMaxBuckets; i += kBucketThreads) (&cnt[0][0])[i] = 0;
+        __syncthreads();
+        // (four loads in flight per thread: the walk is latency-bound otherwise)
+        for (int32_t e0 = s_lo + (int32_t)threadIdx.x; e0 < s_hi; e0 += 4 * kBucketThreads) {
+            int32_t id[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) id[u] = e0 + u * kBucketThreads < s_hi ? id_at(e0 + u * kBucketThreads) : -1;
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (e0 + u * kBucketThreads < s_hi) atomicAdd(&cnt[warp][dedup_bucket(id[u], nb)], 1u);
+        }
+        __syncthreads();
+        if (threadIdx.x < nb) {   // this bucket's pairs of the share: warp after warp
+            uint32_t run = 0;
+            for (int w = 0; w < kWarps; ++w) { const uint32_t c = cnt[w][threadIdx.x]; cnt[w][threadIdx.x] = run; run += c; }
+            base[threadIdx.x] = run;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint32_t run = 0;
+            for (uint32_t q = 0; q < nb; ++q) { const uint32_t c = base[q]; base[q] = run; run += c; }
+            base[nb] = run;
+        }
+        __syncthreads();
+        const int64_t dst0 = out0 + (s_lo - first);
+        if (threadIdx.x <= nb)
+            a.share_off[(((int64_t)pass * a.B + b) * nb + r) * (nb + 1) + threadIdx.x] = (int32_t)(dst0 + base[threadIdx.x]);
+        for (int32_t e0 = s_lo + (int32_t)threadIdx.x; e0 < s_hi; e0 += 4 * kBucketThreads) {
+            int32_t id[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) id[u] = e0 + u * kBucketThreads < s_hi ? id_at(e0 + u * kBucketThreads) : -1;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int32_t e = e0 + u * kBucketThreads;
+                if (e >= s_hi) continue;
+                const uint32_t q = dedup_bucket(id[u], nb);
+                a.pairs[dst0 + base[q] + atomicAdd(&cnt[warp][q], 1u)] = make_int2(id[u], e);
+            }
+        }
+        __syncthreads();
     }
 }
 
 __global__ void __launch_bounds__(kDedupThreads) k_dedupe_last(DedupArgs a) {
     extern __shared__ int32_t dedup_sm[];
     __shared__ uint32_t row_base, list_base, warp_tot[kDedupThreads / 32];
-    __shared__ int32_t run_lo[kDedupMaxBuckets], run_start[kDedupMaxBuckets + 1];
+    __shared__ int32_t run_lo[2][kDedupMaxBuckets], run_start[2][kDedupMaxBuckets + 1];
     if (a.hdr->status) return;
     const uint32_t S = (uint32_t)a.S, nb = (uint32_t)a.nb;
     int32_t* keys = dedup_sm;
@@ -603,73 +629,52 @@ __global__ void __launch_bounds__(kDedupThreads) k_dedupe_last(DedupArgs a) {
     const uint32_t bucket = blockIdx.x % nb;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (uint32_t i = threadIdx.x; i < S; i += kDedupThreads) keys[i] = -1;
-    if (threadIdx.x < nb) {   // this bucket's runs of pairs, one per share ...
-        const int32_t* so = a.share_off + ((int64_t)b * nb + threadIdx.x) * (nb + 1) + bucket;
-        run_lo[threadIdx.x] = so[0];
-        run_start[threadIdx.x + 1] = so[1] - so[0];
+    if (threadIdx.x < 2 * nb) {   // this bucket's runs of pairs, one per share: entries [0], earlier nodes [1] ...
+        const uint32_t which = threadIdx.x / nb, r = threadIdx.x % nb;
+        const int32_t* so = a.share_off + (((int64_t)which * a.B + b) * nb + r) * (nb + 1) + bucket;
+        run_lo[which][r] = so[0];
+        run_start[which][r + 1] = so[1] - so[0];
     }
     __syncthreads();
-    if (threadIdx.x == 0) {   // ... and their lengths' prefix
+    if (threadIdx.x < 2) {   // ... and their lengths' prefix
         int32_t run = 0;
-        for (uint32_t r = 0; r < nb; ++r) { const int32_t c = run_start[r + 1]; run_start[r] = run; run += c; }
-        run_start[nb] = run;
+        for (uint32_t r = 0; r < nb; ++r) { const int32_t c = run_start[threadIdx.x][r + 1]; run_start[threadIdx.x][r] = run; run += c; }
+        run_start[threadIdx.x][nb] = run;
     }
     __syncthreads();
-    // the nodes the mini-batch already has: a warp compacts the ids of this bucket and enters 32 at a time
-    {
-        uint2* q = reinterpret_cast<uint2*>(dedup_sm + 2 * S) + warp * kDedupQueue;
-        const uint32_t lt = (1u << lane) - 1u;
-        uint32_t waiting = 0;
-        auto enter = [&](uint2 it) {
-            const int32_t u = (int32_t)it.x;
-            uint32_t s = dedup_slot(u, nb, S), probe = 0;
-            for (; probe < S; ++probe) {
-                const int32_t old = atomicCAS(&keys[s], -1, u);
-                if (old == -1) { vals[s] = (int32_t)it.y; break; }
-                if (old == u) { atomicOr(&a.hdr->status, ST_DUPLICATE); break; }   // only targets can repeat
-                s = s + 1u == S ? 0u : s + 1u;
-            }
-            if (probe >= S) atomicOr(&a.hdr->status, ST_CAP_TABLE);
-        };
-        for (int j = 0; j <= a.hop; ++j) {
-            const int32_t lo = a.node_off[j * (a.B + 1) + b], hi = a.node_off[j * (a.B + 1) + b + 1];
-            const int32_t row0 = a.cum[b * (a.k + 2) + j];
-            for (int32_t p0 = lo + warp * 32; p0 < hi; p0 += 4 * kDedupThreads) {
-                int32_t us[4];   // four loads in flight per lane
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const int32_t p = p0 + c * kDedupThreads + lane;
-                    us[c] = p < hi ? a.nodes[p] : 0;
-                }
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const int32_t p = p0 + c * kDedupThreads + lane;
-                    const bool m = p < hi && dedup_bucket(us[c], nb) == bucket;
-                    const uint32_t mask = __ballot_sync(0xFFFFFFFFu, m);
-                    if (m) q[waiting + __popc(mask & lt)] = make_uint2((uint32_t)us[c], (uint32_t)(row0 + (p - lo)));
-                    waiting += __popc(mask);
-                    __syncwarp();
-                    if (waiting >= 32) {
-                        enter(q[waiting - 32 + lane]);
-                        waiting -= 32;
-                    }
-                    __syncwarp();
-                }
-            }
-        }
-        if ((uint32_t)lane < waiting) enter(q[lane]);
-    }
-    __syncthreads();
-    // this bucket's pairs: enter the id, leave its slot in place of the id
-    const int32_t n_pairs = run_start[nb];
-    auto pair_at = [&](int32_t i) -> int2* {   // i-th pair of the bucket: which share's run it falls in (run_start ascends)
-        uint32_t lo = 0, hi = nb;                // run_start[lo] <= i < run_start[hi]
+    auto pair_at = [&](int which, int32_t i) -> int2* {   // i-th pair of the bucket: which share's run it falls in (run_start ascends)
+        uint32_t lo = 0, hi = nb;                           // run_start[lo] <= i < run_start[hi]
         while (hi - lo > 1) {
             const uint32_t mid = (lo + hi) >> 1;
-            if (run_start[mid] <= i) lo = mid; else hi = mid;
+            if (run_start[which][mid] <= i) lo = mid; else hi = mid;
         }
-        return a.pairs + run_lo[lo] + (i - run_start[lo]);
+        return a.pairs + run_lo[which][lo] + (i - run_start[which][lo]);
     };
+    // the nodes the mini-batch already has (this bucket's): rows = positions
+    {
+        const int32_t n_old = run_start[1][nb];
+        for (int32_t i0 = threadIdx.x; i0 < n_old; i0 += 4 * kDedupThreads) {
+            int2 it[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) it[u] = *pair_at(1, min(i0 + u * kDedupThreads, n_old - 1));
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (i0 + u * kDedupThreads >= n_old) continue;
+                const int32_t id = it[u].x;
+                uint32_t s = dedup_slot(id, nb, S), probe = 0;
+                for (; probe < S; ++probe) {
+                    const int32_t old = atomicCAS(&keys[s], -1, id);
+                    if (old == -1) { vals[s] = it[u].y; break; }
+                    if (old == id) { atomicOr(&a.hdr->status, ST_DUPLICATE); break; }   // only targets can repeat
+                    s = s + 1u == S ? 0u : s + 1u;
+                }
+                if (probe >= S) atomicOr(&a.hdr->status, ST_CAP_TABLE);
+            }
+        }
+    }
+    __syncthreads();
+    // this bucket's entries: enter the id, leave its slot in place of the id
+    const int32_t n_pairs = run_start[0][nb];
     for (int32_t i0 = threadIdx.x; i0 < n_pairs; i0 += 4 * kDedupThreads) {
         int2* pp[4];
         int32_t id[4], old[4];
@@ -677,7 +682,7 @@ __global__ void __launch_bounds__(kDedupThreads) k_dedupe_last(DedupArgs a) {
 #pragma unroll
         for (int u = 0; u < 4; ++u) {   // four loads, then four first-probe compare-and-swaps, in flight per thread
             const int32_t i = i0 + u * kDedupThreads;
-            pp[u] = pair_at(min(i, n_pairs - 1));
+            pp[u] = pair_at(0, min(i, n_pairs - 1));
             id[u] = i < n_pairs ? pp[u]->x : -1;
         }
 #pragma unroll
@@ -711,9 +716,9 @@ __global__ void __launch_bounds__(kDedupThreads) k_dedupe_last(DedupArgs a) {
     if (lane == 31) warp_tot[warp] = inc;
     __syncthreads();
     if (warp == 0) {
-        const uint32_t w = warp_tot[lane];
+        const uint32_t w = lane < kDedupThreads / 32 ? warp_tot[lane] : 0u;
         const uint32_t wi = warp_incl_scan(w);
-        warp_tot[lane] = wi - w;
+        if (lane < kDedupThreads / 32) warp_tot[lane] = wi - w;
         if (lane == 31) {
             row_base = wi ? atomicAdd(&a.batch_cnt[b], wi) : 0u;
             list_base = wi ? atomicAdd(&a.hdr->n_new, wi) : 0u;
@@ -740,7 +745,7 @@ __global__ void __launch_bounds__(kDedupThreads) k_dedupe_last(DedupArgs a) {
     for (int32_t i0 = threadIdx.x; i0 < n_pairs; i0 += 4 * kDedupThreads) {
         int2 p[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) p[u] = *pair_at(min(i0 + u * kDedupThreads, n_pairs - 1));
+        for (int u = 0; u < 4; ++u) p[u] = *pair_at(0, min(i0 + u * kDedupThreads, n_pairs - 1));
 #pragma unroll
         for (int u = 0; u < 4; ++u)
             if (i0 + u * kDedupThreads < n_pairs) a.ent_repr[p[u].y] = vals[p[u].x];
@@ -1282,12 +1287,12 @@ static int dense_alloc(mg_ctx* ctx, mg_dense* d, int32_t B, int32_t k, int64_t c
         d->cap_pairs = 0;
     }
     if (smem_nb > 0) {
-        if (d->cap_pairs < d->cap_entries) {
+        if (d->cap_pairs < d->cap_entries + d->cap_nodes) {   // (id, entry) of the last hop's entries, then (id, row) of the earlier nodes
             d->cap_pairs = 0;
-            if ((rc = dev_realloc(ctx, &d->pairs, (size_t)d->cap_entries))) return rc;
-            d->cap_pairs = d->cap_entries;
+            if ((rc = dev_realloc(ctx, &d->pairs, (size_t)(d->cap_entries + d->cap_nodes)))) return rc;
+            d->cap_pairs = d->cap_entries + d->cap_nodes;
         }
-        const int64_t need_share = (int64_t)B * smem_nb * (smem_nb + 1);
+        const int64_t need_share = 2 * (int64_t)B * smem_nb * (smem_nb + 1);
         if (d->cap_share < need_share) {
             d->cap_share = 0;
             if ((rc = dev_realloc(ctx, &d->share_off, (size_t)need_share))) return rc;
@@ -1395,7 +1400,7 @@ static void sample_kernel_attributes() {
     static bool done = false;
     if (done) return;
     cudaFuncSetAttribute(k_radix_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScatterSmem);
-    cudaFuncSetAttribute(k_dedupe_last, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kDedupMaxSlots * 2 * sizeof(int32_t) + kDedupQueueBytes));
+    cudaFuncSetAttribute(k_dedupe_last, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kDedupMaxSlots * 2 * sizeof(int32_t)));
     cudaFuncSetAttribute(k_pick_wide, cudaFuncAttributeMaxDynamicSharedMemorySize,
                          (int)((size_t)(kThreads / 32) * 2 * MG_MAX_FANOUT * sizeof(uint32_t)));
     done = true;
@@ -1463,7 +1468,8 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
     // buckets of a hash differ by a per cent or so at these sizes), nb blocks per mini-batch.
     const int32_t dedup_slots = (int32_t)std::min<int64_t>(kDedupMaxSlots, (cap_batch + cap_batch / 4 + 64 + 1023) / 1024 * 1024);
     const int64_t dedup_nb = (cap_batch + (cap_batch * 7 + 79) / 80 + dedup_slots - 1) / dedup_slots;
-    const bool smem_last = dedup_nb <= kDedupMaxBuckets && dedup_nb * n_batches < (1ll << 24) && !getenv("MG_GLOBAL_TABLES");
+    const bool smem_last = dedup_nb <= kDedupMaxBuckets && dedup_nb * n_batches < (1ll << 24) && cap_entries + cap_nodes < (1ll << 31) &&
+                           !getenv("MG_GLOBAL_TABLES");
     // With the last hop deduplicated in shared memory the global tables only ever hold the nodes that are sampled from
     // (targets and the inner deltas): a caller who bounds those gets tables several times smaller.
     int64_t table_nodes = cap_batch;
@@ -1611,9 +1617,9 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
             if (smem_last && h == k - 1) {
                 DedupArgs da{d->hdr, h, B, k, (int32_t)dedup_nb, dedup_slots, d->nodes, d->node_off, d->ent_off, d->ent_nbrs,
                              d->ent_repr, d->pairs, d->share_off, d->cum, batch_cnt + (size_t)h * B, d->newlist[0], d->cap_nodes,
-                             id_bits, (int32_t)cap_batch};
+                             id_bits, (int32_t)cap_batch, d->cap_entries};
                 k_bucket_entries<<<(unsigned)(B * dedup_nb), kBucketThreads, 0, st>>>(da);
-                k_dedupe_last<<<(unsigned)(B * dedup_nb), kDedupThreads, (size_t)dedup_slots * 2 * sizeof(int32_t) + kDedupQueueBytes, st>>>(da);
+                k_dedupe_last<<<(unsigned)(B * dedup_nb), kDedupThreads, (size_t)dedup_slots * 2 * sizeof(int32_t), st>>>(da);
                 ctx->launches += 2;
             } else {
                 InsertArgs ia{d->hdr, h, d->ent_nbrs, d->ent_repr, d->hkeys, tg, d->newlist[0], d->cap_nodes, id_bits,
