@@ -830,43 +830,196 @@ __global__ void __launch_bounds__(256) k_grad_weights(const float* __restrict__ 
         }
 }
 
-struct ScatterArgs {
+// ---- dX of a layer -> the gradient of the layer's input rows ----
+// A source row receives the self part of its own output row and a share of the neighbour part of every output row that
+// aggregates it.  Instead of adding row by row with atomics (a read-modify-write of the target for every sampled
+// entry), the entries are first turned round -- for every source row the list of (output row, weight) that name it: a
+// count per source row, an exclusive scan, a fill -- and a warp then sums a source row's contributions in registers and
+// stores the row once, through the ReLU of the layer below and into that layer's bias gradient on the way.
+struct RevArgs {
     RowGeom g;
-    int32_t layer;             // the layer whose inputs receive the gradient (1 .. k)
-    int64_t row_lo, row_hi;    // packed output rows of this chunk
+    int32_t layer;             // the layer whose entries are turned round (1 .. k)
+    int64_t rows_out;          // its packed output rows
     const int32_t* ent_off;
     const int32_t* ent_repr;
-    const float* dx;           // [row_hi - row_lo, 2 d_in]
-    int32_t d_in, sum_aggr;
-    float* g_in;               // [rows of layer - 1, d_in]
+    uint32_t* cnt;             // [rows of layer - 1]: counts (FILL = false) / fill cursors (FILL = true)
+    const uint32_t* off;       // [rows of layer - 1 + 1] exclusive prefix of the counts
+    int2* rev;                 // (output row, weight as float bits)
+    int32_t sum_aggr;
 };
 
-// one warp per output row: its self row and the source rows of its entries receive their share of dX
-__global__ void __launch_bounds__(kThreads) k_scatter_grad(ScatterArgs a) {
-    const int lane = threadIdx.x & 31;
-    const int64_t warps = (int64_t)gridDim.x * (kThreads / 32);
+template <bool FILL>
+__global__ void __launch_bounds__(kThreads) k_rev_entries(RevArgs a) {
     const int32_t* rb_in = a.g.rowbase + (int64_t)(a.layer - 1) * (a.g.B + 1);
-    for (int64_t row = a.row_lo + blockIdx.x * (int64_t)(kThreads / 32) + (threadIdx.x >> 5); row < a.row_hi; row += warps) {
+    for (int64_t row = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; row < a.rows_out; row += (int64_t)gridDim.x * blockDim.x) {
         int32_t b, local, node;
         locate_row(a.g, a.layer, row, &b, &local, &node);
-        const int64_t in0 = rb_in[b];
-        const float* dxr = a.dx + (row - a.row_lo) * 2 * a.d_in;
-        // (16-byte vector atomics: widths are multiples of 4 and every row starts 16-byte aligned)
-        float4* self = reinterpret_cast<float4*>(a.g_in + (in0 + local) * a.d_in);
-        const float4* dx4 = reinterpret_cast<const float4*>(dxr);
-        const int n4 = a.d_in / 4;
-        for (int c = lane; c < n4; c += 32) atomicAdd(&self[c], dx4[c]);
         const int32_t e0 = a.ent_off[node], e1 = a.ent_off[node + 1];
         if (e1 <= e0) continue;
-        const float scale = a.sum_aggr ? 1.f : 1.f / (float)(e1 - e0);
+        const int64_t in0 = rb_in[b];
+        const float w = a.sum_aggr ? 1.f : 1.f / (float)(e1 - e0);
         for (int32_t e = e0; e < e1; ++e) {
-            float4* src = reinterpret_cast<float4*>(a.g_in + (in0 + a.ent_repr[e]) * a.d_in);
-            for (int c = lane; c < n4; c += 32) {
-                const float4 v = dx4[n4 + c];
-                atomicAdd(&src[c], make_float4(v.x * scale, v.y * scale, v.z * scale, v.w * scale));
-            }
+            const int64_t src = in0 + a.ent_repr[e];
+            const uint32_t pos = atomicAdd(&a.cnt[src], 1u);
+            if (FILL) a.rev[a.off[src] + pos] = make_int2((int32_t)row, __float_as_int(w));
         }
     }
+}
+
+// exclusive scan of data[0 .. n) in place, the total to data[n]: tile sums, their scan by one block, the tiles again
+constexpr int kRevTile = kThreads * 16;
+__global__ void __launch_bounds__(kThreads) k_rev_tile_sums(const uint32_t* __restrict__ data, int64_t n, uint32_t* sums) {
+    __shared__ uint32_t part[kThreads / 32];
+    const int64_t t0 = (int64_t)blockIdx.x * kRevTile;
+    uint32_t s = 0;
+    for (int i = threadIdx.x; i < kRevTile; i += kThreads) s += t0 + i < n ? data[t0 + i] : 0u;
+    for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t t = 0;
+        for (int w = 0; w < kThreads / 32; ++w) t += part[w];
+        sums[blockIdx.x] = t;
+    }
+}
+__global__ void __launch_bounds__(1024) k_rev_scan_sums(uint32_t* sums, int n_tiles) {
+    __shared__ uint32_t part[32];
+    __shared__ uint32_t carry;
+    if (threadIdx.x == 0) carry = 0;
+    __syncthreads();
+    for (int i0 = 0; i0 < n_tiles; i0 += 1024) {
+        const int i = i0 + threadIdx.x;
+        const uint32_t v = i < n_tiles ? sums[i] : 0u;
+        const uint32_t inc = warp_incl_scan(v);
+        if ((threadIdx.x & 31) == 31) part[threadIdx.x >> 5] = inc;
+        __syncthreads();
+        if (threadIdx.x < 32) { const uint32_t w = part[threadIdx.x]; part[threadIdx.x] = warp_incl_scan(w) - w; }
+        __syncthreads();
+        const uint32_t excl = carry + part[threadIdx.x >> 5] + inc - v;
+        if (i < n_tiles) sums[i] = excl;
+        __syncthreads();
+        if (threadIdx.x == 1023) carry = excl + v;
+        __syncthreads();
+    }
+}
+__global__ void __launch_bounds__(kThreads) k_rev_scan_tiles(uint32_t* data, int64_t n, const uint32_t* __restrict__ sums) {
+    __shared__ uint32_t part[kThreads / 32];
+    const int64_t t0 = (int64_t)blockIdx.x * kRevTile + (int64_t)threadIdx.x * 16;   // 16 consecutive elements per thread
+    uint32_t v[16], s = 0;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) { v[i] = t0 + i < n ? data[t0 + i] : 0u; s += v[i]; }
+    const uint32_t inc = warp_incl_scan(s);
+    if ((threadIdx.x & 31) == 31) part[threadIdx.x >> 5] = inc;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        const uint32_t w = threadIdx.x < kThreads / 32 ? part[threadIdx.x] : 0u;
+        const uint32_t wi = warp_incl_scan(w);
+        if (threadIdx.x < kThreads / 32) part[threadIdx.x] = wi - w;
+    }
+    __syncthreads();
+    uint32_t run = sums[blockIdx.x] + part[threadIdx.x >> 5] + inc - s;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        if (t0 + i < n) data[t0 + i] = run;
+        run += v[i];
+        if (t0 + i == n - 1) data[n] = run;
+    }
+}
+
+struct GatherArgs {
+    RowGeom g;
+    int32_t layer;             // the layer whose dX is handed down (1 .. k); its inputs are the rows of layer - 1
+    int64_t rows_in;
+    const uint32_t* off;       // [rows_in + 1]
+    const int2* rev;
+    const float* dx;           // [rows of layer, 2 d_in]
+    int32_t d_in;
+    const float* y;            // [rows_in, d_in] kept outputs of layer - 1 (MASK), else null
+    float* g_in;               // [rows_in, d_in]
+    float* db;                 // [d_in] bias gradient of layer - 1 (MASK)
+};
+
+// one warp per source row; a lane keeps NCH groups of four columns (d_in <= 128 NCH)
+template <bool MASK, int NCH>
+__global__ void __launch_bounds__(kThreads) k_grad_gather(GatherArgs a) {
+    __shared__ float sums[MASK ? 128 * NCH : 1];
+    const int lane = threadIdx.x & 31;
+    const int n4 = a.d_in / 4;
+    const int32_t* rb_out = a.g.rowbase + (int64_t)a.layer * (a.g.B + 1);
+    if (MASK) {
+        for (int c = threadIdx.x; c < 128 * NCH; c += kThreads) sums[c] = 0.f;
+        __syncthreads();
+    }
+    float4 bias[NCH];
+#pragma unroll
+    for (int q = 0; q < NCH; ++q) bias[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int64_t warps = (int64_t)gridDim.x * (kThreads / 32);
+    for (int64_t s = blockIdx.x * (int64_t)(kThreads / 32) + (threadIdx.x >> 5); s < a.rows_in; s += warps) {
+        int32_t b, local, node;
+        locate_row(a.g, a.layer - 1, s, &b, &local, &node);
+        const int32_t n_out = rb_out[b + 1] - rb_out[b];
+        const uint32_t i0 = a.off[s], i1 = a.off[s + 1];
+        float4 acc[NCH];
+#pragma unroll
+        for (int q = 0; q < NCH; ++q) {
+            const int c = lane + 32 * q;
+            acc[q] = (local < n_out && c < n4)
+                         ? reinterpret_cast<const float4*>(a.dx + ((int64_t)rb_out[b] + local) * 2 * a.d_in)[c]
+                         : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        for (uint32_t i = i0; i < i1; i += 2) {   // two contributions in flight
+            const int2 r0 = a.rev[i];
+            const bool two = i + 1 < i1;
+            const int2 r1 = two ? a.rev[i + 1] : r0;
+            const float w0 = __int_as_float(r0.y), w1 = two ? __int_as_float(r1.y) : 0.f;
+            const float4* p0 = reinterpret_cast<const float4*>(a.dx + (int64_t)r0.x * 2 * a.d_in + a.d_in);
+            const float4* p1 = reinterpret_cast<const float4*>(a.dx + (int64_t)r1.x * 2 * a.d_in + a.d_in);
+            float4 v0[NCH], v1[NCH];
+#pragma unroll
+            for (int q = 0; q < NCH; ++q) {
+                const int c = lane + 32 * q;
+                v0[q] = c < n4 ? p0[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+                v1[q] = c < n4 ? p1[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int q = 0; q < NCH; ++q) {
+                acc[q].x += w0 * v0[q].x + w1 * v1[q].x; acc[q].y += w0 * v0[q].y + w1 * v1[q].y;
+                acc[q].z += w0 * v0[q].z + w1 * v1[q].z; acc[q].w += w0 * v0[q].w + w1 * v1[q].w;
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < NCH; ++q) {
+            const int c = lane + 32 * q;
+            if (c >= n4) continue;
+            float4 v = acc[q];
+            if (MASK) {
+                const float4 yy = reinterpret_cast<const float4*>(a.y + s * a.d_in)[c];
+                v = make_float4(yy.x > 0.f ? v.x : 0.f, yy.y > 0.f ? v.y : 0.f, yy.z > 0.f ? v.z : 0.f, yy.w > 0.f ? v.w : 0.f);
+                bias[q].x += v.x; bias[q].y += v.y; bias[q].z += v.z; bias[q].w += v.w;
+            }
+            reinterpret_cast<float4*>(a.g_in + s * a.d_in)[c] = v;
+        }
+    }
+    if (MASK) {
+#pragma unroll
+        for (int q = 0; q < NCH; ++q) {
+            const int c = lane + 32 * q;
+            if (c >= n4) continue;
+            atomicAdd(&sums[4 * c], bias[q].x); atomicAdd(&sums[4 * c + 1], bias[q].y);
+            atomicAdd(&sums[4 * c + 2], bias[q].z); atomicAdd(&sums[4 * c + 3], bias[q].w);
+        }
+        __syncthreads();
+        for (int c = threadIdx.x; c < a.d_in; c += kThreads) atomicAdd(&a.db[c], sums[c]);
+    }
+}
+
+template <bool MASK>
+static void launch_grad_gather(const GatherArgs& a, int grid, cudaStream_t st) {
+    const int nch = (a.d_in + 127) / 128;
+    if (nch <= 1) k_grad_gather<MASK, 1><<<grid, kThreads, 0, st>>>(a);
+    else if (nch <= 2) k_grad_gather<MASK, 2><<<grid, kThreads, 0, st>>>(a);
+    else if (nch <= 4) k_grad_gather<MASK, 4><<<grid, kThreads, 0, st>>>(a);
+    else k_grad_gather<MASK, 8><<<grid, kThreads, 0, st>>>(a);
 }
 
 __global__ void __launch_bounds__(kThreads) k_sgd(float* w, const float* __restrict__ g, float lr, int64_t n) {
@@ -924,26 +1077,34 @@ extern "C" int mg_backward(mg_ctx* ctx, mg_model* m, mg_dense* d, const float* d
     // (chunks 16 times the forward pass's: nothing here gains from a chunk that stays in L2, and fewer, longer launches
     // mean fewer atomic adds into the weight gradients: 18.2 -> 14.6 ms at 128 mini-batches of the 1M-node workload)
     const int64_t bw_mult = 16;
-    int64_t max_x = 0;
-    for (int l = 1; l <= k; ++l)
+    int64_t max_x = 0, max_dx = 0, max_in = 0, max_ent = 0;
+    for (int l = 1; l <= k; ++l) {
         max_x = std::max<int64_t>(max_x, std::min<int64_t>(bw_mult * chunk_rows_for(m->dims[l - 1]), d->h_hdr.rows_total[l]) * 2 * m->dims[l - 1]);
+        if (l > 1 || d_h0_dev) {   // layers whose dX is handed down: dX of the whole layer, the turned-round entries
+            max_dx = std::max<int64_t>(max_dx, (int64_t)d->h_hdr.rows_total[l] * 2 * m->dims[l - 1]);
+            max_in = std::max<int64_t>(max_in, d->h_hdr.rows_total[l - 1]);
+            max_ent = std::max<int64_t>(max_ent, d->h_hdr.ent_base[k]);   // (entries of all hops bound any layer's)
+        }
+    }
+    const int64_t n_sum_tiles = (max_in + kRevTile - 1) / kRevTile + 1;
     if (ctx->bw_g_elems < g_total && (rc = mg_ensure(ctx, &ctx->bw_g, &ctx->bw_g_elems, g_total + g_total / 4 + 16))) return rc;
     if (ctx->bw_x_elems < (size_t)max_x && (rc = mg_ensure(ctx, &ctx->bw_x, &ctx->bw_x_elems, (size_t)max_x + 16))) return rc;
-    if (ctx->bw_dx_elems < (size_t)max_x && (rc = mg_ensure(ctx, &ctx->bw_dx, &ctx->bw_dx_elems, (size_t)max_x + 16))) return rc;
-    if (g_total) MG_CUDA(ctx, cudaMemsetAsync(ctx->bw_g, 0, g_total * sizeof(float), st));
-    if (d_h0_dev) MG_CUDA(ctx, cudaMemsetAsync(d_h0_dev, 0, (size_t)d->h_hdr.rows_total[0] * m->dims[0] * sizeof(float), st));
+    if (ctx->bw_dx_elems < (size_t)max_dx && (rc = mg_ensure(ctx, &ctx->bw_dx, &ctx->bw_dx_elems, (size_t)max_dx + 16))) return rc;
+    if (ctx->bw_off_elems < (size_t)(2 * max_in + n_sum_tiles + 2) &&
+        (rc = mg_ensure(ctx, &ctx->bw_off, &ctx->bw_off_elems, (size_t)(2 * max_in + n_sum_tiles + 2) + 16))) return rc;
+    if (ctx->bw_rev_elems < (size_t)max_ent && (rc = mg_ensure(ctx, &ctx->bw_rev, &ctx->bw_rev_elems, (size_t)max_ent + 16))) return rc;
     const RowGeom geom{B, k, d->rowbase, d->cum, d->node_off};
     const bool half = ctx->feat_dtype == MG_DTYPE_F16;
     const int grid = mg_grid(ctx, 8);
     for (int l = k; l >= 1; --l) {
         const int d_in = m->dims[l - 1], d_out = m->dims[l];
         const int64_t M = d->h_hdr.rows_total[l];
-        if (M == 0) continue;
+        // dPre of the last layer is the caller's gradient; below it, the gather of the layer above has already gone through
+        // the ReLU and summed the bias gradient
         const float* dpre_all = l == k ? d_out_dev : ctx->bw_g + g_off[l];
-        {   // through the ReLU (layers below the last), and the bias gradient
+        if (l == k && M > 0) {
             const int blocks = (int)std::min<int64_t>(grid, (M + kThreads / (d_out / 4) - 1) / (kThreads / (d_out / 4)));
-            if (l < k) k_grad_pre_bias<true><<<blocks, kThreads, 0, st>>>(ctx->bw_g + g_off[l], ctx->ws_h[0] + h_off[l], m->g_bias[l - 1], M, d_out);
-            else k_grad_pre_bias<false><<<blocks, kThreads, 0, st>>>(const_cast<float*>(d_out_dev), nullptr, m->g_bias[l - 1], M, d_out);
+            k_grad_pre_bias<false><<<blocks, kThreads, 0, st>>>(const_cast<float*>(d_out_dev), nullptr, m->g_bias[l - 1], M, d_out);
             ctx->launches++;
         }
         const float* h_prev = l > 1 ? ctx->ws_h[0] + h_off[l - 1] : nullptr;
@@ -981,20 +1142,38 @@ extern "C" int mg_backward(mg_ctx* ctx, mg_model* m, mg_dense* d, const float* d
             }
             ctx->launches++;   // (the aggregation above)
             if (!g_in) continue;   // layer 1 without a gradient of the base representations
+            float* dx = ctx->bw_dx + r0 * 2 * d_in;
             if (m->precision == MG_GEMM_TF32) {
                 // dX = dPre W^T on the tensor cores: the K-major operand the kernel wants is W itself ([2 d_in, d_out])
-                if ((rc = mg_gemm_tf32(ctx, dpre, m->w_cat[l - 1], m->zeros, ctx->bw_dx, rows, 2 * d_in, d_out, false))) return rc;
-                ctx->launches--;
+                if ((rc = mg_gemm_tf32(ctx, dpre, m->w_cat[l - 1], m->zeros, dx, rows, 2 * d_in, d_out, false))) return rc;
             } else {
                 dim3 gx((unsigned)((rows + 63) / 64), (unsigned)((2 * d_in + 63) / 64));
-                k_gemm_fp32<false><<<gx, 256, 0, st>>>(dpre, m->w_cat_t[l - 1], m->zeros, ctx->bw_dx, rows, 2 * d_in, d_out);
+                k_gemm_fp32<false><<<gx, 256, 0, st>>>(dpre, m->w_cat_t[l - 1], m->zeros, dx, rows, 2 * d_in, d_out);
+                ctx->launches++;
             }
-            ScatterArgs s;
-            s.g = geom; s.layer = l; s.row_lo = r0; s.row_hi = r1; s.ent_off = d->ent_off; s.ent_repr = d->ent_repr;
-            s.dx = ctx->bw_dx; s.d_in = d_in; s.sum_aggr = m->sum_aggr ? 1 : 0; s.g_in = g_in;
-            k_scatter_grad<<<grid, kThreads, 0, st>>>(s);
-            ctx->launches += 2;
         }
+        if (!g_in) continue;
+        // dX -> the gradient of the layer's input rows (see k_grad_gather)
+        const int64_t rows_in = d->h_hdr.rows_total[l - 1];
+        if (rows_in == 0) continue;
+        uint32_t* off = ctx->bw_off;
+        uint32_t* cur = ctx->bw_off + (rows_in + 1);
+        uint32_t* tile_sums = cur + rows_in;
+        const int n_tiles = (int)((rows_in + kRevTile - 1) / kRevTile);
+        MG_CUDA(ctx, cudaMemsetAsync(off, 0, sizeof(uint32_t) * (size_t)(2 * rows_in + 1), st));
+        RevArgs ra{geom, l, M, d->ent_off, d->ent_repr, off, off, ctx->bw_rev, m->sum_aggr ? 1 : 0};
+        const int rgrid = (int)std::max<int64_t>(1, std::min<int64_t>(grid, (M + kThreads - 1) / kThreads));
+        if (M > 0) k_rev_entries<false><<<rgrid, kThreads, 0, st>>>(ra);
+        k_rev_tile_sums<<<n_tiles, kThreads, 0, st>>>(off, rows_in, tile_sums);
+        k_rev_scan_sums<<<1, 1024, 0, st>>>(tile_sums, n_tiles);
+        k_rev_scan_tiles<<<n_tiles, kThreads, 0, st>>>(off, rows_in, tile_sums);
+        ra.cnt = cur;
+        if (M > 0) k_rev_entries<true><<<rgrid, kThreads, 0, st>>>(ra);
+        GatherArgs ga{geom, l, rows_in, off, ctx->bw_rev, ctx->bw_dx, d_in, l > 1 ? ctx->ws_h[0] + h_off[l - 1] : nullptr, g_in,
+                      l > 1 ? m->g_bias[l - 2] : nullptr};
+        const int ggrid = (int)std::max<int64_t>(1, std::min<int64_t>(grid, (rows_in + kThreads / 32 - 1) / (kThreads / 32)));
+        if (l > 1) launch_grad_gather<true>(ga, ggrid, st); else launch_grad_gather<false>(ga, ggrid, st);
+        ctx->launches += 6;
     }
     MG_CUDA(ctx, cudaGetLastError());
     MG_CUDA(ctx, cudaStreamSynchronize(st));

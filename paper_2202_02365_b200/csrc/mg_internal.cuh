@@ -152,6 +152,8 @@ struct mg_ctx {
     const struct mg_model* last_fwd_model = nullptr; const struct mg_dense* last_fwd_dense = nullptr;   // what mg_backward may follow
     float* bw_g = nullptr; float* bw_x = nullptr; float* bw_dx = nullptr;   // mg_backward scratch
     size_t bw_g_elems = 0, bw_x_elems = 0, bw_dx_elems = 0;
+    uint32_t* bw_off = nullptr; int2* bw_rev = nullptr;   // mg_backward: the turned-round entries of a layer
+    size_t bw_off_elems = 0, bw_rev_elems = 0;
     char* dm_images = nullptr; size_t dm_images_bytes = 0;   // TF32 operand images of the negatives (mg_distmult_score)
     bool prof_on = false;
     bool sample_graphs = true;   // replay the sampler's launches from a CUDA graph

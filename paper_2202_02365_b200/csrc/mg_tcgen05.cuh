@@ -191,13 +191,39 @@ __device__ __forceinline__ void store_slice_coalesced(const uint32_t* v, float* 
                                                       float* __restrict__ out, int64_t row0, int64_t M, int N, int c0,
                                                       bool relu) {
     const int lane = threadIdx.x & 31;
+    const int rows = (int)min((int64_t)32, M - row0);
+    if (N % 4 == 0 && ((reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(bias)) & 15) == 0) {
+        // rows start 16-byte aligned: the lane's 8 16-byte pieces go to slots piece ^ (row % 8) of its 128-byte row (no bank
+        // conflicts either way); then 8 lanes store one row's 128 bytes, 4 rows per instruction
+        uint8_t* sb = reinterpret_cast<uint8_t*>(stage);
+#pragma unroll
+        for (int p = 0; p < 8; ++p)
+            *reinterpret_cast<float4*>(sb + lane * 128 + ((p ^ (lane & 7)) << 4)) =
+                make_float4(__uint_as_float(v[4 * p]), __uint_as_float(v[4 * p + 1]), __uint_as_float(v[4 * p + 2]), __uint_as_float(v[4 * p + 3]));
+        __syncwarp();
+        const int p = lane & 7;
+        const int n = c0 + 4 * p;
+        if (n < N) {
+            const float4 b = __ldg(reinterpret_cast<const float4*>(bias + n));
+#pragma unroll
+            for (int r4 = 0; r4 < 32; r4 += 4) {
+                const int rr = r4 + (lane >> 3);
+                if (rr >= rows) continue;
+                float4 o = *reinterpret_cast<const float4*>(sb + rr * 128 + ((p ^ (rr & 7)) << 4));
+                o.x += b.x; o.y += b.y; o.z += b.z; o.w += b.w;
+                if (relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f); }
+                *reinterpret_cast<float4*>(out + (row0 + rr) * N + n) = o;
+            }
+        }
+        __syncwarp();
+        return;
+    }
 #pragma unroll
     for (int j = 0; j < 32; ++j) stage[lane * 33 + j] = __uint_as_float(v[j]);
     __syncwarp();
     const int n = c0 + lane;
     if (n < N) {
         const float b = __ldg(bias + n);
-        const int rows = (int)min((int64_t)32, M - row0);
         for (int rr = 0; rr < rows; ++rr) {
             float o = stage[rr * 33 + lane] + b;
             if (relu) o = fmaxf(o, 0.f);
