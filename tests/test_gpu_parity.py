@@ -1273,7 +1273,8 @@ def test_graph_attention_errors_and_fp16_features():
 
 
 @pytest.mark.parametrize("aggregator,prec,dims", [("mean", "fp32", [16, 24, 8]), ("sum", "fp32", [16, 24, 8]), ("mean", "tf32", [16, 24, 8]),
-                                                  ("mean", "tf32", [16, 64, 32])])
+                                                  ("mean", "tf32", [16, 64, 32]), ("mean", "tf32", [16, 520, 36]),
+                                                  ("sum", "fp32", [16, 300, 260])])
 def test_backward_pass_and_sgd_step(tiny, aggregator, prec, dims):
     """Gradients of a scalar loss through the GraphSage layers against the oracle's chain rule (itself pinned by
     finite differences): weights, biases and the base representations' rows; then one SGD step."""
