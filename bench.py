@@ -880,7 +880,7 @@ def run_lp(args, peaks, rank, local_rank, world):
         nonlocal dense, h
         src, rel, dst = batches[i]
         lp = ctx.lp_prepare(src, rel, dst, c["chunks"], c["negs"], seed=77 + i)
-        targets = lp.view()["targets"]
+        targets = lp.targets()
         dense = ctx.sample(targets, [c["fanout"]], seed=i, out=dense)
         if h is None or h.shape[0] < targets.numel():
             h = torch.empty((int(targets.numel() * 1.2) + 16, c["dim"]), dtype=torch.float32, device=device)

@@ -288,6 +288,13 @@ class LpBatch:
         self.n_edges = 0
         self.negs = 0
 
+    def targets(self) -> torch.Tensor:
+        """The batch's target union (distinct ids, ascending) alone: what the sampler is called with."""
+        n = C.c_int32(0)
+        p = C.c_void_p(0)
+        self.ctx._check(self.ctx.lib.mg_lp_view(self.handle, C.byref(n), C.byref(p), None, None, None, None))
+        return _from_dev(p.value, n.value, self.ctx.device)
+
     def view(self):
         n = C.c_int32(0)
         p = [C.c_void_p(0) for _ in range(5)]

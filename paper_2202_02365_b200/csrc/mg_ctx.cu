@@ -357,7 +357,8 @@ extern "C" int mg_destroy(mg_ctx* c) {
     cudaFree(c->ws_x); cudaFree(c->ws_h[0]); cudaFree(c->ws_h[1]);
     cudaEventDestroy(c->ev_fwd_done); cudaEventDestroy(c->ev_out_done); cudaEventDestroy(c->ev_user);
     for (int i = 0; i < 2; ++i) { if (c->ev_hk_done[i]) cudaEventDestroy(c->ev_hk_done[i]); cudaFree(c->hk_buf[i]); }
-    cudaFree(c->lp_ws); cudaFree(c->lp_spare); cudaFree(c->dm_images);
+    cudaFree(c->lp_ws); cudaFree(c->lp_spare); cudaFree(c->dm_images); cudaFree(c->lp_range);
+    if (c->lp_words) cudaFreeHost(c->lp_words);
     cudaFree(c->bw_g); cudaFree(c->bw_x); cudaFree(c->bw_dx); cudaFree(c->bw_off); cudaFree(c->bw_rev);
     cudaFree(c->gat_x); cudaFree(c->gat_z); cudaFree(c->gat_s); cudaFree(c->gat_h[0]); cudaFree(c->gat_h[1]);
     cudaStreamDestroy(c->sample_stream);

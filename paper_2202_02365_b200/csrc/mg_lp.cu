@@ -12,12 +12,15 @@ namespace {
 
 constexpr int kThreads = 256;
 
-// Builds the sort keys (id << 32 | origin) for sources, destinations and negatives.
-// origin: [0, E) sources, [E, 2E) destinations, [2E, 2E + C * negs) negatives.
+// The target union of a batch = the distinct ids among sources, destinations and negatives, ascending.  It is taken
+// with a bit per node: every id sets its bit (k_lp_mark, which also draws the negatives), the words' population counts
+// are scanned, a word's set bits are written out from its prefix on (k_lp_emit), and the row of an id is its word's prefix
+// plus the set bits below it (k_lp_index).  Seven short launches, none of them a sort.
+// Origins: [0, E) sources, [E, 2E) destinations, [2E, 2E + C * negs) negatives.
 __global__ void __launch_bounds__(kThreads)
-k_lp_keys(const int32_t* __restrict__ src, const int32_t* __restrict__ dst, int64_t E, int32_t n_chunks, int32_t negs,
+k_lp_mark(const int32_t* __restrict__ src, const int32_t* __restrict__ dst, int64_t E, int32_t n_chunks, int32_t negs,
           uint64_t seed, const int64_t* __restrict__ res_prefix, int32_t n_parts, int64_t n_resident, int64_t n_nodes, FeatGeom feat,
-          const int64_t* __restrict__ part_start, const int32_t* __restrict__ nodes_by_part, int32_t* neg_ids, uint64_t* keys,
+          const int64_t* __restrict__ part_start, const int32_t* __restrict__ nodes_by_part, int32_t* neg_ids, uint32_t* bitmap,
           uint32_t* status) {
     const int64_t total = 2 * E + (int64_t)n_chunks * negs;
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
@@ -39,30 +42,45 @@ k_lp_keys(const int32_t* __restrict__ src, const int32_t* __restrict__ dst, int6
             id = nodes_by_part ? nodes_by_part[part_start[p] + (r - res_prefix[p])] : (int32_t)(part_start[p] + (r - res_prefix[p]));
             neg_ids[j] = id;
         }
-        keys[i] = ((uint64_t)(uint32_t)id << 32) | (uint64_t)(uint32_t)i;
+        atomicOr(&bitmap[(uint32_t)id >> 5], 1u << (id & 31));
     }
 }
 
-__global__ void __launch_bounds__(kThreads) k_lp_heads(const uint64_t* __restrict__ sorted, int32_t n, uint32_t* heads) {
-    for (int32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
-        heads[i] = (i > 0 && (sorted[i] >> 32) != (sorted[i - 1] >> 32)) ? 1u : 0u;
+__global__ void __launch_bounds__(kThreads) k_lp_popc(const uint32_t* __restrict__ bitmap, int32_t n_words, uint32_t* counts) {
+    for (int32_t w = blockIdx.x * blockDim.x + threadIdx.x; w < n_words; w += gridDim.x * blockDim.x) counts[w] = __popc(bitmap[w]);
 }
 
-// after an exclusive scan of heads: rank[i] = scanned[i] + heads[i] is the target row of key i.
-// An exclusive scan of h gives rank[i] - h[i]; recompute h from the keys.
+// after the exclusive scan of the counts: the ids of the set bits, ascending
 __global__ void __launch_bounds__(kThreads)
-k_lp_scatter(const uint64_t* __restrict__ sorted, const uint32_t* __restrict__ scanned, int32_t n, int64_t E,
-             int32_t* targets, int32_t* src_idx, int32_t* dst_idx, int32_t* neg_idx, int32_t* n_targets) {
-    for (int32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
-        const uint64_t key = sorted[i];
-        const bool head = i > 0 && (key >> 32) != (sorted[i - 1] >> 32);
-        const int32_t rank = (int32_t)scanned[i] + (head ? 1 : 0);
-        const uint32_t origin = (uint32_t)key;
-        if (i == 0 || head) targets[rank] = (int32_t)(key >> 32);
-        if ((int64_t)origin < E) src_idx[origin] = rank;
-        else if ((int64_t)origin < 2 * E) dst_idx[origin - E] = rank;
-        else neg_idx[origin - 2 * E] = rank;
-        if (i == n - 1) *n_targets = rank + 1;
+k_lp_emit(const uint32_t* __restrict__ bitmap, const uint32_t* __restrict__ prefix, int32_t n_words, int32_t* targets) {
+    for (int32_t w = blockIdx.x * blockDim.x + threadIdx.x; w < n_words; w += gridDim.x * blockDim.x) {
+        uint32_t bits = bitmap[w];
+        if (!bits) continue;
+        uint32_t at = prefix[w];
+        while (bits) {
+            const int bpos = __ffs(bits) - 1;
+            targets[at++] = w * 32 + bpos;
+            bits &= bits - 1;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_lp_index(const int32_t* __restrict__ src, const int32_t* __restrict__ dst, const int32_t* __restrict__ neg_ids, int64_t E,
+           int64_t total, int64_t n_nodes, const uint32_t* __restrict__ bitmap, const uint32_t* __restrict__ prefix,
+           int32_t* src_idx, int32_t* dst_idx, int32_t* neg_idx, const uint32_t* status, const int32_t* n_targets, int32_t* host_words) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) {   // the call's two results, straight into mapped host memory
+        host_words[0] = (int32_t)*status;
+        host_words[1] = *n_targets;
+    }
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        int32_t id = i < E ? src[i] : (i < 2 * E ? dst[i - E] : neg_ids[i - 2 * E]);
+        if (id < 0 || (int64_t)id >= n_nodes) id = 0;   // (as k_lp_mark: the call fails with the range error anyway)
+        const uint32_t w = (uint32_t)id >> 5;
+        const int32_t rank = (int32_t)(prefix[w] + __popc(bitmap[w] & ((1u << (id & 31)) - 1u)));
+        if (i < E) src_idx[i] = rank;
+        else if (i < 2 * E) dst_idx[i - E] = rank;
+        else neg_idx[i - 2 * E] = rank;
     }
 }
 
@@ -430,12 +448,11 @@ extern "C" int mg_lp_prepare(mg_ctx* ctx, const int32_t* src, const int32_t* rel
     lp->ctx = ctx; lp->device = ctx->device; lp->n_edges = n_edges; lp->n_chunks = n_chunks; lp->negs = negs;
 
     const size_t n_neg = (size_t)std::max<int64_t>((int64_t)n_chunks * negs, 1);
-    const size_t hist_elems = mg_sort_hist_elems(total);
-    const size_t scan_elems = std::max(mg_scan_tmp_elems(total), mg_scan_tmp_elems((int64_t)hist_elems));
+    const int64_t n_words = (ctx->n_nodes + 31) / 32;
+    const size_t scan_elems = mg_scan_tmp_elems(n_words);
     auto up = [](size_t b) { return (b + 255) / 256 * 256; };
     // scratch: one block of the context that only grows
-    const size_t ws_bytes = 2 * up(4 * (size_t)n_edges) + 2 * up(8 * (size_t)total) + up(4 * (size_t)total) + up(4 * hist_elems) +
-                            up(4 * scan_elems) + 3 * 256;
+    const size_t ws_bytes = 2 * up(4 * (size_t)n_edges) + 2 * up(4 * (size_t)n_words) + up(4 * scan_elems) + 3 * 256;
     if (ctx->lp_ws_bytes < ws_bytes) {
         cudaFree(ctx->lp_ws);
         ctx->lp_ws = nullptr; ctx->lp_ws_bytes = 0;
@@ -449,15 +466,28 @@ extern "C" int mg_lp_prepare(mg_ctx* ctx, const int32_t* src, const int32_t* rel
     auto take = [&](size_t b) { char* p = w; w += up(b); return p; };
     int32_t* d_src = (int32_t*)take(4 * (size_t)n_edges);
     int32_t* d_dst = (int32_t*)take(4 * (size_t)n_edges);
-    uint64_t* keys[2];
-    keys[0] = (uint64_t*)take(8 * (size_t)total);
-    keys[1] = (uint64_t*)take(8 * (size_t)total);
-    uint32_t* heads = (uint32_t*)take(4 * (size_t)total);
-    uint32_t* hist = (uint32_t*)take(4 * hist_elems);
+    uint32_t* bitmap = (uint32_t*)take(4 * (size_t)n_words);
+    uint32_t* prefix = (uint32_t*)take(4 * (size_t)n_words);
     uint32_t* scan_tmp = (uint32_t*)take(4 * scan_elems);
     uint32_t* d_status = (uint32_t*)take(4);
     int32_t* d_nt = (int32_t*)take(4);
-    SortParams* sp = (SortParams*)take(sizeof(SortParams));
+    if (!ctx->lp_words) {
+        if (cudaHostAlloc((void**)&ctx->lp_words, 2 * sizeof(int32_t), cudaHostAllocMapped) != cudaSuccess ||
+            cudaHostGetDevicePointer((void**)&ctx->lp_words_dev, ctx->lp_words, 0) != cudaSuccess ||
+            cudaMalloc((void**)&ctx->lp_range, 2 * sizeof(int32_t)) != cudaSuccess) {
+            cudaGetLastError(); delete lp;
+            return mg_fail(ctx, MG_ERR_OOM, "allocation of the link-prediction scratch failed");
+        }
+    }
+    if (ctx->lp_range_words != n_words) {   // (once per graph)
+        const int32_t h_range[2] = {0, (int32_t)n_words};
+        if (cudaMemcpy(ctx->lp_range, h_range, sizeof(h_range), cudaMemcpyHostToDevice) != cudaSuccess) {
+            cudaGetLastError(); delete lp;
+            return mg_fail(ctx, MG_ERR_CUDA, "copy failed");
+        }
+        ctx->lp_range_words = n_words;
+    }
+    const int32_t* d_range = ctx->lp_range;
     // results: one block, taken from the context's spare when that is large enough
     const size_t blk_bytes = up(4 * (size_t)total) + 3 * up(4 * (size_t)n_edges) + 2 * up(4 * n_neg);
     if (ctx->lp_spare && ctx->lp_spare_bytes >= blk_bytes) {
@@ -478,30 +508,24 @@ extern "C" int mg_lp_prepare(mg_ctx* ctx, const int32_t* src, const int32_t* rel
     lp->neg_idx = (int32_t*)take(4 * n_neg);
     auto cleanup = [&]() {};
 
-    SortParams h_sp;
-    mg_sort_params_host(&h_sp, total);
-    cudaMemcpyAsync(sp, &h_sp, sizeof(h_sp), cudaMemcpyHostToDevice, st);
     cudaMemcpyAsync(d_src, src, 4 * n_edges, cudaMemcpyHostToDevice, st);
     cudaMemcpyAsync(d_dst, dst, 4 * n_edges, cudaMemcpyHostToDevice, st);
     cudaMemcpyAsync(lp->rel, rel, 4 * n_edges, cudaMemcpyHostToDevice, st);
     cudaMemsetAsync(d_status, 0, 4, st);
+    cudaMemsetAsync(bitmap, 0, 4 * (size_t)n_words, st);
     const int grid = mg_grid(ctx, 4);
-    k_lp_keys<<<grid, kThreads, 0, st>>>(d_src, d_dst, n_edges, n_chunks, negs, seed, ctx->d_res_prefix, ctx->n_parts,
+    k_lp_mark<<<grid, kThreads, 0, st>>>(d_src, d_dst, n_edges, n_chunks, negs, seed, ctx->d_res_prefix, ctx->n_parts,
                                          ctx->n_resident_nodes, ctx->n_nodes, mg_feat_geom(ctx), ctx->d_part_start, ctx->d_nodes_by_part,
-                                         lp->neg_ids, keys[0], d_status);
-    int id_bits = 1;
-    while ((1ll << id_bits) < ctx->n_nodes) ++id_bits;
-    int res = 0;
-    mg_sort_u64(ctx, keys, sp, 32, id_bits, hist, scan_tmp, &res);
-    k_lp_heads<<<grid, kThreads, 0, st>>>(keys[res], (int32_t)total, heads);
-    mg_scan_u32(ctx, heads, &sp->zero, &sp->n, nullptr, scan_tmp, nullptr);
-    k_lp_scatter<<<grid, kThreads, 0, st>>>(keys[res], heads, (int32_t)total, n_edges, lp->targets, lp->src_idx, lp->dst_idx,
-                                            lp->neg_idx, d_nt);
-    ctx->launches += 3;
-    uint32_t h_status = 0;
-    cudaMemcpyAsync(&h_status, d_status, 4, cudaMemcpyDeviceToHost, st);
-    cudaMemcpyAsync(&lp->n_targets, d_nt, 4, cudaMemcpyDeviceToHost, st);
+                                         lp->neg_ids, bitmap, d_status);
+    k_lp_popc<<<grid, kThreads, 0, st>>>(bitmap, (int32_t)n_words, prefix);
+    mg_scan_u32(ctx, prefix, d_range, d_range + 1, nullptr, scan_tmp, reinterpret_cast<uint32_t*>(d_nt));
+    k_lp_emit<<<grid, kThreads, 0, st>>>(bitmap, prefix, (int32_t)n_words, lp->targets);
+    k_lp_index<<<grid, kThreads, 0, st>>>(d_src, d_dst, lp->neg_ids, n_edges, total, ctx->n_nodes, bitmap, prefix, lp->src_idx,
+                                          lp->dst_idx, lp->neg_idx, d_status, d_nt, ctx->lp_words_dev);
+    ctx->launches += 4;
     cudaError_t e = cudaStreamSynchronize(st);
+    const uint32_t h_status = e == cudaSuccess ? (uint32_t)ctx->lp_words[0] : 0u;
+    lp->n_targets = e == cudaSuccess ? ctx->lp_words[1] : 0;
     if (e == cudaSuccess) e = cudaGetLastError();
     cleanup();
     if (e != cudaSuccess) { mg_lp_free(lp); return mg_cuda_fail(ctx, e, "mg_lp_prepare"); }
