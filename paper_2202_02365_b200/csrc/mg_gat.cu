@@ -21,8 +21,6 @@
 int mg_gemm_tf32(mg_ctx* ctx, const float* x, const float* w_t, const float* bias, float* out, int64_t M, int N, int K,
                  bool relu);
 int mg_gemm_tf32_status(mg_ctx* ctx);
-int mg_gemm_tf32_dots(mg_ctx* ctx, const float* x, const float* w_t, const float* zero_bias, float* out, int64_t M, int N, int K,
-                      const float* a, const float* b, float* s_a, float* s_b);
 
 struct mg_gat_model {
     mg_ctx* ctx = nullptr;
@@ -37,6 +35,8 @@ struct mg_gat_model {
     float* a_src[MG_MAX_HOPS] = {nullptr};   // device [d_out]
     float* a_dst[MG_MAX_HOPS] = {nullptr};
     float* bias[MG_MAX_HOPS] = {nullptr};
+    float* u_src[MG_MAX_HOPS] = {nullptr};   // device [d_in]: W a_src and W a_dst -- the score terms taken on the layer's
+    float* u_dst[MG_MAX_HOPS] = {nullptr};   // INPUT rows (single head: Z a = (H W) a = H (W a))
     float* zeros = nullptr;                  // device [max d_out]: the GEMM's bias
 };
 
@@ -118,9 +118,9 @@ __global__ void __launch_bounds__(kThreads) k_gat_gather0(GatherArgs a) {
     }
 }
 
-// fp32 GEMM on CUDA cores (the precision option): out[M, N] = x[M, K] w[K, N]
+// fp32 GEMM on CUDA cores (the precision option): out[M, N] = act(x[M, K] w[K, N] + bias) (bias may be null)
 __global__ void __launch_bounds__(256) k_gat_gemm_fp32(const float* __restrict__ x, const float* __restrict__ w, float* out,
-                                                       int64_t M, int N, int K) {
+                                                       int64_t M, int N, int K, const float* __restrict__ bias = nullptr, int relu = 0) {
     constexpr int BM = 64, BN = 64, BK = 16;
     __shared__ float xs[BK][BM + 4];
     __shared__ float ws[BK][BN + 4];
@@ -155,28 +155,16 @@ __global__ void __launch_bounds__(256) k_gat_gemm_fp32(const float* __restrict__
         if (m >= M) continue;
         for (int j = 0; j < 4; ++j) {
             const int n = n0 + tx * 4 + j;
-            if (n < N) out[m * N + n] = acc[i][j];
+            if (n < N) {
+                float v = acc[i][j] + (bias ? bias[n] : 0.f);
+                if (relu) v = fmaxf(v, 0.f);
+                out[m * N + n] = v;
+            }
         }
     }
 }
 
-// s_src[r] = Z[r] . a_src, s_dst[r] = Z[r] . a_dst (one warp per row, fixed summation order)
-__global__ void __launch_bounds__(kThreads) k_gat_scores(const float* __restrict__ z, const float* __restrict__ a_src,
-                                                         const float* __restrict__ a_dst, int64_t n_rows, int dim, float* s_src,
-                                                         float* s_dst) {
-    const int lane = threadIdx.x & 31;
-    const int64_t warps = (int64_t)gridDim.x * (kThreads / 32);
-    for (int64_t row = blockIdx.x * (int64_t)(kThreads / 32) + (threadIdx.x >> 5); row < n_rows; row += warps) {
-        const float* zr = z + row * dim;
-        float ps = 0.f, pd = 0.f;
-        for (int c = lane; c < dim; c += 32) { const float v = zr[c]; ps = fmaf(v, a_src[c], ps); pd = fmaf(v, a_dst[c], pd); }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) { ps += __shfl_xor_sync(0xFFFFFFFFu, ps, o); pd += __shfl_xor_sync(0xFFFFFFFFu, pd, o); }
-        if (lane == 0) { s_src[row] = ps; s_dst[row] = pd; }
-    }
-}
-
-// the same per head: s[row * heads + h] over the head's columns [h * dh, (h + 1) * dh)
+// per head: s_src[row * heads + h] = Z[row] . a_src, s_dst likewise, over the head's columns [h * dh, (h + 1) * dh) (one warp per row)
 __global__ void __launch_bounds__(kThreads) k_gat_scores_heads(const float* __restrict__ z, const float* __restrict__ a_src,
                                                                const float* __restrict__ a_dst, int64_t n_rows, int dim, int heads,
                                                                float* s_src, float* s_dst) {
@@ -213,53 +201,123 @@ struct AttendArgs {
 
 __device__ __forceinline__ float leaky(float v, float slope) { return v > 0.f ? v : slope * v; }
 
-// one warp per output row: softmax over {self} + entries, then the weighted sum of their Z rows
-template <int W>   // W = 32-column slices a lane owns: the row is at most 32 W wide
-__global__ void __launch_bounds__(kThreads) k_gat_attend(AttendArgs a) {
+// Single head, attention taken in the layer's input space.  Z a = (H W) a = H (W a): the two score terms of a row are
+// dot products of its INPUT row with u_src = W a_src and u_dst = W a_dst, and sum_j alpha_ij Z_j = (sum_j alpha_ij H_j) W:
+// one warp per OUTPUT row reads the row's own input row and its entries' input rows once each (layer 1: straight from
+// the partition buffer), keeps a running softmax (maximum, denominator, weighted sum, rescaled when the maximum
+// grows) and stores the attention-weighted input row; the linear map then runs over the output rows only.  Nothing of
+// the width of Z exists for the input rows, and no H^0 copy.
+struct InAttendArgs {
+    GatGeom g;
+    int32_t layer;              // 1 .. k
+    const int32_t* nodes;
+    const int32_t* ent_off;
+    const int32_t* ent_nbrs;    // layer 1: the entries' node ids
+    const int32_t* ent_repr;    // later layers: the entries' local rows of layer - 1
+    const char* slots; FeatGeom feat; int64_t row_bytes;   // layer 1
+    const float* h_prev;        // later layers: [rows of layer - 1, dim]
+    const float* u_src; const float* u_dst;   // [dim]
+    int64_t n_rows;             // rows of this layer
+    int32_t dim, round;
+    float slope;
+    float* x;                   // [n_rows, dim]
+};
+
+template <bool FIRST, bool HALF, int NCH>   // a lane owns NCH groups of four columns: rows up to 128 NCH wide
+__global__ void __launch_bounds__(kThreads) k_gat_attend_inputs(InAttendArgs a) {
+    constexpr int U = NCH == 1 ? 4 : (NCH == 2 ? 2 : 1);   // entries whose rows are in flight together
     const int lane = threadIdx.x & 31;
+    const int n4 = a.dim / 4;
     const int64_t warps = (int64_t)gridDim.x * (kThreads / 32);
     const int32_t* rb_in = a.g.rowbase + (int64_t)(a.layer - 1) * (a.g.B + 1);
+    float4 us[NCH], ud[NCH];
+#pragma unroll
+    for (int q = 0; q < NCH; ++q) {
+        const int c = lane + 32 * q;
+        us[q] = c < n4 ? reinterpret_cast<const float4*>(a.u_src)[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+        ud[q] = c < n4 ? reinterpret_cast<const float4*>(a.u_dst)[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    auto load_row = [&](const char* p, float4* v) {
+#pragma unroll
+        for (int q = 0; q < NCH; ++q) {
+            const int c = lane + 32 * q;
+            if (c >= n4) { v[q] = make_float4(0.f, 0.f, 0.f, 0.f); continue; }
+            if (HALF) {
+                const uint2 raw = reinterpret_cast<const uint2*>(p)[c];
+                const float2 lo = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
+                const float2 hi = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
+                v[q] = make_float4(lo.x, lo.y, hi.x, hi.y);
+            } else {
+                v[q] = reinterpret_cast<const float4*>(p)[c];
+            }
+        }
+    };
+    auto dot = [&](const float4* v, const float4* u) {
+        float s = 0.f;
+#pragma unroll
+        for (int q = 0; q < NCH; ++q) s += v[q].x * u[q].x + v[q].y * u[q].y + v[q].z * u[q].z + v[q].w * u[q].w;
+        return s;
+    };
     for (int64_t row = blockIdx.x * (int64_t)(kThreads / 32) + (threadIdx.x >> 5); row < a.n_rows; row += warps) {
         int32_t b, local, node;
         locate(a.g, a.layer, row, &b, &local, &node);
-        const int64_t in0 = rb_in[b];            // the mini-batch's first input row; a local row keeps its index
-        const int64_t me = in0 + local;
+        const int64_t in0 = rb_in[b];
+        auto row_of = [&](bool self, int32_t e) -> const char* {
+            if (FIRST) return a.slots + feat_row(a.feat, self ? a.nodes[node] : a.ent_nbrs[e]) * a.row_bytes;
+            return reinterpret_cast<const char*>(a.h_prev + (in0 + (self ? local : a.ent_repr[e])) * a.dim);
+        };
         const int32_t e0 = a.ent_off[node], e1 = a.ent_off[node + 1];
-        const float sd = a.s_dst[me];
-        const float self_score = leaky(sd + a.s_src[me], a.slope);
-        float mx = self_score;
-        for (int32_t e = e0 + lane; e < e1; e += 32) mx = fmaxf(mx, leaky(sd + a.s_src[in0 + a.ent_repr[e]], a.slope));
+        float4 acc[NCH];
+        load_row(row_of(true, 0), acc);
+        float ss = dot(acc, us), sd = dot(acc, ud);
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
-        float den = lane == 0 ? __expf(self_score - mx) : 0.f;
-        for (int32_t e = e0 + lane; e < e1; e += 32) den += __expf(leaky(sd + a.s_src[in0 + a.ent_repr[e]], a.slope) - mx);
+        for (int o = 16; o > 0; o >>= 1) { ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o); sd += __shfl_xor_sync(0xFFFFFFFFu, sd, o); }
+        float mx = leaky(sd + ss, a.slope), den = 1.f;   // the row itself: weight exp(0) so far
+        for (int32_t e = e0; e < e1; e += U) {
+            float4 v[U][NCH];
+            float s[U];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xFFFFFFFFu, den, o);
+            for (int u = 0; u < U; ++u) load_row(row_of(false, min(e + u, e1 - 1)), v[u]);
+#pragma unroll
+            for (int u = 0; u < U; ++u) s[u] = dot(v[u], us);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+                for (int u = 0; u < U; ++u) s[u] += __shfl_xor_sync(0xFFFFFFFFu, s[u], o);
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (e + u >= e1) continue;
+                const float logit = leaky(sd + s[u], a.slope);
+                const float m_new = fmaxf(mx, logit);
+                const float keep = __expf(mx - m_new), w = __expf(logit - m_new);
+                den = den * keep + w;
+#pragma unroll
+                for (int q = 0; q < NCH; ++q) {
+                    acc[q].x = acc[q].x * keep + w * v[u][q].x; acc[q].y = acc[q].y * keep + w * v[u][q].y;
+                    acc[q].z = acc[q].z * keep + w * v[u][q].z; acc[q].w = acc[q].w * keep + w * v[u][q].w;
+                }
+                mx = m_new;
+            }
+        }
         const float inv = 1.f / den;
-        float acc[W];
-        {
-            const float w = __expf(self_score - mx) * inv;
-            const float* zr = a.z + me * a.dim;
 #pragma unroll
-            for (int q = 0; q < W; ++q) { const int c = lane + 32 * q; acc[q] = c < a.dim ? w * zr[c] : 0.f; }
-        }
-        for (int32_t e = e0; e < e1; ++e) {
-            const int64_t src = in0 + a.ent_repr[e];
-            const float w = __expf(leaky(sd + a.s_src[src], a.slope) - mx) * inv;
-            const float* zr = a.z + src * a.dim;
-#pragma unroll
-            for (int q = 0; q < W; ++q) { const int c = lane + 32 * q; if (c < a.dim) acc[q] = fmaf(w, zr[c], acc[q]); }
-        }
-        float* dst = a.out + row * a.dim;
-#pragma unroll
-        for (int q = 0; q < W; ++q) {
+        for (int q = 0; q < NCH; ++q) {
             const int c = lane + 32 * q;
-            if (c >= a.dim) continue;
-            float v = acc[q] + a.bias[c];
-            if (a.relu) v = fmaxf(v, 0.f);
-            dst[c] = a.round ? round_tf32(v) : v;
+            if (c >= n4) continue;
+            float4 o = make_float4(acc[q].x * inv, acc[q].y * inv, acc[q].z * inv, acc[q].w * inv);
+            if (a.round) o = make_float4(round_tf32(o.x), round_tf32(o.y), round_tf32(o.z), round_tf32(o.w));
+            reinterpret_cast<float4*>(a.x + row * a.dim)[c] = o;
         }
     }
+}
+
+template <bool FIRST, bool HALF>
+void launch_attend_inputs(const InAttendArgs& a, int grid, cudaStream_t st) {
+    const int nch = (a.dim + 127) / 128;
+    if (nch <= 1) k_gat_attend_inputs<FIRST, HALF, 1><<<grid, kThreads, 0, st>>>(a);
+    else if (nch <= 2) k_gat_attend_inputs<FIRST, HALF, 2><<<grid, kThreads, 0, st>>>(a);
+    else if (nch <= 4) k_gat_attend_inputs<FIRST, HALF, 4><<<grid, kThreads, 0, st>>>(a);
+    else k_gat_attend_inputs<FIRST, HALF, 8><<<grid, kThreads, 0, st>>>(a);
 }
 
 constexpr int kMaxHeads = 8;
@@ -342,6 +400,7 @@ extern "C" int mg_gat_model_free(mg_gat_model* m) {
     cudaSetDevice(m->device);
     for (int l = 0; l < MG_MAX_HOPS; ++l) {
         cudaFree(m->w[l]); cudaFree(m->w_t[l]); cudaFree(m->a_src[l]); cudaFree(m->a_dst[l]); cudaFree(m->bias[l]);
+        cudaFree(m->u_src[l]); cudaFree(m->u_dst[l]);
     }
     cudaFree(m->zeros);
     delete m;
@@ -384,6 +443,17 @@ extern "C" int mg_gat_model_create(mg_ctx* ctx, int32_t k, const int32_t* dims, 
         cudaMemcpyAsync(m->bias[l], bias[l], sizeof(float) * dn, cudaMemcpyHostToDevice, ctx->stream);
         k_gat_transpose<<<mg_grid(ctx, 2), kThreads, 0, ctx->stream>>>(m->w[l], m->w_t[l], (int)di, (int)dn, gemm_precision == MG_GEMM_TF32);
         ctx->launches++;
+        // W a_src and W a_dst (double sums, rounded once): the score terms on the layer's input rows
+        std::vector<float> us(di), ud(di);
+        for (size_t r = 0; r < di; ++r) {
+            double s1 = 0.0, s2 = 0.0;
+            for (size_t c = 0; c < dn; ++c) { s1 += (double)w[l][r * dn + c] * a_src[l][c]; s2 += (double)w[l][r * dn + c] * a_dst[l][c]; }
+            us[r] = (float)s1; ud[r] = (float)s2;
+        }
+        ok = cudaMalloc((void**)&m->u_src[l], sizeof(float) * di) == cudaSuccess &&
+             cudaMalloc((void**)&m->u_dst[l], sizeof(float) * di) == cudaSuccess &&
+             cudaMemcpy(m->u_src[l], us.data(), sizeof(float) * di, cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMemcpy(m->u_dst[l], ud.data(), sizeof(float) * di, cudaMemcpyHostToDevice) == cudaSuccess;
     }
     if (!ok) {
         cudaGetLastError();
@@ -411,6 +481,59 @@ extern "C" int mg_gat_forward(mg_ctx* ctx, const mg_gat_model* m, mg_dense* d, f
     const int k = d->k, B = d->n_batches;
     cudaStream_t st = ctx->stream;
     const bool tf32 = m->precision == MG_GEMM_TF32;
+    int rc;
+    // (a quarter of headroom when a buffer grows: calls of slightly different sizes then share it)
+    auto grow = [&](float** p, size_t* have, size_t need) { return *have >= need && *p ? MG_OK : mg_ensure(ctx, p, have, need + need / 4 + 16); };
+    const GatGeom geom{B, k, d->rowbase, d->cum, d->node_off};
+    const int grid = mg_grid(ctx, 8);
+    if (m->heads == 1) {
+        // single head: attention on the input rows, then the linear map over the output rows (k_gat_attend_inputs)
+        size_t need_x = 0, need_h = 0;
+        for (int l = 1; l <= k; ++l) {
+            need_x = std::max(need_x, (size_t)d->h_hdr.rows_total[l] * m->dims[l - 1]);
+            if (l < k) need_h = std::max(need_h, (size_t)d->h_hdr.rows_total[l] * m->dims[l]);
+        }
+        if ((rc = grow(&ctx->gat_x, &ctx->gat_x_elems, need_x))) return rc;
+        for (int i = 0; i < 2; ++i)
+            if ((rc = grow(&ctx->gat_h[i], &ctx->gat_h_elems[i], need_h))) return rc;
+        if (d->h_hdr.rows_total[k] == 0) return MG_OK;
+        const float* h_in = nullptr;
+        for (int l = 1; l <= k; ++l) {
+            const int d_in = m->dims[l - 1], d_out = m->dims[l];
+            const int64_t rows_out = d->h_hdr.rows_total[l];
+            {
+                ProfScope ps(ctx, l == 1 ? PH_AGG_L1 : PH_AGG_REST, 1);
+                InAttendArgs a;
+                a.g = geom; a.layer = l; a.nodes = d->nodes; a.ent_off = d->ent_off; a.ent_nbrs = d->ent_nbrs; a.ent_repr = d->ent_repr;
+                a.slots = ctx->slots; a.feat = mg_feat_geom(ctx); a.row_bytes = ctx->row_bytes; a.h_prev = h_in;
+                a.u_src = m->u_src[l - 1]; a.u_dst = m->u_dst[l - 1]; a.n_rows = rows_out; a.dim = d_in; a.round = tf32 ? 1 : 0;
+                a.slope = m->slope; a.x = ctx->gat_x;
+                if (l == 1) {
+                    if (ctx->feat_dtype == MG_DTYPE_F16) launch_attend_inputs<true, true>(a, grid, st);
+                    else launch_attend_inputs<true, false>(a, grid, st);
+                } else {
+                    launch_attend_inputs<false, false>(a, grid, st);
+                }
+                ctx->launches++;
+            }
+            float* out_l = l == k ? out_dev : ctx->gat_h[l & 1];
+            {
+                ProfScope ps(ctx, PH_GEMM, 1);
+                if (tf32) {
+                    if ((rc = mg_gemm_tf32(ctx, ctx->gat_x, m->w_t[l - 1], m->bias[l - 1], out_l, rows_out, d_out, d_in, l < k))) return rc;
+                } else {
+                    dim3 g2((unsigned)((rows_out + 63) / 64), (unsigned)((d_out + 63) / 64));
+                    k_gat_gemm_fp32<<<g2, 256, 0, st>>>(ctx->gat_x, m->w[l - 1], out_l, rows_out, d_out, d_in, m->bias[l - 1], l < k ? 1 : 0);
+                    ctx->launches++;
+                }
+            }
+            h_in = out_l;
+        }
+        MG_CUDA(ctx, cudaGetLastError());
+        MG_CUDA(ctx, cudaStreamSynchronize(st));
+        return tf32 ? mg_gemm_tf32_status(ctx) : MG_OK;
+    }
+    // several heads: Z = H W for the input rows, per-head scores, attention over Z
     // scratch: H^0, Z and the two score vectors of the widest layer, two buffers for the layer outputs
     size_t need_x = (size_t)d->h_hdr.rows_total[0] * m->dims[0], need_z = 0, need_s = 0, need_h = 0;
     for (int l = 1; l <= k; ++l) {
@@ -418,17 +541,12 @@ extern "C" int mg_gat_forward(mg_ctx* ctx, const mg_gat_model* m, mg_dense* d, f
         need_s = std::max(need_s, (size_t)d->h_hdr.rows_total[l - 1] * 2 * m->heads);
         if (l < k) need_h = std::max(need_h, (size_t)d->h_hdr.rows_total[l] * m->dims[l]);
     }
-    int rc;
-    // (a quarter of headroom when a buffer grows: calls of slightly different sizes then share it)
-    auto grow = [&](float** p, size_t* have, size_t need) { return *have >= need && *p ? MG_OK : mg_ensure(ctx, p, have, need + need / 4 + 16); };
     if ((rc = grow(&ctx->gat_x, &ctx->gat_x_elems, need_x))) return rc;
     if ((rc = grow(&ctx->gat_z, &ctx->gat_z_elems, need_z))) return rc;
     if ((rc = grow(&ctx->gat_s, &ctx->gat_s_elems, need_s))) return rc;
     for (int i = 0; i < 2; ++i)
         if ((rc = grow(&ctx->gat_h[i], &ctx->gat_h_elems[i], need_h))) return rc;
     if (d->h_hdr.rows_total[k] == 0) return MG_OK;
-    const GatGeom geom{B, k, d->rowbase, d->cum, d->node_off};
-    const int grid = mg_grid(ctx, 8);
     {
         ProfScope ps(ctx, PH_AGG_L1, 1);
         GatherArgs a;
@@ -446,13 +564,9 @@ extern "C" int mg_gat_forward(mg_ctx* ctx, const mg_gat_model* m, mg_dense* d, f
         float* s_src = ctx->gat_s;
         const int H = m->heads;
         float* s_dst = ctx->gat_s + rows_in * H;
-        const bool fused_scores = tf32 && d_out <= 256 && H == 1;   // the GEMM's epilogue also leaves Z a_src and Z a_dst
         {
             ProfScope ps(ctx, PH_GEMM, 1);
-            if (fused_scores) {
-                if ((rc = mg_gemm_tf32_dots(ctx, h_prev, m->w_t[l - 1], m->zeros, ctx->gat_z, rows_in, d_out, d_in, m->a_src[l - 1],
-                                            m->a_dst[l - 1], s_src, s_dst))) return rc;
-            } else if (tf32) {
+            if (tf32) {
                 if ((rc = mg_gemm_tf32(ctx, h_prev, m->w_t[l - 1], m->zeros, ctx->gat_z, rows_in, d_out, d_in, false))) return rc;
             } else {
                 dim3 g2((unsigned)((rows_in + 63) / 64), (unsigned)((d_out + 63) / 64));
@@ -461,8 +575,7 @@ extern "C" int mg_gat_forward(mg_ctx* ctx, const mg_gat_model* m, mg_dense* d, f
             }
         }
         ProfScope ps(ctx, PH_AGG_REST, 2);
-        if (H > 1) k_gat_scores_heads<<<grid, kThreads, 0, st>>>(ctx->gat_z, m->a_src[l - 1], m->a_dst[l - 1], rows_in, d_out, H, s_src, s_dst);
-        else if (!fused_scores) k_gat_scores<<<grid, kThreads, 0, st>>>(ctx->gat_z, m->a_src[l - 1], m->a_dst[l - 1], rows_in, d_out, s_src, s_dst);
+        k_gat_scores_heads<<<grid, kThreads, 0, st>>>(ctx->gat_z, m->a_src[l - 1], m->a_dst[l - 1], rows_in, d_out, H, s_src, s_dst);
         AttendArgs a;
         a.g = geom; a.layer = l; a.ent_off = d->ent_off; a.ent_repr = d->ent_repr; a.z = ctx->gat_z; a.s_src = s_src; a.s_dst = s_dst;
         a.bias = m->bias[l - 1]; a.n_rows = rows_out; a.dim = d_out; a.relu = l < k; a.round = (tf32 && l < k) ? 1 : 0;
@@ -470,18 +583,12 @@ extern "C" int mg_gat_forward(mg_ctx* ctx, const mg_gat_model* m, mg_dense* d, f
         a.heads = H;
         a.out = l == k ? out_dev : ctx->gat_h[l & 1];
         const int slices = (d_out + 31) / 32;   // instantiations for rows of up to 32, 64, 128, 256, 512 floats
-        if (H > 1) {
-            if (slices <= 1) k_gat_attend_heads<1><<<grid, kThreads, 0, st>>>(a);
-            else if (slices <= 2) k_gat_attend_heads<2><<<grid, kThreads, 0, st>>>(a);
-            else if (slices <= 4) k_gat_attend_heads<4><<<grid, kThreads, 0, st>>>(a);
-            else if (slices <= 8) k_gat_attend_heads<8><<<grid, kThreads, 0, st>>>(a);
-            else k_gat_attend_heads<kMaxWidthPerLane><<<grid, kThreads, 0, st>>>(a);
-        } else if (slices <= 1) k_gat_attend<1><<<grid, kThreads, 0, st>>>(a);
-        else if (slices <= 2) k_gat_attend<2><<<grid, kThreads, 0, st>>>(a);
-        else if (slices <= 4) k_gat_attend<4><<<grid, kThreads, 0, st>>>(a);
-        else if (slices <= 8) k_gat_attend<8><<<grid, kThreads, 0, st>>>(a);
-        else k_gat_attend<kMaxWidthPerLane><<<grid, kThreads, 0, st>>>(a);
-        ctx->launches += fused_scores ? 1 : 2;
+        if (slices <= 1) k_gat_attend_heads<1><<<grid, kThreads, 0, st>>>(a);
+        else if (slices <= 2) k_gat_attend_heads<2><<<grid, kThreads, 0, st>>>(a);
+        else if (slices <= 4) k_gat_attend_heads<4><<<grid, kThreads, 0, st>>>(a);
+        else if (slices <= 8) k_gat_attend_heads<8><<<grid, kThreads, 0, st>>>(a);
+        else k_gat_attend_heads<kMaxWidthPerLane><<<grid, kThreads, 0, st>>>(a);
+        ctx->launches += 2;
         h_prev = a.out;
     }
     MG_CUDA(ctx, cudaGetLastError());

@@ -31,9 +31,6 @@ struct GemmParams {
     const float* bias;
     int64_t M;
     int32_t N, K, BN, stages, tmem_cols, relu;
-    // optional: two dot products of every output row (before bias and activation) with the vectors dot_a, dot_b [N],
-    // written to dot_out_a, dot_out_b [M]; only when one tile spans the whole width (N <= BN)
-    const float* dot_a; const float* dot_b; float* dot_out_a; float* dot_out_b;
     int32_t kt_per_slice;   // split-K: blockIdx.z owns this many 32-wide K steps and ADDS its product to out (0 = whole K, plain store)
     int32_t mn_major;       // 1: the operands are stored [K, M] and [K, N] (the contraction runs over their rows)
     uint32_t* error;  // device word: 0 = ok, else the role that gave up waiting
@@ -44,12 +41,9 @@ k_gemm_tf32(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[8], empty_bar[8], acc_bar;
     __shared__ uint32_t tmem_slot;
-    __shared__ float dot_vec[2][256];   // the two vectors of the optional row dot products
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t m0 = (int64_t)blockIdx.x * BM;
-    if (p.dot_a)
-        for (int i = threadIdx.x; i < p.N; i += kGemmThreads) { dot_vec[0][i] = p.dot_a[i]; dot_vec[1][i] = p.dot_b[i]; }
     const int n0 = blockIdx.y * p.BN;
     const int kt_all = (p.K + BK - 1) / BK;
     const int kt_first = p.kt_per_slice ? (int)blockIdx.z * p.kt_per_slice : 0;
@@ -131,27 +125,14 @@ k_gemm_tf32(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         // warps' transpose buffers for coalesced stores
         float* out_stage = reinterpret_cast<float*>(stage_base);
         if (ok) {
-            float dot_a = 0.f, dot_b = 0.f;   // every lane holds one row of the tile: its dot products need no shuffles
             for (int c0 = 0; c0 < p.BN; c0 += 32) {
                 uint32_t v[32];
                 tmem_ld_32(tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)c0, v);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 if (row0 >= p.M) continue;
-                if (p.dot_a) {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int n = n0 + c0 + j;
-                        if (n < p.N) {
-                            const float z = __uint_as_float(v[j]);
-                            dot_a = fmaf(z, dot_vec[0][n], dot_a);
-                            dot_b = fmaf(z, dot_vec[1][n], dot_b);
-                        }
-                    }
-                }
                 if (p.kt_per_slice) add_slice_coalesced(v, out_stage + lane_group * (32 * 33), p.out, row0, p.M, p.N, n0 + c0);
                 else store_slice_coalesced(v, out_stage + lane_group * (32 * 33), p.bias, p.out, row0, p.M, p.N, n0 + c0, p.relu != 0);
             }
-            if (p.dot_a && row0 + lane < p.M) { p.dot_out_a[row0 + lane] = dot_a; p.dot_out_b[row0 + lane] = dot_b; }
         }
     }
     tc_fence_before();
@@ -165,16 +146,13 @@ k_gemm_tf32(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 }  // namespace
 
 static int gemm_tf32_launch(mg_ctx* ctx, const float* x, const float* w_t, const float* bias, float* out, int64_t M, int N, int K,
-                            bool relu, int kt_per_slice, const float* dot_a = nullptr, const float* dot_b = nullptr,
-                            float* dot_out_a = nullptr, float* dot_out_b = nullptr, bool mn_major = false) {
+                            bool relu, int kt_per_slice, bool mn_major = false) {
     if (M <= 0) return MG_OK;
     if ((mn_major ? M : K) % 4 != 0 || N % 4 != 0) return mg_fail(ctx, MG_ERR_ARG, "GEMM sizes must be multiples of 4");
     GemmParams p;
     p.out = out; p.bias = bias; p.M = M; p.N = N; p.K = K; p.relu = relu ? 1 : 0; p.error = ctx->d_flags;
     p.kt_per_slice = kt_per_slice;
     p.mn_major = mn_major ? 1 : 0;
-    p.dot_a = dot_a; p.dot_b = dot_b; p.dot_out_a = dot_out_a; p.dot_out_b = dot_out_b;
-    if (dot_a && N > 256) return mg_fail(ctx, MG_ERR_ARG, "row dot products need a single tile across the width");
     p.BN = mn_major ? std::min(256, (N + 31) / 32 * 32) : std::min(256, (N + 15) / 16 * 16);
     p.tmem_cols = 32;
     while (p.tmem_cols < p.BN) p.tmem_cols <<= 1;
@@ -204,19 +182,12 @@ int mg_gemm_tf32(mg_ctx* ctx, const float* x, const float* w_t, const float* bia
     return gemm_tf32_launch(ctx, x, w_t, bias, out, M, N, K, relu, 0);
 }
 
-// out = x . w_t^T (no bias, no activation) and, from the same accumulators, s_a[r] = out[r] . a, s_b[r] = out[r] . b
-// (N <= 256): the attention layers' transformed rows and their two score terms in one pass.
-int mg_gemm_tf32_dots(mg_ctx* ctx, const float* x, const float* w_t, const float* zero_bias, float* out, int64_t M, int N, int K,
-                      const float* a, const float* b, float* s_a, float* s_b) {
-    return gemm_tf32_launch(ctx, x, w_t, zero_bias, out, M, N, K, false, 0, a, b, s_a, s_b);
-}
-
 // out[M, N] += x[K, M]^T . g[K, N], both operands as they lie in memory (rows = the contraction, far longer than M and
 // N: weight gradients), the contraction split over CTAs (kt_per_slice steps of 32 rows each; atomic adds, any order).
 // M and N are multiples of 4; rows past K and columns past M, N read as zeros.
 int mg_gemm_tf32_splitk_add_rows(mg_ctx* ctx, const float* x, const float* g, float* out, int M, int N, int64_t K, int kt_per_slice) {
     if (K >= (1ll << 31)) return mg_fail(ctx, MG_ERR_ARG, "too many rows for one product");
-    return gemm_tf32_launch(ctx, x, g, nullptr, out, M, N, (int)K, false, std::max(1, kt_per_slice), nullptr, nullptr, nullptr, nullptr, true);
+    return gemm_tf32_launch(ctx, x, g, nullptr, out, M, N, (int)K, false, std::max(1, kt_per_slice), true);
 }
 
 // After the stream has drained: MG_ERR_TIMEOUT if a GEMM gave up on a barrier (the word is cleared).
