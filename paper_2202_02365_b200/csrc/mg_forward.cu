@@ -939,13 +939,18 @@ struct GatherArgs {
     float* db;                 // [d_in] bias gradient of layer - 1 (MASK)
 };
 
-// one warp per source row; a lane keeps NCH groups of four columns (d_in <= 128 NCH)
+// A warp takes 32 consecutive source rows.  Lane = row first: where the row lies, its list bounds and its first
+// contribution, one coalesced round of loads for all 32 rows instead of a chain of dependent look-ups per row.  Then
+// row after row, lane = four columns (NCH groups of them: d_in <= 128 NCH), with the loads of the next row issued
+// before the current one is summed.
 template <bool MASK, int NCH>
 __global__ void __launch_bounds__(kThreads) k_grad_gather(GatherArgs a) {
     __shared__ float sums[MASK ? 128 * NCH : 1];
     const int lane = threadIdx.x & 31;
     const int n4 = a.d_in / 4;
     const int32_t* rb_out = a.g.rowbase + (int64_t)a.layer * (a.g.B + 1);
+    const float* __restrict__ dx = a.dx;
+    const int64_t ld = 2 * (int64_t)a.d_in;
     if (MASK) {
         for (int c = threadIdx.x; c < 128 * NCH; c += kThreads) sums[c] = 0.f;
         __syncthreads();
@@ -953,51 +958,70 @@ __global__ void __launch_bounds__(kThreads) k_grad_gather(GatherArgs a) {
     float4 bias[NCH];
 #pragma unroll
     for (int q = 0; q < NCH; ++q) bias[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-    const int64_t warps = (int64_t)gridDim.x * (kThreads / 32);
-    for (int64_t s = blockIdx.x * (int64_t)(kThreads / 32) + (threadIdx.x >> 5); s < a.rows_in; s += warps) {
-        int32_t b, local, node;
-        locate_row(a.g, a.layer - 1, s, &b, &local, &node);
-        const int32_t n_out = rb_out[b + 1] - rb_out[b];
-        const uint32_t i0 = a.off[s], i1 = a.off[s + 1];
-        float4 acc[NCH];
+    const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    // the self part and the first contribution of row r of the warp's 32 (both optional), as loads in flight
+    auto fetch = [&](int64_t self_row, int32_t first_row, float4* vs, float4* vf) {
 #pragma unroll
         for (int q = 0; q < NCH; ++q) {
             const int c = lane + 32 * q;
-            acc[q] = (local < n_out && c < n4)
-                         ? reinterpret_cast<const float4*>(a.dx + ((int64_t)rb_out[b] + local) * 2 * a.d_in)[c]
-                         : make_float4(0.f, 0.f, 0.f, 0.f);
+            vs[q] = (self_row >= 0 && c < n4) ? reinterpret_cast<const float4*>(dx + self_row * ld)[c] : zero4;
+            vf[q] = (first_row >= 0 && c < n4) ? reinterpret_cast<const float4*>(dx + (int64_t)first_row * ld + a.d_in)[c] : zero4;
         }
-        for (uint32_t i = i0; i < i1; i += 2) {   // two contributions in flight
-            const int2 r0 = a.rev[i];
-            const bool two = i + 1 < i1;
-            const int2 r1 = two ? a.rev[i + 1] : r0;
-            const float w0 = __int_as_float(r0.y), w1 = two ? __int_as_float(r1.y) : 0.f;
-            const float4* p0 = reinterpret_cast<const float4*>(a.dx + (int64_t)r0.x * 2 * a.d_in + a.d_in);
-            const float4* p1 = reinterpret_cast<const float4*>(a.dx + (int64_t)r1.x * 2 * a.d_in + a.d_in);
-            float4 v0[NCH], v1[NCH];
+    };
+    const int64_t warps = (int64_t)gridDim.x * (kThreads / 32);
+    for (int64_t s0 = (blockIdx.x * (int64_t)(kThreads / 32) + (threadIdx.x >> 5)) * 32; s0 < a.rows_in; s0 += warps * 32) {
+        // lane = row
+        const int64_t sl = s0 + lane;
+        uint32_t i0 = 0, i1 = 0;
+        int64_t self_l = -1;
+        int2 first_l = make_int2(-1, 0);
+        if (sl < a.rows_in) {
+            int32_t b, local, node;
+            locate_row(a.g, a.layer - 1, sl, &b, &local, &node);
+            i0 = a.off[sl]; i1 = a.off[sl + 1];
+            if (local < rb_out[b + 1] - rb_out[b]) self_l = (int64_t)rb_out[b] + local;
+            if (i1 > i0) first_l = a.rev[i0];
+        }
+        const int n_here = (int)min((int64_t)32, a.rows_in - s0);
+        float4 vs[NCH], vf[NCH];
+        fetch(__shfl_sync(0xFFFFFFFFu, self_l, 0), __shfl_sync(0xFFFFFFFFu, first_l.x, 0), vs, vf);
+        for (int r = 0; r < n_here; ++r) {
+            const float w_first = __int_as_float(__shfl_sync(0xFFFFFFFFu, first_l.y, r));
+            const uint32_t j0 = __shfl_sync(0xFFFFFFFFu, i0, r), j1 = __shfl_sync(0xFFFFFFFFu, i1, r);
+            float4 acc[NCH];
+#pragma unroll
+            for (int q = 0; q < NCH; ++q)
+                acc[q] = make_float4(vs[q].x + w_first * vf[q].x, vs[q].y + w_first * vf[q].y, vs[q].z + w_first * vf[q].z,
+                                     vs[q].w + w_first * vf[q].w);
+            // the next row's loads go out before this row's remaining contributions and its store
+            const int rn = min(r + 1, 31);
+            fetch(r + 1 < n_here ? __shfl_sync(0xFFFFFFFFu, self_l, rn) : (int64_t)-1,
+                  r + 1 < n_here ? __shfl_sync(0xFFFFFFFFu, first_l.x, rn) : -1, vs, vf);
+            for (uint32_t i = j0 + 1; i < j1; ++i) {   // (most rows are named by one entry: this loop is the exception)
+                const int2 rr = a.rev[i];
+                const float w = __int_as_float(rr.y);
+                const float4* pp = reinterpret_cast<const float4*>(dx + (int64_t)rr.x * ld + a.d_in);
+#pragma unroll
+                for (int q = 0; q < NCH; ++q) {
+                    const int c = lane + 32 * q;
+                    if (c >= n4) continue;
+                    const float4 v = pp[c];
+                    acc[q].x += w * v.x; acc[q].y += w * v.y; acc[q].z += w * v.z; acc[q].w += w * v.w;
+                }
+            }
+            const int64_t s = s0 + r;
 #pragma unroll
             for (int q = 0; q < NCH; ++q) {
                 const int c = lane + 32 * q;
-                v0[q] = c < n4 ? p0[c] : make_float4(0.f, 0.f, 0.f, 0.f);
-                v1[q] = c < n4 ? p1[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+                if (c >= n4) continue;
+                float4 v = acc[q];
+                if (MASK) {
+                    const float4 yy = reinterpret_cast<const float4*>(a.y + s * a.d_in)[c];
+                    v = make_float4(yy.x > 0.f ? v.x : 0.f, yy.y > 0.f ? v.y : 0.f, yy.z > 0.f ? v.z : 0.f, yy.w > 0.f ? v.w : 0.f);
+                    bias[q].x += v.x; bias[q].y += v.y; bias[q].z += v.z; bias[q].w += v.w;
+                }
+                reinterpret_cast<float4*>(a.g_in + s * a.d_in)[c] = v;
             }
-#pragma unroll
-            for (int q = 0; q < NCH; ++q) {
-                acc[q].x += w0 * v0[q].x + w1 * v1[q].x; acc[q].y += w0 * v0[q].y + w1 * v1[q].y;
-                acc[q].z += w0 * v0[q].z + w1 * v1[q].z; acc[q].w += w0 * v0[q].w + w1 * v1[q].w;
-            }
-        }
-#pragma unroll
-        for (int q = 0; q < NCH; ++q) {
-            const int c = lane + 32 * q;
-            if (c >= n4) continue;
-            float4 v = acc[q];
-            if (MASK) {
-                const float4 yy = reinterpret_cast<const float4*>(a.y + s * a.d_in)[c];
-                v = make_float4(yy.x > 0.f ? v.x : 0.f, yy.y > 0.f ? v.y : 0.f, yy.z > 0.f ? v.z : 0.f, yy.w > 0.f ? v.w : 0.f);
-                bias[q].x += v.x; bias[q].y += v.y; bias[q].z += v.z; bias[q].w += v.w;
-            }
-            reinterpret_cast<float4*>(a.g_in + s * a.d_in)[c] = v;
         }
     }
     if (MASK) {
@@ -1171,7 +1195,7 @@ extern "C" int mg_backward(mg_ctx* ctx, mg_model* m, mg_dense* d, const float* d
         if (M > 0) k_rev_entries<true><<<rgrid, kThreads, 0, st>>>(ra);
         GatherArgs ga{geom, l, rows_in, off, ctx->bw_rev, ctx->bw_dx, d_in, l > 1 ? ctx->ws_h[0] + h_off[l - 1] : nullptr, g_in,
                       l > 1 ? m->g_bias[l - 2] : nullptr};
-        const int ggrid = (int)std::max<int64_t>(1, std::min<int64_t>(grid, (rows_in + kThreads / 32 - 1) / (kThreads / 32)));
+        const int ggrid = (int)std::max<int64_t>(1, std::min<int64_t>(grid, (rows_in + kThreads - 1) / kThreads));   // 32 rows per warp
         if (l > 1) launch_grad_gather<true>(ga, ggrid, st); else launch_grad_gather<false>(ga, ggrid, st);
         ctx->launches += 6;
     }
