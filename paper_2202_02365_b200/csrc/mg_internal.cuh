@@ -149,7 +149,7 @@ struct mg_ctx {
     char* lp_spare = nullptr; size_t lp_spare_bytes = 0;
     int32_t* lp_words = nullptr;       // mapped pinned host words {status, n_targets} that mg_lp_prepare's last kernel writes
     int32_t* lp_words_dev = nullptr;   // their device address
-    int32_t* lp_range = nullptr;       // device {0, words of the node bitmap}: the bounds of mg_lp_prepare's scan
+    int32_t* lp_range = nullptr;       // device {0, 32-word groups of the node bitmap}: the bounds of mg_lp_prepare's scan
     int64_t lp_range_words = -1;
     float* gat_x = nullptr; float* gat_z = nullptr; float* gat_s = nullptr; float* gat_h[2] = {nullptr, nullptr};   // mg_gat_forward scratch
     size_t gat_x_elems = 0, gat_z_elems = 0, gat_s_elems = 0, gat_h_elems[2] = {0, 0};

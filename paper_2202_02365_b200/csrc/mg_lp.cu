@@ -15,7 +15,8 @@ constexpr int kThreads = 256;
 // The target union of a batch = the distinct ids among sources, destinations and negatives, ascending.  It is taken
 // with a bit per node: every id sets its bit (k_lp_mark, which also draws the negatives), the words' population counts
 // are scanned, a word's set bits are written out from its prefix on (k_lp_emit), and the row of an id is its word's prefix
-// plus the set bits below it (k_lp_index).  Seven short launches, none of them a sort.
+// plus the set bits below it (k_lp_index); counts and prefixes are kept per group of 32 words, so the scan runs over
+// n_nodes / 1024 values.  Seven short launches, none of them a sort.
 // Origins: [0, E) sources, [E, 2E) destinations, [2E, 2E + C * negs) negatives.
 __global__ void __launch_bounds__(kThreads)
 k_lp_mark(const int32_t* __restrict__ src, const int32_t* __restrict__ dst, int64_t E, int32_t n_chunks, int32_t negs,
@@ -46,17 +47,30 @@ k_lp_mark(const int32_t* __restrict__ src, const int32_t* __restrict__ dst, int6
     }
 }
 
-__global__ void __launch_bounds__(kThreads) k_lp_popc(const uint32_t* __restrict__ bitmap, int32_t n_words, uint32_t* counts) {
-    for (int32_t w = blockIdx.x * blockDim.x + threadIdx.x; w < n_words; w += gridDim.x * blockDim.x) counts[w] = __popc(bitmap[w]);
+// population count of every group of 32 words (1,024 nodes): the scan then runs over n_words / 32 counts
+constexpr int kLpGroup = 32;
+__global__ void __launch_bounds__(kThreads) k_lp_popc(const uint32_t* __restrict__ bitmap, int32_t n_words, int32_t n_groups, uint32_t* counts) {
+    const int lane = threadIdx.x & 31;
+    const int32_t warps = gridDim.x * (kThreads / 32);
+    for (int32_t g = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5); g < n_groups; g += warps) {
+        const int32_t w = g * kLpGroup + lane;
+        uint32_t c = w < n_words ? __popc(bitmap[w]) : 0u;
+        for (int o = 16; o; o >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
+        if (lane == 0) counts[g] = c;
+    }
 }
 
-// after the exclusive scan of the counts: the ids of the set bits, ascending
+// after the exclusive scan of the group counts: the ids of the set bits, ascending (a warp per group: lane = word)
 __global__ void __launch_bounds__(kThreads)
-k_lp_emit(const uint32_t* __restrict__ bitmap, const uint32_t* __restrict__ prefix, int32_t n_words, int32_t* targets) {
-    for (int32_t w = blockIdx.x * blockDim.x + threadIdx.x; w < n_words; w += gridDim.x * blockDim.x) {
-        uint32_t bits = bitmap[w];
-        if (!bits) continue;
-        uint32_t at = prefix[w];
+k_lp_emit(const uint32_t* __restrict__ bitmap, const uint32_t* __restrict__ prefix, int32_t n_words, int32_t n_groups, int32_t* targets) {
+    const int lane = threadIdx.x & 31;
+    const int32_t warps = gridDim.x * (kThreads / 32);
+    for (int32_t g = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5); g < n_groups; g += warps) {
+        const int32_t w = g * kLpGroup + lane;
+        uint32_t bits = w < n_words ? bitmap[w] : 0u;
+        if (!__any_sync(0xFFFFFFFFu, bits != 0u)) continue;
+        const uint32_t c = __popc(bits);
+        uint32_t at = prefix[g] + warp_incl_scan(c) - c;
         while (bits) {
             const int bpos = __ffs(bits) - 1;
             targets[at++] = w * 32 + bpos;
@@ -77,10 +91,12 @@ k_lp_index(const int32_t* __restrict__ src, const int32_t* __restrict__ dst, con
         int32_t id = i < E ? src[i] : (i < 2 * E ? dst[i - E] : neg_ids[i - 2 * E]);
         if (id < 0 || (int64_t)id >= n_nodes) id = 0;   // (as k_lp_mark: the call fails with the range error anyway)
         const uint32_t w = (uint32_t)id >> 5;
-        const int32_t rank = (int32_t)(prefix[w] + __popc(bitmap[w] & ((1u << (id & 31)) - 1u)));
-        if (i < E) src_idx[i] = rank;
-        else if (i < 2 * E) dst_idx[i - E] = rank;
-        else neg_idx[i - 2 * E] = rank;
+        // the group's prefix, the set bits of the group's words before this one, the set bits below the id in its word
+        uint32_t rank = prefix[w / kLpGroup] + __popc(bitmap[w] & ((1u << (id & 31)) - 1u));
+        for (uint32_t v = w - w % kLpGroup; v < w; ++v) rank += __popc(bitmap[v]);
+        if (i < E) src_idx[i] = (int32_t)rank;
+        else if (i < 2 * E) dst_idx[i - E] = (int32_t)rank;
+        else neg_idx[i - 2 * E] = (int32_t)rank;
     }
 }
 
@@ -449,10 +465,11 @@ extern "C" int mg_lp_prepare(mg_ctx* ctx, const int32_t* src, const int32_t* rel
 
     const size_t n_neg = (size_t)std::max<int64_t>((int64_t)n_chunks * negs, 1);
     const int64_t n_words = (ctx->n_nodes + 31) / 32;
-    const size_t scan_elems = mg_scan_tmp_elems(n_words);
+    const int64_t n_groups = (n_words + kLpGroup - 1) / kLpGroup;
+    const size_t scan_elems = mg_scan_tmp_elems(n_groups);
     auto up = [](size_t b) { return (b + 255) / 256 * 256; };
     // scratch: one block of the context that only grows
-    const size_t ws_bytes = 2 * up(4 * (size_t)n_edges) + 2 * up(4 * (size_t)n_words) + up(4 * scan_elems) + 3 * 256;
+    const size_t ws_bytes = 2 * up(4 * (size_t)n_edges) + up(4 * (size_t)n_words) + up(4 * (size_t)n_groups) + up(4 * scan_elems) + 3 * 256;
     if (ctx->lp_ws_bytes < ws_bytes) {
         cudaFree(ctx->lp_ws);
         ctx->lp_ws = nullptr; ctx->lp_ws_bytes = 0;
@@ -467,7 +484,7 @@ extern "C" int mg_lp_prepare(mg_ctx* ctx, const int32_t* src, const int32_t* rel
     int32_t* d_src = (int32_t*)take(4 * (size_t)n_edges);
     int32_t* d_dst = (int32_t*)take(4 * (size_t)n_edges);
     uint32_t* bitmap = (uint32_t*)take(4 * (size_t)n_words);
-    uint32_t* prefix = (uint32_t*)take(4 * (size_t)n_words);
+    uint32_t* prefix = (uint32_t*)take(4 * (size_t)n_groups);
     uint32_t* scan_tmp = (uint32_t*)take(4 * scan_elems);
     uint32_t* d_status = (uint32_t*)take(4);
     int32_t* d_nt = (int32_t*)take(4);
@@ -480,7 +497,7 @@ extern "C" int mg_lp_prepare(mg_ctx* ctx, const int32_t* src, const int32_t* rel
         }
     }
     if (ctx->lp_range_words != n_words) {   // (once per graph)
-        const int32_t h_range[2] = {0, (int32_t)n_words};
+        const int32_t h_range[2] = {0, (int32_t)n_groups};
         if (cudaMemcpy(ctx->lp_range, h_range, sizeof(h_range), cudaMemcpyHostToDevice) != cudaSuccess) {
             cudaGetLastError(); delete lp;
             return mg_fail(ctx, MG_ERR_CUDA, "copy failed");
@@ -517,9 +534,9 @@ extern "C" int mg_lp_prepare(mg_ctx* ctx, const int32_t* src, const int32_t* rel
     k_lp_mark<<<grid, kThreads, 0, st>>>(d_src, d_dst, n_edges, n_chunks, negs, seed, ctx->d_res_prefix, ctx->n_parts,
                                          ctx->n_resident_nodes, ctx->n_nodes, mg_feat_geom(ctx), ctx->d_part_start, ctx->d_nodes_by_part,
                                          lp->neg_ids, bitmap, d_status);
-    k_lp_popc<<<grid, kThreads, 0, st>>>(bitmap, (int32_t)n_words, prefix);
+    k_lp_popc<<<grid, kThreads, 0, st>>>(bitmap, (int32_t)n_words, (int32_t)n_groups, prefix);
     mg_scan_u32(ctx, prefix, d_range, d_range + 1, nullptr, scan_tmp, reinterpret_cast<uint32_t*>(d_nt));
-    k_lp_emit<<<grid, kThreads, 0, st>>>(bitmap, prefix, (int32_t)n_words, lp->targets);
+    k_lp_emit<<<grid, kThreads, 0, st>>>(bitmap, prefix, (int32_t)n_words, (int32_t)n_groups, lp->targets);
     k_lp_index<<<grid, kThreads, 0, st>>>(d_src, d_dst, lp->neg_ids, n_edges, total, ctx->n_nodes, bitmap, prefix, lp->src_idx,
                                           lp->dst_idx, lp->neg_idx, d_status, d_nt, ctx->lp_words_dev);
     ctx->launches += 4;
