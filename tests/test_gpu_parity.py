@@ -409,6 +409,7 @@ def test_link_prediction_distmult():
     prep = O.lp_prepare(view, src.tolist(), dst.tolist(), n_chunks, negs, 2024)
     got = lp.view()
     assert got["targets"].cpu().tolist() == prep["targets"]
+    assert lp.targets().cpu().tolist() == prep["targets"]     # (the accessor that builds the target tensor alone)
     assert got["src_idx"].cpu().tolist() == prep["src_idx"]
     assert got["dst_idx"].cpu().tolist() == prep["dst_idx"]
     assert got["neg_ids"].cpu().tolist() == prep["neg_ids"]
