@@ -875,16 +875,6 @@ constexpr size_t kScatterSmem = (size_t)kSortTile * 8 + (size_t)(kThreads / 32) 
 // -------------------------------------------------------------------------------------
 // place the sorted new nodes as the next hop
 // -------------------------------------------------------------------------------------
-__global__ void k_hop_advance(DenseHeader* hdr, int hop, int32_t B, int32_t* node_off_next, int64_t cap_nodes) {
-    if (hdr->status) return;
-    const int32_t start = hdr->hop_base[hop + 1];
-    const int64_t end = (int64_t)start + hdr->n_new;
-    if (end > cap_nodes) { if (threadIdx.x == 0) atomicOr(&hdr->status, ST_CAP_NODES); return; }
-    if (threadIdx.x == 0) hdr->hop_base[hop + 2] = (int32_t)end;
-    if (hdr->n_new == 0)
-        for (int b = threadIdx.x; b <= B; b += blockDim.x) node_off_next[b] = start;
-}
-
 __global__ void __launch_bounds__(kThreads)
 k_relabel(const DenseHeader* hdr, int hop, const int32_t* __restrict__ hvals, int32_t* ent_repr) {
     if (hdr->status) return;
@@ -895,14 +885,18 @@ k_relabel(const DenseHeader* hdr, int hop, const int32_t* __restrict__ hvals, in
     }
 }
 
-// Outermost hop: per-batch counts -> node offsets of the hop and the batches' row totals (one block)
+// End of a hop (one block): the node arena's next bound, then per-batch counts -> node offsets of the next hop and the
+// batches' row totals
 __global__ void __launch_bounds__(1024)
 k_outer_offsets(DenseHeader* hdr, int hop, int32_t B, int32_t k, const uint32_t* __restrict__ batch_cnt, int32_t* node_off_next,
-                int32_t* cum, int32_t max_nodes_per_batch) {
+                int32_t* cum, int32_t max_nodes_per_batch, int64_t cap_nodes) {
     __shared__ uint32_t warp_tot[33];
     if (hdr->status) return;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int32_t start = hdr->hop_base[hop + 1];
+    const int64_t end = (int64_t)start + hdr->n_new;
+    if (end > cap_nodes) { if (threadIdx.x == 0) atomicOr(&hdr->status, ST_CAP_NODES); return; }
+    if (threadIdx.x == 0) hdr->hop_base[hop + 2] = (int32_t)end;
     uint32_t carry = 0;
     for (int s0 = 0; s0 < B; s0 += 1024) {
         const int b = s0 + threadIdx.x;
@@ -1634,12 +1628,11 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
         {
             // rows were handed out at insert time, in discovery order: per-batch counts -> offsets, then every list
             // entry (mini-batch, id, rank) goes to its place.  No sort, no second pass over the id tables.
-            ProfScope ps(ctx, PH_SAMPLE_PLACE, 3);
+            ProfScope ps(ctx, PH_SAMPLE_PLACE, 2);
             int32_t* off_next = d->node_off + (size_t)(h + 1) * (B + 1);
-            k_hop_advance<<<1, 256, 0, st>>>(d->hdr, h, B, off_next, d->cap_nodes);
-            k_outer_offsets<<<1, 1024, 0, st>>>(d->hdr, h, B, k, batch_cnt + (size_t)h * B, off_next, d->cum, (int32_t)cap_batch);
+            k_outer_offsets<<<1, 1024, 0, st>>>(d->hdr, h, B, k, batch_cnt + (size_t)h * B, off_next, d->cum, (int32_t)cap_batch, d->cap_nodes);
             k_place_nodes_outer<<<grid, kThreads, 0, st>>>(d->hdr, d->newlist[0], id_bits, off_next, d->nodes, d->node_batch);
-            ctx->launches += 3;
+            ctx->launches += 2;
         }
         if (!(smem_last && h == k - 1)) {   // (the last hop's shared-memory kernel leaves final rows)
             ProfScope ps(ctx, PH_SAMPLE_RELABEL, 1);
