@@ -70,8 +70,16 @@ __global__ void __launch_bounds__(kThreads) k_scan_reduce(const uint32_t* data, 
     }
 }
 
+// what the scan of a hop's entry counts also does once the total is known: close the hop's entry range, check the arena
+struct HopClose {
+    DenseHeader* hdr;      // null: a plain scan
+    int hop;
+    int32_t* ent_off;
+    int64_t cap_entries;
+};
+
 // single block: exclusive scan of the tile sums in place; total (plus base) to *total_out
-__global__ void __launch_bounds__(1024) k_scan_tiles(uint32_t* tile_sums, ScanRange r, uint32_t* total_out) {
+__global__ void __launch_bounds__(1024) k_scan_tiles(uint32_t* tile_sums, ScanRange r, uint32_t* total_out, HopClose hc) {
     __shared__ uint32_t warp_tot[33];
     const int n = *r.hi - *r.lo;
     const int ntiles = (n + kScanTile - 1) / kScanTile;
@@ -94,7 +102,18 @@ __global__ void __launch_bounds__(1024) k_scan_tiles(uint32_t* tile_sums, ScanRa
         carry += warp_tot[32];
         __syncthreads();
     }
-    if (threadIdx.x == 0 && total_out) *total_out = carry + (r.base ? (uint32_t)*r.base : 0u);
+    if (threadIdx.x == 0) {
+        const uint32_t end = carry + (r.base ? (uint32_t)*r.base : 0u);
+        if (total_out) *total_out = end;
+        if (hc.hdr && !hc.hdr->status) {
+            if ((int64_t)end > hc.cap_entries) atomicOr(&hc.hdr->status, ST_CAP_ENTRIES);
+            else {
+                hc.hdr->ent_base[hc.hop + 1] = (int32_t)end;
+                hc.ent_off[hc.hdr->hop_base[hc.hop + 1]] = (int32_t)end;   // (past the range the scan's last kernel writes)
+                hc.hdr->n_new = 0;
+            }
+        }
+    }
 }
 
 __global__ void __launch_bounds__(kThreads) k_scan_down(uint32_t* data, ScanRange r, const uint32_t* tile_sums) {
@@ -192,16 +211,6 @@ k_count(const DenseHeader* hdr, int hop, int32_t fanout, const int32_t* __restri
         }
         ent_off[i] = n;
     }
-}
-
-// after the scan: close the hop's entry range and check the arena
-__global__ void k_entries_done(DenseHeader* hdr, int hop, const uint32_t* total, int32_t* ent_off, int64_t cap_entries) {
-    if (hdr->status) return;
-    const uint32_t end = *total;  // already includes ent_base[hop]
-    if ((int64_t)end > cap_entries) { atomicOr(&hdr->status, ST_CAP_ENTRIES); return; }
-    hdr->ent_base[hop + 1] = (int32_t)end;
-    ent_off[hdr->hop_base[hop + 1]] = (int32_t)end;
-    hdr->n_new = 0;
 }
 
 struct PickArgs {
@@ -1213,7 +1222,7 @@ void mg_sort_u64(mg_ctx* ctx, uint64_t* const buf[2], const SortParams* sp, int 
         const int shift = lo_bit + kRadixBits * p;
         k_radix_hist<<<grid, kThreads, 0, st>>>(buf[cur], sp, shift, hist);
         k_scan_reduce<<<grid, kThreads, 0, st>>>(hist, r, scan_tmp);
-        k_scan_tiles<<<1, 1024, 0, st>>>(scan_tmp, r, nullptr);
+        k_scan_tiles<<<1, 1024, 0, st>>>(scan_tmp, r, nullptr, HopClose{nullptr, 0, nullptr, 0});
         k_scan_down<<<grid, kThreads, 0, st>>>(hist, r, scan_tmp);
         k_radix_scatter<<<grid, kThreads, kScatterSmem, st>>>(buf[cur], buf[cur ^ 1], sp, shift, hist);
         cur ^= 1;
@@ -1229,7 +1238,7 @@ void mg_scan_u32(mg_ctx* ctx, uint32_t* data, const int32_t* lo, const int32_t* 
     const int grid = mg_grid(ctx, 8);
     ScanRange r{lo, hi, base};
     k_scan_reduce<<<grid, kThreads, 0, st>>>(data, r, scan_tmp);
-    k_scan_tiles<<<1, 1024, 0, st>>>(scan_tmp, r, total_out);
+    k_scan_tiles<<<1, 1024, 0, st>>>(scan_tmp, r, total_out, HopClose{nullptr, 0, nullptr, 0});
     k_scan_down<<<grid, kThreads, 0, st>>>(data, r, scan_tmp);
     ctx->launches += 3;
 }
@@ -1581,10 +1590,13 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
                                                inout ? ctx->view_off_out : nullptr, d->node_r0_out, d->node_deg_out);
         }
         {
-            ProfScope ps(ctx, PH_SAMPLE_SCAN, 4);
-            mg_scan_u32(ctx, (uint32_t*)d->ent_off, &d->hdr->hop_base[h], &d->hdr->hop_base[h + 1], &d->hdr->ent_base[h],
-                        (uint32_t*)d->scan_tmp, scan_total);
-            k_entries_done<<<1, 1, 0, st>>>(d->hdr, h, scan_total, d->ent_off, d->cap_entries);
+            ProfScope ps(ctx, PH_SAMPLE_SCAN, 3);
+            // (the scan's middle kernel also closes the hop's entry range: ent_base, the sentinel offset, the arena check)
+            const ScanRange sr{&d->hdr->hop_base[h], &d->hdr->hop_base[h + 1], &d->hdr->ent_base[h]};
+            k_scan_reduce<<<grid, kThreads, 0, st>>>((uint32_t*)d->ent_off, sr, (uint32_t*)d->scan_tmp);
+            k_scan_tiles<<<1, 1024, 0, st>>>((uint32_t*)d->scan_tmp, sr, scan_total, HopClose{d->hdr, h, d->ent_off, d->cap_entries});
+            k_scan_down<<<grid, kThreads, 0, st>>>((uint32_t*)d->ent_off, sr, (uint32_t*)d->scan_tmp);
+            ctx->launches += 3;
         }
         {
             ProfScope ps(ctx, PH_SAMPLE_PICK, 1);
@@ -1639,7 +1651,7 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
             k_relabel<<<grid, kThreads, 0, st>>>(d->hdr, h, d->hvals, d->ent_repr);
             ctx->launches++;
         }
-        ctx->launches += 1 + 1 + 1;  // count, entries_done, pick
+        ctx->launches += 1 + 1;  // count, pick
     }
     {
         ProfScope ps(ctx, PH_SAMPLE_FINAL, 1);
