@@ -948,14 +948,17 @@ k_place_nodes_outer(const DenseHeader* hdr, const uint64_t* __restrict__ list, i
     }
 }
 
-// one block: packed row bases of every layer and the per-batch entry bounds of every hop
+// one block: packed row bases of every layer and the per-batch entry bounds of every hop; then the sample's summary
+// (header, per-batch tables) for the host, stored straight into mapped pinned memory.  A copy engine is not used on
+// purpose: a large output copy of a forward pass may be queued on it, and the host would wait for that copy before it
+// learned the sample's sizes.  (After an error the summary still goes out: it carries the status word.)
 __global__ void __launch_bounds__(1024)
-k_finalize(DenseHeader* hdr, int32_t B, int32_t k, const int32_t* __restrict__ cum, const int32_t* __restrict__ node_off,
-           const int32_t* __restrict__ ent_off, int32_t* rowbase, int32_t* ent_hop) {
+k_finalize(DenseHeader* hdr, int32_t B, int32_t k, const int32_t* cum, const int32_t* node_off,
+           const int32_t* __restrict__ ent_off, int32_t* rowbase, int32_t* ent_hop, int32_t n_hdr, int32_t* out) {
     __shared__ uint32_t warp_tot[33];
-    if (hdr->status) return;
+    const bool bad = hdr->status != 0;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int l = 0; l <= k; ++l) {
+    for (int l = 0; l <= k && !bad; ++l) {
         uint32_t carry = 0;
         for (int start = 0; start < B; start += 1024) {
             const int b = start + threadIdx.x;
@@ -979,24 +982,16 @@ k_finalize(DenseHeader* hdr, int32_t B, int32_t k, const int32_t* __restrict__ c
             hdr->rows_total[l] = (int32_t)carry;
         }
     }
-    for (int h = 0; h < k; ++h)
+    for (int h = 0; h < k && !bad; ++h)
         for (int b = threadIdx.x; b <= B; b += blockDim.x)
             ent_hop[h * (B + 1) + b] = ent_off[node_off[h * (B + 1) + b]];
-}
-
-
-// The sample's summary (header, per-batch tables) for the host: stored straight into mapped pinned memory.  A copy
-// engine is not used on purpose: a large output copy of a forward pass may be queued on it, and the host would wait
-// for that copy before it learned the sample's sizes.
-__global__ void __launch_bounds__(kThreads)
-k_summary(const DenseHeader* hdr, const int32_t* __restrict__ cum, const int32_t* __restrict__ node_off,
-          const int32_t* __restrict__ rowbase, const int32_t* __restrict__ ent_hop, int32_t n_hdr, int32_t n_cum, int32_t n_off,
-          int32_t n_ent, int32_t* out) {
+    __syncthreads();   // (one block: its own writes above are what the summary reads)
+    const int32_t n_cum = B * (k + 2), n_off = (k + 1) * (B + 1), n_ent = k * (B + 1);
     const int32_t total = n_hdr + n_cum + 2 * n_off + n_ent;
-    const int32_t* h = reinterpret_cast<const int32_t*>(hdr);
-    for (int32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+    const volatile int32_t* h32 = reinterpret_cast<const volatile int32_t*>(hdr);
+    for (int32_t i = threadIdx.x; i < total; i += blockDim.x) {
         int32_t j = i, v;
-        if (j < n_hdr) v = j < (int32_t)(sizeof(DenseHeader) / 4) ? h[j] : 0;
+        if (j < n_hdr) v = j < (int32_t)(sizeof(DenseHeader) / 4) ? h32[j] : 0;
         else if ((j -= n_hdr) < n_cum) v = cum[j];
         else if ((j -= n_cum) < n_off) v = node_off[j];
         else if ((j -= n_off) < n_off) v = rowbase[j];
@@ -1004,6 +999,7 @@ k_summary(const DenseHeader* hdr, const int32_t* __restrict__ cum, const int32_t
         out[i] = v;
     }
 }
+
 
 // -------------------------------------------------------------------------------------
 // export to the paper's layout (mg_dense_view)
@@ -1655,14 +1651,12 @@ static int sample_begin_impl(mg_ctx* ctx, const int32_t* targets, int targets_on
     }
     {
         ProfScope ps(ctx, PH_SAMPLE_FINAL, 1);
-        k_finalize<<<1, 1024, 0, st>>>(d->hdr, B, k, d->cum, d->node_off, d->ent_off, d->rowbase, d->d_ent_hop);
+        // (the summary goes to pinned host memory behind the kernels; mg_sample_many_end waits for it)
+        static_assert(sizeof(DenseHeader) % 4 == 0, "the header is copied as 32-bit words");
+        k_finalize<<<1, 1024, 0, st>>>(d->hdr, B, k, d->cum, d->node_off, d->ent_off, d->rowbase, d->d_ent_hop,
+                                       (int32_t)((sizeof(DenseHeader) + 3) / 4), d->h_pinned_dev);
         ctx->launches++;
     }
-    // the summary goes to pinned host memory behind the kernels; mg_sample_many_end waits for it
-    static_assert(sizeof(DenseHeader) % 4 == 0, "the header is copied as 32-bit words");
-    k_summary<<<8, kThreads, 0, st>>>(d->hdr, d->cum, d->node_off, d->rowbase, d->d_ent_hop, (int32_t)((sizeof(DenseHeader) + 3) / 4),
-                                     B * (k + 2), (k + 1) * (B + 1), k * (B + 1), d->h_pinned_dev);
-    ctx->launches++;
     MG_CUDA(ctx, cudaGetLastError());
     return MG_OK;
     };   // enqueue
