@@ -206,6 +206,8 @@ struct mg_dense {
     int32_t* scan_tmp = nullptr;    // block sums
     uint32_t* sort_hist = nullptr;  // radix histograms
     size_t scan_tmp_elems = 0, sort_hist_elems = 0;
+    void* seg_tiles = nullptr;      // tile table of the export's sort inside (mini-batch, delta) segments
+    int64_t cap_sort_tiles = 0;     // tiles the sort scratch (histograms, block sums, tile table) is sized for
     int64_t alloc_batches = 0, alloc_table = 0;
 
     // export buffer for mg_dense_view
@@ -350,6 +352,6 @@ void mg_sort_params_host(SortParams* sp, int64_t n);
 int mg_dense_batch_perm(mg_ctx* ctx, mg_dense* d, int b, const int32_t** perm, const int32_t** inv);
 size_t mg_scan_tmp_elems(int64_t max_elems);
 void mg_sort_u64(mg_ctx* ctx, uint64_t* const buf[2], const SortParams* sp, int lo_bit, int bits, uint32_t* hist,
-                 uint32_t* scan_tmp, int* res_buf);
+                 uint32_t* scan_tmp, int* res_buf, const void* seg_tiles = nullptr);
 void mg_scan_u32(mg_ctx* ctx, uint32_t* data, const int32_t* lo, const int32_t* hi, const int32_t* base,
                  uint32_t* scan_tmp, uint32_t* total_out);

@@ -771,25 +771,39 @@ constexpr int kBins = 1 << kRadixBits;
 constexpr int kBinsPerThread = kBins / kThreads;
 
 
+// A tile of a segmented sort: a run of at most kSortTile keys of one segment.  Its histogram sits with its segment's
+// (digit-major inside the segment), so that one exclusive scan over all histograms in segment order gives every
+// (segment, digit, tile) its place in the output, where segment follows segment.
+struct SegTile {
+    int32_t in0;      // first key of the tile in the input of the first pass (the segments lie elsewhere there)
+    int32_t out0;     // first key of the tile in every pass's output and the later passes' input
+    int32_t count;
+    int32_t hist0;    // index of the tile's count of digit 0
+    int32_t stride;   // distance between its counts of consecutive digits: the segment's tiles
+};
+
+// (tiles == nullptr: one segment, tile t = keys [t * kSortTile, ...), histograms digit-major over all tiles)
 __global__ void __launch_bounds__(kThreads)
-k_radix_hist(const uint64_t* __restrict__ keys, const SortParams* sp, int shift, uint32_t* hist) {
+k_radix_hist(const uint64_t* __restrict__ keys, const SortParams* sp, int shift, uint32_t* hist,
+             const SegTile* __restrict__ tiles, bool first_pass) {
     __shared__ uint32_t sh[kBins];
     const int32_t n = sp->n, ntiles = sp->ntiles;
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x) {
 #pragma unroll
         for (int q = 0; q < kBinsPerThread; ++q) sh[threadIdx.x + q * kThreads] = 0;
         __syncthreads();
-        const int32_t tb = t * kSortTile;
+        int32_t tb = t * kSortTile, tn = min(kSortTile, n - tb), h0 = t, hs = ntiles;
+        if (tiles) { const SegTile st = tiles[t]; tb = first_pass ? st.in0 : st.out0; tn = st.count; h0 = st.hist0; hs = st.stride; }
 #pragma unroll 4
         for (int j = 0; j < kSortKeysPerThread; ++j) {
-            const int32_t i = tb + j * kThreads + threadIdx.x;
-            if (i < n) atomicAdd(&sh[(uint32_t)(keys[i] >> shift) & (kBins - 1)], 1u);
+            const int32_t l = j * kThreads + threadIdx.x;
+            if (l < tn) atomicAdd(&sh[(uint32_t)(keys[tb + l] >> shift) & (kBins - 1)], 1u);
         }
         __syncthreads();
 #pragma unroll
         for (int q = 0; q < kBinsPerThread; ++q) {
             const int bin = threadIdx.x + q * kThreads;
-            hist[(size_t)bin * ntiles + t] = sh[bin];
+            hist[(size_t)h0 + (size_t)bin * hs] = sh[bin];
         }
         __syncthreads();
     }
@@ -800,7 +814,7 @@ k_radix_hist(const uint64_t* __restrict__ keys, const SortParams* sp, int shift,
 // equal digits leaves the SM as consecutive addresses.
 __global__ void __launch_bounds__(kThreads)
 k_radix_scatter(const uint64_t* __restrict__ keys, uint64_t* __restrict__ out, const SortParams* sp, int shift,
-                const uint32_t* __restrict__ hist_scanned) {
+                const uint32_t* __restrict__ hist_scanned, const SegTile* __restrict__ tiles, bool first_pass) {
     extern __shared__ __align__(16) uint8_t sort_smem[];
     uint64_t* stage = reinterpret_cast<uint64_t*>(sort_smem);                          // [kSortTile]
     uint32_t (*cnt)[kBins] = reinterpret_cast<uint32_t (*)[kBins]>(stage + kSortTile);   // [warps][kBins]
@@ -818,12 +832,13 @@ k_radix_scatter(const uint64_t* __restrict__ keys, uint64_t* __restrict__ out, c
         __syncthreads();
         uint64_t key[kSortKeysPerThread];
         uint32_t rank[kSortKeysPerThread];
-        const int32_t wb = t * kSortTile + warp * kPerWarp;
+        int32_t tb = t * kSortTile, tile_n = min(kSortTile, n - tb), h0 = t, hs = ntiles;
+        if (tiles) { const SegTile st = tiles[t]; tb = first_pass ? st.in0 : st.out0; tile_n = st.count; h0 = st.hist0; hs = st.stride; }
+        const int32_t wl = warp * kPerWarp;   // the warp's first key inside the tile
 #pragma unroll
         for (int r = 0; r < kSortKeysPerThread; ++r) {
-            const int32_t i = wb + r * 32 + lane;
-            const bool ok = i < n;
-            key[r] = ok ? keys[i] : 0ull;
+            const bool ok = wl + r * 32 + lane < tile_n;
+            key[r] = ok ? keys[tb + wl + r * 32 + lane] : 0ull;
             const uint32_t dg = ok ? ((uint32_t)(key[r] >> shift) & (kBins - 1)) : 0xFFFFFFFFu;
             const uint32_t peers = __match_any_sync(0xFFFFFFFFu, dg);
             const int leader = __ffs(peers) - 1;
@@ -856,20 +871,18 @@ k_radix_scatter(const uint64_t* __restrict__ keys, uint64_t* __restrict__ out, c
         for (int q = 0; q < kBinsPerThread; ++q) {
             const int bin = threadIdx.x * kBinsPerThread + q;
             tile_base[bin] = before;
-            glob_base[bin] = hist_scanned[(size_t)bin * ntiles + t];
+            glob_base[bin] = hist_scanned[(size_t)h0 + (size_t)bin * hs];
             before += mine[q];
         }
         __syncthreads();
 #pragma unroll
         for (int r = 0; r < kSortKeysPerThread; ++r) {
-            const int32_t i = wb + r * 32 + lane;
-            if (i < n) {
+            if (wl + r * 32 + lane < tile_n) {
                 const uint32_t dg = (uint32_t)(key[r] >> shift) & (kBins - 1);
                 stage[tile_base[dg] + cnt[warp][dg] + rank[r]] = key[r];
             }
         }
         __syncthreads();
-        const int32_t tile_n = min(kSortTile, n - t * kSortTile);
         for (int32_t i = threadIdx.x; i < tile_n; i += kThreads) {
             const uint64_t kx = stage[i];
             const uint32_t dg = (uint32_t)(kx >> shift) & (kBins - 1);
@@ -1123,9 +1136,47 @@ __device__ __forceinline__ int hop_of_arena(const ExportManyArgs& a, int32_t i) 
     return h;
 }
 
-__global__ void k_export_params(SortParams* sp, int32_t* range, int32_t n) {
-    sp->zero = 0; sp->n = n; sp->ntiles = (n + kSortTile - 1) / kSortTile; sp->hist_len = kBins * sp->ntiles;
-    range[0] = 0; range[1] = n;
+// The segments of the export's sort in output order -- mini-batch after mini-batch, inside it the farthest delta
+// first -- cut into tiles: where a tile's keys lie in the arenas (hop-major), where in the output, and where its
+// histogram goes.  One block; also the sort's parameters and the range of the entry-count scan.
+__global__ void __launch_bounds__(1024) k_export_tiles(ExportManyArgs a, SegTile* tiles, SortParams* sp, int32_t* range) {
+    __shared__ int32_t warp_t[32], warp_n[32];
+    __shared__ int32_t carry_t, carry_n;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) { carry_t = 0; carry_n = 0; }
+    __syncthreads();
+    const int32_t n_seg = a.B * (a.k + 1);
+    for (int32_t s0 = 0; s0 < n_seg; s0 += 1024) {
+        const int32_t s = s0 + (int32_t)threadIdx.x;
+        int32_t in0 = 0, len = 0;
+        if (s < n_seg) {
+            const int32_t b = s / (a.k + 1), h = a.k - s % (a.k + 1);
+            in0 = a.node_off[h * (a.B + 1) + b];
+            len = a.node_off[h * (a.B + 1) + b + 1] - in0;
+        }
+        const int32_t nt = (len + kSortTile - 1) / kSortTile;
+        const int32_t it = (int32_t)warp_incl_scan((uint32_t)nt), in = (int32_t)warp_incl_scan((uint32_t)len);
+        if (lane == 31) { warp_t[warp] = it; warp_n[warp] = in; }
+        __syncthreads();
+        int32_t t0 = carry_t + it - nt, o0 = carry_n + in - len;
+        for (int w = 0; w < warp; ++w) { t0 += warp_t[w]; o0 += warp_n[w]; }
+        for (int32_t t = 0; t < nt; ++t) {
+            SegTile st;
+            st.in0 = in0 + t * kSortTile;
+            st.out0 = o0 + t * kSortTile;
+            st.count = min(kSortTile, len - t * kSortTile);
+            st.hist0 = t0 * kBins + t;
+            st.stride = nt;
+            tiles[t0 + t] = st;
+        }
+        __syncthreads();
+        if (threadIdx.x == 1023) { carry_t = t0 + nt; carry_n = o0 + len; }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        sp->zero = 0; sp->n = a.n_nodes_total; sp->ntiles = carry_t; sp->hist_len = kBins * carry_t;
+        range[0] = 0; range[1] = a.n_nodes_total;
+    }
 }
 
 __global__ void __launch_bounds__(kThreads) k_export_keys(ExportManyArgs a, uint64_t* keys) {
@@ -1133,8 +1184,7 @@ __global__ void __launch_bounds__(kThreads) k_export_keys(ExportManyArgs a, uint
         const int h = hop_of_arena(a, i);
         const int32_t b = a.node_batch[i];
         const uint32_t id = h == 0 ? (uint32_t)(i - a.node_off[b]) : (uint32_t)a.nodes[i];
-        const uint64_t seg = (uint64_t)b * (a.k + 1) + (uint64_t)(a.k - h);
-        keys[i] = (seg << (a.id_bits + a.pay_bits)) | ((uint64_t)id << a.pay_bits) | (uint64_t)(uint32_t)i;
+        keys[i] = ((uint64_t)id << a.pay_bits) | (uint64_t)(uint32_t)i;   // sorted inside its (mini-batch, delta) segment
     }
     // node_id_offsets of every mini-batch
     for (int32_t t = blockIdx.x * blockDim.x + threadIdx.x; t < a.B; t += gridDim.x * blockDim.x) {
@@ -1206,8 +1256,11 @@ static void sample_kernel_attributes();
 
 // LSD radix sort of 64-bit keys on bits [lo_bit, lo_bit + bits); sp (device) holds the key count.
 // Keys start in buf[0]; *res_buf tells which buffer holds the result.
+// With a tile table (seg_tiles, SegTile per tile; sp->ntiles tiles): a sort inside segments -- the first pass reads
+// every segment where its tiles say and all passes write segment after segment.
 void mg_sort_u64(mg_ctx* ctx, uint64_t* const buf[2], const SortParams* sp, int lo_bit, int bits, uint32_t* hist,
-                 uint32_t* scan_tmp, int* res_buf) {
+                 uint32_t* scan_tmp, int* res_buf, const void* seg_tiles) {
+    const SegTile* tiles = static_cast<const SegTile*>(seg_tiles);
     cudaStream_t st = ctx->stream;
     const int grid = mg_grid(ctx, 8);
     const int passes = (bits + kRadixBits - 1) / kRadixBits;
@@ -1216,11 +1269,11 @@ void mg_sort_u64(mg_ctx* ctx, uint64_t* const buf[2], const SortParams* sp, int 
     int cur = 0;
     for (int p = 0; p < passes; ++p) {
         const int shift = lo_bit + kRadixBits * p;
-        k_radix_hist<<<grid, kThreads, 0, st>>>(buf[cur], sp, shift, hist);
+        k_radix_hist<<<grid, kThreads, 0, st>>>(buf[cur], sp, shift, hist, tiles, p == 0);
         k_scan_reduce<<<grid, kThreads, 0, st>>>(hist, r, scan_tmp);
         k_scan_tiles<<<1, 1024, 0, st>>>(scan_tmp, r, nullptr, HopClose{nullptr, 0, nullptr, 0});
         k_scan_down<<<grid, kThreads, 0, st>>>(hist, r, scan_tmp);
-        k_radix_scatter<<<grid, kThreads, kScatterSmem, st>>>(buf[cur], buf[cur ^ 1], sp, shift, hist);
+        k_radix_scatter<<<grid, kThreads, kScatterSmem, st>>>(buf[cur], buf[cur ^ 1], sp, shift, hist, tiles, p == 0);
         cur ^= 1;
     }
     ctx->launches += 5 * passes;
@@ -1258,6 +1311,9 @@ static int dense_alloc(mg_ctx* ctx, mg_dense* d, int32_t B, int32_t k, int64_t c
                        int32_t table_size, int32_t smem_nb) {
     int rc;
     if (!d->hdr && (rc = dev_realloc(ctx, &d->hdr, 1))) return rc;
+    // sort scratch: a tile per 4096 keys, and one more per (mini-batch, delta) segment for the export's segmented sort
+    const int64_t want_sort_tiles = (std::max(cap_nodes, d->cap_nodes) + kSortTile - 1) / kSortTile + (int64_t)B * (k + 1);
+    const bool grow_sort = d->cap_nodes < cap_nodes || d->cap_sort_tiles < want_sort_tiles;
     if (d->cap_nodes < cap_nodes) {
         d->cap_nodes = 0;
         if ((rc = dev_realloc(ctx, &d->nodes, (size_t)cap_nodes))) return rc;
@@ -1268,15 +1324,21 @@ static int dense_alloc(mg_ctx* ctx, mg_dense* d, int32_t B, int32_t k, int64_t c
         d->cap_nodes_out = 0;
         if ((rc = dev_realloc(ctx, &d->newlist[0], (size_t)cap_nodes))) return rc;
         if ((rc = dev_realloc(ctx, &d->newlist[1], (size_t)cap_nodes))) return rc;
-        const int64_t sort_tiles = (cap_nodes + kSortTile - 1) / kSortTile;
-        const int64_t scan_tiles = std::max<int64_t>((cap_nodes + kScanTile - 1) / kScanTile,
+        d->cap_nodes = cap_nodes;
+    }
+    if (grow_sort) {
+        d->cap_sort_tiles = 0;
+        const int64_t sort_tiles = want_sort_tiles;
+        const int64_t scan_tiles = std::max<int64_t>((d->cap_nodes + kScanTile - 1) / kScanTile,
                                                      (kBins * sort_tiles + kScanTile - 1) / kScanTile);
         d->scan_tmp_elems = (size_t)scan_tiles + 16;
-        (void)scan_tiles;
         if ((rc = dev_realloc(ctx, &d->scan_tmp, d->scan_tmp_elems))) return rc;
         d->sort_hist_elems = (size_t)kBins * sort_tiles + kBins;
         if ((rc = dev_realloc(ctx, &d->sort_hist, d->sort_hist_elems))) return rc;
-        d->cap_nodes = cap_nodes;
+        SegTile* tiles = static_cast<SegTile*>(d->seg_tiles);
+        if ((rc = dev_realloc(ctx, &tiles, (size_t)sort_tiles + 1))) { d->seg_tiles = nullptr; return rc; }
+        d->seg_tiles = tiles;
+        d->cap_sort_tiles = sort_tiles;
     }
     if (d->cap_entries < cap_entries) {
         d->cap_entries = 0;
@@ -1856,9 +1918,10 @@ extern "C" int mg_dense_export_many(mg_ctx* ctx, mg_dense* d) {
     const int32_t n_total = d->h_hdr.hop_base[k + 1];
     const int id_bits = std::max({1, ilog2_ceil(ctx->n_nodes), ilog2_ceil(d->n_targets_total + 1)});
     const int pay_bits = std::max(1, ilog2_ceil((int64_t)n_total + 1));
-    const int seg_bits = std::max(1, ilog2_ceil((int64_t)B * (k + 1)));
-    if (id_bits + pay_bits + seg_bits > 64)
-        return mg_fail(ctx, MG_ERR_CAPACITY, "sample too large for a one-pass export (%d key bits): export fewer mini-batches per sample", id_bits + pay_bits + seg_bits);
+    if (id_bits + pay_bits > 64)
+        return mg_fail(ctx, MG_ERR_CAPACITY, "sample too large for a one-pass export (%d key bits): export fewer mini-batches per sample", id_bits + pay_bits);
+    if ((int64_t)(n_total + kSortTile - 1) / kSortTile + (int64_t)B * (k + 1) > d->cap_sort_tiles)
+        return mg_fail(ctx, MG_ERR_STATE, "the sort scratch of this mg_dense is too small for its sample");
     const ExportLayout L = export_layout(d);
     int rc = mg_ensure(ctx, &d->expm_buf, &d->expm_elems, L.total);
     if (rc) return rc;
@@ -1883,10 +1946,10 @@ extern "C" int mg_dense_export_many(mg_ctx* ctx, mg_dense* d) {
         ctx->stream = st;   // the sort and scan helpers (and the phase events) use ctx->stream
         {
         ProfScope ps(ctx, PH_SAMPLE_SORT, 0);
-        k_export_params<<<1, 1, 0, st>>>(sp, range, n_total);
+        k_export_tiles<<<1, 1024, 0, st>>>(a, static_cast<SegTile*>(d->seg_tiles), sp, range);
         k_export_keys<<<grid, kThreads, 0, st>>>(a, d->newlist[0]);
         int res = 0;
-        mg_sort_u64(ctx, d->newlist, sp, pay_bits, id_bits + seg_bits, d->sort_hist, (uint32_t*)d->scan_tmp, &res);
+        mg_sort_u64(ctx, d->newlist, sp, pay_bits, id_bits, d->sort_hist, (uint32_t*)d->scan_tmp, &res, d->seg_tiles);
         k_export_place<<<grid, kThreads, 0, st>>>(a, d->newlist[res]);
         mg_scan_u32(ctx, a.cnt, &range[0], &range[1], nullptr, (uint32_t*)d->scan_tmp, nullptr);
         k_export_many_entries<<<grid, kThreads, 0, st>>>(a);
@@ -1938,7 +2001,7 @@ extern "C" int mg_dense_free(mg_dense* d) {
     cudaFree(d->hdr); cudaFree(d->nodes); cudaFree(d->node_batch); cudaFree(d->ent_off); cudaFree(d->node_r0); cudaFree(d->node_deg); cudaFree(d->node_r0_out); cudaFree(d->node_deg_out); cudaFree(d->pairs); cudaFree(d->share_off);
     cudaFree(d->ent_nbrs); cudaFree(d->ent_repr); cudaFree(d->node_off); cudaFree(d->cum);
     cudaFree(d->rowbase); cudaFree(d->hkeys); cudaFree(d->hvals); cudaFree(d->newlist[0]);
-    cudaFree(d->newlist[1]); cudaFree(d->d_seeds); cudaFree(d->batch_cnt); cudaFree(d->scan_tmp); cudaFree(d->sort_hist);
+    cudaFree(d->newlist[1]); cudaFree(d->d_seeds); cudaFree(d->batch_cnt); cudaFree(d->scan_tmp); cudaFree(d->sort_hist); cudaFree(d->seg_tiles);
     cudaFree(d->exp_buf); cudaFree(d->perm_buf); cudaFree(d->d_ent_hop); cudaFree(d->expm_buf);
     if (d->ev_exported) cudaEventDestroy(d->ev_exported);
     if (d->h_pinned) cudaFreeHost(d->h_pinned);
