@@ -1199,9 +1199,11 @@ __global__ void __launch_bounds__(kThreads) k_export_keys(ExportManyArgs a, uint
 __global__ void __launch_bounds__(kThreads) k_export_place(ExportManyArgs a, const uint64_t* __restrict__ sorted) {
     const uint64_t pay_mask = (1ull << a.pay_bits) - 1ull;
     for (int32_t c = blockIdx.x * blockDim.x + threadIdx.x; c < a.n_nodes_total; c += gridDim.x * blockDim.x) {
-        const int32_t i = (int32_t)(sorted[c] & pay_mask);
+        const uint64_t key = sorted[c];
+        const int32_t i = (int32_t)(key & pay_mask);
         a.inv[i] = c;
-        a.o_node_ids[c] = a.nodes[i];
+        // the key carries the node id (for the targets their position: they keep the caller's order)
+        a.o_node_ids[c] = i < a.hop_base[1] ? a.nodes[i] : (int32_t)((key >> a.pay_bits) & ((1ull << a.id_bits) - 1ull));
         a.cnt[c] = i < a.hop_base[a.k] ? (uint32_t)(a.ent_off[i + 1] - a.ent_off[i]) : 0u;   // the farthest delta has no entries
     }
 }
