@@ -96,6 +96,7 @@ struct FusedArgs {
     int64_t row_lo;              // first packed output row this launch computes
     int64_t M;                   // one past its last packed output row
     int32_t sa, sb;              // A and B stages
+    const float* w_rows;         // weights-in-tensor-memory form: the padded weight matrix [N][2 * d_in_pad], K order of the slices
     int32_t tmem_cols;
     int32_t relu;
     int32_t sum_aggr;            // neighbour term = sum of the sampled neighbours instead of their mean
@@ -178,7 +179,11 @@ template <> struct PieceSum<true> {
     static __device__ __forceinline__ uint4 self_operand(const uint4& r) { return r; }   // fp16 rows are operands as they are
 };
 
-template <bool FIRST, bool HALF, bool F16>
+// TS: the weights stay in tensor memory for the whole kernel and are the MMAs' first operand (M = 256 output columns over
+// the pair, a CTA's 128 in its 128 lanes, K <= 256 columns), the gathered rows the second (N = 128: a half tile of either
+// CTA); the accumulator is the transposed output, [output column][row].  Nothing is streamed per half tile then -- with
+// the weights in shared memory a half tile waits for eight 16 KB slices through a two-stage ring (4 us of latency).
+template <bool FIRST, bool HALF, bool F16, bool TS = false>
 __global__ void __cluster_dims__(2, 1, 1) __maxnreg__(MG_FUSED_MAXNREG)
 k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_out, FusedArgs a) {
     constexpr int KCE = Geo<F16>::kKC, GC = Geo<F16>::kGroup, LC = Geo<F16>::kLaneCols;
@@ -233,6 +238,29 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
     const uint32_t acc_stride = (uint32_t)(a.tmem_cols / kAccBufs);  // columns per accumulator buffer (a multiple of 32)
+    constexpr uint32_t kTsAcc0 = 256, kTsAccCols = 128;              // TS: weights in columns [0, 256), two accumulators behind them
+    if constexpr (TS) {
+        if (warp >= kFirstEpilogueWarp && warp < kTmaWarp) {   // (the warps that may touch lanes 32 q .. 32 q + 31)
+            const int q = warp & 3;
+            const int n = (int)rank * 128 + q * 32 + lane;     // this lane's output column = its row of the weights
+            const int K = 2 * a.d_in_pad;
+            const float4* wrow = reinterpret_cast<const float4*>(a.w_rows + (size_t)min(n, a.N - 1) * K);
+            for (int k0 = 0; k0 < K; k0 += 32) {
+                uint32_t v[32];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float4 x = n < a.N ? __ldg(wrow + k0 / 4 + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    v[4 * j] = __float_as_uint(x.x); v[4 * j + 1] = __float_as_uint(x.y);
+                    v[4 * j + 2] = __float_as_uint(x.z); v[4 * j + 3] = __float_as_uint(x.w);
+                }
+                tmem_st_32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)k0, v);
+            }
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        }
+        tc_fence_before();
+        cluster_sync_all();   // both CTAs' weights are in place before the leader's first MMA reads them
+        tc_fence_after();
+    }
     const int n_groups = (a.d_in_pad + GC - 1) / GC;
 
     // (Build option) registers move from the epilogue's and the control warpgroup to the producers': each warpgroup
@@ -257,7 +285,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
     MG_REG_SET(MG_REG_CTL);
     if (warp == kTmaWarp) {
         // ---------------- weight slices: each CTA stages its half of the output columns (TMA from L2) ----------------
-        if (lane == 0) {
+        if (!TS && lane == 0) {
             uint32_t cnt = 0;
             bool ok = true;
             // the weight slices of a group are streamed once per half tile, in the order the MMAs consume them
@@ -277,7 +305,29 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
         __syncwarp();
     } else if (warp == kMmaWarp) {
         // ---------------- MMA issue: one thread of the leader, for both CTAs ----------------
-        if (lane == 0 && leader) {
+        if (TS && lane == 0 && leader) {
+            // M = 256 output columns over the pair, N = 128 rows (a half tile of each CTA), fp32 accumulate, TF32, K-major
+            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+            bool ok = true;
+            for (uint32_t it = 0; it < my_iters && ok; ++it)
+                for (int h = 0; h < 2 && ok; ++h) {
+                    const uint32_t hu = it * 2 + h, buf = hu & 1;
+                    if (hu >= 2 && !mbar_wait(&acc_empty[buf], ((hu >> 1) - 1) & 1)) { atomicExch(a.error, 12u); ok = false; break; }
+                    tc_fence_after();
+                    if (!mbar_wait(&a_ready[h], it & 1)) { atomicExch(a.error, 13u); ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + kTsAcc0 + buf * kTsAccCols;
+                    for (int c = 0; c < n_chunks; ++c) {
+                        const uint64_t db = smem_desc_sw128(smem_u32(a_base + (size_t)c * kABytes + (size_t)h * (HM * 128)));
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)
+                            mma_tf32_pair_ts(d_tmem, tmem_base + (uint32_t)(c * 32 + kk * 8), db + (uint64_t)(kk * 2), idesc, (c | kk) ? 1u : 0u);
+                    }
+                    mma_commit_pair(&a_free[h]);
+                    mma_commit_pair(&acc_full[buf]);
+                }
+        }
+        if (!TS && lane == 0 && leader) {
             // M = 128 over the pair: 64 rows (a half tile) of each CTA per instruction
             // fp32 accumulate; operands TF32 (format 2) or fp16 (format 0), both K-major
             const uint32_t idesc = (1u << 4) | ((F16 ? 0u : 2u) << 7) | ((F16 ? 0u : 2u) << 10) | ((uint32_t)(a.BN >> 3) << 17) |
@@ -393,7 +443,50 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
         const int col_base = (lane_group >> 1) * half_n;
         const int n_cols = half_n;
         bool ok = true;
-        for (uint32_t hu = 0; hu < 2 * my_iters && ok; ++hu) {
+        if constexpr (TS) {
+            // The accumulator of a half-tile pair: lane = output column (this CTA's 128), column j = row j of the
+            // leader's half tile (j < 64) or row j - 64 of the peer's.  A warp turns 32 x 32 pieces round through its
+            // staging tile (lane = column of the box, 128-byte swizzle) and stores them with TMA.
+            const int n0 = (int)rank * 128 + lane_group * 32;
+            const float bias_n = n0 + lane < a.N ? __ldg(a.bias + n0 + lane) : 0.f;
+            uint8_t* stage = reinterpret_cast<uint8_t*>(out_stage[lane_group]);
+            for (uint32_t hu = 0; hu < 2 * my_iters && ok; ++hu) {
+                const uint32_t buf = hu & 1;
+                if (!mbar_wait(&acc_full[buf], (hu >> 1) & 1)) { if (lane == 0) atomicExch(a.error, 14u); ok = false; break; }
+                tc_fence_after();
+                for (int g = 0; g < 4; ++g) {
+                    uint32_t v[32];
+                    tmem_ld_32(tmem_base + kTsAcc0 + buf * kTsAccCols + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)(g * 32), v);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    const int64_t t = 2 * ((int64_t)pair + (int64_t)(hu >> 1) * n_pairs) + (g >> 1);   // the tile of CTA g / 2
+                    const int64_t row0 = a.row_lo + t * BM + (hu & 1) * HM + (g & 1) * 32;
+                    if (row0 >= a.M || n0 >= a.N) continue;
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the previous box has left the tile
+                    __syncwarp();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        float o = __uint_as_float(v[j]) + bias_n;
+                        if (a.relu) o = fmaxf(o, 0.f);
+                        *reinterpret_cast<float*>(stage + j * 128 + (((lane >> 2) ^ (j & 7)) << 4) + ((lane & 3) << 2)) = o;
+                    }
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        // rows past the end of the layer and columns past its width are clipped by the tensor map
+                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                                     ::"l"(&map_out), "r"(smem_u32(stage)), "r"(n0), "r"((int)row0) : "memory");
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    if (leader) mbar_arrive(&acc_empty[buf]);
+                    else mbar_arrive_cluster(mapa_u32(smem_u32(&acc_empty[buf]), 0));
+                }
+            }
+        }
+        for (uint32_t hu = 0; !TS && hu < 2 * my_iters && ok; ++hu) {
             const int64_t t = tile_of(hu >> 1);
             const uint32_t buf = hu % kAccBufs;
             if (!mbar_wait(&acc_full[buf], (hu / kAccBufs) & 1)) { if (lane == 0) atomicExch(a.error, 14u); ok = false; break; }
@@ -793,6 +886,9 @@ int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_ou
     // A shallow weight ring (32 KB) on purpose: with 128 KB of A stages the CTA then fits the 196 KB shared-memory
     // carve-out, which leaves the gathers twice the L1 (measured: layer 1 of the bench 2.92 -> 2.75 ms).
     a.sb = std::max(2, std::min({kMaxStages, n_chunks, (32 * 1024) / b_bytes}));
+    // weights in tensor memory: TF32 operands, fp32 output, all of K in 256 columns, at most 256 output columns
+    const bool ts = !f16 && !out_f16 && n_chunks <= 8 && d_out <= 256 && !getenv("MG_FUSED_NO_TS");
+    if (ts) { a.tmem_cols = 512; a.sb = 0; a.w_rows = w_pad_t; }
     const size_t smem = (size_t)a.sa * kABytes + (size_t)a.sb * b_bytes + 1024;
     CUtensorMap mw;
     if (!(f16 ? make_map_f16(&mw, w_pad_h, d_out, 2 * a.d_in_pad, a.BN / 2) : make_map_f32(&mw, w_pad_t, d_out, 2 * a.d_in_pad, a.BN / 2)))
@@ -805,6 +901,8 @@ int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_ou
     const bool first = layer == 1, half = first && ctx->feat_dtype == MG_DTYPE_F16;
     auto kern = first ? (f16 ? k_sage_layer_fused<true, true, true> : half ? k_sage_layer_fused<true, true, false> : k_sage_layer_fused<true, false, false>)
                       : (f16 ? k_sage_layer_fused<false, true, true> : k_sage_layer_fused<false, false, false>);
+    if (ts) kern = first ? (half ? k_sage_layer_fused<true, true, false, true> : k_sage_layer_fused<true, false, false, true>)
+                         : k_sage_layer_fused<false, false, false, true>;
     MG_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const int64_t n_tiles = (row_hi - row_lo + BM - 1) / BM;
     const int grid = 2 * (int)std::min<int64_t>((n_tiles + 1) / 2, ctx->n_sms / 2);   // CTA pairs
