@@ -106,6 +106,7 @@ struct FusedArgs {
     uint32_t* error;
 };
 
+constexpr int kLaneEntries = 32;   // rows up to this long are translated by their own lane of the planner warp
 constexpr int kKeyCap = 704;    // source-row indices of a row block's entries cached in shared memory (22 per row: what still fits the 196 KB carve-out)
 
 // What a producer needs to build one output row: x = source row of the row's own representation; y = first
@@ -283,9 +284,9 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                   "the warpgroups' registers must fit what the CTA was launched with");
     if (warp >= kTmaWarp) {
     MG_REG_SET(MG_REG_CTL);
-    if (warp == kTmaWarp) {
+    if (warp == kTmaWarp && !TS) {
         // ---------------- weight slices: each CTA stages its half of the output columns (TMA from L2) ----------------
-        if (!TS && lane == 0) {
+        if (lane == 0) {
             uint32_t cnt = 0;
             bool ok = true;
             // the weight slices of a group are streamed once per half tile, in the order the MMAs consume them
@@ -372,10 +373,12 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
         // A planner warp takes every kPlannerWarps-th row block: lane = row.  It reads the rows' metadata, scans the
         // entry counts, and translates the block's entries to source rows in shared memory, so that the producers'
         // gathers depend on nothing but shared memory.
-        const int plw = warp - kFirstPlannerWarp;
+        // (with the weights in tensor memory nothing is streamed and the weight warp is a third planner)
+        constexpr int kPlanners = TS ? kPlannerWarps + 1 : kPlannerWarps;
+        const int plw = warp == kTmaWarp ? kPlannerWarps : warp - kFirstPlannerWarp;
         const int32_t* keys = FIRST ? a.ent_nbrs : a.ent_repr;
         bool ok = true;
-        for (uint32_t q = plw; ok; q += kPlannerWarps) {
+        for (uint32_t q = plw; ok; q += kPlanners) {
             if (q / kBlocksPerTile >= my_iters) break;
             const int64_t t = tile_of(q / kBlocksPerTile);   // past the end for the peer of an odd last tile: all padding
             const int slot = q % kPlanSlots;
@@ -393,7 +396,19 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
             const bool cached = total <= kKeyCap;
             const int32_t in_base = rm.w, koff = end - max(rm.z, 0);
             meta[slot][lane] = make_int4(rm.x, rm.y, rm.z, cached ? koff : in_base);
-            if (cached) {
+            const int32_t zmax = (int32_t)__reduce_max_sync(0xFFFFFFFFu, (uint32_t)max(rm.z, 0));
+            if (cached && zmax <= kLaneEntries) {
+                // short rows (the usual case): every lane translates its own row's entries, kUnroll loads in flight
+                // (the entries of consecutive rows are consecutive, so the lanes' loads share their cache lines)
+                for (int32_t i0 = 0; i0 < zmax; i0 += kUnroll) {
+                    int32_t key[kUnroll];
+#pragma unroll
+                    for (int u = 0; u < kUnroll; ++u) key[u] = i0 + u < rm.z ? __ldg(keys + rm.y + i0 + u) : 0;
+#pragma unroll
+                    for (int u = 0; u < kUnroll; ++u)
+                        if (i0 + u < rm.z) src_rows[slot][koff + i0 + u] = source_row<FIRST>(a, in_base, key[u]);
+                }
+            } else if (cached) {
                 // entry j belongs to the first row whose end exceeds j
                 for (int32_t j0 = 0; j0 < total; j0 += 32 * 4) {
                     int32_t key[4], base[4];
