@@ -96,7 +96,7 @@ struct FusedArgs {
     int64_t row_lo;              // first packed output row this launch computes
     int64_t M;                   // one past its last packed output row
     int32_t sa, sb;              // A and B stages
-    const float* w_rows;         // weights-in-tensor-memory form: the padded weight matrix [N][2 * d_in_pad], K order of the slices
+    const void* w_rows;          // weights-in-tensor-memory form: the padded weight matrix [N][2 * d_in_pad] (fp32 or fp16), K order of the slices
     int32_t tmem_cols;
     int32_t relu;
     int32_t sum_aggr;            // neighbour term = sum of the sampled neighbours instead of their mean
@@ -244,8 +244,8 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
         if (warp >= kFirstEpilogueWarp && warp < kTmaWarp) {   // (the warps that may touch lanes 32 q .. 32 q + 31)
             const int q = warp & 3;
             const int n = (int)rank * 128 + q * 32 + lane;     // this lane's output column = its row of the weights
-            const int K = 2 * a.d_in_pad;
-            const float4* wrow = reinterpret_cast<const float4*>(a.w_rows + (size_t)min(n, a.N - 1) * K);
+            const int K = F16 ? a.d_in_pad : 2 * a.d_in_pad;   // 32-bit words per row of the weights (two fp16 values per word)
+            const float4* wrow = reinterpret_cast<const float4*>(static_cast<const uint32_t*>(a.w_rows) + (size_t)min(n, a.N - 1) * K);
             for (int k0 = 0; k0 < K; k0 += 32) {
                 uint32_t v[32];
 #pragma unroll
@@ -307,8 +307,8 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
     } else if (warp == kMmaWarp) {
         // ---------------- MMA issue: one thread of the leader, for both CTAs ----------------
         if (TS && lane == 0 && leader) {
-            // M = 256 output columns over the pair, N = 128 rows (a half tile of each CTA), fp32 accumulate, TF32, K-major
-            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+            // M = 256 output columns over the pair, N = 128 rows (a half tile of each CTA), fp32 accumulate, K-major
+            const uint32_t idesc = (1u << 4) | ((F16 ? 0u : 2u) << 7) | ((F16 ? 0u : 2u) << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
             bool ok = true;
             for (uint32_t it = 0; it < my_iters && ok; ++it)
                 for (int h = 0; h < 2 && ok; ++h) {
@@ -321,8 +321,10 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     for (int c = 0; c < n_chunks; ++c) {
                         const uint64_t db = smem_desc_sw128(smem_u32(a_base + (size_t)c * kABytes + (size_t)h * (HM * 128)));
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk)
-                            mma_tf32_pair_ts(d_tmem, tmem_base + (uint32_t)(c * 32 + kk * 8), db + (uint64_t)(kk * 2), idesc, (c | kk) ? 1u : 0u);
+                        for (int kk = 0; kk < 4; ++kk) {   // 32 bytes of every slice row = 8 columns of the weights per instruction
+                            if (F16) mma_f16_pair_ts(d_tmem, tmem_base + (uint32_t)(c * 32 + kk * 8), db + (uint64_t)(kk * 2), idesc, (c | kk) ? 1u : 0u);
+                            else mma_tf32_pair_ts(d_tmem, tmem_base + (uint32_t)(c * 32 + kk * 8), db + (uint64_t)(kk * 2), idesc, (c | kk) ? 1u : 0u);
+                        }
                     }
                     mma_commit_pair(&a_free[h]);
                     mma_commit_pair(&acc_full[buf]);
@@ -482,7 +484,8 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     for (int j = 0; j < 32; ++j) {
                         float o = __uint_as_float(v[j]) + bias_n;
                         if (a.relu) o = fmaxf(o, 0.f);
-                        *reinterpret_cast<float*>(stage + j * 128 + (((lane >> 2) ^ (j & 7)) << 4) + ((lane & 3) << 2)) = o;
+                        if (a.out_f16) *reinterpret_cast<__half*>(stage + j * 64 + lane * 2) = __float2half_rn(o);   // (boxes of 32 fp16 columns, not swizzled)
+                        else *reinterpret_cast<float*>(stage + j * 128 + (((lane >> 2) ^ (j & 7)) << 4) + ((lane & 3) << 2)) = o;
                     }
                     fence_async_smem();
                     __syncwarp();
@@ -801,6 +804,18 @@ __global__ void k_pack_weights(const float* __restrict__ w_cat /*[2 d_in, N]*/, 
 }
 
 // row-major [rows, K] fp16 matrix, boxes of 64 halves x box_rows, 128-byte swizzle, zero fill
+// the same matrix in boxes of 32 halves x 32 rows, not swizzled (the transposed epilogue's fp16 stores)
+static bool make_map_f16_box32(CUtensorMap* map, const void* base, int64_t rows, int K) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    const cuuint32_t box[2] = {32u, 32u};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 static bool make_map_f16(CUtensorMap* map, const void* base, int64_t rows, int K, int box_rows) {
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
@@ -902,8 +917,8 @@ int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_ou
     // carve-out, which leaves the gathers twice the L1 (measured: layer 1 of the bench 2.92 -> 2.75 ms).
     a.sb = std::max(2, std::min({kMaxStages, n_chunks, (32 * 1024) / b_bytes}));
     // weights in tensor memory: TF32 operands, fp32 output, all of K in 256 columns, at most 256 output columns
-    const bool ts = !f16 && !out_f16 && n_chunks <= 8 && d_out <= 256 && !getenv("MG_FUSED_NO_TS");
-    if (ts) { a.tmem_cols = 512; a.sb = 0; a.w_rows = w_pad_t; }
+    const bool ts = n_chunks <= 8 && d_out <= 256 && !getenv("MG_FUSED_NO_TS");
+    if (ts) { a.tmem_cols = 512; a.sb = 0; a.w_rows = f16 ? (const void*)w_pad_h : (const void*)w_pad_t; }
     const size_t smem = (size_t)a.sa * kABytes + (size_t)a.sb * b_bytes + 1024;
     CUtensorMap mw;
     if (!(f16 ? make_map_f16(&mw, w_pad_h, d_out, 2 * a.d_in_pad, a.BN / 2) : make_map_f32(&mw, w_pad_t, d_out, 2 * a.d_in_pad, a.BN / 2)))
@@ -911,13 +926,14 @@ int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_ou
     // output [row_hi rows, d_out] fp32, 32 x 32 boxes, 128-byte swizzle; rows are global packed rows, so a window's
     // shifted base pointer works unchanged (rows below row_lo are never stored)
     CUtensorMap mo;
-    if (!(out_f16 ? make_map_f16(&mo, h_out, row_hi, d_out, 32) : make_map_f32(&mo, h_out, row_hi, d_out, 32)))
+    if (!(out_f16 ? (ts ? make_map_f16_box32(&mo, h_out, row_hi, d_out) : make_map_f16(&mo, h_out, row_hi, d_out, 32))
+                  : make_map_f32(&mo, h_out, row_hi, d_out, 32)))
         return mg_fail(ctx, MG_ERR_CUDA, "cuTensorMapEncodeTiled failed for the layer output");
     const bool first = layer == 1, half = first && ctx->feat_dtype == MG_DTYPE_F16;
     auto kern = first ? (f16 ? k_sage_layer_fused<true, true, true> : half ? k_sage_layer_fused<true, true, false> : k_sage_layer_fused<true, false, false>)
                       : (f16 ? k_sage_layer_fused<false, true, true> : k_sage_layer_fused<false, false, false>);
-    if (ts) kern = first ? (half ? k_sage_layer_fused<true, true, false, true> : k_sage_layer_fused<true, false, false, true>)
-                         : k_sage_layer_fused<false, false, false, true>;
+    if (ts) kern = first ? (f16 ? k_sage_layer_fused<true, true, true, true> : half ? k_sage_layer_fused<true, true, false, true> : k_sage_layer_fused<true, false, false, true>)
+                         : (f16 ? k_sage_layer_fused<false, true, true, true> : k_sage_layer_fused<false, false, false, true>);
     MG_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const int64_t n_tiles = (row_hi - row_lo + BM - 1) / BM;
     const int grid = 2 * (int)std::min<int64_t>((n_tiles + 1) / 2, ctx->n_sms / 2);   // CTA pairs
