@@ -106,6 +106,7 @@ struct FusedArgs {
     uint32_t* error;
 };
 
+constexpr int kTsMaxEntriesPerRow = 8;   // layers with more entries per output row than this stream their weights
 constexpr int kLaneEntries = 32;   // rows up to this long are translated by their own lane of the planner warp
 constexpr int kKeyCap = 704;    // source-row indices of a row block's entries cached in shared memory (22 per row: what still fits the 196 KB carve-out)
 
@@ -917,7 +918,11 @@ int mg_layer_fused(mg_ctx* ctx, const mg_dense* d, int layer, int d_in, int d_ou
     // carve-out, which leaves the gathers twice the L1 (measured: layer 1 of the bench 2.92 -> 2.75 ms).
     a.sb = std::max(2, std::min({kMaxStages, n_chunks, (32 * 1024) / b_bytes}));
     // weights in tensor memory: TF32 operands, fp32 output, all of K in 256 columns, at most 256 output columns
-    const bool ts = n_chunks <= 8 && d_out <= 256 && !getenv("MG_FUSED_NO_TS");
+    // ... and rows with few entries: a half tile of long rows is gathered for longer than its weight slices take to
+    // arrive, so the stream costs nothing there, while the transposed epilogue does (measured: 5.3 entries per row,
+    // 2.03 -> 1.92 ms with the weights in tensor memory; 20 per row, 0.83 -> 0.90 ms)
+    const int64_t layer_entries = d->h_hdr.ent_base[d->k - layer + 1], layer_rows = d->h_hdr.rows_total[layer];
+    const bool ts = n_chunks <= 8 && d_out <= 256 && layer_entries <= kTsMaxEntriesPerRow * layer_rows && !getenv("MG_FUSED_NO_TS");
     if (ts) { a.tmem_cols = 512; a.sb = 0; a.w_rows = f16 ? (const void*)w_pad_h : (const void*)w_pad_t; }
     const size_t smem = (size_t)a.sa * kABytes + (size_t)a.sb * b_bytes + 1024;
     CUtensorMap mw;
