@@ -550,6 +550,51 @@ def test_fp16_intermediate_layer_outputs(dims):
     ctx.keep_layer_outputs(False)
 
 
+@pytest.mark.parametrize("dims,fanouts,fp16_feats", [([128, 256, 256], [5, 4], False), ([96, 200, 36], [3, 6], False),
+                                                     ([128, 256, 128], [4, 4], True), ([128, 128, 64], [20, 3], False)])
+def test_layer_weights_in_tensor_memory_and_streamed(dims, fanouts, fp16_feats, monkeypatch):
+    """The fused layer kernel keeps a layer's weights in tensor memory (as the MMAs' first operand, the accumulator
+    transposed) when all of K fits there and the layer's rows are short, and streams them through shared memory
+    otherwise.  Both forms on the same sample: each within the tensor-core tolerance of the fp64 oracle and next to
+    each other; widths that are no multiples of 32, ragged tiles, a mini-batch of one target, fp16 base
+    representations, fp16 intermediates, and a layer of long rows (which streams in either case)."""
+    n = 40_000
+    g = inputs.rmat_graph(n, 700_000, seed=31)
+    feats = inputs.normal_features(n, dims[0], seed=32)
+    table = feats.half() if fp16_feats else feats
+    ctx = make_ctx(g, table)
+    sizes = [513, 1, 130]
+    tg = [inputs.distinct_targets(n, s_, seed=33 + i) for i, s_ in enumerate(sizes)]
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    seeds = [17, 18, 19]
+    d = ctx.sample_many(torch.cat(tg), offs, fanouts, seeds)
+    layers = inputs.random_bias_layers(dims, seed=34)
+    np_layers = [(w.numpy(), nn.numpy(), b.numpy()) for w, nn, b in layers]
+    view = oracle_view(g)
+    base = table.float().numpy()
+    want = []
+    for b in range(3):
+        ref = O.sample_dense(view, tg[b].tolist(), fanouts, seeds[b])
+        want.append(O.forward(ref, base[ref["node_ids"]], np_layers))
+    model = ctx.model(layers, mg.GEMM_TF32)
+    got = {}
+    for intermediates in (torch.float32, torch.float16):
+        model.set_intermediates(intermediates)
+        for streamed in (False, True):
+            if streamed:
+                monkeypatch.setenv("MG_FUSED_NO_TS", "1")
+            else:
+                monkeypatch.delenv("MG_FUSED_NO_TS", raising=False)
+            out = torch.full((int(offs[-1]), dims[-1]), float("nan"), dtype=torch.float32, device="cuda")
+            ctx.forward(model, d, out)
+            got[(intermediates, streamed)] = out.cpu().numpy()
+            for b in range(3):
+                close(got[(intermediates, streamed)][offs[b]:offs[b + 1]], want[b], RTOL_TC)
+        # the two forms contract the same TF32 (or fp16) operands in the same K order
+        close(got[(intermediates, False)], got[(intermediates, True)], 3e-4)
+    monkeypatch.delenv("MG_FUSED_NO_TS", raising=False)
+
+
 def test_config2_shaped_power_law_three_layers():
     """R-MAT, dim 128, hidden 256, fanouts [15, 10, 5], batches of 1000 (config 2 at 1/5 scale so
     the oracle finishes in seconds); hub rows, zero-degree nodes, several batches per pass."""
