@@ -243,8 +243,8 @@ int mg_dense_view(mg_ctx* ctx, mg_dense* d, int32_t batch, mg_dense_arrays* out)
 /* The canonical DENSE ordering for the whole sample in one pass (Algorithm 1's computeNextDelta leaves every delta
  * as the ascending list of its ids; on the device a delta is kept in the order its nodes were found).
  * mg_dense_export_many queues, on the library's sampling stream, ONE sort of all nodes of all mini-batches by id
- * inside their (mini-batch, delta) segments and the translation of every entry, and returns at once: no host synchronisation, no work
- * per mini-batch.  It overlaps whatever runs on the context's stream (the layers of this or another sample); a later
+ * inside their (mini-batch, delta) segments and the translation of every entry, and returns at once: no host
+ * synchronisation, no work per mini-batch.  It overlaps whatever runs on the context's stream (the layers of this or another sample); a later
  * sample into `d` is ordered behind it.  mg_dense_export_view waits for that export (first call only) and hands out
  * mini-batch `batch` of it: the same five arrays as mg_dense_view, bit for bit, as DEVICE pointers into a buffer owned
  * by `d` that holds all mini-batches packed one after the other; valid until the next mg_dense_export_many or
