@@ -172,6 +172,41 @@ def test_export_of_all_mini_batches_at_once(tiny):
         assert_dense_equal(d.view(2), O.sample_dense(view, tg[2].tolist(), fanouts, seeds[2]))   # the per-batch path still works
 
 
+def test_export_with_many_segments_and_segments_longer_than_a_tile():
+    """The export sorts the ids inside their (mini-batch, delta) segments.  1,600 segments (more than the 1,024 the
+    tile-table kernel takes per round, empty mini-batches among them), and, in a second sample, deltas of more than
+    4,096 nodes (more than one sort tile per segment, the last one ragged): every checked mini-batch bit for bit the
+    oracle's."""
+    n = 60_000
+    g = inputs.rmat_graph(n, 1_200_000, seed=41)
+    ctx = make_ctx(g)
+    view = oracle_view(g)
+    # many short segments
+    B = 400
+    sizes = [(3 if b % 7 else 0) + (b % 3) for b in range(B)]
+    tg = [inputs.distinct_targets(n, s_, seed=1000 + b) for b, s_ in enumerate(sizes)]
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    seeds = [11 * b + 1 for b in range(B)]
+    fanouts = [3, 2, 2]
+    d = ctx.sample_many(torch.cat(tg), offs, fanouts, seeds)
+    d.export_many()
+    for b in (0, 1, 7, 255, 256, 257, 341, 342, B - 2, B - 1):
+        assert_dense_equal(d.export_view(b), O.sample_dense(view, tg[b].tolist(), fanouts, seeds[b]))
+    # few long segments
+    sizes = [1500, 2, 700]
+    tg = [inputs.distinct_targets(n, s_, seed=2000 + b) for b, s_ in enumerate(sizes)]
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    fanouts = [10, 6]
+    d = ctx.sample_many(torch.cat(tg), offs, fanouts, [5, 6, 7])
+    d.export_many()
+    longest = 0
+    for b in range(3):
+        ref = O.sample_dense(view, tg[b].tolist(), fanouts, [5, 6, 7][b])
+        assert_dense_equal(d.export_view(b), ref)
+        longest = max(longest, int(np.diff(np.asarray(ref["node_id_offsets"])).max()))
+    assert longest > 4096   # (the case is what it claims to be)
+
+
 @pytest.mark.parametrize("fanouts", [[1], [3, 1], [33, 2], [40, 70]])
 def test_odd_fanouts(fanouts):
     g = inputs.rmat_graph(3000, 60_000, seed=3)
