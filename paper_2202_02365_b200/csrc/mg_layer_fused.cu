@@ -195,6 +195,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
     // the leader.
     __shared__ uint64_t a_ready[2], a_free[2], b_full[kMaxStages], b_empty[kMaxStages];   // a_*: one per half tile
     __shared__ uint64_t acc_full[kAccBufs], acc_empty[kAccBufs];
+    __shared__ uint64_t w_ready;   // TS, leader only: both CTAs' weights are in tensor memory
     __shared__ uint32_t tmem_slot;
     __shared__ uint64_t plan_full[kPlanSlots], plan_empty[kPlanSlots];
     __shared__ RowMeta meta[kPlanSlots][kBlockRows];
@@ -225,6 +226,7 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
         for (int s = 0; s < 2; ++s) { mbar_init(&a_ready[s], 2 * kProducerWarps); mbar_init(&a_free[s], 1); }
         for (int s = 0; s < a.sb; ++s) { mbar_init(&b_full[s], 1); mbar_init(&b_empty[s], 1); }
         for (int s = 0; s < kAccBufs; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 2 * 4); }
+        mbar_init(&w_ready, 2 * 4);   // the four loading warps of both CTAs
         for (int s = 0; s < kPlanSlots; ++s) { mbar_init(&plan_full[s], 1); mbar_init(&plan_empty[s], kProducerWarps); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
@@ -258,10 +260,14 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 tmem_st_32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)k0, v);
             }
             asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            // only the leader's MMA thread waits for the weights: planners and gather warps start at once
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                if (leader) mbar_arrive(&w_ready);
+                else mbar_arrive_cluster(mapa_u32(smem_u32(&w_ready), 0));
+            }
         }
-        tc_fence_before();
-        cluster_sync_all();   // both CTAs' weights are in place before the leader's first MMA reads them
-        tc_fence_after();
     }
     const int n_groups = (a.d_in_pad + GC - 1) / GC;
 
@@ -310,7 +316,9 @@ k_sage_layer_fused(const __grid_constant__ CUtensorMap map_w, const __grid_const
         if (TS && lane == 0 && leader) {
             // M = 256 output columns over the pair, N = 128 rows (a half tile of each CTA), fp32 accumulate, K-major
             const uint32_t idesc = (1u << 4) | ((F16 ? 0u : 2u) << 7) | ((F16 ? 0u : 2u) << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
-            bool ok = true;
+            bool ok = mbar_wait(&w_ready, 0);
+            if (!ok) atomicExch(a.error, 18u);
+            tc_fence_after();
             for (uint32_t it = 0; it < my_iters && ok; ++it)
                 for (int h = 0; h < 2 && ok; ++h) {
                     const uint32_t hu = it * 2 + h, buf = hu & 1;
